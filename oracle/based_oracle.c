@@ -1,0 +1,212 @@
+/*
+ * CPU oracle for the Based sequence-mixing hot path (arXiv 2402.18668).
+ *
+ * THIS FILE IS TEST INFRASTRUCTURE.  It is a plain, slow, fp64 restatement of
+ * the paper's definitions, used only to check the CUDA library and to time a
+ * CPU baseline.  It shares no code with the CUDA path and the product never
+ * calls it.
+ *
+ * What it implements, and where the paper defines it:
+ *   oracle_phi                  2nd-order Taylor feature map: Eq. (3) of Sec. 4.1
+ *                               with the scale factors of the TaylorExp module in
+ *                               the App. B.1 PyTorch listing (x / d'^(1/4) and
+ *                               (x (x) x) / (sqrt(2) sqrt(d'))).
+ *   oracle_linattn_quadratic    causal linear attention in its "attention" form,
+ *                               left-hand side of Eq. (2), Sec. 4.1: every (i, j<=i)
+ *                               pair visited explicitly.  This is the authority.
+ *   oracle_linattn_row          one output row of the same definition.
+ *   oracle_linattn_recurrent    recurrent form (KV-state / K-state recurrences and
+ *                               Eq. (2b) of Sec. 4.1; update-then-read order of the
+ *                               App. B.2 step() listing).  L = 1 is one decode step.
+ *   oracle_swa                  exact softmax attention, Eq. (1) of Sec. 2,
+ *                               restricted to the causal window
+ *                               {k_{i-w+1}, ..., k_i} of Sec. 4.2.
+ *   oracle_linattn_quadratic_ld the quadratic form again with long double
+ *                               accumulators (adequacy check of fp64 on tiny inputs).
+ *
+ * Parity pins: every function above is pinned by tests/test_oracle_*.py
+ * (closed forms, special cases, library softmax attention, the Taylor remainder
+ * bound, brute force in extended precision).  Nothing here is "parity unpinned".
+ *
+ * Layouts (row-major, last index contiguous), all double:
+ *   q, k : [B, H, L, dp]      v, y : [B, H, L, dv]
+ *   S    : [B, H, D, dv]      z    : [B, H, D]        D = 1 + dp + dp*dp
+ * Feature order inside D: index 0 the constant, 1..dp the linear terms,
+ * 1 + dp + m*dp + n the (m, n) product.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_EPS 1e-12 /* the eps of the App. B listings, added to the denominator */
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+int oracle_feature_dim(int dp) { return 1 + dp + dp * dp; }
+
+/* phi(x) = [1, x / d'^(1/4), vec(x x^T) / (sqrt 2 * sqrt d')] */
+void oracle_phi(const double *x, int dp, double *out) {
+    const double rd = sqrt((double)dp);
+    const double rrd = sqrt(rd);
+    const double r2 = sqrt(2.0);
+    out[0] = 1.0;
+    for (int m = 0; m < dp; ++m) out[1 + m] = x[m] / rrd;
+    for (int m = 0; m < dp; ++m)
+        for (int n = 0; n < dp; ++n) out[1 + dp + m * dp + n] = (x[m] * x[n] / r2) / rd;
+}
+
+/* The similarity phi(q).phi(k) in closed form: 1 + s/sqrt(d') + s^2/(2 d'), s = q.k */
+static double taylor_weight(const double *qi, const double *kj, int dp) {
+    double s = 0.0;
+    for (int m = 0; m < dp; ++m) s += qi[m] * kj[m];
+    return 1.0 + s / sqrt((double)dp) + s * s / (2.0 * (double)dp);
+}
+
+/* One output row i of one head, straight from the definition. */
+void oracle_linattn_row(const double *q, const double *k, const double *v, int L, int dp, int dv,
+                        int i, double *y_row) {
+    (void)L;
+    double den = 0.0;
+    for (int c = 0; c < dv; ++c) y_row[c] = 0.0;
+    for (int j = 0; j <= i; ++j) {
+        const double w = taylor_weight(q + (size_t)i * dp, k + (size_t)j * dp, dp);
+        den += w;
+        for (int c = 0; c < dv; ++c) y_row[c] += w * v[(size_t)j * dv + c];
+    }
+    for (int c = 0; c < dv; ++c) y_row[c] /= (den + ORACLE_EPS);
+}
+
+/*
+ * Quadratic definition for all heads.  S and z (nullable together) receive the
+ * final state sum_j phi(k_j) v_j^T and sum_j phi(k_j), accumulated directly.
+ */
+void oracle_linattn_quadratic(const double *q, const double *k, const double *v, double *y, double *S,
+                              double *z, int B, int H, int L, int dp, int dv) {
+    const int D = oracle_feature_dim(dp);
+    const long nh = (long)B * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long bh = 0; bh < nh; ++bh) {
+        const double *qh = q + (size_t)bh * L * dp;
+        const double *kh = k + (size_t)bh * L * dp;
+        const double *vh = v + (size_t)bh * L * dv;
+        double *yh = y + (size_t)bh * L * dv;
+        for (int i = 0; i < L; ++i) oracle_linattn_row(qh, kh, vh, L, dp, dv, i, yh + (size_t)i * dv);
+        if (S && z) {
+            double *Sh = S + (size_t)bh * D * dv;
+            double *zh = z + (size_t)bh * D;
+            double *f = (double *)malloc(sizeof(double) * (size_t)D);
+            memset(Sh, 0, sizeof(double) * (size_t)D * dv);
+            memset(zh, 0, sizeof(double) * (size_t)D);
+            for (int j = 0; j < L; ++j) {
+                oracle_phi(kh + (size_t)j * dp, dp, f);
+                for (int a = 0; a < D; ++a) {
+                    zh[a] += f[a];
+                    for (int c = 0; c < dv; ++c) Sh[(size_t)a * dv + c] += f[a] * vh[(size_t)j * dv + c];
+                }
+            }
+            free(f);
+        }
+    }
+}
+
+/*
+ * Recurrent form.  S, z are read as the initial state and overwritten with the
+ * final one.  Per token: S += phi(k) v^T; z += phi(k); then
+ * y = phi(q) S / (phi(q) z + eps).
+ */
+void oracle_linattn_recurrent(const double *q, const double *k, const double *v, double *y, double *S,
+                              double *z, int B, int H, int L, int dp, int dv) {
+    const int D = oracle_feature_dim(dp);
+    const long nh = (long)B * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long bh = 0; bh < nh; ++bh) {
+        const double *qh = q + (size_t)bh * L * dp;
+        const double *kh = k + (size_t)bh * L * dp;
+        const double *vh = v + (size_t)bh * L * dv;
+        double *yh = y + (size_t)bh * L * dv;
+        double *Sh = S + (size_t)bh * D * dv;
+        double *zh = z + (size_t)bh * D;
+        double *f = (double *)malloc(sizeof(double) * (size_t)D);
+        double *g = (double *)malloc(sizeof(double) * (size_t)D);
+        for (int i = 0; i < L; ++i) {
+            oracle_phi(kh + (size_t)i * dp, dp, f);
+            for (int a = 0; a < D; ++a) {
+                zh[a] += f[a];
+                for (int c = 0; c < dv; ++c) Sh[(size_t)a * dv + c] += f[a] * vh[(size_t)i * dv + c];
+            }
+            oracle_phi(qh + (size_t)i * dp, dp, g);
+            double den = 0.0;
+            for (int a = 0; a < D; ++a) den += g[a] * zh[a];
+            for (int c = 0; c < dv; ++c) {
+                double num = 0.0;
+                for (int a = 0; a < D; ++a) num += g[a] * Sh[(size_t)a * dv + c];
+                yh[(size_t)i * dv + c] = num / (den + ORACLE_EPS);
+            }
+        }
+        free(f);
+        free(g);
+    }
+}
+
+/* Sliding-window softmax attention: query i sees keys max(0, i-w+1) .. i. */
+void oracle_swa(const double *q, const double *k, const double *v, double *y, int B, int H, int L, int d,
+                int w, double scale) {
+    const long nh = (long)B * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long bh = 0; bh < nh; ++bh) {
+        const double *qh = q + (size_t)bh * L * d;
+        const double *kh = k + (size_t)bh * L * d;
+        const double *vh = v + (size_t)bh * L * d;
+        double *yh = y + (size_t)bh * L * d;
+        double *p = (double *)malloc(sizeof(double) * (size_t)(w > 0 ? w : 1));
+        for (int i = 0; i < L; ++i) {
+            const int lo = (i - w + 1 > 0) ? i - w + 1 : 0;
+            double mx = -INFINITY;
+            for (int j = lo; j <= i; ++j) {
+                double s = 0.0;
+                for (int m = 0; m < d; ++m) s += qh[(size_t)i * d + m] * kh[(size_t)j * d + m];
+                p[j - lo] = s * scale;
+                if (p[j - lo] > mx) mx = p[j - lo];
+            }
+            double sum = 0.0;
+            for (int j = lo; j <= i; ++j) {
+                p[j - lo] = exp(p[j - lo] - mx);
+                sum += p[j - lo];
+            }
+            for (int c = 0; c < d; ++c) {
+                double acc = 0.0;
+                for (int j = lo; j <= i; ++j) acc += p[j - lo] * vh[(size_t)j * d + c];
+                yh[(size_t)i * d + c] = acc / sum;
+            }
+        }
+        free(p);
+    }
+}
+
+/* Quadratic definition, one head, long double accumulation (tiny inputs only). */
+void oracle_linattn_quadratic_ld(const double *q, const double *k, const double *v, double *y, int L,
+                                 int dp, int dv) {
+    for (int i = 0; i < L; ++i) {
+        long double den = 0.0L;
+        long double *num = (long double *)calloc((size_t)dv, sizeof(long double));
+        for (int j = 0; j <= i; ++j) {
+            long double s = 0.0L;
+            for (int m = 0; m < dp; ++m) s += (long double)q[(size_t)i * dp + m] * (long double)k[(size_t)j * dp + m];
+            const long double w = 1.0L + s / sqrtl((long double)dp) + s * s / (2.0L * (long double)dp);
+            den += w;
+            for (int c = 0; c < dv; ++c) num[c] += w * (long double)v[(size_t)j * dv + c];
+        }
+        for (int c = 0; c < dv; ++c) y[(size_t)i * dv + c] = (double)(num[c] / (den + (long double)ORACLE_EPS));
+        free(num);
+    }
+}
