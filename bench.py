@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the Based hot path on B200 (one process per GPU).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line on rank 0.  The headline `value` is prefill tokens/s of
+`based_prefill` on the named workload (device-resident inputs, rotating buffer sets
+larger than L2); the same line carries the decode-step and sliding-window results
+(`decode`, `swa`), the other prefill configurations (`prefill_configs`), the
+end-to-end number through host buffers (`e2e`), the roofline of the dominant kernel
+and the CPU oracle timed on the host cores (`cpu_baseline`).
+
+Every (b, h) head is independent, so N GPUs run N copies of the per-GPU workload with
+no data-path collective ("weak" scaling); time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed
+    regions run (read-only queries)."""
+
+    BAD = {"hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40}
+    NOTE = {"sw_power_cap": 0x4}
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self.active = False     # set True by the bench while GPU work is in flight
+
+    def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+            return self
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+        return self
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                if self.active:
+                    self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)) if hasattr(
+                        nv, "nvmlDeviceGetCurrentClocksEventReasons") else int(
+                        nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                    for name, bit in {**self.BAD, **self.NOTE}.items():
+                        if mask & bit:
+                            self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join(timeout=1.0)
+        return {
+            "sm_mhz": statistics.median(self.samples) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": sorted(self.reasons),
+            "samples": len(self.samples),
+        }
+
+
+# --------------------------------------------------------------------------- helpers
+def io_code(w):
+    return 0 if w.dtype == "f32" else 1
+
+
+def prefill_alg_flops_per_token_head(d_v: int, chunk: int = 64) -> float:
+    """Tensor-core work the method itself needs per token and head: read-out and state
+    update over the 273 features (4*273*d_v) plus the in-chunk quadratic part
+    (2*chunk*(16+d_v)) at the reference chunk of 64 tokens."""
+    return 4.0 * 273 * d_v + 2.0 * chunk * (16 + d_v)
+
+
+def prefill_alg_bytes(w, with_state: bool) -> float:
+    esz = 4 if w.dtype == "f32" else 2
+    per_tok = esz * (2 * w.d_feat + 2 * w.d_v)
+    b = float(w.B * w.H * w.L) * per_tok
+    if with_state:
+        b += w.B * w.H * (273 * w.d_v + 273) * 4.0
+    return b
+
+
+def time_region(fn_step, steps: int, warmup: int, torch, dist_on: bool):
+    """W warm-up steps, then K steps between two events on the current stream, with a
+    barrier and a device synchronise on both sides.  Returns ms for the K steps (max
+    over ranks when distributed)."""
+    import torch.distributed as dist
+    for i in range(warmup):
+        fn_step(i)
+    torch.cuda.synchronize()
+    if dist_on:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        fn_step(warmup + i)
+    e1.record()
+    torch.cuda.synchronize()
+    if dist_on:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    if dist_on:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms
+
+
+def device_inputs(w, n_sets: int, torch, seed: int = 0):
+    """n_sets independent device-resident (q, k, v, out) sets drawn on the device with the
+    workload's distributions (seeded)."""
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    dt = w.torch_dtype
+    sets = []
+    for _ in range(n_sets):
+        q = (torch.randn(w.B, w.H, w.L, w.d_feat, generator=g, device="cuda") * w.qk_scale).to(dt)
+        k = (torch.randn(w.B, w.H, w.L, w.d_feat, generator=g, device="cuda") * w.qk_scale).to(dt)
+        v = torch.randn(w.B, w.H, w.L, w.d_v, generator=g, device="cuda").to(dt)
+        sets.append((q, k, v, torch.empty_like(v)))
+    return sets
+
+
+def n_sets_for(bytes_per_set: float) -> int:
+    return max(2, int(-(-1.5 * L2_BYTES // bytes_per_set)))
+
+
+# --------------------------------------------------------------------------- the arms
+def bench_prefill(w, steps, warmup, torch, based, dist_on, peaks):
+    with_state = w.return_state
+    per_set = prefill_alg_bytes(w, with_state)
+    sets = device_inputs(w, n_sets_for(per_set), torch)
+    kv, z = based.new_state(w.B, w.H, w.d_v) if with_state else (None, None)
+    need = based.based_prefill_workspace_bytes(w.B, w.H, w.L, w.d_feat, w.d_v, io_code(w))
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
+
+    def step(i):
+        q, k, v, o = sets[i % len(sets)]
+        based.based_prefill(q, k, v, out=o, kv_state=kv, z_state=z, workspace=ws)
+
+    n0 = based.launch_count()
+    ms = time_region(step, steps, warmup, torch, dist_on)
+    launches = (based.launch_count() - n0) * steps // (steps + warmup)
+    assert based.based_poll_error() == 0
+    t = ms * 1e-3 / steps
+    tokens = w.B * w.L
+    flops = prefill_alg_flops_per_token_head(w.d_v) * w.B * w.H * w.L
+    res = {
+        "workload": w.name, "tokens_per_s": tokens / t, "ms_per_step": ms / steps,
+        "alg_tflops": flops / t / 1e12, "alg_gbs": per_set / t / 1e9,
+        "frac_tensor_peak": flops / t / 1e12 / peaks["bf16_tflops"],
+        "frac_hbm_peak": per_set / t / 1e9 / peaks["hbm_gbs"],
+        "buffer_sets": len(sets), "launches_per_step": launches // steps if steps else 0,
+    }
+    return res, launches, sets
+
+
+def bench_prefill_e2e(w, steps, warmup, torch, based, dist_on):
+    """Same call, but every step copies q, k, v from pinned host memory and reads the
+    output back to pinned host memory inside the timed region."""
+    gen = torch.Generator(device="cpu").manual_seed(0)
+    dt = w.torch_dtype
+    hq = (torch.randn(w.B, w.H, w.L, w.d_feat, generator=gen) * w.qk_scale).to(dt).pin_memory()
+    hk = (torch.randn(w.B, w.H, w.L, w.d_feat, generator=gen) * w.qk_scale).to(dt).pin_memory()
+    hv = torch.randn(w.B, w.H, w.L, w.d_v, generator=gen).to(dt).pin_memory()
+    ho = torch.empty_like(hv).pin_memory()
+    dq, dk, dv_ = (torch.empty_like(t, device="cuda") for t in (hq, hk, hv))
+    do = torch.empty_like(dv_)
+    kv, z = based.new_state(w.B, w.H, w.d_v) if w.return_state else (None, None)
+    need = based.based_prefill_workspace_bytes(w.B, w.H, w.L, w.d_feat, w.d_v, io_code(w))
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
+
+    def step(i):
+        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv_.copy_(hv, non_blocking=True)
+        based.based_prefill(dq, dk, dv_, out=do, kv_state=kv, z_state=z, workspace=ws)
+        ho.copy_(do, non_blocking=True)
+
+    ms = time_region(step, steps, warmup, torch, dist_on)
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
+    d2h = ho.numel() * ho.element_size()
+    return {"value": w.B * w.L / (ms * 1e-3 / steps), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms / steps}
+
+
+def bench_decode(w, steps, warmup, torch, based, dist_on, peaks):
+    """cfg-4 style generation: `steps` sequential decode steps on a batch whose fp32 state
+    (B*H*273*d_v*4 bytes, larger than L2) comes from a prompt prefill."""
+    g = torch.Generator(device="cuda").manual_seed(1)
+    dt = w.torch_dtype
+    Lp = min(w.L, 256)     # the state's size does not depend on the prompt length
+    q = torch.randn(w.B, w.H, Lp, w.d_feat, generator=g, device="cuda").to(dt)
+    k = torch.randn(w.B, w.H, Lp, w.d_feat, generator=g, device="cuda").to(dt)
+    v = torch.randn(w.B, w.H, Lp, w.d_v, generator=g, device="cuda").to(dt)
+    kv, z = based.new_state(w.B, w.H, w.d_v)
+    based.based_prefill(q, k, v, kv_state=kv, z_state=z)
+    del q, k, v
+    nbuf = 8
+    qs = torch.randn(nbuf, w.B, w.H, w.d_feat, generator=g, device="cuda").to(dt)
+    ks = torch.randn(nbuf, w.B, w.H, w.d_feat, generator=g, device="cuda").to(dt)
+    vs = torch.randn(nbuf, w.B, w.H, w.d_v, generator=g, device="cuda").to(dt)
+    out = torch.empty(w.B, w.H, w.d_v, device="cuda", dtype=dt)
+
+    def step(i):
+        j = i % nbuf
+        based.based_decode_step(qs[j], ks[j], vs[j], kv, z, out=out)
+
+    ms = time_region(step, steps, warmup, torch, dist_on)
+    assert based.based_poll_error() == 0
+    t = ms * 1e-3 / steps
+    state_bytes = 2.0 * w.B * w.H * 273 * w.d_v * 4
+    esz = 2 if w.dtype == "bf16" else 4
+    all_bytes = state_bytes + w.B * w.H * (2 * 273 * 4 + esz * (2 * w.d_feat + 2 * w.d_v))
+    return {
+        "workload": w.name, "metric": "decode_tokens_per_s", "value": w.B / t, "unit": "tokens/s",
+        "us_per_step": t * 1e6, "steps": steps,
+        "roofline": {"bound": "hbm", "achieved": state_bytes / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": state_bytes / t / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                     "achieved_all_bytes": all_bytes / t / 1e9, "peak_source": peaks["source"]},
+    }
+
+
+def bench_swa(w, steps, warmup, torch, based, dist_on, peaks):
+    g = torch.Generator(device="cuda").manual_seed(2)
+    dt = w.torch_dtype
+    d = w.swa_d
+    per_set = 4.0 * w.B * w.H * w.L * d * 2
+    sets = []
+    for _ in range(n_sets_for(per_set)):
+        q, k, v = (torch.randn(w.B, w.H, w.L, d, generator=g, device="cuda").to(dt) for _ in range(3))
+        sets.append((q, k, v, torch.empty_like(v)))
+
+    def step(i):
+        q, k, v, o = sets[i % len(sets)]
+        based.swa_forward(q, k, v, out=o, window=w.swa_window)
+
+    ms = time_region(step, steps, warmup, torch, dist_on)
+    assert based.based_poll_error() == 0
+    t = ms * 1e-3 / steps
+    return {
+        "workload": w.name, "metric": "swa_tokens_per_s", "value": w.B * w.L / t, "unit": "tokens/s",
+        "ms_per_step": t * 1e3, "window": w.swa_window,
+        "roofline": {"bound": "hbm", "achieved": per_set / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": per_set / t / 1e9 / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
+    }
+
+
+def cpu_oracle_sample(w, budget_heads: int):
+    """The oracle's recurrent form, as it stands, on the first `budget_heads` heads of the
+    workload's seeded host inputs.  Returns (tokens/s scaled to whole tokens, cores, text)."""
+    import oracle
+    from paper_2402_18668_b200 import workloads as wl
+    heads = min(budget_heads, w.B * w.H)
+    ws = w.scaled(B=1, H=heads)
+    q, k, v = wl.prefill_inputs(ws, wl.generator(0))
+    q, k, v = wl.to_f64(q), wl.to_f64(k), wl.to_f64(v)
+    t0 = time.perf_counter()
+    oracle.linattn_recurrent(q, k, v)
+    dt = time.perf_counter() - t0
+    token_heads_per_s = heads * w.L / dt
+    return token_heads_per_s / w.H, oracle.num_threads(), (
+        f"recurrent-form oracle (fp64, OpenMP) on {heads} of {w.B * w.H} heads x {w.L} tokens of {w.name}, "
+        f"{dt:.2f} s; tokens/s = token-heads/s / H")
+
+
+# --------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2_360m_prefill")
+    ap.add_argument("--skip-extras", action="store_true", help="only the headline prefill workload")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    from paper_2402_18668_b200 import workloads as wl
+    w = wl.CONFIGS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        # the reference arm of this build is the CPU oracle: rank 0 alone runs it
+        if rank != 0:
+            return
+        vals = []
+        for _ in range(args.warmup + args.steps):
+            v, cores, sample = cpu_oracle_sample(w, budget_heads=16)
+            vals.append(v)
+        vals = vals[args.warmup:]
+        value = statistics.mean(vals)
+        print(json.dumps({
+            "impl": "reference", "metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": w.B * w.L / value * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d_feat": w.d_feat, "d_v": w.d_v},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0,
+        }))
+        return
+
+    import torch
+    import torch.distributed as dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libbased has no CPU path")
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist_on = world > 1
+    if dist_on:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    import paper_2402_18668_b200 as based
+    based.lib()
+    peaks = load_peaks()
+
+    phys = local
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            phys = int(vis.split(",")[local])
+        except ValueError:
+            phys = local
+    sampler = ClockSampler(phys).start()
+    sampler.active = True
+
+    res, launches, _ = bench_prefill(w, args.steps, args.warmup, torch, based, dist_on, peaks)
+    torch.cuda.empty_cache()
+    e2e = bench_prefill_e2e(w, max(5, args.steps // 5), 3, torch, based, dist_on)
+    torch.cuda.empty_cache()
+    extras = {}
+    if not args.skip_extras:
+        others = {}
+        for name in ("cfg2_360m_prefill", "cfg3_1p3b_prefill", "cfg5_mixer_pair"):
+            if name != w.name:
+                r, _, _ = bench_prefill(wl.CONFIGS[name], max(5, args.steps // 2), 3, torch, based, dist_on, peaks)
+                others[name] = r
+                torch.cuda.empty_cache()
+        extras["prefill_configs"] = others
+        extras["decode"] = bench_decode(wl.CONFIGS["cfg4_generation"], 1024, 16, torch, based, dist_on, peaks)
+        torch.cuda.empty_cache()
+        extras["swa"] = bench_swa(wl.CONFIGS["cfg5_mixer_pair"], max(5, args.steps // 2), 3, torch, based, dist_on,
+                                  peaks)
+        torch.cuda.empty_cache()
+    sampler.active = False
+    clocks = sampler.stop()
+
+    if rank == 0:
+        cpu_val, cores, sample = cpu_oracle_sample(w, budget_heads=w.B * w.H)
+        value = res["tokens_per_s"] * world
+        e2e["value"] *= world
+        bound_tensor = res["frac_tensor_peak"] >= res["frac_hbm_peak"]
+        line = {
+            "metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": res["ms_per_step"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
+            "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d_feat": w.d_feat, "d_v": w.d_v,
+                       "per_gpu": True, "l2": f"rotating {res['buffer_sets']} input sets larger than L2 in total"},
+            "roofline": {
+                "bound": "tensor" if bound_tensor else "hbm",
+                "achieved": res["alg_tflops"] if bound_tensor else res["alg_gbs"],
+                "peak": peaks["bf16_tflops"] if bound_tensor else peaks["hbm_gbs"],
+                "unit": "TFLOP/s" if bound_tensor else "GB/s",
+                "frac": res["frac_tensor_peak"] if bound_tensor else res["frac_hbm_peak"],
+                "traffic": None, "peak_source": peaks["source"],
+                "tensor": {"achieved": res["alg_tflops"], "peak": peaks["bf16_tflops"], "frac": res["frac_tensor_peak"]},
+                "hbm": {"achieved": res["alg_gbs"], "peak": peaks["hbm_gbs"], "frac": res["frac_hbm_peak"]},
+            },
+            "cpu_baseline": {"value": cpu_val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": e2e, "gpu_launches": launches, "clocks": clocks, **extras,
+        }
+        print(json.dumps(line))
+    if dist_on:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

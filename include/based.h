@@ -1,0 +1,122 @@
+/*
+ * based.h — C ABI of the B200 (sm_100a) implementation of the Based sequence
+ * mixers (arXiv 2402.18668): causal linear attention with the 2nd-order Taylor
+ * feature map, its recurrent decode step, and exact sliding-window softmax
+ * attention.
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers to contiguous row-major arrays, owned
+ *     by the caller, 16-byte aligned (else BASED_ERR_ALIGNMENT).  `cuda_stream` is a
+ *     cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Launches are asynchronous on the given stream; no entry point synchronises
+ *     except based_poll_error.  Arguments are validated before anything is launched.
+ *   - The library never falls back to another implementation: an unsupported shape
+ *     or dtype returns BASED_ERR_UNSUPPORTED.
+ *   - No entry point allocates device memory, except where stated otherwise.
+ *   - Errors are returned as based_status; nothing throws, aborts or exits.
+ *
+ * Notation: B batch, H heads, L sequence length, d_feat = d' (width of q, k, 16),
+ * d_v head dimension of v, D = 1 + d_feat + d_feat^2 (= 273) expanded feature size.
+ *
+ * State layout (ABI-visible): kv_state [B, H, D, d_v] fp32 with d_v contiguous,
+ * z_state [B, H, D] fp32.  Feature index 0 is the constant term, 1..d_feat the
+ * linear terms x_m / d'^(1/4), and 1 + d_feat + m*d_feat + n the product
+ * x_m x_n / (sqrt(2) sqrt(d')) (the concatenation order of the feature-map module
+ * in the paper's App. B.1 listing).  Rows are not padded.
+ */
+#ifndef BASED_H_
+#define BASED_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BASED_OK = 0,
+    BASED_ERR_INVALID_ARG = 1,    /* NULL pointer, non-positive size, bad enum value */
+    BASED_ERR_UNSUPPORTED = 2,    /* valid request outside the supported set */
+    BASED_ERR_ALIGNMENT = 3,      /* a pointer is not 16-byte aligned */
+    BASED_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed */
+    BASED_ERR_DEVICE_TIMEOUT = 5, /* a bounded on-device wait gave up (reported by based_poll_error) */
+    BASED_ERR_WORKSPACE = 6       /* workspace missing or smaller than based_prefill_workspace_bytes */
+} based_status;
+
+typedef enum { BASED_F32 = 0, BASED_BF16 = 1 } based_dtype;
+
+/* flags of based_prefill */
+enum {
+    BASED_STATE_ZERO_INIT = 0, /* start from the empty state */
+    BASED_STATE_CONTINUE = 1   /* start from the state held in kv_state / z_state */
+};
+
+/*
+ * Causal Taylor linear attention over whole sequences (Sec. 4.1, Eq. (2) with the
+ * feature map of Eq. (3) scaled as in the App. B.1 listing; chunked evaluation as in
+ * Sec. 5.2 / Algorithm 1, here with the normalising denominator included):
+ *
+ *   out[i] = sum_{j<=i} w_ij v_j / (sum_{j<=i} w_ij + 1e-12),
+ *   w_ij   = phi(q_i).phi(k_j) = 1 + q_i.k_j/sqrt(d') + (q_i.k_j)^2 / (2 d')
+ *
+ * q, k      [B,H,L,d_feat]  io dtype          v, out  [B,H,L,d_v]  io dtype
+ * kv_state  [B,H,D,d_v] fp32, z_state [B,H,D] fp32: both NULL (state not wanted) or
+ *           both non-NULL.  With BASED_STATE_CONTINUE they are read as the state
+ *           before token 0 (then they must be non-NULL); on return they hold the
+ *           state after token L-1.  Accumulation and state are fp32 for both io dtypes.
+ * workspace device scratch of at least based_prefill_workspace_bytes(...) bytes
+ *           (may be NULL when that size is 0); contents are undefined afterwards.
+ * Supported: d_feat = 16; d_v in {64, 128}; io in {F32, BF16}; any L >= 1.
+ * out must not alias an input.
+ */
+based_status based_prefill(const void* q, const void* k, const void* v, void* out, float* kv_state,
+                           float* z_state, int B, int H, int L, int d_feat, int d_v, based_dtype io,
+                           int flags, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Scratch bytes based_prefill needs for these arguments (0 is possible). */
+size_t based_prefill_workspace_bytes(int B, int H, int L, int d_feat, int d_v, based_dtype io);
+
+/*
+ * One recurrent step of the same mixer (Sec. 4.1 recurrences; App. B.2 step()
+ * listing and Algorithm 2, here on raw q, k with the feature map applied on chip and
+ * with the denominator): per (b, h), update then read,
+ *
+ *   kv_state += phi(k) v^T ;  z_state += phi(k) ;
+ *   out = phi(q) kv_state / (phi(q).z_state + 1e-12)
+ *
+ * q, k [B,H,d_feat], v, out [B,H,d_v] in the io dtype; kv_state / z_state as above,
+ * updated IN PLACE.  Supported: d_feat = 16; d_v in {64, 128}; io in {F32, BF16}.
+ */
+based_status based_decode_step(const void* q, const void* k, const void* v, float* kv_state, float* z_state,
+                               void* out, int B, int H, int d_feat, int d_v, based_dtype io,
+                               void* cuda_stream);
+
+/*
+ * Exact causal softmax attention in a sliding window (Eq. (1) of Sec. 2 restricted as
+ * in Sec. 4.2: query i attends keys max(0, i-window+1) .. i):
+ *
+ *   out[i] = sum_j softmax_j(scale * q_i.k_j) v_j
+ *
+ * q, k, v, out [B,H,L,d] in the io dtype.  softmax_scale <= 0 selects 1/sqrt(d).
+ * Supported: d = 64; 1 <= window <= 128; io in {F32, BF16}; any L >= 1.
+ */
+based_status swa_forward(const void* q, const void* k, const void* v, void* out, int B, int H, int L, int d,
+                         int window, float softmax_scale, based_dtype io, void* cuda_stream);
+
+/*
+ * Synchronises the stream and returns the sticky device-side status: BASED_OK, or
+ * BASED_ERR_DEVICE_TIMEOUT if a kernel abandoned a bounded wait (its outputs are then
+ * undefined), or BASED_ERR_CUDA if the stream reported a CUDA error.  Clears the flag.
+ */
+based_status based_poll_error(void* cuda_stream);
+
+const char* based_status_string(based_status s);
+int based_version(void);
+
+/* Number of kernels this library has launched in this process (all entry points). */
+unsigned long long based_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BASED_H_ */

@@ -1,0 +1,8 @@
+"""B200-native (sm_100a) Based sequence mixers: Taylor linear attention prefill and
+decode, and sliding-window softmax attention, behind the C ABI of include/based.h."""
+from . import workloads  # noqa: F401
+from .binding import (  # noqa: F401
+    BASED_BF16, BASED_F32, BASED_OK, BASED_STATE_CONTINUE, BASED_STATE_ZERO_INIT, D_EXPANDED, D_FEAT, BasedError,
+    based_decode_step, based_poll_error, based_prefill, based_prefill_workspace_bytes, launch_count, lib,
+    new_state, status_string, swa_forward, version,
+)

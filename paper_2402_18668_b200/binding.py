@@ -1,0 +1,169 @@
+"""Thin ctypes binding of libbased.so: argument marshalling only.
+
+Every function here has the name and argument order of the C entry point it calls
+(see include/based.h); all arithmetic runs in the CUDA kernels of the library.
+torch is used for device memory and streams.  If the shared library is missing the
+import of this module's functions fails loudly — there is no other implementation.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libbased.so"
+
+BASED_OK = 0
+BASED_F32, BASED_BF16 = 0, 1
+BASED_STATE_ZERO_INIT, BASED_STATE_CONTINUE = 0, 1
+D_FEAT = 16
+D_EXPANDED = 1 + D_FEAT + D_FEAT * D_FEAT
+
+EXPORTS = (
+    "based_prefill", "based_prefill_workspace_bytes", "based_decode_step", "swa_forward", "based_poll_error",
+    "based_status_string", "based_version", "based_launch_count",
+)
+
+_lib = None
+
+
+class BasedError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libbased.so (built by paper_2402_18668_b200.build); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2402_18668_b200.build` "
+                "(there is no fallback implementation)")
+        L = ctypes.CDLL(str(LIB_PATH))
+        vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        L.based_prefill.restype = i
+        L.based_prefill.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
+        L.based_prefill_workspace_bytes.restype = sz
+        L.based_prefill_workspace_bytes.argtypes = [i, i, i, i, i, i]
+        L.based_decode_step.restype = i
+        L.based_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+        L.swa_forward.restype = i
+        L.swa_forward.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
+        L.based_poll_error.restype = i
+        L.based_poll_error.argtypes = [vp]
+        L.based_status_string.restype = ctypes.c_char_p
+        L.based_status_string.argtypes = [i]
+        L.based_version.restype = i
+        L.based_launch_count.restype = ctypes.c_ulonglong
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().based_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(lib().based_version())
+
+
+def launch_count() -> int:
+    return int(lib().based_launch_count())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return BASED_F32
+    if t.dtype == torch.bfloat16:
+        return BASED_BF16
+    raise TypeError(f"unsupported io dtype {t.dtype}")
+
+
+def _dev(*ts):
+    for t in ts:
+        if t is None:
+            continue
+        if not t.is_cuda:
+            raise ValueError("libbased takes CUDA tensors only (there is no CPU path)")
+        if not t.is_contiguous():
+            raise ValueError("tensors must be contiguous")
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != BASED_OK:
+        raise BasedError(status, where)
+
+
+def based_prefill_workspace_bytes(B: int, H: int, L: int, d_feat: int, d_v: int, io: int) -> int:
+    return int(lib().based_prefill_workspace_bytes(B, H, L, d_feat, d_v, io))
+
+
+def based_prefill(q, k, v, out=None, kv_state=None, z_state=None, flags: int = BASED_STATE_ZERO_INIT,
+                  workspace=None, stream=None):
+    """q,k [B,H,L,16], v [B,H,L,d_v] -> out [B,H,L,d_v]; kv_state/z_state (fp32) in/out if given."""
+    _dev(q, k, v, out, kv_state, z_state, workspace)
+    B, H, L, d_feat = q.shape
+    d_v = v.shape[-1]
+    if k.shape != q.shape or v.shape[:3] != q.shape[:3] or k.dtype != q.dtype or v.dtype != q.dtype:
+        raise ValueError("q, k, v shapes/dtypes disagree")
+    io = _dtype_code(q)
+    if out is None:
+        out = torch.empty_like(v)
+    need = based_prefill_workspace_bytes(B, H, L, d_feat, d_v, io)
+    if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    st = lib().based_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(kv_state), _ptr(z_state), B, H, L, d_feat,
+                             d_v, io, flags, _ptr(workspace), ws_bytes, _stream(stream))
+    _check(st, "based_prefill")
+    return out
+
+
+def based_decode_step(q, k, v, kv_state, z_state, out=None, stream=None):
+    """q,k [B,H,16], v [B,H,d_v]; kv_state [B,H,273,d_v], z_state [B,H,273] updated in place."""
+    _dev(q, k, v, kv_state, z_state, out)
+    B, H, d_feat = q.shape
+    d_v = v.shape[-1]
+    if kv_state.dtype != torch.float32 or z_state.dtype != torch.float32:
+        raise TypeError("state tensors are fp32")
+    if out is None:
+        out = torch.empty_like(v)
+    st = lib().based_decode_step(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_state), _ptr(z_state), _ptr(out), B, H, d_feat,
+                                 d_v, _dtype_code(q), _stream(stream))
+    _check(st, "based_decode_step")
+    return out
+
+
+def swa_forward(q, k, v, out=None, window: int = 64, softmax_scale: float = 0.0, stream=None):
+    """q,k,v [B,H,L,d] -> out; causal softmax over keys i-window+1..i; scale<=0 -> 1/sqrt(d)."""
+    _dev(q, k, v, out)
+    B, H, L, d = q.shape
+    if out is None:
+        out = torch.empty_like(v)
+    st = lib().swa_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, L, d, int(window), float(softmax_scale),
+                           _dtype_code(q), _stream(stream))
+    _check(st, "swa_forward")
+    return out
+
+
+def based_poll_error(stream=None) -> int:
+    return int(lib().based_poll_error(_stream(stream)))
+
+
+def new_state(B: int, H: int, d_v: int, device="cuda"):
+    """Zero-initialised (kv_state, z_state) in the ABI layout."""
+    return (torch.zeros(B, H, D_EXPANDED, d_v, dtype=torch.float32, device=device),
+            torch.zeros(B, H, D_EXPANDED, dtype=torch.float32, device=device))

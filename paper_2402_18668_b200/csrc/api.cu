@@ -1,0 +1,119 @@
+// C ABI of libbased: argument validation and dispatch.  See include/based.h for the
+// contract of every entry point.
+#include <atomic>
+#include <cstdio>
+
+#include "common.cuh"
+
+namespace based {
+
+__device__ unsigned int g_error_word = 0;
+
+based_status error_word_ptr(unsigned int** ptr) {
+    // the symbol has one instance per device: resolve it with that device current
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_error_word) != cudaSuccess) return BASED_ERR_CUDA;
+    *ptr = static_cast<unsigned int*>(p);
+    return BASED_OK;
+}
+
+static std::atomic<unsigned long long> g_launches{0};
+
+void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+based_status check_launch(const char* what) {
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        std::fprintf(stderr, "libbased: launch of %s failed: %s\n", what, cudaGetErrorString(e));
+        return BASED_ERR_CUDA;
+    }
+    return BASED_OK;
+}
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace based
+
+using namespace based;
+
+extern "C" {
+
+int based_version(void) { return 1; }
+
+unsigned long long based_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* based_status_string(based_status s) {
+    switch (s) {
+        case BASED_OK: return "ok";
+        case BASED_ERR_INVALID_ARG: return "invalid argument";
+        case BASED_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+        case BASED_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case BASED_ERR_CUDA: return "CUDA error";
+        case BASED_ERR_DEVICE_TIMEOUT: return "bounded device-side wait timed out";
+        case BASED_ERR_WORKSPACE: return "workspace missing or too small";
+    }
+    return "unknown status";
+}
+
+size_t based_prefill_workspace_bytes(int B, int H, int L, int d_feat, int d_v, based_dtype io) {
+    (void)B; (void)H; (void)L; (void)d_feat; (void)d_v; (void)io;
+    return 0;
+}
+
+based_status based_prefill(const void* q, const void* k, const void* v, void* out, float* kv_state, float* z_state,
+                           int B, int H, int L, int d_feat, int d_v, based_dtype io, int flags, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream) {
+    if (!q || !k || !v || !out || B <= 0 || H <= 0 || L <= 0) return BASED_ERR_INVALID_ARG;
+    if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
+    if (flags != BASED_STATE_ZERO_INIT && flags != BASED_STATE_CONTINUE) return BASED_ERR_INVALID_ARG;
+    if ((kv_state == nullptr) != (z_state == nullptr)) return BASED_ERR_INVALID_ARG;
+    if (flags == BASED_STATE_CONTINUE && !kv_state) return BASED_ERR_INVALID_ARG;
+    if (out == q || out == k || out == v) return BASED_ERR_INVALID_ARG;
+    if (d_feat != kDFeat || (d_v != 64 && d_v != 128)) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
+        !aligned16(z_state) || !aligned16(workspace))
+        return BASED_ERR_ALIGNMENT;
+    const size_t need = based_prefill_workspace_bytes(B, H, L, d_feat, d_v, io);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return BASED_ERR_WORKSPACE;
+    return launch_prefill_simt(q, k, v, out, kv_state, z_state, B * H, L, d_v, io, flags,
+                               static_cast<cudaStream_t>(cuda_stream));
+}
+
+based_status based_decode_step(const void* q, const void* k, const void* v, float* kv_state, float* z_state,
+                               void* out, int B, int H, int d_feat, int d_v, based_dtype io, void* cuda_stream) {
+    if (!q || !k || !v || !out || !kv_state || !z_state || B <= 0 || H <= 0) return BASED_ERR_INVALID_ARG;
+    if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
+    if (d_feat != kDFeat || (d_v != 64 && d_v != 128)) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
+        !aligned16(z_state))
+        return BASED_ERR_ALIGNMENT;
+    return launch_decode(q, k, v, kv_state, z_state, out, B * H, d_v, io, static_cast<cudaStream_t>(cuda_stream));
+}
+
+based_status swa_forward(const void* q, const void* k, const void* v, void* out, int B, int H, int L, int d,
+                         int window, float softmax_scale, based_dtype io, void* cuda_stream) {
+    if (!q || !k || !v || !out || B <= 0 || H <= 0 || L <= 0 || window <= 0) return BASED_ERR_INVALID_ARG;
+    if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
+    if (out == q || out == k || out == v) return BASED_ERR_INVALID_ARG;
+    if (d != 64 || window > 128) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return BASED_ERR_ALIGNMENT;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 0.125f;   // 1/sqrt(64)
+    return launch_swa_simt(q, k, v, out, B * H, L, window, scale, io, static_cast<cudaStream_t>(cuda_stream));
+}
+
+based_status based_poll_error(void* cuda_stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return BASED_ERR_CUDA;
+    unsigned int word = 0;
+    if (cudaMemcpyFromSymbol(&word, g_error_word, sizeof(word)) != cudaSuccess) return BASED_ERR_CUDA;
+    if (word != 0) {
+        const unsigned int zero = 0;
+        if (cudaMemcpyToSymbol(g_error_word, &zero, sizeof(zero)) != cudaSuccess) return BASED_ERR_CUDA;
+        return BASED_ERR_DEVICE_TIMEOUT;
+    }
+    return BASED_OK;
+}
+
+}  // extern "C"

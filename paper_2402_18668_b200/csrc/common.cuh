@@ -1,0 +1,50 @@
+// Shared host/device helpers of libbased (sm_100a only).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "based.h"
+
+namespace based {
+
+constexpr int kDFeat = 16;                              // d' of the paper
+constexpr int kD = 1 + kDFeat + kDFeat * kDFeat;        // 273 expanded features
+constexpr float kEps = 1e-12f;                          // eps of the paper's listings
+// feature-map scales: x / d'^(1/4) and x_m x_n / (sqrt(2) sqrt(d')), d' = 16
+constexpr float kLinScale = 0.5f;
+constexpr float kQuadScale = 0.17677669529663687f;      // 1 / (4 sqrt 2)
+
+// Device address of the sticky status word of the current device (bit 0: a bounded
+// wait timed out).  Kernels that can time out receive it as an argument.
+based_status error_word_ptr(unsigned int** ptr);
+
+// host-side bookkeeping
+void note_launch();                                     // ++launch counter
+based_status check_launch(const char* what);            // cudaGetLastError -> status
+
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// value of expanded feature f (0..272) of a raw 16-vector x held in registers/shared memory
+__device__ __forceinline__ float phi_at(const float* x, int f) {
+    if (f == 0) return 1.0f;
+    if (f <= kDFeat) return x[f - 1] * kLinScale;
+    const int p = f - 1 - kDFeat;
+    return x[p >> 4] * x[p & 15] * kQuadScale;
+}
+
+// kernel launchers (defined in the .cu files; all asynchronous on `stream`)
+based_status launch_decode(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
+                           int BH, int d_v, based_dtype io, cudaStream_t stream);
+based_status launch_prefill_simt(const void* q, const void* k, const void* v, void* out, float* kv, float* z,
+                                 int BH, int L, int d_v, based_dtype io, int flags, cudaStream_t stream);
+based_status launch_swa_simt(const void* q, const void* k, const void* v, void* out, int BH, int L, int window,
+                             float scale, based_dtype io, cudaStream_t stream);
+
+}  // namespace based

@@ -1,0 +1,122 @@
+// based_decode_step: one recurrent step of Taylor linear attention per (b, h).
+//
+// Computes the KV-state / K-state recurrences of Sec. 4.1 in the update-then-read
+// order of the App. B.2 step() listing:  S += phi(k) v^T,  z += phi(k),
+// y = phi(q) S / (phi(q).z + eps).  Unlike Algorithm 2, q and k arrive raw (16 wide)
+// and the 273 features are expanded on chip.
+//
+// The step is a pure stream over the fp32 state: each head's [273, d_v] block is
+// read once and written once (2 * 273 * d_v * 4 bytes per head), 0.5 flop per byte,
+// so the kernel is bounded by HBM bandwidth.  One CTA of 256 threads owns one head.
+// A state row is covered by d_v/4 consecutive threads with one 128-bit load each, so
+// every warp instruction touches whole 512-byte (d_v=128) or two 256-byte (d_v=64)
+// rows; loads of several rows are issued before the first dependent FMA to keep
+// many bytes in flight per SM.
+#include "common.cuh"
+
+namespace based {
+
+template <int DV, typename T>
+__global__ void __launch_bounds__(256) decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                          const T* __restrict__ v, float* __restrict__ kv,
+                                                          float* __restrict__ z, T* __restrict__ out) {
+    constexpr int TPR = DV / 4;                    // threads per state row (one float4 each)
+    constexpr int RPP = 256 / TPR;                 // rows per pass: 8 (d_v 128) or 16 (d_v 64)
+    constexpr int NPASS = (kD + RPP - 1) / RPP;    // 35 or 18
+    constexpr int UNROLL = (DV == 128) ? 7 : 6;    // 35 = 5*7, 18 = 3*6 loads in flight per thread
+    static_assert(NPASS % UNROLL == 0, "pass count must divide");
+    constexpr int DPAD = NPASS * RPP;
+
+    __shared__ float s_x[2][kDFeat];
+    __shared__ float s_pq[DPAD], s_pk[DPAD];
+    __shared__ __align__(16) float s_num[RPP][DV];
+    __shared__ float s_den[8];
+
+    const int tid = threadIdx.x;
+    const size_t head = blockIdx.x;
+    const int c4 = tid % TPR, rslot = tid / TPR;
+
+    if (tid < kDFeat) s_x[0][tid] = to_f32(q[head * kDFeat + tid]);
+    else if (tid < 2 * kDFeat) s_x[1][tid - kDFeat] = to_f32(k[head * kDFeat + tid - kDFeat]);
+    float vv[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) vv[e] = to_f32(v[head * DV + c4 * 4 + e]);
+    __syncthreads();
+    for (int f = tid; f < DPAD; f += 256) {
+        s_pq[f] = f < kD ? phi_at(s_x[0], f) : 0.f;
+        s_pk[f] = f < kD ? phi_at(s_x[1], f) : 0.f;
+    }
+    __syncthreads();
+
+    // K-state update and denominator phi(q).z
+    float dpart = 0.f;
+    float* zh = z + head * kD;
+    for (int f = tid; f < kD; f += 256) {
+        const float zn = zh[f] + s_pk[f];
+        zh[f] = zn;
+        dpart = fmaf(s_pq[f], zn, dpart);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dpart += __shfl_xor_sync(0xffffffffu, dpart, o);
+    if ((tid & 31) == 0) s_den[tid >> 5] = dpart;
+
+    // KV-state stream: S[r, :] += phi(k)[r] * v ; num += phi(q)[r] * S[r, :]
+    float4* S = reinterpret_cast<float4*>(kv + head * (size_t)kD * DV) + c4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int p0 = 0; p0 < NPASS; p0 += UNROLL) {
+        float4 s[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int r = (p0 + u) * RPP + rslot;
+            if (r < kD) s[u] = S[(size_t)r * TPR];
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int r = (p0 + u) * RPP + rslot;
+            if (r < kD) {
+                const float pk = s_pk[r], pq = s_pq[r];
+                s[u].x = fmaf(pk, vv[0], s[u].x);
+                s[u].y = fmaf(pk, vv[1], s[u].y);
+                s[u].z = fmaf(pk, vv[2], s[u].z);
+                s[u].w = fmaf(pk, vv[3], s[u].w);
+                acc.x = fmaf(pq, s[u].x, acc.x);
+                acc.y = fmaf(pq, s[u].y, acc.y);
+                acc.z = fmaf(pq, s[u].z, acc.z);
+                acc.w = fmaf(pq, s[u].w, acc.w);
+                S[(size_t)r * TPR] = s[u];
+            }
+        }
+    }
+    *reinterpret_cast<float4*>(&s_num[rslot][c4 * 4]) = acc;
+    __syncthreads();
+    if (tid < DV) {
+        float num = 0.f;
+#pragma unroll
+        for (int r = 0; r < RPP; ++r) num += s_num[r][tid];
+        float den = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) den += s_den[w];
+        out[head * DV + tid] = from_f32<T>(num / (den + kEps));
+    }
+}
+
+template <int DV, typename T>
+static based_status launch_t(const void* q, const void* k, const void* v, float* kv, float* z, void* out, int BH,
+                             cudaStream_t stream) {
+    decode_step_kernel<DV, T><<<BH, 256, 0, stream>>>(static_cast<const T*>(q), static_cast<const T*>(k),
+                                                      static_cast<const T*>(v), kv, z, static_cast<T*>(out));
+    note_launch();
+    return check_launch("decode_step_kernel");
+}
+
+based_status launch_decode(const void* q, const void* k, const void* v, float* kv, float* z, void* out, int BH,
+                           int d_v, based_dtype io, cudaStream_t stream) {
+    if (d_v == 64) {
+        return io == BASED_F32 ? launch_t<64, float>(q, k, v, kv, z, out, BH, stream)
+                               : launch_t<64, __nv_bfloat16>(q, k, v, kv, z, out, BH, stream);
+    }
+    return io == BASED_F32 ? launch_t<128, float>(q, k, v, kv, z, out, BH, stream)
+                           : launch_t<128, __nv_bfloat16>(q, k, v, kv, z, out, BH, stream);
+}
+
+}  // namespace based

@@ -1,0 +1,89 @@
+"""Host-side checks of the C ABI that need no GPU: the shared library builds, loads,
+exports every function include/based.h declares, and rejects bad arguments before
+anything is launched."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2402_18668_b200 import build
+    build.build()
+    from paper_2402_18668_b200 import binding
+    return binding.lib()
+
+
+def _declared_functions():
+    text = (ROOT / "include" / "based.h").read_text()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"\b([a-z_0-9]+)\s*\(", text)
+    return sorted({n for n in names if n.startswith(("based_", "swa_"))})
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_functions()
+    assert {"based_prefill", "based_decode_step", "swa_forward", "based_poll_error"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in based.h but not exported by libbased.so"
+    from paper_2402_18668_b200 import binding
+    assert set(binding.EXPORTS) <= set(names)
+
+
+def test_version_and_status_strings(lib):
+    assert lib.based_version() >= 1
+    seen = {lib.based_status_string(s).decode() for s in range(7)}
+    assert len(seen) == 7 and "ok" in seen
+
+
+P = ctypes.c_void_p(0x1000)        # aligned, never dereferenced: validation fails first
+U = ctypes.c_void_p(0x1008)        # misaligned
+
+
+def test_prefill_validation(lib):
+    f = lib.based_prefill
+    ok_args = dict(B=1, H=1, L=8, d_feat=16, d_v=64, io=1, flags=0)
+
+    def call(q=P, k=P, v=P, out=ctypes.c_void_p(0x2000), kv=None, z=None, ws=None, ws_bytes=0, **kw):
+        a = {**ok_args, **kw}
+        return f(q, k, v, out, kv, z, a["B"], a["H"], a["L"], a["d_feat"], a["d_v"], a["io"], a["flags"], ws,
+                 ws_bytes, None)
+
+    assert call(q=None) == 1
+    assert call(L=0) == 1
+    assert call(io=7) == 1
+    assert call(flags=5) == 1
+    assert call(kv=P, z=None) == 1                      # state pointers come in pairs
+    assert call(flags=1) == 1                           # CONTINUE needs a state
+    assert call(out=P) == 1                             # out aliases q
+    assert call(d_feat=8) == 2
+    assert call(d_v=96) == 2
+    assert call(q=U) == 3
+
+
+def test_decode_and_swa_validation(lib):
+    d = lib.based_decode_step
+    assert d(P, P, P, None, P, P, 1, 1, 16, 64, 0, None) == 1
+    assert d(P, P, P, P, P, P, 0, 1, 16, 64, 0, None) == 1
+    assert d(P, P, P, P, P, P, 1, 1, 16, 80, 0, None) == 2
+    assert d(P, P, P, P, U, P, 1, 1, 16, 64, 0, None) == 3
+    s = lib.swa_forward
+    O = ctypes.c_void_p(0x2000)
+    assert s(P, P, P, O, 1, 1, 16, 64, 0, 0.0, 1, None) == 1          # window 0
+    assert s(P, P, P, P, 1, 1, 16, 64, 64, 0.0, 1, None) == 1         # out aliases
+    assert s(P, P, P, O, 1, 1, 16, 32, 64, 0.0, 1, None) == 2         # head dim
+    assert s(P, P, P, O, 1, 1, 16, 64, 256, 0.0, 1, None) == 2        # window > 128
+    assert s(P, U, P, O, 1, 1, 16, 64, 64, 0.0, 1, None) == 3
+
+
+def test_binding_rejects_cpu_tensors():
+    import torch
+    from paper_2402_18668_b200 import binding
+    q = torch.zeros(1, 1, 4, 16)
+    v = torch.zeros(1, 1, 4, 64)
+    with pytest.raises(ValueError):
+        binding.based_prefill(q, q.clone(), v)

@@ -1,0 +1,269 @@
+"""Parity of the CUDA library against the CPU oracle (needs a B200).
+
+All calls go through the C ABI (via the thin ctypes binding).  Small and ragged
+shapes are compared element by element; the contract's full-size configurations are
+checked on sampled rows and heads that the oracle computes one by one.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2402_18668_b200 as based
+from paper_2402_18668_b200 import workloads as wl
+from parity import TOL_BF16, TOL_F32, head_err, row_err, tol_for
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+
+
+def _np(t):
+    return wl.to_f64(t)
+
+
+def _poll():
+    assert based.based_poll_error() == based.BASED_OK
+
+
+# --------------------------------------------------------------------------- cfg 1
+def test_cfg1_prefill_then_decode_fp32():
+    w = wl.CONFIGS["cfg1_tiny_f32"]
+    gen = wl.generator(0)
+    q, k, v = wl.prefill_inputs(w, gen)
+    qs, ks, vs = wl.decode_inputs(w, gen)
+    y_ref, S_ref, z_ref = oracle.linattn_quadratic(_np(q), _np(k), _np(v))
+
+    kv, z = based.new_state(w.B, w.H, w.d_v)
+    y = based.based_prefill(q.to(DEV), k.to(DEV), v.to(DEV), kv_state=kv, z_state=z)
+    _poll()
+    assert row_err(_np(y), y_ref) <= TOL_F32
+    assert head_err(_np(kv), S_ref) <= TOL_F32
+    assert head_err(_np(z), z_ref) <= TOL_F32
+
+    S, zz = S_ref, z_ref
+    for t in range(w.decode_steps):
+        y_t, S, zz = oracle.decode_step(_np(qs[t]), _np(ks[t]), _np(vs[t]), S, zz)
+        out = based.based_decode_step(qs[t].to(DEV), ks[t].to(DEV), vs[t].to(DEV), kv, z)
+        assert row_err(_np(out), y_t) <= TOL_F32, f"decode step {t}"
+    _poll()
+    assert head_err(_np(kv), S) <= TOL_F32
+    assert head_err(_np(z), zz) <= TOL_F32
+
+
+# --------------------------------------------------------------------------- prefill, element by element
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d_v", [64, 128])
+@pytest.mark.parametrize("L", [1, 7, 64, 129, 300, 515])
+def test_prefill_small_shapes(dtype, d_v, L):
+    w = wl.Workload("small", 2, 3, L, 16, d_v, dtype, 0.25 if dtype == "bf16" else 1.0)
+    q, k, v = wl.prefill_inputs(w, wl.generator(L * 7 + d_v))
+    y_ref, S_ref, z_ref = oracle.linattn_quadratic(_np(q), _np(k), _np(v))
+    kv, z = based.new_state(w.B, w.H, d_v)
+    kv.fill_(float("nan")); z.fill_(float("nan"))          # ZERO_INIT must not read the buffers
+    out = torch.full_like(v, float("nan"), device=DEV)
+    based.based_prefill(q.to(DEV), k.to(DEV), v.to(DEV), out=out, kv_state=kv, z_state=z)
+    _poll()
+    tol = tol_for(dtype)
+    assert row_err(_np(out), y_ref) <= tol
+    assert head_err(_np(kv), S_ref) <= tol
+    assert head_err(_np(z), z_ref) <= tol
+    # without state pointers the outputs are the same
+    out2 = based.based_prefill(q.to(DEV), k.to(DEV), v.to(DEV))
+    assert torch.equal(out2, out)
+
+
+@pytest.mark.parametrize("dtype,d_v,L,L1", [("f32", 64, 200, 77), ("bf16", 128, 384, 128), ("bf16", 64, 450, 131)])
+def test_prefill_continue_equals_one_pass(dtype, d_v, L, L1):
+    w = wl.Workload("split", 1, 4, L, 16, d_v, dtype, 0.5)
+    q, k, v = wl.prefill_inputs(w, wl.generator(3))
+    y_ref, S_ref, z_ref = oracle.linattn_quadratic(_np(q), _np(k), _np(v))
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    kv, z = based.new_state(w.B, w.H, d_v)
+    y1 = based.based_prefill(qd[:, :, :L1].contiguous(), kd[:, :, :L1].contiguous(), vd[:, :, :L1].contiguous(),
+                             kv_state=kv, z_state=z)
+    y2 = based.based_prefill(qd[:, :, L1:].contiguous(), kd[:, :, L1:].contiguous(), vd[:, :, L1:].contiguous(),
+                             kv_state=kv, z_state=z, flags=based.BASED_STATE_CONTINUE)
+    _poll()
+    tol = tol_for(dtype)
+    assert row_err(_np(torch.cat([y1, y2], dim=2)), y_ref) <= tol
+    assert head_err(_np(kv), S_ref) <= tol
+    assert head_err(_np(z), z_ref) <= tol
+
+
+# --------------------------------------------------------------------------- decode
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d_v", [64, 128])
+def test_decode_step_from_given_state(dtype, d_v):
+    """Steps from a non-trivial state: the state a 24-token prefix leaves (rounded to the
+    fp32 the ABI stores), so both sides start from identical numbers."""
+    B, H = 3, 5
+    w = wl.Workload("dec", B, H, 24, 16, d_v, dtype, 1.0, decode_steps=6)
+    gen = wl.generator(11)
+    qp, kp, vp = wl.prefill_inputs(w, gen)
+    qs, ks, vs = wl.decode_inputs(w, gen)
+    _, S0, z0 = oracle.linattn_recurrent(_np(qp), _np(kp), _np(vp))
+    kv0, zz0 = torch.from_numpy(S0).float(), torch.from_numpy(z0).float()
+    kv, z = kv0.to(DEV), zz0.to(DEV)
+    S, zz = _np(kv0), _np(zz0)
+    tol = tol_for(dtype)
+    for t in range(w.decode_steps):
+        y_t, S, zz = oracle.decode_step(_np(qs[t]), _np(ks[t]), _np(vs[t]), S, zz)
+        out = torch.full_like(vs[t], float("nan"), device=DEV)
+        based.based_decode_step(qs[t].to(DEV), ks[t].to(DEV), vs[t].to(DEV), kv, z, out=out)
+        assert row_err(_np(out), y_t) <= tol, f"step {t}"
+        assert head_err(_np(kv), S) <= TOL_F32          # the state is fp32 for both io dtypes
+        assert head_err(_np(z), zz) <= TOL_F32
+    _poll()
+
+
+def test_decode_chain_equals_prefill_on_gpu():
+    """Prefill over T tokens and T chained decode steps agree with each other and the oracle."""
+    B, H, T, d_v = 2, 2, 48, 64
+    w = wl.Workload("chain", B, H, T, 16, d_v, "f32", 0.7)
+    q, k, v = wl.prefill_inputs(w, wl.generator(5))
+    y_ref, S_ref, z_ref = oracle.linattn_quadratic(_np(q), _np(k), _np(v))
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    kv, z = based.new_state(B, H, d_v)
+    ys = [based.based_decode_step(qd[:, :, t].contiguous(), kd[:, :, t].contiguous(), vd[:, :, t].contiguous(), kv, z)
+          for t in range(T)]
+    y_chain = torch.stack(ys, dim=2)
+    kv2, z2 = based.new_state(B, H, d_v)
+    y_pre = based.based_prefill(qd, kd, vd, kv_state=kv2, z_state=z2)
+    _poll()
+    assert row_err(_np(y_chain), y_ref) <= TOL_F32
+    assert row_err(_np(y_pre), y_ref) <= TOL_F32
+    assert head_err(_np(kv), S_ref) <= TOL_F32 and head_err(_np(kv2), S_ref) <= TOL_F32
+    assert head_err(_np(z), z_ref) <= TOL_F32 and head_err(_np(z2), z_ref) <= TOL_F32
+
+
+# --------------------------------------------------------------------------- sliding window
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("L,window", [(1, 64), (63, 64), (64, 64), (333, 64), (200, 1), (257, 17), (400, 128), (130, 100)])
+def test_swa_small_shapes(dtype, L, window):
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    q, k, v = wl.swa_standalone_inputs(2, 3, L, 64, tdt, wl.generator(L + window))
+    ref = oracle.swa(_np(q), _np(k), _np(v), window)
+    out = torch.full_like(v, float("nan"), device=DEV)
+    based.swa_forward(q.to(DEV), k.to(DEV), v.to(DEV), out=out, window=window)
+    _poll()
+    assert row_err(_np(out), ref) <= tol_for(dtype)
+
+
+def test_swa_explicit_scale_and_large_logits():
+    q, k, v = wl.swa_standalone_inputs(1, 2, 150, 64, torch.float32, wl.generator(9))
+    q = q * 6.0
+    ref = oracle.swa(_np(q), _np(k), _np(v), 64, scale=1.0)
+    out = based.swa_forward(q.to(DEV), k.to(DEV), v.to(DEV), window=64, softmax_scale=1.0)
+    _poll()
+    assert row_err(_np(out), ref) <= TOL_F32
+
+
+# --------------------------------------------------------------------------- full-size configurations, sampled
+def _sample_rows(L, n, rng):
+    fixed = [0, 1, 63, 64, 127, 128, L // 2, L - 2, L - 1]
+    extra = rng.integers(0, L, size=n).tolist()
+    return sorted({i for i in fixed + extra if 0 <= i < L})
+
+
+@pytest.mark.parametrize("name", ["cfg2_360m_prefill", "cfg3_1p3b_prefill"])
+def test_full_size_prefill_sampled(name):
+    w = wl.CONFIGS[name]
+    q, k, v = wl.prefill_inputs(w, wl.generator(0))
+    kv, z = based.new_state(w.B, w.H, w.d_v) if w.return_state else (None, None)
+    out = based.based_prefill(q.to(DEV), k.to(DEV), v.to(DEV), kv_state=kv, z_state=z)
+    _poll()
+    out = out.cpu()
+    rng = np.random.default_rng(0)
+    heads = sorted({0, w.B * w.H - 1, *rng.integers(0, w.B * w.H, size=6).tolist()})
+    worst = 0.0
+    for bh in heads:
+        b, h = divmod(bh, w.H)
+        qh, kh, vh = _np(q[b, h]), _np(k[b, h]), _np(v[b, h])
+        for i in _sample_rows(w.L, 24, rng):
+            want = oracle.linattn_row(qh, kh, vh, i)
+            worst = max(worst, row_err(_np(out[b, h, i]), want))
+    assert worst <= TOL_BF16
+    if w.return_state:
+        for bh in heads[:3]:
+            b, h = divmod(bh, w.H)
+            _, S_ref, z_ref = oracle.linattn_recurrent(_np(q[b:b + 1, h:h + 1]), _np(k[b:b + 1, h:h + 1]),
+                                                       _np(v[b:b + 1, h:h + 1]))
+            assert head_err(_np(kv[b:b + 1, h:h + 1]), S_ref) <= TOL_BF16
+            assert head_err(_np(z[b:b + 1, h:h + 1]), z_ref) <= TOL_BF16
+
+
+def test_full_size_mixer_pair_sampled():
+    """cfg 5: L = 32768 linear-attention prefill and window-64 softmax on shared v."""
+    w = wl.CONFIGS["cfg5_mixer_pair"]
+    gen = wl.generator(0)
+    q, k, v = wl.prefill_inputs(w, gen)
+    qs, ks = wl.swa_inputs(w, gen)
+    vd = v.to(DEV)
+    out_lin = based.based_prefill(q.to(DEV), k.to(DEV), vd).cpu()
+    out_swa = based.swa_forward(qs.to(DEV), ks.to(DEV), vd, window=w.swa_window).cpu()
+    _poll()
+    rng = np.random.default_rng(1)
+    worst = 0.0
+    for bh in (0, 13, w.B * w.H - 1):
+        b, h = divmod(bh, w.H)
+        qh, kh, vh = _np(q[b, h]), _np(k[b, h]), _np(v[b, h])
+        for i in _sample_rows(w.L, 12, rng):
+            worst = max(worst, row_err(_np(out_lin[b, h, i]), oracle.linattn_row(qh, kh, vh, i)))
+    assert worst <= TOL_BF16
+    # the sliding-window oracle is cheap enough to check four whole heads
+    for bh in (0, 7, 22, w.B * w.H - 1):
+        b, h = divmod(bh, w.H)
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        ref = oracle.swa(_np(qs[sl]), _np(ks[sl]), _np(v[sl]), w.swa_window)
+        assert row_err(_np(out_swa[sl]), ref) <= TOL_BF16
+
+
+def test_full_size_generation_sampled():
+    """cfg 4: batch 128 prompt prefill, then decode steps from the resulting fp32 state
+    (a reduced number of steps here; the benchmark runs all 1024)."""
+    w = wl.CONFIGS["cfg4_generation"]
+    steps = 64
+    gen = wl.generator(0)
+    q, k, v = wl.prefill_inputs(w, gen)
+    qs, ks, vs = wl.decode_inputs(w, gen, steps=steps)
+    kv, z = based.new_state(w.B, w.H, w.d_v)
+    out = based.based_prefill(q.to(DEV), k.to(DEV), v.to(DEV), kv_state=kv, z_state=z)
+    heads = [0, 777, w.B * w.H - 1]
+    refs = {}
+    for bh in heads:
+        b, h = divmod(bh, w.H)
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        y_ref, S, zz = oracle.linattn_recurrent(_np(q[sl]), _np(k[sl]), _np(v[sl]))
+        assert row_err(_np(out[sl]), y_ref) <= TOL_BF16
+        assert head_err(_np(kv[sl]), S) <= TOL_BF16
+        refs[bh] = (S, zz)
+    del out
+    qsd, ksd, vsd = qs.to(DEV), ks.to(DEV), vs.to(DEV)
+    for t in range(steps):
+        o = based.based_decode_step(qsd[t], ksd[t], vsd[t], kv, z)
+        for bh in heads:
+            b, h = divmod(bh, w.H)
+            sl = (slice(b, b + 1), slice(h, h + 1))
+            S, zz = refs[bh]
+            y_t, S, zz = oracle.decode_step(_np(qs[t][sl]), _np(ks[t][sl]), _np(vs[t][sl]), S, zz)
+            refs[bh] = (S, zz)
+            assert row_err(_np(o[sl]), y_t) <= TOL_BF16, (t, bh)
+    _poll()
+    for bh in heads:
+        b, h = divmod(bh, w.H)
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        assert head_err(_np(kv[sl]), refs[bh][0]) <= TOL_BF16
+        assert head_err(_np(z[sl]), refs[bh][1]) <= TOL_BF16
+
+
+# --------------------------------------------------------------------------- errors on the device box
+def test_unsupported_requests_fail_loudly():
+    q = torch.zeros(1, 1, 4, 16, device=DEV)
+    v = torch.zeros(1, 1, 4, 96, device=DEV)
+    with pytest.raises(based.BasedError) as e:
+        based.based_prefill(q, q.clone(), v)
+    assert e.value.status == 2
+    n0 = based.launch_count()
+    based.based_prefill(q, q.clone(), torch.zeros(1, 1, 4, 64, device=DEV))
+    assert based.launch_count() > n0
