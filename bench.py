@@ -309,8 +309,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_360m_prefill")
     ap.add_argument("--skip-extras", action="store_true", help="only the headline prefill workload")
+    ap.add_argument("--profile", choices=["prefill", "decode", "swa"],
+                    help="run only this arm on --shape (small cases for ncu captures) and print its result")
+    ap.add_argument("--shape", default="", help="B,H,L,d_v for --profile (defaults to the arm's benchmark shape)")
     args = ap.parse_args()
-    if args.warmup < 3:
+    if args.warmup < 3 and not args.profile:
         args.warmup = 3
 
     from paper_2402_18668_b200 import workloads as wl
@@ -352,6 +355,23 @@ def main():
     import paper_2402_18668_b200 as based
     based.lib()
     peaks = load_peaks()
+
+    if args.profile:
+        base = {"prefill": w, "decode": wl.CONFIGS["cfg4_generation"], "swa": wl.CONFIGS["cfg5_mixer_pair"]}[args.profile]
+        if args.shape:
+            B, H, L, dv = (int(x) for x in args.shape.split(","))
+            base = base.scaled(name=f"{base.name}[{args.shape}]", B=B, H=H, L=L, d_v=dv)
+        if args.profile == "prefill":
+            r, _, _ = bench_prefill(base, args.steps, args.warmup, torch, based, dist_on, peaks)
+        elif args.profile == "decode":
+            r = bench_decode(base, args.steps, args.warmup, torch, based, dist_on, peaks)
+        else:
+            r = bench_swa(base, args.steps, args.warmup, torch, based, dist_on, peaks)
+        if rank == 0:
+            print(json.dumps({"profile": args.profile, **r}))
+        if dist_on:
+            dist.destroy_process_group()
+        return
 
     phys = local
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")

@@ -21,7 +21,7 @@ NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xptxas=-v",
     "-I", str(INCLUDE), "-I", str(CSRC),
-]
+] + (os.environ.get("BASED_NVCC_EXTRA", "").split())
 
 
 def _nvcc() -> str:

@@ -56,8 +56,9 @@ const char* based_status_string(based_status s) {
 }
 
 size_t based_prefill_workspace_bytes(int B, int H, int L, int d_feat, int d_v, based_dtype io) {
-    (void)B; (void)H; (void)L; (void)d_feat; (void)d_v; (void)io;
-    return 0;
+    if (B <= 0 || H <= 0 || L <= 0 || d_feat != kDFeat || (d_v != 64 && d_v != 128)) return 0;
+    if (io != BASED_BF16) return 0;            // the fp32 path keeps its state in registers
+    return prefill_tc_workspace_bytes(B * H, L, d_v);
 }
 
 based_status based_prefill(const void* q, const void* k, const void* v, void* out, float* kv_state, float* z_state,
@@ -76,6 +77,10 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
         return BASED_ERR_ALIGNMENT;
     const size_t need = based_prefill_workspace_bytes(B, H, L, d_feat, d_v, io);
     if (need > 0 && (!workspace || workspace_bytes < need)) return BASED_ERR_WORKSPACE;
+    if ((long long)B * H > 65535 && io == BASED_BF16) return BASED_ERR_UNSUPPORTED;
+    if (io == BASED_BF16)
+        return launch_prefill_tc(q, k, v, out, kv_state, z_state, B * H, L, d_v, flags, workspace,
+                                 static_cast<cudaStream_t>(cuda_stream));
     return launch_prefill_simt(q, k, v, out, kv_state, z_state, B * H, L, d_v, io, flags,
                                static_cast<cudaStream_t>(cuda_stream));
 }

@@ -1,0 +1,751 @@
+// based_prefill, bf16 tensor-core path (tcgen05 + TMEM + TMA, sm_100a).
+//
+// Causal Taylor linear attention (Sec. 4.1, Eq. (2)/(3)) evaluated chunk by chunk as in
+// Sec. 5.2: within a chunk of 128 tokens the quadratic "attention" form, across chunks
+// the running KV-state.  Unlike Algorithm 1 the whole expanded state of a head lives in
+// tensor memory as one fp32 accumulator, and the expanded features never leave the SM.
+//
+// Per chunk c of one (b, h) (or of one sequence segment of it) five tensor-core steps:
+//   (1) scores   T[128,128]  = Q_c K_c^T                        (K = 16)
+//   (z) z       += colsum(phi(K_c))         as  phi(K_c)^T x ones   (M = features, N = 16)
+//   (5) S^T     += V_c^T phi(K_c)           [d_v lanes x 160 feature columns, fp32 in TMEM]
+//   (4) Y        = phi(Q_c) [S_prev | z_prev]   (K = 160; the extra column is the
+//                                                cross-chunk part of the denominator)
+//   (3) Y       += P V_c,  P = (1 + T/4 + T^2/32) masked to j <= i, bf16, read from TMEM
+// and three ALU jobs: the polynomial + mask + row sum on the scores, the expansion of
+// q and k rows into feature rows (shared memory, UMMA operand layout), and a bf16 copy of
+// the fp32 state into shared memory as the B operand of (4).
+//
+// Features are kept in a symmetric basis of 153 (padded to 160) instead of 273: with
+// x' = x/2,  [x' (16) | x'_m x'_(m+o) for o = 0..7 (the o = 0 block scaled by 1/sqrt 2) |
+// x'_m x'_(m+8), m < 8 | 1 | 0 x 7].  Its inner products equal those of the 273-feature
+// map; the state is expanded to / folded from the 273-row ABI layout at the kernel's edges.
+//
+// Warp roles (448 threads): warps 0-3 "row" group (one thread per query row / TMEM lane:
+// polynomial + mask), warps 4-7 "feature" group (one thread per token: phi expansion),
+// warps 8-11 "state" group (one thread per TMEM lane: bf16 state copy, normalise + store,
+// state I/O), warp 12 TMA producer, warp 13 MMA issuer.  All cross-role hand-offs are
+// mbarriers with bounded waits.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "sm100.cuh"
+
+namespace based {
+
+using namespace sm100;
+
+namespace {
+
+constexpr int kC = 128;            // tokens per chunk
+constexpr int kF = 160;            // internal feature count (153 padded to a multiple of 16)
+constexpr int kFBlk = 5;           // 32-feature SWIZZLE_64B blocks
+constexpr int kStages = 2;
+constexpr int kThreads = 448;
+constexpr int kWarpTma = 12, kWarpMma = 13;
+constexpr float kRsqrt2 = 0.70710678118654752f;
+
+// ---- workspace layout of one (head, segment) partial state: [kF][DV] fp32 then [kF] fp32
+__host__ __device__ constexpr size_t seg_state_floats(int dv) { return (size_t)kF * dv + kF; }
+
+template <int DV>
+struct Cfg {
+    static constexpr int kNY = DV + 16;                         // Y columns: d_v numerators + denominator block
+    static constexpr uint32_t kQKBytes = kC * 32;               // one q or k tile (16 bf16 per token)
+    static constexpr uint32_t kVBytes = kC * DV * 2;
+    static constexpr uint32_t kStageBytes = 2 * kQKBytes + kVBytes;
+    static constexpr uint32_t kPhiBytes = kFBlk * kC * 64;      // 40 KB
+    static constexpr uint32_t kPhiBlk = kC * 64;                // bytes of one 32-feature block
+    static constexpr uint32_t kScBlk = kNY * 64;
+    static constexpr uint32_t kScBytes = kFBlk * kScBlk;
+    static constexpr uint32_t kOnesBytes = 4096;
+    static constexpr uint32_t offStage = 0;
+    static constexpr uint32_t offPK = kStages * kStageBytes;
+    static constexpr uint32_t offPQ = offPK + kPhiBytes;        // must follow PK (the last z tile over-reads into it)
+    static constexpr uint32_t offSc = offPQ + kPhiBytes;
+    static constexpr uint32_t offOnes = offSc + kScBytes;
+    static constexpr uint32_t offBars = offOnes + kOnesBytes;
+    static constexpr uint32_t kSmemBytes = offBars + 256 + 1024 + 1024;   // barriers, row sums, alignment slack
+    // TMEM columns
+    static constexpr uint32_t colT = 0;                          // scores, overwritten in place by P
+    static constexpr uint32_t colY = 128;
+    static constexpr uint32_t colS = colY + kNY;
+    static constexpr uint32_t colZ0 = colS + kF;
+    static constexpr uint32_t colZ1 = colZ0 + 16;
+    static_assert(colZ1 + 16 <= 512, "TMEM budget");
+    static_assert(kScBlk % 1024 == 0 && kStageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligned");
+};
+
+enum Bar { kFull0 = 0, kFull1, kEmpty0, kEmpty1, kG1, kP, kG2, kG4, kG3, kYfree, kPK, kPQ, kSC, kNumBars };
+
+struct Params {
+    __nv_bfloat16* out;
+    float* kv_abi;        // [BH, 273, DV] or null
+    float* z_abi;         // [BH, 273] or null
+    float* ws;            // per (head, segment) partial states, internal layout
+    unsigned int* err;
+    int L;                // tokens per head
+    int nseg;             // segments per head
+    int seg_len;          // tokens per segment (multiple of kC)
+    int continue_abi;     // start from the ABI state in kv_abi / z_abi
+#ifdef BASED_TRACE
+    unsigned long long* trace;
+#endif
+};
+
+#ifdef BASED_TRACE
+#define TRACE(role, c, ev)                                                                   \
+    do {                                                                                     \
+        if (p.trace && blockIdx.x == gridDim.x - 1 && blockIdx.y == 0 && (c) < 64)           \
+            p.trace[((role) * 64 + (c)) * 8 + (ev)] = clock64();                             \
+    } while (0)
+#else
+#define TRACE(role, c, ev) do {} while (0)
+#endif
+
+// ---- internal feature index -> rows of the 273-row ABI layout -------------------------
+struct AbiRows { int a, b; float scale; };   // b < 0: single row
+__host__ __device__ constexpr AbiRows abi_rows(int i) {
+    if (i < 16) return {1 + i, -1, 1.f};
+    if (i < 144) {
+        const int o = (i - 16) / 16, m = (i - 16) % 16, n = (m + o) % 16;
+        if (o == 0) return {17 + 17 * m, -1, 1.f};
+        return {17 + 16 * m + n, 17 + 16 * n + m, kRsqrt2};
+    }
+    if (i < 152) {
+        const int m = i - 144, n = m + 8;
+        return {17 + 16 * m + n, 17 + 16 * n + m, kRsqrt2};
+    }
+    if (i == 152) return {0, -1, 1.f};
+    return {-1, -1, 0.f};
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ uint32_t mul2(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmul2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
+    return *reinterpret_cast<uint32_t*>(&r);
+}
+
+// Expand one raw 16-vector (8 packed bf16 pairs) into its 160 internal features and write
+// them as row t of a [128 tokens][160 features] tile made of five SWIZZLE_64B blocks.
+__device__ __forceinline__ void write_phi_row(const uint32_t (&x)[8], uint8_t* tile, int t, bool valid) {
+    const uint32_t kHalf = 0x3F003F00u;      // (0.5, 0.5)
+    const uint32_t kRs2 = 0x3F353F35u;       // (1/sqrt2, 1/sqrt2) rounded to bf16
+    uint32_t E[8], O[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) E[i] = valid ? mul2(x[i], kHalf) : 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) O[i] = __byte_perm(E[i], E[(i + 1) & 7], 0x5432);   // (x'_{2i+1}, x'_{2i+2})
+    uint8_t* row = tile + (t >> 3) * 512 + (t & 7) * 64;
+    const uint32_t sw = (t >> 1) & 3;
+    auto store = [&](int j, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+        *reinterpret_cast<uint4*>(row + (j >> 2) * (kC * 64) + (((j & 3) ^ sw) << 4)) = make_uint4(a, b, c, d);
+    };
+    store(0, E[0], E[1], E[2], E[3]);
+    store(1, E[4], E[5], E[6], E[7]);
+    {   // o = 0: squares, scaled by 1/sqrt 2
+        uint32_t p[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) p[i] = mul2(E[i], mul2(E[i], kRs2));
+        store(2, p[0], p[1], p[2], p[3]);
+        store(3, p[4], p[5], p[6], p[7]);
+    }
+#pragma unroll
+    for (int o = 1; o < 8; ++o) {
+        uint32_t p[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t r = (o & 1) ? O[(i + (o - 1) / 2) & 7] : E[(i + o / 2) & 7];
+            p[i] = mul2(E[i], r);
+        }
+        store(2 + 2 * o, p[0], p[1], p[2], p[3]);
+        store(3 + 2 * o, p[4], p[5], p[6], p[7]);
+    }
+    store(18, mul2(E[0], E[4]), mul2(E[1], E[5]), mul2(E[2], E[6]), mul2(E[3], E[7]));
+    store(19, valid ? 0x00003F80u : 0u, 0u, 0u, 0u);   // the constant feature 1.0
+}
+
+// Row t of a [128][16] bf16 tile written by TMA with SWIZZLE_32B.
+__device__ __forceinline__ void read_qk_row(const uint8_t* tile, int t, uint32_t (&x)[8]) {
+    const uint8_t* row = tile + (t >> 3) * 256 + (t & 7) * 32;
+    const uint32_t sw = ((t >> 2) & 1) << 4;
+    const uint4 lo = *reinterpret_cast<const uint4*>(row + (0 ^ sw));
+    const uint4 hi = *reinterpret_cast<const uint4*>(row + (16 ^ sw));
+    x[0] = lo.x; x[1] = lo.y; x[2] = lo.z; x[3] = lo.w;
+    x[4] = hi.x; x[5] = hi.y; x[6] = hi.z; x[7] = hi.w;
+}
+
+}  // namespace
+
+// One 32-column batch of scores -> 16 packed bf16 weight pairs; adds the weights to den.
+// DIAG: the batch straddles the diagonal (key column i of the batch is visible iff i <= lane).
+template <bool DIAG>
+__device__ __forceinline__ void poly_batch(const uint32_t (&sc)[32], uint32_t (&pk)[16], float& den, int lane) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float s0 = __uint_as_float(sc[2 * i]), s1 = __uint_as_float(sc[2 * i + 1]);
+        float w0 = fmaf(s0, fmaf(s0, 0.03125f, 0.25f), 1.0f);
+        float w1 = fmaf(s1, fmaf(s1, 0.03125f, 0.25f), 1.0f);
+        if (DIAG) {
+            w0 = (2 * i <= lane) ? w0 : 0.f;
+            w1 = (2 * i + 1 <= lane) ? w1 : 0.f;
+        }
+        den += w0 + w1;
+        pk[i] = pack_bf16(w0, w1);
+    }
+}
+
+template <int DV, bool STATE_ONLY>
+__global__ void __launch_bounds__(kThreads, 1)
+    prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                      const __grid_constant__ CUtensorMap tm_v, const Params p) {
+    using C = Cfg<DV>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offBars);
+    uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + kNumBars);
+    volatile uint32_t* abort_flag = tmem_base_s + 1;
+    float* s_den = reinterpret_cast<float*>(tmem_base_s + 2);      // [2][128] row sums of the in-chunk weights
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int seg = blockIdx.x, head = blockIdx.y;
+    const int tok_begin = seg * p.seg_len;
+    const int tok_end = min(p.L, tok_begin + p.seg_len);
+    const int nch = (tok_end - tok_begin + kC - 1) / kC;
+
+    uint8_t* sPK = smem + C::offPK;
+    uint8_t* sPQ = smem + C::offPQ;
+    uint8_t* sSc = smem + C::offSc;
+    uint8_t* sOnes = smem + C::offOnes;
+
+    if (tid == 0) {
+        mbar_init(&bars[kFull0], 1); mbar_init(&bars[kFull1], 1);
+        mbar_init(&bars[kEmpty0], 1); mbar_init(&bars[kEmpty1], 1);
+        mbar_init(&bars[kG1], 1); mbar_init(&bars[kG2], 1); mbar_init(&bars[kG4], 1); mbar_init(&bars[kG3], 1);
+        mbar_init(&bars[kP], 128); mbar_init(&bars[kYfree], 128); mbar_init(&bars[kPK], 128);
+        mbar_init(&bars[kPQ], 128); mbar_init(&bars[kSC], 128);
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
+    }
+    if (warp == kWarpMma) { tmem_alloc(tmem_base_s, 512); tmem_relinquish(); }
+    // ones tile (bf16 1.0) and a zeroed state-copy tile (its rows d_v+1.. stay zero for good)
+    for (uint32_t i = tid * 16; i < C::kOnesBytes; i += kThreads * 16)
+        *reinterpret_cast<uint4*>(sOnes + i) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+    for (uint32_t i = tid * 16; i < C::kScBytes; i += kThreads * 16)
+        *reinterpret_cast<uint4*>(sSc + i) = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = *tmem_base_s;
+    const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;     // TMEM lanes this warp may touch
+    bool ok = true;
+
+    if (warp == kWarpTma) {
+        // ===================================================================== TMA producer
+        if (lane == 0) {
+            for (int c = 0; c < nch && ok; ++c) {
+                const int s = c & 1;
+                ok = mbar_wait(&bars[kEmpty0 + s], ((c >> 1) & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                uint8_t* st = smem + C::offStage + s * C::kStageBytes;
+                const int tok0 = tok_begin + c * kC;
+                mbar_arrive_expect_tx(&bars[kFull0 + s], (STATE_ONLY ? 1 : 2) * C::kQKBytes + C::kVBytes);
+                if (!STATE_ONLY) tma_load_3d(st, &tm_q, &bars[kFull0 + s], 0, tok0, head);
+                tma_load_3d(st + C::kQKBytes, &tm_k, &bars[kFull0 + s], 0, tok0, head);
+#pragma unroll
+                for (int b = 0; b < DV / 64; ++b)
+                    tma_load_3d(st + 2 * C::kQKBytes + b * (kC * 128), &tm_v, &bars[kFull0 + s], b * 64, tok0, head);
+            }
+        }
+    } else if (warp == kWarpMma) {
+        // ===================================================================== MMA issuer
+        if (lane == 0) {
+            constexpr uint64_t dQK = make_smem_desc_base(16, 256, kSwizzle32B);           // K-major [128][16]
+            constexpr uint64_t dPhiK = make_smem_desc_base(16, 512, kSwizzle64B);         // K-major, 64-byte rows
+            constexpr uint64_t dPhiMN = make_smem_desc_base(C::kPhiBlk, 512, kSwizzle64B);// MN-major view of a phi tile
+            constexpr uint64_t dV = make_smem_desc_base(kC * 128, 1024, kSwizzle128B);    // MN-major [128 tok][DV]
+            constexpr uint64_t dOnes = make_smem_desc_base(16, 1024, kSwizzle128B);
+            constexpr uint32_t i1 = make_idesc_bf16(128, 128, 0, 0);
+            constexpr uint32_t iZ0 = make_idesc_bf16(128, 16, 1, 0);
+            constexpr uint32_t iZ1 = make_idesc_bf16(64, 16, 1, 0);
+            constexpr uint32_t i5 = make_idesc_bf16(DV, kF, 1, 1);
+            constexpr uint32_t i4 = make_idesc_bf16(128, C::kNY, 0, 0);
+            constexpr uint32_t i3 = make_idesc_bf16(128, DV, 0, 1);
+            const uint32_t aPK = smem_u32(sPK), aPQ = smem_u32(sPQ), aSc = smem_u32(sSc), aOnes = smem_u32(sOnes);
+            for (int c = 0; c < nch && ok; ++c) {
+                const int s = c & 1;
+                const uint32_t ph = c & 1;
+                const uint32_t aSt = smem_u32(smem + C::offStage + s * C::kStageBytes);
+                const uint32_t aVt = aSt + 2 * C::kQKBytes;
+                ok = mbar_wait(&bars[kFull0 + s], (c >> 1) & 1, abort_flag);
+                if (!ok) break;
+                TRACE(1, c, 0);
+                tc_fence_after();
+                if (!STATE_ONLY) {
+                    mma_ss(tb + C::colT, smem_desc(dQK, aSt), smem_desc(dQK, aSt + C::kQKBytes), i1, 0);
+                    mma_commit(&bars[kG1]);
+                }
+                ok = mbar_wait(&bars[kPK], ph, abort_flag);
+                // the state group has read (or, before chunk 0, initialised) the state in TMEM
+                if (ok && (!STATE_ONLY || c == 0)) ok = mbar_wait(&bars[kSC], ph, abort_flag);
+                if (!ok) break;
+                TRACE(1, c, 1);
+                tc_fence_after();
+#pragma unroll
+                for (int k = 0; k < kC / 16; ++k) {
+                    const uint64_t bOnes = smem_desc(dOnes, aOnes + (k >> 2) * 2048 + (k & 3) * 32);
+                    mma_ss(tb + C::colZ0, smem_desc(dPhiMN, aPK + k * 1024), bOnes, iZ0, 1);
+                    mma_ss(tb + C::colZ1, smem_desc(dPhiMN, aPK + 4 * C::kPhiBlk + k * 1024), bOnes, iZ1, 1);
+                }
+#pragma unroll
+                for (int k = 0; k < kC / 16; ++k)
+                    mma_ss(tb + C::colS, smem_desc(dV, aVt + k * 2048), smem_desc(dPhiMN, aPK + k * 1024), i5, 1);
+                mma_commit(&bars[kG2]);
+                TRACE(1, c, 2);
+                if (STATE_ONLY) {
+                    mma_commit(&bars[kEmpty0 + s]);
+                    continue;
+                }
+                ok = mbar_wait(&bars[kPQ], ph, abort_flag);
+                if (ok && c > 0) ok = mbar_wait(&bars[kYfree], ph ^ 1, abort_flag);
+                if (!ok) break;
+                TRACE(1, c, 3);
+                tc_fence_after();
+#pragma unroll
+                for (int k = 0; k < kF / 16; ++k)
+                    mma_ss(tb + C::colY, smem_desc(dPhiK, aPQ + (k >> 1) * C::kPhiBlk + (k & 1) * 32),
+                           smem_desc(dPhiK, aSc + (k >> 1) * C::kScBlk + (k & 1) * 32), i4, k > 0);
+                mma_commit(&bars[kG4]);
+                TRACE(1, c, 4);
+                ok = mbar_wait(&bars[kP], ph, abort_flag);
+                if (!ok) break;
+                TRACE(1, c, 5);
+                tc_fence_after();
+#pragma unroll
+                for (int k = 0; k < kC / 16; ++k)
+                    mma_ts(tb + C::colY, tb + C::colT + k * 8, smem_desc(dV, aVt + k * 2048), i3, 1);
+                mma_commit(&bars[kG3]);
+                mma_commit(&bars[kEmpty0 + s]);
+                TRACE(1, c, 6);
+            }
+        }
+    } else if (warp >= 8) {
+        // ===================================================================== state group
+        // One thread per TMEM lane: initial state, per-chunk bf16 copy of the state for
+        // step (4), normalise + store of Y, final state.
+        const int t = tid - 256;
+        // state row (V column) held by this thread's TMEM lane (64-row accumulators use lanes 0-15 of each quarter)
+        const int srow = (DV == 128) ? t : (((t & 31) < 16) ? ((t >> 5) * 16 + (t & 15)) : -1);
+        // feature of the second z tile (64-row MMA: rows 0..31 sit in lanes 0-15 and 32-47)
+        const int z1f = ((t & 31) < 16 && (t >> 5) < 2) ? 128 + (t >> 5) * 16 + (t & 15) : -1;
+        const size_t seg_stride = seg_state_floats(DV);
+        const float* wsh = p.ws + (size_t)head * (p.nseg > 1 ? p.nseg - 1 : 0) * seg_stride;
+
+        // ---- initial state -> TMEM (zeros, the caller's ABI state, and/or earlier segments' partial states)
+        {
+            const float* kvh = p.kv_abi ? p.kv_abi + (size_t)head * kD * DV : nullptr;
+            const bool from_abi = !STATE_ONLY && p.continue_abi;
+            const int nprev = STATE_ONLY ? 0 : seg;
+#pragma unroll 1
+            for (int b = 0; b < kF / 32; ++b) {
+                uint32_t r[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int f = b * 32 + i;
+                    float acc = 0.f;
+                    if (srow >= 0) {
+                        if (from_abi) {
+                            const AbiRows ar = abi_rows(f);
+                            if (ar.a >= 0) {
+                                float v = kvh[(size_t)ar.a * DV + srow];
+                                if (ar.b >= 0) v += kvh[(size_t)ar.b * DV + srow];
+                                acc = v * ar.scale;
+                            }
+                        }
+                        for (int sp = 0; sp < nprev; ++sp) acc += wsh[(size_t)sp * seg_stride + (size_t)f * DV + srow];
+                    }
+                    r[i] = __float_as_uint(acc);
+                }
+                tmem_st32(tmem_addr(tb, lane_base, C::colS + b * 32), r);
+            }
+            // z: feature t of tile 0, feature z1f of tile 1, value in column 0 of each 16-column tile
+            auto z_init = [&](int f) -> float {
+                if (f < 0) return 0.f;
+                float acc = 0.f;
+                if (from_abi) {
+                    const float* zh = p.z_abi + (size_t)head * kD;
+                    const AbiRows ar = abi_rows(f);
+                    if (ar.a >= 0) {
+                        float v = zh[ar.a];
+                        if (ar.b >= 0) v += zh[ar.b];
+                        acc = v * ar.scale;
+                    }
+                }
+                for (int sp = 0; sp < nprev; ++sp) acc += wsh[(size_t)sp * seg_stride + (size_t)kF * DV + f];
+                return acc;
+            };
+            uint32_t r0[16], r1[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) r0[i] = r1[i] = 0u;
+            r0[0] = __float_as_uint(z_init(t));
+            r1[0] = __float_as_uint(z_init(z1f));
+            tmem_st16(tmem_addr(tb, lane_base, C::colZ0), r0);
+            tmem_st16(tmem_addr(tb, lane_base, C::colZ1), r1);
+            tmem_wait_st();
+        }
+        if (STATE_ONLY) {
+            tc_fence_before();
+            mbar_arrive(&bars[kSC]);
+        }
+
+        __nv_bfloat16* outh = p.out + ((size_t)head * p.L + tok_begin) * DV;
+        // normalise + store chunk c (its Y is complete once step (3) of chunk c has finished)
+        auto epilogue = [&](int c) -> bool {
+            if (!mbar_wait(&bars[kG3], c & 1, abort_flag)) return false;
+            if (t == 0) TRACE(4, c, 4);
+            tc_fence_after();
+            uint32_t dcol;
+            tmem_ld1(tmem_addr(tb, lane_base, C::colY + DV), dcol);
+            const bool valid = tok_begin + c * kC + t < tok_end;
+            uint4* dst = reinterpret_cast<uint4*>(outh + ((size_t)c * kC + t) * DV);
+            float inv = 0.f;
+#pragma unroll
+            for (int h = 0; h < DV / 64; ++h) {
+                uint32_t y0[32], y1[32];
+                tmem_ld32(tmem_addr(tb, lane_base, C::colY + h * 64), y0);
+                tmem_ld32(tmem_addr(tb, lane_base, C::colY + h * 64 + 32), y1);
+                tmem_wait_ld();
+                if (h == 0) inv = 1.0f / (s_den[(c & 1) * kC + t] + __uint_as_float(dcol) + kEps);
+                if (h == DV / 64 - 1) {            // everything of Y is in registers: release the accumulator
+                    tc_fence_before();
+                    mbar_arrive(&bars[kYfree]);
+                    if (t == 0) TRACE(4, c, 5);
+                }
+                if (valid) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 v4;
+                        v4.x = pack_bf16(__uint_as_float(y0[8 * j + 0]) * inv, __uint_as_float(y0[8 * j + 1]) * inv);
+                        v4.y = pack_bf16(__uint_as_float(y0[8 * j + 2]) * inv, __uint_as_float(y0[8 * j + 3]) * inv);
+                        v4.z = pack_bf16(__uint_as_float(y0[8 * j + 4]) * inv, __uint_as_float(y0[8 * j + 5]) * inv);
+                        v4.w = pack_bf16(__uint_as_float(y0[8 * j + 6]) * inv, __uint_as_float(y0[8 * j + 7]) * inv);
+                        dst[h * 8 + j] = v4;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 v4;
+                        v4.x = pack_bf16(__uint_as_float(y1[8 * j + 0]) * inv, __uint_as_float(y1[8 * j + 1]) * inv);
+                        v4.y = pack_bf16(__uint_as_float(y1[8 * j + 2]) * inv, __uint_as_float(y1[8 * j + 3]) * inv);
+                        v4.z = pack_bf16(__uint_as_float(y1[8 * j + 4]) * inv, __uint_as_float(y1[8 * j + 5]) * inv);
+                        v4.w = pack_bf16(__uint_as_float(y1[8 * j + 6]) * inv, __uint_as_float(y1[8 * j + 7]) * inv);
+                        dst[h * 8 + 4 + j] = v4;
+                    }
+                }
+            }
+            if (t == 0) TRACE(4, c, 6);
+            return true;
+        };
+
+        if (!STATE_ONLY) {
+            for (int c = 0; c < nch && ok; ++c) {
+                if (c > 0) {
+                    ok = mbar_wait(&bars[kG2], (c - 1) & 1, abort_flag);   // state after chunk c-1 is final
+                    if (!ok) break;
+                }
+                if (t == 0) TRACE(4, c, 0);
+                tc_fence_after();
+                // bf16 copy of this lane's state row, held in registers until the tile is free
+                uint32_t pkd[kF / 2];
+#pragma unroll
+                for (int b = 0; b < kF / 32; ++b) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_addr(tb, lane_base, C::colS + b * 32), r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        pkd[b * 16 + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                }
+                uint32_t z0, z1;
+                tmem_ld1(tmem_addr(tb, lane_base, C::colZ0), z0);
+                tmem_ld1(tmem_addr(tb, lane_base, C::colZ1), z1);
+                tmem_wait_ld();
+                if (t == 0) TRACE(4, c, 1);
+                if (c > 0) {
+                    ok = mbar_wait(&bars[kG4], (c - 1) & 1, abort_flag);   // step (4) of chunk c-1 has read the tile
+                    if (!ok) break;
+                }
+                if (t == 0) TRACE(4, c, 2);
+                if (srow >= 0) {
+                    uint8_t* row = sSc + (srow >> 3) * 512 + (srow & 7) * 64;
+                    const uint32_t sw = (srow >> 1) & 3;
+#pragma unroll
+                    for (int j = 0; j < kF / 8; ++j)
+                        *reinterpret_cast<uint4*>(row + (j >> 2) * C::kScBlk + (((j & 3) ^ sw) << 4)) =
+                            make_uint4(pkd[4 * j], pkd[4 * j + 1], pkd[4 * j + 2], pkd[4 * j + 3]);
+                }
+                // z row (row DV of the tile); DV is a multiple of 64, so its swizzle term is zero
+                uint8_t* zrow = sSc + (DV >> 3) * 512;
+                *reinterpret_cast<__nv_bfloat16*>(zrow + (t >> 5) * C::kScBlk + (t & 31) * 2) =
+                    __float2bfloat16_rn(__uint_as_float(z0));
+                if (z1f >= 0)
+                    *reinterpret_cast<__nv_bfloat16*>(zrow + (z1f >> 5) * C::kScBlk + (z1f & 31) * 2) =
+                        __float2bfloat16_rn(__uint_as_float(z1));
+                fence_proxy_async_smem();
+                tc_fence_before();
+                mbar_arrive(&bars[kSC]);
+                if (t == 0) TRACE(4, c, 3);
+                if (c > 0) {
+                    ok = epilogue(c - 1);
+                    if (!ok) break;
+                }
+            }
+            if (ok && nch > 0) ok = epilogue(nch - 1);
+        }
+
+        // ---- final state: wait for the last update, then write it out.  A parity wait only
+        // tells the current phase from the one before, so a group that has not followed the
+        // barrier chunk by chunk walks through every phase.
+        if (STATE_ONLY) {
+            for (int c = 0; c < nch && ok; ++c) ok = mbar_wait(&bars[kG2], c & 1, abort_flag);
+        } else if (ok && nch > 0) {
+            ok = mbar_wait(&bars[kG2], (nch - 1) & 1, abort_flag);
+        }
+        tc_fence_after();
+        const bool write_ws = STATE_ONLY;
+        const bool write_abi = !STATE_ONLY && p.kv_abi != nullptr && seg == p.nseg - 1;
+        if (ok && (write_ws || write_abi)) {
+            float* wseg = p.ws + ((size_t)head * (p.nseg > 1 ? p.nseg - 1 : 0) + seg) * seg_stride;
+            float* kvh = write_abi ? p.kv_abi + (size_t)head * kD * DV : nullptr;
+#pragma unroll 1
+            for (int b = 0; b < kF / 32; ++b) {
+                uint32_t r[32];
+                tmem_ld32(tmem_addr(tb, lane_base, C::colS + b * 32), r);
+                tmem_wait_ld();
+                if (srow >= 0) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int f = b * 32 + i;
+                        const float v = __uint_as_float(r[i]);
+                        if (write_ws) wseg[(size_t)f * DV + srow] = v;
+                        else {
+                            const AbiRows ar = abi_rows(f);
+                            if (ar.a >= 0) kvh[(size_t)ar.a * DV + srow] = v * ar.scale;
+                            if (ar.b >= 0) kvh[(size_t)ar.b * DV + srow] = v * ar.scale;
+                        }
+                    }
+                }
+            }
+            uint32_t z0, z1;
+            tmem_ld1(tmem_addr(tb, lane_base, C::colZ0), z0);
+            tmem_ld1(tmem_addr(tb, lane_base, C::colZ1), z1);
+            tmem_wait_ld();
+            auto put_z = [&](int f, float v) {
+                if (f < 0) return;
+                if (write_ws) { wseg[(size_t)kF * DV + f] = v; return; }
+                float* zh = p.z_abi + (size_t)head * kD;
+                const AbiRows ar = abi_rows(f);
+                if (ar.a >= 0) zh[ar.a] = v * ar.scale;
+                if (ar.b >= 0) zh[ar.b] = v * ar.scale;
+            };
+            put_z(t, __uint_as_float(z0));
+            put_z(z1f, __uint_as_float(z1));
+        }
+    } else if (warp >= 4) {
+        // ===================================================================== feature group
+        // One thread per token of the chunk: expands its k row (and q row) into feature rows.
+        const int t = tid - 128;
+        for (int c = 0; c < nch && ok; ++c) {
+            const int s = c & 1;
+            const uint8_t* st = smem + C::offStage + s * C::kStageBytes;
+            const bool valid = tok_begin + c * kC + t < tok_end;
+            ok = mbar_wait(&bars[kFull0 + s], (c >> 1) & 1, abort_flag);
+            if (!ok) break;
+            if (t == 0) TRACE(3, c, 0);
+            uint32_t xk[8], xq[8];
+            read_qk_row(st + C::kQKBytes, t, xk);
+            if (!STATE_ONLY) read_qk_row(st, t, xq);
+            if (c > 0) {
+                ok = mbar_wait(&bars[kG2], (c - 1) & 1, abort_flag);   // steps (z), (5) of chunk c-1 have read phi(K)
+                if (!ok) break;
+            }
+            if (t == 0) TRACE(3, c, 1);
+            write_phi_row(xk, sPK, t, valid);
+            fence_proxy_async_smem();
+            mbar_arrive(&bars[kPK]);
+            if (t == 0) TRACE(3, c, 2);
+            if (!STATE_ONLY) {
+                if (c > 0) {
+                    ok = mbar_wait(&bars[kG4], (c - 1) & 1, abort_flag);   // step (4) of chunk c-1 has read phi(Q)
+                    if (!ok) break;
+                }
+                if (t == 0) TRACE(3, c, 3);
+                write_phi_row(xq, sPQ, t, true);
+                fence_proxy_async_smem();
+                mbar_arrive(&bars[kPQ]);
+                if (t == 0) TRACE(3, c, 4);
+            }
+        }
+    } else if (!STATE_ONLY) {
+        // ===================================================================== row group
+        // One thread per query row: polynomial of the scores, causal mask, row sum; the
+        // bf16 weights overwrite the scores in place (columns [0, 64) of the same lanes).
+        const int q4 = warp;                            // lane quarter == 32-row block of the chunk
+        for (int c = 0; c < nch && ok; ++c) {
+            ok = mbar_wait(&bars[kG1], c & 1, abort_flag);
+            if (!ok) break;
+            if (tid == 96) TRACE(2, c, 0);
+            tc_fence_after();
+            float den = 0.f;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int b0 = 2 * half, b1 = b0 + 1;
+                uint32_t sc0[32], sc1[32], pk0[16], pk1[16];
+                if (b0 <= q4) tmem_ld32(tmem_addr(tb, lane_base, C::colT + b0 * 32), sc0);
+                if (b1 <= q4) tmem_ld32(tmem_addr(tb, lane_base, C::colT + b1 * 32), sc1);
+                tmem_wait_ld();
+                if (b0 < q4) poly_batch<false>(sc0, pk0, den, lane);
+                else if (b0 == q4) poly_batch<true>(sc0, pk0, den, lane);
+                else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pk0[i] = 0u;
+                }
+                if (b1 < q4) poly_batch<false>(sc1, pk1, den, lane);
+                else if (b1 == q4) poly_batch<true>(sc1, pk1, den, lane);
+                else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pk1[i] = 0u;
+                }
+                tmem_st16(tmem_addr(tb, lane_base, C::colT + b0 * 16), pk0);
+                tmem_st16(tmem_addr(tb, lane_base, C::colT + b1 * 16), pk1);
+            }
+            s_den[(c & 1) * kC + tid] = den;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&bars[kP]);
+            if (tid == 96) TRACE(2, c, 1);
+        }
+    }
+
+    if (!ok && lane == 0) atomicOr(p.err, 1u);
+    // ---- teardown: everyone meets; after a give-up, loads still in flight get time to land
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int it = 0; it < 200; ++it) __nanosleep(1000);   // ~0.2 ms: far longer than any TMA load in flight
+    }
+    __syncthreads();
+    if (warp == kWarpMma) tmem_dealloc(tb, 512);
+}
+
+// --------------------------------------------------------------------------------- host side
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// [BH][L][width] bf16, box = [1][128][box_w]
+bool make_map(CUtensorMap* m, const void* base, int BH, int L, int width, int box_w, CUtensorMapSwizzle sw) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)width, (cuuint64_t)L, (cuuint64_t)BH};
+    cuuint64_t strides[2] = {(cuuint64_t)width * 2, (cuuint64_t)L * width * 2};
+    cuuint32_t box[3] = {(cuuint32_t)box_w, (cuuint32_t)kC, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+#ifdef BASED_TRACE
+unsigned long long* g_trace = nullptr;
+#endif
+
+template <int DV>
+based_status launch_dv(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH, int L,
+                       int flags, float* ws, int nseg, cudaStream_t stream) {
+    using C = Cfg<DV>;
+    CUtensorMap tq, tk, tv;
+    if (!make_map(&tq, q, BH, L, kDFeat, kDFeat, CU_TENSOR_MAP_SWIZZLE_32B) ||
+        !make_map(&tk, k, BH, L, kDFeat, kDFeat, CU_TENSOR_MAP_SWIZZLE_32B) ||
+        !make_map(&tv, v, BH, L, DV, 64, CU_TENSOR_MAP_SWIZZLE_128B))
+        return BASED_ERR_CUDA;
+    Params p;
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.kv_abi = kv;
+    p.z_abi = z;
+    p.ws = ws;
+    if (error_word_ptr(&p.err) != BASED_OK) return BASED_ERR_CUDA;
+    p.L = L;
+    p.nseg = nseg;
+    const int nch = (L + kC - 1) / kC;
+    p.seg_len = ((nch + nseg - 1) / nseg) * kC;
+    p.continue_abi = (flags & BASED_STATE_CONTINUE) ? 1 : 0;
+#ifdef BASED_TRACE
+    p.trace = g_trace;
+#endif
+    if (cudaFuncSetAttribute(prefill_tc_kernel<DV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)C::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(prefill_tc_kernel<DV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)C::kSmemBytes) != cudaSuccess)
+        return BASED_ERR_CUDA;
+    if (nseg > 1) {
+        prefill_tc_kernel<DV, true><<<dim3(nseg - 1, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, p);
+        note_launch();
+        const based_status st = check_launch("prefill_tc_kernel<state>");
+        if (st != BASED_OK) return st;
+    }
+    prefill_tc_kernel<DV, false><<<dim3(nseg, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, p);
+    note_launch();
+    return check_launch("prefill_tc_kernel");
+}
+
+}  // namespace
+
+// Number of sequence segments a head is split into so that about one CTA per SM is busy.
+int prefill_tc_segments(int BH, int L) {
+    const int nch = (L + kC - 1) / kC;
+    int nseg = 148 / BH;
+    if (nseg < 1) nseg = 1;
+    if (nseg > 8) nseg = 8;
+    if (nseg > nch) nseg = nch;
+    // every segment must own at least one chunk
+    while (nseg > 1 && ((nch + nseg - 1) / nseg) * (nseg - 1) >= nch) --nseg;
+    return nseg;
+}
+
+size_t prefill_tc_workspace_bytes(int BH, int L, int d_v) {
+    const int nseg = prefill_tc_segments(BH, L);
+    return nseg > 1 ? (size_t)BH * (nseg - 1) * seg_state_floats(d_v) * sizeof(float) : 0;
+}
+
+based_status launch_prefill_tc(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH,
+                               int L, int d_v, int flags, void* workspace, cudaStream_t stream) {
+    const int nseg = prefill_tc_segments(BH, L);
+    float* ws = static_cast<float*>(workspace);
+    if (d_v == 64) return launch_dv<64>(q, k, v, out, kv, z, BH, L, flags, ws, nseg, stream);
+    return launch_dv<128>(q, k, v, out, kv, z, BH, L, flags, ws, nseg, stream);
+}
+
+}  // namespace based
+
+#ifdef BASED_TRACE
+extern "C" void based_debug_set_trace(void* ptr) { based::g_trace = static_cast<unsigned long long*>(ptr); }
+#endif

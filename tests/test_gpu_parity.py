@@ -73,6 +73,22 @@ def test_prefill_small_shapes(dtype, d_v, L):
     assert torch.equal(out2, out)
 
 
+@pytest.mark.parametrize("B,H,d_v,L", [(10, 16, 64, 300), (5, 16, 128, 515), (4, 16, 64, 700), (2, 16, 128, 1100),
+                                       (1, 16, 64, 2048), (1, 3, 128, 1000)])
+def test_prefill_bf16_many_chunks(B, H, d_v, L):
+    """Several 128-token chunks per CTA, with and without the sequence split into segments
+    (the split depends on B*H), ragged tails included."""
+    w = wl.Workload("chunks", B, H, L, 16, d_v, "bf16", 0.25)
+    q, k, v = wl.prefill_inputs(w, wl.generator(B * 1000 + L))
+    y_ref, S_ref, z_ref = oracle.linattn_recurrent(_np(q), _np(k), _np(v))
+    kv, z = based.new_state(B, H, d_v)
+    out = based.based_prefill(q.to(DEV), k.to(DEV), v.to(DEV), kv_state=kv, z_state=z)
+    _poll()
+    assert row_err(_np(out), y_ref) <= TOL_BF16
+    assert head_err(_np(kv), S_ref) <= TOL_BF16
+    assert head_err(_np(z), z_ref) <= TOL_BF16
+
+
 @pytest.mark.parametrize("dtype,d_v,L,L1", [("f32", 64, 200, 77), ("bf16", 128, 384, 128), ("bf16", 64, 450, 131)])
 def test_prefill_continue_equals_one_pass(dtype, d_v, L, L1):
     w = wl.Workload("split", 1, 4, L, 16, d_v, dtype, 0.5)
