@@ -139,9 +139,8 @@ def time_region(fn_step, steps: int, warmup: int, torch, dist_on: bool):
         dist.barrier()
     ms = e0.elapsed_time(e1)
     if dist_on:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+        from paper_2402_18668_b200.dist import max_over_ranks
+        ms = max_over_ranks(ms, device="cuda")
     return ms
 
 
