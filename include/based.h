@@ -104,6 +104,33 @@ based_status swa_forward(const void* q, const void* k, const void* v, void* out,
                          int window, float softmax_scale, based_dtype io, void* cuda_stream);
 
 /*
+ * The same computation as based_prefill, for callers that cannot give the library scratch
+ * memory.  (The paper has no counterpart: this is a deployment convenience.)  Some hosts
+ * may not allocate device memory around a call at all - a serving process that has handed
+ * the whole GPU to its own arena and exposes no allocator to plug-ins, a latency-critical
+ * loop in which cudaMalloc's device-wide synchronisation is not acceptable, a sandbox that
+ * forbids the allocation calls.  For them the scratch lives in a fixed array of
+ * BASED_STATIC_SCRATCH_BYTES (8 MiB) of device memory inside the library image; every GPU
+ * that loads the library holds that array until the process exits.  This entry point, and
+ * everything it calls, allocates nothing.
+ *
+ * Arguments, layouts, supported set and results are those of based_prefill without the
+ * workspace pair.  A request whose based_prefill_workspace_bytes exceeds the array returns
+ * BASED_ERR_WORKSPACE (and says so on stderr); use based_prefill with your own buffer then.
+ * The first call on a device looks up the array's device address (one
+ * cudaGetSymbolAddress, no allocation); make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's contents:
+ * nothing in it needs clearing (each call overwrites what it later reads), but two calls
+ * whose kernels can overlap on the GPU - different streams, or different threads - race on
+ * it and must be serialised by the caller.
+ */
+#define BASED_STATIC_SCRATCH_BYTES (8u << 20)
+based_status based_prefill_static_scratch(const void* q, const void* k, const void* v, void* out, float* kv_state,
+                                          float* z_state, int B, int H, int L, int d_feat, int d_v, based_dtype io,
+                                          int flags, void* cuda_stream);
+size_t based_static_scratch_bytes(void);
+
+/*
  * Synchronises the stream and returns the sticky device-side status: BASED_OK, or
  * BASED_ERR_DEVICE_TIMEOUT if a kernel abandoned a bounded wait (its outputs are then
  * undefined), or BASED_ERR_CUDA if the stream reported a CUDA error.  Clears the flag.

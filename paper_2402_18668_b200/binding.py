@@ -23,7 +23,8 @@ D_EXPANDED = 1 + D_FEAT + D_FEAT * D_FEAT
 
 EXPORTS = (
     "based_prefill", "based_prefill_workspace_bytes", "based_decode_step", "swa_forward", "based_poll_error",
-    "based_status_string", "based_version", "based_launch_count",
+    "based_status_string", "based_version", "based_launch_count", "based_prefill_static_scratch",
+    "based_static_scratch_bytes",
 )
 
 _lib = None
@@ -49,6 +50,9 @@ def lib() -> ctypes.CDLL:
         L.based_prefill.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
         L.based_prefill_workspace_bytes.restype = sz
         L.based_prefill_workspace_bytes.argtypes = [i, i, i, i, i, i]
+        L.based_prefill_static_scratch.restype = i
+        L.based_prefill_static_scratch.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
+        L.based_static_scratch_bytes.restype = sz
         L.based_decode_step.restype = i
         L.based_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
         L.swa_forward.restype = i
@@ -129,6 +133,23 @@ def based_prefill(q, k, v, out=None, kv_state=None, z_state=None, flags: int = B
     st = lib().based_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(kv_state), _ptr(z_state), B, H, L, d_feat,
                              d_v, io, flags, _ptr(workspace), ws_bytes, _stream(stream))
     _check(st, "based_prefill")
+    return out
+
+
+def based_static_scratch_bytes() -> int:
+    return int(lib().based_static_scratch_bytes())
+
+
+def based_prefill_static_scratch(q, k, v, out, kv_state=None, z_state=None, flags: int = BASED_STATE_ZERO_INIT,
+                                 stream=None):
+    """based_prefill without a workspace argument: the library's built-in scratch array is
+    used, so the call allocates nothing (the caller passes `out`, too).  Calls that may
+    overlap on the GPU must be serialised by the caller: they share that one array."""
+    _dev(q, k, v, out, kv_state, z_state)
+    B, H, L, d_feat = q.shape
+    st = lib().based_prefill_static_scratch(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(kv_state), _ptr(z_state), B, H,
+                                            L, d_feat, v.shape[-1], _dtype_code(q), flags, _stream(stream))
+    _check(st, "based_prefill_static_scratch")
     return out
 
 
