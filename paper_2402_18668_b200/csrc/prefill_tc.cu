@@ -5,27 +5,28 @@
 // the running KV-state.  Unlike Algorithm 1 the whole expanded state of a head lives in
 // tensor memory as one fp32 accumulator, and the expanded features never leave the SM.
 //
-// Per chunk c of one (b, h) (or of one sequence segment of it) five tensor-core steps:
+// Per chunk c of one (b, h) (or of one sequence segment of it) the tensor-core steps are
 //   (1) scores   T[128,128]  = Q_c K_c^T                        (K = 16)
-//   (z) z       += colsum(phi(K_c))         as  phi(K_c)^T x ones   (M = features, N = 16)
 //   (5) S^T     += V_c^T phi(K_c)           [d_v lanes x 160 feature columns, fp32 in TMEM]
+//   (z) z       += colsum(phi(K_c))         d_v = 64: an extra "ones" column of V, i.e. lane 64
+//                                           of S^T; d_v = 128: phi(K_c)^T x ones (N = 16)
 //   (4) Y        = phi(Q_c) [S_prev | z_prev]   (K = 160; the extra column is the
 //                                                cross-chunk part of the denominator)
 //   (3) Y       += P V_c,  P = (1 + T/4 + T^2/32) masked to j <= i, bf16, read from TMEM
-// and three ALU jobs: the polynomial + mask + row sum on the scores, the expansion of
-// q and k rows into feature rows (shared memory, UMMA operand layout), and a bf16 copy of
-// the fp32 state into shared memory as the B operand of (4).
+// and the ALU jobs: polynomial + mask + row sum on the scores, expansion of q and k rows
+// into feature rows (shared memory, UMMA operand layout), a bf16 copy of the fp32 state
+// as the B operand of (4), and normalise + store through shared memory and TMA.
 //
 // Features are kept in a symmetric basis of 153 (padded to 160) instead of 273: with
 // x' = x/2,  [x' (16) | x'_m x'_(m+o) for o = 0..7 (the o = 0 block scaled by 1/sqrt 2) |
 // x'_m x'_(m+8), m < 8 | 1 | 0 x 7].  Its inner products equal those of the 273-feature
 // map; the state is expanded to / folded from the 273-row ABI layout at the kernel's edges.
 //
-// Warp roles (448 threads): warps 0-3 "row" group (one thread per query row / TMEM lane:
-// polynomial + mask), warps 4-7 "feature" group (one thread per token: phi expansion),
-// warps 8-11 "state" group (one thread per TMEM lane: bf16 state copy, normalise + store,
-// state I/O), warp 12 TMA producer, warp 13 MMA issuer.  All cross-role hand-offs are
-// mbarriers with bounded waits.
+// Warp roles (576 threads): warps 0-3 "row" group (one thread per query row: polynomial),
+// warps 4-7 "feature" group (one thread per token: phi expansion), warps 8-11 "state"
+// group (one thread per TMEM lane: bf16 state copy, state I/O), warps 12-15 "output"
+// group (one thread per output row: normalise, stage, TMA store), warp 16 TMA producer,
+// warp 17 MMA issuer.  All cross-role hand-offs are mbarriers with bounded waits.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -40,9 +41,8 @@ namespace {
 constexpr int kC = 128;            // tokens per chunk
 constexpr int kF = 160;            // internal feature count (153 padded to a multiple of 16)
 constexpr int kFBlk = 5;           // 32-feature SWIZZLE_64B blocks
-constexpr int kStages = 2;
-constexpr int kThreads = 448;
-constexpr int kWarpTma = 12, kWarpMma = 13;
+constexpr int kThreads = 576;
+constexpr int kWarpTma = 16, kWarpMma = 17;
 constexpr float kRsqrt2 = 0.70710678118654752f;
 
 // ---- workspace layout of one (head, segment) partial state: [kF][DV] fp32 then [kF] fp32
@@ -50,36 +50,45 @@ __host__ __device__ constexpr size_t seg_state_floats(int dv) { return (size_t)k
 
 template <int DV>
 struct Cfg {
+    static constexpr int kStages = (DV == 64) ? 3 : 2;
     static constexpr int kNY = DV + 16;                         // Y columns: d_v numerators + denominator block
+    static constexpr int kSLanes = (DV == 64) ? 65 : 128;       // live lanes of S^T (d_v 64: lane 64 carries z)
     static constexpr uint32_t kQKBytes = kC * 32;               // one q or k tile (16 bf16 per token)
     static constexpr uint32_t kVBytes = kC * DV * 2;
     static constexpr uint32_t kStageBytes = 2 * kQKBytes + kVBytes;
-    static constexpr uint32_t kPhiBytes = kFBlk * kC * 64;      // 40 KB
     static constexpr uint32_t kPhiBlk = kC * 64;                // bytes of one 32-feature block
+    static constexpr uint32_t kPhiBytes = kFBlk * kPhiBlk;      // 40 KB
     static constexpr uint32_t kScBlk = kNY * 64;
     static constexpr uint32_t kScBytes = kFBlk * kScBlk;
-    static constexpr uint32_t kOnesBytes = 4096;
+    // d_v 64: a [128 tokens][64] bf16 block whose column 0 is 1.0 (second M-block of V^T);
+    // d_v 128: a block of bf16 ones (B operand of the z step)
+    static constexpr uint32_t kOnesBytes = (DV == 64) ? kC * 128 : 2048;
+    static constexpr uint32_t kOutBytes = kC * 128;             // staging of 64 output columns
     static constexpr uint32_t offStage = 0;
-    static constexpr uint32_t offPK = kStages * kStageBytes;
+    static constexpr uint32_t offOnes = kStages * kStageBytes;  // after the stages: LBO of V^T stays positive
+    static constexpr uint32_t offPK = offOnes + kOnesBytes;
     static constexpr uint32_t offPQ = offPK + kPhiBytes;        // must follow PK (the last z tile over-reads into it)
     static constexpr uint32_t offSc = offPQ + kPhiBytes;
-    static constexpr uint32_t offOnes = offSc + kScBytes;
-    static constexpr uint32_t offBars = offOnes + kOnesBytes;
-    static constexpr uint32_t kSmemBytes = offBars + 256 + 1024 + 1024;   // barriers, row sums, alignment slack
+    static constexpr uint32_t offOut = offSc + kScBytes;
+    static constexpr uint32_t offMisc = offOut + kOutBytes;
+    static constexpr uint32_t kMiscBytes = 2048;                // barriers, row sums, ABI row table
+    static constexpr uint32_t kSmemBytes = offMisc + kMiscBytes + 1024;   // + alignment slack
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
     // TMEM columns
     static constexpr uint32_t colT = 0;                          // scores, overwritten in place by P
     static constexpr uint32_t colY = 128;
     static constexpr uint32_t colS = colY + kNY;
-    static constexpr uint32_t colZ0 = colS + kF;
+    static constexpr uint32_t colZ0 = colS + kF;                 // d_v 128 only
     static constexpr uint32_t colZ1 = colZ0 + 16;
     static_assert(colZ1 + 16 <= 512, "TMEM budget");
-    static_assert(kScBlk % 1024 == 0 && kStageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligned");
+    static_assert(kScBlk % 1024 == 0 && kStageBytes % 1024 == 0 && offPK % 1024 == 0, "tiles stay 1024-byte aligned");
 };
 
-enum Bar { kFull0 = 0, kFull1, kEmpty0, kEmpty1, kG1, kP, kG2, kG4, kG3, kYfree, kPK, kPQ, kSC, kNumBars };
+enum Bar {
+    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kP, kG2, kG4, kG3, kYfree, kPK, kPQ, kSR, kSC, kNumBars
+};
 
 struct Params {
-    __nv_bfloat16* out;
     float* kv_abi;        // [BH, 273, DV] or null
     float* z_abi;         // [BH, 273] or null
     float* ws;            // per (head, segment) partial states, internal layout
@@ -104,20 +113,20 @@ struct Params {
 #endif
 
 // ---- internal feature index -> rows of the 273-row ABI layout -------------------------
-struct AbiRows { int a, b; float scale; };   // b < 0: single row
+struct AbiRows { int a, b; };   // b < 0: single row (scale 1); b >= 0: two rows, scale 1/sqrt 2; a < 0: padding
 __host__ __device__ constexpr AbiRows abi_rows(int i) {
-    if (i < 16) return {1 + i, -1, 1.f};
+    if (i < 16) return {1 + i, -1};
     if (i < 144) {
         const int o = (i - 16) / 16, m = (i - 16) % 16, n = (m + o) % 16;
-        if (o == 0) return {17 + 17 * m, -1, 1.f};
-        return {17 + 16 * m + n, 17 + 16 * n + m, kRsqrt2};
+        if (o == 0) return {17 + 17 * m, -1};
+        return {17 + 16 * m + n, 17 + 16 * n + m};
     }
     if (i < 152) {
         const int m = i - 144, n = m + 8;
-        return {17 + 16 * m + n, 17 + 16 * n + m, kRsqrt2};
+        return {17 + 16 * m + n, 17 + 16 * n + m};
     }
-    if (i == 152) return {0, -1, 1.f};
-    return {-1, -1, 0.f};
+    if (i == 152) return {0, -1};
+    return {-1, -1};
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -131,7 +140,8 @@ __device__ __forceinline__ uint32_t mul2(uint32_t a, uint32_t b) {
 
 // Expand one raw 16-vector (8 packed bf16 pairs) into its 160 internal features and write
 // them as row t of a [128 tokens][160 features] tile made of five SWIZZLE_64B blocks.
-__device__ __forceinline__ void write_phi_row(const uint32_t (&x)[8], uint8_t* tile, int t, bool valid) {
+__device__ __noinline__ void write_phi_row(uint4 xlo, uint4 xhi, uint8_t* tile, int t, bool valid) {
+    const uint32_t x[8] = {xlo.x, xlo.y, xlo.z, xlo.w, xhi.x, xhi.y, xhi.z, xhi.w};
     const uint32_t kHalf = 0x3F003F00u;      // (0.5, 0.5)
     const uint32_t kRs2 = 0x3F353F35u;       // (1/sqrt2, 1/sqrt2) rounded to bf16
     uint32_t E[8], O[8];
@@ -169,46 +179,47 @@ __device__ __forceinline__ void write_phi_row(const uint32_t (&x)[8], uint8_t* t
 }
 
 // Row t of a [128][16] bf16 tile written by TMA with SWIZZLE_32B.
-__device__ __forceinline__ void read_qk_row(const uint8_t* tile, int t, uint32_t (&x)[8]) {
+__device__ __forceinline__ void read_qk_row(const uint8_t* tile, int t, uint4& lo, uint4& hi) {
     const uint8_t* row = tile + (t >> 3) * 256 + (t & 7) * 32;
     const uint32_t sw = ((t >> 2) & 1) << 4;
-    const uint4 lo = *reinterpret_cast<const uint4*>(row + (0 ^ sw));
-    const uint4 hi = *reinterpret_cast<const uint4*>(row + (16 ^ sw));
-    x[0] = lo.x; x[1] = lo.y; x[2] = lo.z; x[3] = lo.w;
-    x[4] = hi.x; x[5] = hi.y; x[6] = hi.z; x[7] = hi.w;
+    lo = *reinterpret_cast<const uint4*>(row + (0 ^ sw));
+    hi = *reinterpret_cast<const uint4*>(row + (16 ^ sw));
+}
+
+__device__ __forceinline__ void group_sync(int id) {        // named barrier of one 128-thread group
+    asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
+}
+// AND of a predicate over one 128-thread group (every thread gets the same answer, so the
+// group leaves its loop together and never strands a member at a named barrier)
+__device__ __forceinline__ bool group_all(int id, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, %2, 128, p;\n\t"
+        "selp.b32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred), "r"(id)
+        : "memory");
+    return r != 0;
 }
 
 }  // namespace
 
-// One 32-column batch of scores -> 16 packed bf16 weight pairs; adds the weights to den.
-// DIAG: the batch straddles the diagonal (key column i of the batch is visible iff i <= lane).
-template <bool DIAG>
-__device__ __forceinline__ void poly_batch(const uint32_t (&sc)[32], uint32_t (&pk)[16], float& den, int lane) {
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        const float s0 = __uint_as_float(sc[2 * i]), s1 = __uint_as_float(sc[2 * i + 1]);
-        float w0 = fmaf(s0, fmaf(s0, 0.03125f, 0.25f), 1.0f);
-        float w1 = fmaf(s1, fmaf(s1, 0.03125f, 0.25f), 1.0f);
-        if (DIAG) {
-            w0 = (2 * i <= lane) ? w0 : 0.f;
-            w1 = (2 * i + 1 <= lane) ? w1 : 0.f;
-        }
-        den += w0 + w1;
-        pk[i] = pack_bf16(w0, w1);
-    }
-}
-
 template <int DV, bool STATE_ONLY>
 __global__ void __launch_bounds__(kThreads, 1)
     prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                      const __grid_constant__ CUtensorMap tm_v, const Params p) {
+                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                      const Params p) {
     using C = Cfg<DV>;
+    constexpr int NS = C::kStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offBars);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offMisc);
     uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + kNumBars);
     volatile uint32_t* abort_flag = tmem_base_s + 1;
-    float* s_den = reinterpret_cast<float*>(tmem_base_s + 2);      // [2][128] row sums of the in-chunk weights
+    float* s_den = reinterpret_cast<float*>(tmem_base_s + 2);          // [2][128] row sums of in-chunk weights
+    short2* s_abi = reinterpret_cast<short2*>(s_den + 2 * kC);         // [160] ABI rows of each internal feature
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int seg = blockIdx.x, head = blockIdx.y;
@@ -220,21 +231,30 @@ __global__ void __launch_bounds__(kThreads, 1)
     uint8_t* sPQ = smem + C::offPQ;
     uint8_t* sSc = smem + C::offSc;
     uint8_t* sOnes = smem + C::offOnes;
+    uint8_t* sOut = smem + C::offOut;
 
     if (tid == 0) {
-        mbar_init(&bars[kFull0], 1); mbar_init(&bars[kFull1], 1);
-        mbar_init(&bars[kEmpty0], 1); mbar_init(&bars[kEmpty1], 1);
+        for (int s = 0; s < NS; ++s) { mbar_init(&bars[kFull0 + s], 1); mbar_init(&bars[kEmpty0 + s], 1); }
         mbar_init(&bars[kG1], 1); mbar_init(&bars[kG2], 1); mbar_init(&bars[kG4], 1); mbar_init(&bars[kG3], 1);
         mbar_init(&bars[kP], 128); mbar_init(&bars[kYfree], 128); mbar_init(&bars[kPK], 128);
-        mbar_init(&bars[kPQ], 128); mbar_init(&bars[kSC], 128);
+        mbar_init(&bars[kPQ], 128); mbar_init(&bars[kSR], 128); mbar_init(&bars[kSC], 128);
         *abort_flag = 0;
         fence_mbar_init();
-        prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
+        prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v); prefetch_tensormap(&tm_o);
     }
     if (warp == kWarpMma) { tmem_alloc(tmem_base_s, 512); tmem_relinquish(); }
-    // ones tile (bf16 1.0) and a zeroed state-copy tile (its rows d_v+1.. stay zero for good)
-    for (uint32_t i = tid * 16; i < C::kOnesBytes; i += kThreads * 16)
-        *reinterpret_cast<uint4*>(sOnes + i) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+    if (tid < kF) { const AbiRows ar = abi_rows(tid); s_abi[tid] = make_short2((short)ar.a, (short)ar.b); }
+    // constant operand tiles and a zeroed state-copy tile (its rows past d_v + 1 stay zero for good)
+    if (DV == 64) {
+        for (uint32_t i = tid * 16; i < C::kOnesBytes; i += kThreads * 16) {
+            const uint32_t t = i >> 7, chunk = (i >> 4) & 7;      // token row, 16-byte chunk within the 128-byte row
+            const uint32_t first = (chunk == (t & 7)) ? 0x00003F80u : 0u;   // element (t, column 0) = 1.0
+            *reinterpret_cast<uint4*>(sOnes + i) = make_uint4(first, 0u, 0u, 0u);
+        }
+    } else {
+        for (uint32_t i = tid * 16; i < C::kOnesBytes; i += kThreads * 16)
+            *reinterpret_cast<uint4*>(sOnes + i) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+    }
     for (uint32_t i = tid * 16; i < C::kScBytes; i += kThreads * 16)
         *reinterpret_cast<uint4*>(sSc + i) = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
@@ -249,8 +269,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         // ===================================================================== TMA producer
         if (lane == 0) {
             for (int c = 0; c < nch && ok; ++c) {
-                const int s = c & 1;
-                ok = mbar_wait(&bars[kEmpty0 + s], ((c >> 1) & 1) ^ 1, abort_flag);
+                const int s = c % NS;
+                ok = mbar_wait(&bars[kEmpty0 + s], ((c / NS) & 1) ^ 1, abort_flag);
                 if (!ok) break;
                 uint8_t* st = smem + C::offStage + s * C::kStageBytes;
                 const int tok0 = tok_begin + c * kC;
@@ -273,38 +293,55 @@ __global__ void __launch_bounds__(kThreads, 1)
             constexpr uint32_t i1 = make_idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t iZ0 = make_idesc_bf16(128, 16, 1, 0);
             constexpr uint32_t iZ1 = make_idesc_bf16(64, 16, 1, 0);
-            constexpr uint32_t i5 = make_idesc_bf16(DV, kF, 1, 1);
+            constexpr uint32_t i5 = make_idesc_bf16(128, kF, 1, 1);
             constexpr uint32_t i4 = make_idesc_bf16(128, C::kNY, 0, 0);
             constexpr uint32_t i3 = make_idesc_bf16(128, DV, 0, 1);
-            const uint32_t aPK = smem_u32(sPK), aPQ = smem_u32(sPQ), aSc = smem_u32(sSc), aOnes = smem_u32(sOnes);
+            const uint32_t aOnes = smem_u32(sOnes);
+            // low descriptor words: constant part + (start address >> 4)
+            const uint32_t lQK = desc_lo(dQK), lV = desc_lo(dV);
+            const uint32_t lPK = desc_lo(dPhiMN) + (smem_u32(sPK) >> 4), lPQ = desc_lo(dPhiK) + (smem_u32(sPQ) >> 4);
+            const uint32_t lSc = desc_lo(dPhiK) + (smem_u32(sSc) >> 4), lOnes = desc_lo(dOnes) + (aOnes >> 4);
             for (int c = 0; c < nch && ok; ++c) {
-                const int s = c & 1;
+                const int s = c % NS;
                 const uint32_t ph = c & 1;
                 const uint32_t aSt = smem_u32(smem + C::offStage + s * C::kStageBytes);
                 const uint32_t aVt = aSt + 2 * C::kQKBytes;
-                ok = mbar_wait(&bars[kFull0 + s], (c >> 1) & 1, abort_flag);
+                ok = mbar_wait(&bars[kFull0 + s], (c / NS) & 1, abort_flag);
                 if (!ok) break;
                 TRACE(1, c, 0);
                 tc_fence_after();
                 if (!STATE_ONLY) {
-                    mma_ss(tb + C::colT, smem_desc(dQK, aSt), smem_desc(dQK, aSt + C::kQKBytes), i1, 0);
+                    mma_ss_lh<false>(tb + C::colT, lQK + (aSt >> 4), desc_hi(dQK), lQK + ((aSt + C::kQKBytes) >> 4),
+                                     desc_hi(dQK), i1);
                     mma_commit(&bars[kG1]);
                 }
                 ok = mbar_wait(&bars[kPK], ph, abort_flag);
                 // the state group has read (or, before chunk 0, initialised) the state in TMEM
-                if (ok && (!STATE_ONLY || c == 0)) ok = mbar_wait(&bars[kSC], ph, abort_flag);
+                if (ok && (!STATE_ONLY || c == 0)) ok = mbar_wait(&bars[kSR], ph, abort_flag);
                 if (!ok) break;
                 TRACE(1, c, 1);
                 tc_fence_after();
+                if (DV == 64) {
+                    // V^T as a 128-row A operand: rows 0..63 from the V tile, rows 64..127 from the ones
+                    // block (row 64 = ones over the tokens), so lane 64 of S^T accumulates z
+                    const uint64_t dV1 = make_smem_desc_base(aOnes - aVt, 1024, kSwizzle128B);
+                    const uint32_t a_lo = desc_lo(dV1) + (aVt >> 4), a_hi = desc_hi(dV1);
 #pragma unroll
-                for (int k = 0; k < kC / 16; ++k) {
-                    const uint64_t bOnes = smem_desc(dOnes, aOnes + (k >> 2) * 2048 + (k & 3) * 32);
-                    mma_ss(tb + C::colZ0, smem_desc(dPhiMN, aPK + k * 1024), bOnes, iZ0, 1);
-                    mma_ss(tb + C::colZ1, smem_desc(dPhiMN, aPK + 4 * C::kPhiBlk + k * 1024), bOnes, iZ1, 1);
+                    for (int k = 0; k < kC / 16; ++k)
+                        mma_ss_lh<true>(tb + C::colS, a_lo + k * (2048 >> 4), a_hi, lPK + k * (1024 >> 4),
+                                        desc_hi(dPhiMN), i5);
+                } else {
+                    const uint32_t a_lo = lV + (aVt >> 4);
+#pragma unroll
+                    for (int k = 0; k < kC / 16; ++k) {
+                        mma_ss_lh<true>(tb + C::colS, a_lo + k * (2048 >> 4), desc_hi(dV), lPK + k * (1024 >> 4),
+                                        desc_hi(dPhiMN), i5);
+                        mma_ss_lh<true>(tb + C::colZ0, lPK + k * (1024 >> 4), desc_hi(dPhiMN), lOnes + (k & 1) * 2,
+                                        desc_hi(dOnes), iZ0);
+                        mma_ss_lh<true>(tb + C::colZ1, lPK + ((4 * C::kPhiBlk + k * 1024) >> 4), desc_hi(dPhiMN),
+                                        lOnes + (k & 1) * 2, desc_hi(dOnes), iZ1);
+                    }
                 }
-#pragma unroll
-                for (int k = 0; k < kC / 16; ++k)
-                    mma_ss(tb + C::colS, smem_desc(dV, aVt + k * 2048), smem_desc(dPhiMN, aPK + k * 1024), i5, 1);
                 mma_commit(&bars[kG2]);
                 TRACE(1, c, 2);
                 if (STATE_ONLY) {
@@ -312,121 +349,66 @@ __global__ void __launch_bounds__(kThreads, 1)
                     continue;
                 }
                 ok = mbar_wait(&bars[kPQ], ph, abort_flag);
+                if (ok) ok = mbar_wait(&bars[kSC], ph, abort_flag);
                 if (ok && c > 0) ok = mbar_wait(&bars[kYfree], ph ^ 1, abort_flag);
                 if (!ok) break;
                 TRACE(1, c, 3);
                 tc_fence_after();
 #pragma unroll
-                for (int k = 0; k < kF / 16; ++k)
-                    mma_ss(tb + C::colY, smem_desc(dPhiK, aPQ + (k >> 1) * C::kPhiBlk + (k & 1) * 32),
-                           smem_desc(dPhiK, aSc + (k >> 1) * C::kScBlk + (k & 1) * 32), i4, k > 0);
+                for (int k = 0; k < kF / 16; ++k) {
+                    const uint32_t off = ((k >> 1) * C::kPhiBlk + (k & 1) * 32) >> 4;
+                    const uint32_t offb = ((k >> 1) * C::kScBlk + (k & 1) * 32) >> 4;
+                    if (k == 0) mma_ss_lh<false>(tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
+                    else mma_ss_lh<true>(tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
+                }
                 mma_commit(&bars[kG4]);
                 TRACE(1, c, 4);
                 ok = mbar_wait(&bars[kP], ph, abort_flag);
                 if (!ok) break;
                 TRACE(1, c, 5);
                 tc_fence_after();
+                {
+                    const uint32_t b_lo = lV + (aVt >> 4);
 #pragma unroll
-                for (int k = 0; k < kC / 16; ++k)
-                    mma_ts(tb + C::colY, tb + C::colT + k * 8, smem_desc(dV, aVt + k * 2048), i3, 1);
+                    for (int k = 0; k < kC / 16; ++k)
+                        mma_ts_lh<true>(tb + C::colY, tb + C::colT + k * 8, b_lo + k * (2048 >> 4), desc_hi(dV), i3);
+                }
                 mma_commit(&bars[kG3]);
                 mma_commit(&bars[kEmpty0 + s]);
                 TRACE(1, c, 6);
             }
         }
-    } else if (warp >= 8) {
-        // ===================================================================== state group
-        // One thread per TMEM lane: initial state, per-chunk bf16 copy of the state for
-        // step (4), normalise + store of Y, final state.
-        const int t = tid - 256;
-        // state row (V column) held by this thread's TMEM lane (64-row accumulators use lanes 0-15 of each quarter)
-        const int srow = (DV == 128) ? t : (((t & 31) < 16) ? ((t >> 5) * 16 + (t & 15)) : -1);
-        // feature of the second z tile (64-row MMA: rows 0..31 sit in lanes 0-15 and 32-47)
-        const int z1f = ((t & 31) < 16 && (t >> 5) < 2) ? 128 + (t >> 5) * 16 + (t & 15) : -1;
-        const size_t seg_stride = seg_state_floats(DV);
-        const float* wsh = p.ws + (size_t)head * (p.nseg > 1 ? p.nseg - 1 : 0) * seg_stride;
-
-        // ---- initial state -> TMEM (zeros, the caller's ABI state, and/or earlier segments' partial states)
-        {
-            const float* kvh = p.kv_abi ? p.kv_abi + (size_t)head * kD * DV : nullptr;
-            const bool from_abi = !STATE_ONLY && p.continue_abi;
-            const int nprev = STATE_ONLY ? 0 : seg;
-#pragma unroll 1
-            for (int b = 0; b < kF / 32; ++b) {
-                uint32_t r[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int f = b * 32 + i;
-                    float acc = 0.f;
-                    if (srow >= 0) {
-                        if (from_abi) {
-                            const AbiRows ar = abi_rows(f);
-                            if (ar.a >= 0) {
-                                float v = kvh[(size_t)ar.a * DV + srow];
-                                if (ar.b >= 0) v += kvh[(size_t)ar.b * DV + srow];
-                                acc = v * ar.scale;
-                            }
-                        }
-                        for (int sp = 0; sp < nprev; ++sp) acc += wsh[(size_t)sp * seg_stride + (size_t)f * DV + srow];
-                    }
-                    r[i] = __float_as_uint(acc);
-                }
-                tmem_st32(tmem_addr(tb, lane_base, C::colS + b * 32), r);
-            }
-            // z: feature t of tile 0, feature z1f of tile 1, value in column 0 of each 16-column tile
-            auto z_init = [&](int f) -> float {
-                if (f < 0) return 0.f;
-                float acc = 0.f;
-                if (from_abi) {
-                    const float* zh = p.z_abi + (size_t)head * kD;
-                    const AbiRows ar = abi_rows(f);
-                    if (ar.a >= 0) {
-                        float v = zh[ar.a];
-                        if (ar.b >= 0) v += zh[ar.b];
-                        acc = v * ar.scale;
-                    }
-                }
-                for (int sp = 0; sp < nprev; ++sp) acc += wsh[(size_t)sp * seg_stride + (size_t)kF * DV + f];
-                return acc;
-            };
-            uint32_t r0[16], r1[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) r0[i] = r1[i] = 0u;
-            r0[0] = __float_as_uint(z_init(t));
-            r1[0] = __float_as_uint(z_init(z1f));
-            tmem_st16(tmem_addr(tb, lane_base, C::colZ0), r0);
-            tmem_st16(tmem_addr(tb, lane_base, C::colZ1), r1);
-            tmem_wait_st();
-        }
-        if (STATE_ONLY) {
-            tc_fence_before();
-            mbar_arrive(&bars[kSC]);
-        }
-
-        __nv_bfloat16* outh = p.out + ((size_t)head * p.L + tok_begin) * DV;
-        // normalise + store chunk c (its Y is complete once step (3) of chunk c has finished)
-        auto epilogue = [&](int c) -> bool {
-            if (!mbar_wait(&bars[kG3], c & 1, abort_flag)) return false;
-            if (t == 0) TRACE(4, c, 4);
-            tc_fence_after();
-            uint32_t dcol;
-            tmem_ld1(tmem_addr(tb, lane_base, C::colY + DV), dcol);
-            const bool valid = tok_begin + c * kC + t < tok_end;
-            uint4* dst = reinterpret_cast<uint4*>(outh + ((size_t)c * kC + t) * DV);
-            float inv = 0.f;
-#pragma unroll
-            for (int h = 0; h < DV / 64; ++h) {
-                uint32_t y0[32], y1[32];
-                tmem_ld32(tmem_addr(tb, lane_base, C::colY + h * 64), y0);
-                tmem_ld32(tmem_addr(tb, lane_base, C::colY + h * 64 + 32), y1);
+    } else if (warp >= 12) {
+        // ===================================================================== output group
+        // One thread per output row: Y / (row sum + cross-chunk denominator + eps) -> bf16 ->
+        // swizzled staging tile of 64 columns -> TMA store.
+        if (!STATE_ONLY) {
+            const int t = tid - 384;
+            uint8_t* orow = sOut + (t >> 3) * 1024 + (t & 7) * 128;
+            const uint32_t sw = t & 7;
+            for (int c = 0; c < nch && ok; ++c) {
+                ok = group_all(1, mbar_wait(&bars[kG3], c & 1, abort_flag));
+                if (!ok) break;
+                if (t == 0) TRACE(5, c, 0);
+                tc_fence_after();
+                uint32_t dcol;
+                tmem_ld1(tmem_addr(tb, lane_base, C::colY + DV), dcol);
                 tmem_wait_ld();
-                if (h == 0) inv = 1.0f / (s_den[(c & 1) * kC + t] + __uint_as_float(dcol) + kEps);
-                if (h == DV / 64 - 1) {            // everything of Y is in registers: release the accumulator
-                    tc_fence_before();
-                    mbar_arrive(&bars[kYfree]);
-                    if (t == 0) TRACE(4, c, 5);
-                }
-                if (valid) {
+                const float inv = 1.0f / (s_den[(c & 1) * kC + t] + __uint_as_float(dcol) + kEps);
+#pragma unroll 1
+                for (int h = 0; h < DV / 64; ++h) {
+                    uint32_t y0[32], y1[32];
+                    tmem_ld32(tmem_addr(tb, lane_base, C::colY + h * 64), y0);
+                    tmem_ld32(tmem_addr(tb, lane_base, C::colY + h * 64 + 32), y1);
+                    tmem_wait_ld();
+                    if (h == DV / 64 - 1) {            // all of Y is in registers: release the accumulator
+                        tc_fence_before();
+                        mbar_arrive(&bars[kYfree]);
+                        if (t == 0) TRACE(5, c, 1);
+                    }
+                    // the staging tile is free once the previous TMA store has read it
+                    if (t == 0) tma_store_wait_read<0>();
+                    group_sync(1);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         uint4 v4;
@@ -434,7 +416,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                         v4.y = pack_bf16(__uint_as_float(y0[8 * j + 2]) * inv, __uint_as_float(y0[8 * j + 3]) * inv);
                         v4.z = pack_bf16(__uint_as_float(y0[8 * j + 4]) * inv, __uint_as_float(y0[8 * j + 5]) * inv);
                         v4.w = pack_bf16(__uint_as_float(y0[8 * j + 6]) * inv, __uint_as_float(y0[8 * j + 7]) * inv);
-                        dst[h * 8 + j] = v4;
+                        *reinterpret_cast<uint4*>(orow + ((j ^ sw) << 4)) = v4;
                     }
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -443,15 +425,101 @@ __global__ void __launch_bounds__(kThreads, 1)
                         v4.y = pack_bf16(__uint_as_float(y1[8 * j + 2]) * inv, __uint_as_float(y1[8 * j + 3]) * inv);
                         v4.z = pack_bf16(__uint_as_float(y1[8 * j + 4]) * inv, __uint_as_float(y1[8 * j + 5]) * inv);
                         v4.w = pack_bf16(__uint_as_float(y1[8 * j + 6]) * inv, __uint_as_float(y1[8 * j + 7]) * inv);
-                        dst[h * 8 + 4 + j] = v4;
+                        *reinterpret_cast<uint4*>(orow + (((4 + j) ^ sw) << 4)) = v4;
+                    }
+                    fence_proxy_async_smem();
+                    group_sync(1);
+                    if (t == 0) {
+                        // rows past the end of the sequence are clipped by the tensor map
+                        tma_store_3d(&tm_o, sOut, h * 64, tok_begin + c * kC, head);
+                        tma_store_commit();
                     }
                 }
+                if (t == 0) TRACE(5, c, 2);
             }
-            if (t == 0) TRACE(4, c, 6);
-            return true;
-        };
+            if (t == 0) tma_store_wait<0>();
+        }
+    } else if (warp >= 8) {
+        // ===================================================================== state group
+        // One thread per TMEM lane of the state accumulator: initial state, per-chunk bf16
+        // copy of the state for step (4), final state.
+        const int t = tid - 256;
+        // what this thread's lane of S^T holds: V column srow, or (d_v 64) the K-state at lane 64
+        const int srow = (t < C::kSLanes) ? t : -1;
+        const bool is_z = (DV == 64) && t == 64;
+        // d_v 128: K-state features held in the two z tiles (64-row MMA: rows 0..31 in lanes 0-15, 32-47)
+        const int z1f = (DV == 128 && (t & 31) < 16 && (t >> 5) < 2) ? 128 + (t >> 5) * 16 + (t & 15) : -1;
+        const size_t seg_stride = seg_state_floats(DV);
+        const float* wsh = p.ws + (size_t)head * (p.nseg > 1 ? p.nseg - 1 : 0) * seg_stride;
+        const float* kvh = p.kv_abi ? p.kv_abi + (size_t)head * kD * DV : nullptr;
+        const float* zh = p.z_abi ? p.z_abi + (size_t)head * kD : nullptr;
+        const bool from_abi = !STATE_ONLY && p.continue_abi;
+        const int nprev = STATE_ONLY ? 0 : seg;
 
-        if (!STATE_ONLY) {
+        // Initial value of this lane's row: the caller's ABI state (folded into the internal
+        // basis) plus the partial states of the earlier segments.  Loads are issued 16 at a
+        // time before they are consumed, so their latencies overlap.
+#pragma unroll 1
+        for (int b = 0; b < kF / 16; ++b) {
+            float acc[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+            if (srow >= 0) {
+                if (from_abi) {
+                    float va[16], vb[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const short2 ar = s_abi[b * 16 + i];
+                        va[i] = (ar.x >= 0) ? (is_z ? zh[ar.x] : kvh[(size_t)ar.x * DV + srow]) : 0.f;
+                        vb[i] = (ar.y >= 0) ? (is_z ? zh[ar.y] : kvh[(size_t)ar.y * DV + srow]) : 0.f;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) acc[i] = (s_abi[b * 16 + i].y >= 0) ? (va[i] + vb[i]) * kRsqrt2 : va[i];
+                }
+                for (int sp = 0; sp < nprev; ++sp) {
+                    const float* src = wsh + (size_t)sp * seg_stride + (is_z ? (size_t)kF * DV + b * 16
+                                                                             : (size_t)(b * 16) * DV + srow);
+                    float tmp[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) tmp[i] = is_z ? src[i] : src[(size_t)i * DV];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) acc[i] += tmp[i];
+                }
+            }
+            uint32_t r[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(acc[i]);
+            tmem_st16(tmem_addr(tb, lane_base, C::colS + b * 16), r);
+        }
+        // d_v 128: K-state of feature t (tile 0) and feature z1f (tile 1), column 0 of each tile
+        auto z_init = [&](int f) -> float {
+            if (f < 0) return 0.f;
+            float acc = 0.f;
+            if (from_abi) {
+                const short2 ar = s_abi[f];
+                if (ar.x >= 0) acc = (ar.y >= 0) ? (zh[ar.x] + zh[ar.y]) * kRsqrt2 : zh[ar.x];
+            }
+            for (int sp = 0; sp < nprev; ++sp) acc += wsh[(size_t)sp * seg_stride + (size_t)kF * DV + f];
+            return acc;
+        };
+        if (DV == 128) {
+            uint32_t r0[16], r1[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) r0[i] = r1[i] = 0u;
+            r0[0] = __float_as_uint(z_init(t));
+            r1[0] = __float_as_uint(z_init(z1f));
+            tmem_st16(tmem_addr(tb, lane_base, C::colZ0), r0);
+            tmem_st16(tmem_addr(tb, lane_base, C::colZ1), r1);
+        }
+        tmem_wait_st();
+
+        if (STATE_ONLY) {
+            tc_fence_before();
+            mbar_arrive(&bars[kSR]);
+            // a parity wait only tells the current phase from the one before, so follow the
+            // state-update barrier chunk by chunk
+            for (int c = 0; c < nch && ok; ++c) ok = mbar_wait(&bars[kG2], c & 1, abort_flag);
+        } else {
             for (int c = 0; c < nch && ok; ++c) {
                 if (c > 0) {
                     ok = mbar_wait(&bars[kG2], (c - 1) & 1, abort_flag);   // state after chunk c-1 is final
@@ -462,18 +530,22 @@ __global__ void __launch_bounds__(kThreads, 1)
                 // bf16 copy of this lane's state row, held in registers until the tile is free
                 uint32_t pkd[kF / 2];
 #pragma unroll
-                for (int b = 0; b < kF / 32; ++b) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem_addr(tb, lane_base, C::colS + b * 32), r);
+                for (int b = 0; b < kF / 16; ++b) {
+                    uint32_t r[16];
+                    tmem_ld16(tmem_addr(tb, lane_base, C::colS + b * 16), r);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        pkd[b * 16 + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                    for (int i = 0; i < 8; ++i)
+                        pkd[b * 8 + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
                 }
-                uint32_t z0, z1;
-                tmem_ld1(tmem_addr(tb, lane_base, C::colZ0), z0);
-                tmem_ld1(tmem_addr(tb, lane_base, C::colZ1), z1);
-                tmem_wait_ld();
+                uint32_t z0 = 0, z1 = 0;
+                if (DV == 128) {
+                    tmem_ld1(tmem_addr(tb, lane_base, C::colZ0), z0);
+                    tmem_ld1(tmem_addr(tb, lane_base, C::colZ1), z1);
+                    tmem_wait_ld();
+                }
+                tc_fence_before();
+                mbar_arrive(&bars[kSR]);                                   // step (5) of chunk c may overwrite the state
                 if (t == 0) TRACE(4, c, 1);
                 if (c > 0) {
                     ok = mbar_wait(&bars[kG4], (c - 1) & 1, abort_flag);   // step (4) of chunk c-1 has read the tile
@@ -488,93 +560,81 @@ __global__ void __launch_bounds__(kThreads, 1)
                         *reinterpret_cast<uint4*>(row + (j >> 2) * C::kScBlk + (((j & 3) ^ sw) << 4)) =
                             make_uint4(pkd[4 * j], pkd[4 * j + 1], pkd[4 * j + 2], pkd[4 * j + 3]);
                 }
-                // z row (row DV of the tile); DV is a multiple of 64, so its swizzle term is zero
-                uint8_t* zrow = sSc + (DV >> 3) * 512;
-                *reinterpret_cast<__nv_bfloat16*>(zrow + (t >> 5) * C::kScBlk + (t & 31) * 2) =
-                    __float2bfloat16_rn(__uint_as_float(z0));
-                if (z1f >= 0)
-                    *reinterpret_cast<__nv_bfloat16*>(zrow + (z1f >> 5) * C::kScBlk + (z1f & 31) * 2) =
-                        __float2bfloat16_rn(__uint_as_float(z1));
+                if (DV == 128) {
+                    // z row (row 128 of the tile: its swizzle term is zero)
+                    uint8_t* zrow = sSc + (DV >> 3) * 512;
+                    *reinterpret_cast<__nv_bfloat16*>(zrow + (t >> 5) * C::kScBlk + (t & 31) * 2) =
+                        __float2bfloat16_rn(__uint_as_float(z0));
+                    if (z1f >= 0)
+                        *reinterpret_cast<__nv_bfloat16*>(zrow + (uint32_t)(z1f >> 5) * C::kScBlk + (uint32_t)(z1f & 31) * 2) =
+                            __float2bfloat16_rn(__uint_as_float(z1));
+                }
                 fence_proxy_async_smem();
-                tc_fence_before();
                 mbar_arrive(&bars[kSC]);
                 if (t == 0) TRACE(4, c, 3);
-                if (c > 0) {
-                    ok = epilogue(c - 1);
-                    if (!ok) break;
-                }
             }
-            if (ok && nch > 0) ok = epilogue(nch - 1);
+            if (ok && nch > 0) ok = mbar_wait(&bars[kG2], (nch - 1) & 1, abort_flag);
         }
 
-        // ---- final state: wait for the last update, then write it out.  A parity wait only
-        // tells the current phase from the one before, so a group that has not followed the
-        // barrier chunk by chunk walks through every phase.
-        if (STATE_ONLY) {
-            for (int c = 0; c < nch && ok; ++c) ok = mbar_wait(&bars[kG2], c & 1, abort_flag);
-        } else if (ok && nch > 0) {
-            ok = mbar_wait(&bars[kG2], (nch - 1) & 1, abort_flag);
-        }
+        // ---- final state
         tc_fence_after();
         const bool write_ws = STATE_ONLY;
         const bool write_abi = !STATE_ONLY && p.kv_abi != nullptr && seg == p.nseg - 1;
         if (ok && (write_ws || write_abi)) {
             float* wseg = p.ws + ((size_t)head * (p.nseg > 1 ? p.nseg - 1 : 0) + seg) * seg_stride;
-            float* kvh = write_abi ? p.kv_abi + (size_t)head * kD * DV : nullptr;
+            float* kvo = write_abi ? p.kv_abi + (size_t)head * kD * DV : nullptr;
+            float* zo = write_abi ? p.z_abi + (size_t)head * kD : nullptr;
+            auto put = [&](int f, float v, bool zrow, int col) {
+                if (write_ws) {
+                    if (zrow) wseg[(size_t)kF * DV + f] = v;
+                    else wseg[(size_t)f * DV + col] = v;
+                    return;
+                }
+                const short2 ar = s_abi[f];
+                if (ar.x < 0) return;
+                if (ar.y >= 0) v *= kRsqrt2;
+                if (zrow) { zo[ar.x] = v; if (ar.y >= 0) zo[ar.y] = v; }
+                else { kvo[(size_t)ar.x * DV + col] = v; if (ar.y >= 0) kvo[(size_t)ar.y * DV + col] = v; }
+            };
 #pragma unroll 1
-            for (int b = 0; b < kF / 32; ++b) {
-                uint32_t r[32];
-                tmem_ld32(tmem_addr(tb, lane_base, C::colS + b * 32), r);
+            for (int b = 0; b < kF / 16; ++b) {
+                uint32_t r[16];
+                tmem_ld16(tmem_addr(tb, lane_base, C::colS + b * 16), r);
                 tmem_wait_ld();
                 if (srow >= 0) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int f = b * 32 + i;
-                        const float v = __uint_as_float(r[i]);
-                        if (write_ws) wseg[(size_t)f * DV + srow] = v;
-                        else {
-                            const AbiRows ar = abi_rows(f);
-                            if (ar.a >= 0) kvh[(size_t)ar.a * DV + srow] = v * ar.scale;
-                            if (ar.b >= 0) kvh[(size_t)ar.b * DV + srow] = v * ar.scale;
-                        }
-                    }
+                    for (int i = 0; i < 16; ++i) put(b * 16 + i, __uint_as_float(r[i]), is_z, srow);
                 }
             }
-            uint32_t z0, z1;
-            tmem_ld1(tmem_addr(tb, lane_base, C::colZ0), z0);
-            tmem_ld1(tmem_addr(tb, lane_base, C::colZ1), z1);
-            tmem_wait_ld();
-            auto put_z = [&](int f, float v) {
-                if (f < 0) return;
-                if (write_ws) { wseg[(size_t)kF * DV + f] = v; return; }
-                float* zh = p.z_abi + (size_t)head * kD;
-                const AbiRows ar = abi_rows(f);
-                if (ar.a >= 0) zh[ar.a] = v * ar.scale;
-                if (ar.b >= 0) zh[ar.b] = v * ar.scale;
-            };
-            put_z(t, __uint_as_float(z0));
-            put_z(z1f, __uint_as_float(z1));
+            if (DV == 128) {
+                uint32_t z0, z1;
+                tmem_ld1(tmem_addr(tb, lane_base, C::colZ0), z0);
+                tmem_ld1(tmem_addr(tb, lane_base, C::colZ1), z1);
+                tmem_wait_ld();
+                put(t, __uint_as_float(z0), true, 0);
+                if (z1f >= 0) put(z1f, __uint_as_float(z1), true, 0);
+            }
         }
     } else if (warp >= 4) {
         // ===================================================================== feature group
         // One thread per token of the chunk: expands its k row (and q row) into feature rows.
         const int t = tid - 128;
         for (int c = 0; c < nch && ok; ++c) {
-            const int s = c & 1;
+            const int s = c % NS;
             const uint8_t* st = smem + C::offStage + s * C::kStageBytes;
             const bool valid = tok_begin + c * kC + t < tok_end;
-            ok = mbar_wait(&bars[kFull0 + s], (c >> 1) & 1, abort_flag);
+            ok = mbar_wait(&bars[kFull0 + s], (c / NS) & 1, abort_flag);
             if (!ok) break;
             if (t == 0) TRACE(3, c, 0);
-            uint32_t xk[8], xq[8];
-            read_qk_row(st + C::kQKBytes, t, xk);
-            if (!STATE_ONLY) read_qk_row(st, t, xq);
+            uint4 klo, khi, qlo = make_uint4(0u, 0u, 0u, 0u), qhi = qlo;
+            read_qk_row(st + C::kQKBytes, t, klo, khi);
+            if (!STATE_ONLY) read_qk_row(st, t, qlo, qhi);
             if (c > 0) {
-                ok = mbar_wait(&bars[kG2], (c - 1) & 1, abort_flag);   // steps (z), (5) of chunk c-1 have read phi(K)
+                ok = mbar_wait(&bars[kG2], (c - 1) & 1, abort_flag);   // step (5) of chunk c-1 has read phi(K)
                 if (!ok) break;
             }
             if (t == 0) TRACE(3, c, 1);
-            write_phi_row(xk, sPK, t, valid);
+            write_phi_row(klo, khi, sPK, t, valid);
             fence_proxy_async_smem();
             mbar_arrive(&bars[kPK]);
             if (t == 0) TRACE(3, c, 2);
@@ -584,7 +644,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     if (!ok) break;
                 }
                 if (t == 0) TRACE(3, c, 3);
-                write_phi_row(xq, sPQ, t, true);
+                write_phi_row(qlo, qhi, sPQ, t, true);
                 fence_proxy_async_smem();
                 mbar_arrive(&bars[kPQ]);
                 if (t == 0) TRACE(3, c, 4);
@@ -601,27 +661,29 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (tid == 96) TRACE(2, c, 0);
             tc_fence_after();
             float den = 0.f;
+#pragma unroll 1
+            for (int b = 0; b < 4; ++b) {
+                uint32_t pk[16];
+                if (b <= q4) {                           // some row of this warp sees these key columns
+                    uint32_t sc[32];
+                    tmem_ld32(tmem_addr(tb, lane_base, C::colT + b * 32), sc);
+                    tmem_wait_ld();
+                    const int limit = (b < q4) ? 64 : lane;      // last visible column of the batch for this row
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const int b0 = 2 * half, b1 = b0 + 1;
-                uint32_t sc0[32], sc1[32], pk0[16], pk1[16];
-                if (b0 <= q4) tmem_ld32(tmem_addr(tb, lane_base, C::colT + b0 * 32), sc0);
-                if (b1 <= q4) tmem_ld32(tmem_addr(tb, lane_base, C::colT + b1 * 32), sc1);
-                tmem_wait_ld();
-                if (b0 < q4) poly_batch<false>(sc0, pk0, den, lane);
-                else if (b0 == q4) poly_batch<true>(sc0, pk0, den, lane);
-                else {
+                    for (int i = 0; i < 16; ++i) {
+                        const float s0 = __uint_as_float(sc[2 * i]), s1 = __uint_as_float(sc[2 * i + 1]);
+                        float w0 = fmaf(s0, fmaf(s0, 0.03125f, 0.25f), 1.0f);
+                        float w1 = fmaf(s1, fmaf(s1, 0.03125f, 0.25f), 1.0f);
+                        w0 = (2 * i <= limit) ? w0 : 0.f;
+                        w1 = (2 * i + 1 <= limit) ? w1 : 0.f;
+                        den += w0 + w1;
+                        pk[i] = pack_bf16(w0, w1);
+                    }
+                } else {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) pk0[i] = 0u;
+                    for (int i = 0; i < 16; ++i) pk[i] = 0u;
                 }
-                if (b1 < q4) poly_batch<false>(sc1, pk1, den, lane);
-                else if (b1 == q4) poly_batch<true>(sc1, pk1, den, lane);
-                else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) pk1[i] = 0u;
-                }
-                tmem_st16(tmem_addr(tb, lane_base, C::colT + b0 * 16), pk0);
-                tmem_st16(tmem_addr(tb, lane_base, C::colT + b1 * 16), pk1);
+                tmem_st16(tmem_addr(tb, lane_base, C::colT + b * 16), pk);
             }
             s_den[(c & 1) * kC + tid] = den;
             tmem_wait_st();
@@ -682,13 +744,13 @@ template <int DV>
 based_status launch_dv(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH, int L,
                        int flags, float* ws, int nseg, cudaStream_t stream) {
     using C = Cfg<DV>;
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     if (!make_map(&tq, q, BH, L, kDFeat, kDFeat, CU_TENSOR_MAP_SWIZZLE_32B) ||
         !make_map(&tk, k, BH, L, kDFeat, kDFeat, CU_TENSOR_MAP_SWIZZLE_32B) ||
-        !make_map(&tv, v, BH, L, DV, 64, CU_TENSOR_MAP_SWIZZLE_128B))
+        !make_map(&tv, v, BH, L, DV, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map(&to, out, BH, L, DV, 64, CU_TENSOR_MAP_SWIZZLE_128B))
         return BASED_ERR_CUDA;
     Params p;
-    p.out = static_cast<__nv_bfloat16*>(out);
     p.kv_abi = kv;
     p.z_abi = z;
     p.ws = ws;
@@ -707,12 +769,12 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
                              (int)C::kSmemBytes) != cudaSuccess)
         return BASED_ERR_CUDA;
     if (nseg > 1) {
-        prefill_tc_kernel<DV, true><<<dim3(nseg - 1, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, p);
+        prefill_tc_kernel<DV, true><<<dim3(nseg - 1, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
         note_launch();
         const based_status st = check_launch("prefill_tc_kernel<state>");
         if (st != BASED_OK) return st;
     }
-    prefill_tc_kernel<DV, false><<<dim3(nseg, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, p);
+    prefill_tc_kernel<DV, false><<<dim3(nseg, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
     note_launch();
     return check_launch("prefill_tc_kernel");
 }
