@@ -106,6 +106,8 @@ based_status swa_forward(const void* q, const void* k, const void* v, void* out,
     if ((long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return BASED_ERR_ALIGNMENT;
     const float scale = softmax_scale > 0.f ? softmax_scale : 0.125f;   // 1/sqrt(64)
+    if (io == BASED_BF16 && swa_tc_supported(window))
+        return launch_swa_tc(q, k, v, out, B * H, L, window, scale, static_cast<cudaStream_t>(cuda_stream));
     return launch_swa_simt(q, k, v, out, B * H, L, window, scale, io, static_cast<cudaStream_t>(cuda_stream));
 }
 
