@@ -26,7 +26,9 @@
 // warps 4-7 "feature" group (one thread per token: phi expansion), warps 8-11 "state"
 // group (one thread per TMEM lane: bf16 state copy, state I/O), warps 12-15 "output"
 // group (one thread per output row: normalise, stage, TMA store), warp 16 TMA producer,
-// warp 17 MMA issuer.  All cross-role hand-offs are mbarriers with bounded waits.
+// warp 17 issues the state-update MMAs (5)/(z), warp 18 the output-side MMAs (1)/(4)/(3):
+// two independent in-order streams, so the state chain runs ahead of the output chain.
+// All cross-role hand-offs are mbarriers with bounded waits.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -41,8 +43,8 @@ namespace {
 constexpr int kC = 128;            // tokens per chunk
 constexpr int kF = 160;            // internal feature count (153 padded to a multiple of 16)
 constexpr int kFBlk = 5;           // 32-feature SWIZZLE_64B blocks
-constexpr int kThreads = 576;
-constexpr int kWarpTma = 16, kWarpMma = 17;
+constexpr int kThreads = 608;
+constexpr int kWarpTma = 16, kWarpMma = 17, kWarpMmaY = 18;
 constexpr float kRsqrt2 = 0.70710678118654752f;
 
 // ---- workspace layout of one (head, segment) partial state: [kF][DV] fp32 then [kF] fp32
@@ -85,7 +87,7 @@ struct Cfg {
 };
 
 enum Bar {
-    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kP, kG2, kG4, kG3, kYfree, kPK, kPQ, kSR, kSC, kNumBars
+    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kP, kG2, kG2b, kG4, kG3, kYfree, kPK, kPQ, kSR, kSC, kNumBars
 };
 
 struct Params {
@@ -234,8 +236,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     uint8_t* sOut = smem + C::offOut;
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(&bars[kFull0 + s], 1); mbar_init(&bars[kEmpty0 + s], 1); }
-        mbar_init(&bars[kG1], 1); mbar_init(&bars[kG2], 1); mbar_init(&bars[kG4], 1); mbar_init(&bars[kG3], 1);
+        for (int s = 0; s < NS; ++s) { mbar_init(&bars[kFull0 + s], 1); mbar_init(&bars[kEmpty0 + s], STATE_ONLY ? 1 : 2); }
+        mbar_init(&bars[kG1], 1); mbar_init(&bars[kG2], 1); mbar_init(&bars[kG2b], 1); mbar_init(&bars[kG4], 1);
+        mbar_init(&bars[kG3], 1);
         mbar_init(&bars[kP], 128); mbar_init(&bars[kYfree], 128); mbar_init(&bars[kPK], 128);
         mbar_init(&bars[kPQ], 128); mbar_init(&bars[kSR], 128); mbar_init(&bars[kSC], 128);
         *abort_flag = 0;
@@ -264,6 +267,11 @@ __global__ void __launch_bounds__(kThreads, 1)
     const uint32_t tb = *tmem_base_s;
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;     // TMEM lanes this warp may touch
     bool ok = true;
+    // "State update of chunk c done".  A parity wait can only tell a phase from the one before it,
+    // so a waiter may lag its barrier by at most one phase: the state-only pass, whose feature group
+    // works two chunks ahead on two alternating tiles, uses one barrier per tile.
+    auto g2_bar = [&](int c) -> uint64_t* { return &bars[(STATE_ONLY && (c & 1)) ? kG2b : kG2]; };
+    auto g2_parity = [&](int c) -> uint32_t { return STATE_ONLY ? ((c >> 1) & 1) : (c & 1); };
 
     if (warp == kWarpTma) {
         // ===================================================================== TMA producer
@@ -283,39 +291,25 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
         }
     } else if (warp == kWarpMma) {
-        // ===================================================================== MMA issuer
+        // ===================================================================== MMA issuer, state chain
         if (lane == 0) {
-            constexpr uint64_t dQK = make_smem_desc_base(16, 256, kSwizzle32B);           // K-major [128][16]
-            constexpr uint64_t dPhiK = make_smem_desc_base(16, 512, kSwizzle64B);         // K-major, 64-byte rows
             constexpr uint64_t dPhiMN = make_smem_desc_base(C::kPhiBlk, 512, kSwizzle64B);// MN-major view of a phi tile
             constexpr uint64_t dV = make_smem_desc_base(kC * 128, 1024, kSwizzle128B);    // MN-major [128 tok][DV]
             constexpr uint64_t dOnes = make_smem_desc_base(16, 1024, kSwizzle128B);
-            constexpr uint32_t i1 = make_idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t iZ0 = make_idesc_bf16(128, 16, 1, 0);
             constexpr uint32_t iZ1 = make_idesc_bf16(64, 16, 1, 0);
             constexpr uint32_t i5 = make_idesc_bf16(128, kF, 1, 1);
-            constexpr uint32_t i4 = make_idesc_bf16(128, C::kNY, 0, 0);
-            constexpr uint32_t i3 = make_idesc_bf16(128, DV, 0, 1);
             const uint32_t aOnes = smem_u32(sOnes);
-            // low descriptor words: constant part + (start address >> 4)
-            const uint32_t lQK = desc_lo(dQK), lV = desc_lo(dV);
-            const uint32_t lPK = desc_lo(dPhiMN) + (smem_u32(sPK) >> 4), lPQ = desc_lo(dPhiK) + (smem_u32(sPQ) >> 4);
-            const uint32_t lSc = desc_lo(dPhiK) + (smem_u32(sSc) >> 4), lOnes = desc_lo(dOnes) + (aOnes >> 4);
+            const uint32_t lV = desc_lo(dV), lOnes = desc_lo(dOnes) + (aOnes >> 4);
+            // STATE_ONLY alternates between two phi(K) tiles (the phi(Q) tile is unused there)
+            const uint32_t lPK0 = desc_lo(dPhiMN) + (smem_u32(sPK) >> 4), lPK1 = desc_lo(dPhiMN) + (smem_u32(sPQ) >> 4);
             for (int c = 0; c < nch && ok; ++c) {
                 const int s = c % NS;
                 const uint32_t ph = c & 1;
-                const uint32_t aSt = smem_u32(smem + C::offStage + s * C::kStageBytes);
-                const uint32_t aVt = aSt + 2 * C::kQKBytes;
+                const uint32_t aVt = smem_u32(smem + C::offStage + s * C::kStageBytes) + 2 * C::kQKBytes;
+                const uint32_t lPK = (STATE_ONLY && (c & 1)) ? lPK1 : lPK0;
                 ok = mbar_wait(&bars[kFull0 + s], (c / NS) & 1, abort_flag);
-                if (!ok) break;
-                TRACE(1, c, 0);
-                tc_fence_after();
-                if (!STATE_ONLY) {
-                    mma_ss_lh<false>(tb + C::colT, lQK + (aSt >> 4), desc_hi(dQK), lQK + ((aSt + C::kQKBytes) >> 4),
-                                     desc_hi(dQK), i1);
-                    mma_commit(&bars[kG1]);
-                }
-                ok = mbar_wait(&bars[kPK], ph, abort_flag);
+                if (ok) ok = mbar_wait(&bars[kPK], ph, abort_flag);
                 // the state group has read (or, before chunk 0, initialised) the state in TMEM
                 if (ok && (!STATE_ONLY || c == 0)) ok = mbar_wait(&bars[kSR], ph, abort_flag);
                 if (!ok) break;
@@ -342,17 +336,39 @@ __global__ void __launch_bounds__(kThreads, 1)
                                         lOnes + (k & 1) * 2, desc_hi(dOnes), iZ1);
                     }
                 }
-                mma_commit(&bars[kG2]);
+                mma_commit(g2_bar(c));
+                mma_commit(&bars[kEmpty0 + s]);
                 TRACE(1, c, 2);
-                if (STATE_ONLY) {
-                    mma_commit(&bars[kEmpty0 + s]);
-                    continue;
-                }
+            }
+        }
+    } else if (warp == kWarpMmaY) {
+        // ===================================================================== MMA issuer, output chain
+        if (lane == 0 && !STATE_ONLY) {
+            constexpr uint64_t dQK = make_smem_desc_base(16, 256, kSwizzle32B);           // K-major [128][16]
+            constexpr uint64_t dPhiK = make_smem_desc_base(16, 512, kSwizzle64B);         // K-major, 64-byte rows
+            constexpr uint64_t dV = make_smem_desc_base(kC * 128, 1024, kSwizzle128B);    // MN-major [128 tok][DV]
+            constexpr uint32_t i1 = make_idesc_bf16(128, 128, 0, 0);
+            constexpr uint32_t i4 = make_idesc_bf16(128, C::kNY, 0, 0);
+            constexpr uint32_t i3 = make_idesc_bf16(128, DV, 0, 1);
+            const uint32_t lQK = desc_lo(dQK), lV = desc_lo(dV);
+            const uint32_t lPQ = desc_lo(dPhiK) + (smem_u32(sPQ) >> 4), lSc = desc_lo(dPhiK) + (smem_u32(sSc) >> 4);
+            for (int c = 0; c < nch && ok; ++c) {
+                const int s = c % NS;
+                const uint32_t ph = c & 1;
+                const uint32_t aSt = smem_u32(smem + C::offStage + s * C::kStageBytes);
+                const uint32_t aVt = aSt + 2 * C::kQKBytes;
+                ok = mbar_wait(&bars[kFull0 + s], (c / NS) & 1, abort_flag);
+                if (!ok) break;
+                TRACE(0, c, 0);
+                tc_fence_after();
+                mma_ss_lh<false>(tb + C::colT, lQK + (aSt >> 4), desc_hi(dQK), lQK + ((aSt + C::kQKBytes) >> 4),
+                                 desc_hi(dQK), i1);
+                mma_commit(&bars[kG1]);
                 ok = mbar_wait(&bars[kPQ], ph, abort_flag);
                 if (ok) ok = mbar_wait(&bars[kSC], ph, abort_flag);
                 if (ok && c > 0) ok = mbar_wait(&bars[kYfree], ph ^ 1, abort_flag);
                 if (!ok) break;
-                TRACE(1, c, 3);
+                TRACE(0, c, 3);
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < kF / 16; ++k) {
@@ -362,10 +378,10 @@ __global__ void __launch_bounds__(kThreads, 1)
                     else mma_ss_lh<true>(tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
                 }
                 mma_commit(&bars[kG4]);
-                TRACE(1, c, 4);
+                TRACE(0, c, 4);
                 ok = mbar_wait(&bars[kP], ph, abort_flag);
                 if (!ok) break;
-                TRACE(1, c, 5);
+                TRACE(0, c, 5);
                 tc_fence_after();
                 {
                     const uint32_t b_lo = lV + (aVt >> 4);
@@ -375,7 +391,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 }
                 mma_commit(&bars[kG3]);
                 mma_commit(&bars[kEmpty0 + s]);
-                TRACE(1, c, 6);
+                TRACE(0, c, 6);
             }
         }
     } else if (warp >= 12) {
@@ -518,7 +534,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             mbar_arrive(&bars[kSR]);
             // a parity wait only tells the current phase from the one before, so follow the
             // state-update barrier chunk by chunk
-            for (int c = 0; c < nch && ok; ++c) ok = mbar_wait(&bars[kG2], c & 1, abort_flag);
+            for (int c = 0; c < nch && ok; ++c) ok = mbar_wait(g2_bar(c), g2_parity(c), abort_flag);
         } else {
             for (int c = 0; c < nch && ok; ++c) {
                 if (c > 0) {
@@ -629,12 +645,15 @@ __global__ void __launch_bounds__(kThreads, 1)
             uint4 klo, khi, qlo = make_uint4(0u, 0u, 0u, 0u), qhi = qlo;
             read_qk_row(st + C::kQKBytes, t, klo, khi);
             if (!STATE_ONLY) read_qk_row(st, t, qlo, qhi);
-            if (c > 0) {
-                ok = mbar_wait(&bars[kG2], (c - 1) & 1, abort_flag);   // step (5) of chunk c-1 has read phi(K)
+            // the tile being overwritten was last read by step (5) of chunk c-1 (c-2 in STATE_ONLY,
+            // which alternates between two tiles)
+            constexpr int kLag = STATE_ONLY ? 2 : 1;
+            if (c >= kLag) {
+                ok = mbar_wait(g2_bar(c - kLag), g2_parity(c - kLag), abort_flag);
                 if (!ok) break;
             }
             if (t == 0) TRACE(3, c, 1);
-            write_phi_row(klo, khi, sPK, t, valid);
+            write_phi_row(klo, khi, (STATE_ONLY && (c & 1)) ? sPQ : sPK, t, valid);
             fence_proxy_async_smem();
             mbar_arrive(&bars[kPK]);
             if (t == 0) TRACE(3, c, 2);
