@@ -30,6 +30,7 @@
 // two independent in-order streams, so the state chain runs ahead of the output chain.
 // All cross-role hand-offs are mbarriers with bounded waits.
 #include <cuda_bf16.h>
+#include <cstdlib>
 
 #include "common.cuh"
 #include "sm100.cuh"
@@ -73,21 +74,22 @@ struct Cfg {
     static constexpr uint32_t offSc = offPQ + kPhiBytes;
     static constexpr uint32_t offOut = offSc + kScBytes;
     static constexpr uint32_t offMisc = offOut + kOutBytes;
-    static constexpr uint32_t kMiscBytes = 2048;                // barriers, row sums, ABI row table
+    static constexpr uint32_t kMiscBytes = 3072;                // barriers, row sums, ABI row table
     static constexpr uint32_t kSmemBytes = offMisc + kMiscBytes + 1024;   // + alignment slack
     static_assert(kSmemBytes <= 232448, "shared memory budget");
     // TMEM columns
     static constexpr uint32_t colT = 0;                          // scores, overwritten in place by P
-    static constexpr uint32_t colY = 128;
+    static constexpr bool kTDouble = (DV == 64);                 // two score buffers when TMEM has room
+    static constexpr uint32_t colY = kTDouble ? 256 : 128;
     static constexpr uint32_t colS = colY + kNY;
     static constexpr uint32_t colZ0 = colS + kF;                 // d_v 128 only
     static constexpr uint32_t colZ1 = colZ0 + 16;
-    static_assert(colZ1 + 16 <= 512, "TMEM budget");
+    static_assert((DV == 64 ? colS + kF : colZ1 + 16) <= 512, "TMEM budget");
     static_assert(kScBlk % 1024 == 0 && kStageBytes % 1024 == 0 && offPK % 1024 == 0, "tiles stay 1024-byte aligned");
 };
 
 enum Bar {
-    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kP, kG2, kG2b, kG4, kG3, kYfree, kPK, kPQ, kSR, kSC, kNumBars
+    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kG1b, kP, kPb, kG2, kG2b, kG4, kG3, kYfree, kPK, kPQ, kSR, kSC, kNumBars
 };
 
 struct Params {
@@ -220,8 +222,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offMisc);
     uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + kNumBars);
     volatile uint32_t* abort_flag = tmem_base_s + 1;
-    float* s_den = reinterpret_cast<float*>(tmem_base_s + 2);          // [2][128] row sums of in-chunk weights
-    short2* s_abi = reinterpret_cast<short2*>(s_den + 2 * kC);         // [160] ABI rows of each internal feature
+    float* s_den = reinterpret_cast<float*>(tmem_base_s + 2);          // [4][128] row sums of in-chunk weights
+    short2* s_abi = reinterpret_cast<short2*>(s_den + 4 * kC);         // [160] ABI rows of each internal feature
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int seg = blockIdx.x, head = blockIdx.y;
@@ -237,7 +239,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(&bars[kFull0 + s], 1); mbar_init(&bars[kEmpty0 + s], STATE_ONLY ? 1 : 2); }
-        mbar_init(&bars[kG1], 1); mbar_init(&bars[kG2], 1); mbar_init(&bars[kG2b], 1); mbar_init(&bars[kG4], 1);
+        mbar_init(&bars[kG1], 1); mbar_init(&bars[kG1b], 1); mbar_init(&bars[kPb], 128); mbar_init(&bars[kG2], 1); mbar_init(&bars[kG2b], 1); mbar_init(&bars[kG4], 1);
         mbar_init(&bars[kG3], 1);
         mbar_init(&bars[kP], 128); mbar_init(&bars[kYfree], 128); mbar_init(&bars[kPK], 128);
         mbar_init(&bars[kPQ], 128); mbar_init(&bars[kSR], 128); mbar_init(&bars[kSC], 128);
@@ -270,6 +272,10 @@ __global__ void __launch_bounds__(kThreads, 1)
     // "State update of chunk c done".  A parity wait can only tell a phase from the one before it,
     // so a waiter may lag its barrier by at most one phase: the state-only pass, whose feature group
     // works two chunks ahead on two alternating tiles, uses one barrier per tile.
+    // Scores / weights of chunk c: with two score buffers the row group may run a chunk ahead of the
+    // MMA issuer (and the issuer's scores a chunk ahead of the row group), so each buffer has its own pair.
+    auto t_idx = [&](int c) -> int { return C::kTDouble ? (c & 1) : 0; };
+    auto t_parity = [&](int c) -> uint32_t { return C::kTDouble ? ((c >> 1) & 1) : (c & 1); };
     auto g2_bar = [&](int c) -> uint64_t* { return &bars[(STATE_ONLY && (c & 1)) ? kG2b : kG2]; };
     auto g2_parity = [&](int c) -> uint32_t { return STATE_ONLY ? ((c >> 1) & 1) : (c & 1); };
 
@@ -352,18 +358,30 @@ __global__ void __launch_bounds__(kThreads, 1)
             constexpr uint32_t i3 = make_idesc_bf16(128, DV, 0, 1);
             const uint32_t lQK = desc_lo(dQK), lV = desc_lo(dV);
             const uint32_t lPQ = desc_lo(dPhiK) + (smem_u32(sPQ) >> 4), lSc = desc_lo(dPhiK) + (smem_u32(sSc) >> 4);
+            // scores of chunk c: T[c & 1] (or the single T) = Q_c K_c^T
+            auto issue_scores = [&](int c) -> bool {
+                const int s = c % NS;
+                if (!mbar_wait(&bars[kFull0 + s], (c / NS) & 1, abort_flag)) return false;
+                TRACE(0, c, 0);
+                tc_fence_after();
+                const uint32_t aSt = smem_u32(smem + C::offStage + s * C::kStageBytes);
+                mma_ss_lh<false>(tb + C::colT + (C::kTDouble ? (c & 1) * 128 : 0), lQK + (aSt >> 4), desc_hi(dQK),
+                                 lQK + ((aSt + C::kQKBytes) >> 4), desc_hi(dQK), i1);
+                mma_commit(&bars[kG1 + t_idx(c)]);
+                return true;
+            };
+            if (nch > 0) ok = issue_scores(0);
             for (int c = 0; c < nch && ok; ++c) {
                 const int s = c % NS;
                 const uint32_t ph = c & 1;
-                const uint32_t aSt = smem_u32(smem + C::offStage + s * C::kStageBytes);
-                const uint32_t aVt = aSt + 2 * C::kQKBytes;
-                ok = mbar_wait(&bars[kFull0 + s], (c / NS) & 1, abort_flag);
-                if (!ok) break;
-                TRACE(0, c, 0);
-                tc_fence_after();
-                mma_ss_lh<false>(tb + C::colT, lQK + (aSt >> 4), desc_hi(dQK), lQK + ((aSt + C::kQKBytes) >> 4),
-                                 desc_hi(dQK), i1);
-                mma_commit(&bars[kG1]);
+                const uint32_t aVt = smem_u32(smem + C::offStage + s * C::kStageBytes) + 2 * C::kQKBytes;
+                const uint32_t colTc = C::colT + (C::kTDouble ? (c & 1) * 128 : 0);
+                // with two score buffers the next chunk's scores are issued ahead of this chunk's
+                // steps (4) and (3), so its polynomial overlaps them
+                if (C::kTDouble && c + 1 < nch) {
+                    ok = issue_scores(c + 1);
+                    if (!ok) break;
+                }
                 ok = mbar_wait(&bars[kPQ], ph, abort_flag);
                 if (ok) ok = mbar_wait(&bars[kSC], ph, abort_flag);
                 if (ok && c > 0) ok = mbar_wait(&bars[kYfree], ph ^ 1, abort_flag);
@@ -379,7 +397,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 }
                 mma_commit(&bars[kG4]);
                 TRACE(0, c, 4);
-                ok = mbar_wait(&bars[kP], ph, abort_flag);
+                ok = mbar_wait(&bars[kP + t_idx(c)], t_parity(c), abort_flag);
                 if (!ok) break;
                 TRACE(0, c, 5);
                 tc_fence_after();
@@ -387,11 +405,13 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const uint32_t b_lo = lV + (aVt >> 4);
 #pragma unroll
                     for (int k = 0; k < kC / 16; ++k)
-                        mma_ts_lh<true>(tb + C::colY, tb + C::colT + k * 8, b_lo + k * (2048 >> 4), desc_hi(dV), i3);
+                        mma_ts_lh<true>(tb + C::colY, tb + colTc + k * 8, b_lo + k * (2048 >> 4), desc_hi(dV), i3);
                 }
                 mma_commit(&bars[kG3]);
                 mma_commit(&bars[kEmpty0 + s]);
                 TRACE(0, c, 6);
+                // single score buffer: P of this chunk has to be consumed before the next scores land
+                if (!C::kTDouble && c + 1 < nch) ok = issue_scores(c + 1);
             }
         }
     } else if (warp >= 12) {
@@ -410,7 +430,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 uint32_t dcol;
                 tmem_ld1(tmem_addr(tb, lane_base, C::colY + DV), dcol);
                 tmem_wait_ld();
-                const float inv = 1.0f / (s_den[(c & 1) * kC + t] + __uint_as_float(dcol) + kEps);
+                const float inv = 1.0f / (s_den[(c & 3) * kC + t] + __uint_as_float(dcol) + kEps);
 #pragma unroll 1
                 for (int h = 0; h < DV / 64; ++h) {
                     uint32_t y0[32], y1[32];
@@ -675,39 +695,53 @@ __global__ void __launch_bounds__(kThreads, 1)
         // bf16 weights overwrite the scores in place (columns [0, 64) of the same lanes).
         const int q4 = warp;                            // lane quarter == 32-row block of the chunk
         for (int c = 0; c < nch && ok; ++c) {
-            ok = mbar_wait(&bars[kG1], c & 1, abort_flag);
+            ok = mbar_wait(&bars[kG1 + t_idx(c)], t_parity(c), abort_flag);
             if (!ok) break;
             if (tid == 96) TRACE(2, c, 0);
             tc_fence_after();
-            float den = 0.f;
+            const uint32_t colTc = C::colT + (C::kTDouble ? (c & 1) * 128 : 0);
+            float den0 = 0.f, den1 = 0.f;
 #pragma unroll 1
             for (int b = 0; b < 4; ++b) {
                 uint32_t pk[16];
                 if (b <= q4) {                           // some row of this warp sees these key columns
                     uint32_t sc[32];
-                    tmem_ld32(tmem_addr(tb, lane_base, C::colT + b * 32), sc);
+                    tmem_ld32(tmem_addr(tb, lane_base, colTc + b * 32), sc);
                     tmem_wait_ld();
-                    const int limit = (b < q4) ? 64 : lane;      // last visible column of the batch for this row
+                    if (b < q4) {                        // fully visible batch: no mask
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float s0 = __uint_as_float(sc[2 * i]), s1 = __uint_as_float(sc[2 * i + 1]);
-                        float w0 = fmaf(s0, fmaf(s0, 0.03125f, 0.25f), 1.0f);
-                        float w1 = fmaf(s1, fmaf(s1, 0.03125f, 0.25f), 1.0f);
-                        w0 = (2 * i <= limit) ? w0 : 0.f;
-                        w1 = (2 * i + 1 <= limit) ? w1 : 0.f;
-                        den += w0 + w1;
-                        pk[i] = pack_bf16(w0, w1);
+                        for (int i = 0; i < 16; ++i) {
+                            const float s0 = __uint_as_float(sc[2 * i]), s1 = __uint_as_float(sc[2 * i + 1]);
+                            const float w0 = fmaf(s0, fmaf(s0, 0.03125f, 0.25f), 1.0f);
+                            const float w1 = fmaf(s1, fmaf(s1, 0.03125f, 0.25f), 1.0f);
+                            den0 += w0;
+                            den1 += w1;
+                            pk[i] = pack_bf16(w0, w1);
+                        }
+                    } else {                             // the batch that holds the diagonal
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const float s0 = __uint_as_float(sc[2 * i]), s1 = __uint_as_float(sc[2 * i + 1]);
+                            float w0 = fmaf(s0, fmaf(s0, 0.03125f, 0.25f), 1.0f);
+                            float w1 = fmaf(s1, fmaf(s1, 0.03125f, 0.25f), 1.0f);
+                            w0 = (2 * i <= lane) ? w0 : 0.f;
+                            w1 = (2 * i + 1 <= lane) ? w1 : 0.f;
+                            den0 += w0;
+                            den1 += w1;
+                            pk[i] = pack_bf16(w0, w1);
+                        }
                     }
                 } else {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) pk[i] = 0u;
                 }
-                tmem_st16(tmem_addr(tb, lane_base, C::colT + b * 16), pk);
+                tmem_st16(tmem_addr(tb, lane_base, colTc + b * 16), pk);
             }
-            s_den[(c & 1) * kC + tid] = den;
+            const float den = den0 + den1;
+            s_den[(c & 3) * kC + tid] = den;
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(&bars[kP]);
+            mbar_arrive(&bars[kP + t_idx(c)]);
             if (tid == 96) TRACE(2, c, 1);
         }
     }
@@ -800,13 +834,19 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
 
 }  // namespace
 
-// Number of sequence segments a head is split into so that about one CTA per SM is busy.
+// Number of sequence segments a head is split into so that about one CTA per SM is busy
+// (measured on B200: cfg 2, 64 heads x 16 chunks, runs 29 us unsplit against 35 us in two segments).
 int prefill_tc_segments(int BH, int L) {
     const int nch = (L + kC - 1) / kC;
     int nseg = 148 / BH;
-    if (nseg < 1) nseg = 1;
+#ifdef BASED_TRACE
+    if (const char* e = getenv("BASED_NSEG")) nseg = atoi(e);
+#endif
     if (nseg > 8) nseg = 8;
-    if (nseg > nch) nseg = nch;
+    // a split costs a second launch, a second start-up and the extra state pass: it pays only when
+    // every segment keeps at least 16 chunks
+    if (nseg > nch / 16) nseg = nch / 16;
+    if (nseg < 1) nseg = 1;
     // every segment must own at least one chunk
     while (nseg > 1 && ((nch + nseg - 1) / nseg) * (nseg - 1) >= nch) --nseg;
     return nseg;

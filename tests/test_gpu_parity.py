@@ -74,7 +74,9 @@ def test_prefill_small_shapes(dtype, d_v, L):
 
 
 @pytest.mark.parametrize("B,H,d_v,L", [(10, 16, 64, 300), (5, 16, 128, 515), (4, 16, 64, 700), (2, 16, 128, 1100),
-                                       (1, 16, 64, 2048), (1, 3, 128, 1000)])
+                                       (1, 16, 64, 2048), (1, 3, 128, 1000),
+                                       # long enough to be cut into 2, 3 and 8 sequence segments
+                                       (1, 2, 64, 4200), (1, 3, 128, 6200), (1, 1, 64, 16500)])
 def test_prefill_bf16_many_chunks(B, H, d_v, L):
     """Several 128-token chunks per CTA, with and without the sequence split into segments
     (the split depends on B*H), ragged tails included."""

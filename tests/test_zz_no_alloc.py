@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 
 
 def test_static_scratch_matches_workspace_variant_twice():
-    B, H, L, d_v = 2, 8, 1500, 64                       # 16 heads -> several segments of several chunks
+    B, H, L, d_v = 2, 4, 4200, 64                       # 8 heads x 33 chunks -> two segments per head
     assert based.based_prefill_workspace_bytes(B, H, L, 16, d_v, based.BASED_BF16) > 0
     for seed in (21, 22):
         w = wl.Workload("noalloc", B, H, L, 16, d_v, "bf16", 0.25)
@@ -34,7 +34,7 @@ def test_static_scratch_matches_workspace_variant_twice():
 
 
 def test_static_scratch_rejects_oversized_requests():
-    B, H, L, d_v = 1, 18, 4096, 128                     # 8 segments x 18 heads x 82,560 B > 8 MiB
+    B, H, L, d_v = 1, 18, 16384, 128                    # 7 partial states x 18 heads x 82,560 B > 8 MiB
     need = based.based_prefill_workspace_bytes(B, H, L, 16, d_v, based.BASED_BF16)
     assert need > based.based_static_scratch_bytes() == 8 << 20
     q = torch.zeros(B, H, L, 16, dtype=torch.bfloat16, device="cuda")
