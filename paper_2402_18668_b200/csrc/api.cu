@@ -1,6 +1,7 @@
 // C ABI of libbased: argument validation and dispatch.  See include/based.h for the
 // contract of every entry point.
 #include <atomic>
+#include <mutex>
 #include <cstdio>
 
 #include "common.cuh"
@@ -10,11 +11,24 @@ namespace based {
 __device__ unsigned int g_error_word = 0;
 
 based_status error_word_ptr(unsigned int** ptr) {
-    // the symbol has one instance per device: resolve it with that device current
-    void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_error_word) != cudaSuccess) return BASED_ERR_CUDA;
-    *ptr = static_cast<unsigned int*>(p);
+    // the symbol has one instance per device: resolve it once per device, with that device current
+    static std::atomic<unsigned int*> cache[64];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BASED_ERR_CUDA;
+    unsigned int* p = cache[dev].load(std::memory_order_acquire);
+    if (p == nullptr) {
+        void* q = nullptr;
+        if (cudaGetSymbolAddress(&q, g_error_word) != cudaSuccess) return BASED_ERR_CUDA;
+        p = static_cast<unsigned int*>(q);
+        cache[dev].store(p, std::memory_order_release);
+    }
+    *ptr = p;
     return BASED_OK;
+}
+
+std::mutex& setup_mutex() {
+    static std::mutex mu;
+    return mu;
 }
 
 static std::atomic<unsigned long long> g_launches{0};

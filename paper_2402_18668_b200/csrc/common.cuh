@@ -4,6 +4,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "based.h"
 
 namespace based {
@@ -18,6 +21,9 @@ constexpr float kQuadScale = 0.17677669529663687f;      // 1 / (4 sqrt 2)
 // Device address of the sticky status word of the current device (bit 0: a bounded
 // wait timed out).  Kernels that can time out receive it as an argument.
 based_status error_word_ptr(unsigned int** ptr);
+
+// serialises the per-device one-time set-up of the launchers (function attributes and the like)
+std::mutex& setup_mutex();
 
 // host-side bookkeeping
 void note_launch();                                     // ++launch counter

@@ -816,11 +816,20 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
 #ifdef BASED_TRACE
     p.trace = g_trace;
 #endif
-    if (cudaFuncSetAttribute(prefill_tc_kernel<DV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)C::kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(prefill_tc_kernel<DV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)C::kSmemBytes) != cudaSuccess)
-        return BASED_ERR_CUDA;
+    {
+        static bool configured[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BASED_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(setup_mutex());
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(prefill_tc_kernel<DV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)C::kSmemBytes) != cudaSuccess ||
+                cudaFuncSetAttribute(prefill_tc_kernel<DV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)C::kSmemBytes) != cudaSuccess)
+                return BASED_ERR_CUDA;
+            configured[dev] = true;
+        }
+    }
     if (nseg > 1) {
         prefill_tc_kernel<DV, true><<<dim3(nseg - 1, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
         note_launch();

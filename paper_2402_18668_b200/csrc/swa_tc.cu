@@ -341,11 +341,21 @@ based_status launch_swa_tc(const void* q, const void* k, const void* v, void* ou
     p.tiles_per_head = (L + kQT - 1) / kQT;
     p.total_tiles = p.tiles_per_head * BH;
     p.scale_log2e = scale * 1.4426950408889634f;
-    if (cudaFuncSetAttribute(swa_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) !=
-        cudaSuccess)
-        return BASED_ERR_CUDA;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    static int sm_count[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BASED_ERR_CUDA;
+    {
+        std::lock_guard<std::mutex> lock(setup_mutex());
+        if (sm_count[dev] == 0) {
+            if (cudaFuncSetAttribute(swa_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) !=
+                cudaSuccess)
+                return BASED_ERR_CUDA;
+            int n = 148;
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+            sm_count[dev] = n > 0 ? n : 148;
+        }
+    }
+    const int sms = sm_count[dev];
     const int grid = p.total_tiles < sms ? p.total_tiles : sms;
     swa_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tq, tk, tv, to, p);
     note_launch();
