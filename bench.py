@@ -28,6 +28,16 @@ ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
 L2_BYTES = 126 * 1024 * 1024
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/.  cfg 2 was captured at full size; the decode and sliding-window
+# captures used half-size cases (sizing rule for profiler runs) and are scaled by the units
+# processed.  Written bytes still resident in L2 when a launch ends are not in these figures.
+NCU_TRAFFIC = {
+    "cfg2_360m_prefill": 25.23e6,                 # profiles/prefill_tc_kernel_dv64_cfg2.md (output stays in L2)
+    "cfg4_generation": 2 * (144.59e6 + 88.45e6),  # profiles/decode_step_kernel_dv128.md, 1024 -> 2048 heads
+    "cfg5_mixer_pair:swa": 2 * (201.37e6 + 43.87e6),  # profiles/swa_tc_kernel.md, 16 -> 32 heads
+}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -274,7 +284,8 @@ def bench_decode(w, steps, warmup, torch, based, dist_on, peaks):
         "workload": w.name, "metric": "decode_tokens_per_s", "value": w.B / t, "unit": "tokens/s",
         "us_per_step": t * 1e6, "steps": steps,
         "roofline": {"bound": "hbm", "achieved": state_bytes / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": state_bytes / t / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                     "frac": state_bytes / t / 1e9 / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC.get(w.name),
+                     "kernel": "decode_step_kernel", "algorithmic_bytes": state_bytes,
                      "achieved_all_bytes": all_bytes / t / 1e9, "peak_source": peaks["source"]},
     }
 
@@ -300,7 +311,8 @@ def bench_swa(w, steps, warmup, torch, based, dist_on, peaks):
         "workload": w.name, "metric": "swa_tokens_per_s", "value": w.B * w.L / t, "unit": "tokens/s",
         "ms_per_step": t * 1e3, "window": w.swa_window,
         "roofline": {"bound": "hbm", "achieved": per_set / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": per_set / t / 1e9 / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
+                     "frac": per_set / t / 1e9 / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC.get(w.name + ":swa"),
+                     "kernel": "swa_tc_kernel", "algorithmic_bytes": per_set, "peak_source": peaks["source"]},
     }
 
 
@@ -444,7 +456,10 @@ def main():
                 "peak": peaks["bf16_tflops"] if bound_tensor else peaks["hbm_gbs"],
                 "unit": "TFLOP/s" if bound_tensor else "GB/s",
                 "frac": res["frac_tensor_peak"] if bound_tensor else res["frac_hbm_peak"],
-                "traffic": None, "peak_source": peaks["source"],
+                "traffic": NCU_TRAFFIC.get(w.name), "peak_source": peaks["source"],
+                "kernel": "prefill_tc_kernel", "kernel_us": res["ms_per_step"] * 1e3 / max(1, res["launches_per_step"]),
+                "algorithmic_flops": prefill_alg_flops_per_token_head(w.d_v) * w.B * w.H * w.L,
+                "algorithmic_bytes": prefill_alg_bytes(w, w.return_state),
                 "tensor": {"achieved": res["alg_tflops"], "peak": peaks["bf16_tflops"], "frac": res["frac_tensor_peak"]},
                 "hbm": {"achieved": res["alg_gbs"], "peak": peaks["hbm_gbs"], "frac": res["frac_hbm_peak"]},
             },
