@@ -137,6 +137,15 @@ size_t based_static_scratch_bytes(void);
  */
 based_status based_poll_error(void* cuda_stream);
 
+/*
+ * Diagnostic (no counterpart in the paper): launches a one-CTA kernel whose bounded wait is
+ * made to run out after limit_ms (1..2000) - it waits on a barrier nothing signals - so the
+ * error path "wait gives up -> sticky status word -> clean kernel exit" can be checked on a
+ * live GPU without faulting or hanging it.  based_poll_error then returns
+ * BASED_ERR_DEVICE_TIMEOUT once, and the context stays usable.
+ */
+based_status based_selftest_bounded_wait(unsigned int limit_ms, void* cuda_stream);
+
 const char* based_status_string(based_status s);
 int based_version(void);
 

@@ -24,7 +24,7 @@ D_EXPANDED = 1 + D_FEAT + D_FEAT * D_FEAT
 EXPORTS = (
     "based_prefill", "based_prefill_workspace_bytes", "based_decode_step", "swa_forward", "based_poll_error",
     "based_status_string", "based_version", "based_launch_count", "based_prefill_static_scratch",
-    "based_static_scratch_bytes",
+    "based_static_scratch_bytes", "based_selftest_bounded_wait",
 )
 
 _lib = None
@@ -53,6 +53,8 @@ def lib() -> ctypes.CDLL:
         L.based_prefill_static_scratch.restype = i
         L.based_prefill_static_scratch.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
         L.based_static_scratch_bytes.restype = sz
+        L.based_selftest_bounded_wait.restype = i
+        L.based_selftest_bounded_wait.argtypes = [ctypes.c_uint, vp]
         L.based_decode_step.restype = i
         L.based_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
         L.swa_forward.restype = i
@@ -178,6 +180,11 @@ def swa_forward(q, k, v, out=None, window: int = 64, softmax_scale: float = 0.0,
                            _dtype_code(q), _stream(stream))
     _check(st, "swa_forward")
     return out
+
+
+def based_selftest_bounded_wait(limit_ms: int = 20, stream=None) -> None:
+    """Makes a device-side bounded wait run out on purpose (see based.h); poll afterwards."""
+    _check(lib().based_selftest_bounded_wait(int(limit_ms), _stream(stream)), "based_selftest_bounded_wait")
 
 
 def based_poll_error(stream=None) -> int:

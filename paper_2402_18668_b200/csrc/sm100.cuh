@@ -48,7 +48,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // (shared memory) short-circuits every later wait of the CTA once one wait has given
 // up, so the kernel drains to its exit instead of hanging.  Returns false on give-up.
 constexpr uint64_t kWaitLimitNs = 1500ull * 1000ull * 1000ull;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t deadline = 0;
     for (uint32_t it = 1;; ++it) {
@@ -56,7 +57,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         if ((it & 255u) == 0) {
             if (*abort_flag) return false;
             const uint64_t now = global_timer_ns();
-            if (deadline == 0) deadline = now + kWaitLimitNs;
+            if (deadline == 0) deadline = now + limit_ns;
             else if (now > deadline) {
                 *abort_flag = 1;
                 return false;

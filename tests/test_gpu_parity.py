@@ -285,3 +285,17 @@ def test_unsupported_requests_fail_loudly():
     n0 = based.launch_count()
     based.based_prefill(q, q.clone(), torch.zeros(1, 1, 4, 64, device=DEV))
     assert based.launch_count() > n0
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A device-side wait that can never be satisfied gives up after its limit, the sticky status
+    is reported once, and the library keeps working afterwards (no fault, no hang)."""
+    assert based.based_poll_error() == based.BASED_OK
+    based.based_selftest_bounded_wait(limit_ms=20)
+    assert based.based_poll_error() == 5          # BASED_ERR_DEVICE_TIMEOUT
+    assert based.based_poll_error() == based.BASED_OK
+    q = torch.randn(1, 2, 130, 16, device=DEV).bfloat16()
+    v = torch.randn(1, 2, 130, 64, device=DEV).bfloat16()
+    out = based.based_prefill(q, q.clone(), v)
+    _poll()
+    assert torch.isfinite(out.float()).all()
