@@ -44,6 +44,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+// try_wait with a suspend-time hint: the thread is parked by the hardware until the phase completes
+// or the hint (in ns) runs out, instead of spinning and taking issue slots from the warps that work.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
+
 // Wait for the phase with the given parity, for at most ~kWaitLimitNs.  `abort_flag`
 // (shared memory) short-circuits every later wait of the CTA once one wait has given
 // up, so the kernel drains to its exit instead of hanging.  Returns false on give-up.
@@ -52,16 +66,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
                                           uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t deadline = 0;
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 0) {
-            if (*abort_flag) return false;
-            const uint64_t now = global_timer_ns();
-            if (deadline == 0) deadline = now + limit_ns;
-            else if (now > deadline) {
-                *abort_flag = 1;
-                return false;
-            }
+    for (;;) {
+        if (mbar_try_wait_hint(bar, parity, 20000u)) return true;      // parked for up to 20 us per attempt
+        if (*abort_flag) return false;
+        const uint64_t now = global_timer_ns();
+        if (deadline == 0) deadline = now + limit_ns;
+        else if (now > deadline) {
+            *abort_flag = 1;
+            return false;
         }
     }
 }
