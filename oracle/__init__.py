@@ -47,8 +47,9 @@ def _load():
         lib.oracle_linattn_recurrent.argtypes = [_dp, _dp, _dp, _dp, _dp, _dp, i, i, i, i, i]
         lib.oracle_swa.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, ctypes.c_double]
         lib.oracle_linattn_quadratic_ld.argtypes = [_dp, _dp, _dp, _dp, i, i, i]
+        lib.oracle_swa_decode_step.argtypes = [_dp, _dp, _dp, _dp, _dp, _dp, i, i, i, i, i, ctypes.c_double]
         for name in ("oracle_phi", "oracle_linattn_row", "oracle_linattn_quadratic", "oracle_linattn_recurrent",
-                     "oracle_swa", "oracle_linattn_quadratic_ld"):
+                     "oracle_swa", "oracle_linattn_quadratic_ld", "oracle_swa_decode_step"):
             getattr(lib, name).restype = None
         _lib = lib
     return _lib
@@ -150,3 +151,18 @@ def linattn_quadratic_ld(q, k, v) -> np.ndarray:
     y = np.empty((L, dv))
     _load().oracle_linattn_quadratic_ld(_p(q), _p(k), _p(v), _p(y), L, dp, dv)
     return y
+
+
+def swa_decode_step(q, k, v, k_cache, v_cache, pos: int, scale: float | None = None):
+    """One generation step on a rolling cache: q,k,v [B,H,d]; caches [B,H,w,d] (slot = pos % w).
+    Returns y [B,H,d] and the updated caches (new arrays)."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    kc, vc = _f64(k_cache).copy(), _f64(v_cache).copy()
+    B, H, d = q.shape
+    w = kc.shape[2]
+    assert kc.shape == vc.shape == (B, H, w, d)
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    y = np.empty((B, H, d))
+    _load().oracle_swa_decode_step(_p(q), _p(k), _p(v), _p(kc), _p(vc), _p(y), B, H, d, w, int(pos), float(scale))
+    return y, kc, vc

@@ -21,6 +21,10 @@
  *   oracle_swa                  exact softmax attention, Eq. (1) of Sec. 2,
  *                               restricted to the causal window
  *                               {k_{i-w+1}, ..., k_i} of Sec. 4.2.
+ *   oracle_swa_decode_step      one generation step of the same sliding-window attention on a
+ *                               rolling cache of the last w keys and values (the PyTorch
+ *                               sliding-window listing and Algorithm 3 of App. B.2, plus the
+ *                               cache update the paper's benchmark leaves out).
  *   oracle_linattn_quadratic_ld the quadratic form again with long double
  *                               accumulators (adequacy check of fp64 on tiny inputs).
  *
@@ -188,6 +192,47 @@ void oracle_swa(const double *q, const double *k, const double *v, double *y, in
                 for (int j = lo; j <= i; ++j) acc += p[j - lo] * vh[(size_t)j * d + c];
                 yh[(size_t)i * d + c] = acc / sum;
             }
+        }
+        free(p);
+    }
+}
+
+/*
+ * One decode step on a rolling window cache.  kc, vc: [B, H, w, d]; the token at absolute
+ * position t is kept in slot t % w.  The new k, v (position pos) are written first, then the
+ * query attends over the cached positions max(0, pos-w+1) .. pos (softmax does not depend on
+ * the slot order).  q, k, v, y: [B, H, d].
+ */
+void oracle_swa_decode_step(const double *q, const double *k, const double *v, double *kc, double *vc, double *y,
+                            int B, int H, int d, int w, int pos, double scale) {
+    const long nh = (long)B * H;
+    const int nvalid = (pos + 1 < w) ? pos + 1 : w;
+#pragma omp parallel for schedule(static)
+    for (long bh = 0; bh < nh; ++bh) {
+        double *kh = kc + (size_t)bh * w * d;
+        double *vh = vc + (size_t)bh * w * d;
+        const int slot = pos % w;
+        for (int m = 0; m < d; ++m) {
+            kh[(size_t)slot * d + m] = k[(size_t)bh * d + m];
+            vh[(size_t)slot * d + m] = v[(size_t)bh * d + m];
+        }
+        double *p = (double *)malloc(sizeof(double) * (size_t)w);
+        double mx = -INFINITY;
+        for (int j = 0; j < nvalid; ++j) {          /* before the ring is full, slots 0..pos are the valid ones */
+            double s = 0.0;
+            for (int m = 0; m < d; ++m) s += q[(size_t)bh * d + m] * kh[(size_t)j * d + m];
+            p[j] = s * scale;
+            if (p[j] > mx) mx = p[j];
+        }
+        double sum = 0.0;
+        for (int j = 0; j < nvalid; ++j) {
+            p[j] = exp(p[j] - mx);
+            sum += p[j];
+        }
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int j = 0; j < nvalid; ++j) acc += p[j] * vh[(size_t)j * d + c];
+            y[(size_t)bh * d + c] = acc / sum;
         }
         free(p);
     }

@@ -71,3 +71,32 @@ def test_softmax_shift_invariance_and_default_scale():
     # large logits must not overflow (max-subtraction)
     ybig = oracle.swa(q * 100.0, k * 100.0, v, w)
     assert np.isfinite(ybig).all()
+
+
+@pytest.mark.parametrize("L,w,d", [(150, 64, 64), (40, 16, 8), (9, 128, 32), (20, 1, 4)])
+def test_decode_chain_on_rolling_cache_equals_prefill_form(L, w, d):
+    """T steps on the ring cache reproduce the rows of the whole-sequence form (itself pinned
+    against library attention above), before and after the ring wraps around."""
+    B, H = 2, 2
+    q, k, v = _rand(B, H, L, d), _rand(B, H, L, d), _rand(B, H, L, d)
+    ref = oracle.swa(q, k, v, w)
+    kc = np.full((B, H, w, d), np.nan)
+    vc = np.full((B, H, w, d), np.nan)          # unwritten slots must never be read
+    for t in range(L):
+        y, kc, vc = oracle.swa_decode_step(q[:, :, t], k[:, :, t], v[:, :, t], kc, vc, t)
+        np.testing.assert_allclose(y, ref[:, :, t], rtol=1e-11, atol=1e-12)
+        np.testing.assert_array_equal(kc[:, :, t % w], k[:, :, t])
+        np.testing.assert_array_equal(vc[:, :, t % w], v[:, :, t])
+
+
+def test_decode_step_closed_forms():
+    B, H, w, d = 1, 3, 8, 4
+    kc, vc = _rand(B, H, w, d), _rand(B, H, w, d)
+    q, v = _rand(B, H, d), _rand(B, H, d)
+    # zero query: uniform weights over the (full) window after the new entry is written
+    y, kc2, vc2 = oracle.swa_decode_step(np.zeros((B, H, d)), _rand(B, H, d), v, kc, vc, pos=21)
+    np.testing.assert_allclose(y, vc2.mean(axis=2), rtol=1e-12, atol=1e-13)
+    assert np.array_equal(vc2[:, :, 21 % w], v)
+    # first token of a sequence: output is its own v whatever the cache holds
+    y, _, _ = oracle.swa_decode_step(q, _rand(B, H, d), v, kc, vc, pos=0)
+    np.testing.assert_allclose(y, v, rtol=0, atol=1e-15)
