@@ -356,6 +356,37 @@ def bench_swa(w, steps, warmup, torch, based, dist_on, peaks):
     }
 
 
+def bench_swa_decode(w, steps, warmup, torch, based, dist_on, peaks):
+    """Generation steps of the sliding-window mixer at the generation configuration's batch
+    (B x H heads, window w.swa_window, head dim 64).  One cache set is smaller than L2, so the
+    steps rotate over several independent request groups whose caches together exceed it."""
+    g = torch.Generator(device="cuda").manual_seed(3)
+    dt = w.torch_dtype
+    d, win = 64, 64
+    per_set = 2.0 * w.B * w.H * win * d * 2
+    n = n_sets_for(per_set)
+    kcs = [torch.randn(w.B, w.H, win, d, generator=g, device="cuda").to(dt) for _ in range(n)]
+    vcs = [torch.randn(w.B, w.H, win, d, generator=g, device="cuda").to(dt) for _ in range(n)]
+    q, k, v = (torch.randn(w.B, w.H, d, generator=g, device="cuda").to(dt) for _ in range(3))
+    out = torch.empty_like(v)
+
+    def step(i):
+        j = i % n
+        based.swa_decode_step(q, k, v, kcs[j], vcs[j], win + i // n, out=out)
+
+    ms = time_region(step, steps, warmup, torch, dist_on, graph=True)
+    assert based.based_poll_error() == 0
+    t = ms * 1e-3 / steps
+    bytes_step = per_set + w.B * w.H * d * 2 * 6.0        # cache read + (k, v slot write, q, k, v, out)
+    return {
+        "workload": f"B{w.B} H{w.H} window {win} d {d} {w.dtype}", "metric": "swa_decode_tokens_per_s",
+        "value": w.B / t, "unit": "tokens/s", "us_per_step": t * 1e6, "steps": steps, "cache_sets": n,
+        "roofline": {"bound": "hbm", "achieved": bytes_step / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": bytes_step / t / 1e9 / peaks["hbm_gbs"], "traffic": None, "kernel": "swa_decode_kernel",
+                     "algorithmic_bytes": bytes_step, "peak_source": peaks["source"]},
+    }
+
+
 def cpu_oracle_sample(w, budget_heads: int):
     """The oracle's recurrent form, as it stands, on the first `budget_heads` heads of the
     workload's seeded host inputs.  Returns (tokens/s scaled to whole tokens, cores, text)."""
@@ -383,7 +414,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_360m_prefill")
     ap.add_argument("--skip-extras", action="store_true", help="only the headline prefill workload")
-    ap.add_argument("--profile", choices=["prefill", "decode", "swa"],
+    ap.add_argument("--profile", choices=["prefill", "decode", "swa", "swa_decode"],
                     help="run only this arm on --shape (small cases for ncu captures) and print its result")
     ap.add_argument("--shape", default="", help="B,H,L,d_v for --profile (defaults to the arm's benchmark shape)")
     args = ap.parse_args()
@@ -431,7 +462,8 @@ def main():
     peaks = load_peaks()
 
     if args.profile:
-        base = {"prefill": w, "decode": wl.CONFIGS["cfg4_generation"], "swa": wl.CONFIGS["cfg5_mixer_pair"]}[args.profile]
+        base = {"prefill": w, "decode": wl.CONFIGS["cfg4_generation"], "swa": wl.CONFIGS["cfg5_mixer_pair"],
+                "swa_decode": wl.CONFIGS["cfg4_generation"]}[args.profile]
         if args.shape:
             B, H, L, dv = (int(x) for x in args.shape.split(","))
             base = base.scaled(name=f"{base.name}[{args.shape}]", B=B, H=H, L=L, d_v=dv)
@@ -439,6 +471,8 @@ def main():
             r, _, _ = bench_prefill(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         elif args.profile == "decode":
             r = bench_decode(base, args.steps, args.warmup, torch, based, dist_on, peaks)
+        elif args.profile == "swa_decode":
+            r = bench_swa_decode(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         else:
             r = bench_swa(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         if rank == 0:
@@ -472,6 +506,7 @@ def main():
         extras["prefill_configs"] = others
         extras["decode"] = bench_decode(wl.CONFIGS["cfg4_generation"], 1024, 16, torch, based, dist_on, peaks)
         torch.cuda.empty_cache()
+        extras["swa_decode"] = bench_swa_decode(wl.CONFIGS["cfg4_generation"], 200, 10, torch, based, dist_on, peaks)
         extras["swa"] = bench_swa(wl.CONFIGS["cfg5_mixer_pair"], max(5, args.steps // 2), 3, torch, based, dist_on,
                                   peaks)
         torch.cuda.empty_cache()

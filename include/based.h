@@ -104,6 +104,25 @@ based_status swa_forward(const void* q, const void* k, const void* v, void* out,
                          int window, float softmax_scale, based_dtype io, void* cuda_stream);
 
 /*
+ * One generation step of the sliding-window mixer on a rolling cache of the last `window` keys
+ * and values (the sliding-window PyTorch listing and Algorithm 3 of App. B.2; the cache update,
+ * which the paper's micro-benchmark leaves out, is part of the call):
+ *
+ *   k_cache[pos % window] = k ;  v_cache[pos % window] = v ;
+ *   out = sum_j softmax_j(scale * q.k_cache[j]) v_cache[j]   over the cached positions
+ *         max(0, pos-window+1) .. pos
+ *
+ * q, k, v, out [B,H,d]; k_cache, v_cache [B,H,window,d], all in the io dtype; the caches are
+ * ring buffers updated IN PLACE: the token at absolute position t lives in slot t % window, and
+ * slots of positions that have not occurred yet are never read.  `pos` is the absolute position
+ * of the new token (the same for the whole batch).  softmax_scale <= 0 selects 1/sqrt(d).
+ * Supported: d = 64; 1 <= window <= 128; io in {F32, BF16}.
+ */
+based_status swa_decode_step(const void* q, const void* k, const void* v, void* k_cache, void* v_cache, void* out,
+                             int B, int H, int d, int window, int pos, float softmax_scale, based_dtype io,
+                             void* cuda_stream);
+
+/*
  * The same computation as based_prefill, for callers that cannot give the library scratch
  * memory.  (The paper has no counterpart: this is a deployment convenience.)  Some hosts
  * may not allocate device memory around a call at all - a serving process that has handed

@@ -24,7 +24,7 @@ D_EXPANDED = 1 + D_FEAT + D_FEAT * D_FEAT
 EXPORTS = (
     "based_prefill", "based_prefill_workspace_bytes", "based_decode_step", "swa_forward", "based_poll_error",
     "based_status_string", "based_version", "based_launch_count", "based_prefill_static_scratch",
-    "based_static_scratch_bytes", "based_selftest_bounded_wait",
+    "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step",
 )
 
 _lib = None
@@ -59,6 +59,8 @@ def lib() -> ctypes.CDLL:
         L.based_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
         L.swa_forward.restype = i
         L.swa_forward.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
+        L.swa_decode_step.restype = i
+        L.swa_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
         L.based_poll_error.restype = i
         L.based_poll_error.argtypes = [vp]
         L.based_status_string.restype = ctypes.c_char_p
@@ -179,6 +181,21 @@ def swa_forward(q, k, v, out=None, window: int = 64, softmax_scale: float = 0.0,
     st = lib().swa_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, L, d, int(window), float(softmax_scale),
                            _dtype_code(q), _stream(stream))
     _check(st, "swa_forward")
+    return out
+
+
+def swa_decode_step(q, k, v, k_cache, v_cache, pos: int, out=None, softmax_scale: float = 0.0, stream=None):
+    """q,k,v [B,H,d]; k_cache,v_cache [B,H,window,d] ring buffers updated in place (slot pos % window)."""
+    _dev(q, k, v, k_cache, v_cache, out)
+    B, H, d = q.shape
+    window = k_cache.shape[2]
+    if k_cache.shape != (B, H, window, d) or v_cache.shape != k_cache.shape or k_cache.dtype != q.dtype:
+        raise ValueError("cache shapes/dtypes disagree with q")
+    if out is None:
+        out = torch.empty_like(v)
+    st = lib().swa_decode_step(_ptr(q), _ptr(k), _ptr(v), _ptr(k_cache), _ptr(v_cache), _ptr(out), B, H, d, window,
+                               int(pos), float(softmax_scale), _dtype_code(q), _stream(stream))
+    _check(st, "swa_decode_step")
     return out
 
 

@@ -58,6 +58,8 @@ based_status launch_prefill_tc(const void* q, const void* k, const void* v, void
 bool swa_tc_supported(int window);
 based_status launch_swa_tc(const void* q, const void* k, const void* v, void* out, int BH, int L, int window,
                            float scale, cudaStream_t stream);
+based_status launch_swa_decode(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
+                               int window, int pos, float scale, based_dtype io, cudaStream_t stream);
 based_status launch_swa_simt(const void* q, const void* k, const void* v, void* out, int BH, int L, int window,
                              float scale, based_dtype io, cudaStream_t stream);
 

@@ -80,6 +80,16 @@ def test_decode_and_swa_validation(lib):
     assert s(P, U, P, O, 1, 1, 16, 64, 64, 0.0, 1, None) == 3
 
 
+def test_swa_decode_validation(lib):
+    f = lib.swa_decode_step
+    O = ctypes.c_void_p(0x2000)
+    assert f(P, P, P, P, P, O, 1, 1, 64, 64, -1, 0.0, 1, None) == 1          # negative position
+    assert f(P, P, P, None, P, O, 1, 1, 64, 64, 0, 0.0, 1, None) == 1
+    assert f(P, P, P, P, P, O, 1, 1, 32, 64, 0, 0.0, 1, None) == 2           # head dim
+    assert f(P, P, P, P, P, O, 1, 1, 64, 129, 0, 0.0, 1, None) == 2          # window
+    assert f(P, P, P, P, U, O, 1, 1, 64, 64, 0, 0.0, 1, None) == 3
+
+
 def test_binding_rejects_cpu_tensors():
     import torch
     from paper_2402_18668_b200 import binding

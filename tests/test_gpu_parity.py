@@ -177,6 +177,63 @@ def test_swa_explicit_scale_and_large_logits():
     assert row_err(_np(out), ref) <= TOL_F32
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("window,steps", [(64, 150), (128, 140), (17, 40), (1, 5)])
+def test_swa_decode_chain(dtype, window, steps):
+    """Generation on the rolling cache, before and after the ring wraps: every step's output and the
+    cache contents (bit-exact copies of k, v) against the oracle; caches start NaN-filled."""
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    B, H, d = 3, 5, 64
+    q, k, v = wl.swa_standalone_inputs(B, H, steps, d, tdt, wl.generator(window * 3 + steps))
+    kc = torch.full((B, H, window, d), float("nan"), dtype=tdt, device=DEV)
+    vc = torch.full((B, H, window, d), float("nan"), dtype=tdt, device=DEV)
+    kc_ref = np.full((B, H, window, d), np.nan)
+    vc_ref = np.full((B, H, window, d), np.nan)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    for t in range(steps):
+        y_ref, kc_ref, vc_ref = oracle.swa_decode_step(_np(q[:, :, t]), _np(k[:, :, t]), _np(v[:, :, t]), kc_ref,
+                                                       vc_ref, t)
+        out = based.swa_decode_step(qd[:, :, t].contiguous(), kd[:, :, t].contiguous(), vd[:, :, t].contiguous(), kc,
+                                    vc, t)
+        assert row_err(_np(out), y_ref) <= tol_for(dtype), f"step {t}"
+    _poll()
+    nv = min(steps, window)
+    got_k, got_v = _np(kc), _np(vc)
+    filled = [t % window for t in range(steps - nv, steps)]
+    assert np.array_equal(got_k[:, :, filled], kc_ref[:, :, filled])
+    assert np.array_equal(got_v[:, :, filled], vc_ref[:, :, filled])
+
+
+def test_swa_decode_full_batch():
+    """Batch 128 x 16 heads (the generation configuration's size), window 64, around a ring wrap."""
+    B, H, d, w = 128, 16, 64, 64
+    gen = wl.generator(5)
+    kc0 = torch.randn(B, H, w, d, generator=gen).bfloat16()
+    vc0 = torch.randn(B, H, w, d, generator=gen).bfloat16()
+    kc, vc = kc0.to(DEV), vc0.to(DEV)
+    kc_ref, vc_ref = _np(kc0), _np(vc0)
+    for pos in (126, 127, 128, 129):
+        q, k, v = (torch.randn(B, H, d, generator=gen).bfloat16() for _ in range(3))
+        y_ref, kc_ref, vc_ref = oracle.swa_decode_step(_np(q), _np(k), _np(v), kc_ref, vc_ref, pos)
+        out = based.swa_decode_step(q.to(DEV), k.to(DEV), v.to(DEV), kc, vc, pos)
+        assert row_err(_np(out), y_ref) <= TOL_BF16
+    _poll()
+    assert np.array_equal(_np(kc), kc_ref) and np.array_equal(_np(vc), vc_ref)
+
+
+def test_swa_decode_matches_forward_on_gpu():
+    """The decode chain and swa_forward agree on the same sequence (both against the oracle above)."""
+    B, H, L, d, w = 2, 4, 200, 64, 64
+    q, k, v = (t.to(DEV) for t in wl.swa_standalone_inputs(B, H, L, d, torch.bfloat16, wl.generator(77)))
+    full = based.swa_forward(q, k, v, window=w)
+    kc = torch.zeros(B, H, w, d, dtype=torch.bfloat16, device=DEV)
+    vc = torch.zeros_like(kc)
+    outs = [based.swa_decode_step(q[:, :, t].contiguous(), k[:, :, t].contiguous(), v[:, :, t].contiguous(), kc, vc, t)
+            for t in range(L)]
+    _poll()
+    assert row_err(_np(torch.stack(outs, dim=2)), _np(full)) <= TOL_BF16
+
+
 # --------------------------------------------------------------------------- full-size configurations, sampled
 def _sample_rows(L, n, rng):
     fixed = [0, 1, 63, 64, 127, 128, L // 2, L - 2, L - 1]
