@@ -2,27 +2,42 @@
 // of the last `window` keys and values (the PyTorch sliding-window listing and Algorithm 3 of
 // App. B.2, here with the cache update included and for any position of the ring).
 //
-// One CTA of 128 threads per (b, h).  All loads are issued up front and kept packed (as loaded)
-// in registers: thread j holds cached key j (one row per thread, 128-bit loads) and, as one of 8
-// threads per row in 16 row groups, its share of the cached values; the new k, v are written into
-// slot pos % window; then scores, block-wide max and sum, and the weighted sum run from registers.
-// The step reads 2 * window * 64 elements per head once: it is bound by HBM bandwidth and, at
-// small batch, by launch latency.
+// One CTA of four warps per (b, h).  Thread 0 fetches the head's valid cache rows and the new q, k,
+// v with five untiled bulk copies that complete on one mbarrier, so a head's whole
+// 2 * window * 64 elements are in flight from the first instruction and up to 13 heads per SM
+// stream at once.  The warps then work from shared memory: 8 lanes share a row (8 columns each),
+// 4 rows per pass, passes dealt round-robin to the warps; scores are reduced with three shuffles
+// and kept in registers; each warp forms the softmax numerator and denominator of its own rows
+// relative to their maximum, and one block-wide barrier later the four partial results are
+// rescaled and added.  The new k, v replace the row of slot pos % window on the fly and are
+// stored to the cache.  The step reads the cache once: it is bound by HBM bandwidth and, at small
+// batch, by launch latency.
 #include <math.h>
 
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace based {
 
 namespace {
 constexpr int kHD = 64;
-constexpr int kMaxWin = 128;
+constexpr int kWarps = 4;
 
-template <typename T> struct Raw8;   // 8 consecutive elements as loaded (converted to fp32 only when used)
-template <> struct Raw8<__nv_bfloat16> {
-    uint4 u;
-    __device__ __forceinline__ void load(const __nv_bfloat16* p) { u = *reinterpret_cast<const uint4*>(p); }
-    __device__ __forceinline__ void get(float (&x)[8]) const {
+// Per-warp partial results (flash-style: each warp works relative to the maximum of its own rows
+// and the partials are rescaled when they are combined).
+struct Partials {
+    float acc[kWarps][kHD];
+    float mx[kWarps];
+    float sum[kWarps];
+};
+
+// The 8 columns lane-slot c owns in a 64-wide row: one 16-byte piece of a bf16 row, two 16-byte
+// pieces (32 columns apart) of an fp32 row, so that a warp always reads consecutive 16-byte words.
+template <typename T> struct Cols;
+template <> struct Cols<__nv_bfloat16> {
+    static __device__ __forceinline__ int col(int c, int i) { return c * 8 + i; }
+    static __device__ __forceinline__ void load(const __nv_bfloat16* row, int c, float (&x)[8]) {
+        const uint4 u = *reinterpret_cast<const uint4*>(row + c * 8);
         const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -31,137 +46,198 @@ template <> struct Raw8<__nv_bfloat16> {
             x[2 * i + 1] = f.y;
         }
     }
-};
-template <> struct Raw8<float> {
-    float4 a, b;
-    __device__ __forceinline__ void load(const float* p) {
-        a = *reinterpret_cast<const float4*>(p);
-        b = *reinterpret_cast<const float4*>(p + 4);
+    static __device__ __forceinline__ void store(__nv_bfloat16* row, int c, const float (&x)[8]) {
+        uint4 u;
+        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
+        *reinterpret_cast<uint4*>(row + c * 8) = u;
     }
-    __device__ __forceinline__ void get(float (&x)[8]) const {
+};
+template <> struct Cols<float> {
+    static __device__ __forceinline__ int col(int c, int i) { return i < 4 ? c * 4 + i : 32 + c * 4 + i - 4; }
+    static __device__ __forceinline__ void load(const float* row, int c, float (&x)[8]) {
+        const float4 a = *reinterpret_cast<const float4*>(row + c * 4);
+        const float4 b = *reinterpret_cast<const float4*>(row + 32 + c * 4);
         x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
     }
+    static __device__ __forceinline__ void store(float* row, int c, const float (&x)[8]) {
+        *reinterpret_cast<float4*>(row + c * 4) = make_float4(x[0], x[1], x[2], x[3]);
+        *reinterpret_cast<float4*>(row + 32 + c * 4) = make_float4(x[4], x[5], x[6], x[7]);
+    }
 };
 
+// Shared memory: K rows [window][64], V rows [window][64], new q, k, v [64] each (all of type T),
+// then the mbarrier, the give-up flag of the bounded wait, and the warps' partial results.
+template <typename T>
+size_t swa_decode_smem_bytes(int window) {
+    return ((size_t)2 * window * kHD + 3 * kHD) * sizeof(T) + 16 + sizeof(Partials);
+}
 }  // namespace
 
-template <typename T, int VROWS>     // VROWS: value rows per thread = ceil(window / 16)
-__global__ void __launch_bounds__(128, (sizeof(T) == 2 && VROWS <= 4) ? 8 : 4)
-swa_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, T* __restrict__ kc,
-                  T* __restrict__ vc, T* __restrict__ out, int window, int pos, float scale) {
-    __shared__ float s_q[kHD];
-    __shared__ float s_p[kMaxWin];
-    __shared__ float s_red[8];
-    __shared__ __align__(16) float s_acc[16][kHD];
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+template <typename T, int NPW>     // NPW >= ceil(window / (4 * kWarps)): passes of 4 rows per warp
+__global__ void __launch_bounds__(32 * kWarps)
+swa_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, T* __restrict__ kc,
+                  T* __restrict__ vc, T* __restrict__ out, int window, int pos, float scale,
+                  unsigned int* __restrict__ error_word) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    T* s_K = reinterpret_cast<T*>(smem);
+    T* s_V = s_K + (size_t)window * kHD;
+    T* s_qn = s_V + (size_t)window * kHD;
+    T* s_kn = s_qn + kHD;
+    T* s_vn = s_kn + kHD;
+    uint64_t* bar = reinterpret_cast<uint64_t*>(s_vn + kHD);
+    volatile uint32_t* give_up = reinterpret_cast<volatile uint32_t*>(bar + 1);
+    Partials& part = *reinterpret_cast<Partials*>(bar + 2);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 3, c = lane & 7;
     const size_t head = blockIdx.x;
     T* kh = kc + head * (size_t)window * kHD;
     T* vh = vc + head * (size_t)window * kHD;
     const int slot = pos % window;
     const int nvalid = min(pos + 1, window);          // before the ring is full, slots 0..pos are the valid ones
 
-    // Every global load of the step is issued before anything is consumed: this thread's key row
-    // and its (up to 8) value rows.  The new token's row is taken from the k, v inputs, so the loads
-    // do not wait for the cache update below.
-    const int cg = tid & 7, jg = tid >> 3;
-    Raw8<T> kx[kHD / 8];
-    if (tid < nvalid) {
-        const T* kr = (tid == slot) ? k + head * kHD : kh + (size_t)tid * kHD;
-#pragma unroll
-        for (int m = 0; m < kHD / 8; ++m) kx[m].load(kr + m * 8);
-    }
-    Raw8<T> vx[VROWS];
-#pragma unroll
-    for (int u = 0; u < VROWS; ++u) {
-        const int j = jg + 16 * u;
-        if (j < nvalid) {
-            const T* vr = (j == slot) ? v + head * kHD : vh + (size_t)j * kHD;
-            vx[u].load(vr + cg * 8);
-        }
-    }
-    // cache update, and q to shared memory
-    if (tid < kHD) {
-        kh[(size_t)slot * kHD + tid] = k[head * kHD + tid];
-        s_q[tid] = to_f32(q[head * kHD + tid]) * scale;
-    } else {
-        vh[(size_t)slot * kHD + tid - kHD] = v[head * kHD + tid - kHD];
+    if (tid == 0) {
+        sm100::mbar_init(bar, 1);
+        *give_up = 0;
+        sm100::fence_mbar_init();
+        const uint32_t rows = (uint32_t)nvalid * kHD * sizeof(T), one = kHD * sizeof(T);
+        sm100::mbar_arrive_expect_tx(bar, 2 * rows + 3 * one);
+        sm100::bulk_load_1d(s_K, kh, rows, bar);
+        sm100::bulk_load_1d(s_V, vh, rows, bar);
+        sm100::bulk_load_1d(s_qn, q + head * kHD, one, bar);
+        sm100::bulk_load_1d(s_kn, k + head * kHD, one, bar);
+        sm100::bulk_load_1d(s_vn, v + head * kHD, one, bar);
     }
     __syncthreads();
+    if (!sm100::mbar_wait(bar, 0, give_up)) {
+        if (tid == 0) atomicExch(error_word, 1u);
+        return;
+    }
 
-    // scores: thread j <-> cached key j
-    float s = -INFINITY;
-    if (tid < nvalid) {
+    // cache update (warp 0): 16-byte pieces of the new key row, then of the new value row
+    if (warp == 0) {
+        constexpr int kPieces = kHD * sizeof(T) / 16;          // 8 (bf16) or 16 (fp32) per row
+        if (lane < kPieces)
+            reinterpret_cast<uint4*>(kh + (size_t)slot * kHD)[lane] = reinterpret_cast<const uint4*>(s_kn)[lane];
+        else if (lane < 2 * kPieces)
+            reinterpret_cast<uint4*>(vh + (size_t)slot * kHD)[lane - kPieces] =
+                reinterpret_cast<const uint4*>(s_vn)[lane - kPieces];
+    }
+
+    float qx[8];
+    Cols<T>::load(s_qn, c, qx);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) qx[i] *= scale;
+
+    // scores: pass p of this warp, row group g <-> cached key 4 * (p * kWarps + warp) + g
+    float s[NPW];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int p = 0; p < NPW; ++p) {
+        const int row = 4 * (p * kWarps + warp) + g;
         float a = 0.f;
-#pragma unroll
-        for (int m = 0; m < kHD / 8; ++m) {
+        if (row < nvalid) {
             float x[8];
-            kx[m].get(x);
+            Cols<T>::load(row == slot ? s_kn : s_K + (size_t)row * kHD, c, x);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) a = fmaf(x[i], s_q[m * 8 + i], a);
+            for (int i = 0; i < 8; ++i) a = fmaf(x[i], qx[i], a);
         }
-        s = a;
+        a += __shfl_xor_sync(0xffffffffu, a, 1);
+        a += __shfl_xor_sync(0xffffffffu, a, 2);
+        a += __shfl_xor_sync(0xffffffffu, a, 4);
+        s[p] = row < nvalid ? a : -INFINITY;
+        mx = fmaxf(mx, s[p]);
     }
-    float mx = s;
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+    const float ref = mx == -INFINITY ? 0.f : mx;     // a warp whose rows all lie outside the window
+    float sum = 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (lane == 0) s_red[warp] = mx;
-    __syncthreads();
-    mx = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
-    const float e = tid < nvalid ? expf(s - mx) : 0.f;
-    s_p[tid] = e;
-    float sum = e;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if (lane == 0) s_red[4 + warp] = sum;
-    __syncthreads();
-    sum = s_red[4] + s_red[5] + s_red[6] + s_red[7];
+    for (int p = 0; p < NPW; ++p) {
+        s[p] = expf(s[p] - ref);                      // exp(-inf) = 0 for rows outside the window
+        sum += s[p];
+    }
+    sum += __shfl_xor_sync(0xffffffffu, sum, 8);
+    sum += __shfl_xor_sync(0xffffffffu, sum, 16);
 
-    // weighted sum of the cached values: 8 threads per row (8 columns each), 16 row groups
+    // this warp's weighted sum of cached values
     float acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
 #pragma unroll
-    for (int u = 0; u < VROWS; ++u) {
-        const int j = jg + 16 * u;
-        if (j < nvalid) {
-            const float pj = s_p[j];
+    for (int p = 0; p < NPW; ++p) {
+        const int row = 4 * (p * kWarps + warp) + g;
+        if (row < nvalid) {
             float x[8];
-            vx[u].get(x);
+            Cols<T>::load(row == slot ? s_vn : s_V + (size_t)row * kHD, c, x);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i] = fmaf(pj, x[i], acc[i]);
+            for (int i = 0; i < 8; ++i) acc[i] = fmaf(s[p], x[i], acc[i]);
         }
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) s_acc[jg][cg * 8 + i] = acc[i];
-    __syncthreads();
-    if (tid < kHD) {
-        float a = 0.f;
+    for (int i = 0; i < 8; ++i) {
+        acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 8);
+        acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 16);
+    }
+    if (g == 0) {
 #pragma unroll
-        for (int g = 0; g < 16; ++g) a += s_acc[g][tid];
-        out[head * kHD + tid] = from_f32<T>(a / sum);
+        for (int i = 0; i < 8; ++i) part.acc[warp][Cols<T>::col(c, i)] = acc[i];
+    }
+    if (lane == 0) {
+        part.mx[warp] = mx;
+        part.sum[warp] = sum;
+    }
+    __syncthreads();
+
+    // combine the warps' partials (warp 0 always holds row 0, so the overall maximum is finite)
+    if (tid < kHD) {
+        float M = part.mx[0];
+#pragma unroll
+        for (int w = 1; w < kWarps; ++w) M = fmaxf(M, part.mx[w]);
+        float num = 0.f, den = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const float f = expf(part.mx[w] - M);
+            num = fmaf(f, part.acc[w][tid], num);
+            den = fmaf(f, part.sum[w], den);
+        }
+        out[head * kHD + tid] = from_f32<T>(num / den);
     }
 }
 
+template <typename T, int NPW>
+static based_status launch_n(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
+                             int window, int pos, float scale, unsigned int* err, cudaStream_t stream) {
+    const size_t smem = swa_decode_smem_bytes<T>(window);
+    if (smem > 48 * 1024) {
+        if (cudaFuncSetAttribute(swa_decode_kernel<T, NPW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem) != cudaSuccess)
+            return BASED_ERR_CUDA;
+    }
+    swa_decode_kernel<T, NPW><<<BH, 32 * kWarps, smem, stream>>>(static_cast<const T*>(q), static_cast<const T*>(k),
+                                                          static_cast<const T*>(v), static_cast<T*>(kc),
+                                                          static_cast<T*>(vc), static_cast<T*>(out), window, pos,
+                                                          scale, err);
+    note_launch();
+    return check_launch("swa_decode_kernel");
+}
+
 template <typename T>
-static void launch_t(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH, int window,
-                     int pos, float scale, cudaStream_t stream) {
-    const T* qq = static_cast<const T*>(q);
-    const T* kk = static_cast<const T*>(k);
-    const T* vv = static_cast<const T*>(v);
-    T* kcc = static_cast<T*>(kc);
-    T* vcc = static_cast<T*>(vc);
-    T* oo = static_cast<T*>(out);
-    if (window <= 64) swa_decode_kernel<T, 4><<<BH, 128, 0, stream>>>(qq, kk, vv, kcc, vcc, oo, window, pos, scale);
-    else swa_decode_kernel<T, 8><<<BH, 128, 0, stream>>>(qq, kk, vv, kcc, vcc, oo, window, pos, scale);
+static based_status launch_t(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
+                             int window, int pos, float scale, unsigned int* err, cudaStream_t stream) {
+    if (window <= 64) return launch_n<T, 4>(q, k, v, kc, vc, out, BH, window, pos, scale, err, stream);
+    return launch_n<T, 8>(q, k, v, kc, vc, out, BH, window, pos, scale, err, stream);
 }
 
 based_status launch_swa_decode(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
                                int window, int pos, float scale, based_dtype io, cudaStream_t stream) {
-    if (io == BASED_F32) launch_t<float>(q, k, v, kc, vc, out, BH, window, pos, scale, stream);
-    else launch_t<__nv_bfloat16>(q, k, v, kc, vc, out, BH, window, pos, scale, stream);
-    note_launch();
-    return check_launch("swa_decode_kernel");
+    unsigned int* err = nullptr;
+    const based_status st = error_word_ptr(&err);
+    if (st != BASED_OK) return st;
+    if (io == BASED_F32) return launch_t<float>(q, k, v, kc, vc, out, BH, window, pos, scale, err, stream);
+    return launch_t<__nv_bfloat16>(q, k, v, kc, vc, out, BH, window, pos, scale, err, stream);
 }
 
 }  // namespace based
