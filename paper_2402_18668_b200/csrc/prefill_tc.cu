@@ -45,6 +45,7 @@ constexpr int kC = 128;            // tokens per chunk
 constexpr int kF = 160;            // internal feature count (153 padded to a multiple of 16)
 constexpr int kFBlk = 5;           // 32-feature SWIZZLE_64B blocks
 constexpr int kThreads = 608;
+constexpr int kModeMain = 0, kModeState = 1, kModePre = 2;
 constexpr int kWarpTma = 16, kWarpMma = 17, kWarpMmaY = 18;
 constexpr float kRsqrt2 = 0.70710678118654752f;
 
@@ -89,8 +90,11 @@ struct Cfg {
 };
 
 enum Bar {
-    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kG1b, kP, kPb, kG2, kG2b, kG4, kG3, kYfree, kPK, kPQ, kSR, kSC, kNumBars
+    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kG1b, kP, kPb, kG2, kG2b, kG4, kG3, kYfree, kPK, kPKb, kPQ, kSR, kSC, kDone, kNumBars
 };
+
+// segments per head, chunks per segment (the last one takes the rest), mode
+struct SegPlan { int nseg; int per; bool recompute; };
 
 struct Params {
     float* kv_abi;        // [BH, 273, DV] or null
@@ -109,11 +113,17 @@ struct Params {
 #ifdef BASED_TRACE
 #define TRACE(role, c, ev)                                                                   \
     do {                                                                                     \
-        if (p.trace && blockIdx.x == gridDim.x - 1 && blockIdx.y == 0 && (c) < 64)           \
+        if (p.trace && blockIdx.x == gridDim.x - 1 && blockIdx.y == 0 && (c) >= 0 && (c) < 64)           \
             p.trace[((role) * 64 + (c)) * 8 + (ev)] = clock64();                             \
+    } while (0)
+// wall-clock entry / exit of every CTA, after the per-role events
+#define TRACE_CTA(which)                                                                                      \
+    do {                                                                                                      \
+        if (p.trace) p.trace[6 * 64 * 8 + (blockIdx.y * gridDim.x + blockIdx.x) * 2 + (which)] = global_timer_ns(); \
     } while (0)
 #else
 #define TRACE(role, c, ev) do {} while (0)
+#define TRACE_CTA(which) do {} while (0)
 #endif
 
 // ---- internal feature index -> rows of the 273-row ABI layout -------------------------
@@ -210,13 +220,18 @@ __device__ __forceinline__ bool group_all(int id, bool pred) {
 
 }  // namespace
 
-template <int DV, bool STATE_ONLY>
+// MODE: kModeMain = chunk loop from a given initial state; kModeState = state-update-only pass over
+// a segment (partial state to the workspace); kModePre = kModeMain preceded by state-update-only
+// "pre-chunks" over everything before the segment (recompute mode).
+template <int DV, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
     prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
                       const Params p) {
     using C = Cfg<DV>;
     constexpr int NS = C::kStages;
+    constexpr bool STATE_ONLY = MODE == kModeState;
+    constexpr bool PRE = MODE == kModePre;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offMisc);
@@ -230,6 +245,12 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int tok_begin = seg * p.seg_len;
     const int tok_end = min(p.L, tok_begin + p.seg_len);
     const int nch = (tok_end - tok_begin + kC - 1) / kC;
+    // Recompute mode: before its own chunks the CTA runs the state update alone ("pre-chunks") over
+    // every chunk that precedes its segment.  g counts pre-chunks and own chunks together; stage
+    // ring, phi(K) tile and state-update barriers are indexed by g, everything else by c = g - npre.
+    const int npre = PRE ? tok_begin / kC : 0;
+    const int ntot = npre + nch;
+    const int tok_first = tok_begin - npre * kC;
 
     uint8_t* sPK = smem + C::offPK;
     uint8_t* sPQ = smem + C::offPQ;
@@ -237,11 +258,12 @@ __global__ void __launch_bounds__(kThreads, 1)
     uint8_t* sOnes = smem + C::offOnes;
     uint8_t* sOut = smem + C::offOut;
 
+    if (tid == 0) { TRACE(5, 0, 7); TRACE_CTA(0); }     // kernel entry
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(&bars[kFull0 + s], 1); mbar_init(&bars[kEmpty0 + s], STATE_ONLY ? 1 : 2); }
         mbar_init(&bars[kG1], 1); mbar_init(&bars[kG1b], 1); mbar_init(&bars[kPb], 128); mbar_init(&bars[kG2], 1); mbar_init(&bars[kG2b], 1); mbar_init(&bars[kG4], 1);
         mbar_init(&bars[kG3], 1);
-        mbar_init(&bars[kP], 128); mbar_init(&bars[kYfree], 128); mbar_init(&bars[kPK], 128);
+        mbar_init(&bars[kP], 128); mbar_init(&bars[kYfree], 128); mbar_init(&bars[kPK], 128); mbar_init(&bars[kPKb], 128); mbar_init(&bars[kDone], 1);
         mbar_init(&bars[kPQ], 128); mbar_init(&bars[kSR], 128); mbar_init(&bars[kSC], 128);
         *abort_flag = 0;
         fence_mbar_init();
@@ -276,20 +298,30 @@ __global__ void __launch_bounds__(kThreads, 1)
     // MMA issuer (and the issuer's scores a chunk ahead of the row group), so each buffer has its own pair.
     auto t_idx = [&](int c) -> int { return C::kTDouble ? (c & 1) : 0; };
     auto t_parity = [&](int c) -> uint32_t { return C::kTDouble ? ((c >> 1) & 1) : (c & 1); };
-    auto g2_bar = [&](int c) -> uint64_t* { return &bars[(STATE_ONLY && (c & 1)) ? kG2b : kG2]; };
-    auto g2_parity = [&](int c) -> uint32_t { return STATE_ONLY ? ((c >> 1) & 1) : (c & 1); };
+    // The state-only pass and the pre-chunks alternate between two phi(K) tiles (the phi(Q) tile is
+    // free there), even chunks on kG2, odd ones on kG2b; own chunks of the main pass use kG2 alone,
+    // continuing its phase count after the even pre-chunks.
+    auto alt = [&](int g) -> bool { return STATE_ONLY || g < npre; };
+    auto g2_bar = [&](int g) -> uint64_t* { return &bars[(alt(g) && (g & 1)) ? kG2b : kG2]; };
+    auto g2_parity = [&](int g) -> uint32_t {
+        return alt(g) ? ((g >> 1) & 1) : (uint32_t)(((npre + 1) >> 1) + (g - npre)) & 1u;
+    };
+    // "phi(K) of chunk g written": one barrier per tile for the same reason (the feature group may be
+    // two chunks ahead of the issuer where tiles alternate); same phase numbering as above
+    auto pk_bar = [&](int g) -> uint64_t* { return &bars[(alt(g) && (g & 1)) ? kPKb : kPK]; };
 
     if (warp == kWarpTma) {
         // ===================================================================== TMA producer
         if (lane == 0) {
-            for (int c = 0; c < nch && ok; ++c) {
-                const int s = c % NS;
-                ok = mbar_wait(&bars[kEmpty0 + s], ((c / NS) & 1) ^ 1, abort_flag);
+            for (int g = 0; g < ntot && ok; ++g) {
+                const int s = g % NS;
+                ok = mbar_wait(&bars[kEmpty0 + s], ((g / NS) & 1) ^ 1, abort_flag);
                 if (!ok) break;
                 uint8_t* st = smem + C::offStage + s * C::kStageBytes;
-                const int tok0 = tok_begin + c * kC;
-                mbar_arrive_expect_tx(&bars[kFull0 + s], (STATE_ONLY ? 1 : 2) * C::kQKBytes + C::kVBytes);
-                if (!STATE_ONLY) tma_load_3d(st, &tm_q, &bars[kFull0 + s], 0, tok0, head);
+                const int tok0 = tok_first + g * kC;
+                const bool with_q = !STATE_ONLY && g >= npre;
+                mbar_arrive_expect_tx(&bars[kFull0 + s], (with_q ? 2 : 1) * C::kQKBytes + C::kVBytes);
+                if (with_q) tma_load_3d(st, &tm_q, &bars[kFull0 + s], 0, tok0, head);
                 tma_load_3d(st + C::kQKBytes, &tm_k, &bars[kFull0 + s], 0, tok0, head);
 #pragma unroll
                 for (int b = 0; b < DV / 64; ++b)
@@ -309,15 +341,22 @@ __global__ void __launch_bounds__(kThreads, 1)
             const uint32_t lV = desc_lo(dV), lOnes = desc_lo(dOnes) + (aOnes >> 4);
             // STATE_ONLY alternates between two phi(K) tiles (the phi(Q) tile is unused there)
             const uint32_t lPK0 = desc_lo(dPhiMN) + (smem_u32(sPK) >> 4), lPK1 = desc_lo(dPhiMN) + (smem_u32(sPQ) >> 4);
-            for (int c = 0; c < nch && ok; ++c) {
+            for (int c = 0; c < ntot && ok; ++c) {      // c counts pre-chunks and own chunks here
                 const int s = c % NS;
-                const uint32_t ph = c & 1;
                 const uint32_t aVt = smem_u32(smem + C::offStage + s * C::kStageBytes) + 2 * C::kQKBytes;
-                const uint32_t lPK = (STATE_ONLY && (c & 1)) ? lPK1 : lPK0;
+                const uint32_t lPK = (alt(c) && (c & 1)) ? lPK1 : lPK0;
                 ok = mbar_wait(&bars[kFull0 + s], (c / NS) & 1, abort_flag);
-                if (ok) ok = mbar_wait(&bars[kPK], ph, abort_flag);
-                // the state group has read (or, before chunk 0, initialised) the state in TMEM
-                if (ok && (!STATE_ONLY || c == 0)) ok = mbar_wait(&bars[kSR], ph, abort_flag);
+                if (ok) ok = mbar_wait(pk_bar(c), g2_parity(c), abort_flag);
+                // the state group has read (or, before the first chunk, initialised) the state in TMEM:
+                // phase 0 of the barrier is the initialisation when there are pre-chunks (or in the
+                // state-only pass), and own chunk i is phase i (+1 after pre-chunks)
+                if (ok) {
+                    if (STATE_ONLY || c < npre) {
+                        if (c == 0) ok = mbar_wait(&bars[kSR], 0, abort_flag);
+                    } else {
+                        ok = mbar_wait(&bars[kSR], (uint32_t)(c - npre + (npre > 0 ? 1 : 0)) & 1u, abort_flag);
+                    }
+                }
                 if (!ok) break;
                 TRACE(1, c, 1);
                 tc_fence_after();
@@ -344,6 +383,9 @@ __global__ void __launch_bounds__(kThreads, 1)
                 }
                 mma_commit(g2_bar(c));
                 mma_commit(&bars[kEmpty0 + s]);
+                // every state update without a read-out in between is done (state-only pass: all of
+                // them; main pass: the pre-chunks)
+                if (c + 1 == (STATE_ONLY ? nch : npre)) mma_commit(&bars[kDone]);
                 TRACE(1, c, 2);
             }
         }
@@ -360,8 +402,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             const uint32_t lPQ = desc_lo(dPhiK) + (smem_u32(sPQ) >> 4), lSc = desc_lo(dPhiK) + (smem_u32(sSc) >> 4);
             // scores of chunk c: T[c & 1] (or the single T) = Q_c K_c^T
             auto issue_scores = [&](int c) -> bool {
-                const int s = c % NS;
-                if (!mbar_wait(&bars[kFull0 + s], (c / NS) & 1, abort_flag)) return false;
+                const int s = (c + npre) % NS;
+                if (!mbar_wait(&bars[kFull0 + s], ((c + npre) / NS) & 1, abort_flag)) return false;
                 TRACE(0, c, 0);
                 tc_fence_after();
                 const uint32_t aSt = smem_u32(smem + C::offStage + s * C::kStageBytes);
@@ -370,9 +412,14 @@ __global__ void __launch_bounds__(kThreads, 1)
                 mma_commit(&bars[kG1 + t_idx(c)]);
                 return true;
             };
-            if (nch > 0) ok = issue_scores(0);
+            // pre-chunks: nothing to issue, but the stage is released by two arrivals
+            for (int g = 0; g < npre && ok; ++g) {
+                ok = mbar_wait(&bars[kFull0 + g % NS], (g / NS) & 1, abort_flag);
+                if (ok) mbar_arrive(&bars[kEmpty0 + g % NS]);
+            }
+            if (nch > 0 && ok) ok = issue_scores(0);
             for (int c = 0; c < nch && ok; ++c) {
-                const int s = c % NS;
+                const int s = (c + npre) % NS;
                 const uint32_t ph = c & 1;
                 const uint32_t aVt = smem_u32(smem + C::offStage + s * C::kStageBytes) + 2 * C::kQKBytes;
                 const uint32_t colTc = C::colT + (C::kTDouble ? (c & 1) * 128 : 0);
@@ -473,7 +520,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                 }
                 if (t == 0) TRACE(5, c, 2);
             }
-            if (t == 0) tma_store_wait<0>();
+            // the staging tile must outlive the last store's read of it; the global writes complete on their own
+            if (t == 0) tma_store_wait_read<0>();
         }
     } else if (warp >= 8) {
         // ===================================================================== state group
@@ -490,7 +538,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const float* kvh = p.kv_abi ? p.kv_abi + (size_t)head * kD * DV : nullptr;
         const float* zh = p.z_abi ? p.z_abi + (size_t)head * kD : nullptr;
         const bool from_abi = !STATE_ONLY && p.continue_abi;
-        const int nprev = STATE_ONLY ? 0 : seg;
+        const int nprev = (STATE_ONLY || PRE) ? 0 : seg;
 
         // Initial value of this lane's row: the caller's ABI state (folded into the internal
         // basis) plus the partial states of the earlier segments.  Loads are issued 16 at a
@@ -548,17 +596,21 @@ __global__ void __launch_bounds__(kThreads, 1)
             tmem_st16(tmem_addr(tb, lane_base, C::colZ1), r1);
         }
         tmem_wait_st();
+        if (t == 0) TRACE(5, 2, 7);   // state initialised
 
         if (STATE_ONLY) {
             tc_fence_before();
             mbar_arrive(&bars[kSR]);
-            // a parity wait only tells the current phase from the one before, so follow the
-            // state-update barrier chunk by chunk
-            for (int c = 0; c < nch && ok; ++c) ok = mbar_wait(g2_bar(c), g2_parity(c), abort_flag);
+            if (nch > 0) ok = mbar_wait(&bars[kDone], 0, abort_flag);
         } else {
+            if (npre > 0) {
+                tc_fence_before();
+                mbar_arrive(&bars[kSR]);                                   // the state is initialised
+                ok = mbar_wait(&bars[kDone], 0, abort_flag);               // all pre-chunks are folded in
+            }
             for (int c = 0; c < nch && ok; ++c) {
                 if (c > 0) {
-                    ok = mbar_wait(&bars[kG2], (c - 1) & 1, abort_flag);   // state after chunk c-1 is final
+                    ok = mbar_wait(g2_bar(c + npre - 1), g2_parity(c + npre - 1), abort_flag);   // state after chunk c-1 is final
                     if (!ok) break;
                 }
                 if (t == 0) TRACE(4, c, 0);
@@ -609,10 +661,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                 mbar_arrive(&bars[kSC]);
                 if (t == 0) TRACE(4, c, 3);
             }
-            if (ok && nch > 0) ok = mbar_wait(&bars[kG2], (nch - 1) & 1, abort_flag);
+            if (ok && nch > 0) ok = mbar_wait(g2_bar(ntot - 1), g2_parity(ntot - 1), abort_flag);
         }
 
         // ---- final state
+        if (t == 0) TRACE(5, 3, 7);   // chunk loop done
         tc_fence_after();
         const bool write_ws = STATE_ONLY;
         const bool write_abi = !STATE_ONLY && p.kv_abi != nullptr && seg == p.nseg - 1;
@@ -655,31 +708,41 @@ __global__ void __launch_bounds__(kThreads, 1)
         // ===================================================================== feature group
         // One thread per token of the chunk: expands its k row (and q row) into feature rows.
         const int t = tid - 128;
-        for (int c = 0; c < nch && ok; ++c) {
-            const int s = c % NS;
+        for (int g = 0; g < ntot && ok; ++g) {
+            const int c = g - npre;                     // own chunk index (negative: pre-chunk)
+            const int s = g % NS;
             const uint8_t* st = smem + C::offStage + s * C::kStageBytes;
-            const bool valid = tok_begin + c * kC + t < tok_end;
-            ok = mbar_wait(&bars[kFull0 + s], (c / NS) & 1, abort_flag);
+            const bool valid = tok_first + g * kC + t < tok_end;
+            ok = mbar_wait(&bars[kFull0 + s], (g / NS) & 1, abort_flag);
             if (!ok) break;
             if (t == 0) TRACE(3, c, 0);
             uint4 klo, khi, qlo = make_uint4(0u, 0u, 0u, 0u), qhi = qlo;
             read_qk_row(st + C::kQKBytes, t, klo, khi);
-            if (!STATE_ONLY) read_qk_row(st, t, qlo, qhi);
-            // the tile being overwritten was last read by step (5) of chunk c-1 (c-2 in STATE_ONLY,
-            // which alternates between two tiles)
-            constexpr int kLag = STATE_ONLY ? 2 : 1;
-            if (c >= kLag) {
-                ok = mbar_wait(g2_bar(c - kLag), g2_parity(c - kLag), abort_flag);
-                if (!ok) break;
+            if (!STATE_ONLY && c >= 0) read_qk_row(st, t, qlo, qhi);
+            // the tile being overwritten was last read by step (5) of the chunk before (two chunks
+            // before where tiles alternate; own chunk 0 after pre-chunks: the last even pre-chunk)
+            {
+                int last = -1;
+                if (alt(g)) last = g - 2;
+                else if (c > 0) last = g - 1;
+                else if (npre > 0) last = (npre - 1) & ~1;
+                if (last >= 0) {
+                    ok = mbar_wait(g2_bar(last), g2_parity(last), abort_flag);
+                    if (!ok) break;
+                }
             }
             if (t == 0) TRACE(3, c, 1);
-            write_phi_row(klo, khi, (STATE_ONLY && (c & 1)) ? sPQ : sPK, t, valid);
+            write_phi_row(klo, khi, (alt(g) && (g & 1)) ? sPQ : sPK, t, valid);
             fence_proxy_async_smem();
-            mbar_arrive(&bars[kPK]);
+            mbar_arrive(pk_bar(g));
             if (t == 0) TRACE(3, c, 2);
-            if (!STATE_ONLY) {
+            if (!STATE_ONLY && c >= 0) {
                 if (c > 0) {
                     ok = mbar_wait(&bars[kG4], (c - 1) & 1, abort_flag);   // step (4) of chunk c-1 has read phi(Q)
+                    if (!ok) break;
+                } else if (npre > 1) {
+                    const int last = ((npre & 1) ? npre - 2 : npre - 1);   // last odd pre-chunk used this tile for phi(K)
+                    ok = mbar_wait(g2_bar(last), g2_parity(last), abort_flag);
                     if (!ok) break;
                 }
                 if (t == 0) TRACE(3, c, 3);
@@ -755,6 +818,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     __syncthreads();
     if (warp == kWarpMma) tmem_dealloc(tb, 512);
+    if (tid == 0) { TRACE(5, 1, 7); TRACE_CTA(1); }     // kernel exit
 }
 
 // --------------------------------------------------------------------------------- host side
@@ -795,7 +859,7 @@ unsigned long long* g_trace = nullptr;
 
 template <int DV>
 based_status launch_dv(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH, int L,
-                       int flags, float* ws, int nseg, cudaStream_t stream) {
+                       int flags, float* ws, const SegPlan plan, cudaStream_t stream) {
     using C = Cfg<DV>;
     CUtensorMap tq, tk, tv, to;
     if (!make_map(&tq, q, BH, L, kDFeat, kDFeat, CU_TENSOR_MAP_SWIZZLE_32B) ||
@@ -809,9 +873,10 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
     p.ws = ws;
     if (error_word_ptr(&p.err) != BASED_OK) return BASED_ERR_CUDA;
     p.L = L;
+    const int nseg = plan.nseg;
+    const bool recompute = plan.recompute;
     p.nseg = nseg;
-    const int nch = (L + kC - 1) / kC;
-    p.seg_len = ((nch + nseg - 1) / nseg) * kC;
+    p.seg_len = plan.per * kC;
     p.continue_abi = (flags & BASED_STATE_CONTINUE) ? 1 : 0;
 #ifdef BASED_TRACE
     p.trace = g_trace;
@@ -822,60 +887,108 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
         if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BASED_ERR_CUDA;
         std::lock_guard<std::mutex> lock(setup_mutex());
         if (!configured[dev]) {
-            if (cudaFuncSetAttribute(prefill_tc_kernel<DV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            if (cudaFuncSetAttribute(prefill_tc_kernel<DV, kModeMain>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)C::kSmemBytes) != cudaSuccess ||
-                cudaFuncSetAttribute(prefill_tc_kernel<DV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                cudaFuncSetAttribute(prefill_tc_kernel<DV, kModeState>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)C::kSmemBytes) != cudaSuccess ||
+                cudaFuncSetAttribute(prefill_tc_kernel<DV, kModePre>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)C::kSmemBytes) != cudaSuccess)
                 return BASED_ERR_CUDA;
             configured[dev] = true;
         }
     }
+    if (nseg > 1 && recompute) {
+        prefill_tc_kernel<DV, kModePre><<<dim3(nseg, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
+        note_launch();
+        return check_launch("prefill_tc_kernel<pre>");
+    }
     if (nseg > 1) {
-        prefill_tc_kernel<DV, true><<<dim3(nseg - 1, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
+        prefill_tc_kernel<DV, kModeState><<<dim3(nseg - 1, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
         note_launch();
         const based_status st = check_launch("prefill_tc_kernel<state>");
         if (st != BASED_OK) return st;
     }
-    prefill_tc_kernel<DV, false><<<dim3(nseg, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
+    prefill_tc_kernel<DV, kModeMain><<<dim3(nseg, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
     note_launch();
     return check_launch("prefill_tc_kernel");
 }
 
 }  // namespace
 
-// Number of sequence segments a head is split into so that about one CTA per SM is busy
-// (measured on B200: cfg 2, 64 heads x 16 chunks, runs 29 us unsplit against 35 us in two segments).
-int prefill_tc_segments(int BH, int L) {
+// How a head's sequence is cut into segments so that about one CTA per SM is busy.
+//  - one segment: the plain chunk loop;
+//  - state pass: a first launch computes every segment's own state into the workspace, the main
+//    launch starts each segment from the sum of the earlier ones (long sequences);
+//  - recompute: one launch, no workspace; a segment's CTA first runs the state update alone over
+//    all earlier chunks (short sequences, where a second launch and start-up cost more than that).
+// The choice compares modelled CTA times in thousands of cycles per chunk, measured on B200:
+// full chunk 3.3 (d_v 64) / 3.4 (d_v 128), state-update-only chunk 1.0 / 1.4, a second launch and
+// start-up about 14.  In recompute mode later segments do more redundant work, so the first
+// n - 1 segments get `per` chunks each and the last one the (shorter) rest, `per` chosen to
+// level the modelled times.
+static SegPlan prefill_tc_plan(int BH, int L, int d_v) {
     const int nch = (L + kC - 1) / kC;
-    int nseg = 148 / BH;
-#ifdef BASED_TRACE
-    if (const char* e = getenv("BASED_NSEG")) nseg = atoi(e);
-#endif
-    if (nseg > 8) nseg = 8;
-    // a split costs a second launch, a second start-up and the extra state pass: it pays only when
-    // every segment keeps at least 16 chunks
+    const float full = d_v == 64 ? 3.3f : 3.4f, upd = d_v == 64 ? 1.0f : 1.4f;
+    int nmax = 148 / BH;
+    if (nmax > 8) nmax = 8;
+    // state pass: a split pays only when every segment keeps at least 16 chunks
+    int nseg = nmax;
     if (nseg > nch / 16) nseg = nch / 16;
     if (nseg < 1) nseg = 1;
-    // every segment must own at least one chunk
-    while (nseg > 1 && ((nch + nseg - 1) / nseg) * (nseg - 1) >= nch) --nseg;
-    return nseg;
+    while (nseg > 1 && ((nch + nseg - 1) / nseg) * (nseg - 1) >= nch) --nseg;   // every segment owns a chunk
+    SegPlan best = {nseg, (nch + nseg - 1) / nseg, false};
+    float best_cost = nseg > 1 ? (float)best.per * (upd + full) + 14.f : (float)nch * full;
+    for (int n = 2; n <= nmax; ++n) {
+        for (int per = (nch + n - 1) / n; per * (n - 1) < nch; ++per) {
+            float cost = 0.f;
+            for (int j = 0; j < n; ++j) {
+                const int own = (j == n - 1) ? nch - per * (n - 1) : per;
+                const float c = (float)(j * per) * upd + (float)own * full;
+                if (c > cost) cost = c;
+            }
+            if (cost < 0.95f * best_cost) {
+                best = {n, per, true};
+                best_cost = cost;
+            }
+        }
+    }
+#ifdef BASED_TRACE
+    if (const char* e = getenv("BASED_NSEG")) {
+        const int v = atoi(e);                      // negative: recompute mode with that many segments
+        best.nseg = v < 0 ? -v : (v > 0 ? v : 1);
+        best.recompute = v < 0;
+        best.per = (nch + best.nseg - 1) / best.nseg;
+        if (const char* q = getenv("BASED_PER")) best.per = atoi(q);
+    }
+#endif
+    return best;
 }
 
 size_t prefill_tc_workspace_bytes(int BH, int L, int d_v) {
-    const int nseg = prefill_tc_segments(BH, L);
+    const SegPlan plan = prefill_tc_plan(BH, L, d_v);
+    const int nseg = plan.recompute ? 1 : plan.nseg;
     return nseg > 1 ? (size_t)BH * (nseg - 1) * seg_state_floats(d_v) * sizeof(float) : 0;
 }
 
 based_status launch_prefill_tc(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH,
                                int L, int d_v, int flags, void* workspace, cudaStream_t stream) {
-    const int nseg = prefill_tc_segments(BH, L);
+    const SegPlan plan = prefill_tc_plan(BH, L, d_v);
     float* ws = static_cast<float*>(workspace);
-    if (d_v == 64) return launch_dv<64>(q, k, v, out, kv, z, BH, L, flags, ws, nseg, stream);
-    return launch_dv<128>(q, k, v, out, kv, z, BH, L, flags, ws, nseg, stream);
+    if (d_v == 64) return launch_dv<64>(q, k, v, out, kv, z, BH, L, flags, ws, plan, stream);
+    return launch_dv<128>(q, k, v, out, kv, z, BH, L, flags, ws, plan, stream);
 }
 
 }  // namespace based
 
 #ifdef BASED_TRACE
+// out[0..127]: the per-warp wait records; out[128]: owner CTA; then both are cleared
+extern "C" void based_debug_read_waits(unsigned int* out) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(out, based::sm100::g_wait_dbg, sizeof(unsigned int) * 128);
+    cudaMemcpyFromSymbol(out + 128, based::sm100::g_wait_owner, sizeof(unsigned int));
+    unsigned int zero[129] = {};
+    cudaMemcpyToSymbol(based::sm100::g_wait_dbg, zero, sizeof(unsigned int) * 128);
+    cudaMemcpyToSymbol(based::sm100::g_wait_owner, zero, sizeof(unsigned int));
+}
 extern "C" void based_debug_set_trace(void* ptr) { based::g_trace = static_cast<unsigned long long*>(ptr); }
 #endif

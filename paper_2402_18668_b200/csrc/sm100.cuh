@@ -62,16 +62,36 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parit
 // (shared memory) short-circuits every later wait of the CTA once one wait has given
 // up, so the kernel drains to its exit instead of hanging.  Returns false on give-up.
 constexpr uint64_t kWaitLimitNs = 1500ull * 1000ull * 1000ull;
+#ifdef BASED_TRACE
+// debug builds: which barrier each warp of the first CTA that gives up was waiting on
+static __device__ unsigned int g_wait_owner;
+static __device__ unsigned int g_wait_dbg[32][4];
+static __device__ __noinline__ void record_wait(uint64_t* bar, uint32_t parity, uint32_t why) {
+    const unsigned cta = blockIdx.y * gridDim.x + blockIdx.x + 1;
+    const unsigned old = atomicCAS(&g_wait_owner, 0u, cta);
+    if (old == 0u || old == cta) {
+        unsigned int* d = g_wait_dbg[(threadIdx.x >> 5) & 31];
+        d[0] = smem_u32(bar); d[1] = parity; d[2] = threadIdx.x | (why << 16); d[3] = cta;
+    }
+}
+#define BASED_RECORD_WAIT(bar, parity, why) record_wait(bar, parity, why)
+#else
+#define BASED_RECORD_WAIT(bar, parity, why) do {} while (0)
+#endif
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
                                           uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t deadline = 0;
     for (;;) {
         if (mbar_try_wait_hint(bar, parity, 20000u)) return true;      // parked for up to 20 us per attempt
-        if (*abort_flag) return false;
+        if (*abort_flag) {
+            BASED_RECORD_WAIT(bar, parity, 2u);
+            return false;
+        }
         const uint64_t now = global_timer_ns();
         if (deadline == 0) deadline = now + limit_ns;
         else if (now > deadline) {
+            BASED_RECORD_WAIT(bar, parity, 1u);
             *abort_flag = 1;
             return false;
         }

@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 
 
 def test_static_scratch_matches_workspace_variant_twice():
-    B, H, L, d_v = 2, 4, 4200, 64                       # 8 heads x 33 chunks -> two segments per head
+    B, H, L, d_v = 2, 4, 16500, 64                      # 8 heads x 129 chunks -> 8 segments per head, state pass
     assert based.based_prefill_workspace_bytes(B, H, L, 16, d_v, based.BASED_BF16) > 0
     for seed in (21, 22):
         w = wl.Workload("noalloc", B, H, L, 16, d_v, "bf16", 0.25)
