@@ -48,6 +48,13 @@ def _load():
         lib.oracle_swa.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, ctypes.c_double]
         lib.oracle_linattn_quadratic_ld.argtypes = [_dp, _dp, _dp, _dp, i, i, i]
         lib.oracle_swa_decode_step.argtypes = [_dp, _dp, _dp, _dp, _dp, _dp, i, i, i, i, i, ctypes.c_double]
+        lib.oracle_feature_dim_sym.restype = i
+        lib.oracle_feature_dim_sym.argtypes = [i]
+        lib.oracle_psi.argtypes = [_dp, i, _dp]
+        lib.oracle_state_to_sym.argtypes = [_dp, _dp, ctypes.c_long, i, i]
+        lib.oracle_linattn_recurrent_sym.argtypes = [_dp, _dp, _dp, _dp, _dp, _dp, i, i, i, i, i]
+        for name in ("oracle_psi", "oracle_state_to_sym", "oracle_linattn_recurrent_sym"):
+            getattr(lib, name).restype = None
         for name in ("oracle_phi", "oracle_linattn_row", "oracle_linattn_quadratic", "oracle_linattn_recurrent",
                      "oracle_swa", "oracle_linattn_quadratic_ld", "oracle_swa_decode_step"):
             getattr(lib, name).restype = None
@@ -166,3 +173,48 @@ def swa_decode_step(q, k, v, k_cache, v_cache, pos: int, scale: float | None = N
     y = np.empty((B, H, d))
     _load().oracle_swa_decode_step(_p(q), _p(k), _p(v), _p(kc), _p(vc), _p(y), B, H, d, w, int(pos), float(scale))
     return y, kc, vc
+
+
+def feature_dim_sym(dp: int) -> int:
+    return int(_load().oracle_feature_dim_sym(dp))
+
+
+def psi(x) -> np.ndarray:
+    """Symmetric feature map of one vector x[dp] -> [1 + dp + dp(dp+1)/2]."""
+    x = _f64(x)
+    assert x.ndim == 1
+    out = np.empty(feature_dim_sym(x.shape[0]), dtype=np.float64)
+    _load().oracle_psi(_p(x), x.shape[0], _p(out))
+    return out
+
+
+def state_to_sym(S, z):
+    """Fold a full state S [B,H,D,dv], z [B,H,D] into the symmetric one (Ds rows)."""
+    S, z = _f64(S), _f64(z)
+    B, H, D, dv = S.shape
+    dp = int(round((-1 + np.sqrt(1 + 4 * (D - 1))) / 2))
+    assert feature_dim(dp) == D and z.shape == (B, H, D)
+    Ds = feature_dim_sym(dp)
+    Ss, zs = np.empty((B, H, Ds, dv)), np.empty((B, H, Ds))
+    _load().oracle_state_to_sym(_p(S), _p(Ss), B * H, dp, dv)
+    _load().oracle_state_to_sym(_p(z), _p(zs), B * H, dp, 1)
+    return Ss, zs
+
+
+def linattn_recurrent_sym(q, k, v, S0=None, z0=None):
+    """Recurrent form on the symmetric state. Returns y, S [B,H,Ds,dv], z [B,H,Ds] (new arrays)."""
+    q, k, v, B, H, L, dp, dv = _shapes(q, k, v)
+    D = feature_dim_sym(dp)
+    S = np.zeros((B, H, D, dv)) if S0 is None else _f64(S0).copy()
+    z = np.zeros((B, H, D)) if z0 is None else _f64(z0).copy()
+    assert S.shape == (B, H, D, dv) and z.shape == (B, H, D)
+    y = np.empty((B, H, L, dv))
+    _load().oracle_linattn_recurrent_sym(_p(q), _p(k), _p(v), _p(y), _p(S), _p(z), B, H, L, dp, dv)
+    return y, S, z
+
+
+def decode_step_sym(q, k, v, S, z):
+    """One recurrent step on the symmetric state: q,k [B,H,dp], v [B,H,dv]."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    y, S1, z1 = linattn_recurrent_sym(q[:, :, None, :], k[:, :, None, :], v[:, :, None, :], S, z)
+    return y[:, :, 0, :], S1, z1

@@ -27,6 +27,13 @@
  *                               cache update the paper's benchmark leaves out).
  *   oracle_linattn_quadratic_ld the quadratic form again with long double
  *                               accumulators (adequacy check of fp64 on tiny inputs).
+ *   oracle_psi, oracle_state_to_sym, oracle_linattn_recurrent_sym
+ *                               the same recurrences on the symmetric feature set whose size
+ *                               the appendix "Computing Recurrent State Size" counts,
+ *                               1 + 3d'/2 + d'^2/2 features: the product x_m x_n is kept once
+ *                               per unordered pair.  psi(q).psi(k) = phi(q).phi(k), so outputs
+ *                               are those of the full form; the symmetric state is the full
+ *                               state with each (m,n),(n,m) pair of rows folded into one.
  *
  * Parity pins: every function above is pinned by tests/test_oracle_*.py
  * (closed forms, special cases, library softmax attention, the Taylor remainder
@@ -37,6 +44,8 @@
  *   S    : [B, H, D, dv]      z    : [B, H, D]        D = 1 + dp + dp*dp
  * Feature order inside D: index 0 the constant, 1..dp the linear terms,
  * 1 + dp + m*dp + n the (m, n) product.
+ * Symmetric form: Ds = 1 + dp + dp(dp+1)/2; index 0 the constant, 1..dp the linear terms, then
+ * the pairs m <= n in row-major order of the upper triangle: (0,0), (0,1), ..., (0,dp-1), (1,1), ...
  */
 #include <math.h>
 #include <stddef.h>
@@ -253,5 +262,85 @@ void oracle_linattn_quadratic_ld(const double *q, const double *k, const double 
         }
         for (int c = 0; c < dv; ++c) y[(size_t)i * dv + c] = (double)(num[c] / (den + (long double)ORACLE_EPS));
         free(num);
+    }
+}
+
+/* ---- symmetric feature set (appendix "Computing Recurrent State Size") ------------------- */
+
+int oracle_feature_dim_sym(int dp) { return 1 + dp + dp * (dp + 1) / 2; }
+
+/*
+ * psi(x): constant and linear terms as in phi; one feature per unordered pair {m, n}:
+ * x_m^2 / (sqrt 2 sqrt d') on the diagonal and x_m x_n / sqrt d' off it (the two equal
+ * entries (m,n), (n,m) of phi, each x_m x_n / (sqrt 2 sqrt d'), merged into one of sqrt 2 times
+ * the size, which keeps the inner product).
+ */
+void oracle_psi(const double *x, int dp, double *out) {
+    const double rd = sqrt((double)dp);
+    const double rrd = sqrt(rd);
+    const double r2 = sqrt(2.0);
+    int at = 0;
+    out[at++] = 1.0;
+    for (int m = 0; m < dp; ++m) out[at++] = x[m] / rrd;
+    for (int m = 0; m < dp; ++m)
+        for (int n = m; n < dp; ++n) out[at++] = (m == n) ? (x[m] * x[m] / r2) / rd : (x[m] * x[n]) / rd;
+}
+
+/*
+ * Fold a full state (D rows) into the symmetric one (Ds rows): constant and linear rows are
+ * copied, the diagonal rows too, and rows (m,n), (n,m) become (row_mn + row_nm) / sqrt 2.
+ * `width` is dv for the KV-state and 1 for the K-state.
+ */
+void oracle_state_to_sym(const double *full, double *sym, long nheads, int dp, int width) {
+    const int D = oracle_feature_dim(dp), Ds = oracle_feature_dim_sym(dp);
+    const double r2 = sqrt(2.0);
+    for (long h = 0; h < nheads; ++h) {
+        const double *f = full + (size_t)h * D * width;
+        double *s = sym + (size_t)h * Ds * width;
+        for (int a = 0; a <= dp; ++a)
+            for (int c = 0; c < width; ++c) s[(size_t)a * width + c] = f[(size_t)a * width + c];
+        int at = 1 + dp;
+        for (int m = 0; m < dp; ++m)
+            for (int n = m; n < dp; ++n, ++at)
+                for (int c = 0; c < width; ++c) {
+                    const double a = f[(size_t)(1 + dp + m * dp + n) * width + c];
+                    const double b = f[(size_t)(1 + dp + n * dp + m) * width + c];
+                    s[(size_t)at * width + c] = (m == n) ? a : (a + b) / r2;
+                }
+    }
+}
+
+/* The recurrent form on the symmetric state: S [B,H,Ds,dv], z [B,H,Ds]; otherwise as above. */
+void oracle_linattn_recurrent_sym(const double *q, const double *k, const double *v, double *y, double *S,
+                                  double *z, int B, int H, int L, int dp, int dv) {
+    const int D = oracle_feature_dim_sym(dp);
+    const long nh = (long)B * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long bh = 0; bh < nh; ++bh) {
+        const double *qh = q + (size_t)bh * L * dp;
+        const double *kh = k + (size_t)bh * L * dp;
+        const double *vh = v + (size_t)bh * L * dv;
+        double *yh = y + (size_t)bh * L * dv;
+        double *Sh = S + (size_t)bh * D * dv;
+        double *zh = z + (size_t)bh * D;
+        double *f = (double *)malloc(sizeof(double) * (size_t)D);
+        double *g = (double *)malloc(sizeof(double) * (size_t)D);
+        for (int i = 0; i < L; ++i) {
+            oracle_psi(kh + (size_t)i * dp, dp, f);
+            for (int a = 0; a < D; ++a) {
+                zh[a] += f[a];
+                for (int c = 0; c < dv; ++c) Sh[(size_t)a * dv + c] += f[a] * vh[(size_t)i * dv + c];
+            }
+            oracle_psi(qh + (size_t)i * dp, dp, g);
+            double den = 0.0;
+            for (int a = 0; a < D; ++a) den += g[a] * zh[a];
+            for (int c = 0; c < dv; ++c) {
+                double num = 0.0;
+                for (int a = 0; a < D; ++a) num += g[a] * Sh[(size_t)a * dv + c];
+                yh[(size_t)i * dv + c] = num / (den + ORACLE_EPS);
+            }
+        }
+        free(f);
+        free(g);
     }
 }
