@@ -290,9 +290,10 @@ def bench_prefill_e2e(w, steps, warmup, torch, based, dist_on):
             "how": "pinned host q,k,v -> device, based_prefill, out -> pinned host, every step; 2 streams alternate"}
 
 
-def bench_decode(w, steps, warmup, torch, based, dist_on, peaks):
+def bench_decode(w, steps, warmup, torch, based, dist_on, peaks, sym=False):
     """cfg-4 style generation: `steps` sequential decode steps on a batch whose fp32 state
-    (B*H*273*d_v*4 bytes, larger than L2) comes from a prompt prefill."""
+    (B*H*273*d_v*4 bytes, larger than L2) comes from a prompt prefill.  sym: the state is folded
+    into the 153-row symmetric format after the prefill and the steps run on that."""
     g = torch.Generator(device="cuda").manual_seed(1)
     dt = w.torch_dtype
     Lp = w.L               # the whole prompt, as the configuration says (outside the timed region)
@@ -304,6 +305,14 @@ def bench_decode(w, steps, warmup, torch, based, dist_on, peaks):
     torch.cuda.synchronize()
     del q, k, v, o
     torch.cuda.empty_cache()
+    rows = 273
+    if sym:
+        kv_full, z_full = kv, z
+        kv, z = based.based_state_to_sym(kv_full, z_full)
+        torch.cuda.synchronize()
+        del kv_full, z_full
+        torch.cuda.empty_cache()
+        rows = based.D_SYM
     nbuf = 8
     qs = torch.randn(nbuf, w.B, w.H, w.d_feat, generator=g, device="cuda").to(dt)
     ks = torch.randn(nbuf, w.B, w.H, w.d_feat, generator=g, device="cuda").to(dt)
@@ -312,19 +321,23 @@ def bench_decode(w, steps, warmup, torch, based, dist_on, peaks):
 
     def step(i):
         j = i % nbuf
-        based.based_decode_step(qs[j], ks[j], vs[j], kv, z, out=out)
+        if sym:
+            based.based_decode_step_sym(qs[j], ks[j], vs[j], kv, z, out=out)
+        else:
+            based.based_decode_step(qs[j], ks[j], vs[j], kv, z, out=out)
 
     ms = time_region(step, steps, warmup, torch, dist_on)
     assert based.based_poll_error() == 0
     t = ms * 1e-3 / steps
-    state_bytes = 2.0 * w.B * w.H * 273 * w.d_v * 4
+    state_bytes = 2.0 * w.B * w.H * rows * w.d_v * 4
     esz = 2 if w.dtype == "bf16" else 4
-    all_bytes = state_bytes + w.B * w.H * (2 * 273 * 4 + esz * (2 * w.d_feat + 2 * w.d_v))
+    all_bytes = state_bytes + w.B * w.H * (2 * rows * 4 + esz * (2 * w.d_feat + 2 * w.d_v))
     return {
-        "workload": w.name, "metric": "decode_tokens_per_s", "value": w.B / t, "unit": "tokens/s",
-        "us_per_step": t * 1e6, "steps": steps,
+        "workload": w.name + (" (symmetric 153-row state)" if sym else ""), "metric": "decode_tokens_per_s",
+        "value": w.B / t, "unit": "tokens/s", "us_per_step": t * 1e6, "steps": steps, "state_rows": rows,
         "roofline": {"bound": "hbm", "achieved": state_bytes / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": state_bytes / t / 1e9 / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC.get(w.name),
+                     "frac": state_bytes / t / 1e9 / peaks["hbm_gbs"],
+                     "traffic": None if sym else NCU_TRAFFIC.get(w.name),
                      "kernel": "decode_step_kernel", "algorithmic_bytes": state_bytes,
                      "achieved_all_bytes": all_bytes / t / 1e9, "peak_source": peaks["source"]},
     }
@@ -414,7 +427,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_360m_prefill")
     ap.add_argument("--skip-extras", action="store_true", help="only the headline prefill workload")
-    ap.add_argument("--profile", choices=["prefill", "decode", "swa", "swa_decode"],
+    ap.add_argument("--profile", choices=["prefill", "decode", "decode_sym", "swa", "swa_decode"],
                     help="run only this arm on --shape (small cases for ncu captures) and print its result")
     ap.add_argument("--shape", default="", help="B,H,L,d_v for --profile (defaults to the arm's benchmark shape)")
     args = ap.parse_args()
@@ -462,15 +475,16 @@ def main():
     peaks = load_peaks()
 
     if args.profile:
-        base = {"prefill": w, "decode": wl.CONFIGS["cfg4_generation"], "swa": wl.CONFIGS["cfg5_mixer_pair"],
+        base = {"prefill": w, "decode": wl.CONFIGS["cfg4_generation"], "decode_sym": wl.CONFIGS["cfg4_generation"], "swa": wl.CONFIGS["cfg5_mixer_pair"],
                 "swa_decode": wl.CONFIGS["cfg4_generation"]}[args.profile]
         if args.shape:
             B, H, L, dv = (int(x) for x in args.shape.split(","))
             base = base.scaled(name=f"{base.name}[{args.shape}]", B=B, H=H, L=L, d_v=dv)
         if args.profile == "prefill":
             r, _, _ = bench_prefill(base, args.steps, args.warmup, torch, based, dist_on, peaks)
-        elif args.profile == "decode":
-            r = bench_decode(base, args.steps, args.warmup, torch, based, dist_on, peaks)
+        elif args.profile in ("decode", "decode_sym"):
+            r = bench_decode(base, args.steps, args.warmup, torch, based, dist_on, peaks,
+                             sym=args.profile == "decode_sym")
         elif args.profile == "swa_decode":
             r = bench_swa_decode(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         else:
@@ -505,6 +519,8 @@ def main():
                 torch.cuda.empty_cache()
         extras["prefill_configs"] = others
         extras["decode"] = bench_decode(wl.CONFIGS["cfg4_generation"], 1024, 16, torch, based, dist_on, peaks)
+        extras["decode_sym"] = bench_decode(wl.CONFIGS["cfg4_generation"], 1024, 16, torch, based, dist_on, peaks,
+                                            sym=True)
         torch.cuda.empty_cache()
         extras["swa_decode"] = bench_swa_decode(wl.CONFIGS["cfg4_generation"], 200, 10, torch, based, dist_on, peaks)
         extras["swa"] = bench_swa(wl.CONFIGS["cfg5_mixer_pair"], max(5, args.steps // 2), 3, torch, based, dist_on,

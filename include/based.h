@@ -92,6 +92,36 @@ based_status based_decode_step(const void* q, const void* k, const void* v, floa
                                void* cuda_stream);
 
 /*
+ * The same step on a symmetric state (opt-in format).  The outer product x (x) x has equal
+ * entries (m,n) and (n,m); keeping one feature per unordered pair leaves
+ * BASED_D_SYM = 1 + 3d'/2 + d'^2/2 = 153 rows (the feature count of the paper's appendix
+ * "Computing Recurrent State Size" and of its feature-map ablation table) instead of 273,
+ * with the same outputs and 44 % fewer state bytes read and written per step:
+ *
+ *   psi(x) = [1, x/2, {x_m^2 / (4 sqrt 2)} , {x_m x_n / 4 : m < n}]     psi(q).psi(k) = phi(q).phi(k)
+ *
+ * Row order: 0 the constant, 1..16 the linear terms, then the pairs m <= n in row-major order
+ * of the upper triangle ((0,0), (0,1), ..., (0,15), (1,1), ...).
+ * kv_sym [B,H,153,d_v] fp32 and z_sym [B,H,153] fp32 are updated IN PLACE; everything else as in
+ * based_decode_step.
+ */
+#define BASED_D_SYM 153
+based_status based_decode_step_sym(const void* q, const void* k, const void* v, float* kv_sym, float* z_sym,
+                                   void* out, int B, int H, int d_feat, int d_v, based_dtype io,
+                                   void* cuda_stream);
+
+/*
+ * Conversions between the 273-row state of based_prefill / based_decode_step and the symmetric
+ * one.  to_sym: row (m,n), m < n, = (S_mn + S_nm) / sqrt 2, the other rows are copied.
+ * from_sym: rows (m,n) and (n,m) = S_sym / sqrt 2 (exact inverse on states built by the
+ * recurrences, which are symmetric).  Input and output must not alias; all device pointers, fp32.
+ */
+based_status based_state_to_sym(const float* kv_state, const float* z_state, float* kv_sym, float* z_sym, int B,
+                                int H, int d_feat, int d_v, void* cuda_stream);
+based_status based_state_from_sym(const float* kv_sym, const float* z_sym, float* kv_state, float* z_state, int B,
+                                  int H, int d_feat, int d_v, void* cuda_stream);
+
+/*
  * Exact causal softmax attention in a sliding window (Eq. (1) of Sec. 2 restricted as
  * in Sec. 4.2: query i attends keys max(0, i-window+1) .. i):
  *

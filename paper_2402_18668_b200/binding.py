@@ -20,11 +20,13 @@ BASED_F32, BASED_BF16 = 0, 1
 BASED_STATE_ZERO_INIT, BASED_STATE_CONTINUE = 0, 1
 D_FEAT = 16
 D_EXPANDED = 1 + D_FEAT + D_FEAT * D_FEAT
+D_SYM = 1 + D_FEAT + D_FEAT * (D_FEAT + 1) // 2         # rows of the symmetric state format
 
 EXPORTS = (
     "based_prefill", "based_prefill_workspace_bytes", "based_decode_step", "swa_forward", "based_poll_error",
     "based_status_string", "based_version", "based_launch_count", "based_prefill_static_scratch",
-    "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step",
+    "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step", "based_decode_step_sym",
+    "based_state_to_sym", "based_state_from_sym",
 )
 
 _lib = None
@@ -57,6 +59,12 @@ def lib() -> ctypes.CDLL:
         L.based_selftest_bounded_wait.argtypes = [ctypes.c_uint, vp]
         L.based_decode_step.restype = i
         L.based_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+        L.based_decode_step_sym.restype = i
+        L.based_decode_step_sym.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+        L.based_state_to_sym.restype = i
+        L.based_state_to_sym.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
+        L.based_state_from_sym.restype = i
+        L.based_state_from_sym.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
         L.swa_forward.restype = i
         L.swa_forward.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
         L.swa_decode_step.restype = i
@@ -172,6 +180,47 @@ def based_decode_step(q, k, v, kv_state, z_state, out=None, stream=None):
     return out
 
 
+def based_decode_step_sym(q, k, v, kv_sym, z_sym, out=None, stream=None):
+    """q,k [B,H,16], v [B,H,d_v]; kv_sym [B,H,153,d_v], z_sym [B,H,153] (symmetric state) updated in place."""
+    _dev(q, k, v, kv_sym, z_sym, out)
+    B, H, d_feat = q.shape
+    d_v = v.shape[-1]
+    if kv_sym.dtype != torch.float32 or z_sym.dtype != torch.float32:
+        raise TypeError("state tensors are fp32")
+    if kv_sym.shape != (B, H, D_SYM, d_v) or z_sym.shape != (B, H, D_SYM):
+        raise ValueError("symmetric state has 153 rows")
+    if out is None:
+        out = torch.empty_like(v)
+    st = lib().based_decode_step_sym(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_sym), _ptr(z_sym), _ptr(out), B, H, d_feat,
+                                     d_v, _dtype_code(q), _stream(stream))
+    _check(st, "based_decode_step_sym")
+    return out
+
+
+def based_state_to_sym(kv_state, z_state, kv_sym=None, z_sym=None, stream=None):
+    """[B,H,273,d_v], [B,H,273] -> symmetric [B,H,153,d_v], [B,H,153]."""
+    _dev(kv_state, z_state, kv_sym, z_sym)
+    B, H, _, d_v = kv_state.shape
+    if kv_sym is None:
+        kv_sym, z_sym = new_state(B, H, d_v, device=kv_state.device, sym=True)
+    st = lib().based_state_to_sym(_ptr(kv_state), _ptr(z_state), _ptr(kv_sym), _ptr(z_sym), B, H, D_FEAT, d_v,
+                                  _stream(stream))
+    _check(st, "based_state_to_sym")
+    return kv_sym, z_sym
+
+
+def based_state_from_sym(kv_sym, z_sym, kv_state=None, z_state=None, stream=None):
+    """Symmetric [B,H,153,d_v], [B,H,153] -> [B,H,273,d_v], [B,H,273]."""
+    _dev(kv_sym, z_sym, kv_state, z_state)
+    B, H, _, d_v = kv_sym.shape
+    if kv_state is None:
+        kv_state, z_state = new_state(B, H, d_v, device=kv_sym.device)
+    st = lib().based_state_from_sym(_ptr(kv_sym), _ptr(z_sym), _ptr(kv_state), _ptr(z_state), B, H, D_FEAT, d_v,
+                                    _stream(stream))
+    _check(st, "based_state_from_sym")
+    return kv_state, z_state
+
+
 def swa_forward(q, k, v, out=None, window: int = 64, softmax_scale: float = 0.0, stream=None):
     """q,k,v [B,H,L,d] -> out; causal softmax over keys i-window+1..i; scale<=0 -> 1/sqrt(d)."""
     _dev(q, k, v, out)
@@ -208,7 +257,8 @@ def based_poll_error(stream=None) -> int:
     return int(lib().based_poll_error(_stream(stream)))
 
 
-def new_state(B: int, H: int, d_v: int, device="cuda"):
-    """Zero-initialised (kv_state, z_state) in the ABI layout."""
-    return (torch.zeros(B, H, D_EXPANDED, d_v, dtype=torch.float32, device=device),
-            torch.zeros(B, H, D_EXPANDED, dtype=torch.float32, device=device))
+def new_state(B: int, H: int, d_v: int, device="cuda", sym: bool = False):
+    """Zero-initialised (kv_state, z_state) in the ABI layout (273 rows, or the 153 symmetric ones)."""
+    D = D_SYM if sym else D_EXPANDED
+    return (torch.zeros(B, H, D, d_v, dtype=torch.float32, device=device),
+            torch.zeros(B, H, D, dtype=torch.float32, device=device))

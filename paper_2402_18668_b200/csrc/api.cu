@@ -108,7 +108,42 @@ based_status based_decode_step(const void* q, const void* k, const void* v, floa
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
         !aligned16(z_state))
         return BASED_ERR_ALIGNMENT;
-    return launch_decode(q, k, v, kv_state, z_state, out, B * H, d_v, io, static_cast<cudaStream_t>(cuda_stream));
+    return launch_decode(q, k, v, kv_state, z_state, out, B * H, d_v, io, false,
+                         static_cast<cudaStream_t>(cuda_stream));
+}
+
+based_status based_decode_step_sym(const void* q, const void* k, const void* v, float* kv_sym, float* z_sym,
+                                   void* out, int B, int H, int d_feat, int d_v, based_dtype io,
+                                   void* cuda_stream) {
+    if (!q || !k || !v || !out || !kv_sym || !z_sym || B <= 0 || H <= 0) return BASED_ERR_INVALID_ARG;
+    if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
+    if (d_feat != kDFeat || (d_v != 64 && d_v != 128)) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_sym) ||
+        !aligned16(z_sym))
+        return BASED_ERR_ALIGNMENT;
+    return launch_decode(q, k, v, kv_sym, z_sym, out, B * H, d_v, io, true, static_cast<cudaStream_t>(cuda_stream));
+}
+
+static based_status state_convert(const float* kv_in, const float* z_in, float* kv_out, float* z_out, int B, int H,
+                                  int d_feat, int d_v, bool to_sym, void* cuda_stream) {
+    if (!kv_in || !z_in || !kv_out || !z_out || B <= 0 || H <= 0) return BASED_ERR_INVALID_ARG;
+    if (kv_in == kv_out || z_in == z_out) return BASED_ERR_INVALID_ARG;
+    if (d_feat != kDFeat || (d_v != 64 && d_v != 128)) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
+    if (!aligned16(kv_in) || !aligned16(z_in) || !aligned16(kv_out) || !aligned16(z_out)) return BASED_ERR_ALIGNMENT;
+    return launch_state_convert(kv_in, z_in, kv_out, z_out, B * H, d_v, to_sym,
+                                static_cast<cudaStream_t>(cuda_stream));
+}
+
+based_status based_state_to_sym(const float* kv_state, const float* z_state, float* kv_sym, float* z_sym, int B,
+                                int H, int d_feat, int d_v, void* cuda_stream) {
+    return state_convert(kv_state, z_state, kv_sym, z_sym, B, H, d_feat, d_v, true, cuda_stream);
+}
+
+based_status based_state_from_sym(const float* kv_sym, const float* z_sym, float* kv_state, float* z_state, int B,
+                                  int H, int d_feat, int d_v, void* cuda_stream) {
+    return state_convert(kv_sym, z_sym, kv_state, z_state, B, H, d_feat, d_v, false, cuda_stream);
 }
 
 based_status swa_forward(const void* q, const void* k, const void* v, void* out, int B, int H, int L, int d,

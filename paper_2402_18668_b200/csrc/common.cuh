@@ -13,6 +13,7 @@ namespace based {
 
 constexpr int kDFeat = 16;                              // d' of the paper
 constexpr int kD = 1 + kDFeat + kDFeat * kDFeat;        // 273 expanded features
+constexpr int kDSym = 1 + kDFeat + kDFeat * (kDFeat + 1) / 2;   // 153 features, one per unordered pair
 constexpr float kEps = 1e-12f;                          // eps of the paper's listings
 // feature-map scales: x / d'^(1/4) and x_m x_n / (sqrt(2) sqrt(d')), d' = 16
 constexpr float kLinScale = 0.5f;
@@ -45,9 +46,32 @@ __device__ __forceinline__ float phi_at(const float* x, int f) {
     return x[p >> 4] * x[p & 15] * kQuadScale;
 }
 
+// Symmetric feature set: index 0 the constant, 1..16 the linear terms, then the pairs m <= n in
+// row-major order of the upper triangle.  pair_of(p) returns (m, n) of pair p in [0, 136).
+__host__ __device__ __forceinline__ void pair_of(int p, int& m, int& n) {
+    m = 0;
+    while (p >= kDFeat - m) {
+        p -= kDFeat - m;
+        ++m;
+    }
+    n = m + p;
+}
+// value of symmetric feature f (0..152): x_m^2 / (4 sqrt 2) on the diagonal, x_m x_n / 4 off it
+__device__ __forceinline__ float psi_at(const float* x, int f) {
+    if (f == 0) return 1.0f;
+    if (f <= kDFeat) return x[f - 1] * kLinScale;
+    int m, n;
+    pair_of(f - 1 - kDFeat, m, n);
+    return x[m] * x[n] * (m == n ? kQuadScale : 0.25f);
+}
+
 // kernel launchers (defined in the .cu files; all asynchronous on `stream`)
+// sym: the state has the 153 symmetric rows instead of the 273 full ones
 based_status launch_decode(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
-                           int BH, int d_v, based_dtype io, cudaStream_t stream);
+                           int BH, int d_v, based_dtype io, bool sym, cudaStream_t stream);
+// full (273-row) state -> symmetric (153-row) state, or back
+based_status launch_state_convert(const float* kv_in, const float* z_in, float* kv_out, float* z_out, int BH,
+                                  int d_v, bool to_sym, cudaStream_t stream);
 based_status launch_prefill_simt(const void* q, const void* k, const void* v, void* out, float* kv, float* z,
                                  int BH, int L, int d_v, based_dtype io, int flags, cudaStream_t stream);
 // bf16 tensor-core prefill (tcgen05); workspace holds partial states of sequence segments

@@ -19,14 +19,18 @@ namespace based {
 // STREAM: the state of all heads together is larger than L2, so every line is used exactly once
 // per step: load and store it with the evict-first (streaming) policy.  Measured on B200 at batch
 // 128 x 16 heads, d_v 128: 94.4 us per step against 96.9 us with the default policy.
-template <int DV, typename T, bool STREAM>
+// SYM: the state holds the 153 symmetric features (one per unordered pair, the feature count of the
+// appendix "Computing Recurrent State Size") instead of the 273 of the full outer product: the
+// same outputs from 44 % fewer state bytes per step.
+template <int DV, typename T, bool STREAM, bool SYM>
 __global__ void __launch_bounds__(256, 4) decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k,
                                                           const T* __restrict__ v, float* __restrict__ kv,
                                                           float* __restrict__ z, T* __restrict__ out) {
     constexpr int TPR = DV / 4;                    // threads per state row (one float4 each)
     constexpr int RPP = 256 / TPR;                 // rows per pass: 8 (d_v 128) or 16 (d_v 64)
-    constexpr int NPASS = (kD + RPP - 1) / RPP;    // 35 or 18
-    constexpr int UNROLL = (DV == 128) ? 7 : 6;    // 35 = 5*7, 18 = 3*6 loads in flight per thread
+    constexpr int ND = SYM ? kDSym : kD;           // state rows
+    constexpr int NPASS = (ND + RPP - 1) / RPP;    // full: 35 or 18; symmetric: 20 or 10
+    constexpr int UNROLL = SYM ? 5 : (DV == 128) ? 7 : 6;   // loads in flight per thread (35 = 5*7, 18 = 3*6, 20 = 4*5)
     static_assert(NPASS % UNROLL == 0, "pass count must divide");
     constexpr int DPAD = NPASS * RPP;
 
@@ -46,15 +50,15 @@ __global__ void __launch_bounds__(256, 4) decode_step_kernel(const T* __restrict
     for (int e = 0; e < 4; ++e) vv[e] = to_f32(v[head * DV + c4 * 4 + e]);
     __syncthreads();
     for (int f = tid; f < DPAD; f += 256) {
-        s_pq[f] = f < kD ? phi_at(s_x[0], f) : 0.f;
-        s_pk[f] = f < kD ? phi_at(s_x[1], f) : 0.f;
+        s_pq[f] = f < ND ? (SYM ? psi_at(s_x[0], f) : phi_at(s_x[0], f)) : 0.f;
+        s_pk[f] = f < ND ? (SYM ? psi_at(s_x[1], f) : phi_at(s_x[1], f)) : 0.f;
     }
     __syncthreads();
 
     // K-state update and denominator phi(q).z
     float dpart = 0.f;
-    float* zh = z + head * kD;
-    for (int f = tid; f < kD; f += 256) {
+    float* zh = z + head * ND;
+    for (int f = tid; f < ND; f += 256) {
         const float zn = zh[f] + s_pk[f];
         zh[f] = zn;
         dpart = fmaf(s_pq[f], zn, dpart);
@@ -64,19 +68,19 @@ __global__ void __launch_bounds__(256, 4) decode_step_kernel(const T* __restrict
     if ((tid & 31) == 0) s_den[tid >> 5] = dpart;
 
     // KV-state stream: S[r, :] += phi(k)[r] * v ; num += phi(q)[r] * S[r, :]
-    float4* S = reinterpret_cast<float4*>(kv + head * (size_t)kD * DV) + c4;
+    float4* S = reinterpret_cast<float4*>(kv + head * (size_t)ND * DV) + c4;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int p0 = 0; p0 < NPASS; p0 += UNROLL) {
         float4 s[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const int r = (p0 + u) * RPP + rslot;
-            if (r < kD) s[u] = STREAM ? __ldcs(&S[(size_t)r * TPR]) : S[(size_t)r * TPR];
+            if (r < ND) s[u] = STREAM ? __ldcs(&S[(size_t)r * TPR]) : S[(size_t)r * TPR];
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const int r = (p0 + u) * RPP + rslot;
-            if (r < kD) {
+            if (r < ND) {
                 const float pk = s_pk[r], pq = s_pq[r];
                 s[u].x = fmaf(pk, vv[0], s[u].x);
                 s[u].y = fmaf(pk, vv[1], s[u].y);
@@ -104,29 +108,95 @@ __global__ void __launch_bounds__(256, 4) decode_step_kernel(const T* __restrict
     }
 }
 
-template <int DV, typename T>
+template <int DV, typename T, bool SYM>
 static based_status launch_t(const void* q, const void* k, const void* v, float* kv, float* z, void* out, int BH,
                              cudaStream_t stream) {
     // 96 MB: safely above what L2 (126 MB, shared with everything else) keeps from one step to the next
-    const bool streaming = (size_t)BH * kD * DV * sizeof(float) > (size_t)96 << 20;
+    const bool streaming = (size_t)BH * (SYM ? kDSym : kD) * DV * sizeof(float) > (size_t)96 << 20;
     if (streaming)
-        decode_step_kernel<DV, T, true><<<BH, 256, 0, stream>>>(static_cast<const T*>(q), static_cast<const T*>(k),
-                                                                static_cast<const T*>(v), kv, z, static_cast<T*>(out));
+        decode_step_kernel<DV, T, true, SYM><<<BH, 256, 0, stream>>>(
+            static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), kv, z, static_cast<T*>(out));
     else
-        decode_step_kernel<DV, T, false><<<BH, 256, 0, stream>>>(static_cast<const T*>(q), static_cast<const T*>(k),
-                                                                 static_cast<const T*>(v), kv, z, static_cast<T*>(out));
+        decode_step_kernel<DV, T, false, SYM><<<BH, 256, 0, stream>>>(
+            static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), kv, z, static_cast<T*>(out));
     note_launch();
     return check_launch("decode_step_kernel");
 }
 
+template <int DV, bool SYM>
+static based_status launch_dv(const void* q, const void* k, const void* v, float* kv, float* z, void* out, int BH,
+                              based_dtype io, cudaStream_t stream) {
+    return io == BASED_F32 ? launch_t<DV, float, SYM>(q, k, v, kv, z, out, BH, stream)
+                           : launch_t<DV, __nv_bfloat16, SYM>(q, k, v, kv, z, out, BH, stream);
+}
+
 based_status launch_decode(const void* q, const void* k, const void* v, float* kv, float* z, void* out, int BH,
-                           int d_v, based_dtype io, cudaStream_t stream) {
-    if (d_v == 64) {
-        return io == BASED_F32 ? launch_t<64, float>(q, k, v, kv, z, out, BH, stream)
-                               : launch_t<64, __nv_bfloat16>(q, k, v, kv, z, out, BH, stream);
+                           int d_v, based_dtype io, bool sym, cudaStream_t stream) {
+    if (d_v == 64)
+        return sym ? launch_dv<64, true>(q, k, v, kv, z, out, BH, io, stream)
+                   : launch_dv<64, false>(q, k, v, kv, z, out, BH, io, stream);
+    return sym ? launch_dv<128, true>(q, k, v, kv, z, out, BH, io, stream)
+               : launch_dv<128, false>(q, k, v, kv, z, out, BH, io, stream);
+}
+
+// ------------------------------------------------------------------ full <-> symmetric state
+// One CTA per head.  to_sym: row (m,n), m < n, becomes (S_mn + S_nm) / sqrt 2, the other rows are
+// copied; from_sym: rows (m,n) and (n,m) both become S_sym / sqrt 2 (a full state that gives the
+// same outputs; a state built by the recurrences is symmetric, so this is its inverse).
+__global__ void __launch_bounds__(256) state_convert_kernel(const float* __restrict__ kv_in,
+                                                            const float* __restrict__ z_in,
+                                                            float* __restrict__ kv_out, float* __restrict__ z_out,
+                                                            int d_v, bool to_sym) {
+    constexpr float kRs2 = 0.70710678118654752f;
+    const size_t head = blockIdx.x;
+    const int nin = to_sym ? kD : kDSym, nout = to_sym ? kDSym : kD;
+    const float* kvi = kv_in + head * (size_t)nin * d_v;
+    const float* zi = z_in + head * (size_t)nin;
+    float* kvo = kv_out + head * (size_t)nout * d_v;
+    float* zo = z_out + head * (size_t)nout;
+    // source rows of output row r: (a, b >= 0 -> (a + b) scaled, b < 0 -> copy of a, scaled for from_sym pairs)
+    auto src = [&](int r, int& a, int& b, float& scale) {
+        b = -1;
+        scale = 1.f;
+        if (r <= kDFeat) { a = r; return; }
+        if (to_sym) {
+            int m, n;
+            pair_of(r - 1 - kDFeat, m, n);
+            a = 1 + kDFeat + m * kDFeat + n;
+            if (m != n) { b = 1 + kDFeat + n * kDFeat + m; scale = kRs2; }
+        } else {
+            const int p = r - 1 - kDFeat;
+            int m = p >> 4, n = p & 15;
+            if (m > n) { const int t = m; m = n; n = t; }
+            a = 1 + kDFeat + m * kDFeat - m * (m - 1) / 2 + (n - m);
+            if (m != n) scale = kRs2;
+        }
+    };
+    const int total = nout * d_v;
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        const int r = i / d_v, c = i - r * d_v;
+        int a, b;
+        float scale;
+        src(r, a, b, scale);
+        float x = kvi[(size_t)a * d_v + c];
+        if (b >= 0) x += kvi[(size_t)b * d_v + c];
+        kvo[i] = x * scale;
     }
-    return io == BASED_F32 ? launch_t<128, float>(q, k, v, kv, z, out, BH, stream)
-                           : launch_t<128, __nv_bfloat16>(q, k, v, kv, z, out, BH, stream);
+    for (int r = threadIdx.x; r < nout; r += blockDim.x) {
+        int a, b;
+        float scale;
+        src(r, a, b, scale);
+        float x = zi[a];
+        if (b >= 0) x += zi[b];
+        zo[r] = x * scale;
+    }
+}
+
+based_status launch_state_convert(const float* kv_in, const float* z_in, float* kv_out, float* z_out, int BH,
+                                  int d_v, bool to_sym, cudaStream_t stream) {
+    state_convert_kernel<<<BH, 256, 0, stream>>>(kv_in, z_in, kv_out, z_out, d_v, to_sym);
+    note_launch();
+    return check_launch("state_convert_kernel");
 }
 
 }  // namespace based

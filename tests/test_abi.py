@@ -90,6 +90,19 @@ def test_swa_decode_validation(lib):
     assert f(P, P, P, P, U, O, 1, 1, 64, 64, 0, 0.0, 1, None) == 3
 
 
+def test_sym_state_validation(lib):
+    d = lib.based_decode_step_sym
+    assert d(P, P, P, None, P, P, 1, 1, 16, 64, 0, None) == 1
+    assert d(P, P, P, P, P, P, 1, 1, 8, 64, 0, None) == 2                    # d' other than 16
+    assert d(P, P, P, P, U, P, 1, 1, 16, 64, 0, None) == 3
+    O = ctypes.c_void_p(0x2000)
+    for f in (lib.based_state_to_sym, lib.based_state_from_sym):
+        assert f(P, P, O, None, 1, 1, 16, 64, None) == 1
+        assert f(P, P, P, O, 1, 1, 16, 64, None) == 1                        # in and out alias
+        assert f(P, P, O, O, 1, 1, 16, 96, None) == 2
+        assert f(P, U, O, O, 1, 1, 16, 64, None) == 3
+
+
 def test_binding_rejects_cpu_tensors():
     import torch
     from paper_2402_18668_b200 import binding

@@ -155,6 +155,92 @@ def test_decode_chain_equals_prefill_on_gpu():
     assert head_err(_np(z), z_ref) <= TOL_F32 and head_err(_np(z2), z_ref) <= TOL_F32
 
 
+# --------------------------------------------------------------------------- symmetric state
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d_v", [64, 128])
+def test_decode_step_sym_from_folded_state(dtype, d_v):
+    """Steps on the 153-row state, starting from the fold of the state a 24-token prefix leaves."""
+    B, H = 3, 5
+    w = wl.Workload("decsym", B, H, 24, 16, d_v, dtype, 1.0, decode_steps=6)
+    gen = wl.generator(12)
+    qp, kp, vp = wl.prefill_inputs(w, gen)
+    qs, ks, vs = wl.decode_inputs(w, gen)
+    _, S0, z0 = oracle.linattn_recurrent_sym(_np(qp), _np(kp), _np(vp))
+    kv0, zz0 = torch.from_numpy(S0).float(), torch.from_numpy(z0).float()
+    kv, z = kv0.to(DEV), zz0.to(DEV)
+    S, zz = _np(kv0), _np(zz0)
+    assert kv.shape == (B, H, based.D_SYM, d_v)
+    tol = tol_for(dtype)
+    for t in range(w.decode_steps):
+        y_t, S, zz = oracle.decode_step_sym(_np(qs[t]), _np(ks[t]), _np(vs[t]), S, zz)
+        out = torch.full_like(vs[t], float("nan"), device=DEV)
+        based.based_decode_step_sym(qs[t].to(DEV), ks[t].to(DEV), vs[t].to(DEV), kv, z, out=out)
+        assert row_err(_np(out), y_t) <= tol, f"step {t}"
+        assert head_err(_np(kv), S) <= TOL_F32
+        assert head_err(_np(z), zz) <= TOL_F32
+    _poll()
+
+
+@pytest.mark.parametrize("d_v", [64, 128])
+def test_state_conversions_and_prefill_to_sym_decode(d_v):
+    """bf16 prefill -> fold on the GPU -> symmetric decode steps, against the oracle's definition
+    form over the whole sequence; the fold and its inverse against the oracle's fold."""
+    B, H, L, T = 2, 3, 300, 5
+    w = wl.Workload("p2s", B, H, L + T, 16, d_v, "bf16", 0.5)
+    q, k, v = wl.prefill_inputs(w, wl.generator(31))
+    y_ref, _, _ = oracle.linattn_quadratic(_np(q), _np(k), _np(v), return_state=False)
+    _, S_ref, z_ref = oracle.linattn_quadratic(_np(q[:, :, :L]), _np(k[:, :, :L]), _np(v[:, :, :L]))
+    Ss_ref, zs_ref = oracle.state_to_sym(S_ref, z_ref)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    kv, z = based.new_state(B, H, d_v)
+    based.based_prefill(qd[:, :, :L].contiguous(), kd[:, :, :L].contiguous(), vd[:, :, :L].contiguous(),
+                        kv_state=kv, z_state=z)
+    kvs, zs = based.based_state_to_sym(kv, z)
+    assert head_err(_np(kvs), Ss_ref) <= TOL_BF16 and head_err(_np(zs), zs_ref) <= TOL_BF16
+    # the fold itself is exact fp32 arithmetic on the GPU's own state
+    Ss_own, zs_own = oracle.state_to_sym(_np(kv), _np(z))
+    assert head_err(_np(kvs), Ss_own) <= 1e-6 and head_err(_np(zs), zs_own) <= 1e-6
+    # and back: the inverse reproduces the (symmetric) full state
+    kv_back, z_back = based.based_state_from_sym(kvs, zs)
+    assert head_err(_np(kv_back), _np(kv)) <= 1e-6 and head_err(_np(z_back), _np(z)) <= 1e-6
+    for t in range(L, L + T):
+        out = based.based_decode_step_sym(qd[:, :, t].contiguous(), kd[:, :, t].contiguous(),
+                                          vd[:, :, t].contiguous(), kvs, zs)
+        assert row_err(_np(out), y_ref[:, :, t]) <= TOL_BF16, f"token {t}"
+    _poll()
+
+
+def test_sym_and_full_decode_agree_at_generation_batch():
+    """Full-size batch (128 x 16 heads, d_v 128): one step of both formats from the same random
+    state; sampled heads against the oracle, all outputs against each other."""
+    w = wl.CONFIGS["cfg4_generation"]
+    B, H, d_v = w.B, w.H, w.d_v
+    g = torch.Generator(device=DEV).manual_seed(77)
+    tdt = torch.bfloat16
+    q = (torch.randn(B, H, 16, generator=g, device=DEV) * 0.5).to(tdt)
+    k = (torch.randn(B, H, 16, generator=g, device=DEV) * 0.5).to(tdt)
+    v = torch.randn(B, H, d_v, generator=g, device=DEV).to(tdt)
+    # a symmetric full state with a positive K-state, so the denominator is well away from zero
+    kvs = torch.randn(B, H, based.D_SYM, d_v, generator=g, device=DEV)
+    zs = torch.rand(B, H, based.D_SYM, generator=g, device=DEV) * 0.1
+    zs[:, :, 0] = 50.0
+    kv, z = based.based_state_from_sym(kvs, zs)
+    out_sym = based.based_decode_step_sym(q, k, v, kvs, zs)
+    out_full = based.based_decode_step(q, k, v, kv, z)
+    _poll()
+    assert row_err(_np(out_sym), _np(out_full)) <= TOL_BF16
+    kv_fold, z_fold = based.based_state_to_sym(kv, z)
+    assert head_err(_np(kv_fold), _np(kvs)) <= 1e-5 and head_err(_np(z_fold), _np(zs)) <= 1e-5
+    # sampled heads, one step recomputed by the oracle from the pre-step state (undo: S - psi(k) v^T)
+    for (b, h) in [(0, 0), (B - 1, H - 1), (63, 7)]:
+        f = oracle.psi(_np(k[b, h]))
+        S_before = _np(kvs[b, h]) - np.outer(f, _np(v[b, h]))
+        z_before = _np(zs[b, h]) - f
+        y, _, _ = oracle.decode_step_sym(_np(q[b:b + 1, h:h + 1]), _np(k[b:b + 1, h:h + 1]), _np(v[b:b + 1, h:h + 1]),
+                                         S_before[None, None], z_before[None, None])
+        assert row_err(_np(out_sym[b:b + 1, h:h + 1]), y) <= TOL_BF16
+
+
 # --------------------------------------------------------------------------- sliding window
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("L,window", [(1, 64), (63, 64), (64, 64), (333, 64), (200, 1), (257, 17), (400, 128), (130, 100)])
