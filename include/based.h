@@ -48,7 +48,9 @@ typedef enum { BASED_F32 = 0, BASED_BF16 = 1 } based_dtype;
 /* flags of based_prefill */
 enum {
     BASED_STATE_ZERO_INIT = 0, /* start from the empty state */
-    BASED_STATE_CONTINUE = 1   /* start from the state held in kv_state / z_state */
+    BASED_STATE_CONTINUE = 1,  /* start from the state held in kv_state / z_state */
+    BASED_STATE_SYM = 2        /* OR-ed in: kv_state / z_state use the 153-row symmetric format
+                                  described at based_decode_step_sym ([B,H,153,d_v], [B,H,153]) */
 };
 
 /*

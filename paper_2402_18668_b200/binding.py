@@ -17,7 +17,7 @@ LIB_PATH = _PKG / "libbased.so"
 
 BASED_OK = 0
 BASED_F32, BASED_BF16 = 0, 1
-BASED_STATE_ZERO_INIT, BASED_STATE_CONTINUE = 0, 1
+BASED_STATE_ZERO_INIT, BASED_STATE_CONTINUE, BASED_STATE_SYM = 0, 1, 2
 D_FEAT = 16
 D_EXPANDED = 1 + D_FEAT + D_FEAT * D_FEAT
 D_SYM = 1 + D_FEAT + D_FEAT * (D_FEAT + 1) // 2         # rows of the symmetric state format

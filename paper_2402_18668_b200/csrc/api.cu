@@ -80,9 +80,9 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
                            size_t workspace_bytes, void* cuda_stream) {
     if (!q || !k || !v || !out || B <= 0 || H <= 0 || L <= 0) return BASED_ERR_INVALID_ARG;
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
-    if (flags != BASED_STATE_ZERO_INIT && flags != BASED_STATE_CONTINUE) return BASED_ERR_INVALID_ARG;
+    if (flags & ~(BASED_STATE_CONTINUE | BASED_STATE_SYM)) return BASED_ERR_INVALID_ARG;
     if ((kv_state == nullptr) != (z_state == nullptr)) return BASED_ERR_INVALID_ARG;
-    if (flags == BASED_STATE_CONTINUE && !kv_state) return BASED_ERR_INVALID_ARG;
+    if ((flags & BASED_STATE_CONTINUE) && !kv_state) return BASED_ERR_INVALID_ARG;
     if (out == q || out == k || out == v) return BASED_ERR_INVALID_ARG;
     if (d_feat != kDFeat || (d_v != 64 && d_v != 128)) return BASED_ERR_UNSUPPORTED;
     if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;

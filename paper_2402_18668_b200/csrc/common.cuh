@@ -56,6 +56,10 @@ __host__ __device__ __forceinline__ void pair_of(int p, int& m, int& n) {
     }
     n = m + p;
 }
+// row of pair (m, n), m <= n, in the symmetric layout
+__host__ __device__ constexpr int sym_pair_row(int m, int n) {
+    return 1 + kDFeat + m * kDFeat - m * (m - 1) / 2 + (n - m);
+}
 // value of symmetric feature f (0..152): x_m^2 / (4 sqrt 2) on the diagonal, x_m x_n / 4 off it
 __device__ __forceinline__ float psi_at(const float* x, int f) {
     if (f == 0) return 1.0f;

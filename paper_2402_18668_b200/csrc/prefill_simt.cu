@@ -41,11 +41,30 @@ __global__ void __launch_bounds__(kGroups* DV + 32, 1)
     float S[kRowsPerGroup];
 #pragma unroll
     for (int j = 0; j < kRowsPerGroup; ++j) S[j] = 0.f;
+    // Symmetric state format: full row (m, n) lives in symmetric row (min, max), scaled by sqrt 2
+    // off the diagonal.  Rows (m, n) and (n, m) of the full state are bitwise equal here (same
+    // products, same order of accumulation), so the fold (S_mn + S_nm) / sqrt 2 is S_mn * sqrt 2.
+    const bool sym = (flags & BASED_STATE_SYM) != 0;
+    const int nrows = sym ? kDSym : kD;
+    auto sym_row = [](int p, float& scale, bool& owner) -> int {
+        scale = 1.f;
+        owner = true;
+        if (p <= kDFeat) return p;
+        const int m = (p - 1 - kDFeat) >> 4, n = (p - 1 - kDFeat) & 15;
+        owner = m <= n;
+        if (m != n) scale = 0.70710678118654752f;
+        return m <= n ? sym_pair_row(m, n) : sym_pair_row(n, m);
+    };
     if (active && (flags & BASED_STATE_CONTINUE)) {
 #pragma unroll
         for (int j = 0; j < kRowsPerGroup; ++j) {
             const int p = g * kRowsPerGroup + j;
-            if (p < kD) S[j] = ones ? z[head * kD + p] : kv[(head * kD + p) * DV + c];
+            if (p < kD) {
+                float scale = 1.f;
+                bool owner;
+                const int r = sym ? sym_row(p, scale, owner) : p;
+                S[j] = (ones ? z[head * nrows + r] : kv[(head * nrows + r) * DV + c]) * scale;
+            }
         }
     }
 
@@ -113,8 +132,13 @@ __global__ void __launch_bounds__(kGroups* DV + 32, 1)
         for (int j = 0; j < kRowsPerGroup; ++j) {
             const int p = g * kRowsPerGroup + j;
             if (p < kD) {
-                if (ones) z[head * kD + p] = S[j];
-                else kv[(head * kD + p) * DV + c] = S[j];
+                float scale = 1.f;
+                bool owner = true;
+                const int r = sym ? sym_row(p, scale, owner) : p;
+                if (!owner) continue;                       // the (n, m) twin writes the shared row
+                const float val = sym && scale != 1.f ? S[j] * 1.41421356237309505f : S[j];
+                if (ones) z[head * nrows + r] = val;
+                else kv[(head * nrows + r) * DV + c] = val;
             }
         }
     }

@@ -105,6 +105,7 @@ struct Params {
     int nseg;             // segments per head
     int seg_len;          // tokens per segment (multiple of kC)
     int continue_abi;     // start from the ABI state in kv_abi / z_abi
+    int sym;              // kv_abi / z_abi use the 153-row symmetric format
 #ifdef BASED_TRACE
     unsigned long long* trace;
 #endif
@@ -139,6 +140,19 @@ __host__ __device__ constexpr AbiRows abi_rows(int i) {
         const int m = i - 144, n = m + 8;
         return {17 + 16 * m + n, 17 + 16 * n + m};
     }
+    if (i == 152) return {0, -1};
+    return {-1, -1};
+}
+
+// ---- the same for the 153-row symmetric state format: the internal basis is that format's
+// feature set in another order, so every feature maps to one row with scale 1
+__host__ __device__ constexpr AbiRows sym_rows(int i) {
+    if (i < 16) return {1 + i, -1};
+    if (i < 144) {
+        const int o = (i - 16) / 16, m = (i - 16) % 16, n = (m + o) % 16;
+        return {m <= n ? sym_pair_row(m, n) : sym_pair_row(n, m), -1};
+    }
+    if (i < 152) return {sym_pair_row(i - 144, i - 144 + 8), -1};
     if (i == 152) return {0, -1};
     return {-1, -1};
 }
@@ -270,7 +284,11 @@ __global__ void __launch_bounds__(kThreads, 1)
         prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v); prefetch_tensormap(&tm_o);
     }
     if (warp == kWarpMma) { tmem_alloc(tmem_base_s, 512); tmem_relinquish(); }
-    if (tid < kF) { const AbiRows ar = abi_rows(tid); s_abi[tid] = make_short2((short)ar.a, (short)ar.b); }
+    if (tid < kF) {
+        const AbiRows ar = p.sym ? sym_rows(tid) : abi_rows(tid);
+        s_abi[tid] = make_short2((short)ar.a, (short)ar.b);
+    }
+    const int abi_nrows = p.sym ? kDSym : kD;
     // constant operand tiles and a zeroed state-copy tile (its rows past d_v + 1 stay zero for good)
     if (DV == 64) {
         for (uint32_t i = tid * 16; i < C::kOnesBytes; i += kThreads * 16) {
@@ -535,8 +553,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int z1f = (DV == 128 && (t & 31) < 16 && (t >> 5) < 2) ? 128 + (t >> 5) * 16 + (t & 15) : -1;
         const size_t seg_stride = seg_state_floats(DV);
         const float* wsh = p.ws + (size_t)head * (p.nseg > 1 ? p.nseg - 1 : 0) * seg_stride;
-        const float* kvh = p.kv_abi ? p.kv_abi + (size_t)head * kD * DV : nullptr;
-        const float* zh = p.z_abi ? p.z_abi + (size_t)head * kD : nullptr;
+        const float* kvh = p.kv_abi ? p.kv_abi + (size_t)head * abi_nrows * DV : nullptr;
+        const float* zh = p.z_abi ? p.z_abi + (size_t)head * abi_nrows : nullptr;
         const bool from_abi = !STATE_ONLY && p.continue_abi;
         const int nprev = (STATE_ONLY || PRE) ? 0 : seg;
 
@@ -671,8 +689,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         const bool write_abi = !STATE_ONLY && p.kv_abi != nullptr && seg == p.nseg - 1;
         if (ok && (write_ws || write_abi)) {
             float* wseg = p.ws + ((size_t)head * (p.nseg > 1 ? p.nseg - 1 : 0) + seg) * seg_stride;
-            float* kvo = write_abi ? p.kv_abi + (size_t)head * kD * DV : nullptr;
-            float* zo = write_abi ? p.z_abi + (size_t)head * kD : nullptr;
+            float* kvo = write_abi ? p.kv_abi + (size_t)head * abi_nrows * DV : nullptr;
+            float* zo = write_abi ? p.z_abi + (size_t)head * abi_nrows : nullptr;
             auto put = [&](int f, float v, bool zrow, int col) {
                 if (write_ws) {
                     if (zrow) wseg[(size_t)kF * DV + f] = v;
@@ -878,6 +896,7 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
     p.nseg = nseg;
     p.seg_len = plan.per * kC;
     p.continue_abi = (flags & BASED_STATE_CONTINUE) ? 1 : 0;
+    p.sym = (flags & BASED_STATE_SYM) ? 1 : 0;
 #ifdef BASED_TRACE
     p.trace = g_trace;
 #endif

@@ -210,6 +210,31 @@ def test_state_conversions_and_prefill_to_sym_decode(d_v):
     _poll()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("L,d_v", [(200, 64), (333, 128), (4200, 64)])
+def test_prefill_with_symmetric_state_in_and_out(dtype, L, d_v):
+    """BASED_STATE_SYM: the state leaves based_prefill in the 153-row format, and a second call
+    continues from it; both against the oracle's symmetric recurrence."""
+    B, H = 1, 2
+    w = wl.Workload("psym", B, H, L, 16, d_v, dtype, 0.5)
+    q, k, v = wl.prefill_inputs(w, wl.generator(L + d_v))
+    half = L // 2 + 3
+    y_ref, S_ref, z_ref = oracle.linattn_recurrent_sym(_np(q), _np(k), _np(v))
+    _, S_half, z_half = oracle.linattn_recurrent_sym(_np(q[:, :, :half]), _np(k[:, :, :half]), _np(v[:, :, :half]))
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    tol = tol_for(dtype)
+    kv, z = based.new_state(B, H, d_v, sym=True)
+    out1 = based.based_prefill(qd[:, :, :half].contiguous(), kd[:, :, :half].contiguous(), vd[:, :, :half].contiguous(),
+                               kv_state=kv, z_state=z, flags=based.BASED_STATE_SYM)
+    assert row_err(_np(out1), y_ref[:, :, :half]) <= tol
+    assert head_err(_np(kv), S_half) <= tol and head_err(_np(z), z_half) <= tol
+    out2 = based.based_prefill(qd[:, :, half:].contiguous(), kd[:, :, half:].contiguous(), vd[:, :, half:].contiguous(),
+                               kv_state=kv, z_state=z, flags=based.BASED_STATE_SYM | based.BASED_STATE_CONTINUE)
+    _poll()
+    assert row_err(_np(out2), y_ref[:, :, half:]) <= tol
+    assert head_err(_np(kv), S_ref) <= tol and head_err(_np(z), z_ref) <= tol
+
+
 def test_sym_and_full_decode_agree_at_generation_batch():
     """Full-size batch (128 x 16 heads, d_v 128): one step of both formats from the same random
     state; sampled heads against the oracle, all outputs against each other."""
