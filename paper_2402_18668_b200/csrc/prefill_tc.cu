@@ -90,7 +90,7 @@ struct Cfg {
 };
 
 enum Bar {
-    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kG1b, kP, kPb, kG2, kG2b, kG4, kG3, kYfree, kPK, kPKb, kPQ, kSR, kSC, kDone, kNumBars
+    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kG1b, kP, kPb, kG2, kG2b, kG4, kG3, kR4, kPK, kPKb, kSR, kDone, kNumBars
 };
 
 // segments per head, chunks per segment (the last one takes the rest), mode
@@ -166,9 +166,9 @@ __device__ __forceinline__ uint32_t mul2(uint32_t a, uint32_t b) {
     return *reinterpret_cast<uint32_t*>(&r);
 }
 
-// Expand one raw 16-vector (8 packed bf16 pairs) into its 160 internal features and write
-// them as row t of a [128 tokens][160 features] tile made of five SWIZZLE_64B blocks.
-__device__ __noinline__ void write_phi_row(uint4 xlo, uint4 xhi, uint8_t* tile, int t, bool valid) {
+// Expand one raw 16-vector (8 packed bf16 pairs) into its 160 internal features: 20 packed
+// 16-byte pieces f[0..19] (piece j = features 8j .. 8j+7).
+__device__ __forceinline__ void compute_phi_row(uint4 xlo, uint4 xhi, bool valid, uint4 (&f)[20]) {
     const uint32_t x[8] = {xlo.x, xlo.y, xlo.z, xlo.w, xhi.x, xhi.y, xhi.z, xhi.w};
     const uint32_t kHalf = 0x3F003F00u;      // (0.5, 0.5)
     const uint32_t kRs2 = 0x3F353F35u;       // (1/sqrt2, 1/sqrt2) rounded to bf16
@@ -177,19 +177,14 @@ __device__ __noinline__ void write_phi_row(uint4 xlo, uint4 xhi, uint8_t* tile, 
     for (int i = 0; i < 8; ++i) E[i] = valid ? mul2(x[i], kHalf) : 0u;
 #pragma unroll
     for (int i = 0; i < 8; ++i) O[i] = __byte_perm(E[i], E[(i + 1) & 7], 0x5432);   // (x'_{2i+1}, x'_{2i+2})
-    uint8_t* row = tile + (t >> 3) * 512 + (t & 7) * 64;
-    const uint32_t sw = (t >> 1) & 3;
-    auto store = [&](int j, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-        *reinterpret_cast<uint4*>(row + (j >> 2) * (kC * 64) + (((j & 3) ^ sw) << 4)) = make_uint4(a, b, c, d);
-    };
-    store(0, E[0], E[1], E[2], E[3]);
-    store(1, E[4], E[5], E[6], E[7]);
+    f[0] = make_uint4(E[0], E[1], E[2], E[3]);
+    f[1] = make_uint4(E[4], E[5], E[6], E[7]);
     {   // o = 0: squares, scaled by 1/sqrt 2
         uint32_t p[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) p[i] = mul2(E[i], mul2(E[i], kRs2));
-        store(2, p[0], p[1], p[2], p[3]);
-        store(3, p[4], p[5], p[6], p[7]);
+        f[2] = make_uint4(p[0], p[1], p[2], p[3]);
+        f[3] = make_uint4(p[4], p[5], p[6], p[7]);
     }
 #pragma unroll
     for (int o = 1; o < 8; ++o) {
@@ -199,11 +194,26 @@ __device__ __noinline__ void write_phi_row(uint4 xlo, uint4 xhi, uint8_t* tile, 
             const uint32_t r = (o & 1) ? O[(i + (o - 1) / 2) & 7] : E[(i + o / 2) & 7];
             p[i] = mul2(E[i], r);
         }
-        store(2 + 2 * o, p[0], p[1], p[2], p[3]);
-        store(3 + 2 * o, p[4], p[5], p[6], p[7]);
+        f[2 + 2 * o] = make_uint4(p[0], p[1], p[2], p[3]);
+        f[3 + 2 * o] = make_uint4(p[4], p[5], p[6], p[7]);
     }
-    store(18, mul2(E[0], E[4]), mul2(E[1], E[5]), mul2(E[2], E[6]), mul2(E[3], E[7]));
-    store(19, valid ? 0x00003F80u : 0u, 0u, 0u, 0u);   // the constant feature 1.0
+    f[18] = make_uint4(mul2(E[0], E[4]), mul2(E[1], E[5]), mul2(E[2], E[6]), mul2(E[3], E[7]));
+    f[19] = make_uint4(valid ? 0x00003F80u : 0u, 0u, 0u, 0u);   // the constant feature 1.0
+}
+
+// Write the 20 pieces as row t of a [128 tokens][160 features] tile made of five SWIZZLE_64B blocks.
+__device__ __forceinline__ void store_phi_row(const uint4 (&f)[20], uint8_t* tile, int t) {
+    uint8_t* row = tile + (t >> 3) * 512 + (t & 7) * 64;
+    const uint32_t sw = (t >> 1) & 3;
+#pragma unroll
+    for (int j = 0; j < 20; ++j)
+        *reinterpret_cast<uint4*>(row + (j >> 2) * (kC * 64) + (((j & 3) ^ sw) << 4)) = f[j];
+}
+
+__device__ __noinline__ void write_phi_row(uint4 xlo, uint4 xhi, uint8_t* tile, int t, bool valid) {
+    uint4 f[20];
+    compute_phi_row(xlo, xhi, valid, f);
+    store_phi_row(f, tile, t);
 }
 
 // Row t of a [128][16] bf16 tile written by TMA with SWIZZLE_32B.
@@ -277,8 +287,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         for (int s = 0; s < NS; ++s) { mbar_init(&bars[kFull0 + s], 1); mbar_init(&bars[kEmpty0 + s], STATE_ONLY ? 1 : 2); }
         mbar_init(&bars[kG1], 1); mbar_init(&bars[kG1b], 1); mbar_init(&bars[kPb], 128); mbar_init(&bars[kG2], 1); mbar_init(&bars[kG2b], 1); mbar_init(&bars[kG4], 1);
         mbar_init(&bars[kG3], 1);
-        mbar_init(&bars[kP], 128); mbar_init(&bars[kYfree], 128); mbar_init(&bars[kPK], 128); mbar_init(&bars[kPKb], 128); mbar_init(&bars[kDone], 1);
-        mbar_init(&bars[kPQ], 128); mbar_init(&bars[kSR], 128); mbar_init(&bars[kSC], 128);
+        mbar_init(&bars[kP], 128); mbar_init(&bars[kR4], 384); mbar_init(&bars[kPK], 128); mbar_init(&bars[kPKb], 128); mbar_init(&bars[kDone], 1);
+        mbar_init(&bars[kSR], 128);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v); prefetch_tensormap(&tm_o);
@@ -335,6 +345,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const int s = g % NS;
                 ok = mbar_wait(&bars[kEmpty0 + s], ((g / NS) & 1) ^ 1, abort_flag);
                 if (!ok) break;
+                TRACE(1, g, 3);
                 uint8_t* st = smem + C::offStage + s * C::kStageBytes;
                 const int tok0 = tok_first + g * kC;
                 const bool with_q = !STATE_ONLY && g >= npre;
@@ -443,13 +454,16 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const uint32_t colTc = C::colT + (C::kTDouble ? (c & 1) * 128 : 0);
                 // with two score buffers the next chunk's scores are issued ahead of this chunk's
                 // steps (4) and (3), so its polynomial overlaps them
+                TRACE(2, c, 3);
                 if (C::kTDouble && c + 1 < nch) {
                     ok = issue_scores(c + 1);
                     if (!ok) break;
                 }
-                ok = mbar_wait(&bars[kPQ], ph, abort_flag);
-                if (ok) ok = mbar_wait(&bars[kSC], ph, abort_flag);
-                if (ok && c > 0) ok = mbar_wait(&bars[kYfree], ph ^ 1, abort_flag);
+                TRACE(0, c, 1);
+                // step (4) of chunk c needs phi(Q) of chunk c (feature group), the state copy after chunk
+                // c-1 (state group) and the Y accumulator read out for chunk c-1 (output group, which
+                // arrives once before its first chunk): one barrier, three groups of 128 arrivals
+                ok = mbar_wait(&bars[kR4], ph, abort_flag);
                 if (!ok) break;
                 TRACE(0, c, 3);
                 tc_fence_after();
@@ -472,6 +486,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     for (int k = 0; k < kC / 16; ++k)
                         mma_ts_lh<true>(tb + C::colY, tb + colTc + k * 8, b_lo + k * (2048 >> 4), desc_hi(dV), i3);
                 }
+                TRACE(2, c, 2);
                 mma_commit(&bars[kG3]);
                 mma_commit(&bars[kEmpty0 + s]);
                 TRACE(0, c, 6);
@@ -487,6 +502,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             const int t = tid - 384;
             uint8_t* orow = sOut + (t >> 3) * 1024 + (t & 7) * 128;
             const uint32_t sw = t & 7;
+            if (nch > 0) mbar_arrive(&bars[kR4]);            // the Y accumulator starts out free
             for (int c = 0; c < nch && ok; ++c) {
                 ok = group_all(1, mbar_wait(&bars[kG3], c & 1, abort_flag));
                 if (!ok) break;
@@ -504,7 +520,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     tmem_wait_ld();
                     if (h == DV / 64 - 1) {            // all of Y is in registers: release the accumulator
                         tc_fence_before();
-                        mbar_arrive(&bars[kYfree]);
+                        mbar_arrive(&bars[kR4]);
                         if (t == 0) TRACE(5, c, 1);
                     }
                     // the staging tile is free once the previous TMA store has read it
@@ -676,7 +692,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                             __float2bfloat16_rn(__uint_as_float(z1));
                 }
                 fence_proxy_async_smem();
-                mbar_arrive(&bars[kSC]);
+                mbar_arrive(&bars[kR4]);
                 if (t == 0) TRACE(4, c, 3);
             }
             if (ok && nch > 0) ok = mbar_wait(g2_bar(ntot - 1), g2_parity(ntot - 1), abort_flag);
@@ -766,7 +782,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 if (t == 0) TRACE(3, c, 3);
                 write_phi_row(qlo, qhi, sPQ, t, true);
                 fence_proxy_async_smem();
-                mbar_arrive(&bars[kPQ]);
+                mbar_arrive(&bars[kR4]);
                 if (t == 0) TRACE(3, c, 4);
             }
         }
