@@ -37,6 +37,7 @@ NCU_TRAFFIC = {
     "cfg2_360m_prefill": 25.23e6,                 # profiles/prefill_tc_kernel_dv64_cfg2.md (output stays in L2)
     "cfg4_generation": 2 * (144.59e6 + 88.45e6),  # profiles/decode_step_kernel_dv128.md, 1024 -> 2048 heads
     "cfg5_mixer_pair:swa": 2 * (201.37e6 + 43.87e6),  # profiles/swa_tc_kernel.md, 16 -> 32 heads
+    "swa_decode": 34.36e6,                        # profiles/swa_decode_kernel.md (full size; writes stay in L2)
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -395,7 +396,8 @@ def bench_swa_decode(w, steps, warmup, torch, based, dist_on, peaks):
         "workload": f"B{w.B} H{w.H} window {win} d {d} {w.dtype}", "metric": "swa_decode_tokens_per_s",
         "value": w.B / t, "unit": "tokens/s", "us_per_step": t * 1e6, "steps": steps, "cache_sets": n,
         "roofline": {"bound": "hbm", "achieved": bytes_step / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": bytes_step / t / 1e9 / peaks["hbm_gbs"], "traffic": None, "kernel": "swa_decode_kernel",
+                     "frac": bytes_step / t / 1e9 / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC["swa_decode"],
+                     "kernel": "swa_decode_kernel",
                      "algorithmic_bytes": bytes_step, "peak_source": peaks["source"]},
     }
 
