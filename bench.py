@@ -402,6 +402,41 @@ def bench_swa_decode(w, steps, warmup, torch, based, dist_on, peaks):
     }
 
 
+def bench_generation_graph(w, steps, warmup, torch, based, dist_on, peaks):
+    """One generated token through the mixer pair at the generation configuration's batch: the
+    linear-attention decode step on the 153-row symmetric state plus the window-64 decode step on
+    its rolling cache, captured once as a CUDA graph (paper_2402_18668_b200.generation.DecodeGraph)
+    and replayed per token.  The state (321 MB) is larger than L2; the caches (34 MB) are not, as
+    in a real generation loop."""
+    from paper_2402_18668_b200.generation import DecodeGraph
+    g = torch.Generator(device="cuda").manual_seed(4)
+    dt = w.torch_dtype
+    win, d = 64, 64
+    kv = torch.randn(w.B, w.H, based.D_SYM, w.d_v, generator=g, device="cuda")
+    z = torch.rand(w.B, w.H, based.D_SYM, generator=g, device="cuda") + 1.0
+    kc = torch.randn(w.B, w.H, win, d, generator=g, device="cuda").to(dt)
+    vc = torch.randn(w.B, w.H, win, d, generator=g, device="cuda").to(dt)
+    graph = DecodeGraph(kv, z, kc, vc, pos=w.L, dtype=dt, sym=True)
+    for buf, scale in ((graph.q, 0.25), (graph.k, 0.25), (graph.v, 1.0), (graph.qw, 1.0), (graph.kw, 1.0),
+                       (graph.vw, 1.0)):
+        buf.copy_((torch.randn(buf.shape, generator=g, device="cuda") * scale).to(dt))
+
+    ms = time_region(lambda i: graph.replay(), steps, warmup, torch, dist_on)
+    assert based.based_poll_error() == 0
+    t = ms * 1e-3 / steps
+    esz = 2
+    bytes_step = 2.0 * w.B * w.H * based.D_SYM * w.d_v * 4 + 2.0 * w.B * w.H * win * d * esz
+    return {
+        "workload": f"B{w.B} H{w.H}: decode step on the 153-row state (d_v {w.d_v}) + window-{win} decode step, "
+                    "one CUDA graph per token",
+        "metric": "generation_tokens_per_s", "value": w.B / t, "unit": "tokens/s", "us_per_token_step": t * 1e6,
+        "steps": steps, "kernels_per_replay": 3,
+        "roofline": {"bound": "hbm", "achieved": bytes_step / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": bytes_step / t / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                     "algorithmic_bytes": bytes_step, "peak_source": peaks["source"]},
+    }
+
+
 def cpu_oracle_sample(w, budget_heads: int):
     """The oracle's recurrent form, as it stands, on the first `budget_heads` heads of the
     workload's seeded host inputs.  Returns (tokens/s scaled to whole tokens, cores, text)."""
@@ -429,7 +464,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_360m_prefill")
     ap.add_argument("--skip-extras", action="store_true", help="only the headline prefill workload")
-    ap.add_argument("--profile", choices=["prefill", "decode", "decode_sym", "swa", "swa_decode"],
+    ap.add_argument("--profile", choices=["prefill", "decode", "decode_sym", "swa", "swa_decode", "generation_graph"],
                     help="run only this arm on --shape (small cases for ncu captures) and print its result")
     ap.add_argument("--shape", default="", help="B,H,L,d_v for --profile (defaults to the arm's benchmark shape)")
     args = ap.parse_args()
@@ -478,7 +513,8 @@ def main():
 
     if args.profile:
         base = {"prefill": w, "decode": wl.CONFIGS["cfg4_generation"], "decode_sym": wl.CONFIGS["cfg4_generation"], "swa": wl.CONFIGS["cfg5_mixer_pair"],
-                "swa_decode": wl.CONFIGS["cfg4_generation"]}[args.profile]
+                "swa_decode": wl.CONFIGS["cfg4_generation"],
+                "generation_graph": wl.CONFIGS["cfg4_generation"]}[args.profile]
         if args.shape:
             B, H, L, dv = (int(x) for x in args.shape.split(","))
             base = base.scaled(name=f"{base.name}[{args.shape}]", B=B, H=H, L=L, d_v=dv)
@@ -489,6 +525,8 @@ def main():
                              sym=args.profile == "decode_sym")
         elif args.profile == "swa_decode":
             r = bench_swa_decode(base, args.steps, args.warmup, torch, based, dist_on, peaks)
+        elif args.profile == "generation_graph":
+            r = bench_generation_graph(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         else:
             r = bench_swa(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         if rank == 0:
@@ -524,6 +562,8 @@ def main():
         extras["decode_sym"] = bench_decode(wl.CONFIGS["cfg4_generation"], 1024, 16, torch, based, dist_on, peaks,
                                             sym=True)
         torch.cuda.empty_cache()
+        extras["generation_graph"] = bench_generation_graph(wl.CONFIGS["cfg4_generation"], 512, 16, torch, based,
+                                                            dist_on, peaks)
         extras["swa_decode"] = bench_swa_decode(wl.CONFIGS["cfg4_generation"], 200, 10, torch, based, dist_on, peaks)
         extras["swa"] = bench_swa(wl.CONFIGS["cfg5_mixer_pair"], max(5, args.steps // 2), 3, torch, based, dist_on,
                                   peaks)

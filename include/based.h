@@ -155,6 +155,24 @@ based_status swa_decode_step(const void* q, const void* k, const void* v, void* 
                              void* cuda_stream);
 
 /*
+ * Loads the kernels of the generation step (based_decode_step, based_decode_step_sym,
+ * swa_decode_step, swa_decode_step_at, the state conversions) into the current device's
+ * context and resolves the library's device symbols, so that their first use may happen inside
+ * a stream capture.  Launches nothing.
+ */
+based_status based_preload_decode(void);
+
+/*
+ * The same step with the position read from device memory (one int, >= 0) when the kernel runs,
+ * so that a launch captured into a CUDA graph (as the paper does for next-token prediction,
+ * Sec. 6 "Efficiency Benchmarks") can be replayed while the sequence grows: the caller advances
+ * *pos_device between replays, e.g. with a node of the same graph.
+ */
+based_status swa_decode_step_at(const void* q, const void* k, const void* v, void* k_cache, void* v_cache,
+                                void* out, int B, int H, int d, int window, const int* pos_device,
+                                float softmax_scale, based_dtype io, void* cuda_stream);
+
+/*
  * The same computation as based_prefill, for callers that cannot give the library scratch
  * memory.  (The paper has no counterpart: this is a deployment convenience.)  Some hosts
  * may not allocate device memory around a call at all - a serving process that has handed

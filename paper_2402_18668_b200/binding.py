@@ -26,7 +26,7 @@ EXPORTS = (
     "based_prefill", "based_prefill_workspace_bytes", "based_decode_step", "swa_forward", "based_poll_error",
     "based_status_string", "based_version", "based_launch_count", "based_prefill_static_scratch",
     "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step", "based_decode_step_sym",
-    "based_state_to_sym", "based_state_from_sym",
+    "based_state_to_sym", "based_state_from_sym", "swa_decode_step_at", "based_preload_decode",
 )
 
 _lib = None
@@ -69,6 +69,9 @@ def lib() -> ctypes.CDLL:
         L.swa_forward.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
         L.swa_decode_step.restype = i
         L.swa_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
+        L.swa_decode_step_at.restype = i
+        L.swa_decode_step_at.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, i, vp]
+        L.based_preload_decode.restype = i
         L.based_poll_error.restype = i
         L.based_poll_error.argtypes = [vp]
         L.based_status_string.restype = ctypes.c_char_p

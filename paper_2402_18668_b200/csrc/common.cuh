@@ -86,8 +86,13 @@ based_status launch_prefill_tc(const void* q, const void* k, const void* v, void
 bool swa_tc_supported(int window);
 based_status launch_swa_tc(const void* q, const void* k, const void* v, void* out, int BH, int L, int window,
                            float scale, cudaStream_t stream);
+// pos_dev != nullptr: the position is read from device memory by the kernel (pos is ignored)
 based_status launch_swa_decode(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
-                               int window, int pos, float scale, based_dtype io, cudaStream_t stream);
+                               int window, int pos, const int* pos_dev, float scale, based_dtype io,
+                               cudaStream_t stream);
+// load the generation-step kernels into the current context
+based_status preload_decode();
+based_status preload_swa_decode();
 based_status launch_swa_simt(const void* q, const void* k, const void* v, void* out, int BH, int L, int window,
                              float scale, based_dtype io, cudaStream_t stream);
 

@@ -192,6 +192,28 @@ __global__ void __launch_bounds__(256) state_convert_kernel(const float* __restr
     }
 }
 
+namespace {
+template <typename K>
+bool load_kernel(K kernel) {
+    cudaFuncAttributes attr;
+    return cudaFuncGetAttributes(&attr, kernel) == cudaSuccess;
+}
+template <int DV, typename T>
+bool load_decode_variants() {
+    return load_kernel(decode_step_kernel<DV, T, false, false>) && load_kernel(decode_step_kernel<DV, T, true, false>) &&
+           load_kernel(decode_step_kernel<DV, T, false, true>) && load_kernel(decode_step_kernel<DV, T, true, true>);
+}
+}  // namespace
+
+// Forces the decode kernels into the current context (first use inside a stream capture would
+// otherwise load them there).
+based_status preload_decode() {
+    const bool ok = load_decode_variants<64, float>() && load_decode_variants<64, __nv_bfloat16>() &&
+                    load_decode_variants<128, float>() && load_decode_variants<128, __nv_bfloat16>() &&
+                    load_kernel(state_convert_kernel);
+    return ok ? BASED_OK : BASED_ERR_CUDA;
+}
+
 based_status launch_state_convert(const float* kv_in, const float* z_in, float* kv_out, float* z_out, int BH,
                                   int d_v, bool to_sym, cudaStream_t stream) {
     state_convert_kernel<<<BH, 256, 0, stream>>>(kv_in, z_in, kv_out, z_out, d_v, to_sym);

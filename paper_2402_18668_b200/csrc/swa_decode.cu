@@ -79,8 +79,11 @@ size_t swa_decode_smem_bytes(int window) {
 template <typename T, int NPW>     // NPW >= ceil(window / (4 * kWarps)): passes of 4 rows per warp
 __global__ void __launch_bounds__(32 * kWarps)
 swa_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, T* __restrict__ kc,
-                  T* __restrict__ vc, T* __restrict__ out, int window, int pos, float scale,
-                  unsigned int* __restrict__ error_word) {
+                  T* __restrict__ vc, T* __restrict__ out, int window, int pos_arg,
+                  const int* __restrict__ pos_dev, float scale, unsigned int* __restrict__ error_word) {
+    // the position comes from device memory when the launch is part of a captured graph that is
+    // replayed as the sequence grows
+    const int pos = pos_dev ? *pos_dev : pos_arg;
     extern __shared__ __align__(128) unsigned char smem[];
     T* s_K = reinterpret_cast<T*>(smem);
     T* s_V = s_K + (size_t)window * kHD;
@@ -209,7 +212,8 @@ swa_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
 
 template <typename T, int NPW>
 static based_status launch_n(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
-                             int window, int pos, float scale, unsigned int* err, cudaStream_t stream) {
+                             int window, int pos, const int* pos_dev, float scale, unsigned int* err,
+                             cudaStream_t stream) {
     const size_t smem = swa_decode_smem_bytes<T>(window);
     if (smem > 48 * 1024) {
         if (cudaFuncSetAttribute(swa_decode_kernel<T, NPW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -219,25 +223,36 @@ static based_status launch_n(const void* q, const void* k, const void* v, void* 
     swa_decode_kernel<T, NPW><<<BH, 32 * kWarps, smem, stream>>>(static_cast<const T*>(q), static_cast<const T*>(k),
                                                           static_cast<const T*>(v), static_cast<T*>(kc),
                                                           static_cast<T*>(vc), static_cast<T*>(out), window, pos,
-                                                          scale, err);
+                                                          pos_dev, scale, err);
     note_launch();
     return check_launch("swa_decode_kernel");
 }
 
 template <typename T>
 static based_status launch_t(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
-                             int window, int pos, float scale, unsigned int* err, cudaStream_t stream) {
-    if (window <= 64) return launch_n<T, 4>(q, k, v, kc, vc, out, BH, window, pos, scale, err, stream);
-    return launch_n<T, 8>(q, k, v, kc, vc, out, BH, window, pos, scale, err, stream);
+                             int window, int pos, const int* pos_dev, float scale, unsigned int* err,
+                             cudaStream_t stream) {
+    if (window <= 64) return launch_n<T, 4>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, scale, err, stream);
+    return launch_n<T, 8>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, scale, err, stream);
+}
+
+based_status preload_swa_decode() {
+    cudaFuncAttributes attr;
+    const bool ok = cudaFuncGetAttributes(&attr, swa_decode_kernel<float, 4>) == cudaSuccess &&
+                    cudaFuncGetAttributes(&attr, swa_decode_kernel<float, 8>) == cudaSuccess &&
+                    cudaFuncGetAttributes(&attr, swa_decode_kernel<__nv_bfloat16, 4>) == cudaSuccess &&
+                    cudaFuncGetAttributes(&attr, swa_decode_kernel<__nv_bfloat16, 8>) == cudaSuccess;
+    return ok ? BASED_OK : BASED_ERR_CUDA;
 }
 
 based_status launch_swa_decode(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
-                               int window, int pos, float scale, based_dtype io, cudaStream_t stream) {
+                               int window, int pos, const int* pos_dev, float scale, based_dtype io,
+                               cudaStream_t stream) {
     unsigned int* err = nullptr;
     const based_status st = error_word_ptr(&err);
     if (st != BASED_OK) return st;
-    if (io == BASED_F32) return launch_t<float>(q, k, v, kc, vc, out, BH, window, pos, scale, err, stream);
-    return launch_t<__nv_bfloat16>(q, k, v, kc, vc, out, BH, window, pos, scale, err, stream);
+    if (io == BASED_F32) return launch_t<float>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, scale, err, stream);
+    return launch_t<__nv_bfloat16>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, scale, err, stream);
 }
 
 }  // namespace based

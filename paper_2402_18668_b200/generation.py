@@ -1,0 +1,80 @@
+"""Next-token step of the mixer pair as one replayable CUDA graph.
+
+The paper runs next-token prediction under CUDA graphs (Sec. 6, "Efficiency Benchmarks"): at
+batch sizes where a decode step lasts tens of microseconds the launch overhead of separate
+calls is a visible share of it.  `DecodeGraph` captures one step of both mixers, the Taylor
+linear-attention decode step (on the 273-row or the 153-row symmetric state) and the
+sliding-window decode step on its rolling cache, together with the increment of the position
+counter the latter reads from device memory, and replays it once per generated token.
+
+Only plumbing lives here (static buffers, stream capture); every arithmetic step runs in the
+library's kernels.
+"""
+from __future__ import annotations
+
+import ctypes
+
+import torch
+
+from . import binding as _b
+
+
+class DecodeGraph:
+    """One generation step of a linear-attention mixer and a sliding-window mixer.
+
+    q, k: [B,H,16]; v: [B,H,d_v] (linear attention).  qw, kw, vw: [B,H,64] (sliding window).
+    State and caches are owned by the caller and updated in place by every `step`.
+    """
+
+    def __init__(self, kv_state, z_state, k_cache, v_cache, pos: int, dtype=torch.bfloat16, sym: bool = False,
+                 softmax_scale: float = 0.0):
+        B, H, rows, d_v = kv_state.shape
+        if rows != (_b.D_SYM if sym else _b.D_EXPANDED):
+            raise ValueError("state rows do not match the format")
+        window, d = k_cache.shape[2], k_cache.shape[3]
+        dev = kv_state.device
+        self.sym, self.kv, self.z, self.kc, self.vc = sym, kv_state, z_state, k_cache, v_cache
+        self.q = torch.zeros(B, H, _b.D_FEAT, dtype=dtype, device=dev)
+        self.k = torch.zeros_like(self.q)
+        self.v = torch.zeros(B, H, d_v, dtype=dtype, device=dev)
+        self.qw = torch.zeros(B, H, d, dtype=dtype, device=dev)
+        self.kw = torch.zeros_like(self.qw)
+        self.vw = torch.zeros_like(self.qw)
+        self.out_lin = torch.empty_like(self.v)
+        self.out_swa = torch.empty_like(self.qw)
+        self.pos = torch.full((1,), int(pos), dtype=torch.int32, device=dev)
+        self._scale, self._window, self._d = float(softmax_scale), window, d
+        self._stream = torch.cuda.Stream(device=dev)
+        self._graph = torch.cuda.CUDAGraph()
+        # an eager warm-up pass would advance the state, so the kernels are loaded explicitly and
+        # the step is captured directly (the library allocates nothing: the calls only enqueue kernels)
+        _b._check(_b.lib().based_preload_decode(), "based_preload_decode")
+        self.pos.add_(0)                                   # loads torch's add kernel outside the capture
+        self._stream.wait_stream(torch.cuda.current_stream(dev))
+        with torch.cuda.stream(self._stream):
+            with torch.cuda.graph(self._graph, stream=self._stream):
+                self._enqueue()
+        torch.cuda.current_stream(dev).wait_stream(self._stream)
+
+    def _enqueue(self):
+        dec = _b.based_decode_step_sym if self.sym else _b.based_decode_step
+        dec(self.q, self.k, self.v, self.kv, self.z, out=self.out_lin)
+        B, H, d = self.qw.shape
+        st = _b.lib().swa_decode_step_at(_b._ptr(self.qw), _b._ptr(self.kw), _b._ptr(self.vw), _b._ptr(self.kc),
+                                         _b._ptr(self.vc), _b._ptr(self.out_swa), B, H, d, self._window,
+                                         ctypes.c_void_p(self.pos.data_ptr()), self._scale,
+                                         _b._dtype_code(self.qw), _b._stream())
+        _b._check(st, "swa_decode_step_at")
+        self.pos.add_(1)
+
+    def step(self, q, k, v, qw, kw, vw):
+        """Copies the token's inputs into the graph's buffers, replays it; returns the two outputs
+        (views of buffers that the next step overwrites)."""
+        self.q.copy_(q); self.k.copy_(k); self.v.copy_(v)
+        self.qw.copy_(qw); self.kw.copy_(kw); self.vw.copy_(vw)
+        self._graph.replay()
+        return self.out_lin, self.out_swa
+
+    def replay(self):
+        """Replays the step on whatever the input buffers hold (benchmarks)."""
+        self._graph.replay()

@@ -107,6 +107,14 @@ def test_sym_state_validation(lib):
         assert f(P, U, O, O, 1, 1, 16, 64, None) == 3
 
 
+def test_swa_decode_at_validation(lib):
+    f = lib.swa_decode_step_at
+    O = ctypes.c_void_p(0x2000)
+    assert f(P, P, P, P, P, O, 1, 1, 64, 64, None, 0.0, 1, None) == 1            # no position pointer
+    assert f(P, P, P, P, P, O, 1, 1, 64, 64, ctypes.c_void_p(0x3002), 0.0, 1, None) == 3
+    assert f(P, P, P, P, P, O, 1, 1, 48, 64, P, 0.0, 1, None) == 2
+
+
 def test_binding_rejects_cpu_tensors():
     import torch
     from paper_2402_18668_b200 import binding

@@ -155,6 +155,44 @@ def test_decode_chain_equals_prefill_on_gpu():
     assert head_err(_np(z), z_ref) <= TOL_F32 and head_err(_np(z2), z_ref) <= TOL_F32
 
 
+# --------------------------------------------------------------------------- graph-replayed generation step
+@pytest.mark.parametrize("sym", [False, True])
+def test_decode_graph_replays_match_oracle_chain(sym):
+    """The mixer pair's generation step captured once and replayed T times (position advanced on the
+    device): linear-attention outputs against the oracle's recurrence, sliding-window outputs against
+    the whole-sequence form, across the point where the ring cache wraps."""
+    from paper_2402_18668_b200.generation import DecodeGraph
+    B, H, d_v, win, T, L0 = 2, 3, 64, 16, 40, 5
+    g = wl.generator(404)
+    tdt = torch.bfloat16
+    def rnd(*shape, scale=1.0):
+        return (torch.randn(*shape, generator=g) * scale).to(tdt)
+    q, k, v = rnd(B, H, L0 + T, 16, scale=0.5), rnd(B, H, L0 + T, 16, scale=0.5), rnd(B, H, L0 + T, d_v)
+    qw, kw, vw = rnd(B, H, L0 + T, 64), rnd(B, H, L0 + T, 64), rnd(B, H, L0 + T, 64)
+    y_ref, _, _ = oracle.linattn_quadratic(_np(q), _np(k), _np(v), return_state=False)
+    w_ref = oracle.swa(_np(qw), _np(kw), _np(vw), win)
+    # prompt of L0 tokens: state by prefill, caches by L0 eager sliding-window steps
+    kv, z = based.new_state(B, H, d_v, sym=sym)
+    flags = based.BASED_STATE_SYM if sym else based.BASED_STATE_ZERO_INIT
+    based.based_prefill(q[:, :, :L0].contiguous().to(DEV), k[:, :, :L0].contiguous().to(DEV),
+                        v[:, :, :L0].contiguous().to(DEV), kv_state=kv, z_state=z, flags=flags)
+    kc = torch.full((B, H, win, 64), float("nan"), dtype=tdt, device=DEV)
+    vc = torch.full_like(kc, float("nan"))
+    for t in range(L0):
+        based.swa_decode_step(qw[:, :, t].contiguous().to(DEV), kw[:, :, t].contiguous().to(DEV),
+                              vw[:, :, t].contiguous().to(DEV), kc, vc, pos=t)
+    graph = DecodeGraph(kv, z, kc, vc, pos=L0, dtype=tdt, sym=sym)
+    n0 = based.launch_count()
+    for t in range(L0, L0 + T):
+        o_lin, o_swa = graph.step(q[:, :, t].to(DEV), k[:, :, t].to(DEV), v[:, :, t].to(DEV),
+                                  qw[:, :, t].to(DEV), kw[:, :, t].to(DEV), vw[:, :, t].to(DEV))
+        assert row_err(_np(o_lin), y_ref[:, :, t]) <= TOL_BF16, f"linear, token {t}"
+        assert row_err(_np(o_swa), w_ref[:, :, t]) <= TOL_BF16, f"window, token {t}"
+    _poll()
+    assert int(graph.pos.item()) == L0 + T
+    assert based.launch_count() == n0          # replays enqueue no new launches through the library
+
+
 # --------------------------------------------------------------------------- symmetric state
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d_v", [64, 128])
