@@ -55,6 +55,10 @@ def _load():
         lib.oracle_linattn_recurrent_sym.argtypes = [_dp, _dp, _dp, _dp, _dp, _dp, i, i, i, i, i]
         for name in ("oracle_psi", "oracle_state_to_sym", "oracle_linattn_recurrent_sym"):
             getattr(lib, name).restype = None
+        lib.oracle_baseconv_gate.argtypes = [_dp, _dp, _dp, _dp, _dp, i, i, i, i]
+        lib.oracle_baseconv_gate_step.argtypes = [_dp, _dp, _dp, _dp, _dp, _dp, i, i, i]
+        lib.oracle_baseconv_gate.restype = None
+        lib.oracle_baseconv_gate_step.restype = None
         for name in ("oracle_phi", "oracle_linattn_row", "oracle_linattn_quadratic", "oracle_linattn_recurrent",
                      "oracle_swa", "oracle_linattn_quadratic_ld", "oracle_swa_decode_step"):
             getattr(lib, name).restype = None
@@ -218,3 +222,26 @@ def decode_step_sym(q, k, v, S, z):
     q, k, v = _f64(q), _f64(k), _f64(v)
     y, S1, z1 = linattn_recurrent_sym(q[:, :, None, :], k[:, :, None, :], v[:, :, None, :], S, z)
     return y[:, :, 0, :], S1, z1
+
+
+def baseconv_gate(a, g, h, b2) -> np.ndarray:
+    """a, g [B,N,C]; h [w,C] (h[0] taps the current token); b2 [C] -> a * SiLU(causal_conv(h, g) + b2)."""
+    a, g, h, b2 = _f64(a), _f64(g), _f64(h), _f64(b2)
+    B, N, C = a.shape
+    w = h.shape[0]
+    assert g.shape == a.shape and h.shape == (w, C) and b2.shape == (C,)
+    out = np.empty_like(a)
+    _load().oracle_baseconv_gate(_p(a), _p(g), _p(h), _p(b2), _p(out), B, N, C, w)
+    return out
+
+
+def baseconv_gate_step(a, g, h, b2, state):
+    """One token: a, g [B,C]; state [B,w-1,C] (row j = g of the token j+1 steps back). Returns out, new state."""
+    a, g, h, b2 = _f64(a), _f64(g), _f64(h), _f64(b2)
+    st = _f64(state).copy()
+    B, C = a.shape
+    w = h.shape[0]
+    assert st.shape == (B, w - 1, C)
+    out = np.empty_like(a)
+    _load().oracle_baseconv_gate_step(_p(a), _p(g), _p(h), _p(b2), _p(st), _p(out), B, C, w)
+    return out, st

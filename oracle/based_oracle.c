@@ -35,6 +35,13 @@
  *                               are those of the full form; the symmetric state is the full
  *                               state with each (m,n),(n,m) pair of rows folded into one.
  *
+ *   oracle_baseconv_gate        the gated short convolution at the core of the BaseConv layer of
+ *                               App. "Extended Architecture Details" (paragraph "Convolution"):
+ *                               z = a (.) SiLU(h * g + b2), h * g a causal depthwise convolution
+ *                               of width w (the paper suggests 3); the three projections around
+ *                               it are plain matrix products and are not part of this function.
+ *   oracle_baseconv_gate_step   the same for one new token, from the last w-1 rows of g.
+ *
  * Parity pins: every function above is pinned by tests/test_oracle_*.py
  * (closed forms, special cases, library softmax attention, the Taylor remainder
  * bound, brute force in extended precision).  Nothing here is "parity unpinned".
@@ -342,5 +349,44 @@ void oracle_linattn_recurrent_sym(const double *q, const double *k, const double
         }
         free(f);
         free(g);
+    }
+}
+
+/* ---- gated short convolution of the BaseConv layer (App. "Extended Architecture Details") ---- */
+
+static double silu(double x) { return x / (1.0 + exp(-x)); }
+
+/*
+ * a, g, out: [B, N, C]; h: [w, C] (h[0] is the tap on the current token, h[j] on the token j
+ * steps back); b2: [C].  out[b,i,c] = a[b,i,c] * SiLU(sum_{j<w, j<=i} h[j,c] g[b,i-j,c] + b2[c]).
+ */
+void oracle_baseconv_gate(const double *a, const double *g, const double *h, const double *b2, double *out,
+                          int B, int N, int C, int w) {
+#pragma omp parallel for schedule(static)
+    for (long bi = 0; bi < (long)B * N; ++bi) {
+        const long b = bi / N, i = bi % N;
+        for (int c = 0; c < C; ++c) {
+            double acc = b2[c];
+            for (int j = 0; j < w && j <= i; ++j) acc += h[(size_t)j * C + c] * g[((size_t)b * N + (i - j)) * C + c];
+            out[(size_t)bi * C + c] = a[(size_t)bi * C + c] * silu(acc);
+        }
+    }
+}
+
+/*
+ * One token: a, g, out [B, C]; state [B, w-1, C] holds the previous rows of g, state[b,j] = g of
+ * the token j+1 steps back (zeros before the sequence start); it is shifted and g stored in slot 0.
+ */
+void oracle_baseconv_gate_step(const double *a, const double *g, const double *h, const double *b2, double *state,
+                               double *out, int B, int C, int w) {
+    for (int b = 0; b < B; ++b) {
+        double *st = state + (size_t)b * (w - 1) * C;
+        for (int c = 0; c < C; ++c) {
+            double acc = b2[c] + h[c] * g[(size_t)b * C + c];
+            for (int j = 1; j < w; ++j) acc += h[(size_t)j * C + c] * st[(size_t)(j - 1) * C + c];
+            out[(size_t)b * C + c] = a[(size_t)b * C + c] * silu(acc);
+            for (int j = w - 2; j >= 1; --j) st[(size_t)j * C + c] = st[(size_t)(j - 1) * C + c];
+            if (w > 1) st[c] = g[(size_t)b * C + c];
+        }
     }
 }
