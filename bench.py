@@ -37,6 +37,7 @@ NCU_TRAFFIC = {
     "cfg2_360m_prefill": 25.23e6,                 # profiles/prefill_tc_kernel_dv64_cfg2.md (output stays in L2)
     "cfg4_generation": 2 * (144.59e6 + 88.45e6),  # profiles/decode_step_kernel_dv128.md, 1024 -> 2048 heads
     "cfg5_mixer_pair:swa": 2 * (201.37e6 + 43.87e6),  # profiles/swa_tc_kernel.md, 16 -> 32 heads
+    "baseconv": 4 * (272.67e6 + 96.72e6),         # profiles/baseconv_gate_kernel.md, batch 2 -> 8 (part of the writes still in L2)
     "swa_decode": 34.36e6,                        # profiles/swa_decode_kernel.md (full size; writes stay in L2)
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -437,6 +438,35 @@ def bench_generation_graph(w, steps, warmup, torch, based, dist_on, peaks):
     }
 
 
+def bench_baseconv(shape, steps, warmup, torch, based, dist_on, peaks):
+    """Gated short convolution of a BaseConv layer (width 3, expansion 4): B x N tokens, C = 4 d
+    channels, bf16.  Three tensors of B*N*C elements cross HBM once per call (a, g in, out);
+    input sets rotate so that consecutive calls do not find their inputs in L2."""
+    B, N, C = shape
+    g_ = torch.Generator(device="cuda").manual_seed(6)
+    per_set = 3.0 * B * N * C * 2
+    n = n_sets_for(per_set)
+    sets = [(torch.randn(B, N, C, generator=g_, device="cuda").bfloat16(),
+             torch.randn(B, N, C, generator=g_, device="cuda").bfloat16(),
+             torch.empty(B, N, C, device="cuda", dtype=torch.bfloat16)) for _ in range(n)]
+    h = torch.randn(3, C, generator=g_, device="cuda") * 0.6
+    b2 = torch.randn(C, generator=g_, device="cuda") * 0.3
+
+    def step(i):
+        a, g, o = sets[i % n]
+        based.baseconv_gate_forward(a, g, h, b2, out=o)
+
+    ms = time_region(step, steps, warmup, torch, dist_on)
+    t = ms * 1e-3 / steps
+    return {
+        "workload": f"B{B} N{N} C{C} width 3 bf16", "metric": "baseconv_tokens_per_s", "value": B * N / t,
+        "unit": "tokens/s", "ms_per_step": t * 1e3, "steps": steps, "buffer_sets": n,
+        "roofline": {"bound": "hbm", "achieved": per_set / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": per_set / t / 1e9 / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC.get("baseconv"),
+                     "kernel": "baseconv_gate_kernel", "algorithmic_bytes": per_set, "peak_source": peaks["source"]},
+    }
+
+
 def cpu_oracle_sample(w, budget_heads: int):
     """The oracle's recurrent form, as it stands, on the first `budget_heads` heads of the
     workload's seeded host inputs.  Returns (tokens/s scaled to whole tokens, cores, text)."""
@@ -464,7 +494,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_360m_prefill")
     ap.add_argument("--skip-extras", action="store_true", help="only the headline prefill workload")
-    ap.add_argument("--profile", choices=["prefill", "decode", "decode_sym", "swa", "swa_decode", "generation_graph"],
+    ap.add_argument("--profile", choices=["prefill", "decode", "decode_sym", "swa", "swa_decode", "generation_graph", "baseconv"],
                     help="run only this arm on --shape (small cases for ncu captures) and print its result")
     ap.add_argument("--shape", default="", help="B,H,L,d_v for --profile (defaults to the arm's benchmark shape)")
     args = ap.parse_args()
@@ -514,8 +544,9 @@ def main():
     if args.profile:
         base = {"prefill": w, "decode": wl.CONFIGS["cfg4_generation"], "decode_sym": wl.CONFIGS["cfg4_generation"], "swa": wl.CONFIGS["cfg5_mixer_pair"],
                 "swa_decode": wl.CONFIGS["cfg4_generation"],
-                "generation_graph": wl.CONFIGS["cfg4_generation"]}[args.profile]
-        if args.shape:
+                "generation_graph": wl.CONFIGS["cfg4_generation"],
+                "baseconv": wl.CONFIGS["cfg3_1p3b_prefill"]}[args.profile]
+        if args.shape and args.profile != "baseconv":
             B, H, L, dv = (int(x) for x in args.shape.split(","))
             base = base.scaled(name=f"{base.name}[{args.shape}]", B=B, H=H, L=L, d_v=dv)
         if args.profile == "prefill":
@@ -525,6 +556,12 @@ def main():
                              sym=args.profile == "decode_sym")
         elif args.profile == "swa_decode":
             r = bench_swa_decode(base, args.steps, args.warmup, torch, based, dist_on, peaks)
+        elif args.profile == "baseconv":
+            shp = (8, 4096, 8192)
+            if args.shape:
+                B_, _, L_, C_ = (int(x) for x in args.shape.split(","))
+                shp = (B_, L_, C_)
+            r = bench_baseconv(shp, args.steps, args.warmup, torch, based, dist_on, peaks)
         elif args.profile == "generation_graph":
             r = bench_generation_graph(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         else:
@@ -562,6 +599,7 @@ def main():
         extras["decode_sym"] = bench_decode(wl.CONFIGS["cfg4_generation"], 1024, 16, torch, based, dist_on, peaks,
                                             sym=True)
         torch.cuda.empty_cache()
+        extras["baseconv"] = bench_baseconv((8, 4096, 8192), 10, 3, torch, based, dist_on, peaks)
         extras["generation_graph"] = bench_generation_graph(wl.CONFIGS["cfg4_generation"], 512, 16, torch, based,
                                                             dist_on, peaks)
         extras["swa_decode"] = bench_swa_decode(wl.CONFIGS["cfg4_generation"], 200, 10, torch, based, dist_on, peaks)

@@ -155,6 +155,31 @@ based_status swa_decode_step(const void* q, const void* k, const void* v, void* 
                              void* cuda_stream);
 
 /*
+ * The gated short convolution at the core of the BaseConv layer (App. "Extended Architecture
+ * Details", paragraph "Convolution": y = ((u W1 + b1) (.) SiLU(h * (u W2) + b2)) W3 + b3).
+ * The three projections are plain matrix products and stay with the caller; this call is the
+ * fused middle:
+ *
+ *   out[b,i,c] = a[b,i,c] * SiLU( sum_{j < width, j <= i} h[j,c] * g[b,i-j,c] + b2[c] )
+ *
+ * a = u W1 + b1, g = u W2, out: [B,N,C] in the io dtype; h [width,C] fp32, a causal depthwise
+ * filter whose row 0 is the tap on the current token; b2 [C] fp32.  SiLU(x) = x / (1 + exp(-x)).
+ * Supported: 1 <= width <= 4 (the paper uses 3); C a multiple of 8; io in {F32, BF16}.
+ * out may alias a; it must not alias g.
+ */
+based_status baseconv_gate_forward(const void* a, const void* g, const float* h, const float* b2, void* out, int B,
+                                   int N, int C, int width, based_dtype io, void* cuda_stream);
+
+/*
+ * The same for one new token per sequence (generation): a, g, out [B,C]; conv_state
+ * [B,width-1,C] in the io dtype holds the previous rows of g (row j = the token j+1 steps back,
+ * zeros before the sequence start) and is updated IN PLACE (shifted, g stored in row 0).
+ * conv_state may be NULL when width = 1.
+ */
+based_status baseconv_gate_step(const void* a, const void* g, const float* h, const float* b2, void* conv_state,
+                                void* out, int B, int C, int width, based_dtype io, void* cuda_stream);
+
+/*
  * Loads the kernels of the generation step (based_decode_step, based_decode_step_sym,
  * swa_decode_step, swa_decode_step_at, the state conversions) into the current device's
  * context and resolves the library's device symbols, so that their first use may happen inside

@@ -27,6 +27,7 @@ EXPORTS = (
     "based_status_string", "based_version", "based_launch_count", "based_prefill_static_scratch",
     "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step", "based_decode_step_sym",
     "based_state_to_sym", "based_state_from_sym", "swa_decode_step_at", "based_preload_decode",
+    "baseconv_gate_forward", "baseconv_gate_step",
 )
 
 _lib = None
@@ -72,6 +73,10 @@ def lib() -> ctypes.CDLL:
         L.swa_decode_step_at.restype = i
         L.swa_decode_step_at.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, i, vp]
         L.based_preload_decode.restype = i
+        L.baseconv_gate_forward.restype = i
+        L.baseconv_gate_forward.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+        L.baseconv_gate_step.restype = i
+        L.baseconv_gate_step.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp]
         L.based_poll_error.restype = i
         L.based_poll_error.argtypes = [vp]
         L.based_status_string.restype = ctypes.c_char_p
@@ -222,6 +227,38 @@ def based_state_from_sym(kv_sym, z_sym, kv_state=None, z_state=None, stream=None
                                     _stream(stream))
     _check(st, "based_state_from_sym")
     return kv_state, z_state
+
+
+def baseconv_gate_forward(a, g, h, b2, out=None, stream=None):
+    """a, g [B,N,C] (io dtype); h [width,C] fp32 (row 0 taps the current token); b2 [C] fp32
+    -> a * SiLU(causal depthwise conv(h, g) + b2)."""
+    _dev(a, g, h, b2, out)
+    B, N, C = a.shape
+    if g.shape != a.shape or g.dtype != a.dtype or h.dtype != torch.float32 or b2.dtype != torch.float32:
+        raise ValueError("a, g disagree or the filter/bias are not fp32")
+    if h.shape[1] != C or b2.shape != (C,):
+        raise ValueError("filter/bias shapes disagree with C")
+    if out is None:
+        out = torch.empty_like(a)
+    st = lib().baseconv_gate_forward(_ptr(a), _ptr(g), _ptr(h), _ptr(b2), _ptr(out), B, N, C, h.shape[0],
+                                     _dtype_code(a), _stream(stream))
+    _check(st, "baseconv_gate_forward")
+    return out
+
+
+def baseconv_gate_step(a, g, h, b2, conv_state, out=None, stream=None):
+    """One token: a, g [B,C]; conv_state [B,width-1,C] (io dtype) updated in place."""
+    _dev(a, g, h, b2, conv_state, out)
+    B, C = a.shape
+    width = h.shape[0]
+    if conv_state is not None and (conv_state.shape != (B, width - 1, C) or conv_state.dtype != a.dtype):
+        raise ValueError("conv_state must be [B, width-1, C] in the io dtype")
+    if out is None:
+        out = torch.empty_like(a)
+    st = lib().baseconv_gate_step(_ptr(a), _ptr(g), _ptr(h), _ptr(b2), _ptr(conv_state), _ptr(out), B, C, width,
+                                  _dtype_code(a), _stream(stream))
+    _check(st, "baseconv_gate_step")
+    return out
 
 
 def swa_forward(q, k, v, out=None, window: int = 64, softmax_scale: float = 0.0, stream=None):

@@ -192,6 +192,34 @@ based_status swa_decode_step_at(const void* q, const void* k, const void* v, voi
                              static_cast<cudaStream_t>(cuda_stream));
 }
 
+static based_status baseconv_check(const void* a, const void* g, const float* h, const float* b2, const void* out,
+                                   int B, int N, int C, int width, based_dtype io) {
+    if (!a || !g || !h || !b2 || !out || B <= 0 || N <= 0 || C <= 0 || width <= 0) return BASED_ERR_INVALID_ARG;
+    if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
+    if (out == g) return BASED_ERR_INVALID_ARG;
+    if (width > 4 || C % 8 != 0 || B > 65535 || (N + 63) / 64 > 65535) return BASED_ERR_UNSUPPORTED;
+    if (!aligned16(a) || !aligned16(g) || !aligned16(h) || !aligned16(b2) || !aligned16(out)) return BASED_ERR_ALIGNMENT;
+    return BASED_OK;
+}
+
+based_status baseconv_gate_forward(const void* a, const void* g, const float* h, const float* b2, void* out, int B,
+                                   int N, int C, int width, based_dtype io, void* cuda_stream) {
+    const based_status st = baseconv_check(a, g, h, b2, out, B, N, C, width, io);
+    if (st != BASED_OK) return st;
+    return launch_baseconv(a, g, h, b2, nullptr, out, B, N, C, width, false, io,
+                           static_cast<cudaStream_t>(cuda_stream));
+}
+
+based_status baseconv_gate_step(const void* a, const void* g, const float* h, const float* b2, void* conv_state,
+                                void* out, int B, int C, int width, based_dtype io, void* cuda_stream) {
+    const based_status st = baseconv_check(a, g, h, b2, out, B, 1, C, width, io);
+    if (st != BASED_OK) return st;
+    if (width > 1 && !conv_state) return BASED_ERR_INVALID_ARG;
+    if (!aligned16(conv_state)) return BASED_ERR_ALIGNMENT;
+    return launch_baseconv(a, g, h, b2, conv_state, out, B, 1, C, width, true, io,
+                           static_cast<cudaStream_t>(cuda_stream));
+}
+
 based_status based_preload_decode(void) {
     unsigned int* err = nullptr;
     based_status st = error_word_ptr(&err);

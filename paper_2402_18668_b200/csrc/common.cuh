@@ -90,6 +90,9 @@ based_status launch_swa_tc(const void* q, const void* k, const void* v, void* ou
 based_status launch_swa_decode(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
                                int window, int pos, const int* pos_dev, float scale, based_dtype io,
                                cudaStream_t stream);
+// gated short convolution (BaseConv core); step: one token on a [B, width-1, C] state, N ignored
+based_status launch_baseconv(const void* a, const void* g, const float* h, const float* b2, void* state, void* out,
+                             int B, int N, int C, int width, bool step, based_dtype io, cudaStream_t stream);
 // load the generation-step kernels into the current context
 based_status preload_decode();
 based_status preload_swa_decode();

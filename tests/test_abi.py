@@ -22,7 +22,7 @@ def _declared_functions():
     text = (ROOT / "include" / "based.h").read_text()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     names = re.findall(r"\b([a-z_0-9]+)\s*\(", text)
-    return sorted({n for n in names if n.startswith(("based_", "swa_"))})
+    return sorted({n for n in names if n.startswith(("based_", "swa_", "baseconv_"))})
 
 
 def test_every_declared_symbol_is_exported(lib):
@@ -113,6 +113,19 @@ def test_swa_decode_at_validation(lib):
     assert f(P, P, P, P, P, O, 1, 1, 64, 64, None, 0.0, 1, None) == 1            # no position pointer
     assert f(P, P, P, P, P, O, 1, 1, 64, 64, ctypes.c_void_p(0x3002), 0.0, 1, None) == 3
     assert f(P, P, P, P, P, O, 1, 1, 48, 64, P, 0.0, 1, None) == 2
+
+
+def test_baseconv_validation(lib):
+    f = lib.baseconv_gate_forward
+    O = ctypes.c_void_p(0x2000)
+    assert f(P, P, P, P, O, 1, 4, 64, 0, 1, None) == 1                    # width 0
+    assert f(P, O, P, P, O, 1, 4, 64, 3, 1, None) == 1                    # out aliases g
+    assert f(P, P, P, P, O, 1, 4, 60, 3, 1, None) == 2                    # C not a multiple of 8
+    assert f(P, P, P, P, O, 1, 4, 64, 5, 1, None) == 2                    # width > 4
+    assert f(P, U, P, P, O, 1, 4, 64, 3, 1, None) == 3
+    s = lib.baseconv_gate_step
+    assert s(P, P, P, P, None, O, 1, 64, 3, 1, None) == 1                 # state missing for width > 1
+    assert s(P, P, P, P, U, O, 1, 64, 3, 1, None) == 3
 
 
 def test_binding_rejects_cpu_tensors():

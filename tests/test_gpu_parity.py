@@ -155,6 +155,68 @@ def test_decode_chain_equals_prefill_on_gpu():
     assert head_err(_np(z), z_ref) <= TOL_F32 and head_err(_np(z2), z_ref) <= TOL_F32
 
 
+# --------------------------------------------------------------------------- gated short convolution
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,N,C,w", [(2, 100, 64, 3), (1, 33, 1032, 3), (3, 1, 8, 3), (2, 70, 256, 1), (1, 65, 136, 2),
+                                     (2, 64, 2048, 4)])
+def test_baseconv_gate_forward_small(dtype, B, N, C, w):
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    g_ = wl.generator(N * 7 + C + w)
+    a = torch.randn(B, N, C, generator=g_).to(tdt)
+    g = torch.randn(B, N, C, generator=g_).to(tdt)
+    h = torch.randn(w, C, generator=g_) * 0.6
+    b2 = torch.randn(C, generator=g_) * 0.3
+    ref = oracle.baseconv_gate(_np(a), _np(g), _np(h), _np(b2))
+    out = torch.full_like(a, float("nan"), device=DEV)
+    based.baseconv_gate_forward(a.to(DEV), g.to(DEV), h.to(DEV), b2.to(DEV), out=out)
+    # element-wise op: the tolerance applies per element, relative to the row's largest value
+    assert row_err(_np(out), ref) <= tol_for(dtype)
+    # in place over a
+    a_dev = a.to(DEV)
+    based.baseconv_gate_forward(a_dev, g.to(DEV), h.to(DEV), b2.to(DEV), out=a_dev)
+    assert torch.equal(a_dev, out)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("w", [1, 3, 4])
+def test_baseconv_gate_step_chain(dtype, w):
+    """Token-by-token calls on the rolling state reproduce the whole-sequence oracle."""
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    B, N, C = 3, 12, 264
+    g_ = wl.generator(50 + w)
+    a = torch.randn(B, N, C, generator=g_).to(tdt)
+    g = torch.randn(B, N, C, generator=g_).to(tdt)
+    h = torch.randn(w, C, generator=g_) * 0.6
+    b2 = torch.randn(C, generator=g_) * 0.3
+    ref = oracle.baseconv_gate(_np(a), _np(g), _np(h), _np(b2))
+    state = torch.zeros(B, w - 1, C, dtype=tdt, device=DEV) if w > 1 else None
+    hd, bd = h.to(DEV), b2.to(DEV)
+    for t in range(N):
+        out = based.baseconv_gate_step(a[:, t].contiguous().to(DEV), g[:, t].contiguous().to(DEV), hd, bd, state)
+        assert row_err(_np(out), ref[:, t]) <= tol_for(dtype), f"token {t}"
+    if w > 1:
+        assert torch.equal(state[:, 0].cpu(), g[:, N - 1])           # the state holds g exactly
+
+
+def test_baseconv_gate_full_size_sampled():
+    """A 1.3B-layer-sized call (B8 N4096 C8192, bf16): sampled (batch, token-run, channel-block)
+    tiles recomputed by the oracle, including run boundaries and the sequence start."""
+    B, N, C, w = 8, 4096, 8192, 3
+    g_ = torch.Generator(device=DEV).manual_seed(9)
+    a = torch.randn(B, N, C, generator=g_, device=DEV).bfloat16()
+    g = torch.randn(B, N, C, generator=g_, device=DEV).bfloat16()
+    h = torch.randn(w, C, generator=g_, device=DEV) * 0.6
+    b2 = torch.randn(C, generator=g_, device=DEV) * 0.3
+    out = based.baseconv_gate_forward(a, g, h, b2)
+    for (b, i0, c0) in [(0, 0, 0), (7, 4096 - 40, 8192 - 64), (3, 30, 1000), (5, 2047, 4096)]:
+        i_lo = max(0, i0 - (w - 1))
+        sl = (slice(b, b + 1), slice(i_lo, i0 + 40), slice(c0, c0 + 64))
+        a_s, g_s = _np(a[sl]), _np(g[sl])
+        ref = oracle.baseconv_gate(a_s, g_s, _np(h[:, c0:c0 + 64]), _np(b2[c0:c0 + 64]))
+        skip = i0 - i_lo            # rows that only serve as history (exact at the sequence start, where skip = 0)
+        assert row_err(_np(out[sl])[:, skip:], ref[:, skip:]) <= TOL_BF16
+
+
 # --------------------------------------------------------------------------- graph-replayed generation step
 @pytest.mark.parametrize("sym", [False, True])
 def test_decode_graph_replays_match_oracle_chain(sym):
