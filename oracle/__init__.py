@@ -59,6 +59,8 @@ def _load():
         lib.oracle_baseconv_gate_step.argtypes = [_dp, _dp, _dp, _dp, _dp, _dp, i, i, i]
         lib.oracle_baseconv_gate.restype = None
         lib.oracle_baseconv_gate_step.restype = None
+        lib.oracle_linattn_numerator.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i]
+        lib.oracle_linattn_numerator.restype = None
         for name in ("oracle_phi", "oracle_linattn_row", "oracle_linattn_quadratic", "oracle_linattn_recurrent",
                      "oracle_swa", "oracle_linattn_quadratic_ld", "oracle_swa_decode_step"):
             getattr(lib, name).restype = None
@@ -245,3 +247,11 @@ def baseconv_gate_step(a, g, h, b2, state):
     out = np.empty_like(a)
     _load().oracle_baseconv_gate_step(_p(a), _p(g), _p(h), _p(b2), _p(st), _p(out), B, C, w)
     return out, st
+
+
+def linattn_numerator(q, k, v) -> np.ndarray:
+    """Numerator of the definition form: y_i = sum_{j<=i} phi(q_i).phi(k_j) v_j (no division)."""
+    q, k, v, B, H, L, dp, dv = _shapes(q, k, v)
+    y = np.empty((B, H, L, dv))
+    _load().oracle_linattn_numerator(_p(q), _p(k), _p(v), _p(y), B, H, L, dp, dv)
+    return y

@@ -27,6 +27,9 @@
  *                               cache update the paper's benchmark leaves out).
  *   oracle_linattn_quadratic_ld the quadratic form again with long double
  *                               accumulators (adequacy check of fp64 on tiny inputs).
+ *   oracle_linattn_numerator    the numerator alone, sum_{j<=i} phi(q_i).phi(k_j) v_j: what Algorithm 1
+ *                               and the kernel micro-benchmarks of App. "IO Aware Implementations" (their
+ *                               captions say they time the numerator) compute.
  *   oracle_psi, oracle_state_to_sym, oracle_linattn_recurrent_sym
  *                               the same recurrences on the symmetric feature set whose size
  *                               the appendix "Computing Recurrent State Size" counts,
@@ -387,6 +390,26 @@ void oracle_baseconv_gate_step(const double *a, const double *g, const double *h
             out[(size_t)b * C + c] = a[(size_t)b * C + c] * silu(acc);
             for (int j = w - 2; j >= 1; --j) st[(size_t)j * C + c] = st[(size_t)(j - 1) * C + c];
             if (w > 1) st[c] = g[(size_t)b * C + c];
+        }
+    }
+}
+
+/* ---- numerator only (Algorithm 1 stops here; the micro-benchmark figures time this) ---------- */
+void oracle_linattn_numerator(const double *q, const double *k, const double *v, double *y, int B, int H, int L,
+                              int dp, int dv) {
+    const long nh = (long)B * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long bh = 0; bh < nh; ++bh) {
+        const double *qh = q + (size_t)bh * L * dp;
+        const double *kh = k + (size_t)bh * L * dp;
+        const double *vh = v + (size_t)bh * L * dv;
+        double *yh = y + (size_t)bh * L * dv;
+        for (int i = 0; i < L; ++i) {
+            for (int c = 0; c < dv; ++c) yh[(size_t)i * dv + c] = 0.0;
+            for (int j = 0; j <= i; ++j) {
+                const double w = taylor_weight(qh + (size_t)i * dp, kh + (size_t)j * dp, dp);
+                for (int c = 0; c < dv; ++c) yh[(size_t)i * dv + c] += w * vh[(size_t)j * dv + c];
+            }
         }
     }
 }

@@ -227,3 +227,18 @@ def test_long_double_brute_force_agrees():
 
 def test_oracle_reports_threads():
     assert oracle.num_threads() >= 1
+
+
+def test_numerator_only_form():
+    """Numerator alone (what Algorithm 1 computes): against an explicit masked matrix product written
+    with numpy, and against normalised output x denominator (the denominator is the numerator of v = 1)."""
+    B, H, L, dp, dv = 1, 2, 45, 16, 6
+    rng = np.random.default_rng(31)
+    q, k, v = rng.standard_normal((B, H, L, dp)) * 0.6, rng.standard_normal((B, H, L, dp)) * 0.6, rng.standard_normal((B, H, L, dv))
+    num = oracle.linattn_numerator(q, k, v)
+    s = np.einsum("bhid,bhjd->bhij", q, k)
+    wmat = np.tril(1.0 + s / 4.0 + s * s / 32.0)
+    np.testing.assert_allclose(num, wmat @ v, rtol=1e-12, atol=1e-12)
+    den = oracle.linattn_numerator(q, k, np.ones((B, H, L, 1)))
+    y, _, _ = oracle.linattn_quadratic(q, k, v, return_state=False)
+    np.testing.assert_allclose(num, y * (den + 1e-12), rtol=1e-11, atol=1e-12)
