@@ -49,8 +49,11 @@ typedef enum { BASED_F32 = 0, BASED_BF16 = 1 } based_dtype;
 enum {
     BASED_STATE_ZERO_INIT = 0, /* start from the empty state */
     BASED_STATE_CONTINUE = 1,  /* start from the state held in kv_state / z_state */
-    BASED_STATE_SYM = 2        /* OR-ed in: kv_state / z_state use the 153-row symmetric format
+    BASED_STATE_SYM = 2,       /* OR-ed in: kv_state / z_state use the 153-row symmetric format
                                   described at based_decode_step_sym ([B,H,153,d_v], [B,H,153]) */
+    BASED_NUMERATOR_ONLY = 4   /* OR-ed in: out = sum_j w_ij v_j without the division by sum_j w_ij
+                                  (what Algorithm 1 and the kernel micro-benchmarks of App. "IO Aware
+                                  Implementations" compute); the state is updated as usual */
 };
 
 /*
@@ -111,6 +114,14 @@ based_status based_decode_step(const void* q, const void* k, const void* v, floa
 based_status based_decode_step_sym(const void* q, const void* k, const void* v, float* kv_sym, float* z_sym,
                                    void* out, int B, int H, int d_feat, int d_v, based_dtype io,
                                    void* cuda_stream);
+
+/*
+ * based_decode_step with flags: 0, BASED_STATE_SYM (the state has the symmetric format, as
+ * based_decode_step_sym), BASED_NUMERATOR_ONLY (out = phi(q) kv_state, no division), or both.
+ */
+based_status based_decode_step_flags(const void* q, const void* k, const void* v, float* kv_state, float* z_state,
+                                     void* out, int B, int H, int d_feat, int d_v, based_dtype io, int flags,
+                                     void* cuda_stream);
 
 /*
  * Conversions between the 273-row state of based_prefill / based_decode_step and the symmetric

@@ -17,7 +17,7 @@ LIB_PATH = _PKG / "libbased.so"
 
 BASED_OK = 0
 BASED_F32, BASED_BF16 = 0, 1
-BASED_STATE_ZERO_INIT, BASED_STATE_CONTINUE, BASED_STATE_SYM = 0, 1, 2
+BASED_STATE_ZERO_INIT, BASED_STATE_CONTINUE, BASED_STATE_SYM, BASED_NUMERATOR_ONLY = 0, 1, 2, 4
 D_FEAT = 16
 D_EXPANDED = 1 + D_FEAT + D_FEAT * D_FEAT
 D_SYM = 1 + D_FEAT + D_FEAT * (D_FEAT + 1) // 2         # rows of the symmetric state format
@@ -27,7 +27,7 @@ EXPORTS = (
     "based_status_string", "based_version", "based_launch_count", "based_prefill_static_scratch",
     "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step", "based_decode_step_sym",
     "based_state_to_sym", "based_state_from_sym", "swa_decode_step_at", "based_preload_decode",
-    "baseconv_gate_forward", "baseconv_gate_step",
+    "baseconv_gate_forward", "baseconv_gate_step", "based_decode_step_flags",
 )
 
 _lib = None
@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.based_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
         L.based_decode_step_sym.restype = i
         L.based_decode_step_sym.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+        L.based_decode_step_flags.restype = i
+        L.based_decode_step_flags.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, vp]
         L.based_state_to_sym.restype = i
         L.based_state_to_sym.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
         L.based_state_from_sym.restype = i
@@ -202,6 +204,19 @@ def based_decode_step_sym(q, k, v, kv_sym, z_sym, out=None, stream=None):
     st = lib().based_decode_step_sym(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_sym), _ptr(z_sym), _ptr(out), B, H, d_feat,
                                      d_v, _dtype_code(q), _stream(stream))
     _check(st, "based_decode_step_sym")
+    return out
+
+
+def based_decode_step_flags(q, k, v, kv_state, z_state, flags: int, out=None, stream=None):
+    """based_decode_step with flags (BASED_STATE_SYM and/or BASED_NUMERATOR_ONLY)."""
+    _dev(q, k, v, kv_state, z_state, out)
+    B, H, d_feat = q.shape
+    d_v = v.shape[-1]
+    if out is None:
+        out = torch.empty_like(v)
+    st = lib().based_decode_step_flags(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_state), _ptr(z_state), _ptr(out), B, H,
+                                       d_feat, d_v, _dtype_code(q), int(flags), _stream(stream))
+    _check(st, "based_decode_step_flags")
     return out
 
 

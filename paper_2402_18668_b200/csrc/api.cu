@@ -80,7 +80,7 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
                            size_t workspace_bytes, void* cuda_stream) {
     if (!q || !k || !v || !out || B <= 0 || H <= 0 || L <= 0) return BASED_ERR_INVALID_ARG;
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
-    if (flags & ~(BASED_STATE_CONTINUE | BASED_STATE_SYM)) return BASED_ERR_INVALID_ARG;
+    if (flags & ~(BASED_STATE_CONTINUE | BASED_STATE_SYM | BASED_NUMERATOR_ONLY)) return BASED_ERR_INVALID_ARG;
     if ((kv_state == nullptr) != (z_state == nullptr)) return BASED_ERR_INVALID_ARG;
     if ((flags & BASED_STATE_CONTINUE) && !kv_state) return BASED_ERR_INVALID_ARG;
     if (out == q || out == k || out == v) return BASED_ERR_INVALID_ARG;
@@ -108,8 +108,23 @@ based_status based_decode_step(const void* q, const void* k, const void* v, floa
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
         !aligned16(z_state))
         return BASED_ERR_ALIGNMENT;
-    return launch_decode(q, k, v, kv_state, z_state, out, B * H, d_v, io, false,
+    return launch_decode(q, k, v, kv_state, z_state, out, B * H, d_v, io, false, false,
                          static_cast<cudaStream_t>(cuda_stream));
+}
+
+based_status based_decode_step_flags(const void* q, const void* k, const void* v, float* kv_state, float* z_state,
+                                     void* out, int B, int H, int d_feat, int d_v, based_dtype io, int flags,
+                                     void* cuda_stream) {
+    if (!q || !k || !v || !out || !kv_state || !z_state || B <= 0 || H <= 0) return BASED_ERR_INVALID_ARG;
+    if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
+    if (flags & ~(BASED_STATE_SYM | BASED_NUMERATOR_ONLY)) return BASED_ERR_INVALID_ARG;
+    if (d_feat != kDFeat || (d_v != 64 && d_v != 128)) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
+        !aligned16(z_state))
+        return BASED_ERR_ALIGNMENT;
+    return launch_decode(q, k, v, kv_state, z_state, out, B * H, d_v, io, (flags & BASED_STATE_SYM) != 0,
+                         (flags & BASED_NUMERATOR_ONLY) != 0, static_cast<cudaStream_t>(cuda_stream));
 }
 
 based_status based_decode_step_sym(const void* q, const void* k, const void* v, float* kv_sym, float* z_sym,
@@ -122,7 +137,8 @@ based_status based_decode_step_sym(const void* q, const void* k, const void* v, 
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_sym) ||
         !aligned16(z_sym))
         return BASED_ERR_ALIGNMENT;
-    return launch_decode(q, k, v, kv_sym, z_sym, out, B * H, d_v, io, true, static_cast<cudaStream_t>(cuda_stream));
+    return launch_decode(q, k, v, kv_sym, z_sym, out, B * H, d_v, io, true, false,
+                         static_cast<cudaStream_t>(cuda_stream));
 }
 
 static based_status state_convert(const float* kv_in, const float* z_in, float* kv_out, float* z_out, int B, int H,

@@ -72,7 +72,7 @@ __device__ __forceinline__ float psi_at(const float* x, int f) {
 // kernel launchers (defined in the .cu files; all asynchronous on `stream`)
 // sym: the state has the 153 symmetric rows instead of the 273 full ones
 based_status launch_decode(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
-                           int BH, int d_v, based_dtype io, bool sym, cudaStream_t stream);
+                           int BH, int d_v, based_dtype io, bool sym, bool numerator_only, cudaStream_t stream);
 // full (273-row) state -> symmetric (153-row) state, or back
 based_status launch_state_convert(const float* kv_in, const float* z_in, float* kv_out, float* z_out, int BH,
                                   int d_v, bool to_sym, cudaStream_t stream);

@@ -25,7 +25,8 @@ namespace based {
 template <int DV, typename T, bool STREAM, bool SYM>
 __global__ void __launch_bounds__(256, 4) decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k,
                                                           const T* __restrict__ v, float* __restrict__ kv,
-                                                          float* __restrict__ z, T* __restrict__ out) {
+                                                          float* __restrict__ z, T* __restrict__ out,
+                                                          int numerator_only) {
     constexpr int TPR = DV / 4;                    // threads per state row (one float4 each)
     constexpr int RPP = 256 / TPR;                 // rows per pass: 8 (d_v 128) or 16 (d_v 64)
     constexpr int ND = SYM ? kDSym : kD;           // state rows
@@ -104,39 +105,42 @@ __global__ void __launch_bounds__(256, 4) decode_step_kernel(const T* __restrict
         float den = 0.f;
 #pragma unroll
         for (int w = 0; w < 8; ++w) den += s_den[w];
-        out[head * DV + tid] = from_f32<T>(num / (den + kEps));
+        out[head * DV + tid] = from_f32<T>(numerator_only ? num : num / (den + kEps));
     }
 }
 
 template <int DV, typename T, bool SYM>
 static based_status launch_t(const void* q, const void* k, const void* v, float* kv, float* z, void* out, int BH,
-                             cudaStream_t stream) {
+                             int num_only, cudaStream_t stream) {
     // 96 MB: safely above what L2 (126 MB, shared with everything else) keeps from one step to the next
     const bool streaming = (size_t)BH * (SYM ? kDSym : kD) * DV * sizeof(float) > (size_t)96 << 20;
     if (streaming)
         decode_step_kernel<DV, T, true, SYM><<<BH, 256, 0, stream>>>(
-            static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), kv, z, static_cast<T*>(out));
+            static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), kv, z, static_cast<T*>(out),
+            num_only);
     else
         decode_step_kernel<DV, T, false, SYM><<<BH, 256, 0, stream>>>(
-            static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), kv, z, static_cast<T*>(out));
+            static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), kv, z, static_cast<T*>(out),
+            num_only);
     note_launch();
     return check_launch("decode_step_kernel");
 }
 
 template <int DV, bool SYM>
 static based_status launch_dv(const void* q, const void* k, const void* v, float* kv, float* z, void* out, int BH,
-                              based_dtype io, cudaStream_t stream) {
-    return io == BASED_F32 ? launch_t<DV, float, SYM>(q, k, v, kv, z, out, BH, stream)
-                           : launch_t<DV, __nv_bfloat16, SYM>(q, k, v, kv, z, out, BH, stream);
+                              based_dtype io, int num_only, cudaStream_t stream) {
+    return io == BASED_F32 ? launch_t<DV, float, SYM>(q, k, v, kv, z, out, BH, num_only, stream)
+                           : launch_t<DV, __nv_bfloat16, SYM>(q, k, v, kv, z, out, BH, num_only, stream);
 }
 
 based_status launch_decode(const void* q, const void* k, const void* v, float* kv, float* z, void* out, int BH,
-                           int d_v, based_dtype io, bool sym, cudaStream_t stream) {
+                           int d_v, based_dtype io, bool sym, bool numerator_only, cudaStream_t stream) {
+    const int n = numerator_only ? 1 : 0;
     if (d_v == 64)
-        return sym ? launch_dv<64, true>(q, k, v, kv, z, out, BH, io, stream)
-                   : launch_dv<64, false>(q, k, v, kv, z, out, BH, io, stream);
-    return sym ? launch_dv<128, true>(q, k, v, kv, z, out, BH, io, stream)
-               : launch_dv<128, false>(q, k, v, kv, z, out, BH, io, stream);
+        return sym ? launch_dv<64, true>(q, k, v, kv, z, out, BH, io, n, stream)
+                   : launch_dv<64, false>(q, k, v, kv, z, out, BH, io, n, stream);
+    return sym ? launch_dv<128, true>(q, k, v, kv, z, out, BH, io, n, stream)
+               : launch_dv<128, false>(q, k, v, kv, z, out, BH, io, n, stream);
 }
 
 // ------------------------------------------------------------------ full <-> symmetric state

@@ -123,7 +123,7 @@ __global__ void __launch_bounds__(kGroups* DV + 32, 1)
                 num += s_part[gg][t][cc];
                 den += s_part[gg][t][DV];
             }
-            oh[(size_t)t0 * DV + i] = from_f32<T>(num / (den + kEps));
+            oh[(size_t)t0 * DV + i] = from_f32<T>((flags & BASED_NUMERATOR_ONLY) ? num : num / (den + kEps));
         }
     }
 

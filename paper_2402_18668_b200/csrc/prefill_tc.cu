@@ -106,6 +106,7 @@ struct Params {
     int seg_len;          // tokens per segment (multiple of kC)
     int continue_abi;     // start from the ABI state in kv_abi / z_abi
     int sym;              // kv_abi / z_abi use the 153-row symmetric format
+    int numerator_only;   // outputs are not divided by the denominator
 #ifdef BASED_TRACE
     unsigned long long* trace;
 #endif
@@ -511,7 +512,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 uint32_t dcol;
                 tmem_ld1(tmem_addr(tb, lane_base, C::colY + DV), dcol);
                 tmem_wait_ld();
-                const float inv = 1.0f / (s_den[(c & 3) * kC + t] + __uint_as_float(dcol) + kEps);
+                const float inv = p.numerator_only ? 1.0f : 1.0f / (s_den[(c & 3) * kC + t] + __uint_as_float(dcol) + kEps);
 #pragma unroll 1
                 for (int h = 0; h < DV / 64; ++h) {
                     uint32_t y0[32], y1[32];
@@ -913,6 +914,7 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
     p.seg_len = plan.per * kC;
     p.continue_abi = (flags & BASED_STATE_CONTINUE) ? 1 : 0;
     p.sym = (flags & BASED_STATE_SYM) ? 1 : 0;
+    p.numerator_only = (flags & BASED_NUMERATOR_ONLY) ? 1 : 0;
 #ifdef BASED_TRACE
     p.trace = g_trace;
 #endif

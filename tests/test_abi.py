@@ -93,7 +93,9 @@ def test_swa_decode_validation(lib):
 def test_sym_state_validation(lib):
     pf = lib.based_prefill
     O2 = ctypes.c_void_p(0x2000)
-    assert pf(P, P, P, O2, None, None, 1, 1, 8, 16, 64, 1, 4, None, 0, None) == 1     # unknown flag bit
+    assert pf(P, P, P, O2, None, None, 1, 1, 8, 16, 64, 1, 8, None, 0, None) == 1     # unknown flag bit
+    df = lib.based_decode_step_flags
+    assert df(P, P, P, P, P, O2, 1, 1, 16, 64, 1, 1, None) == 1                       # CONTINUE is not a decode flag
     assert pf(P, P, P, O2, None, None, 1, 1, 8, 16, 64, 1, 3, None, 0, None) == 1     # continue without a state
     d = lib.based_decode_step_sym
     assert d(P, P, P, None, P, P, 1, 1, 16, 64, 0, None) == 1

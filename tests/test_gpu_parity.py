@@ -155,6 +155,30 @@ def test_decode_chain_equals_prefill_on_gpu():
     assert head_err(_np(z), z_ref) <= TOL_F32 and head_err(_np(z2), z_ref) <= TOL_F32
 
 
+# --------------------------------------------------------------------------- numerator only
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("L,d_v", [(300, 64), (200, 128)])
+def test_numerator_only_prefill_and_decode(dtype, L, d_v):
+    """BASED_NUMERATOR_ONLY: prefill rows and two decode steps against the oracle's numerator."""
+    B, H, T = 2, 2, 2
+    w = wl.Workload("num", B, H, L + T, 16, d_v, dtype, 0.5)
+    q, k, v = wl.prefill_inputs(w, wl.generator(L))
+    ref = oracle.linattn_numerator(_np(q), _np(k), _np(v))
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    kv, z = based.new_state(B, H, d_v)
+    out = based.based_prefill(qd[:, :, :L].contiguous(), kd[:, :, :L].contiguous(), vd[:, :, :L].contiguous(),
+                              kv_state=kv, z_state=z, flags=based.BASED_NUMERATOR_ONLY)
+    tol = tol_for(dtype)
+    assert row_err(_np(out), ref[:, :, :L]) <= tol
+    kvs, zs = based.based_state_to_sym(kv, z)
+    for t in range(L, L + T):
+        args = (qd[:, :, t].contiguous(), kd[:, :, t].contiguous(), vd[:, :, t].contiguous())
+        o_full = based.based_decode_step_flags(*args, kv, z, based.BASED_NUMERATOR_ONLY)
+        o_sym = based.based_decode_step_flags(*args, kvs, zs, based.BASED_NUMERATOR_ONLY | based.BASED_STATE_SYM)
+        assert row_err(_np(o_full), ref[:, :, t]) <= tol and row_err(_np(o_sym), ref[:, :, t]) <= tol
+    _poll()
+
+
 # --------------------------------------------------------------------------- gated short convolution
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("B,N,C,w", [(2, 100, 64, 3), (1, 33, 1032, 3), (3, 1, 8, 3), (2, 70, 256, 1), (1, 65, 136, 2),
