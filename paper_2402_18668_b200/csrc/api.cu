@@ -45,6 +45,8 @@ based_status check_launch(const char* what) {
 }
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+// value head dimensions: 64 (360M-scale heads), 128, and 112 (the 1.3B configuration's 1792 / 16)
+static inline bool dv_ok(int d_v) { return d_v == 64 || d_v == 112 || d_v == 128; }
 
 }  // namespace based
 
@@ -70,7 +72,7 @@ const char* based_status_string(based_status s) {
 }
 
 size_t based_prefill_workspace_bytes(int B, int H, int L, int d_feat, int d_v, based_dtype io) {
-    if (B <= 0 || H <= 0 || L <= 0 || d_feat != kDFeat || (d_v != 64 && d_v != 128)) return 0;
+    if (B <= 0 || H <= 0 || L <= 0 || d_feat != kDFeat || !dv_ok(d_v)) return 0;
     if (io != BASED_BF16) return 0;            // the fp32 path keeps its state in registers
     return prefill_tc_workspace_bytes(B * H, L, d_v);
 }
@@ -84,7 +86,7 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
     if ((kv_state == nullptr) != (z_state == nullptr)) return BASED_ERR_INVALID_ARG;
     if ((flags & BASED_STATE_CONTINUE) && !kv_state) return BASED_ERR_INVALID_ARG;
     if (out == q || out == k || out == v) return BASED_ERR_INVALID_ARG;
-    if (d_feat != kDFeat || (d_v != 64 && d_v != 128)) return BASED_ERR_UNSUPPORTED;
+    if (d_feat != kDFeat || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
     if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
         !aligned16(z_state) || !aligned16(workspace))
@@ -103,7 +105,7 @@ based_status based_decode_step(const void* q, const void* k, const void* v, floa
                                void* out, int B, int H, int d_feat, int d_v, based_dtype io, void* cuda_stream) {
     if (!q || !k || !v || !out || !kv_state || !z_state || B <= 0 || H <= 0) return BASED_ERR_INVALID_ARG;
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
-    if (d_feat != kDFeat || (d_v != 64 && d_v != 128)) return BASED_ERR_UNSUPPORTED;
+    if (d_feat != kDFeat || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
     if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
         !aligned16(z_state))
@@ -118,7 +120,7 @@ based_status based_decode_step_flags(const void* q, const void* k, const void* v
     if (!q || !k || !v || !out || !kv_state || !z_state || B <= 0 || H <= 0) return BASED_ERR_INVALID_ARG;
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
     if (flags & ~(BASED_STATE_SYM | BASED_NUMERATOR_ONLY)) return BASED_ERR_INVALID_ARG;
-    if (d_feat != kDFeat || (d_v != 64 && d_v != 128)) return BASED_ERR_UNSUPPORTED;
+    if (d_feat != kDFeat || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
     if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
         !aligned16(z_state))
@@ -132,7 +134,7 @@ based_status based_decode_step_sym(const void* q, const void* k, const void* v, 
                                    void* cuda_stream) {
     if (!q || !k || !v || !out || !kv_sym || !z_sym || B <= 0 || H <= 0) return BASED_ERR_INVALID_ARG;
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
-    if (d_feat != kDFeat || (d_v != 64 && d_v != 128)) return BASED_ERR_UNSUPPORTED;
+    if (d_feat != kDFeat || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
     if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_sym) ||
         !aligned16(z_sym))
@@ -145,7 +147,7 @@ static based_status state_convert(const float* kv_in, const float* z_in, float* 
                                   int d_feat, int d_v, bool to_sym, void* cuda_stream) {
     if (!kv_in || !z_in || !kv_out || !z_out || B <= 0 || H <= 0) return BASED_ERR_INVALID_ARG;
     if (kv_in == kv_out || z_in == z_out) return BASED_ERR_INVALID_ARG;
-    if (d_feat != kDFeat || (d_v != 64 && d_v != 128)) return BASED_ERR_UNSUPPORTED;
+    if (d_feat != kDFeat || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
     if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(kv_in) || !aligned16(z_in) || !aligned16(kv_out) || !aligned16(z_out)) return BASED_ERR_ALIGNMENT;
     return launch_state_convert(kv_in, z_in, kv_out, z_out, B * H, d_v, to_sym,

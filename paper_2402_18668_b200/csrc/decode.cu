@@ -30,9 +30,10 @@ __global__ void __launch_bounds__(256, 4) decode_step_kernel(const T* __restrict
     constexpr int TPR = DV / 4;                    // threads per state row (one float4 each)
     constexpr int RPP = 256 / TPR;                 // rows per pass: 8 (d_v 128) or 16 (d_v 64)
     constexpr int ND = SYM ? kDSym : kD;           // state rows
-    constexpr int NPASS = (ND + RPP - 1) / RPP;    // full: 35 or 18; symmetric: 20 or 10
-    constexpr int UNROLL = SYM ? 5 : (DV == 128) ? 7 : 6;   // loads in flight per thread (35 = 5*7, 18 = 3*6, 20 = 4*5)
-    static_assert(NPASS % UNROLL == 0, "pass count must divide");
+    constexpr int UNROLL = SYM ? 5 : (DV == 64) ? 6 : 7;    // loads in flight per thread (35 = 5*7, 18 = 3*6, 20 = 4*5)
+    // full: 35 or 18 passes; symmetric: 20 or 10; d_v 112 (28 threads per row, 9 rows per pass, the last
+    // 4 threads idle): 31 and 17 passes, rounded up to the unroll factor (rows past the end are skipped)
+    constexpr int NPASS = ((ND + RPP - 1) / RPP + UNROLL - 1) / UNROLL * UNROLL;
     constexpr int DPAD = NPASS * RPP;
 
     __shared__ float s_x[2][kDFeat];
@@ -43,6 +44,7 @@ __global__ void __launch_bounds__(256, 4) decode_step_kernel(const T* __restrict
     const int tid = threadIdx.x;
     const size_t head = blockIdx.x;
     const int c4 = tid % TPR, rslot = tid / TPR;
+    const bool row_thread = rslot < RPP;             // false only for the idle tail threads of d_v 112
 
     if (tid < kDFeat) s_x[0][tid] = to_f32(q[head * kDFeat + tid]);
     else if (tid < 2 * kDFeat) s_x[1][tid - kDFeat] = to_f32(k[head * kDFeat + tid - kDFeat]);
@@ -76,12 +78,12 @@ __global__ void __launch_bounds__(256, 4) decode_step_kernel(const T* __restrict
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const int r = (p0 + u) * RPP + rslot;
-            if (r < ND) s[u] = STREAM ? __ldcs(&S[(size_t)r * TPR]) : S[(size_t)r * TPR];
+            if (r < ND && row_thread) s[u] = STREAM ? __ldcs(&S[(size_t)r * TPR]) : S[(size_t)r * TPR];
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const int r = (p0 + u) * RPP + rslot;
-            if (r < ND) {
+            if (r < ND && row_thread) {
                 const float pk = s_pk[r], pq = s_pq[r];
                 s[u].x = fmaf(pk, vv[0], s[u].x);
                 s[u].y = fmaf(pk, vv[1], s[u].y);
@@ -96,7 +98,7 @@ __global__ void __launch_bounds__(256, 4) decode_step_kernel(const T* __restrict
             }
         }
     }
-    *reinterpret_cast<float4*>(&s_num[rslot][c4 * 4]) = acc;
+    if (row_thread) *reinterpret_cast<float4*>(&s_num[rslot][c4 * 4]) = acc;
     __syncthreads();
     if (tid < DV) {
         float num = 0.f;
@@ -139,6 +141,9 @@ based_status launch_decode(const void* q, const void* k, const void* v, float* k
     if (d_v == 64)
         return sym ? launch_dv<64, true>(q, k, v, kv, z, out, BH, io, n, stream)
                    : launch_dv<64, false>(q, k, v, kv, z, out, BH, io, n, stream);
+    if (d_v == 112)
+        return sym ? launch_dv<112, true>(q, k, v, kv, z, out, BH, io, n, stream)
+                   : launch_dv<112, false>(q, k, v, kv, z, out, BH, io, n, stream);
     return sym ? launch_dv<128, true>(q, k, v, kv, z, out, BH, io, n, stream)
                : launch_dv<128, false>(q, k, v, kv, z, out, BH, io, n, stream);
 }
@@ -213,6 +218,7 @@ bool load_decode_variants() {
 // otherwise load them there).
 based_status preload_decode() {
     const bool ok = load_decode_variants<64, float>() && load_decode_variants<64, __nv_bfloat16>() &&
+                    load_decode_variants<112, float>() && load_decode_variants<112, __nv_bfloat16>() &&
                     load_decode_variants<128, float>() && load_decode_variants<128, __nv_bfloat16>() &&
                     load_kernel(state_convert_kernel);
     return ok ? BASED_OK : BASED_ERR_CUDA;

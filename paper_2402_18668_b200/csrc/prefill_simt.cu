@@ -160,6 +160,10 @@ based_status launch_prefill_simt(const void* q, const void* k, const void* v, vo
         return io == BASED_F32 ? launch_t<64, float>(q, k, v, out, kv, z, BH, L, flags, stream)
                                : launch_t<64, __nv_bfloat16>(q, k, v, out, kv, z, BH, L, flags, stream);
     }
+    if (d_v == 112) {
+        return io == BASED_F32 ? launch_t<112, float>(q, k, v, out, kv, z, BH, L, flags, stream)
+                               : launch_t<112, __nv_bfloat16>(q, k, v, out, kv, z, BH, L, flags, stream);
+    }
     return io == BASED_F32 ? launch_t<128, float>(q, k, v, out, kv, z, BH, L, flags, stream)
                            : launch_t<128, __nv_bfloat16>(q, k, v, out, kv, z, BH, L, flags, stream);
 }

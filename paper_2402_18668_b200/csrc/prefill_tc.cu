@@ -107,6 +107,8 @@ struct Params {
     int continue_abi;     // start from the ABI state in kv_abi / z_abi
     int sym;              // kv_abi / z_abi use the 153-row symmetric format
     int numerator_only;   // outputs are not divided by the denominator
+    int dv;               // value head dimension of the caller's tensors (112 runs on the d_v 128 kernel:
+                          // the tensor maps zero-fill columns 112..127 on load and clip them on store)
 #ifdef BASED_TRACE
     unsigned long long* trace;
 #endif
@@ -570,7 +572,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int z1f = (DV == 128 && (t & 31) < 16 && (t >> 5) < 2) ? 128 + (t >> 5) * 16 + (t & 15) : -1;
         const size_t seg_stride = seg_state_floats(DV);
         const float* wsh = p.ws + (size_t)head * (p.nseg > 1 ? p.nseg - 1 : 0) * seg_stride;
-        const float* kvh = p.kv_abi ? p.kv_abi + (size_t)head * abi_nrows * DV : nullptr;
+        const int dv = p.dv;                        // row pitch of the caller's state; lanes >= dv hold zeros
+        const float* kvh = p.kv_abi ? p.kv_abi + (size_t)head * abi_nrows * dv : nullptr;
         const float* zh = p.z_abi ? p.z_abi + (size_t)head * abi_nrows : nullptr;
         const bool from_abi = !STATE_ONLY && p.continue_abi;
         const int nprev = (STATE_ONLY || PRE) ? 0 : seg;
@@ -589,8 +592,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const short2 ar = s_abi[b * 16 + i];
-                        va[i] = (ar.x >= 0) ? (is_z ? zh[ar.x] : kvh[(size_t)ar.x * DV + srow]) : 0.f;
-                        vb[i] = (ar.y >= 0) ? (is_z ? zh[ar.y] : kvh[(size_t)ar.y * DV + srow]) : 0.f;
+                        const bool live = is_z || srow < dv;
+                        va[i] = (ar.x >= 0 && live) ? (is_z ? zh[ar.x] : kvh[(size_t)ar.x * dv + srow]) : 0.f;
+                        vb[i] = (ar.y >= 0 && live) ? (is_z ? zh[ar.y] : kvh[(size_t)ar.y * dv + srow]) : 0.f;
                     }
 #pragma unroll
                     for (int i = 0; i < 16; ++i) acc[i] = (s_abi[b * 16 + i].y >= 0) ? (va[i] + vb[i]) * kRsqrt2 : va[i];
@@ -706,7 +710,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const bool write_abi = !STATE_ONLY && p.kv_abi != nullptr && seg == p.nseg - 1;
         if (ok && (write_ws || write_abi)) {
             float* wseg = p.ws + ((size_t)head * (p.nseg > 1 ? p.nseg - 1 : 0) + seg) * seg_stride;
-            float* kvo = write_abi ? p.kv_abi + (size_t)head * abi_nrows * DV : nullptr;
+            float* kvo = write_abi ? p.kv_abi + (size_t)head * abi_nrows * dv : nullptr;
             float* zo = write_abi ? p.z_abi + (size_t)head * abi_nrows : nullptr;
             auto put = [&](int f, float v, bool zrow, int col) {
                 if (write_ws) {
@@ -718,7 +722,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 if (ar.x < 0) return;
                 if (ar.y >= 0) v *= kRsqrt2;
                 if (zrow) { zo[ar.x] = v; if (ar.y >= 0) zo[ar.y] = v; }
-                else { kvo[(size_t)ar.x * DV + col] = v; if (ar.y >= 0) kvo[(size_t)ar.y * DV + col] = v; }
+                else if (col < dv) { kvo[(size_t)ar.x * dv + col] = v; if (ar.y >= 0) kvo[(size_t)ar.y * dv + col] = v; }
             };
 #pragma unroll 1
             for (int b = 0; b < kF / 16; ++b) {
@@ -894,13 +898,13 @@ unsigned long long* g_trace = nullptr;
 
 template <int DV>
 based_status launch_dv(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH, int L,
-                       int flags, float* ws, const SegPlan plan, cudaStream_t stream) {
+                       int dv, int flags, float* ws, const SegPlan plan, cudaStream_t stream) {
     using C = Cfg<DV>;
     CUtensorMap tq, tk, tv, to;
     if (!make_map(&tq, q, BH, L, kDFeat, kDFeat, CU_TENSOR_MAP_SWIZZLE_32B) ||
         !make_map(&tk, k, BH, L, kDFeat, kDFeat, CU_TENSOR_MAP_SWIZZLE_32B) ||
-        !make_map(&tv, v, BH, L, DV, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map(&to, out, BH, L, DV, 64, CU_TENSOR_MAP_SWIZZLE_128B))
+        !make_map(&tv, v, BH, L, dv, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map(&to, out, BH, L, dv, 64, CU_TENSOR_MAP_SWIZZLE_128B))
         return BASED_ERR_CUDA;
     Params p;
     p.kv_abi = kv;
@@ -915,6 +919,7 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
     p.continue_abi = (flags & BASED_STATE_CONTINUE) ? 1 : 0;
     p.sym = (flags & BASED_STATE_SYM) ? 1 : 0;
     p.numerator_only = (flags & BASED_NUMERATOR_ONLY) ? 1 : 0;
+    p.dv = dv;
 #ifdef BASED_TRACE
     p.trace = g_trace;
 #endif
@@ -1002,6 +1007,7 @@ static SegPlan prefill_tc_plan(int BH, int L, int d_v) {
 }
 
 size_t prefill_tc_workspace_bytes(int BH, int L, int d_v) {
+    if (d_v == 112) d_v = 128;                      // runs on the d_v 128 kernel, partial states in its layout
     const SegPlan plan = prefill_tc_plan(BH, L, d_v);
     const int nseg = plan.recompute ? 1 : plan.nseg;
     return nseg > 1 ? (size_t)BH * (nseg - 1) * seg_state_floats(d_v) * sizeof(float) : 0;
@@ -1009,10 +1015,10 @@ size_t prefill_tc_workspace_bytes(int BH, int L, int d_v) {
 
 based_status launch_prefill_tc(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH,
                                int L, int d_v, int flags, void* workspace, cudaStream_t stream) {
-    const SegPlan plan = prefill_tc_plan(BH, L, d_v);
+    const SegPlan plan = prefill_tc_plan(BH, L, d_v == 112 ? 128 : d_v);
     float* ws = static_cast<float*>(workspace);
-    if (d_v == 64) return launch_dv<64>(q, k, v, out, kv, z, BH, L, flags, ws, plan, stream);
-    return launch_dv<128>(q, k, v, out, kv, z, BH, L, flags, ws, plan, stream);
+    if (d_v == 64) return launch_dv<64>(q, k, v, out, kv, z, BH, L, 64, flags, ws, plan, stream);
+    return launch_dv<128>(q, k, v, out, kv, z, BH, L, d_v, flags, ws, plan, stream);      // 112 or 128
 }
 
 }  // namespace based

@@ -155,6 +155,39 @@ def test_decode_chain_equals_prefill_on_gpu():
     assert head_err(_np(z), z_ref) <= TOL_F32 and head_err(_np(z2), z_ref) <= TOL_F32
 
 
+# --------------------------------------------------------------------------- d_v = 112
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("L", [130, 4200])
+def test_head_dim_112_prefill_continue_and_decode(dtype, L):
+    """The 1.3B configuration's true value head dimension (1792 / 16): prefill in two calls
+    (state out, then continued), decode steps on both state formats."""
+    if dtype == "f32" and L > 1000:
+        pytest.skip("the fp32 path is the slow correctness path; the long case adds nothing there")
+    B, H, d_v, T = 2, 2, 112, 3
+    w = wl.Workload("dv112", B, H, L + T, 16, d_v, dtype, 0.5)
+    q, k, v = wl.prefill_inputs(w, wl.generator(112 + L))
+    y_ref, _, _ = oracle.linattn_quadratic(_np(q), _np(k), _np(v), return_state=False)
+    _, S_ref, z_ref = oracle.linattn_recurrent(_np(q[:, :, :L]), _np(k[:, :, :L]), _np(v[:, :, :L]))
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    tol = tol_for(dtype)
+    half = L // 2 + 1
+    kv, z = based.new_state(B, H, d_v)
+    out = torch.full((B, H, L, d_v), float("nan"), dtype=qd.dtype, device=DEV)
+    o1 = based.based_prefill(qd[:, :, :half].contiguous(), kd[:, :, :half].contiguous(), vd[:, :, :half].contiguous(),
+                             kv_state=kv, z_state=z)
+    o2 = based.based_prefill(qd[:, :, half:L].contiguous(), kd[:, :, half:L].contiguous(),
+                             vd[:, :, half:L].contiguous(), kv_state=kv, z_state=z, flags=based.BASED_STATE_CONTINUE)
+    out[:, :, :half], out[:, :, half:] = o1, o2
+    assert row_err(_np(out), y_ref[:, :, :L]) <= tol
+    assert head_err(_np(kv), S_ref) <= tol and head_err(_np(z), z_ref) <= tol
+    kvs, zs = based.based_state_to_sym(kv, z)
+    for t in range(L, L + T):
+        args = (qd[:, :, t].contiguous(), kd[:, :, t].contiguous(), vd[:, :, t].contiguous())
+        assert row_err(_np(based.based_decode_step(*args, kv, z)), y_ref[:, :, t]) <= tol
+        assert row_err(_np(based.based_decode_step_sym(*args, kvs, zs)), y_ref[:, :, t]) <= tol
+    _poll()
+
+
 # --------------------------------------------------------------------------- numerator only
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("L,d_v", [(300, 64), (200, 128)])
