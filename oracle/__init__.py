@@ -61,6 +61,8 @@ def _load():
         lib.oracle_baseconv_gate_step.restype = None
         lib.oracle_linattn_numerator.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i]
         lib.oracle_linattn_numerator.restype = None
+        lib.oracle_linattn_backward.argtypes = [_dp, _dp, _dp, _dp, _dp, _dp, _dp, i, i, i, i, i, i]
+        lib.oracle_linattn_backward.restype = None
         for name in ("oracle_phi", "oracle_linattn_row", "oracle_linattn_quadratic", "oracle_linattn_recurrent",
                      "oracle_swa", "oracle_linattn_quadratic_ld", "oracle_swa_decode_step"):
             getattr(lib, name).restype = None
@@ -255,3 +257,14 @@ def linattn_numerator(q, k, v) -> np.ndarray:
     y = np.empty((B, H, L, dv))
     _load().oracle_linattn_numerator(_p(q), _p(k), _p(v), _p(y), B, H, L, dp, dv)
     return y
+
+
+def linattn_backward(q, k, v, dout, numerator_only: bool = False):
+    """Gradients of the definition form with respect to q, k, v for the output gradient dout [B,H,L,dv]."""
+    q, k, v, B, H, L, dp, dv = _shapes(q, k, v)
+    dout = _f64(dout)
+    assert dout.shape == v.shape
+    dq, dk, dvv = np.empty_like(q), np.empty_like(k), np.empty_like(v)
+    _load().oracle_linattn_backward(_p(q), _p(k), _p(v), _p(dout), _p(dq), _p(dk), _p(dvv), B, H, L, dp, dv,
+                                    1 if numerator_only else 0)
+    return dq, dk, dvv

@@ -30,6 +30,10 @@
  *   oracle_linattn_numerator    the numerator alone, sum_{j<=i} phi(q_i).phi(k_j) v_j: what Algorithm 1
  *                               and the kernel micro-benchmarks of App. "IO Aware Implementations" (their
  *                               captions say they time the numerator) compute.
+ *   oracle_linattn_backward     gradients of the definition form (left-hand side of Eq. (2)) with respect
+ *                               to q, k, v for a given gradient of the output; the paper calls prefill
+ *                               "the forward pass during training" but prints no backward algorithm, so
+ *                               this is the chain rule applied to the definition, pair by pair.
  *   oracle_psi, oracle_state_to_sym, oracle_linattn_recurrent_sym
  *                               the same recurrences on the symmetric feature set whose size
  *                               the appendix "Computing Recurrent State Size" counts,
@@ -411,5 +415,68 @@ void oracle_linattn_numerator(const double *q, const double *k, const double *v,
                 for (int c = 0; c < dv; ++c) yh[(size_t)i * dv + c] += w * vh[(size_t)j * dv + c];
             }
         }
+    }
+}
+
+/* ---- backward of the definition form ------------------------------------------------------ */
+/*
+ * y_i = N_i / D_i,  N_i = sum_{j<=i} w_ij v_j,  D_i = sum_{j<=i} w_ij + eps,
+ * w_ij = 1 + s_ij / sqrt(d') + s_ij^2 / (2 d'),  s_ij = q_i . k_j.
+ * With G_i the gradient of the loss with respect to y_i:
+ *   dN_i = G_i / D_i (a vector),  dD_i = -(G_i . y_i) / D_i (a scalar),
+ *   dw_ij = dN_i . v_j + dD_i,  ds_ij = dw_ij (1 / sqrt(d') + s_ij / d'),
+ *   dv_j = sum_{i>=j} w_ij dN_i,  dq_i = sum_{j<=i} ds_ij k_j,  dk_j = sum_{i>=j} ds_ij q_i.
+ * numerator_only != 0: y_i = N_i (dN_i = G_i, dD_i = 0).
+ */
+void oracle_linattn_backward(const double *q, const double *k, const double *v, const double *dout, double *dq,
+                             double *dk, double *dv, int B, int H, int L, int dp, int dvw, int numerator_only) {
+    const long nh = (long)B * H;
+    const double rd = sqrt((double)dp);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long bh = 0; bh < nh; ++bh) {
+        const double *qh = q + (size_t)bh * L * dp, *kh = k + (size_t)bh * L * dp;
+        const double *vh = v + (size_t)bh * L * dvw, *gh = dout + (size_t)bh * L * dvw;
+        double *dqh = dq + (size_t)bh * L * dp, *dkh = dk + (size_t)bh * L * dp, *dvh = dv + (size_t)bh * L * dvw;
+        double *dN = (double *)malloc(sizeof(double) * (size_t)dvw);
+        double *num = (double *)malloc(sizeof(double) * (size_t)dvw);
+        memset(dqh, 0, sizeof(double) * (size_t)L * dp);
+        memset(dkh, 0, sizeof(double) * (size_t)L * dp);
+        memset(dvh, 0, sizeof(double) * (size_t)L * dvw);
+        for (int i = 0; i < L; ++i) {
+            /* forward quantities of row i */
+            double den = ORACLE_EPS;
+            for (int c = 0; c < dvw; ++c) num[c] = 0.0;
+            for (int j = 0; j <= i; ++j) {
+                const double w = taylor_weight(qh + (size_t)i * dp, kh + (size_t)j * dp, dp);
+                den += w;
+                for (int c = 0; c < dvw; ++c) num[c] += w * vh[(size_t)j * dvw + c];
+            }
+            double dD = 0.0;
+            for (int c = 0; c < dvw; ++c) {
+                const double g = gh[(size_t)i * dvw + c];
+                if (numerator_only) dN[c] = g;
+                else {
+                    dN[c] = g / den;
+                    dD -= g * (num[c] / den) / den;
+                }
+            }
+            for (int j = 0; j <= i; ++j) {
+                double sij = 0.0;
+                for (int m = 0; m < dp; ++m) sij += qh[(size_t)i * dp + m] * kh[(size_t)j * dp + m];
+                const double w = 1.0 + sij / rd + sij * sij / (2.0 * (double)dp);
+                double dw = dD;
+                for (int c = 0; c < dvw; ++c) {
+                    dw += dN[c] * vh[(size_t)j * dvw + c];
+                    dvh[(size_t)j * dvw + c] += w * dN[c];
+                }
+                const double ds = dw * (1.0 / rd + sij / (double)dp);
+                for (int m = 0; m < dp; ++m) {
+                    dqh[(size_t)i * dp + m] += ds * kh[(size_t)j * dp + m];
+                    dkh[(size_t)j * dp + m] += ds * qh[(size_t)i * dp + m];
+                }
+            }
+        }
+        free(dN);
+        free(num);
     }
 }
