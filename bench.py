@@ -467,6 +467,32 @@ def bench_baseconv(shape, steps, warmup, torch, based, dist_on, peaks):
     }
 
 
+def bench_backward(w, steps, warmup, torch, based, dist_on, peaks):
+    """Backward pass of the linear attention (fp32 FMA path, quadratic form) on the workload's shape.
+    Bound by the fp32 pipe: peak = SMs x 128 lanes x 2 flop x SM clock (148 x 128 x 2 x 1.965 GHz)."""
+    g = torch.Generator(device="cuda").manual_seed(8)
+    dt = w.torch_dtype
+    q = (torch.randn(w.B, w.H, w.L, w.d_feat, generator=g, device="cuda") * w.qk_scale).to(dt)
+    k = (torch.randn(w.B, w.H, w.L, w.d_feat, generator=g, device="cuda") * w.qk_scale).to(dt)
+    v = torch.randn(w.B, w.H, w.L, w.d_v, generator=g, device="cuda").to(dt)
+    dout = torch.randn(w.B, w.H, w.L, w.d_v, generator=g, device="cuda").to(dt)
+    ws = torch.empty(w.B * w.H * w.L * 8, dtype=torch.uint8, device="cuda")
+    n0 = based.launch_count()
+    ms = time_region(lambda i: based.based_prefill_backward(q, k, v, dout, workspace=ws), steps, warmup, torch, dist_on)
+    t = ms * 1e-3 / steps
+    pairs = w.B * w.H * w.L * (w.L + 1) / 2.0
+    flops = 2.0 * pairs * (80 + 4 * w.d_v)              # 3 score passes, 3 a.v passes + dv, dq and dk updates
+    alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12
+    return {
+        "workload": w.name + " backward (fp32 FMA, quadratic form)", "metric": "backward_tokens_per_s",
+        "value": w.B * w.L / t, "unit": "tokens/s", "ms_per_step": t * 1e3, "steps": steps,
+        "launches_per_step": (based.launch_count() - n0) // (steps + warmup),
+        "roofline": {"bound": "alu", "achieved": flops / t / 1e12, "peak": alu_peak, "unit": "TFLOP/s",
+                     "frac": flops / t / 1e12 / alu_peak, "traffic": None, "kernel": "bwd_dkdv_kernel",
+                     "algorithmic_flops": flops, "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz"},
+    }
+
+
 def cpu_oracle_sample(w, budget_heads: int):
     """The oracle's recurrent form, as it stands, on the first `budget_heads` heads of the
     workload's seeded host inputs.  Returns (tokens/s scaled to whole tokens, cores, text)."""
@@ -494,7 +520,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_360m_prefill")
     ap.add_argument("--skip-extras", action="store_true", help="only the headline prefill workload")
-    ap.add_argument("--profile", choices=["prefill", "decode", "decode_sym", "swa", "swa_decode", "generation_graph", "baseconv"],
+    ap.add_argument("--profile", choices=["prefill", "decode", "decode_sym", "swa", "swa_decode", "generation_graph", "baseconv", "backward"],
                     help="run only this arm on --shape (small cases for ncu captures) and print its result")
     ap.add_argument("--shape", default="", help="B,H,L,d_v for --profile (defaults to the arm's benchmark shape)")
     args = ap.parse_args()
@@ -545,7 +571,7 @@ def main():
         base = {"prefill": w, "decode": wl.CONFIGS["cfg4_generation"], "decode_sym": wl.CONFIGS["cfg4_generation"], "swa": wl.CONFIGS["cfg5_mixer_pair"],
                 "swa_decode": wl.CONFIGS["cfg4_generation"],
                 "generation_graph": wl.CONFIGS["cfg4_generation"],
-                "baseconv": wl.CONFIGS["cfg3_1p3b_prefill"]}[args.profile]
+                "baseconv": wl.CONFIGS["cfg3_1p3b_prefill"], "backward": w}[args.profile]
         if args.shape and args.profile != "baseconv":
             B, H, L, dv = (int(x) for x in args.shape.split(","))
             base = base.scaled(name=f"{base.name}[{args.shape}]", B=B, H=H, L=L, d_v=dv)
@@ -556,6 +582,8 @@ def main():
                              sym=args.profile == "decode_sym")
         elif args.profile == "swa_decode":
             r = bench_swa_decode(base, args.steps, args.warmup, torch, based, dist_on, peaks)
+        elif args.profile == "backward":
+            r = bench_backward(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         elif args.profile == "baseconv":
             shp = (8, 4096, 8192)
             if args.shape:
@@ -599,6 +627,7 @@ def main():
         extras["decode_sym"] = bench_decode(wl.CONFIGS["cfg4_generation"], 1024, 16, torch, based, dist_on, peaks,
                                             sym=True)
         torch.cuda.empty_cache()
+        extras["backward"] = bench_backward(w, 5, 3, torch, based, dist_on, peaks)
         extras["baseconv"] = bench_baseconv((8, 4096, 8192), 10, 3, torch, based, dist_on, peaks)
         extras["generation_graph"] = bench_generation_graph(wl.CONFIGS["cfg4_generation"], 512, 16, torch, based,
                                                             dist_on, peaks)

@@ -166,6 +166,29 @@ based_status swa_decode_step(const void* q, const void* k, const void* v, void* 
                              void* cuda_stream);
 
 /*
+ * Backward pass of based_prefill from the empty state (the paper calls prefill "the forward pass
+ * during training" but gives no backward algorithm: this is the chain rule on the definition
+ * form of Eq. (2), Sec. 4.1).  With dout the gradient of the loss with respect to out,
+ *
+ *   a_i = dout_i / D_i,  b_i = -(dout_i . out_i) / D_i,  D_i = sum_{j<=i} w_ij + 1e-12,
+ *   ds_ij = (a_i . v_j + b_i)(1/4 + q_i.k_j / 16),
+ *   dq_i = sum_{j<=i} ds_ij k_j,  dk_j = sum_{i>=j} ds_ij q_i,  dv_j = sum_{i>=j} w_ij a_i.
+ *
+ * q, k, dq, dk [B,H,L,d_feat]; v, dout, dv [B,H,L,d_v], all in the io dtype; arithmetic in fp32
+ * (the forward output is not an argument: out_i is recomputed in fp32, because a_i.v_j + b_i
+ * cancels almost completely for short prefixes and a rounded out would dominate the result).
+ * flags: 0, or BASED_NUMERATOR_ONLY for the backward of the numerator-only forward.
+ * workspace: at least based_prefill_backward_workspace_bytes(B, H, L) bytes of device scratch.
+ * Supported: d_feat = 16; d_v in {64, 112, 128}; io in {F32, BF16}; B*H <= 65535.
+ * This path evaluates the quadratic form with fp32 FMAs (O(L^2) per head): a correct first
+ * implementation, not a tensor-core kernel.  Gradient outputs must not alias inputs.
+ */
+based_status based_prefill_backward(const void* q, const void* k, const void* v, const void* dout, void* dq,
+                                    void* dk, void* dv, int B, int H, int L, int d_feat, int d_v, based_dtype io,
+                                    int flags, void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t based_prefill_backward_workspace_bytes(int B, int H, int L);
+
+/*
  * The gated short convolution at the core of the BaseConv layer (App. "Extended Architecture
  * Details", paragraph "Convolution": y = ((u W1 + b1) (.) SiLU(h * (u W2) + b2)) W3 + b3).
  * The three projections are plain matrix products and stay with the caller; this call is the

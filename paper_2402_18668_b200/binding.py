@@ -27,7 +27,8 @@ EXPORTS = (
     "based_status_string", "based_version", "based_launch_count", "based_prefill_static_scratch",
     "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step", "based_decode_step_sym",
     "based_state_to_sym", "based_state_from_sym", "swa_decode_step_at", "based_preload_decode",
-    "baseconv_gate_forward", "baseconv_gate_step", "based_decode_step_flags",
+    "baseconv_gate_forward", "baseconv_gate_step", "based_decode_step_flags", "based_prefill_backward",
+    "based_prefill_backward_workspace_bytes",
 )
 
 _lib = None
@@ -75,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.swa_decode_step_at.restype = i
         L.swa_decode_step_at.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, i, vp]
         L.based_preload_decode.restype = i
+        L.based_prefill_backward.restype = i
+        L.based_prefill_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
+        L.based_prefill_backward_workspace_bytes.restype = sz
+        L.based_prefill_backward_workspace_bytes.argtypes = [i, i, i]
         L.baseconv_gate_forward.restype = i
         L.baseconv_gate_forward.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
         L.baseconv_gate_step.restype = i
@@ -156,6 +161,22 @@ def based_prefill(q, k, v, out=None, kv_state=None, z_state=None, flags: int = B
                              d_v, io, flags, _ptr(workspace), ws_bytes, _stream(stream))
     _check(st, "based_prefill")
     return out
+
+
+def based_prefill_backward(q, k, v, dout, flags: int = 0, workspace=None, stream=None):
+    """Gradients (dq, dk, dv) of based_prefill (empty initial state) for the output gradient dout."""
+    _dev(q, k, v, dout, workspace)
+    B, H, L, d_feat = q.shape
+    d_v = v.shape[-1]
+    need = int(lib().based_prefill_backward_workspace_bytes(B, H, L))
+    if workspace is None or workspace.numel() * workspace.element_size() < need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    st = lib().based_prefill_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv), B, H, L,
+                                      d_feat, d_v, _dtype_code(q), int(flags), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "based_prefill_backward")
+    return dq, dk, dv
 
 
 def based_static_scratch_bytes() -> int:

@@ -238,6 +238,28 @@ based_status baseconv_gate_step(const void* a, const void* g, const float* h, co
                            static_cast<cudaStream_t>(cuda_stream));
 }
 
+size_t based_prefill_backward_workspace_bytes(int B, int H, int L) {
+    if (B <= 0 || H <= 0 || L <= 0) return 0;
+    return (size_t)B * H * L * 2 * sizeof(float);
+}
+
+based_status based_prefill_backward(const void* q, const void* k, const void* v, const void* dout, void* dq,
+                                    void* dk, void* dv, int B, int H, int L, int d_feat, int d_v, based_dtype io,
+                                    int flags, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!q || !k || !v || !dout || !dq || !dk || !dv || B <= 0 || H <= 0 || L <= 0) return BASED_ERR_INVALID_ARG;
+    if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
+    if (flags & ~BASED_NUMERATOR_ONLY) return BASED_ERR_INVALID_ARG;
+    if (dq == q || dq == k || dk == q || dk == k || dv == v || dv == dout) return BASED_ERR_INVALID_ARG;
+    if (d_feat != kDFeat || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) || !aligned16(dk) ||
+        !aligned16(dv) || !aligned16(workspace))
+        return BASED_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < based_prefill_backward_workspace_bytes(B, H, L)) return BASED_ERR_WORKSPACE;
+    return launch_prefill_backward(q, k, v, dout, dq, dk, dv, static_cast<float*>(workspace), B * H, L, d_v, io,
+                                   (flags & BASED_NUMERATOR_ONLY) ? 1 : 0, static_cast<cudaStream_t>(cuda_stream));
+}
+
 based_status based_preload_decode(void) {
     unsigned int* err = nullptr;
     based_status st = error_word_ptr(&err);

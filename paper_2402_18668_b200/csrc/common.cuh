@@ -93,6 +93,10 @@ based_status launch_swa_decode(const void* q, const void* k, const void* v, void
 // gated short convolution (BaseConv core); step: one token on a [B, width-1, C] state, N ignored
 based_status launch_baseconv(const void* a, const void* g, const float* h, const float* b2, void* state, void* out,
                              int B, int N, int C, int width, bool step, based_dtype io, cudaStream_t stream);
+// backward of the linear attention (fp32 FMA, quadratic form); stats: [BH, L] float2 scratch
+based_status launch_prefill_backward(const void* q, const void* k, const void* v, const void* g, void* dq, void* dk,
+                                     void* dv, float* stats, int BH, int L, int d_v, based_dtype io,
+                                     int numerator_only, cudaStream_t stream);
 // load the generation-step kernels into the current context
 based_status preload_decode();
 based_status preload_swa_decode();

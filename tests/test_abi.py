@@ -130,6 +130,20 @@ def test_baseconv_validation(lib):
     assert s(P, P, P, P, U, O, 1, 64, 3, 1, None) == 3
 
 
+def test_backward_validation(lib):
+    f = lib.based_prefill_backward
+    A = [ctypes.c_void_p(0x1000 * n) for n in range(1, 9)]
+    q, k, v, g, dq, dk, dv, ws = A
+    ok = (1, 1, 8, 16, 64, 1)
+    assert lib.based_prefill_backward_workspace_bytes(2, 3, 100) == 2 * 3 * 100 * 8
+    assert f(q, k, v, None, dq, dk, dv, *ok, 0, ws, 1 << 20, None) == 1            # output gradient missing
+    assert f(q, k, v, g, dq, dk, dv, *ok, 1, ws, 1 << 20, None) == 1               # CONTINUE is not a backward flag
+    assert f(q, k, v, g, q, dk, dv, *ok, 0, ws, 1 << 20, None) == 1                # gradient aliases an input
+    assert f(q, k, v, g, dq, dk, dv, 1, 1, 8, 16, 96, 1, 0, ws, 1 << 20, None) == 2
+    assert f(q, k, v, g, dq, dk, dv, *ok, 0, ws, 8, None) == 6                     # workspace too small
+    assert f(q, k, v, g, dq, dk, dv, *ok, 0, None, 0, None) == 6
+
+
 def test_binding_rejects_cpu_tensors():
     import torch
     from paper_2402_18668_b200 import binding

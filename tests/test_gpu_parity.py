@@ -188,6 +188,55 @@ def test_head_dim_112_prefill_continue_and_decode(dtype, L):
     _poll()
 
 
+# --------------------------------------------------------------------------- backward
+def _grad_err(got, want):
+    """Gradients are sums of many signed terms: compare per head against the head's largest entry.
+    Where the true gradient vanishes (one token: y = v whatever q and k are) the reference is
+    the difference of two O(1) terms (a.v and b), so the scale has a floor well below those terms."""
+    got, want = np.asarray(got, dtype=np.float64), np.asarray(want, dtype=np.float64)
+    assert np.isfinite(got).all()
+    g = got.reshape(got.shape[0] * got.shape[1], -1)
+    w = want.reshape(g.shape)
+    return float((np.abs(g - w).max(axis=1) / np.maximum(np.abs(w).max(axis=1), 5e-2)).max())
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("L,d_v", [(200, 64), (64, 128), (333, 112), (1, 64)])
+def test_prefill_backward_small(dtype, L, d_v):
+    B, H = 2, 2
+    w = wl.Workload("bwd", B, H, L, 16, d_v, dtype, 0.5)
+    gen = wl.generator(L * 3 + d_v)
+    q, k, v = wl.prefill_inputs(w, gen)
+    dout = torch.randn(B, H, L, d_v, generator=gen).to(q.dtype)
+    qd, kd, vd, gd = q.to(DEV), k.to(DEV), v.to(DEV), dout.to(DEV)
+    dq, dk, dv = based.based_prefill_backward(qd, kd, vd, gd)
+    _poll()
+    rq, rk, rv = oracle.linattn_backward(_np(q), _np(k), _np(v), _np(dout))
+    tol = tol_for(dtype)
+    assert _grad_err(_np(dq), rq) <= tol and _grad_err(_np(dk), rk) <= tol and _grad_err(_np(dv), rv) <= tol
+    # numerator-only variant (no forward output needed)
+    dq, dk, dv = based.based_prefill_backward(qd, kd, vd, gd, flags=based.BASED_NUMERATOR_ONLY)
+    rq, rk, rv = oracle.linattn_backward(_np(q), _np(k), _np(v), _np(dout), numerator_only=True)
+    assert _grad_err(_np(dq), rq) <= tol and _grad_err(_np(dk), rk) <= tol and _grad_err(_np(dv), rv) <= tol
+    _poll()
+
+
+def test_prefill_backward_cfg2_sampled_heads():
+    """Full 360M-layer shape (B4 H16 L2048 d_v64, bf16): two heads recomputed by the oracle."""
+    w = wl.CONFIGS["cfg2_360m_prefill"]
+    gen = wl.generator(77)
+    q, k, v = wl.prefill_inputs(w, gen)
+    dout = torch.randn(w.B, w.H, w.L, w.d_v, generator=gen).to(q.dtype)
+    qd, kd, vd, gd = q.to(DEV), k.to(DEV), v.to(DEV), dout.to(DEV)
+    dq, dk, dv = based.based_prefill_backward(qd, kd, vd, gd)
+    _poll()
+    for (b, h) in [(0, 0), (w.B - 1, w.H - 1)]:
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        rq, rk, rv = oracle.linattn_backward(_np(q[sl]), _np(k[sl]), _np(v[sl]), _np(dout[sl]))
+        assert _grad_err(_np(dq[sl]), rq) <= TOL_BF16 and _grad_err(_np(dk[sl]), rk) <= TOL_BF16
+        assert _grad_err(_np(dv[sl]), rv) <= TOL_BF16
+
+
 # --------------------------------------------------------------------------- numerator only
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("L,d_v", [(300, 64), (200, 128)])
