@@ -72,6 +72,9 @@ enum {
  * workspace device scratch of at least based_prefill_workspace_bytes(...) bytes
  *           (may be NULL when that size is 0); contents are undefined afterwards.
  * Supported: d_feat = 16; d_v in {64, 112, 128}; io in {F32, BF16}; any L >= 1.
+ * d_feat in {8, 24, 32} (the other dimensions of the paper's feature-map ablation; state rows
+ * D = 1 + d_feat + d_feat^2 = 73, 601, 1057) is served by fp32 definition-form kernels for
+ * both io dtypes: no workspace, no BASED_STATE_SYM, B*H <= 65535.
  * out must not alias an input.
  */
 based_status based_prefill(const void* q, const void* k, const void* v, void* out, float* kv_state,
@@ -90,7 +93,8 @@ size_t based_prefill_workspace_bytes(int B, int H, int L, int d_feat, int d_v, b
  *   out = phi(q) kv_state / (phi(q).z_state + 1e-12)
  *
  * q, k [B,H,d_feat], v, out [B,H,d_v] in the io dtype; kv_state / z_state as above,
- * updated IN PLACE.  Supported: d_feat = 16; d_v in {64, 112, 128}; io in {F32, BF16}.
+ * updated IN PLACE.  Supported: d_feat = 16; d_v in {64, 112, 128}; io in {F32, BF16}; also
+ * d_feat in {8, 24, 32} with D = 1 + d_feat + d_feat^2 state rows (plain streaming kernel).
  */
 based_status based_decode_step(const void* q, const void* k, const void* v, float* kv_state, float* z_state,
                                void* out, int B, int H, int d_feat, int d_v, based_dtype io,

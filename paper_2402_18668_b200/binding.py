@@ -333,8 +333,11 @@ def based_poll_error(stream=None) -> int:
     return int(lib().based_poll_error(_stream(stream)))
 
 
-def new_state(B: int, H: int, d_v: int, device="cuda", sym: bool = False):
-    """Zero-initialised (kv_state, z_state) in the ABI layout (273 rows, or the 153 symmetric ones)."""
-    D = D_SYM if sym else D_EXPANDED
+def new_state(B: int, H: int, d_v: int, device="cuda", sym: bool = False, d_feat: int = D_FEAT):
+    """Zero-initialised (kv_state, z_state) in the ABI layout (1 + d' + d'^2 rows: 273 for d' = 16; or
+    the 153 symmetric ones, d' = 16 only)."""
+    if sym and d_feat != D_FEAT:
+        raise ValueError("the symmetric format exists for d' = 16 only")
+    D = D_SYM if sym else 1 + d_feat + d_feat * d_feat
     return (torch.zeros(B, H, D, d_v, dtype=torch.float32, device=device),
             torch.zeros(B, H, D, dtype=torch.float32, device=device))

@@ -47,6 +47,8 @@ based_status check_launch(const char* what) {
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 // value head dimensions: 64 (360M-scale heads), 128, and 112 (the 1.3B configuration's 1792 / 16)
 static inline bool dv_ok(int d_v) { return d_v == 64 || d_v == 112 || d_v == 128; }
+// feature dimensions of the paper's ablation other than 16: served by the fp32 definition-form kernels
+static inline bool df_generic(int d_feat) { return d_feat == 8 || d_feat == 24 || d_feat == 32; }
 
 }  // namespace based
 
@@ -86,11 +88,16 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
     if ((kv_state == nullptr) != (z_state == nullptr)) return BASED_ERR_INVALID_ARG;
     if ((flags & BASED_STATE_CONTINUE) && !kv_state) return BASED_ERR_INVALID_ARG;
     if (out == q || out == k || out == v) return BASED_ERR_INVALID_ARG;
-    if (d_feat != kDFeat || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
+    if ((d_feat != kDFeat && !df_generic(d_feat)) || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
     if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
         !aligned16(z_state) || !aligned16(workspace))
         return BASED_ERR_ALIGNMENT;
+    if (d_feat != kDFeat) {
+        if ((flags & BASED_STATE_SYM) || (long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
+        return launch_prefill_generic(q, k, v, out, kv_state, z_state, B * H, L, d_feat, d_v, io, flags,
+                                      static_cast<cudaStream_t>(cuda_stream));
+    }
     const size_t need = based_prefill_workspace_bytes(B, H, L, d_feat, d_v, io);
     if (need > 0 && (!workspace || workspace_bytes < need)) return BASED_ERR_WORKSPACE;
     if ((long long)B * H > 65535 && io == BASED_BF16) return BASED_ERR_UNSUPPORTED;
@@ -105,11 +112,14 @@ based_status based_decode_step(const void* q, const void* k, const void* v, floa
                                void* out, int B, int H, int d_feat, int d_v, based_dtype io, void* cuda_stream) {
     if (!q || !k || !v || !out || !kv_state || !z_state || B <= 0 || H <= 0) return BASED_ERR_INVALID_ARG;
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
-    if (d_feat != kDFeat || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
+    if ((d_feat != kDFeat && !df_generic(d_feat)) || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
     if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
         !aligned16(z_state))
         return BASED_ERR_ALIGNMENT;
+    if (d_feat != kDFeat)
+        return launch_decode_generic(q, k, v, kv_state, z_state, out, B * H, d_feat, d_v, io, false,
+                                     static_cast<cudaStream_t>(cuda_stream));
     return launch_decode(q, k, v, kv_state, z_state, out, B * H, d_v, io, false, false,
                          static_cast<cudaStream_t>(cuda_stream));
 }
@@ -120,11 +130,16 @@ based_status based_decode_step_flags(const void* q, const void* k, const void* v
     if (!q || !k || !v || !out || !kv_state || !z_state || B <= 0 || H <= 0) return BASED_ERR_INVALID_ARG;
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
     if (flags & ~(BASED_STATE_SYM | BASED_NUMERATOR_ONLY)) return BASED_ERR_INVALID_ARG;
-    if (d_feat != kDFeat || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
+    if ((d_feat != kDFeat && !df_generic(d_feat)) || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
     if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
         !aligned16(z_state))
         return BASED_ERR_ALIGNMENT;
+    if (d_feat != kDFeat) {
+        if (flags & BASED_STATE_SYM) return BASED_ERR_UNSUPPORTED;
+        return launch_decode_generic(q, k, v, kv_state, z_state, out, B * H, d_feat, d_v, io,
+                                     (flags & BASED_NUMERATOR_ONLY) != 0, static_cast<cudaStream_t>(cuda_stream));
+    }
     return launch_decode(q, k, v, kv_state, z_state, out, B * H, d_v, io, (flags & BASED_STATE_SYM) != 0,
                          (flags & BASED_NUMERATOR_ONLY) != 0, static_cast<cudaStream_t>(cuda_stream));
 }

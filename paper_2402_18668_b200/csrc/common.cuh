@@ -97,6 +97,13 @@ based_status launch_baseconv(const void* a, const void* g, const float* h, const
 based_status launch_prefill_backward(const void* q, const void* k, const void* v, const void* g, void* dq, void* dk,
                                      void* dv, float* stats, int BH, int L, int d_v, based_dtype io,
                                      int numerator_only, cudaStream_t stream);
+// feature dimensions 8, 24, 32 (fp32 FMA, definition form); state layout [1 + d' + d'^2, d_v]
+based_status launch_prefill_generic(const void* q, const void* k, const void* v, void* out, float* kv, float* z,
+                                    int BH, int L, int d_feat, int d_v, based_dtype io, int flags,
+                                    cudaStream_t stream);
+based_status launch_decode_generic(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
+                                   int BH, int d_feat, int d_v, based_dtype io, bool numerator_only,
+                                   cudaStream_t stream);
 // load the generation-step kernels into the current context
 based_status preload_decode();
 based_status preload_swa_decode();

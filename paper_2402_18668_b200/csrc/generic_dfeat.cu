@@ -1,0 +1,332 @@
+// Feature dimensions other than 16: d' in {8, 24, 32} (the paper's feature-map ablation trains
+// Taylor maps of dimension 8, 16, 24 and 32, i.e. 73, 273, 601 and 1057 expanded features).
+// First correct path, fp32 FMAs only:
+//
+//   prefill   the definition form of Eq. (2), Sec. 4.1, tile by tile: 64 queries per CTA loop over
+//             the key tiles j <= i; scores (any d'), weights w = 1 + s/sqrt(d') + s^2/(2 d'), row
+//             sums, and the product of the weight tile (through shared memory) with the value
+//             tile.  A given initial state adds phi(q_i).S0 and phi(q_i).z0 per row.
+//   state     S = S0 + sum_j phi(k_j) v_j^T, z = z0 + sum_j phi(k_j): one CTA per (head, 32 features).
+//   decode    the recurrent step as a plain stream over the [D, d_v] state, D = 1 + d' + d'^2.
+//
+// The state layout is the 273-row layout's generalisation: constant, linear terms, row-major
+// outer product.  The tensor-core kernels and the symmetric format exist for d' = 16 only.
+#include "common.cuh"
+
+namespace based {
+
+namespace {
+constexpr int kT = 64;             // tile edge
+constexpr int kBT = 128;           // threads: 16 row groups (4 rows) x 8 column lanes
+constexpr int kMaxDF = 32;
+constexpr int kQP = kMaxDF + 1;    // padded row length of q/k tiles
+
+__host__ __device__ constexpr int expanded_dim(int df) { return 1 + df + df * df; }
+
+struct FeatScale { float lin, quad, s1, s2; };      // x/d'^(1/4), x x/(sqrt2 sqrt d'), s/sqrt d', s^2/(2 d')
+__device__ __forceinline__ FeatScale feat_scale(int df) {
+    const float rd = sqrtf((float)df);
+    return {rsqrtf(rd), 1.0f / (1.41421356237309505f * rd), 1.0f / rd, 0.5f / (float)df};
+}
+// expanded feature f of x[df]
+__device__ __forceinline__ float phi_gen(const float* x, int df, int f, const FeatScale& sc) {
+    if (f == 0) return 1.0f;
+    if (f <= df) return x[f - 1] * sc.lin;
+    const int p = f - 1 - df;
+    return x[p / df] * x[p % df] * sc.quad;
+}
+
+template <int DV> struct FwdSmem {
+    float q[kT][kQP];
+    float k[kT][kQP];
+    float v[kT][DV + 1];
+    float w[kT][kT + 1];           // weights of the current tile [query][key]
+};
+
+template <typename T>
+__device__ __forceinline__ void load_rows(const T* __restrict__ src, int r0, int L, int W, float* dst, int pitch) {
+    for (int i = threadIdx.x; i < kT * W; i += kBT) {
+        const int r = i / W, c = i - r * W;
+        dst[r * pitch + c] = r0 + r < L ? to_f32(src[(size_t)(r0 + r) * W + c]) : 0.f;
+    }
+}
+}  // namespace
+
+template <typename T, int DV>
+__global__ void __launch_bounds__(kBT) generic_prefill_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                              const T* __restrict__ v, T* __restrict__ out,
+                                                              const float* __restrict__ kv0,
+                                                              const float* __restrict__ z0, int L, int df,
+                                                              int numerator_only) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    FwdSmem<DV>& sm = *reinterpret_cast<FwdSmem<DV>*>(smem_raw);
+    const int i0 = (gridDim.x - 1 - blockIdx.x) * kT;       // longest loops first
+    const size_t head = blockIdx.y;
+    const int ty = threadIdx.x >> 3, tx = threadIdx.x & 7;
+    const FeatScale sc = feat_scale(df);
+    const int D = expanded_dim(df);
+    constexpr int NC = DV / 8;
+    load_rows<T>(q + head * (size_t)L * df, i0, L, df, &sm.q[0][0], kQP);
+    float num[4][NC], den[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < NC; ++c) num[r][c] = 0.f;
+    for (int j0 = 0; j0 <= i0; j0 += kT) {
+        __syncthreads();
+        load_rows<T>(k + head * (size_t)L * df, j0, L, df, &sm.k[0][0], kQP);
+        load_rows<T>(v + head * (size_t)L * DV, j0, L, DV, &sm.v[0][0], DV + 1);
+        __syncthreads();
+        float s[4][8];
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int n = 0; n < 8; ++n) s[r][n] = 0.f;
+        for (int m = 0; m < df; ++m) {
+            float qa[4], kb[8];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) qa[r] = sm.q[ty * 4 + r][m];
+#pragma unroll
+            for (int n = 0; n < 8; ++n) kb[n] = sm.k[tx + 8 * n][m];
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int n = 0; n < 8; ++n) s[r][n] = fmaf(qa[r], kb[n], s[r][n]);
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int n = 0; n < 8; ++n) {
+                const bool live = j0 + tx + 8 * n <= i0 + ty * 4 + r;
+                const float sv = s[r][n];
+                const float w = live ? fmaf(sv, fmaf(sv, sc.s2, sc.s1), 1.0f) : 0.f;
+                den[r] += w;
+                sm.w[ty * 4 + r][tx + 8 * n] = w;
+            }
+        __syncthreads();
+#pragma unroll 4
+        for (int j = 0; j < kT; ++j) {
+            float ww[4], vv[NC];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) ww[r] = sm.w[ty * 4 + r][j];
+#pragma unroll
+            for (int c = 0; c < NC; ++c) vv[c] = sm.v[j][tx + 8 * c];
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int c = 0; c < NC; ++c) num[r][c] = fmaf(ww[r], vv[c], num[r][c]);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        den[r] += __shfl_xor_sync(0xffffffffu, den[r], 1);
+        den[r] += __shfl_xor_sync(0xffffffffu, den[r], 2);
+        den[r] += __shfl_xor_sync(0xffffffffu, den[r], 4);
+    }
+    // contribution of a given initial state: phi(q_i).S0 and phi(q_i).z0
+    if (kv0 != nullptr) {
+        const float* S0 = kv0 + head * (size_t)D * DV;
+        const float* Z0 = z0 + head * (size_t)D;
+        for (int f = 0; f < D; ++f) {
+            float pf[4], srow[NC];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) pf[r] = phi_gen(sm.q[ty * 4 + r], df, f, sc);
+#pragma unroll
+            for (int c = 0; c < NC; ++c) srow[c] = S0[(size_t)f * DV + tx + 8 * c];
+            const float zf = Z0[f];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                den[r] = fmaf(pf[r], zf, den[r]);
+#pragma unroll
+                for (int c = 0; c < NC; ++c) num[r][c] = fmaf(pf[r], srow[c], num[r][c]);
+            }
+        }
+    }
+    T* oh = out + head * (size_t)L * DV;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const int i = i0 + ty * 4 + r;
+        if (i >= L) continue;
+        const float inv = numerator_only ? 1.0f : 1.0f / (den[r] + kEps);
+#pragma unroll
+        for (int c = 0; c < NC; ++c) oh[(size_t)i * DV + tx + 8 * c] = from_f32<T>(num[r][c] * inv);
+    }
+}
+
+// S[f, :] = S0[f, :] + sum_j phi_f(k_j) v_j, z[f] likewise; one CTA per (32 features, head), one thread per
+// value column plus one warp-less extra thread for z (thread DV).
+template <typename T, int DV>
+__global__ void __launch_bounds__(DV + 32) generic_state_kernel(const T* __restrict__ k, const T* __restrict__ v,
+                                                                float* __restrict__ kv, float* __restrict__ z, int L,
+                                                                int df, int accumulate) {
+    constexpr int FB = 32, TOK = 32;
+    __shared__ float s_k[TOK][kMaxDF];
+    __shared__ float s_v[TOK][DV];
+    const int f0 = blockIdx.x * FB;
+    const size_t head = blockIdx.y;
+    const int D = expanded_dim(df);
+    const FeatScale sc = feat_scale(df);
+    const int c = threadIdx.x;                       // value column, or DV for the K-state
+    const bool active = c <= DV;
+    float acc[FB];
+#pragma unroll
+    for (int r = 0; r < FB; ++r) acc[r] = 0.f;
+    const T* kh = k + head * (size_t)L * df;
+    const T* vh = v + head * (size_t)L * DV;
+    for (int t0 = 0; t0 < L; t0 += TOK) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < TOK * df; i += DV + 32) {
+            const int t = i / df, m = i - t * df;
+            s_k[t][m] = t0 + t < L ? to_f32(kh[(size_t)(t0 + t) * df + m]) : 0.f;
+        }
+        for (int i = threadIdx.x; i < TOK * DV; i += DV + 32) {
+            const int t = i / DV, cc = i - t * DV;
+            s_v[t][cc] = t0 + t < L ? to_f32(vh[(size_t)(t0 + t) * DV + cc]) : 0.f;
+        }
+        __syncthreads();
+        if (active) {
+            const int nt = min(TOK, L - t0);
+            for (int t = 0; t < nt; ++t) {
+                const float vc = c < DV ? s_v[t][c] : 1.0f;
+#pragma unroll
+                for (int r = 0; r < FB; ++r) {
+                    const int f = f0 + r;
+                    if (f < D) acc[r] = fmaf(phi_gen(s_k[t], df, f, sc), vc, acc[r]);
+                }
+            }
+        }
+    }
+    if (active) {
+#pragma unroll
+        for (int r = 0; r < FB; ++r) {
+            const int f = f0 + r;
+            if (f >= D) continue;
+            float* dst = c < DV ? &kv[(head * D + f) * DV + c] : &z[head * D + f];
+            *dst = accumulate ? *dst + acc[r] : acc[r];
+        }
+    }
+}
+
+// one recurrent step on the [D, d_v] state of a head (update, then read)
+template <typename T>
+__global__ void __launch_bounds__(256) generic_decode_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                             const T* __restrict__ v, float* __restrict__ kv,
+                                                             float* __restrict__ z, T* __restrict__ out, int df,
+                                                             int dv, int numerator_only) {
+    __shared__ float s_x[2][kMaxDF];
+    __shared__ float s_pq[1 + kMaxDF + kMaxDF * kMaxDF], s_pk[1 + kMaxDF + kMaxDF * kMaxDF];
+    __shared__ __align__(16) float s_num[8][128];      // written with 16-byte stores
+    __shared__ float s_den[8];
+    const int tid = threadIdx.x;
+    const size_t head = blockIdx.x;
+    const int D = expanded_dim(df);
+    const FeatScale sc = feat_scale(df);
+    if (tid < df) s_x[0][tid] = to_f32(q[head * df + tid]);
+    else if (tid >= 32 && tid < 32 + df) s_x[1][tid - 32] = to_f32(k[head * df + tid - 32]);
+    __syncthreads();
+    for (int f = tid; f < D; f += 256) {
+        s_pq[f] = phi_gen(s_x[0], df, f, sc);
+        s_pk[f] = phi_gen(s_x[1], df, f, sc);
+    }
+    __syncthreads();
+    float dpart = 0.f;
+    float* zh = z + head * (size_t)D;
+    for (int f = tid; f < D; f += 256) {
+        const float zn = zh[f] + s_pk[f];
+        zh[f] = zn;
+        dpart = fmaf(s_pq[f], zn, dpart);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dpart += __shfl_xor_sync(0xffffffffu, dpart, o);
+    if ((tid & 31) == 0) s_den[tid >> 5] = dpart;
+    // 32 column lanes (4 columns each for d_v 128; fewer are live for narrower heads) x 8 row slots
+    const int c4 = tid & 31, rslot = tid >> 5;
+    const bool live = c4 * 4 < dv;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), vv = acc;
+    if (live) {
+        vv.x = to_f32(v[head * dv + c4 * 4]); vv.y = to_f32(v[head * dv + c4 * 4 + 1]);
+        vv.z = to_f32(v[head * dv + c4 * 4 + 2]); vv.w = to_f32(v[head * dv + c4 * 4 + 3]);
+        float* S = kv + head * (size_t)D * dv + c4 * 4;
+        for (int r = rslot; r < D; r += 8) {
+            float4 s = *reinterpret_cast<float4*>(S + (size_t)r * dv);
+            const float pk = s_pk[r], pq = s_pq[r];
+            s.x = fmaf(pk, vv.x, s.x); s.y = fmaf(pk, vv.y, s.y); s.z = fmaf(pk, vv.z, s.z); s.w = fmaf(pk, vv.w, s.w);
+            acc.x = fmaf(pq, s.x, acc.x); acc.y = fmaf(pq, s.y, acc.y);
+            acc.z = fmaf(pq, s.z, acc.z); acc.w = fmaf(pq, s.w, acc.w);
+            *reinterpret_cast<float4*>(S + (size_t)r * dv) = s;
+        }
+    }
+    *reinterpret_cast<float4*>(&s_num[rslot][c4 * 4]) = acc;
+    __syncthreads();
+    if (tid < dv) {
+        float num = 0.f, den = 0.f;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            num += s_num[r][tid];
+            den += s_den[r];
+        }
+        out[head * dv + tid] = from_f32<T>(numerator_only ? num : num / (den + kEps));
+    }
+}
+
+template <typename T, int DV>
+static based_status prefill_t(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH,
+                              int L, int df, int flags, cudaStream_t stream) {
+    const size_t smem = sizeof(FwdSmem<DV>);
+    {
+        static bool configured[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BASED_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(setup_mutex());
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(generic_prefill_kernel<T, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem) != cudaSuccess)
+                return BASED_ERR_CUDA;
+            configured[dev] = true;
+        }
+    }
+    const bool cont = (flags & BASED_STATE_CONTINUE) != 0;
+    const T* qq = static_cast<const T*>(q);
+    const T* kk = static_cast<const T*>(k);
+    const T* vv = static_cast<const T*>(v);
+    generic_prefill_kernel<T, DV><<<dim3((L + kT - 1) / kT, BH), kBT, smem, stream>>>(
+        qq, kk, vv, static_cast<T*>(out), cont ? kv : nullptr, cont ? z : nullptr, L, df,
+        (flags & BASED_NUMERATOR_ONLY) ? 1 : 0);
+    note_launch();
+    based_status st = check_launch("generic_prefill_kernel");
+    if (st != BASED_OK || kv == nullptr) return st;
+    const int D = expanded_dim(df);
+    generic_state_kernel<T, DV><<<dim3((D + 31) / 32, BH), DV + 32, 0, stream>>>(kk, vv, kv, z, L, df, cont ? 1 : 0);
+    note_launch();
+    return check_launch("generic_state_kernel");
+}
+
+based_status launch_prefill_generic(const void* q, const void* k, const void* v, void* out, float* kv, float* z,
+                                    int BH, int L, int d_feat, int d_v, based_dtype io, int flags,
+                                    cudaStream_t stream) {
+    if (io == BASED_F32) {
+        if (d_v == 64) return prefill_t<float, 64>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
+        if (d_v == 112) return prefill_t<float, 112>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
+        return prefill_t<float, 128>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
+    }
+    if (d_v == 64) return prefill_t<__nv_bfloat16, 64>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
+    if (d_v == 112) return prefill_t<__nv_bfloat16, 112>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
+    return prefill_t<__nv_bfloat16, 128>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
+}
+
+based_status launch_decode_generic(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
+                                   int BH, int d_feat, int d_v, based_dtype io, bool numerator_only,
+                                   cudaStream_t stream) {
+    if (io == BASED_F32)
+        generic_decode_kernel<float><<<BH, 256, 0, stream>>>(static_cast<const float*>(q), static_cast<const float*>(k),
+                                                             static_cast<const float*>(v), kv, z,
+                                                             static_cast<float*>(out), d_feat, d_v, numerator_only);
+    else
+        generic_decode_kernel<__nv_bfloat16><<<BH, 256, 0, stream>>>(
+            static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
+            static_cast<const __nv_bfloat16*>(v), kv, z, static_cast<__nv_bfloat16*>(out), d_feat, d_v, numerator_only);
+    note_launch();
+    return check_launch("generic_decode_kernel");
+}
+
+}  // namespace based

@@ -60,7 +60,7 @@ def test_prefill_validation(lib):
     assert call(kv=P, z=None) == 1                      # state pointers come in pairs
     assert call(flags=1) == 1                           # CONTINUE needs a state
     assert call(out=P) == 1                             # out aliases q
-    assert call(d_feat=8) == 2
+    assert call(d_feat=12) == 2                         # 8, 16, 24, 32 are the supported feature dimensions
     assert call(d_v=96) == 2
     assert call(q=U) == 3
 
@@ -99,7 +99,7 @@ def test_sym_state_validation(lib):
     assert pf(P, P, P, O2, None, None, 1, 1, 8, 16, 64, 1, 3, None, 0, None) == 1     # continue without a state
     d = lib.based_decode_step_sym
     assert d(P, P, P, None, P, P, 1, 1, 16, 64, 0, None) == 1
-    assert d(P, P, P, P, P, P, 1, 1, 8, 64, 0, None) == 2                    # d' other than 16
+    assert d(P, P, P, P, P, P, 1, 1, 8, 64, 0, None) == 2                    # the symmetric format is d' = 16 only
     assert d(P, P, P, P, U, P, 1, 1, 16, 64, 0, None) == 3
     O = ctypes.c_void_p(0x2000)
     for f in (lib.based_state_to_sym, lib.based_state_from_sym):

@@ -237,6 +237,38 @@ def test_prefill_backward_cfg2_sampled_heads():
         assert _grad_err(_np(dv[sl]), rv) <= TOL_BF16
 
 
+# --------------------------------------------------------------------------- other feature dimensions
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d_feat,L,d_v", [(8, 200, 64), (24, 130, 128), (32, 77, 112), (8, 1, 64)])
+def test_other_feature_dimensions_prefill_continue_decode(dtype, d_feat, L, d_v):
+    """d' in {8, 24, 32} (feature-map ablation): prefill in two calls with state hand-over, then decode
+    steps, against the oracle's definition form; final state against the oracle's."""
+    B, H, T = 2, 2, 3
+    w = wl.Workload("dfeat", B, H, L + T, d_feat, d_v, dtype, 0.5)
+    q, k, v = wl.prefill_inputs(w, wl.generator(d_feat * 1000 + L))
+    y_ref, _, _ = oracle.linattn_quadratic(_np(q), _np(k), _np(v), return_state=False)
+    _, S_ref, z_ref = oracle.linattn_recurrent(_np(q[:, :, :L]), _np(k[:, :, :L]), _np(v[:, :, :L]))
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    tol = tol_for(dtype)
+    kv, z = based.new_state(B, H, d_v, d_feat=d_feat)
+    assert kv.shape[2] == 1 + d_feat + d_feat * d_feat
+    half = L // 2
+    outs = []
+    if half > 0:
+        outs.append(based.based_prefill(qd[:, :, :half].contiguous(), kd[:, :, :half].contiguous(),
+                                        vd[:, :, :half].contiguous(), kv_state=kv, z_state=z))
+    outs.append(based.based_prefill(qd[:, :, half:L].contiguous(), kd[:, :, half:L].contiguous(),
+                                    vd[:, :, half:L].contiguous(), kv_state=kv, z_state=z,
+                                    flags=based.BASED_STATE_CONTINUE if half > 0 else based.BASED_STATE_ZERO_INIT))
+    out = torch.cat(outs, dim=2)
+    assert row_err(_np(out), y_ref[:, :, :L]) <= tol
+    assert head_err(_np(kv), S_ref) <= tol and head_err(_np(z), z_ref) <= tol
+    for t in range(L, L + T):
+        o = based.based_decode_step(qd[:, :, t].contiguous(), kd[:, :, t].contiguous(), vd[:, :, t].contiguous(), kv, z)
+        assert row_err(_np(o), y_ref[:, :, t]) <= tol, f"token {t}"
+    _poll()
+
+
 # --------------------------------------------------------------------------- numerator only
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("L,d_v", [(300, 64), (200, 128)])
