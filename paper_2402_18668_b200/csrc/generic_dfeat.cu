@@ -154,20 +154,32 @@ __global__ void __launch_bounds__(kBT) generic_prefill_kernel(const T* __restric
 }
 
 // S[f, :] = S0[f, :] + sum_j phi_f(k_j) v_j, z[f] likewise; one CTA per (32 features, head), one thread per
-// value column plus one warp-less extra thread for z (thread DV).
+// value column plus one for z (thread DV).  Per block of 32 tokens the 32 x 32 feature values are
+// expanded once into shared memory by all threads, then every column thread accumulates from there.
 template <typename T, int DV>
 __global__ void __launch_bounds__(DV + 32) generic_state_kernel(const T* __restrict__ k, const T* __restrict__ v,
                                                                 float* __restrict__ kv, float* __restrict__ z, int L,
                                                                 int df, int accumulate) {
-    constexpr int FB = 32, TOK = 32;
-    __shared__ float s_k[TOK][kMaxDF];
+    constexpr int FB = 32, TOK = 32, NT = DV + 32;
+    __shared__ float s_k[TOK][kMaxDF + 1];
     __shared__ float s_v[TOK][DV];
+    __shared__ __align__(16) float s_phi[TOK][FB];
+    __shared__ int s_m[FB], s_n[FB];                 // feature -> (m, n) of the product, or (-1, -1) constant, (m, -1) linear
+    __shared__ float s_scale[FB];
     const int f0 = blockIdx.x * FB;
     const size_t head = blockIdx.y;
     const int D = expanded_dim(df);
     const FeatScale sc = feat_scale(df);
     const int c = threadIdx.x;                       // value column, or DV for the K-state
     const bool active = c <= DV;
+    if (threadIdx.x < FB) {
+        const int f = f0 + threadIdx.x;
+        int m = -1, n = -1;
+        float scale = f < D ? 1.0f : 0.0f;           // rows past the end contribute nothing
+        if (f >= 1 && f <= df) { m = f - 1; scale = sc.lin; }
+        else if (f > df && f < D) { m = (f - 1 - df) / df; n = (f - 1 - df) % df; scale = sc.quad; }
+        s_m[threadIdx.x] = m; s_n[threadIdx.x] = n; s_scale[threadIdx.x] = scale;
+    }
     float acc[FB];
 #pragma unroll
     for (int r = 0; r < FB; ++r) acc[r] = 0.f;
@@ -175,23 +187,35 @@ __global__ void __launch_bounds__(DV + 32) generic_state_kernel(const T* __restr
     const T* vh = v + head * (size_t)L * DV;
     for (int t0 = 0; t0 < L; t0 += TOK) {
         __syncthreads();
-        for (int i = threadIdx.x; i < TOK * df; i += DV + 32) {
+        for (int i = threadIdx.x; i < TOK * df; i += NT) {
             const int t = i / df, m = i - t * df;
             s_k[t][m] = t0 + t < L ? to_f32(kh[(size_t)(t0 + t) * df + m]) : 0.f;
         }
-        for (int i = threadIdx.x; i < TOK * DV; i += DV + 32) {
+        for (int i = threadIdx.x; i < TOK * DV; i += NT) {
             const int t = i / DV, cc = i - t * DV;
             s_v[t][cc] = t0 + t < L ? to_f32(vh[(size_t)(t0 + t) * DV + cc]) : 0.f;
         }
         __syncthreads();
+        for (int i = threadIdx.x; i < TOK * FB; i += NT) {
+            const int t = i / FB, r = i - t * FB;
+            const int m = s_m[r], n = s_n[r];
+            float x = s_scale[r];
+            if (m >= 0) x *= s_k[t][m];
+            if (n >= 0) x *= s_k[t][n];
+            s_phi[t][r] = t0 + t < L ? x : 0.f;      // tokens past the end: also no constant feature
+        }
+        __syncthreads();
         if (active) {
-            const int nt = min(TOK, L - t0);
-            for (int t = 0; t < nt; ++t) {
+#pragma unroll 4
+            for (int t = 0; t < TOK; ++t) {
                 const float vc = c < DV ? s_v[t][c] : 1.0f;
 #pragma unroll
-                for (int r = 0; r < FB; ++r) {
-                    const int f = f0 + r;
-                    if (f < D) acc[r] = fmaf(phi_gen(s_k[t], df, f, sc), vc, acc[r]);
+                for (int r4 = 0; r4 < FB / 4; ++r4) {
+                    const float4 p = *reinterpret_cast<const float4*>(&s_phi[t][r4 * 4]);
+                    acc[r4 * 4 + 0] = fmaf(p.x, vc, acc[r4 * 4 + 0]);
+                    acc[r4 * 4 + 1] = fmaf(p.y, vc, acc[r4 * 4 + 1]);
+                    acc[r4 * 4 + 2] = fmaf(p.z, vc, acc[r4 * 4 + 2]);
+                    acc[r4 * 4 + 3] = fmaf(p.w, vc, acc[r4 * 4 + 3]);
                 }
             }
         }
