@@ -468,28 +468,32 @@ def bench_baseconv(shape, steps, warmup, torch, based, dist_on, peaks):
 
 
 def bench_backward(w, steps, warmup, torch, based, dist_on, peaks):
-    """Backward pass of the linear attention (fp32 FMA path, quadratic form) on the workload's shape.
-    Bound by the fp32 pipe: peak = SMs x 128 lanes x 2 flop x SM clock (148 x 128 x 2 x 1.965 GHz)."""
+    """Backward pass of the linear attention (quadratic form) on the workload's shape: bf16 io runs on
+    the tensor cores, fp32 io on the fp32 pipe (peak = SMs x 128 lanes x 2 flop x SM clock)."""
     g = torch.Generator(device="cuda").manual_seed(8)
     dt = w.torch_dtype
     q = (torch.randn(w.B, w.H, w.L, w.d_feat, generator=g, device="cuda") * w.qk_scale).to(dt)
     k = (torch.randn(w.B, w.H, w.L, w.d_feat, generator=g, device="cuda") * w.qk_scale).to(dt)
     v = torch.randn(w.B, w.H, w.L, w.d_v, generator=g, device="cuda").to(dt)
     dout = torch.randn(w.B, w.H, w.L, w.d_v, generator=g, device="cuda").to(dt)
-    ws = torch.empty(w.B * w.H * w.L * 8, dtype=torch.uint8, device="cuda")
+    bf16 = w.dtype == "bf16"
+    ws = torch.empty(based.lib().based_prefill_backward_workspace_bytes(w.B, w.H, w.L, w.d_v, 1 if bf16 else 0),
+                     dtype=torch.uint8, device="cuda")
     n0 = based.launch_count()
     ms = time_region(lambda i: based.based_prefill_backward(q, k, v, dout, workspace=ws), steps, warmup, torch, dist_on)
+    assert based.based_poll_error() == 0
     t = ms * 1e-3 / steps
     pairs = w.B * w.H * w.L * (w.L + 1) / 2.0
-    flops = 2.0 * pairs * (80 + 4 * w.d_v)              # 3 score passes, 3 a.v passes + dv, dq and dk updates
-    alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12
+    flops = 2.0 * pairs * (80 + 4 * w.d_v)              # 3 score passes, 3 dout.v passes + dv, dq and dk updates
+    peak = peaks["bf16_tflops"] if bf16 else 148 * 128 * 2 * 1.965e9 / 1e12
     return {
-        "workload": w.name + " backward (fp32 FMA, quadratic form)", "metric": "backward_tokens_per_s",
-        "value": w.B * w.L / t, "unit": "tokens/s", "ms_per_step": t * 1e3, "steps": steps,
-        "launches_per_step": (based.launch_count() - n0) // (steps + warmup),
-        "roofline": {"bound": "alu", "achieved": flops / t / 1e12, "peak": alu_peak, "unit": "TFLOP/s",
-                     "frac": flops / t / 1e12 / alu_peak, "traffic": None, "kernel": "bwd_dkdv_kernel",
-                     "algorithmic_flops": flops, "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz"},
+        "workload": w.name + (" backward (tensor cores, quadratic form)" if bf16 else " backward (fp32 FMA, quadratic form)"),
+        "metric": "backward_tokens_per_s", "value": w.B * w.L / t, "unit": "tokens/s", "ms_per_step": t * 1e3,
+        "steps": steps, "launches_per_step": (based.launch_count() - n0) // (steps + warmup),
+        "roofline": {"bound": "tensor" if bf16 else "alu", "achieved": flops / t / 1e12, "peak": peak,
+                     "unit": "TFLOP/s", "frac": flops / t / 1e12 / peak, "traffic": None,
+                     "kernel": "backward_tc_kernel" if bf16 else "bwd_dkdv_kernel", "algorithmic_flops": flops,
+                     "peak_source": peaks["source"] if bf16 else "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz"},
     }
 
 

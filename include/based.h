@@ -182,15 +182,16 @@ based_status swa_decode_step(const void* q, const void* k, const void* v, void* 
  * (the forward output is not an argument: out_i is recomputed in fp32, because a_i.v_j + b_i
  * cancels almost completely for short prefixes and a rounded out would dominate the result).
  * flags: 0, or BASED_NUMERATOR_ONLY for the backward of the numerator-only forward.
- * workspace: at least based_prefill_backward_workspace_bytes(B, H, L) bytes of device scratch.
+ * workspace: at least based_prefill_backward_workspace_bytes(B, H, L, d_v, io) bytes of device scratch.
  * Supported: d_feat = 16; d_v in {64, 112, 128}; io in {F32, BF16}; B*H <= 65535.
- * This path evaluates the quadratic form with fp32 FMAs (O(L^2) per head): a correct first
- * implementation, not a tensor-core kernel.  Gradient outputs must not alias inputs.
+ * Both paths evaluate the quadratic form, O(L^2) per head, on 128 x 128 (bf16 io: tcgen05 tensor
+ * cores, bf16 operands, fp32 accumulation) or 64 x 64 (fp32 io: fp32 FMAs) tiles of (query, key)
+ * pairs.  Gradient outputs must not alias inputs.
  */
 based_status based_prefill_backward(const void* q, const void* k, const void* v, const void* dout, void* dq,
                                     void* dk, void* dv, int B, int H, int L, int d_feat, int d_v, based_dtype io,
                                     int flags, void* workspace, size_t workspace_bytes, void* cuda_stream);
-size_t based_prefill_backward_workspace_bytes(int B, int H, int L);
+size_t based_prefill_backward_workspace_bytes(int B, int H, int L, int d_v, based_dtype io);
 
 /*
  * The gated short convolution at the core of the BaseConv layer (App. "Extended Architecture

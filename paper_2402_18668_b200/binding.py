@@ -79,7 +79,7 @@ def lib() -> ctypes.CDLL:
         L.based_prefill_backward.restype = i
         L.based_prefill_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
         L.based_prefill_backward_workspace_bytes.restype = sz
-        L.based_prefill_backward_workspace_bytes.argtypes = [i, i, i]
+        L.based_prefill_backward_workspace_bytes.argtypes = [i, i, i, i, i]
         L.baseconv_gate_forward.restype = i
         L.baseconv_gate_forward.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
         L.baseconv_gate_step.restype = i
@@ -168,7 +168,7 @@ def based_prefill_backward(q, k, v, dout, flags: int = 0, workspace=None, stream
     _dev(q, k, v, dout, workspace)
     B, H, L, d_feat = q.shape
     d_v = v.shape[-1]
-    need = int(lib().based_prefill_backward_workspace_bytes(B, H, L))
+    need = int(lib().based_prefill_backward_workspace_bytes(B, H, L, d_v, _dtype_code(q)))
     if workspace is None or workspace.numel() * workspace.element_size() < need:
         workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
     dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)

@@ -253,8 +253,9 @@ based_status baseconv_gate_step(const void* a, const void* g, const float* h, co
                            static_cast<cudaStream_t>(cuda_stream));
 }
 
-size_t based_prefill_backward_workspace_bytes(int B, int H, int L) {
-    if (B <= 0 || H <= 0 || L <= 0) return 0;
+size_t based_prefill_backward_workspace_bytes(int B, int H, int L, int d_v, based_dtype io) {
+    if (B <= 0 || H <= 0 || L <= 0 || !dv_ok(d_v)) return 0;
+    if (io == BASED_BF16) return backward_tc_workspace_bytes(B * H, L, d_v);
     return (size_t)B * H * L * 2 * sizeof(float);
 }
 
@@ -270,7 +271,12 @@ based_status based_prefill_backward(const void* q, const void* k, const void* v,
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) || !aligned16(dk) ||
         !aligned16(dv) || !aligned16(workspace))
         return BASED_ERR_ALIGNMENT;
-    if (!workspace || workspace_bytes < based_prefill_backward_workspace_bytes(B, H, L)) return BASED_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < based_prefill_backward_workspace_bytes(B, H, L, d_v, io))
+        return BASED_ERR_WORKSPACE;
+    if (io == BASED_BF16)
+        return launch_prefill_backward_tc(q, k, v, dout, dq, dk, dv, static_cast<float*>(workspace), B * H, L, d_v,
+                                          (flags & BASED_NUMERATOR_ONLY) ? 1 : 0,
+                                          static_cast<cudaStream_t>(cuda_stream));
     return launch_prefill_backward(q, k, v, dout, dq, dk, dv, static_cast<float*>(workspace), B * H, L, d_v, io,
                                    (flags & BASED_NUMERATOR_ONLY) ? 1 : 0, static_cast<cudaStream_t>(cuda_stream));
 }

@@ -1,0 +1,430 @@
+// based_prefill_backward, bf16 tensor-core path (tcgen05 / TMEM / TMA): the same three passes as
+// the fp32 path (row statistics, dq, dk + dv; see backward_simt.cu for the formulas), with every
+// 128 x 128 tile of (query, key) pairs evaluated by tensor-core products:
+//
+//   S  = Q_i K_j^T          (K = 16)          GV = G_i V_j^T   (K = d_v; G = dout, exact in bf16)
+//   dq:   DS = (GV / D_i + b_i)(1/4 + S/16) [j<=i]  as bf16 in tensor memory,   dQ_i += DS K_j
+//   dk/dv: the transposed products S^T = K_j Q_i^T, GV^T = V_j G_i^T;  W'^T = w(S^T) / D_i and DS^T in
+//          tensor memory (over the scores, in place);   dV_j += W'^T G_i,   dK_j += DS^T Q_i
+// 1/D_i is applied to the fp32 products, not to the operand: a = dout / D rounded to bf16 would
+// break the near-cancellation of a_i.v_j + b_i for short prefixes.
+//
+// One CTA per (head, 128-row tile), 160 threads: warps 0-3 own one accumulator row each (the
+// polynomial, masks and bf16 packing), lane 0 of warp 4 issues TMA loads and MMAs.  The loop over
+// the other side's tiles is sequential per CTA (loads of the next tile are in flight during the
+// current one); parallelism comes from the (tile, head) grid.  q and k tiles are loaded 32
+// columns wide (columns 16..31 are zero-filled by TMA) so that they serve both as K-major
+// operands of the scores and as MN-major B operands of dQ / dK.  The work is O(L^2) per head, as
+// in the fp32 path.
+#include <mutex>
+
+#include "common.cuh"
+#include "sm100.cuh"
+
+namespace based {
+using namespace sm100;
+
+namespace {
+constexpr int kTile = 128;
+constexpr int kThreadsB = 160;
+constexpr int kModeStats = 0, kModeDq = 1, kModeDkDv = 2;
+constexpr uint32_t kQKTile = kTile * 64;                 // [128][32] bf16, 64-byte rows, SWIZZLE_64B
+
+template <int DV> struct BCfg {
+    static constexpr int kVB = (DV + 63) / 64;           // 64-column blocks of a [128][DV] tile (112 -> 2, second partly zero)
+    static constexpr uint32_t kWide = kVB * kTile * 128; // [128][64 * kVB] bf16 in SWIZZLE_128B blocks
+    // shared memory: resident narrow + wide tile, two stages of (narrow + wide), b of two stages, barriers
+    static constexpr uint32_t offResN = 0, offResW = offResN + kQKTile;
+    static constexpr uint32_t offStage = offResW + kWide, kStage = kQKTile + kWide;
+    static constexpr uint32_t offB = offStage + 2 * kStage;
+    static constexpr uint32_t offMisc = offB + 2 * kTile * 8;      // (1/D, b) of the looped queries, two stages
+    static constexpr uint32_t kSmem = offMisc + 256 + 1024;
+    // tensor memory columns
+    static constexpr uint32_t colS = 0, colG = 128, colD = 256, colAcc = 320, colK = 448;   // colAcc: dQ (32) or dV (<= 128)
+};
+enum { bRes = 0, bFull0, bFull1, bMma, bAlu, bFinal, bNum };
+
+struct BParams {
+    const float2* stats_in;      // (1/D, b) per row (dq, dk/dv passes)
+    float2* stats_out;           // statistics pass
+    __nv_bfloat16* dq;           // [BH, L, 16]
+    __nv_bfloat16* dk;
+    __nv_bfloat16* dvo;          // [BH, L, dvw]
+    unsigned int* err;
+    int L, dvw, numerator_only;  // dvw: value head dimension of the caller's tensors (64, 112, 128)
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// AND of a predicate over the 128 row threads (named barrier 1): all of them get the same answer, so
+// they leave their loop together and the warp-collective tensor-memory accesses stay converged; it
+// also orders their shared-memory writes before the reads that follow
+__device__ __forceinline__ bool rows_all(bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, 1, 128, p;\n\t"
+        "selp.b32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred)
+        : "memory");
+    return r != 0;
+}
+__device__ __forceinline__ float tw(float s) { return fmaf(s, fmaf(s, 0.03125f, 0.25f), 1.0f); }
+__device__ __forceinline__ float tdw(float s) { return fmaf(s, 0.0625f, 0.25f); }
+}  // namespace
+
+// tm_n0 / tm_w0: narrow (q or k) and wide (a/g or v) tensor of the CTA's own (resident) tile;
+// tm_n1 / tm_w1: of the tiles it loops over.
+template <int DV, int MODE>
+__global__ void __launch_bounds__(kThreadsB, 1)
+    backward_tc_kernel(const __grid_constant__ CUtensorMap tm_n0, const __grid_constant__ CUtensorMap tm_w0,
+                       const __grid_constant__ CUtensorMap tm_n1, const __grid_constant__ CUtensorMap tm_w1,
+                       const BParams p) {
+    using C = BCfg<DV>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offMisc);
+    uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + bNum);
+    volatile uint32_t* abort_flag = tmem_base_s + 1;
+    float2* s_b = reinterpret_cast<float2*>(smem + C::offB);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int ntiles = (p.L + kTile - 1) / kTile;
+    // own tile: the longest loops first (dq, statistics: last query tiles; dk/dv: first key tiles)
+    const int own = MODE == kModeDkDv ? blockIdx.x : ntiles - 1 - blockIdx.x;
+    const int head = blockIdx.y;
+    const int r0 = own * kTile;
+    const int first = MODE == kModeDkDv ? own : 0;             // other-side tiles first .. last
+    const int last = MODE == kModeDkDv ? ntiles - 1 : own;
+    const int nloop = last - first + 1;
+
+    if (tid == 0) {
+        mbar_init(&bars[bRes], 1); mbar_init(&bars[bFull0], 1); mbar_init(&bars[bFull1], 1);
+        mbar_init(&bars[bMma], 1); mbar_init(&bars[bAlu], 128); mbar_init(&bars[bFinal], 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 4) { tmem_alloc(tmem_base_s, 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = *tmem_base_s;
+    bool ok = true;
+
+    // descriptors: narrow tiles (64-byte rows, SWIZZLE_64B), wide tiles (128-byte rows, SWIZZLE_128B, 64-column blocks)
+    constexpr uint64_t dN = make_smem_desc_base(16, 512, kSwizzle64B);                  // K-major, or MN-major one block
+    constexpr uint64_t dW = make_smem_desc_base(kTile * 128, 1024, kSwizzle128B);       // K-major, or MN-major blocks
+    constexpr uint32_t iS = make_idesc_bf16(128, 128, 0, 0);                            // both operands K-major
+    constexpr uint32_t iN32 = make_idesc_bf16(128, 32, 0, 1);                           // A from TMEM, B MN-major narrow
+    constexpr uint32_t iNV = make_idesc_bf16(128, 64 * C::kVB, 0, 1);                   // A from TMEM, B MN-major wide
+
+    if (warp == 4) {
+        if (lane == 0) {
+            const uint32_t aResN = smem_u32(smem + C::offResN), aResW = smem_u32(smem + C::offResW);
+            auto load_stage = [&](int it) {
+                const int s = it & 1;
+                uint8_t* st = smem + C::offStage + s * C::kStage;
+                const int row = (first + it) * kTile;
+                mbar_arrive_expect_tx(&bars[bFull0 + s], C::kStage);
+                tma_load_3d(st, &tm_n1, &bars[bFull0 + s], 0, row, head);
+#pragma unroll
+                for (int b = 0; b < C::kVB; ++b)
+                    tma_load_3d(st + kQKTile + b * (kTile * 128), &tm_w1, &bars[bFull0 + s], b * 64, row, head);
+            };
+            mbar_arrive_expect_tx(&bars[bRes], kQKTile + C::kWide);
+            tma_load_3d(smem + C::offResN, &tm_n0, &bars[bRes], 0, r0, head);
+#pragma unroll
+            for (int b = 0; b < C::kVB; ++b)
+                tma_load_3d(smem + C::offResW + b * (kTile * 128), &tm_w0, &bars[bRes], b * 64, r0, head);
+            load_stage(0);
+            ok = mbar_wait(&bars[bRes], 0, abort_flag);
+            for (int it = 0; it < nloop && ok; ++it) {
+                const int s = it & 1;
+                const uint32_t aN = smem_u32(smem + C::offStage + s * C::kStage), aW = aN + kQKTile;
+                ok = mbar_wait(&bars[bFull0 + s], (it >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                // scores: rows = own tile, columns = looped tile
+                mma_ss_lh<false>(tb + C::colS, desc_lo(dN) + (aResN >> 4), desc_hi(dN), desc_lo(dN) + (aN >> 4),
+                                 desc_hi(dN), iS);
+                // own wide tile x looped wide tile^T over d_v
+#pragma unroll
+                for (int kk = 0; kk < DV / 16; ++kk) {
+                    const uint32_t off = ((kk >> 2) * (kTile * 128) + (kk & 3) * 32) >> 4;
+                    if (kk == 0)
+                        mma_ss_lh<false>(tb + C::colG, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW),
+                                         desc_lo(dW) + (aW >> 4) + off, desc_hi(dW), iS);
+                    else
+                        mma_ss_lh<true>(tb + C::colG, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW),
+                                        desc_lo(dW) + (aW >> 4) + off, desc_hi(dW), iS);
+                }
+                mma_commit(&bars[bMma]);
+                // once these products are done, so are the previous iteration's (in-order pipe): its stage is free
+                ok = mbar_wait(&bars[bMma], it & 1, abort_flag);
+                if (!ok) break;
+                if (it + 1 < nloop) load_stage(it + 1);
+                ok = mbar_wait(&bars[bAlu], it & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                if (MODE == kModeDq) {
+                    // dQ += DS (tensor memory, 128 keys = 8 K-steps) x K_j (MN-major, 32 columns)
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        if (it == 0 && k == 0)
+                            mma_ts_lh<false>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                                             desc_hi(dN), iN32);
+                        else
+                            mma_ts_lh<true>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                                            desc_hi(dN), iN32);
+                    }
+                } else if (MODE == kModeDkDv) {
+                    // dV += W^T (over the scores) x A_i;  dK += DS^T (over GV) x Q_i
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        if (it == 0 && k == 0) {
+                            mma_ts_lh<false>(tb + C::colAcc, tb + C::colS + k * 8, desc_lo(dW) + ((aW + k * 2048) >> 4),
+                                             desc_hi(dW), iNV);
+                            mma_ts_lh<false>(tb + C::colK, tb + C::colG + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                                             desc_hi(dN), iN32);
+                        } else {
+                            mma_ts_lh<true>(tb + C::colAcc, tb + C::colS + k * 8, desc_lo(dW) + ((aW + k * 2048) >> 4),
+                                            desc_hi(dW), iNV);
+                            mma_ts_lh<true>(tb + C::colK, tb + C::colG + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                                            desc_hi(dN), iN32);
+                        }
+                    }
+                }
+            }
+            if (ok) mma_commit(&bars[bFinal]);
+        }
+    } else {
+        // ===================================================================== row threads
+        const int t = tid;                                   // accumulator row == TMEM lane
+        const uint32_t lane_base = (uint32_t)warp * 32u;
+        const int row = r0 + t;                              // query (statistics, dq) or key (dk/dv) of this thread
+        float den = 0.f, en = 0.f;
+        float2 st_own = make_float2(0.f, 0.f);               // (1/D, b) of this thread's query (dq pass)
+        if (MODE == kModeDq && row < p.L) st_own = p.stats_in[(size_t)head * p.L + row];
+        for (int it = 0; it < nloop && ok; ++it) {
+            const int c0 = (first + it) * kTile;             // first row of the looped tile (columns of the accumulators)
+            if (MODE == kModeDkDv)                           // (1/D, b) of the looped queries, one per thread
+                s_b[(it & 1) * kTile + t] = c0 + t < p.L ? p.stats_in[(size_t)head * p.L + c0 + t] : make_float2(0.f, 0.f);
+            ok = rows_all(mbar_wait(&bars[bMma], it & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int blk = 0; blk < 4; ++blk) {
+                uint32_t sr[32], gr[32];
+                tmem_ld32(tmem_addr(tb, lane_base, C::colS + blk * 32), sr);
+                tmem_ld32(tmem_addr(tb, lane_base, C::colG + blk * 32), gr);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int col = c0 + blk * 32 + i;
+                    const float s = __uint_as_float(sr[i]), gvv = __uint_as_float(gr[i]);
+                    // pair (query, key): own row is the query except in the dk/dv pass
+                    const bool live = MODE == kModeDkDv ? (row <= col && col < p.L) : (col <= row);
+                    float w = live ? tw(s) : 0.f;
+                    float ds = 0.f;
+                    if (MODE == kModeStats) {
+                        den += w;
+                        en = fmaf(w, gvv, en);
+                    } else {
+                        const float2 stq = MODE == kModeDq ? st_own : s_b[(it & 1) * kTile + blk * 32 + i];
+                        ds = live ? fmaf(gvv, stq.x, stq.y) * tdw(s) : 0.f;
+                        w *= stq.x;                          // dv_j = sum_i (w_ij / D_i) G_i
+                    }
+                    sr[i] = __float_as_uint(w);
+                    gr[i] = __float_as_uint(ds);
+                }
+                uint32_t pw[16], pd[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    pw[i] = pack_bf16x2(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
+                    pd[i] = pack_bf16x2(__uint_as_float(gr[2 * i]), __uint_as_float(gr[2 * i + 1]));
+                }
+                if (MODE == kModeDq) tmem_st16(tmem_addr(tb, lane_base, C::colD + blk * 16), pd);
+                if (MODE == kModeDkDv) {
+                    tmem_st16(tmem_addr(tb, lane_base, C::colS + blk * 16), pw);       // in place: columns already read
+                    tmem_st16(tmem_addr(tb, lane_base, C::colG + blk * 16), pd);
+                }
+            }
+            if (MODE != kModeStats) tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&bars[bAlu]);
+        }
+        if (MODE != kModeStats) ok = rows_all(ok && mbar_wait(&bars[bFinal], 0, abort_flag));
+        tc_fence_after();
+        // tcgen05.ld is a warp-collective: every lane takes part, only the stores depend on the row
+        const bool store = ok && row < p.L;
+        const size_t grow = (size_t)head * p.L + (store ? row : 0);
+        if (MODE == kModeStats) {
+            if (store) {
+                const float dinv = p.numerator_only ? 1.0f : 1.0f / (den + kEps);
+                const float bq = p.numerator_only ? 0.0f : -en * dinv * dinv;
+                p.stats_out[grow] = make_float2(dinv, bq);
+            }
+        } else if (ok) {                                     // ok is uniform over the row threads (rows_all)
+            // 16 gradient columns of dq (colAcc) or dk (colK)
+            uint32_t r[16];
+            tmem_ld16(tmem_addr(tb, lane_base, MODE == kModeDq ? C::colAcc : C::colK), r);
+            tmem_wait_ld();
+            if (store) {
+                uint4 o0, o1;
+                o0.x = pack_bf16x2(__uint_as_float(r[0]), __uint_as_float(r[1]));
+                o0.y = pack_bf16x2(__uint_as_float(r[2]), __uint_as_float(r[3]));
+                o0.z = pack_bf16x2(__uint_as_float(r[4]), __uint_as_float(r[5]));
+                o0.w = pack_bf16x2(__uint_as_float(r[6]), __uint_as_float(r[7]));
+                o1.x = pack_bf16x2(__uint_as_float(r[8]), __uint_as_float(r[9]));
+                o1.y = pack_bf16x2(__uint_as_float(r[10]), __uint_as_float(r[11]));
+                o1.z = pack_bf16x2(__uint_as_float(r[12]), __uint_as_float(r[13]));
+                o1.w = pack_bf16x2(__uint_as_float(r[14]), __uint_as_float(r[15]));
+                uint4* dst = reinterpret_cast<uint4*>((MODE == kModeDq ? p.dq : p.dk) + grow * kDFeat);
+                dst[0] = o0;
+                dst[1] = o1;
+            }
+            if (MODE == kModeDkDv) {
+                uint4* vdst = reinterpret_cast<uint4*>(p.dvo + grow * p.dvw);
+                for (int c = 0; c < p.dvw / 16; ++c) {       // p.dvw is uniform
+                    uint32_t rv[16];
+                    tmem_ld16(tmem_addr(tb, lane_base, C::colAcc + c * 16), rv);
+                    tmem_wait_ld();
+                    if (store) {
+                        uint4 a, b;
+                        a.x = pack_bf16x2(__uint_as_float(rv[0]), __uint_as_float(rv[1]));
+                        a.y = pack_bf16x2(__uint_as_float(rv[2]), __uint_as_float(rv[3]));
+                        a.z = pack_bf16x2(__uint_as_float(rv[4]), __uint_as_float(rv[5]));
+                        a.w = pack_bf16x2(__uint_as_float(rv[6]), __uint_as_float(rv[7]));
+                        b.x = pack_bf16x2(__uint_as_float(rv[8]), __uint_as_float(rv[9]));
+                        b.y = pack_bf16x2(__uint_as_float(rv[10]), __uint_as_float(rv[11]));
+                        b.z = pack_bf16x2(__uint_as_float(rv[12]), __uint_as_float(rv[13]));
+                        b.w = pack_bf16x2(__uint_as_float(rv[14]), __uint_as_float(rv[15]));
+                        vdst[2 * c] = a;
+                        vdst[2 * c + 1] = b;
+                    }
+                }
+            }
+        }
+    }
+    if (!ok && lane == 0) atomicOr(p.err, 1u);
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);     // loads still in flight get time to land
+    }
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tb, 512);
+}
+
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_fn_b() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+// [BH][L][width] bf16, box = [1][128][box_w] (box_w may exceed width: the rest is zero-filled)
+bool make_map_b(CUtensorMap* m, const void* base, int BH, int L, int width, int box_w, CUtensorMapSwizzle sw) {
+    EncodeTiledFn enc = encode_fn_b();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)width, (cuuint64_t)L, (cuuint64_t)BH};
+    cuuint64_t strides[2] = {(cuuint64_t)width * 2, (cuuint64_t)L * width * 2};
+    cuuint32_t box[3] = {(cuuint32_t)box_w, (cuuint32_t)kTile, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int DV>
+based_status launch_dvb(const void* q, const void* k, const void* v, const void* g, void* dq, void* dk, void* dv,
+                        float* ws, int BH, int L, int dvr, int numerator_only, cudaStream_t stream) {
+    using C = BCfg<DV>;
+    float2* stats = reinterpret_cast<float2*>(ws);
+    CUtensorMap tq, tk, tv, tg;
+    if (!make_map_b(&tq, q, BH, L, kDFeat, 32, CU_TENSOR_MAP_SWIZZLE_64B) ||
+        !make_map_b(&tk, k, BH, L, kDFeat, 32, CU_TENSOR_MAP_SWIZZLE_64B) ||
+        !make_map_b(&tv, v, BH, L, dvr, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_b(&tg, g, BH, L, dvr, 64, CU_TENSOR_MAP_SWIZZLE_128B))
+        return BASED_ERR_CUDA;
+    BParams p{};
+    if (error_word_ptr(&p.err) != BASED_OK) return BASED_ERR_CUDA;
+    p.stats_in = stats;
+    p.stats_out = stats;
+    p.dq = static_cast<__nv_bfloat16*>(dq);
+    p.dk = static_cast<__nv_bfloat16*>(dk);
+    p.dvo = static_cast<__nv_bfloat16*>(dv);
+    p.L = L;
+    p.dvw = dvr;
+    p.numerator_only = numerator_only;
+    {
+        static bool configured[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BASED_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(setup_mutex());
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(backward_tc_kernel<DV, kModeStats>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)C::kSmem) != cudaSuccess ||
+                cudaFuncSetAttribute(backward_tc_kernel<DV, kModeDq>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)C::kSmem) != cudaSuccess ||
+                cudaFuncSetAttribute(backward_tc_kernel<DV, kModeDkDv>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)C::kSmem) != cudaSuccess)
+                return BASED_ERR_CUDA;
+            configured[dev] = true;
+        }
+    }
+    const dim3 grid((L + kTile - 1) / kTile, BH);
+    // statistics: own = queries (q, dout), looped = keys (k, v)
+    backward_tc_kernel<DV, kModeStats><<<grid, kThreadsB, C::kSmem, stream>>>(tq, tg, tk, tv, p);
+    note_launch();
+    based_status st = check_launch("backward_tc_kernel<stats>");
+    if (st != BASED_OK) return st;
+    // dq: own = queries (q, dout), looped = keys (k, v)
+    backward_tc_kernel<DV, kModeDq><<<grid, kThreadsB, C::kSmem, stream>>>(tq, tg, tk, tv, p);
+    note_launch();
+    st = check_launch("backward_tc_kernel<dq>");
+    if (st != BASED_OK) return st;
+    // dk, dv: own = keys (k, v), looped = queries (q, dout)
+    backward_tc_kernel<DV, kModeDkDv><<<grid, kThreadsB, C::kSmem, stream>>>(tk, tv, tq, tg, p);
+    note_launch();
+    return check_launch("backward_tc_kernel<dkdv>");
+}
+}  // namespace
+
+size_t backward_tc_workspace_bytes(int BH, int L, int d_v) {
+    (void)d_v;
+    return (size_t)BH * L * 2 * sizeof(float);                 // (1 / D, b) per row
+}
+
+based_status launch_prefill_backward_tc(const void* q, const void* k, const void* v, const void* g, void* dq, void* dk,
+                                        void* dv, float* ws, int BH, int L, int d_v, int numerator_only,
+                                        cudaStream_t stream) {
+    if (d_v == 64) return launch_dvb<64>(q, k, v, g, dq, dk, dv, ws, BH, L, 64, numerator_only, stream);
+    return launch_dvb<128>(q, k, v, g, dq, dk, dv, ws, BH, L, d_v, numerator_only, stream);       // 112 or 128
+}
+
+}  // namespace based
+
+#ifdef BASED_TRACE
+// debug builds: which barrier each warp of the first CTA that gave up was waiting on (this file's copy)
+extern "C" void based_debug_read_waits_bwd(unsigned int* out) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(out, based::sm100::g_wait_dbg, sizeof(unsigned int) * 128);
+    cudaMemcpyFromSymbol(out + 128, based::sm100::g_wait_owner, sizeof(unsigned int));
+    unsigned int zero[129] = {};
+    cudaMemcpyToSymbol(based::sm100::g_wait_dbg, zero, sizeof(unsigned int) * 128);
+    cudaMemcpyToSymbol(based::sm100::g_wait_owner, zero, sizeof(unsigned int));
+}
+#endif

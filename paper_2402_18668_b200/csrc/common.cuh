@@ -104,6 +104,11 @@ based_status launch_prefill_generic(const void* q, const void* k, const void* v,
 based_status launch_decode_generic(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
                                    int BH, int d_feat, int d_v, based_dtype io, bool numerator_only,
                                    cudaStream_t stream);
+// the same on tensor cores (bf16 io); ws: backward_tc_workspace_bytes
+size_t backward_tc_workspace_bytes(int BH, int L, int d_v);
+based_status launch_prefill_backward_tc(const void* q, const void* k, const void* v, const void* g, void* dq, void* dk,
+                                        void* dv, float* ws, int BH, int L, int d_v, int numerator_only,
+                                        cudaStream_t stream);
 // load the generation-step kernels into the current context
 based_status preload_decode();
 based_status preload_swa_decode();

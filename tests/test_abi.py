@@ -135,7 +135,8 @@ def test_backward_validation(lib):
     A = [ctypes.c_void_p(0x1000 * n) for n in range(1, 9)]
     q, k, v, g, dq, dk, dv, ws = A
     ok = (1, 1, 8, 16, 64, 1)
-    assert lib.based_prefill_backward_workspace_bytes(2, 3, 100) == 2 * 3 * 100 * 8
+    assert lib.based_prefill_backward_workspace_bytes(2, 3, 100, 64, 0) == 2 * 3 * 100 * 8
+    assert lib.based_prefill_backward_workspace_bytes(2, 3, 100, 64, 1) == 2 * 3 * 100 * 8
     assert f(q, k, v, None, dq, dk, dv, *ok, 0, ws, 1 << 20, None) == 1            # output gradient missing
     assert f(q, k, v, g, dq, dk, dv, *ok, 1, ws, 1 << 20, None) == 1               # CONTINUE is not a backward flag
     assert f(q, k, v, g, q, dk, dv, *ok, 0, ws, 1 << 20, None) == 1                # gradient aliases an input
