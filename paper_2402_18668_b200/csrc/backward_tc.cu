@@ -30,17 +30,26 @@ constexpr int kThreadsB = 160;
 constexpr int kModeStats = 0, kModeDq = 1, kModeDkDv = 2;
 constexpr uint32_t kQKTile = kTile * 64;                 // [128][32] bf16, 64-byte rows, SWIZZLE_64B
 
-template <int DV> struct BCfg {
-    static constexpr int kVB = (DV + 63) / 64;           // 64-column blocks of a [128][DV] tile (112 -> 2, second partly zero)
-    static constexpr uint32_t kWide = kVB * kTile * 128; // [128][64 * kVB] bf16 in SWIZZLE_128B blocks
-    // shared memory: resident narrow + wide tile, two stages of (narrow + wide), b of two stages, barriers
+// LT: rows of the tiles the CTA loops over (columns of the accumulators): 64 where that lets two CTAs
+// share an SM (256 tensor-memory columns each), so that one CTA's row-thread pass overlaps the
+// other's MMA bursts; 128 for the dk/dv pass at d_v 128, whose accumulators need more columns.
+template <int DV, int MODE, int LT> struct BCfg {
+    static constexpr int kVB = (DV + 63) / 64;           // 64-column blocks of a [rows][DV] tile (112 -> 2, second partly zero)
+    static constexpr uint32_t kWide = kVB * kTile * 128; // own tile: [128][64 * kVB] bf16 in SWIZZLE_128B blocks
+    static constexpr uint32_t kNarrowL = LT * 64, kWideL = kVB * LT * 128;       // looped tiles
+    // shared memory: resident narrow + wide tile, two stages of (narrow + wide), (1/D, b) of two stages, barriers
     static constexpr uint32_t offResN = 0, offResW = offResN + kQKTile;
-    static constexpr uint32_t offStage = offResW + kWide, kStage = kQKTile + kWide;
+    static constexpr uint32_t offStage = offResW + kWide, kStage = kNarrowL + kWideL;
     static constexpr uint32_t offB = offStage + 2 * kStage;
-    static constexpr uint32_t offMisc = offB + 2 * kTile * 8;      // (1/D, b) of the looped queries, two stages
+    static constexpr uint32_t offMisc = offB + 2 * LT * 8;
     static constexpr uint32_t kSmem = offMisc + 256 + 1024;
-    // tensor memory columns
-    static constexpr uint32_t colS = 0, colG = 128, colD = 256, colAcc = 320, colK = 448;   // colAcc: dQ (32) or dV (<= 128)
+    // tensor memory columns: scores, dout.v products, ds (dq pass; the dk/dv pass packs in place), accumulators
+    static constexpr uint32_t colS = 0, colG = LT, colD = 2 * LT;
+    static constexpr uint32_t colAcc = MODE == kModeDq ? 2 * LT + LT / 2 : 2 * LT;        // dQ (32) or dV (64 * kVB)
+    static constexpr uint32_t colK = colAcc + 64 * kVB;                                   // dK (32), dk/dv pass
+    static constexpr uint32_t kColsUsed = MODE == kModeStats ? 2 * LT : MODE == kModeDq ? colAcc + 32 : colK + 32;
+    static constexpr uint32_t kCols = kColsUsed <= 128 ? 128 : kColsUsed <= 256 ? 256 : 512;
+    static_assert(kColsUsed <= 512, "tensor memory budget");
 };
 enum { bRes = 0, bFull0, bFull1, bMma, bAlu, bFinal, bNum };
 
@@ -79,12 +88,12 @@ __device__ __forceinline__ float tdw(float s) { return fmaf(s, 0.0625f, 0.25f); 
 
 // tm_n0 / tm_w0: narrow (q or k) and wide (a/g or v) tensor of the CTA's own (resident) tile;
 // tm_n1 / tm_w1: of the tiles it loops over.
-template <int DV, int MODE>
+template <int DV, int MODE, int LT>
 __global__ void __launch_bounds__(kThreadsB, 1)
     backward_tc_kernel(const __grid_constant__ CUtensorMap tm_n0, const __grid_constant__ CUtensorMap tm_w0,
                        const __grid_constant__ CUtensorMap tm_n1, const __grid_constant__ CUtensorMap tm_w1,
                        const BParams p) {
-    using C = BCfg<DV>;
+    using C = BCfg<DV, MODE, LT>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offMisc);
@@ -98,8 +107,9 @@ __global__ void __launch_bounds__(kThreadsB, 1)
     const int own = MODE == kModeDkDv ? blockIdx.x : ntiles - 1 - blockIdx.x;
     const int head = blockIdx.y;
     const int r0 = own * kTile;
-    const int first = MODE == kModeDkDv ? own : 0;             // other-side tiles first .. last
-    const int last = MODE == kModeDkDv ? ntiles - 1 : own;
+    // looped tiles (LT rows each): keys 0 .. end of the own tile, or queries from the own tile's first row on
+    const int first = MODE == kModeDkDv ? r0 / LT : 0;
+    const int last = MODE == kModeDkDv ? (p.L - 1) / LT : (min(p.L, r0 + kTile) - 1) / LT;
     const int nloop = last - first + 1;
 
     if (tid == 0) {
@@ -108,7 +118,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
         *abort_flag = 0;
         fence_mbar_init();
     }
-    if (warp == 4) { tmem_alloc(tmem_base_s, 512); tmem_relinquish(); }
+    if (warp == 4) { tmem_alloc(tmem_base_s, C::kCols); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -117,8 +127,9 @@ __global__ void __launch_bounds__(kThreadsB, 1)
 
     // descriptors: narrow tiles (64-byte rows, SWIZZLE_64B), wide tiles (128-byte rows, SWIZZLE_128B, 64-column blocks)
     constexpr uint64_t dN = make_smem_desc_base(16, 512, kSwizzle64B);                  // K-major, or MN-major one block
-    constexpr uint64_t dW = make_smem_desc_base(kTile * 128, 1024, kSwizzle128B);       // K-major, or MN-major blocks
-    constexpr uint32_t iS = make_idesc_bf16(128, 128, 0, 0);                            // both operands K-major
+    constexpr uint64_t dW = make_smem_desc_base(kTile * 128, 1024, kSwizzle128B);       // own wide tile (128 rows per block)
+    constexpr uint64_t dWL = make_smem_desc_base(LT * 128, 1024, kSwizzle128B);         // looped wide tile (LT rows per block)
+    constexpr uint32_t iS = make_idesc_bf16(128, LT, 0, 0);                             // both operands K-major
     constexpr uint32_t iN32 = make_idesc_bf16(128, 32, 0, 1);                           // A from TMEM, B MN-major narrow
     constexpr uint32_t iNV = make_idesc_bf16(128, 64 * C::kVB, 0, 1);                   // A from TMEM, B MN-major wide
 
@@ -128,12 +139,12 @@ __global__ void __launch_bounds__(kThreadsB, 1)
             auto load_stage = [&](int it) {
                 const int s = it & 1;
                 uint8_t* st = smem + C::offStage + s * C::kStage;
-                const int row = (first + it) * kTile;
+                const int row = (first + it) * LT;
                 mbar_arrive_expect_tx(&bars[bFull0 + s], C::kStage);
                 tma_load_3d(st, &tm_n1, &bars[bFull0 + s], 0, row, head);
 #pragma unroll
                 for (int b = 0; b < C::kVB; ++b)
-                    tma_load_3d(st + kQKTile + b * (kTile * 128), &tm_w1, &bars[bFull0 + s], b * 64, row, head);
+                    tma_load_3d(st + C::kNarrowL + b * (LT * 128), &tm_w1, &bars[bFull0 + s], b * 64, row, head);
             };
             mbar_arrive_expect_tx(&bars[bRes], kQKTile + C::kWide);
             tma_load_3d(smem + C::offResN, &tm_n0, &bars[bRes], 0, r0, head);
@@ -144,7 +155,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
             ok = mbar_wait(&bars[bRes], 0, abort_flag);
             for (int it = 0; it < nloop && ok; ++it) {
                 const int s = it & 1;
-                const uint32_t aN = smem_u32(smem + C::offStage + s * C::kStage), aW = aN + kQKTile;
+                const uint32_t aN = smem_u32(smem + C::offStage + s * C::kStage), aW = aN + C::kNarrowL;
                 ok = mbar_wait(&bars[bFull0 + s], (it >> 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
@@ -155,12 +166,13 @@ __global__ void __launch_bounds__(kThreadsB, 1)
 #pragma unroll
                 for (int kk = 0; kk < DV / 16; ++kk) {
                     const uint32_t off = ((kk >> 2) * (kTile * 128) + (kk & 3) * 32) >> 4;
+                    const uint32_t offL = ((kk >> 2) * (LT * 128) + (kk & 3) * 32) >> 4;
                     if (kk == 0)
                         mma_ss_lh<false>(tb + C::colG, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW),
-                                         desc_lo(dW) + (aW >> 4) + off, desc_hi(dW), iS);
+                                         desc_lo(dWL) + (aW >> 4) + offL, desc_hi(dWL), iS);
                     else
                         mma_ss_lh<true>(tb + C::colG, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW),
-                                        desc_lo(dW) + (aW >> 4) + off, desc_hi(dW), iS);
+                                        desc_lo(dWL) + (aW >> 4) + offL, desc_hi(dWL), iS);
                 }
                 mma_commit(&bars[bMma]);
                 // once these products are done, so are the previous iteration's (in-order pipe): its stage is free
@@ -171,9 +183,9 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                 if (!ok) break;
                 tc_fence_after();
                 if (MODE == kModeDq) {
-                    // dQ += DS (tensor memory, 128 keys = 8 K-steps) x K_j (MN-major, 32 columns)
+                    // dQ += DS (tensor memory, LT keys = LT/16 K-steps) x K_j (MN-major, 32 columns)
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
+                    for (int k = 0; k < LT / 16; ++k) {
                         if (it == 0 && k == 0)
                             mma_ts_lh<false>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                              desc_hi(dN), iN32);
@@ -182,17 +194,17 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                                             desc_hi(dN), iN32);
                     }
                 } else if (MODE == kModeDkDv) {
-                    // dV += W^T (over the scores) x A_i;  dK += DS^T (over GV) x Q_i
+                    // dV += W'^T (over the scores) x G_i;  dK += DS^T (over GV) x Q_i
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
+                    for (int k = 0; k < LT / 16; ++k) {
                         if (it == 0 && k == 0) {
-                            mma_ts_lh<false>(tb + C::colAcc, tb + C::colS + k * 8, desc_lo(dW) + ((aW + k * 2048) >> 4),
-                                             desc_hi(dW), iNV);
+                            mma_ts_lh<false>(tb + C::colAcc, tb + C::colS + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
+                                             desc_hi(dWL), iNV);
                             mma_ts_lh<false>(tb + C::colK, tb + C::colG + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                              desc_hi(dN), iN32);
                         } else {
-                            mma_ts_lh<true>(tb + C::colAcc, tb + C::colS + k * 8, desc_lo(dW) + ((aW + k * 2048) >> 4),
-                                            desc_hi(dW), iNV);
+                            mma_ts_lh<true>(tb + C::colAcc, tb + C::colS + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
+                                            desc_hi(dWL), iNV);
                             mma_ts_lh<true>(tb + C::colK, tb + C::colG + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                             desc_hi(dN), iN32);
                         }
@@ -210,14 +222,14 @@ __global__ void __launch_bounds__(kThreadsB, 1)
         float2 st_own = make_float2(0.f, 0.f);               // (1/D, b) of this thread's query (dq pass)
         if (MODE == kModeDq && row < p.L) st_own = p.stats_in[(size_t)head * p.L + row];
         for (int it = 0; it < nloop && ok; ++it) {
-            const int c0 = (first + it) * kTile;             // first row of the looped tile (columns of the accumulators)
-            if (MODE == kModeDkDv)                           // (1/D, b) of the looped queries, one per thread
-                s_b[(it & 1) * kTile + t] = c0 + t < p.L ? p.stats_in[(size_t)head * p.L + c0 + t] : make_float2(0.f, 0.f);
+            const int c0 = (first + it) * LT;                // first row of the looped tile (columns of the accumulators)
+            if (MODE == kModeDkDv && t < LT)                 // (1/D, b) of the looped queries
+                s_b[(it & 1) * LT + t] = c0 + t < p.L ? p.stats_in[(size_t)head * p.L + c0 + t] : make_float2(0.f, 0.f);
             ok = rows_all(mbar_wait(&bars[bMma], it & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
 #pragma unroll 1
-            for (int blk = 0; blk < 4; ++blk) {
+            for (int blk = 0; blk < LT / 32; ++blk) {
                 uint32_t sr[32], gr[32];
                 tmem_ld32(tmem_addr(tb, lane_base, C::colS + blk * 32), sr);
                 tmem_ld32(tmem_addr(tb, lane_base, C::colG + blk * 32), gr);
@@ -234,7 +246,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                         den += w;
                         en = fmaf(w, gvv, en);
                     } else {
-                        const float2 stq = MODE == kModeDq ? st_own : s_b[(it & 1) * kTile + blk * 32 + i];
+                        const float2 stq = MODE == kModeDq ? st_own : s_b[(it & 1) * LT + blk * 32 + i];
                         ds = live ? fmaf(gvv, stq.x, stq.y) * tdw(s) : 0.f;
                         w *= stq.x;                          // dv_j = sum_i (w_ij / D_i) G_i
                     }
@@ -317,7 +329,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
         for (int i = 0; i < 200; ++i) __nanosleep(1000);     // loads still in flight get time to land
     }
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tb, 512);
+    if (warp == 4) tmem_dealloc(tb, C::kCols);
 }
 
 namespace {
@@ -336,28 +348,52 @@ EncodeTiledFn encode_fn_b() {
     return fn;
 }
 // [BH][L][width] bf16, box = [1][128][box_w] (box_w may exceed width: the rest is zero-filled)
-bool make_map_b(CUtensorMap* m, const void* base, int BH, int L, int width, int box_w, CUtensorMapSwizzle sw) {
+bool make_map_b(CUtensorMap* m, const void* base, int BH, int L, int width, int box_w, int box_rows,
+                CUtensorMapSwizzle sw) {
     EncodeTiledFn enc = encode_fn_b();
     if (!enc) return false;
     cuuint64_t dims[3] = {(cuuint64_t)width, (cuuint64_t)L, (cuuint64_t)BH};
     cuuint64_t strides[2] = {(cuuint64_t)width * 2, (cuuint64_t)L * width * 2};
-    cuuint32_t box[3] = {(cuuint32_t)box_w, (cuuint32_t)kTile, 1};
+    cuuint32_t box[3] = {(cuuint32_t)box_w, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+template <int DV, int MODE, int LT>
+based_status launch_pass(const CUtensorMap& n0, const CUtensorMap& w0, const CUtensorMap& n1, const CUtensorMap& w1,
+                         const BParams& p, dim3 grid, const char* what, cudaStream_t stream) {
+    using C = BCfg<DV, MODE, LT>;
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BASED_ERR_CUDA;
+    {
+        std::lock_guard<std::mutex> lock(setup_mutex());
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(backward_tc_kernel<DV, MODE, LT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)C::kSmem) != cudaSuccess)
+                return BASED_ERR_CUDA;
+            configured[dev] = true;
+        }
+    }
+    backward_tc_kernel<DV, MODE, LT><<<grid, kThreadsB, C::kSmem, stream>>>(n0, w0, n1, w1, p);
+    note_launch();
+    return check_launch(what);
+}
+
 template <int DV>
 based_status launch_dvb(const void* q, const void* k, const void* v, const void* g, void* dq, void* dk, void* dv,
                         float* ws, int BH, int L, int dvr, int numerator_only, cudaStream_t stream) {
-    using C = BCfg<DV>;
+    constexpr int LTK = (DV == 64) ? 64 : 128;       // looped tile of the dk/dv pass (d_v 128 needs all 512 columns anyway)
     float2* stats = reinterpret_cast<float2*>(ws);
-    CUtensorMap tq, tk, tv, tg;
-    if (!make_map_b(&tq, q, BH, L, kDFeat, 32, CU_TENSOR_MAP_SWIZZLE_64B) ||
-        !make_map_b(&tk, k, BH, L, kDFeat, 32, CU_TENSOR_MAP_SWIZZLE_64B) ||
-        !make_map_b(&tv, v, BH, L, dvr, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map_b(&tg, g, BH, L, dvr, 64, CU_TENSOR_MAP_SWIZZLE_128B))
+    // own tiles: 128 rows; looped tiles: 64 rows (and LTK rows for the dk/dv pass)
+    CUtensorMap tq, tk, tv, tg, tk64, tv64, tqL, tgL;
+    const CUtensorMapSwizzle s64 = CU_TENSOR_MAP_SWIZZLE_64B, s128 = CU_TENSOR_MAP_SWIZZLE_128B;
+    if (!make_map_b(&tq, q, BH, L, kDFeat, 32, kTile, s64) || !make_map_b(&tk, k, BH, L, kDFeat, 32, kTile, s64) ||
+        !make_map_b(&tv, v, BH, L, dvr, 64, kTile, s128) || !make_map_b(&tg, g, BH, L, dvr, 64, kTile, s128) ||
+        !make_map_b(&tk64, k, BH, L, kDFeat, 32, 64, s64) || !make_map_b(&tv64, v, BH, L, dvr, 64, 64, s128) ||
+        !make_map_b(&tqL, q, BH, L, kDFeat, 32, LTK, s64) || !make_map_b(&tgL, g, BH, L, dvr, 64, LTK, s128))
         return BASED_ERR_CUDA;
     BParams p{};
     if (error_word_ptr(&p.err) != BASED_OK) return BASED_ERR_CUDA;
@@ -369,37 +405,15 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
     p.L = L;
     p.dvw = dvr;
     p.numerator_only = numerator_only;
-    {
-        static bool configured[64] = {};
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BASED_ERR_CUDA;
-        std::lock_guard<std::mutex> lock(setup_mutex());
-        if (!configured[dev]) {
-            if (cudaFuncSetAttribute(backward_tc_kernel<DV, kModeStats>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)C::kSmem) != cudaSuccess ||
-                cudaFuncSetAttribute(backward_tc_kernel<DV, kModeDq>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)C::kSmem) != cudaSuccess ||
-                cudaFuncSetAttribute(backward_tc_kernel<DV, kModeDkDv>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)C::kSmem) != cudaSuccess)
-                return BASED_ERR_CUDA;
-            configured[dev] = true;
-        }
-    }
     const dim3 grid((L + kTile - 1) / kTile, BH);
     // statistics: own = queries (q, dout), looped = keys (k, v)
-    backward_tc_kernel<DV, kModeStats><<<grid, kThreadsB, C::kSmem, stream>>>(tq, tg, tk, tv, p);
-    note_launch();
-    based_status st = check_launch("backward_tc_kernel<stats>");
+    based_status st = launch_pass<DV, kModeStats, 64>(tq, tg, tk64, tv64, p, grid, "backward_tc_kernel<stats>", stream);
     if (st != BASED_OK) return st;
     // dq: own = queries (q, dout), looped = keys (k, v)
-    backward_tc_kernel<DV, kModeDq><<<grid, kThreadsB, C::kSmem, stream>>>(tq, tg, tk, tv, p);
-    note_launch();
-    st = check_launch("backward_tc_kernel<dq>");
+    st = launch_pass<DV, kModeDq, 64>(tq, tg, tk64, tv64, p, grid, "backward_tc_kernel<dq>", stream);
     if (st != BASED_OK) return st;
     // dk, dv: own = keys (k, v), looped = queries (q, dout)
-    backward_tc_kernel<DV, kModeDkDv><<<grid, kThreadsB, C::kSmem, stream>>>(tk, tv, tq, tg, p);
-    note_launch();
-    return check_launch("backward_tc_kernel<dkdv>");
+    return launch_pass<DV, kModeDkDv, LTK>(tk, tv, tqL, tgL, p, grid, "backward_tc_kernel<dkdv>", stream);
 }
 }  // namespace
 
