@@ -95,7 +95,16 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
         return BASED_ERR_ALIGNMENT;
     if (d_feat != kDFeat) {
         if ((flags & BASED_STATE_SYM) || (long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
-        return launch_prefill_generic(q, k, v, out, kv_state, z_state, B * H, L, d_feat, d_v, io, flags,
+        // bf16 io from the empty state: outputs on the tensor cores (definition form), the state by the fp32 kernel
+        bool outputs_done = false;
+        if (io == BASED_BF16 && !(flags & BASED_STATE_CONTINUE)) {
+            const based_status st =
+                launch_quadratic_forward_tc(q, k, v, out, B * H, L, d_feat, d_v, (flags & BASED_NUMERATOR_ONLY) ? 1 : 0,
+                                            static_cast<cudaStream_t>(cuda_stream));
+            if (st != BASED_OK) return st;
+            outputs_done = true;
+        }
+        return launch_prefill_generic(q, k, v, out, kv_state, z_state, B * H, L, d_feat, d_v, io, flags, outputs_done,
                                       static_cast<cudaStream_t>(cuda_stream));
     }
     const size_t need = based_prefill_workspace_bytes(B, H, L, d_feat, d_v, io);

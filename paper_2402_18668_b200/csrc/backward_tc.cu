@@ -15,7 +15,11 @@
 // current one); parallelism comes from the (tile, head) grid.  q and k tiles are loaded 32
 // columns wide (columns 16..31 are zero-filled by TMA) so that they serve both as K-major
 // operands of the scores and as MN-major B operands of dQ / dK.  The work is O(L^2) per head, as
-// in the fp32 path.
+// in the fp32 path.  A fourth mode of the same kernel evaluates the forward pass in this form
+// (scores, weights as bf16 in tensor memory, Y += P V, row sums): the tensor-core path of the
+// feature dimensions 8, 24 and 32, which the chunked d' = 16 kernel does not cover.
+#include <math.h>
+
 #include <mutex>
 
 #include "common.cuh"
@@ -27,7 +31,7 @@ using namespace sm100;
 namespace {
 constexpr int kTile = 128;
 constexpr int kThreadsB = 160;
-constexpr int kModeStats = 0, kModeDq = 1, kModeDkDv = 2;
+constexpr int kModeStats = 0, kModeDq = 1, kModeDkDv = 2, kModeFwd = 3;
 constexpr uint32_t kQKTile = kTile * 64;                 // [128][32] bf16, 64-byte rows, SWIZZLE_64B
 
 // LT: rows of the tiles the CTA loops over (columns of the accumulators): 64 where that lets two CTAs
@@ -44,10 +48,15 @@ template <int DV, int MODE, int LT> struct BCfg {
     static constexpr uint32_t offMisc = offB + 2 * LT * 8;
     static constexpr uint32_t kSmem = offMisc + 256 + 1024;
     // tensor memory columns: scores, dout.v products, ds (dq pass; the dk/dv pass packs in place), accumulators
-    static constexpr uint32_t colS = 0, colG = LT, colD = 2 * LT;
-    static constexpr uint32_t colAcc = MODE == kModeDq ? 2 * LT + LT / 2 : 2 * LT;        // dQ (32) or dV (64 * kVB)
+    static constexpr uint32_t colS = 0, colG = LT, colD = MODE == kModeFwd ? LT : 2 * LT;   // forward: no dout.v product
+    static constexpr uint32_t colAcc = MODE == kModeDq ? 2 * LT + LT / 2                  // dQ (32)
+                                       : MODE == kModeFwd ? LT + LT / 2                   // Y (64 * kVB)
+                                                          : 2 * LT;                       // dV (64 * kVB)
     static constexpr uint32_t colK = colAcc + 64 * kVB;                                   // dK (32), dk/dv pass
-    static constexpr uint32_t kColsUsed = MODE == kModeStats ? 2 * LT : MODE == kModeDq ? colAcc + 32 : colK + 32;
+    static constexpr uint32_t kColsUsed = MODE == kModeStats ? 2 * LT
+                                          : MODE == kModeDq ? colAcc + 32
+                                          : MODE == kModeFwd ? colAcc + 64 * kVB
+                                                             : colK + 32;
     static constexpr uint32_t kCols = kColsUsed <= 128 ? 128 : kColsUsed <= 256 ? 256 : 512;
     static_assert(kColsUsed <= 512, "tensor memory budget");
 };
@@ -61,6 +70,8 @@ struct BParams {
     __nv_bfloat16* dvo;          // [BH, L, dvw]
     unsigned int* err;
     int L, dvw, numerator_only;  // dvw: value head dimension of the caller's tensors (64, 112, 128)
+    int kdim;                    // forward mode: feature dimension rounded up to 16 (K extent of the scores)
+    float s1, s2;                // forward mode: w = 1 + s * s1 + s^2 * s2 (1 / sqrt d', 1 / (2 d'))
 };
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -146,11 +157,13 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                 for (int b = 0; b < C::kVB; ++b)
                     tma_load_3d(st + C::kNarrowL + b * (LT * 128), &tm_w1, &bars[bFull0 + s], b * 64, row, head);
             };
-            mbar_arrive_expect_tx(&bars[bRes], kQKTile + C::kWide);
+            mbar_arrive_expect_tx(&bars[bRes], MODE == kModeFwd ? kQKTile : kQKTile + C::kWide);
             tma_load_3d(smem + C::offResN, &tm_n0, &bars[bRes], 0, r0, head);
+            if (MODE != kModeFwd) {
 #pragma unroll
-            for (int b = 0; b < C::kVB; ++b)
-                tma_load_3d(smem + C::offResW + b * (kTile * 128), &tm_w0, &bars[bRes], b * 64, r0, head);
+                for (int b = 0; b < C::kVB; ++b)
+                    tma_load_3d(smem + C::offResW + b * (kTile * 128), &tm_w0, &bars[bRes], b * 64, r0, head);
+            }
             load_stage(0);
             ok = mbar_wait(&bars[bRes], 0, abort_flag);
             for (int it = 0; it < nloop && ok; ++it) {
@@ -162,9 +175,12 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                 // scores: rows = own tile, columns = looped tile
                 mma_ss_lh<false>(tb + C::colS, desc_lo(dN) + (aResN >> 4), desc_hi(dN), desc_lo(dN) + (aN >> 4),
                                  desc_hi(dN), iS);
+                if (MODE == kModeFwd && p.kdim > 16)         // feature dimensions 24 and 32: second K-step
+                    mma_ss_lh<true>(tb + C::colS, desc_lo(dN) + (aResN >> 4) + 2, desc_hi(dN), desc_lo(dN) + (aN >> 4) + 2,
+                                    desc_hi(dN), iS);
                 // own wide tile x looped wide tile^T over d_v
 #pragma unroll
-                for (int kk = 0; kk < DV / 16; ++kk) {
+                for (int kk = 0; kk < (MODE == kModeFwd ? 0 : DV / 16); ++kk) {
                     const uint32_t off = ((kk >> 2) * (kTile * 128) + (kk & 3) * 32) >> 4;
                     const uint32_t offL = ((kk >> 2) * (LT * 128) + (kk & 3) * 32) >> 4;
                     if (kk == 0)
@@ -192,6 +208,17 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                         else
                             mma_ts_lh<true>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                             desc_hi(dN), iN32);
+                    }
+                } else if (MODE == kModeFwd) {
+                    // Y += P (tensor memory) x V_j
+#pragma unroll
+                    for (int k = 0; k < LT / 16; ++k) {
+                        if (it == 0 && k == 0)
+                            mma_ts_lh<false>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
+                                             desc_hi(dWL), iNV);
+                        else
+                            mma_ts_lh<true>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
+                                            desc_hi(dWL), iNV);
                     }
                 } else if (MODE == kModeDkDv) {
                     // dV += W'^T (over the scores) x G_i;  dK += DS^T (over GV) x Q_i
@@ -232,17 +259,19 @@ __global__ void __launch_bounds__(kThreadsB, 1)
             for (int blk = 0; blk < LT / 32; ++blk) {
                 uint32_t sr[32], gr[32];
                 tmem_ld32(tmem_addr(tb, lane_base, C::colS + blk * 32), sr);
-                tmem_ld32(tmem_addr(tb, lane_base, C::colG + blk * 32), gr);
+                if (MODE != kModeFwd) tmem_ld32(tmem_addr(tb, lane_base, C::colG + blk * 32), gr);
                 tmem_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
                     const int col = c0 + blk * 32 + i;
-                    const float s = __uint_as_float(sr[i]), gvv = __uint_as_float(gr[i]);
+                    const float s = __uint_as_float(sr[i]), gvv = MODE == kModeFwd ? 0.f : __uint_as_float(gr[i]);
                     // pair (query, key): own row is the query except in the dk/dv pass
                     const bool live = MODE == kModeDkDv ? (row <= col && col < p.L) : (col <= row);
-                    float w = live ? tw(s) : 0.f;
+                    float w = live ? (MODE == kModeFwd ? fmaf(s, fmaf(s, p.s2, p.s1), 1.0f) : tw(s)) : 0.f;
                     float ds = 0.f;
-                    if (MODE == kModeStats) {
+                    if (MODE == kModeFwd) {
+                        den += w;
+                    } else if (MODE == kModeStats) {
                         den += w;
                         en = fmaf(w, gvv, en);
                     } else {
@@ -260,6 +289,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                     pd[i] = pack_bf16x2(__uint_as_float(gr[2 * i]), __uint_as_float(gr[2 * i + 1]));
                 }
                 if (MODE == kModeDq) tmem_st16(tmem_addr(tb, lane_base, C::colD + blk * 16), pd);
+                if (MODE == kModeFwd) tmem_st16(tmem_addr(tb, lane_base, C::colD + blk * 16), pw);
                 if (MODE == kModeDkDv) {
                     tmem_st16(tmem_addr(tb, lane_base, C::colS + blk * 16), pw);       // in place: columns already read
                     tmem_st16(tmem_addr(tb, lane_base, C::colG + blk * 16), pd);
@@ -283,9 +313,11 @@ __global__ void __launch_bounds__(kThreadsB, 1)
         } else if (ok) {                                     // ok is uniform over the row threads (rows_all)
             // 16 gradient columns of dq (colAcc) or dk (colK)
             uint32_t r[16];
-            tmem_ld16(tmem_addr(tb, lane_base, MODE == kModeDq ? C::colAcc : C::colK), r);
-            tmem_wait_ld();
-            if (store) {
+            if (MODE != kModeFwd) {
+                tmem_ld16(tmem_addr(tb, lane_base, MODE == kModeDq ? C::colAcc : C::colK), r);
+                tmem_wait_ld();
+            }
+            if (store && MODE != kModeFwd) {
                 uint4 o0, o1;
                 o0.x = pack_bf16x2(__uint_as_float(r[0]), __uint_as_float(r[1]));
                 o0.y = pack_bf16x2(__uint_as_float(r[2]), __uint_as_float(r[3]));
@@ -299,7 +331,9 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                 dst[0] = o0;
                 dst[1] = o1;
             }
-            if (MODE == kModeDkDv) {
+            if (MODE == kModeDkDv || MODE == kModeFwd) {
+                // the wide accumulator row: dv, or the forward output scaled by 1 / (denominator + eps)
+                const float sc = (MODE == kModeFwd && !p.numerator_only) ? 1.0f / (den + kEps) : 1.0f;
                 uint4* vdst = reinterpret_cast<uint4*>(p.dvo + grow * p.dvw);
                 for (int c = 0; c < p.dvw / 16; ++c) {       // p.dvw is uniform
                     uint32_t rv[16];
@@ -307,14 +341,14 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                     tmem_wait_ld();
                     if (store) {
                         uint4 a, b;
-                        a.x = pack_bf16x2(__uint_as_float(rv[0]), __uint_as_float(rv[1]));
-                        a.y = pack_bf16x2(__uint_as_float(rv[2]), __uint_as_float(rv[3]));
-                        a.z = pack_bf16x2(__uint_as_float(rv[4]), __uint_as_float(rv[5]));
-                        a.w = pack_bf16x2(__uint_as_float(rv[6]), __uint_as_float(rv[7]));
-                        b.x = pack_bf16x2(__uint_as_float(rv[8]), __uint_as_float(rv[9]));
-                        b.y = pack_bf16x2(__uint_as_float(rv[10]), __uint_as_float(rv[11]));
-                        b.z = pack_bf16x2(__uint_as_float(rv[12]), __uint_as_float(rv[13]));
-                        b.w = pack_bf16x2(__uint_as_float(rv[14]), __uint_as_float(rv[15]));
+                        a.x = pack_bf16x2(__uint_as_float(rv[0]) * sc, __uint_as_float(rv[1]) * sc);
+                        a.y = pack_bf16x2(__uint_as_float(rv[2]) * sc, __uint_as_float(rv[3]) * sc);
+                        a.z = pack_bf16x2(__uint_as_float(rv[4]) * sc, __uint_as_float(rv[5]) * sc);
+                        a.w = pack_bf16x2(__uint_as_float(rv[6]) * sc, __uint_as_float(rv[7]) * sc);
+                        b.x = pack_bf16x2(__uint_as_float(rv[8]) * sc, __uint_as_float(rv[9]) * sc);
+                        b.y = pack_bf16x2(__uint_as_float(rv[10]) * sc, __uint_as_float(rv[11]) * sc);
+                        b.z = pack_bf16x2(__uint_as_float(rv[12]) * sc, __uint_as_float(rv[13]) * sc);
+                        b.w = pack_bf16x2(__uint_as_float(rv[14]) * sc, __uint_as_float(rv[15]) * sc);
                         vdst[2 * c] = a;
                         vdst[2 * c + 1] = b;
                     }
@@ -416,6 +450,29 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
     return launch_pass<DV, kModeDkDv, LTK>(tk, tv, tqL, tgL, p, grid, "backward_tc_kernel<dkdv>", stream);
 }
 }  // namespace
+
+// Forward of the definition form on the same tiles, for feature dimensions other than 16 (bf16 io,
+// empty initial state): out = (sum_j w_ij v_j) / (sum_j w_ij + eps), w = 1 + s/sqrt(d') + s^2/(2 d').
+based_status launch_quadratic_forward_tc(const void* q, const void* k, const void* v, void* out, int BH, int L,
+                                         int d_feat, int d_v, int numerator_only, cudaStream_t stream) {
+    CUtensorMap tq, tk64, tv64;
+    const CUtensorMapSwizzle s64 = CU_TENSOR_MAP_SWIZZLE_64B, s128 = CU_TENSOR_MAP_SWIZZLE_128B;
+    if (!make_map_b(&tq, q, BH, L, d_feat, 32, kTile, s64) || !make_map_b(&tk64, k, BH, L, d_feat, 32, 64, s64) ||
+        !make_map_b(&tv64, v, BH, L, d_v, 64, 64, s128))
+        return BASED_ERR_CUDA;
+    BParams p{};
+    if (error_word_ptr(&p.err) != BASED_OK) return BASED_ERR_CUDA;
+    p.dvo = static_cast<__nv_bfloat16*>(out);
+    p.L = L;
+    p.dvw = d_v;
+    p.numerator_only = numerator_only;
+    p.kdim = d_feat <= 16 ? 16 : 32;
+    p.s1 = 1.0f / sqrtf((float)d_feat);
+    p.s2 = 0.5f / (float)d_feat;
+    const dim3 grid((L + kTile - 1) / kTile, BH);
+    if (d_v == 64) return launch_pass<64, kModeFwd, 64>(tq, tq, tk64, tv64, p, grid, "quadratic forward (tc)", stream);
+    return launch_pass<128, kModeFwd, 64>(tq, tq, tk64, tv64, p, grid, "quadratic forward (tc)", stream);
+}
 
 size_t backward_tc_workspace_bytes(int BH, int L, int d_v) {
     (void)d_v;

@@ -98,8 +98,9 @@ based_status launch_prefill_backward(const void* q, const void* k, const void* v
                                      void* dv, float* stats, int BH, int L, int d_v, based_dtype io,
                                      int numerator_only, cudaStream_t stream);
 // feature dimensions 8, 24, 32 (fp32 FMA, definition form); state layout [1 + d' + d'^2, d_v]
+// outputs_done: out has been written already (tensor-core forward), only the state is still to do
 based_status launch_prefill_generic(const void* q, const void* k, const void* v, void* out, float* kv, float* z,
-                                    int BH, int L, int d_feat, int d_v, based_dtype io, int flags,
+                                    int BH, int L, int d_feat, int d_v, based_dtype io, int flags, bool outputs_done,
                                     cudaStream_t stream);
 based_status launch_decode_generic(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
                                    int BH, int d_feat, int d_v, based_dtype io, bool numerator_only,
@@ -109,6 +110,9 @@ size_t backward_tc_workspace_bytes(int BH, int L, int d_v);
 based_status launch_prefill_backward_tc(const void* q, const void* k, const void* v, const void* g, void* dq, void* dk,
                                         void* dv, float* ws, int BH, int L, int d_v, int numerator_only,
                                         cudaStream_t stream);
+// definition-form forward on tensor cores for d' in {8, 24, 32} (bf16 io, empty initial state)
+based_status launch_quadratic_forward_tc(const void* q, const void* k, const void* v, void* out, int BH, int L,
+                                         int d_feat, int d_v, int numerator_only, cudaStream_t stream);
 // load the generation-step kernels into the current context
 based_status preload_decode();
 based_status preload_swa_decode();

@@ -295,7 +295,7 @@ __global__ void __launch_bounds__(256) generic_decode_kernel(const T* __restrict
 
 template <typename T, int DV>
 static based_status prefill_t(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH,
-                              int L, int df, int flags, cudaStream_t stream) {
+                              int L, int df, int flags, bool outputs_done, cudaStream_t stream) {
     const size_t smem = sizeof(FwdSmem<DV>);
     {
         static bool configured[64] = {};
@@ -313,11 +313,14 @@ static based_status prefill_t(const void* q, const void* k, const void* v, void*
     const T* qq = static_cast<const T*>(q);
     const T* kk = static_cast<const T*>(k);
     const T* vv = static_cast<const T*>(v);
-    generic_prefill_kernel<T, DV><<<dim3((L + kT - 1) / kT, BH), kBT, smem, stream>>>(
-        qq, kk, vv, static_cast<T*>(out), cont ? kv : nullptr, cont ? z : nullptr, L, df,
-        (flags & BASED_NUMERATOR_ONLY) ? 1 : 0);
-    note_launch();
-    based_status st = check_launch("generic_prefill_kernel");
+    based_status st = BASED_OK;
+    if (!outputs_done) {
+        generic_prefill_kernel<T, DV><<<dim3((L + kT - 1) / kT, BH), kBT, smem, stream>>>(
+            qq, kk, vv, static_cast<T*>(out), cont ? kv : nullptr, cont ? z : nullptr, L, df,
+            (flags & BASED_NUMERATOR_ONLY) ? 1 : 0);
+        note_launch();
+        st = check_launch("generic_prefill_kernel");
+    }
     if (st != BASED_OK || kv == nullptr) return st;
     const int D = expanded_dim(df);
     generic_state_kernel<T, DV><<<dim3((D + 31) / 32, BH), DV + 32, 0, stream>>>(kk, vv, kv, z, L, df, cont ? 1 : 0);
@@ -326,16 +329,16 @@ static based_status prefill_t(const void* q, const void* k, const void* v, void*
 }
 
 based_status launch_prefill_generic(const void* q, const void* k, const void* v, void* out, float* kv, float* z,
-                                    int BH, int L, int d_feat, int d_v, based_dtype io, int flags,
+                                    int BH, int L, int d_feat, int d_v, based_dtype io, int flags, bool outputs_done,
                                     cudaStream_t stream) {
     if (io == BASED_F32) {
-        if (d_v == 64) return prefill_t<float, 64>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
-        if (d_v == 112) return prefill_t<float, 112>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
-        return prefill_t<float, 128>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
+        if (d_v == 64) return prefill_t<float, 64>(q, k, v, out, kv, z, BH, L, d_feat, flags, outputs_done, stream);
+        if (d_v == 112) return prefill_t<float, 112>(q, k, v, out, kv, z, BH, L, d_feat, flags, outputs_done, stream);
+        return prefill_t<float, 128>(q, k, v, out, kv, z, BH, L, d_feat, flags, outputs_done, stream);
     }
-    if (d_v == 64) return prefill_t<__nv_bfloat16, 64>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
-    if (d_v == 112) return prefill_t<__nv_bfloat16, 112>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
-    return prefill_t<__nv_bfloat16, 128>(q, k, v, out, kv, z, BH, L, d_feat, flags, stream);
+    if (d_v == 64) return prefill_t<__nv_bfloat16, 64>(q, k, v, out, kv, z, BH, L, d_feat, flags, outputs_done, stream);
+    if (d_v == 112) return prefill_t<__nv_bfloat16, 112>(q, k, v, out, kv, z, BH, L, d_feat, flags, outputs_done, stream);
+    return prefill_t<__nv_bfloat16, 128>(q, k, v, out, kv, z, BH, L, d_feat, flags, outputs_done, stream);
 }
 
 based_status launch_decode_generic(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
