@@ -21,6 +21,7 @@
 #include <math.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "common.cuh"
 #include "sm100.cuh"
@@ -255,46 +256,55 @@ __global__ void __launch_bounds__(kThreadsB, 1)
             ok = rows_all(mbar_wait(&bars[bMma], it & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
+            // one pass over the tile's LT accumulator columns of this row; MASKED: the tile touches the
+            // diagonal or the end of the sequence (the others need no per-pair test)
+            auto pass = [&](auto masked_tag) {
+                constexpr bool MASKED = decltype(masked_tag)::value;
 #pragma unroll 1
-            for (int blk = 0; blk < LT / 32; ++blk) {
-                uint32_t sr[32], gr[32];
-                tmem_ld32(tmem_addr(tb, lane_base, C::colS + blk * 32), sr);
-                if (MODE != kModeFwd) tmem_ld32(tmem_addr(tb, lane_base, C::colG + blk * 32), gr);
-                tmem_wait_ld();
+                for (int blk = 0; blk < LT / 32; ++blk) {
+                    uint32_t sr[32], gr[32];
+                    tmem_ld32(tmem_addr(tb, lane_base, C::colS + blk * 32), sr);
+                    if (MODE != kModeFwd) tmem_ld32(tmem_addr(tb, lane_base, C::colG + blk * 32), gr);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int col = c0 + blk * 32 + i;
-                    const float s = __uint_as_float(sr[i]), gvv = MODE == kModeFwd ? 0.f : __uint_as_float(gr[i]);
-                    // pair (query, key): own row is the query except in the dk/dv pass
-                    const bool live = MODE == kModeDkDv ? (row <= col && col < p.L) : (col <= row);
-                    float w = live ? (MODE == kModeFwd ? fmaf(s, fmaf(s, p.s2, p.s1), 1.0f) : tw(s)) : 0.f;
-                    float ds = 0.f;
-                    if (MODE == kModeFwd) {
-                        den += w;
-                    } else if (MODE == kModeStats) {
-                        den += w;
-                        en = fmaf(w, gvv, en);
-                    } else {
-                        const float2 stq = MODE == kModeDq ? st_own : s_b[(it & 1) * LT + blk * 32 + i];
-                        ds = live ? fmaf(gvv, stq.x, stq.y) * tdw(s) : 0.f;
-                        w *= stq.x;                          // dv_j = sum_i (w_ij / D_i) G_i
+                    for (int i = 0; i < 32; ++i) {
+                        const int col = c0 + blk * 32 + i;
+                        const float s = __uint_as_float(sr[i]), gvv = MODE == kModeFwd ? 0.f : __uint_as_float(gr[i]);
+                        // pair (query, key): own row is the query except in the dk/dv pass
+                        const bool live = !MASKED || (MODE == kModeDkDv ? (row <= col && col < p.L) : (col <= row));
+                        float w = live ? (MODE == kModeFwd ? fmaf(s, fmaf(s, p.s2, p.s1), 1.0f) : tw(s)) : 0.f;
+                        float ds = 0.f;
+                        if (MODE == kModeFwd) {
+                            den += w;
+                        } else if (MODE == kModeStats) {
+                            den += w;
+                            en = fmaf(w, gvv, en);
+                        } else {
+                            const float2 stq = MODE == kModeDq ? st_own : s_b[(it & 1) * LT + blk * 32 + i];
+                            ds = live ? fmaf(gvv, stq.x, stq.y) * tdw(s) : 0.f;
+                            w *= stq.x;                      // dv_j = sum_i (w_ij / D_i) G_i
+                        }
+                        sr[i] = __float_as_uint(w);
+                        gr[i] = __float_as_uint(ds);
                     }
-                    sr[i] = __float_as_uint(w);
-                    gr[i] = __float_as_uint(ds);
-                }
-                uint32_t pw[16], pd[16];
+                    uint32_t pw[16], pd[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    pw[i] = pack_bf16x2(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
-                    pd[i] = pack_bf16x2(__uint_as_float(gr[2 * i]), __uint_as_float(gr[2 * i + 1]));
+                    for (int i = 0; i < 16; ++i) {
+                        pw[i] = pack_bf16x2(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
+                        pd[i] = pack_bf16x2(__uint_as_float(gr[2 * i]), __uint_as_float(gr[2 * i + 1]));
+                    }
+                    if (MODE == kModeDq) tmem_st16(tmem_addr(tb, lane_base, C::colD + blk * 16), pd);
+                    if (MODE == kModeFwd) tmem_st16(tmem_addr(tb, lane_base, C::colD + blk * 16), pw);
+                    if (MODE == kModeDkDv) {
+                        tmem_st16(tmem_addr(tb, lane_base, C::colS + blk * 16), pw);   // in place: columns already read
+                        tmem_st16(tmem_addr(tb, lane_base, C::colG + blk * 16), pd);
+                    }
                 }
-                if (MODE == kModeDq) tmem_st16(tmem_addr(tb, lane_base, C::colD + blk * 16), pd);
-                if (MODE == kModeFwd) tmem_st16(tmem_addr(tb, lane_base, C::colD + blk * 16), pw);
-                if (MODE == kModeDkDv) {
-                    tmem_st16(tmem_addr(tb, lane_base, C::colS + blk * 16), pw);       // in place: columns already read
-                    tmem_st16(tmem_addr(tb, lane_base, C::colG + blk * 16), pd);
-                }
-            }
+            };
+            // uniform over the CTA: every pair of the tile is live
+            const bool all_live = MODE == kModeDkDv ? (r0 + kTile - 1 <= c0 && c0 + LT <= p.L) : (c0 + LT - 1 <= r0);
+            if (all_live) pass(std::false_type{});
+            else pass(std::true_type{});
             if (MODE != kModeStats) tmem_wait_st();
             tc_fence_before();
             mbar_arrive(&bars[bAlu]);
