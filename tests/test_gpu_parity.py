@@ -237,6 +237,25 @@ def test_prefill_backward_cfg2_sampled_heads():
         assert _grad_err(_np(dv[sl]), rv) <= TOL_BF16
 
 
+def test_autograd_wrapper_routes_gradients_through_the_library():
+    """loss.backward() through paper_2402_18668_b200.autograd.linear_attention: gradients against the oracle's."""
+    from paper_2402_18668_b200.autograd import linear_attention
+    B, H, L, d_v = 2, 3, 260, 64
+    w = wl.Workload("ag", B, H, L, 16, d_v, "bf16", 0.5)
+    gen = wl.generator(606)
+    q, k, v = wl.prefill_inputs(w, gen)
+    g = torch.randn(B, H, L, d_v, generator=gen).to(q.dtype)
+    qd, kd, vd = (t.to(DEV).requires_grad_(True) for t in (q, k, v))
+    n0 = based.launch_count()
+    out = linear_attention(qd, kd, vd)
+    (out.float() * g.to(DEV).float()).sum().backward()
+    _poll()
+    assert based.launch_count() - n0 >= 4                   # one forward launch, three backward launches
+    rq, rk, rv = oracle.linattn_backward(_np(q), _np(k), _np(v), _np(g))
+    assert _grad_err(_np(qd.grad), rq) <= TOL_BF16 and _grad_err(_np(kd.grad), rk) <= TOL_BF16
+    assert _grad_err(_np(vd.grad), rv) <= TOL_BF16
+
+
 # --------------------------------------------------------------------------- other feature dimensions
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d_feat,L,d_v", [(8, 200, 64), (24, 130, 128), (32, 77, 112), (8, 1, 64)])
