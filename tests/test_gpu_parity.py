@@ -237,6 +237,43 @@ def test_prefill_backward_cfg2_sampled_heads():
         assert _grad_err(_np(dv[sl]), rv) <= TOL_BF16
 
 
+def test_prefill_backward_cfg3_sampled_heads():
+    """Full 1.3B-layer shape (B8 H16 L4096 d_v128, bf16), the dk/dv pass on 128-row looped tiles: one head
+    recomputed by the oracle (4096^2 / 2 pairs in fp64), gradients drawn on the device."""
+    w = wl.CONFIGS["cfg3_1p3b_prefill"]
+    g_ = torch.Generator(device=DEV).manual_seed(88)
+    q = (torch.randn(w.B, w.H, w.L, 16, generator=g_, device=DEV) * w.qk_scale).bfloat16()
+    k = (torch.randn(w.B, w.H, w.L, 16, generator=g_, device=DEV) * w.qk_scale).bfloat16()
+    v = torch.randn(w.B, w.H, w.L, w.d_v, generator=g_, device=DEV).bfloat16()
+    dout = torch.randn(w.B, w.H, w.L, w.d_v, generator=g_, device=DEV).bfloat16()
+    dq, dk, dv = based.based_prefill_backward(q, k, v, dout)
+    _poll()
+    b, h = w.B - 1, 5
+    sl = (slice(b, b + 1), slice(h, h + 1))
+    rq, rk, rv = oracle.linattn_backward(_np(q[sl]), _np(k[sl]), _np(v[sl]), _np(dout[sl]))
+    assert _grad_err(_np(dq[sl]), rq) <= TOL_BF16 and _grad_err(_np(dk[sl]), rk) <= TOL_BF16
+    assert _grad_err(_np(dv[sl]), rv) <= TOL_BF16
+
+
+@pytest.mark.parametrize("d_feat", [8, 32])
+def test_other_feature_dimensions_full_length_sampled(d_feat):
+    """B4 H16 L2048 d_v64 at d' = 8 and 32 (bf16: tensor-core definition form): two heads against the oracle,
+    outputs and final state."""
+    B, H, L, d_v = 4, 16, 2048, 64
+    g_ = torch.Generator(device=DEV).manual_seed(d_feat)
+    q = (torch.randn(B, H, L, d_feat, generator=g_, device=DEV) * 0.4).bfloat16()
+    k = (torch.randn(B, H, L, d_feat, generator=g_, device=DEV) * 0.4).bfloat16()
+    v = torch.randn(B, H, L, d_v, generator=g_, device=DEV).bfloat16()
+    kv, z = based.new_state(B, H, d_v, d_feat=d_feat)
+    out = based.based_prefill(q, k, v, kv_state=kv, z_state=z)
+    _poll()
+    for (b, h) in [(0, 0), (B - 1, H - 1)]:
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        y_ref, S_ref, z_ref = oracle.linattn_quadratic(_np(q[sl]), _np(k[sl]), _np(v[sl]))
+        assert row_err(_np(out[sl]), y_ref) <= TOL_BF16
+        assert head_err(_np(kv[sl]), S_ref) <= TOL_BF16 and head_err(_np(z[sl]), z_ref) <= TOL_BF16
+
+
 def test_autograd_wrapper_routes_gradients_through_the_library():
     """loss.backward() through paper_2402_18668_b200.autograd.linear_attention: gradients against the oracle's."""
     from paper_2402_18668_b200.autograd import linear_attention
