@@ -405,6 +405,15 @@ bool make_map_b(CUtensorMap* m, const void* base, int BH, int L, int width, int 
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+}  // namespace
+
+// the same map for the other tensor-core kernels of the library
+bool make_rows_map_bf16(CUtensorMap* m, const void* base, int BH, int L, int width, int box_w, int box_rows,
+                        CUtensorMapSwizzle sw) {
+    return make_map_b(m, base, BH, L, width, box_w, box_rows, sw);
+}
+
+namespace {
 template <int DV, int MODE, int LT>
 based_status launch_pass(const CUtensorMap& n0, const CUtensorMap& w0, const CUtensorMap& n1, const CUtensorMap& w1,
                          const BParams& p, dim3 grid, const char* what, cudaStream_t stream) {

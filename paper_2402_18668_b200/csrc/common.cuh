@@ -102,6 +102,9 @@ based_status launch_prefill_backward(const void* q, const void* k, const void* v
 based_status launch_prefill_generic(const void* q, const void* k, const void* v, void* out, float* kv, float* z,
                                     int BH, int L, int d_feat, int d_v, based_dtype io, int flags, bool outputs_done,
                                     cudaStream_t stream);
+// the final state of those feature dimensions on tensor cores (bf16 io); cont: add to the state given
+based_status launch_state_generic_tc(const void* k, const void* v, float* kv, float* z, int BH, int L, int d_feat,
+                                     int d_v, int cont, cudaStream_t stream);
 based_status launch_decode_generic(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
                                    int BH, int d_feat, int d_v, based_dtype io, bool numerator_only,
                                    cudaStream_t stream);

@@ -1,6 +1,7 @@
 // Feature dimensions other than 16: d' in {8, 24, 32} (the paper's feature-map ablation trains
 // Taylor maps of dimension 8, 16, 24 and 32, i.e. 73, 273, 601 and 1057 expanded features).
-// First correct path, fp32 FMAs only:
+// The fp32 FMA paths (fp32 io; with bf16 io the outputs from the empty state and the final state run
+// on tensor cores instead: the tile kernel's forward mode and generic_state_tc.cu):
 //
 //   prefill   the definition form of Eq. (2), Sec. 4.1, tile by tile: 64 queries per CTA loop over
 //             the key tiles j <= i; scores (any d'), weights w = 1 + s/sqrt(d') + s^2/(2 d'), row
@@ -10,7 +11,7 @@
 //   decode    the recurrent step as a plain stream over the [D, d_v] state, D = 1 + d' + d'^2.
 //
 // The state layout is the 273-row layout's generalisation: constant, linear terms, row-major
-// outer product.  The tensor-core kernels and the symmetric format exist for d' = 16 only.
+// outer product.  The chunked tensor-core prefill and the symmetric format exist for d' = 16 only.
 #include "common.cuh"
 
 namespace based {
@@ -322,6 +323,7 @@ static based_status prefill_t(const void* q, const void* k, const void* v, void*
         st = check_launch("generic_prefill_kernel");
     }
     if (st != BASED_OK || kv == nullptr) return st;
+    if (sizeof(T) == 2) return launch_state_generic_tc(k, v, kv, z, BH, L, df, DV, cont ? 1 : 0, stream);
     const int D = expanded_dim(df);
     generic_state_kernel<T, DV><<<dim3((D + 31) / 32, BH), DV + 32, 0, stream>>>(kk, vv, kv, z, L, df, cont ? 1 : 0);
     note_launch();
