@@ -29,6 +29,12 @@
 // warp 17 issues the state-update MMAs (5)/(z), warp 18 the output-side MMAs (1)/(4)/(3):
 // two independent in-order streams, so the state chain runs ahead of the output chain.
 // All cross-role hand-offs are mbarriers with bounded waits.
+//
+// d_v 64, plain chunk loop: phi(Q) does not go through shared memory.  The feature group writes it
+// into tensor memory (the upper half of the chunk's score buffer once the row group has read the
+// scores, plus 16 spare columns) as the A operand of step (4), and the shared-memory tile that
+// frees holds a second state-copy tile, so the copy for chunk c+1 is written while step (4) of
+// chunk c reads its own.
 #include <cuda_bf16.h>
 #include <cstdlib>
 
@@ -85,12 +91,20 @@ struct Cfg {
     static constexpr uint32_t colS = colY + kNY;
     static constexpr uint32_t colZ0 = colS + kF;                 // d_v 128 only
     static constexpr uint32_t colZ1 = colZ0 + 16;
-    static_assert((DV == 64 ? colS + kF : colZ1 + 16) <= 512, "TMEM budget");
+    // d_v 64: phi(Q) of a chunk lives in tensor memory as the A operand of step (4): features 0..127 in
+    // the upper half of the chunk's score buffer (free once the row group has read the scores), features
+    // 128..159 in the 16 columns after the state; the shared-memory tile it leaves free during the own
+    // chunks holds a second copy tile of the state, so the state group writes chunk c+1's copy while
+    // step (4) of chunk c still reads its own
+    static constexpr bool kPQinT = (DV == 64);
+    static constexpr uint32_t colPQhi = colS + kF;
+    static_assert((DV == 64 ? colS + kF + 16 : colZ1 + 16) <= 512, "TMEM budget");
     static_assert(kScBlk % 1024 == 0 && kStageBytes % 1024 == 0 && offPK % 1024 == 0, "tiles stay 1024-byte aligned");
 };
 
 enum Bar {
-    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kG1b, kP, kPb, kG2, kG2b, kG4, kG3, kR4, kPK, kPKb, kSR, kDone, kNumBars
+    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kG1b, kP, kPb, kG2, kG2b, kG4, kG4b, kG3, kR4, kPK, kPKb, kSR, kDone, kTR, kTRb, kSC, kSCb,
+    kNumBars
 };
 
 // segments per head, chunks per segment (the last one takes the rest), mode
@@ -259,6 +273,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     constexpr int NS = C::kStages;
     constexpr bool STATE_ONLY = MODE == kModeState;
     constexpr bool PRE = MODE == kModePre;
+    // phi(Q) in tensor memory and two state-copy tiles: the plain chunk loop only (measured: -7 % where every
+    // SM has a CTA; the recompute mode's kernel loses 5 % with it)
+    constexpr bool PQT = C::kPQinT && MODE == kModeMain;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offMisc);
@@ -288,9 +305,10 @@ __global__ void __launch_bounds__(kThreads, 1)
     if (tid == 0) { TRACE(5, 0, 7); TRACE_CTA(0); }     // kernel entry
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(&bars[kFull0 + s], 1); mbar_init(&bars[kEmpty0 + s], STATE_ONLY ? 1 : 2); }
-        mbar_init(&bars[kG1], 1); mbar_init(&bars[kG1b], 1); mbar_init(&bars[kPb], 128); mbar_init(&bars[kG2], 1); mbar_init(&bars[kG2b], 1); mbar_init(&bars[kG4], 1);
+        mbar_init(&bars[kG1], 1); mbar_init(&bars[kG1b], 1); mbar_init(&bars[kPb], 128); mbar_init(&bars[kG2], 1); mbar_init(&bars[kG2b], 1); mbar_init(&bars[kG4], 1); mbar_init(&bars[kG4b], 1);
+        mbar_init(&bars[kTR], 128); mbar_init(&bars[kTRb], 128); mbar_init(&bars[kSC], 128); mbar_init(&bars[kSCb], 128);
         mbar_init(&bars[kG3], 1);
-        mbar_init(&bars[kP], 128); mbar_init(&bars[kR4], 384); mbar_init(&bars[kPK], 128); mbar_init(&bars[kPKb], 128); mbar_init(&bars[kDone], 1);
+        mbar_init(&bars[kP], 128); mbar_init(&bars[kR4], PQT ? 256 : 384); mbar_init(&bars[kPK], 128); mbar_init(&bars[kPKb], 128); mbar_init(&bars[kDone], 1);
         mbar_init(&bars[kSR], 128);
         *abort_flag = 0;
         fence_mbar_init();
@@ -340,6 +358,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     // "phi(K) of chunk g written": one barrier per tile for the same reason (the feature group may be
     // two chunks ahead of the issuer where tiles alternate); same phase numbering as above
     auto pk_bar = [&](int g) -> uint64_t* { return &bars[(alt(g) && (g & 1)) ? kPKb : kPK]; };
+    // "step (4) of own chunk c done": with two state-copy tiles (kPQinT) one barrier per tile, as above
+    auto g4_bar = [&](int c) -> uint64_t* { return &bars[(PQT && (c & 1)) ? kG4b : kG4]; };
+    auto g4_parity = [&](int c) -> uint32_t { return PQT ? ((c >> 1) & 1) : (c & 1); };
 
     if (warp == kWarpTma) {
         // ===================================================================== TMA producer
@@ -431,7 +452,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             constexpr uint32_t i4 = make_idesc_bf16(128, C::kNY, 0, 0);
             constexpr uint32_t i3 = make_idesc_bf16(128, DV, 0, 1);
             const uint32_t lQK = desc_lo(dQK), lV = desc_lo(dV);
-            const uint32_t lPQ = desc_lo(dPhiK) + (smem_u32(sPQ) >> 4), lSc = desc_lo(dPhiK) + (smem_u32(sSc) >> 4);
+            const uint32_t lPQ = desc_lo(dPhiK) + (smem_u32(sPQ) >> 4), lSc0 = desc_lo(dPhiK) + (smem_u32(sSc) >> 4);
             // scores of chunk c: T[c & 1] (or the single T) = Q_c K_c^T
             auto issue_scores = [&](int c) -> bool {
                 const int s = (c + npre) % NS;
@@ -468,16 +489,28 @@ __global__ void __launch_bounds__(kThreads, 1)
                 // arrives once before its first chunk): one barrier, three groups of 128 arrivals
                 ok = mbar_wait(&bars[kR4], ph, abort_flag);
                 if (!ok) break;
+                // two copy tiles: the state group may be a chunk ahead, so its "copy written" has a barrier per tile
+                if (PQT) {
+                    ok = mbar_wait(&bars[kSC + (c & 1)], (c >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                }
                 TRACE(0, c, 3);
                 tc_fence_after();
+                const uint32_t lSc = (PQT && (c & 1)) ? lPQ : lSc0;      // second copy tile: the phi(Q) tile's place
 #pragma unroll
                 for (int k = 0; k < kF / 16; ++k) {
                     const uint32_t off = ((k >> 1) * C::kPhiBlk + (k & 1) * 32) >> 4;
                     const uint32_t offb = ((k >> 1) * C::kScBlk + (k & 1) * 32) >> 4;
-                    if (k == 0) mma_ss_lh<false>(tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
-                    else mma_ss_lh<true>(tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
+                    if (PQT) {
+                        const uint32_t a = tb + (k < 8 ? colTc + 64 + k * 8 : C::colPQhi + (k - 8) * 8);
+                        if (k == 0) mma_ts_lh<false>(tb + C::colY, a, lSc + offb, desc_hi(dPhiK), i4);
+                        else mma_ts_lh<true>(tb + C::colY, a, lSc + offb, desc_hi(dPhiK), i4);
+                    } else {
+                        if (k == 0) mma_ss_lh<false>(tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
+                        else mma_ss_lh<true>(tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
+                    }
                 }
-                mma_commit(&bars[kG4]);
+                mma_commit(g4_bar(c));
                 TRACE(0, c, 4);
                 ok = mbar_wait(&bars[kP + t_idx(c)], t_parity(c), abort_flag);
                 if (!ok) break;
@@ -674,13 +707,16 @@ __global__ void __launch_bounds__(kThreads, 1)
                 tc_fence_before();
                 mbar_arrive(&bars[kSR]);                                   // step (5) of chunk c may overwrite the state
                 if (t == 0) TRACE(4, c, 1);
-                if (c > 0) {
-                    ok = mbar_wait(&bars[kG4], (c - 1) & 1, abort_flag);   // step (4) of chunk c-1 has read the tile
+                // the tile's last reader: step (4) of chunk c-1, or of chunk c-2 where two tiles alternate
+                constexpr int kBack = PQT ? 2 : 1;
+                if (c >= kBack) {
+                    ok = mbar_wait(g4_bar(c - kBack), g4_parity(c - kBack), abort_flag);
                     if (!ok) break;
                 }
                 if (t == 0) TRACE(4, c, 2);
+                uint8_t* sScC = (PQT && (c & 1)) ? sPQ : sSc;
                 if (srow >= 0) {
-                    uint8_t* row = sSc + (srow >> 3) * 512 + (srow & 7) * 64;
+                    uint8_t* row = sScC + (srow >> 3) * 512 + (srow & 7) * 64;
                     const uint32_t sw = (srow >> 1) & 3;
 #pragma unroll
                     for (int j = 0; j < kF / 8; ++j)
@@ -689,7 +725,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 }
                 if (DV == 128) {
                     // z row (row 128 of the tile: its swizzle term is zero)
-                    uint8_t* zrow = sSc + (DV >> 3) * 512;
+                    uint8_t* zrow = sScC + (DV >> 3) * 512;
                     *reinterpret_cast<__nv_bfloat16*>(zrow + (t >> 5) * C::kScBlk + (t & 31) * 2) =
                         __float2bfloat16_rn(__uint_as_float(z0));
                     if (z1f >= 0)
@@ -697,7 +733,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                             __float2bfloat16_rn(__uint_as_float(z1));
                 }
                 fence_proxy_async_smem();
-                mbar_arrive(&bars[kR4]);
+                mbar_arrive(&bars[PQT ? kSC + (c & 1) : kR4]);
                 if (t == 0) TRACE(4, c, 3);
             }
             if (ok && nch > 0) ok = mbar_wait(g2_bar(ntot - 1), g2_parity(ntot - 1), abort_flag);
@@ -780,8 +816,23 @@ __global__ void __launch_bounds__(kThreads, 1)
                 // wait (measured: 5 % on the 360M-layer shape; at d_v 128 it costs 1 %, so not there)
                 uint4 fq[DV == 64 ? 20 : 1];
                 if constexpr (DV == 64) compute_phi_row(qlo, qhi, true, fq);
+                if constexpr (PQT) {
+                    // the row group has read the scores of chunk c: the upper half of their buffer is free
+                    ok = mbar_wait(&bars[kTR + t_idx(c)], t_parity(c), abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t colTc = C::colT + (c & 1) * 128;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t r[16] = {fq[4 * j].x, fq[4 * j].y, fq[4 * j].z, fq[4 * j].w,
+                                                fq[4 * j + 1].x, fq[4 * j + 1].y, fq[4 * j + 1].z, fq[4 * j + 1].w,
+                                                fq[4 * j + 2].x, fq[4 * j + 2].y, fq[4 * j + 2].z, fq[4 * j + 2].w,
+                                                fq[4 * j + 3].x, fq[4 * j + 3].y, fq[4 * j + 3].z, fq[4 * j + 3].w};
+                        tmem_st16(tmem_addr(tb, lane_base, colTc + 64 + j * 16), r);
+                    }
+                }
                 if (c > 0) {
-                    ok = mbar_wait(&bars[kG4], (c - 1) & 1, abort_flag);   // step (4) of chunk c-1 has read phi(Q)
+                    ok = mbar_wait(g4_bar(c - 1), g4_parity(c - 1), abort_flag);   // step (4) of chunk c-1 has read phi(Q)
                     if (!ok) break;
                 } else if (npre > 1) {
                     const int last = ((npre & 1) ? npre - 2 : npre - 1);   // last odd pre-chunk used this tile for phi(K)
@@ -789,9 +840,18 @@ __global__ void __launch_bounds__(kThreads, 1)
                     if (!ok) break;
                 }
                 if (t == 0) TRACE(3, c, 3);
-                if constexpr (DV == 64) store_phi_row(fq, sPQ, t);
-                else write_phi_row(qlo, qhi, sPQ, t, true);
-                fence_proxy_async_smem();
+                if constexpr (PQT) {
+                    tc_fence_after();
+                    const uint32_t r[16] = {fq[16].x, fq[16].y, fq[16].z, fq[16].w, fq[17].x, fq[17].y, fq[17].z, fq[17].w,
+                                            fq[18].x, fq[18].y, fq[18].z, fq[18].w, fq[19].x, fq[19].y, fq[19].z, fq[19].w};
+                    tmem_st16(tmem_addr(tb, lane_base, C::colPQhi), r);
+                    tmem_wait_st();
+                    tc_fence_before();
+                } else {
+                    if constexpr (DV == 64) store_phi_row(fq, sPQ, t);
+                    else write_phi_row(qlo, qhi, sPQ, t, true);
+                    fence_proxy_async_smem();
+                }
                 mbar_arrive(&bars[kR4]);
                 if (t == 0) TRACE(3, c, 4);
             }
@@ -841,6 +901,10 @@ __global__ void __launch_bounds__(kThreads, 1)
                 } else {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) pk[i] = 0u;
+                }
+                if (PQT && b == 3) {               // every score column has been read: phi(Q) may take the upper half
+                    tc_fence_before();
+                    mbar_arrive(&bars[kTR + t_idx(c)]);
                 }
                 tmem_st16(tmem_addr(tb, lane_base, colTc + b * 16), pk);
             }
