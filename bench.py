@@ -479,15 +479,20 @@ def bench_backward(w, steps, warmup, torch, based, dist_on, peaks):
     bf16 = w.dtype == "bf16"
     ws = torch.empty(based.lib().based_prefill_backward_workspace_bytes(w.B, w.H, w.L, w.d_v, 1 if bf16 else 0),
                      dtype=torch.uint8, device="cuda")
+    # as in training, the forward output exists already (autograd saved it): not part of the timed region
+    out = based.based_prefill(q, k, v)
     n0 = based.launch_count()
-    ms = time_region(lambda i: based.based_prefill_backward(q, k, v, dout, workspace=ws), steps, warmup, torch, dist_on)
+    ms = time_region(lambda i: based.based_prefill_backward(q, k, v, dout, workspace=ws, out=out), steps, warmup, torch,
+                     dist_on)
     assert based.based_poll_error() == 0
     t = ms * 1e-3 / steps
     pairs = w.B * w.H * w.L * (w.L + 1) / 2.0
-    flops = 2.0 * pairs * (80 + 4 * w.d_v)              # 3 score passes, 3 dout.v passes + dv, dq and dk updates
+    # per pair: bf16 (statistics + dq merged): 2 score and 2 dout.v products, dv, X and Y of dq, dk = 80 + 3 d_v;
+    # fp32: 3 score and 3 dout.v products, dv, dq, dk = 80 + 4 d_v
+    flops = 2.0 * pairs * (80 + (3 if bf16 else 4) * w.d_v)
     peak = peaks["bf16_tflops"] if bf16 else 148 * 128 * 2 * 1.965e9 / 1e12
     return {
-        "workload": w.name + (" backward (tensor cores, quadratic form)" if bf16 else " backward (fp32 FMA, quadratic form)"),
+        "workload": w.name + (" backward given the forward output (tensor cores, quadratic form, 2 passes)" if bf16 else " backward (fp32 FMA, quadratic form)"),
         "metric": "backward_tokens_per_s", "value": w.B * w.L / t, "unit": "tokens/s", "ms_per_step": t * 1e3,
         "steps": steps, "launches_per_step": (based.launch_count() - n0) // (steps + warmup),
         "roofline": {"bound": "tensor" if bf16 else "alu", "achieved": flops / t / 1e12, "peak": peak,

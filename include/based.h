@@ -194,6 +194,22 @@ based_status based_prefill_backward(const void* q, const void* k, const void* v,
 size_t based_prefill_backward_workspace_bytes(int B, int H, int L, int d_v, based_dtype io);
 
 /*
+ * The same backward pass for a caller that kept the forward output (training: autograd saves it).
+ * out [B,H,L,d_v], io dtype: what based_prefill returned for these q, k, v from the empty state with
+ * the same flags.  Results and arguments as based_prefill_backward.  With bf16 io the row statistics
+ * and dq then take one sweep over the keys instead of two: dq_i = X_i / D_i + (m_i / D_i + b_i) Y_i
+ * with X_i = sum_j w'_ij (dout_i.v_j - m_i) k_j and Y_i = sum_j w'_ij k_j needs neither D_i nor b_i
+ * while the keys are swept, and m_i = dout_i . out_i, the weighted mean of dout_i . v_j up to the
+ * rounding of out, keeps the cancellation against b_i in fp32.  out is used for this centring
+ * only: D_i and dout_i . N_i are still recomputed in fp32.  fp32 io ignores out's values.
+ * out must not alias a gradient output.
+ */
+based_status based_prefill_backward_with_out(const void* q, const void* k, const void* v, const void* out,
+                                             const void* dout, void* dq, void* dk, void* dv, int B, int H, int L,
+                                             int d_feat, int d_v, based_dtype io, int flags, void* workspace,
+                                             size_t workspace_bytes, void* cuda_stream);
+
+/*
  * The gated short convolution at the core of the BaseConv layer (App. "Extended Architecture
  * Details", paragraph "Convolution": y = ((u W1 + b1) (.) SiLU(h * (u W2) + b2)) W3 + b3).
  * The three projections are plain matrix products and stay with the caller; this call is the

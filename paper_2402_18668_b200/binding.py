@@ -28,7 +28,7 @@ EXPORTS = (
     "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step", "based_decode_step_sym",
     "based_state_to_sym", "based_state_from_sym", "swa_decode_step_at", "based_preload_decode",
     "baseconv_gate_forward", "baseconv_gate_step", "based_decode_step_flags", "based_prefill_backward",
-    "based_prefill_backward_workspace_bytes",
+    "based_prefill_backward_workspace_bytes", "based_prefill_backward_with_out",
 )
 
 _lib = None
@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.based_preload_decode.restype = i
         L.based_prefill_backward.restype = i
         L.based_prefill_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
+        L.based_prefill_backward_with_out.restype = i
+        L.based_prefill_backward_with_out.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
         L.based_prefill_backward_workspace_bytes.restype = sz
         L.based_prefill_backward_workspace_bytes.argtypes = [i, i, i, i, i]
         L.baseconv_gate_forward.restype = i
@@ -163,18 +165,25 @@ def based_prefill(q, k, v, out=None, kv_state=None, z_state=None, flags: int = B
     return out
 
 
-def based_prefill_backward(q, k, v, dout, flags: int = 0, workspace=None, stream=None):
-    """Gradients (dq, dk, dv) of based_prefill (empty initial state) for the output gradient dout."""
-    _dev(q, k, v, dout, workspace)
+def based_prefill_backward(q, k, v, dout, flags: int = 0, workspace=None, stream=None, out=None):
+    """Gradients (dq, dk, dv) of based_prefill (empty initial state) for the output gradient dout.
+    out: the forward output, if the caller kept it (based_prefill_backward_with_out)."""
+    _dev(q, k, v, dout, workspace, out)
     B, H, L, d_feat = q.shape
     d_v = v.shape[-1]
     need = int(lib().based_prefill_backward_workspace_bytes(B, H, L, d_v, _dtype_code(q)))
     if workspace is None or workspace.numel() * workspace.element_size() < need:
         workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
     dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
-    st = lib().based_prefill_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv), B, H, L,
-                                      d_feat, d_v, _dtype_code(q), int(flags), _ptr(workspace),
-                                      workspace.numel() * workspace.element_size(), _stream(stream))
+    tail = (B, H, L, d_feat, d_v, _dtype_code(q), int(flags), _ptr(workspace),
+            workspace.numel() * workspace.element_size(), _stream(stream))
+    if out is None:
+        st = lib().based_prefill_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv), *tail)
+    else:
+        if out.dtype != v.dtype or out.shape != v.shape or not out.is_contiguous():
+            raise ValueError("out must have v's shape and dtype and be contiguous")
+        st = lib().based_prefill_backward_with_out(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(dout), _ptr(dq), _ptr(dk),
+                                                   _ptr(dv), *tail)
     _check(st, "based_prefill_backward")
     return dq, dk, dv
 

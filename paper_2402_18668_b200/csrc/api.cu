@@ -268,9 +268,10 @@ size_t based_prefill_backward_workspace_bytes(int B, int H, int L, int d_v, base
     return (size_t)B * H * L * 2 * sizeof(float);
 }
 
-based_status based_prefill_backward(const void* q, const void* k, const void* v, const void* dout, void* dq,
-                                    void* dk, void* dv, int B, int H, int L, int d_feat, int d_v, based_dtype io,
-                                    int flags, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+static based_status prefill_backward(const void* q, const void* k, const void* v, const void* out, const void* dout,
+                                     void* dq, void* dk, void* dv, int B, int H, int L, int d_feat, int d_v,
+                                     based_dtype io, int flags, void* workspace, size_t workspace_bytes,
+                                     void* cuda_stream) {
     if (!q || !k || !v || !dout || !dq || !dk || !dv || B <= 0 || H <= 0 || L <= 0) return BASED_ERR_INVALID_ARG;
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
     if (flags & ~BASED_NUMERATOR_ONLY) return BASED_ERR_INVALID_ARG;
@@ -278,16 +279,32 @@ based_status based_prefill_backward(const void* q, const void* k, const void* v,
     if (d_feat != kDFeat || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
     if ((long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) || !aligned16(dk) ||
-        !aligned16(dv) || !aligned16(workspace))
+        !aligned16(dv) || !aligned16(workspace) || !aligned16(out))
         return BASED_ERR_ALIGNMENT;
     if (!workspace || workspace_bytes < based_prefill_backward_workspace_bytes(B, H, L, d_v, io))
         return BASED_ERR_WORKSPACE;
     if (io == BASED_BF16)
-        return launch_prefill_backward_tc(q, k, v, dout, dq, dk, dv, static_cast<float*>(workspace), B * H, L, d_v,
-                                          (flags & BASED_NUMERATOR_ONLY) ? 1 : 0,
+        return launch_prefill_backward_tc(q, k, v, out, dout, dq, dk, dv, static_cast<float*>(workspace), B * H, L,
+                                          d_v, (flags & BASED_NUMERATOR_ONLY) ? 1 : 0,
                                           static_cast<cudaStream_t>(cuda_stream));
     return launch_prefill_backward(q, k, v, dout, dq, dk, dv, static_cast<float*>(workspace), B * H, L, d_v, io,
                                    (flags & BASED_NUMERATOR_ONLY) ? 1 : 0, static_cast<cudaStream_t>(cuda_stream));
+}
+
+based_status based_prefill_backward(const void* q, const void* k, const void* v, const void* dout, void* dq,
+                                    void* dk, void* dv, int B, int H, int L, int d_feat, int d_v, based_dtype io,
+                                    int flags, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return prefill_backward(q, k, v, nullptr, dout, dq, dk, dv, B, H, L, d_feat, d_v, io, flags, workspace,
+                            workspace_bytes, cuda_stream);
+}
+
+based_status based_prefill_backward_with_out(const void* q, const void* k, const void* v, const void* out,
+                                             const void* dout, void* dq, void* dk, void* dv, int B, int H, int L,
+                                             int d_feat, int d_v, based_dtype io, int flags, void* workspace,
+                                             size_t workspace_bytes, void* cuda_stream) {
+    if (!out || out == dq || out == dk || out == dv) return BASED_ERR_INVALID_ARG;
+    return prefill_backward(q, k, v, out, dout, dq, dk, dv, B, H, L, d_feat, d_v, io, flags, workspace,
+                            workspace_bytes, cuda_stream);
 }
 
 based_status based_preload_decode(void) {

@@ -9,6 +9,14 @@
 // 1/D_i is applied to the fp32 products, not to the operand: a = dout / D rounded to bf16 would
 // break the near-cancellation of a_i.v_j + b_i for short prefixes.
 //
+// When the caller passes the forward output, statistics and dq take one sweep (a fifth mode):
+//   dq_i = X_i / D_i + (m_i / D_i + b_i) Y_i,   X_i = sum_j w'_ij (gv_ij - m_i) k_j,   Y_i = sum_j w'_ij k_j
+// holds for any m_i and needs neither D_i nor b_i while the keys are swept: D_i and E_i accumulate in
+// registers, X and Y by MMA from two packed bf16 tiles, and 1/D_i, b_i, dq_i are formed in fp32 at the
+// end.  m_i = dout_i . out_i is the weighted mean E_i / D_i of the gv_ij up to the rounding of out, so
+// the packed products are as small as ds above and the part of dq that cancels against b_i stays in
+// fp32 (without a centre the two separately rounded tiles would have to cancel).
+//
 // One CTA per (head, 128-row tile), 160 threads: warps 0-3 own one accumulator row each (the
 // polynomial, masks and bf16 packing), lane 0 of warp 4 issues TMA loads and MMAs.  The loop over
 // the other side's tiles is sequential per CTA (loads of the next tile are in flight during the
@@ -32,7 +40,7 @@ using namespace sm100;
 namespace {
 constexpr int kTile = 128;
 constexpr int kThreadsB = 160;
-constexpr int kModeStats = 0, kModeDq = 1, kModeDkDv = 2, kModeFwd = 3;
+constexpr int kModeStats = 0, kModeDq = 1, kModeDkDv = 2, kModeFwd = 3, kModeDqS = 4;
 constexpr uint32_t kQKTile = kTile * 64;                 // [128][32] bf16, 64-byte rows, SWIZZLE_64B
 
 // LT: rows of the tiles the CTA loops over (columns of the accumulators): 64 where that lets two CTAs
@@ -50,12 +58,16 @@ template <int DV, int MODE, int LT> struct BCfg {
     static constexpr uint32_t kSmem = offMisc + 256 + 1024;
     // tensor memory columns: scores, dout.v products, ds (dq pass; the dk/dv pass packs in place), accumulators
     static constexpr uint32_t colS = 0, colG = LT, colD = MODE == kModeFwd ? LT : 2 * LT;   // forward: no dout.v product
+    static constexpr uint32_t colD2 = colD + LT / 2;                                      // second packed tile (merged pass)
     static constexpr uint32_t colAcc = MODE == kModeDq ? 2 * LT + LT / 2                  // dQ (32)
+                                       : MODE == kModeDqS ? 3 * LT                        // X (32), then Y (32)
                                        : MODE == kModeFwd ? LT + LT / 2                   // Y (64 * kVB)
                                                           : 2 * LT;                       // dV (64 * kVB)
+    static constexpr uint32_t colAcc2 = colAcc + 32;                                      // merged pass: Y
     static constexpr uint32_t colK = colAcc + 64 * kVB;                                   // dK (32), dk/dv pass
     static constexpr uint32_t kColsUsed = MODE == kModeStats ? 2 * LT
                                           : MODE == kModeDq ? colAcc + 32
+                                          : MODE == kModeDqS ? colAcc2 + 32
                                           : MODE == kModeFwd ? colAcc + 64 * kVB
                                                              : colK + 32;
     static constexpr uint32_t kCols = kColsUsed <= 128 ? 128 : kColsUsed <= 256 ? 256 : 512;
@@ -64,6 +76,8 @@ template <int DV, int MODE, int LT> struct BCfg {
 enum { bRes = 0, bFull0, bFull1, bMma, bAlu, bFinal, bNum };
 
 struct BParams {
+    const __nv_bfloat16* g_raw;  // dout and the forward output as plain pointers [BH, L, dvw] (merged pass)
+    const __nv_bfloat16* o_raw;
     const float2* stats_in;      // (1/D, b) per row (dq, dk/dv passes)
     float2* stats_out;           // statistics pass
     __nv_bfloat16* dq;           // [BH, L, 16]
@@ -210,6 +224,22 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                             mma_ts_lh<true>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                             desc_hi(dN), iN32);
                     }
+                } else if (MODE == kModeDqS) {
+                    // X += (w' (gv - m)) K_j and Y += w' K_j: two packed tiles in tensor memory, the same B operand
+#pragma unroll
+                    for (int k = 0; k < LT / 16; ++k) {
+                        if (it == 0 && k == 0) {
+                            mma_ts_lh<false>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                                             desc_hi(dN), iN32);
+                            mma_ts_lh<false>(tb + C::colAcc2, tb + C::colD2 + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                                             desc_hi(dN), iN32);
+                        } else {
+                            mma_ts_lh<true>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                                            desc_hi(dN), iN32);
+                            mma_ts_lh<true>(tb + C::colAcc2, tb + C::colD2 + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                                            desc_hi(dN), iN32);
+                        }
+                    }
                 } else if (MODE == kModeFwd) {
                     // Y += P (tensor memory) x V_j
 #pragma unroll
@@ -249,6 +279,36 @@ __global__ void __launch_bounds__(kThreadsB, 1)
         float den = 0.f, en = 0.f;
         float2 st_own = make_float2(0.f, 0.f);               // (1/D, b) of this thread's query (dq pass)
         if (MODE == kModeDq && row < p.L) st_own = p.stats_in[(size_t)head * p.L + row];
+        // merged pass: the products dout_i . v_j enter the packed tile relative to m_i = dout_i . out_i, which
+        // is their weighted mean E_i / D_i up to the rounding of out: the part of dq that cancels against
+        // b_i is then formed in fp32 at the end, not from two separately rounded bf16 tiles
+        float m_own = 0.f;
+        if (MODE == kModeDqS && !p.numerator_only && row < p.L) {
+            const uint4* gp = reinterpret_cast<const uint4*>(p.g_raw + ((size_t)head * p.L + row) * p.dvw);
+            const uint4* op = reinterpret_cast<const uint4*>(p.o_raw + ((size_t)head * p.L + row) * p.dvw);
+            float part[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int c0 = 0; c0 < p.dvw / 8; c0 += 4) {          // 64, 112, 128 columns: 8, 14, 16 pieces; four in flight
+                uint4 a[4], b[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const bool in = c0 + u < p.dvw / 8;
+                    a[u] = in ? gp[c0 + u] : make_uint4(0u, 0u, 0u, 0u);
+                    b[u] = in ? op[c0 + u] : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const __nv_bfloat162* ha = reinterpret_cast<const __nv_bfloat162*>(&a[u]);
+                    const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&b[u]);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 fa = __bfloat1622float2(ha[e]), fb = __bfloat1622float2(hb[e]);
+                        part[u] = fmaf(fa.x, fb.x, part[u]);
+                        part[u] = fmaf(fa.y, fb.y, part[u]);
+                    }
+                }
+            }
+            m_own = (part[0] + part[1]) + (part[2] + part[3]);
+        }
         for (int it = 0; it < nloop && ok; ++it) {
             const int c0 = (first + it) * LT;                // first row of the looped tile (columns of the accumulators)
             if (MODE == kModeDkDv && t < LT)                 // (1/D, b) of the looped queries
@@ -279,6 +339,11 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                         } else if (MODE == kModeStats) {
                             den += w;
                             en = fmaf(w, gvv, en);
+                        } else if (MODE == kModeDqS) {
+                            den += w;
+                            en = fmaf(w, gvv, en);
+                            w = live ? tdw(s) : 0.f;         // second tile: w'
+                            ds = w * (gvv - m_own);          // first tile: w' (gv - m)
                         } else {
                             const float2 stq = MODE == kModeDq ? st_own : s_b[(it & 1) * LT + blk * 32 + i];
                             ds = live ? fmaf(gvv, stq.x, stq.y) * tdw(s) : 0.f;
@@ -294,6 +359,10 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                         pd[i] = pack_bf16x2(__uint_as_float(gr[2 * i]), __uint_as_float(gr[2 * i + 1]));
                     }
                     if (MODE == kModeDq) tmem_st16(tmem_addr(tb, lane_base, C::colD + blk * 16), pd);
+                    if (MODE == kModeDqS) {
+                        tmem_st16(tmem_addr(tb, lane_base, C::colD + blk * 16), pd);
+                        tmem_st16(tmem_addr(tb, lane_base, C::colD2 + blk * 16), pw);
+                    }
                     if (MODE == kModeFwd) tmem_st16(tmem_addr(tb, lane_base, C::colD + blk * 16), pw);
                     if (MODE == kModeDkDv) {
                         tmem_st16(tmem_addr(tb, lane_base, C::colS + blk * 16), pw);   // in place: columns already read
@@ -314,11 +383,27 @@ __global__ void __launch_bounds__(kThreadsB, 1)
         // tcgen05.ld is a warp-collective: every lane takes part, only the stores depend on the row
         const bool store = ok && row < p.L;
         const size_t grow = (size_t)head * p.L + (store ? row : 0);
-        if (MODE == kModeStats) {
-            if (store) {
-                const float dinv = p.numerator_only ? 1.0f : 1.0f / (den + kEps);
-                const float bq = p.numerator_only ? 0.0f : -en * dinv * dinv;
-                p.stats_out[grow] = make_float2(dinv, bq);
+        if (MODE == kModeStats || MODE == kModeDqS) {
+            const float dinv = p.numerator_only ? 1.0f : 1.0f / (den + kEps);
+            const float bq = p.numerator_only ? 0.0f : -en * dinv * dinv;
+            if (store) p.stats_out[grow] = make_float2(dinv, bq);
+            if (MODE == kModeDqS && ok) {
+                // dq_i = X_i / D_i + (m_i / D_i + b_i) Y_i
+                const float cy = fmaf(m_own, dinv, bq);
+                uint32_t rx[16], ry[16];
+                tmem_ld16(tmem_addr(tb, lane_base, C::colAcc), rx);
+                tmem_ld16(tmem_addr(tb, lane_base, C::colAcc2), ry);
+                tmem_wait_ld();
+                if (store) {
+                    uint32_t o[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        o[i] = pack_bf16x2(fmaf(__uint_as_float(rx[2 * i]), dinv, cy * __uint_as_float(ry[2 * i])),
+                                           fmaf(__uint_as_float(rx[2 * i + 1]), dinv, cy * __uint_as_float(ry[2 * i + 1])));
+                    uint4* dst = reinterpret_cast<uint4*>(p.dq + grow * kDFeat);
+                    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                }
             }
         } else if (ok) {                                     // ok is uniform over the row threads (rows_all)
             // 16 gradient columns of dq (colAcc) or dk (colK)
@@ -436,8 +521,8 @@ based_status launch_pass(const CUtensorMap& n0, const CUtensorMap& w0, const CUt
 }
 
 template <int DV>
-based_status launch_dvb(const void* q, const void* k, const void* v, const void* g, void* dq, void* dk, void* dv,
-                        float* ws, int BH, int L, int dvr, int numerator_only, cudaStream_t stream) {
+based_status launch_dvb(const void* q, const void* k, const void* v, const void* out, const void* g, void* dq, void* dk,
+                        void* dv, float* ws, int BH, int L, int dvr, int numerator_only, cudaStream_t stream) {
     constexpr int LTK = (DV == 64) ? 64 : 128;       // looped tile of the dk/dv pass (d_v 128 needs all 512 columns anyway)
     float2* stats = reinterpret_cast<float2*>(ws);
     // own tiles: 128 rows; looped tiles: 64 rows (and LTK rows for the dk/dv pass)
@@ -452,6 +537,8 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
     if (error_word_ptr(&p.err) != BASED_OK) return BASED_ERR_CUDA;
     p.stats_in = stats;
     p.stats_out = stats;
+    p.g_raw = static_cast<const __nv_bfloat16*>(g);
+    p.o_raw = static_cast<const __nv_bfloat16*>(out);
     p.dq = static_cast<__nv_bfloat16*>(dq);
     p.dk = static_cast<__nv_bfloat16*>(dk);
     p.dvo = static_cast<__nv_bfloat16*>(dv);
@@ -459,12 +546,19 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
     p.dvw = dvr;
     p.numerator_only = numerator_only;
     const dim3 grid((L + kTile - 1) / kTile, BH);
-    // statistics: own = queries (q, dout), looped = keys (k, v)
-    based_status st = launch_pass<DV, kModeStats, 64>(tq, tg, tk64, tv64, p, grid, "backward_tc_kernel<stats>", stream);
-    if (st != BASED_OK) return st;
-    // dq: own = queries (q, dout), looped = keys (k, v)
-    st = launch_pass<DV, kModeDq, 64>(tq, tg, tk64, tv64, p, grid, "backward_tc_kernel<dq>", stream);
-    if (st != BASED_OK) return st;
+    based_status st;
+    if (out != nullptr || numerator_only) {
+        // statistics and dq in one sweep (needs the forward output as the centre of the packed products)
+        st = launch_pass<DV, kModeDqS, 64>(tq, tg, tk64, tv64, p, grid, "backward_tc_kernel<stats+dq>", stream);
+        if (st != BASED_OK) return st;
+    } else {
+        // statistics: own = queries (q, dout), looped = keys (k, v)
+        st = launch_pass<DV, kModeStats, 64>(tq, tg, tk64, tv64, p, grid, "backward_tc_kernel<stats>", stream);
+        if (st != BASED_OK) return st;
+        // dq: own = queries (q, dout), looped = keys (k, v)
+        st = launch_pass<DV, kModeDq, 64>(tq, tg, tk64, tv64, p, grid, "backward_tc_kernel<dq>", stream);
+        if (st != BASED_OK) return st;
+    }
     // dk, dv: own = keys (k, v), looped = queries (q, dout)
     return launch_pass<DV, kModeDkDv, LTK>(tk, tv, tqL, tgL, p, grid, "backward_tc_kernel<dkdv>", stream);
 }
@@ -498,11 +592,11 @@ size_t backward_tc_workspace_bytes(int BH, int L, int d_v) {
     return (size_t)BH * L * 2 * sizeof(float);                 // (1 / D, b) per row
 }
 
-based_status launch_prefill_backward_tc(const void* q, const void* k, const void* v, const void* g, void* dq, void* dk,
-                                        void* dv, float* ws, int BH, int L, int d_v, int numerator_only,
-                                        cudaStream_t stream) {
-    if (d_v == 64) return launch_dvb<64>(q, k, v, g, dq, dk, dv, ws, BH, L, 64, numerator_only, stream);
-    return launch_dvb<128>(q, k, v, g, dq, dk, dv, ws, BH, L, d_v, numerator_only, stream);       // 112 or 128
+based_status launch_prefill_backward_tc(const void* q, const void* k, const void* v, const void* out, const void* g,
+                                        void* dq, void* dk, void* dv, float* ws, int BH, int L, int d_v,
+                                        int numerator_only, cudaStream_t stream) {
+    if (d_v == 64) return launch_dvb<64>(q, k, v, out, g, dq, dk, dv, ws, BH, L, 64, numerator_only, stream);
+    return launch_dvb<128>(q, k, v, out, g, dq, dk, dv, ws, BH, L, d_v, numerator_only, stream);  // 112 or 128
 }
 
 }  // namespace based

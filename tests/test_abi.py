@@ -143,6 +143,12 @@ def test_backward_validation(lib):
     assert f(q, k, v, g, dq, dk, dv, 1, 1, 8, 16, 96, 1, 0, ws, 1 << 20, None) == 2
     assert f(q, k, v, g, dq, dk, dv, *ok, 0, ws, 8, None) == 6                     # workspace too small
     assert f(q, k, v, g, dq, dk, dv, *ok, 0, None, 0, None) == 6
+    w = lib.based_prefill_backward_with_out
+    o = ctypes.c_void_p(0x9000)
+    assert w(q, k, v, None, g, dq, dk, dv, *ok, 0, ws, 1 << 20, None) == 1         # forward output missing
+    assert w(q, k, v, dv, g, dq, dk, dv, *ok, 0, ws, 1 << 20, None) == 1           # out aliases a gradient
+    assert w(q, k, v, U, g, dq, dk, dv, *ok, 0, ws, 1 << 20, None) == 3
+    assert w(q, k, v, o, g, dq, dk, dv, *ok, 0, ws, 8, None) == 6
 
 
 def test_binding_rejects_cpu_tensors():
