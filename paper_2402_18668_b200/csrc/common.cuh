@@ -82,7 +82,7 @@ based_status launch_prefill_simt(const void* q, const void* k, const void* v, vo
 size_t prefill_tc_workspace_bytes(int BH, int L, int d_v);
 based_status launch_prefill_tc(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH,
                                int L, int d_v, int flags, void* workspace, cudaStream_t stream);
-// bf16 tensor-core sliding window (window <= 64)
+// bf16 tensor-core sliding window (window <= 128)
 bool swa_tc_supported(int window);
 based_status launch_swa_tc(const void* q, const void* k, const void* v, void* out, int BH, int L, int window,
                            float scale, cudaStream_t stream);

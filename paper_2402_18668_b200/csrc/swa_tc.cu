@@ -1,6 +1,6 @@
 // swa_forward, bf16 tensor-core path (tcgen05 + TMEM + TMA): exact causal softmax
 // attention in a sliding window (Eq. (1) of Sec. 2 with the key set {i-w+1..i} of
-// Sec. 4.2), head dimension 64, window <= 64.
+// Sec. 4.2), head dimension 64, window <= 128.
 //
 // Persistent CTAs (one per SM) walk tiles of 128 consecutive queries of one head.  The 192
 // keys a tile can see (64 before its first query, then its own 128) are loaded once; per tile
@@ -13,6 +13,11 @@
 // The kernel is bound by HBM (512 B per token and head against ~50 k flop): a 3-stage TMA
 // ring prefetches tiles, and two softmax groups with one TMEM buffer each alternate tiles so
 // that loads, MMAs, softmax and stores of neighbouring tiles overlap.
+//
+// Windows of 65..128 keys run the same kernel with 128 keys before the tile (PAD = 128): 256 keys
+// per tile, a 2-stage ring, S[128,256] filling the tile's 256 tensor-memory columns, and a softmax
+// in two passes over the 160 columns a warp's rows can touch (maximum first, then exponentials and
+// the packed weights, 32 columns at a time, written over columns that have been read already).
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -25,21 +30,24 @@ using namespace sm100;
 namespace {
 
 constexpr int kQT = 128;                 // queries per tile
-constexpr int kPad = 64;                 // keys loaded before the tile's first query (>= window - 1)
-constexpr int kKeys = kQT + kPad;        // 192
 constexpr int kHD = 64;
-constexpr int kStages = 3;
 constexpr int kThreads = 320;            // 2 softmax groups of 4 warps, TMA producer warp, MMA warp
 constexpr int kWarpTma = 8, kWarpMma = 9;
 constexpr uint32_t kQBytes = kQT * kHD * 2;      // 16 KB
-constexpr uint32_t kKVBytes = kKeys * kHD * 2;   // 24 KB
-constexpr uint32_t kStageBytes = kQBytes + 2 * kKVBytes;   // 64 KB
-constexpr uint32_t offOut = kStages * kStageBytes;         // two 16 KB output staging tiles (one per group)
-constexpr uint32_t offBars = offOut + 2 * kQBytes;
-constexpr uint32_t kSmemBytes = offBars + 256 + 1024;
-static_assert(kSmemBytes <= 232448, "shared memory budget");
+// PAD: keys loaded before the tile's first query (>= window - 1): 64 or 128
+template <int PAD> struct SwaCfg {
+    static constexpr int kPad = PAD;
+    static constexpr int kKeys = kQT + PAD;                        // 192 / 256
+    static constexpr int kStages = PAD == 64 ? 3 : 2;
+    static constexpr uint32_t kKVBytes = kKeys * kHD * 2;          // 24 / 32 KB
+    static constexpr uint32_t kStageBytes = kQBytes + 2 * kKVBytes;   // 64 / 80 KB
+    static constexpr uint32_t offOut = kStages * kStageBytes;      // two 16 KB output staging tiles (one per group)
+    static constexpr uint32_t offBars = offOut + 2 * kQBytes;
+    static constexpr uint32_t kSmemBytes = offBars + 256 + 1024;
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
+};
 constexpr uint32_t kBufCols = 256;               // TMEM columns per tile in flight
-constexpr uint32_t colS = 0, colO = 128;         // P overwrites columns [0, 96) of S; O uses dead S columns
+constexpr uint32_t colS = 0, colO = 128;         // P overwrites the first half of S's columns; O uses dead S columns
 
 enum SwaBar { bFull = 0, bEmpty = 3, bS = 6, bP = 8, bO = 10, bOfree = 12, bCount = 14 };
 
@@ -81,10 +89,14 @@ struct SwaParams {
 
 // Persistent kernel: CTA j handles tiles j, j + gridDim.x, ...  Tile n of a CTA uses shared
 // memory stage n % 3 and TMEM buffer n % 2; softmax group n % 2 owns it.
+template <int PAD>
 __global__ void __launch_bounds__(kThreads, 1)
     swa_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
                   const SwaParams p) {
+    using C = SwaCfg<PAD>;
+    constexpr int kPad = C::kPad, kKeys = C::kKeys, kStages = C::kStages;
+    constexpr uint32_t kKVBytes = C::kKVBytes, kStageBytes = C::kStageBytes, offOut = C::offOut, offBars = C::offBars;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + offBars);
@@ -120,7 +132,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const int tile = blockIdx.x + n * gridDim.x;
                 const int head = tile / p.tiles_per_head, i0 = (tile % p.tiles_per_head) * kQT;
                 uint8_t* st = smem + s * kStageBytes;
-                // Q tile, and K, V rows i0-64 .. i0+127 (rows before the sequence start read as zero)
+                // Q tile, and K, V rows i0-PAD .. i0+127 (rows before the sequence start read as zero)
                 mbar_arrive_expect_tx(&bars[bFull + s], kStageBytes);
                 tma_load_3d(st, &tm_q, &bars[bFull + s], 0, i0, head);
                 tma_load_3d(st + kQBytes, &tm_k, &bars[bFull + s], 0, i0 - kPad, head);
@@ -179,7 +191,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int wq = warp & 3;                     // lane quarter
         const int r = tid & 127;
         const uint32_t lane_base = (uint32_t)wq * 32u;
-        const int c0 = wq * 32;                      // first score column this warp reads (96 columns from here)
+        const int c0 = wq * 32;                      // first score column this warp reads (PAD + 32 columns from here)
         uint8_t* ostage = smem + offOut + g * kQBytes;
         uint8_t* orow = ostage + (r >> 3) * 1024 + (r & 7) * 128;
         const uint32_t sw = r & 7;
@@ -188,64 +200,110 @@ __global__ void __launch_bounds__(kThreads, 1)
             const uint32_t ph = (n >> 1) & 1;
             const int tile = blockIdx.x + n * gridDim.x;
             const int head = tile / p.tiles_per_head, i0 = (tile % p.tiles_per_head) * kQT;
-            // visible columns of this row inside the 96-column batch: keys i-w+1 .. i, and key >= 0
+            // visible columns of this row inside its warp's batch of PAD + 32 columns: keys i-w+1 .. i, and key >= 0
             const int jhi = lane + kPad;
             int jlo = lane + kPad + 1 - p.window;
-            jlo = max(jlo, kPad - i0 - c0);          // key index i0 - 64 + c0 + j must not be negative
+            jlo = max(jlo, kPad - i0 - c0);          // key index i0 - PAD + c0 + j must not be negative
             auto mask_word = [&](int base) -> uint32_t {
                 const int a = max(jlo - base, 0), b = min(jhi - base, 31);
                 if (a > b) return 0u;
                 return (b - a == 31) ? 0xffffffffu : (((1u << (b - a + 1)) - 1u) << a);
             };
-            const uint32_t mk[3] = {mask_word(0), mask_word(32), mask_word(64)};
-
-            ok = group_all(1 + g, mbar_wait(&bars[bS + g], ph, abort_flag));
-            if (!ok) break;
-            tc_fence_after();
             float inv_l;
-            {
-                uint32_t s[96];
+            if constexpr (PAD == 64) {
+                const uint32_t mk[3] = {mask_word(0), mask_word(32), mask_word(64)};
+
+                ok = group_all(1 + g, mbar_wait(&bars[bS + g], ph, abort_flag));
+                if (!ok) break;
+                tc_fence_after();
                 {
-                    uint32_t t0[32], t1[32], t2[32];
-                    tmem_ld32(tmem_addr(tbuf, lane_base, colS + c0), t0);
-                    tmem_ld32(tmem_addr(tbuf, lane_base, colS + c0 + 32), t1);
-                    tmem_ld32(tmem_addr(tbuf, lane_base, colS + c0 + 64), t2);
-                    tmem_wait_ld();
+                    uint32_t s[96];
+                    {
+                        uint32_t t0[32], t1[32], t2[32];
+                        tmem_ld32(tmem_addr(tbuf, lane_base, colS + c0), t0);
+                        tmem_ld32(tmem_addr(tbuf, lane_base, colS + c0 + 32), t1);
+                        tmem_ld32(tmem_addr(tbuf, lane_base, colS + c0 + 64), t2);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) { s[i] = t0[i]; s[32 + i] = t1[i]; s[64 + i] = t2[i]; }
+                        for (int i = 0; i < 32; ++i) { s[i] = t0[i]; s[32 + i] = t1[i]; s[64 + i] = t2[i]; }
+                    }
+                    float mx = -INFINITY;
+#pragma unroll
+                    for (int j = 0; j < 96; ++j) {
+                        const bool v = (mk[j >> 5] >> (j & 31)) & 1u;
+                        const float x = v ? __uint_as_float(s[j]) : -INFINITY;
+                        s[j] = __float_as_uint(x);
+                        mx = fmaxf(mx, x);
+                    }
+                    const float mc = mx * p.scale_log2e;     // every row sees at least its own key, so mx is finite
+                    float l = 0.f;
+                    uint32_t pk[48];
+#pragma unroll
+                    for (int j = 0; j < 48; ++j) {
+                        const float e0 = ex2(fmaf(__uint_as_float(s[2 * j]), p.scale_log2e, -mc));
+                        const float e1 = ex2(fmaf(__uint_as_float(s[2 * j + 1]), p.scale_log2e, -mc));
+                        l += e0 + e1;
+                        pk[j] = pack2(e0, e1);
+                    }
+                    inv_l = 1.0f / l;
+                    // P row: 192 keys = 96 packed columns; this warp's batch sits at packed columns [16 wq, 16 wq + 48)
+                    uint32_t zero[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) zero[i] = 0u;
+#pragma unroll
+                    for (int gg = 0; gg < 6; ++gg)
+                        if (gg < wq || gg > wq + 2) tmem_st16(tmem_addr(tbuf, lane_base, colS + gg * 16), zero);
+                    uint32_t d0[16], d1[16], d2[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) { d0[i] = pk[i]; d1[i] = pk[16 + i]; d2[i] = pk[32 + i]; }
+                    tmem_st16(tmem_addr(tbuf, lane_base, colS + wq * 16), d0);
+                    tmem_st16(tmem_addr(tbuf, lane_base, colS + wq * 16 + 16), d1);
+                    tmem_st16(tmem_addr(tbuf, lane_base, colS + wq * 16 + 32), d2);
                 }
+            } else {
+                // 160 columns per row: two passes of five 32-column loads (maximum, then weights); the packed
+                // weights of a block go over columns that this row has read already
+                ok = group_all(1 + g, mbar_wait(&bars[bS + g], ph, abort_flag));
+                if (!ok) break;
+                tc_fence_after();
                 float mx = -INFINITY;
+#pragma unroll 1
+                for (int b = 0; b < 5; ++b) {
+                    uint32_t t[32];
+                    tmem_ld32(tmem_addr(tbuf, lane_base, colS + c0 + 32 * b), t);
+                    tmem_wait_ld();
+                    const uint32_t m = mask_word(32 * b);
 #pragma unroll
-                for (int j = 0; j < 96; ++j) {
-                    const bool v = (mk[j >> 5] >> (j & 31)) & 1u;
-                    const float x = v ? __uint_as_float(s[j]) : -INFINITY;
-                    s[j] = __float_as_uint(x);
-                    mx = fmaxf(mx, x);
+                    for (int i = 0; i < 32; ++i)
+                        if ((m >> i) & 1u) mx = fmaxf(mx, __uint_as_float(t[i]));
                 }
                 const float mc = mx * p.scale_log2e;     // every row sees at least its own key, so mx is finite
                 float l = 0.f;
-                uint32_t pk[48];
+#pragma unroll 1
+                for (int b = 0; b < 5; ++b) {
+                    uint32_t t[32], pk[16];
+                    tmem_ld32(tmem_addr(tbuf, lane_base, colS + c0 + 32 * b), t);
+                    tmem_wait_ld();
+                    const uint32_t m = mask_word(32 * b);
 #pragma unroll
-                for (int j = 0; j < 48; ++j) {
-                    const float e0 = ex2(fmaf(__uint_as_float(s[2 * j]), p.scale_log2e, -mc));
-                    const float e1 = ex2(fmaf(__uint_as_float(s[2 * j + 1]), p.scale_log2e, -mc));
-                    l += e0 + e1;
-                    pk[j] = pack2(e0, e1);
+                    for (int j = 0; j < 16; ++j) {
+                        const float x0 = ((m >> (2 * j)) & 1u) ? __uint_as_float(t[2 * j]) : -INFINITY;
+                        const float x1 = ((m >> (2 * j + 1)) & 1u) ? __uint_as_float(t[2 * j + 1]) : -INFINITY;
+                        const float e0 = ex2(fmaf(x0, p.scale_log2e, -mc));
+                        const float e1 = ex2(fmaf(x1, p.scale_log2e, -mc));
+                        l += e0 + e1;
+                        pk[j] = pack2(e0, e1);
+                    }
+                    tmem_st16(tmem_addr(tbuf, lane_base, colS + wq * 16 + b * 16), pk);
                 }
                 inv_l = 1.0f / l;
-                // P row: 192 keys = 96 packed columns; this warp's batch sits at packed columns [16 wq, 16 wq + 48)
+                // P row: 256 keys = 128 packed columns; this warp's batch sits at packed columns [16 wq, 16 wq + 80)
                 uint32_t zero[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) zero[i] = 0u;
 #pragma unroll
-                for (int gg = 0; gg < 6; ++gg)
-                    if (gg < wq || gg > wq + 2) tmem_st16(tmem_addr(tbuf, lane_base, colS + gg * 16), zero);
-                uint32_t d0[16], d1[16], d2[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) { d0[i] = pk[i]; d1[i] = pk[16 + i]; d2[i] = pk[32 + i]; }
-                tmem_st16(tmem_addr(tbuf, lane_base, colS + wq * 16), d0);
-                tmem_st16(tmem_addr(tbuf, lane_base, colS + wq * 16 + 16), d1);
-                tmem_st16(tmem_addr(tbuf, lane_base, colS + wq * 16 + 32), d2);
+                for (int gg = 0; gg < 8; ++gg)
+                    if (gg < wq || gg > wq + 4) tmem_st16(tmem_addr(tbuf, lane_base, colS + gg * 16), zero);
             }
             tmem_wait_st();
             tc_fence_before();
@@ -326,12 +384,14 @@ bool make_map(CUtensorMap* m, const void* base, int BH, int L, int box_rows) {
 
 }  // namespace
 
-bool swa_tc_supported(int window) { return window >= 1 && window <= kPad; }
+bool swa_tc_supported(int window) { return window >= 1 && window <= 128; }
 
-based_status launch_swa_tc(const void* q, const void* k, const void* v, void* out, int BH, int L, int window,
-                           float scale, cudaStream_t stream) {
+template <int PAD>
+static based_status launch_swa_pad(const void* q, const void* k, const void* v, void* out, int BH, int L, int window,
+                                   float scale, cudaStream_t stream) {
+    using C = SwaCfg<PAD>;
     CUtensorMap tq, tk, tv, to;
-    if (!make_map(&tq, q, BH, L, kQT) || !make_map(&tk, k, BH, L, kKeys) || !make_map(&tv, v, BH, L, kKeys) ||
+    if (!make_map(&tq, q, BH, L, kQT) || !make_map(&tk, k, BH, L, C::kKeys) || !make_map(&tv, v, BH, L, C::kKeys) ||
         !make_map(&to, out, BH, L, kQT))
         return BASED_ERR_CUDA;
     SwaParams p;
@@ -347,8 +407,8 @@ based_status launch_swa_tc(const void* q, const void* k, const void* v, void* ou
     {
         std::lock_guard<std::mutex> lock(setup_mutex());
         if (sm_count[dev] == 0) {
-            if (cudaFuncSetAttribute(swa_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) !=
-                cudaSuccess)
+            if (cudaFuncSetAttribute(swa_tc_kernel<PAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)C::kSmemBytes) != cudaSuccess)
                 return BASED_ERR_CUDA;
             int n = 148;
             cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
@@ -357,9 +417,15 @@ based_status launch_swa_tc(const void* q, const void* k, const void* v, void* ou
     }
     const int sms = sm_count[dev];
     const int grid = p.total_tiles < sms ? p.total_tiles : sms;
-    swa_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tq, tk, tv, to, p);
+    swa_tc_kernel<PAD><<<grid, kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
     note_launch();
     return check_launch("swa_tc_kernel");
+}
+
+based_status launch_swa_tc(const void* q, const void* k, const void* v, void* out, int BH, int L, int window,
+                           float scale, cudaStream_t stream) {
+    if (window <= 64) return launch_swa_pad<64>(q, k, v, out, BH, L, window, scale, stream);
+    return launch_swa_pad<128>(q, k, v, out, BH, L, window, scale, stream);
 }
 
 }  // namespace based

@@ -601,7 +601,8 @@ def test_sym_and_full_decode_agree_at_generation_batch():
 
 # --------------------------------------------------------------------------- sliding window
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("L,window", [(1, 64), (63, 64), (64, 64), (333, 64), (200, 1), (257, 17), (400, 128), (130, 100)])
+@pytest.mark.parametrize("L,window", [(1, 64), (63, 64), (64, 64), (333, 64), (200, 1), (257, 17), (400, 128), (130, 100),
+                                      (1000, 65), (777, 127), (129, 128), (1, 128), (2048, 96)])
 def test_swa_small_shapes(dtype, L, window):
     tdt = torch.float32 if dtype == "f32" else torch.bfloat16
     q, k, v = wl.swa_standalone_inputs(2, 3, L, 64, tdt, wl.generator(L + window))
@@ -736,6 +737,23 @@ def test_full_size_mixer_pair_sampled():
         sl = (slice(b, b + 1), slice(h, h + 1))
         ref = oracle.swa(_np(qs[sl]), _np(ks[sl]), _np(v[sl]), w.swa_window)
         assert row_err(_np(out_swa[sl]), ref) <= TOL_BF16
+
+
+@pytest.mark.parametrize("window", [100, 128])
+def test_full_size_wide_window_sampled(window):
+    """The mixer pair's sequence length (B2 H16 L32768, bf16) with the widest windows the paper allows
+    (tensor-core path with 128 keys before each query tile): three whole heads against the oracle."""
+    w = wl.CONFIGS["cfg5_mixer_pair"]
+    gen = wl.generator(window)
+    _, _, v = wl.prefill_inputs(w, gen)
+    qs, ks = wl.swa_inputs(w, gen)
+    out = based.swa_forward(qs.to(DEV), ks.to(DEV), v.to(DEV), window=window).cpu()
+    _poll()
+    for bh in (0, 9, w.B * w.H - 1):
+        b, h = divmod(bh, w.H)
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        ref = oracle.swa(_np(qs[sl]), _np(ks[sl]), _np(v[sl]), window)
+        assert row_err(_np(out[sl]), ref) <= TOL_BF16
 
 
 def test_full_size_generation_sampled():
