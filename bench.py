@@ -357,7 +357,7 @@ def bench_swa(w, steps, warmup, torch, based, dist_on, peaks):
 
     def step(i):
         q, k, v, o = sets[i % len(sets)]
-        based.swa_forward(q, k, v, out=o, window=w.swa_window)
+        based.swa_forward(q, k, v, out=o, window=w.swa_window)      # windows above 64: the kernel's 128-key-halo variant
 
     ms = time_region(step, steps, warmup, torch, dist_on)
     assert based.based_poll_error() == 0
@@ -368,6 +368,42 @@ def bench_swa(w, steps, warmup, torch, based, dist_on, peaks):
         "roofline": {"bound": "hbm", "achieved": per_set / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": per_set / t / 1e9 / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC.get(w.name + ":swa"),
                      "kernel": "swa_tc_kernel", "algorithmic_bytes": per_set, "peak_source": peaks["source"]},
+    }
+
+
+def bench_prefill_dfeat(w, steps, warmup, torch, based, dist_on, peaks):
+    """based_prefill for a feature dimension other than 16 (bf16, empty initial state, final state
+    returned): the definition form on the tile kernel's forward mode plus the tensor-core state
+    kernel.  Flops: the pairs' scores and weighted values, and the state's 2 D d_v per token."""
+    g = torch.Generator(device="cuda").manual_seed(9)
+    dt = w.torch_dtype
+    sets = []
+    per_set = w.B * w.H * w.L * (2 * w.d_feat + 2 * w.d_v) * 2.0
+    for _ in range(n_sets_for(per_set)):
+        q = (torch.randn(w.B, w.H, w.L, w.d_feat, generator=g, device="cuda") * w.qk_scale).to(dt)
+        k = (torch.randn(w.B, w.H, w.L, w.d_feat, generator=g, device="cuda") * w.qk_scale).to(dt)
+        v = torch.randn(w.B, w.H, w.L, w.d_v, generator=g, device="cuda").to(dt)
+        sets.append((q, k, v, torch.empty_like(v)))
+    kv, z = based.new_state(w.B, w.H, w.d_v, d_feat=w.d_feat)
+
+    def step(i):
+        q, k, v, o = sets[i % len(sets)]
+        based.based_prefill(q, k, v, out=o, kv_state=kv, z_state=z)
+
+    n0 = based.launch_count()
+    ms = time_region(step, steps, warmup, torch, dist_on)
+    assert based.based_poll_error() == 0
+    t = ms * 1e-3 / steps
+    pairs = w.B * w.H * w.L * (w.L + 1) / 2.0
+    flops = 2.0 * pairs * (w.d_feat + w.d_v) + 2.0 * w.B * w.H * w.L * w.D * w.d_v
+    return {
+        "workload": f"{w.name} with d' = {w.d_feat} (D = {w.D}), final state returned", "metric": "prefill_tokens_per_s",
+        "value": w.B * w.L / t, "unit": "tokens/s", "ms_per_step": t * 1e3, "steps": steps,
+        "launches_per_step": (based.launch_count() - n0) // (steps + warmup),
+        "roofline": {"bound": "tensor", "achieved": flops / t / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": flops / t / 1e12 / peaks["bf16_tflops"], "traffic": None,
+                     "kernel": "backward_tc_kernel<fwd> + generic_state_tc_kernel", "algorithmic_flops": flops,
+                     "peak_source": peaks["source"]},
     }
 
 
@@ -529,9 +565,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_360m_prefill")
     ap.add_argument("--skip-extras", action="store_true", help="only the headline prefill workload")
-    ap.add_argument("--profile", choices=["prefill", "decode", "decode_sym", "swa", "swa_decode", "generation_graph", "baseconv", "backward"],
+    ap.add_argument("--profile", choices=["prefill", "decode", "decode_sym", "swa", "swa_decode", "generation_graph", "baseconv", "backward",
+                             "prefill_dfeat"],
                     help="run only this arm on --shape (small cases for ncu captures) and print its result")
     ap.add_argument("--shape", default="", help="B,H,L,d_v for --profile (defaults to the arm's benchmark shape)")
+    ap.add_argument("--window", type=int, default=0, help="--profile swa: window (default: the workload's 64)")
+    ap.add_argument("--d-feat", type=int, default=32, help="--profile prefill_dfeat: feature dimension (8, 24, 32)")
     args = ap.parse_args()
     if args.warmup < 3 and not args.profile:
         args.warmup = 3
@@ -580,7 +619,10 @@ def main():
         base = {"prefill": w, "decode": wl.CONFIGS["cfg4_generation"], "decode_sym": wl.CONFIGS["cfg4_generation"], "swa": wl.CONFIGS["cfg5_mixer_pair"],
                 "swa_decode": wl.CONFIGS["cfg4_generation"],
                 "generation_graph": wl.CONFIGS["cfg4_generation"],
-                "baseconv": wl.CONFIGS["cfg3_1p3b_prefill"], "backward": w}[args.profile]
+                "baseconv": wl.CONFIGS["cfg3_1p3b_prefill"], "backward": w,
+                "prefill_dfeat": w.scaled(d_feat=args.d_feat, qk_scale=0.4)}[args.profile]
+        if args.profile == "swa" and args.window > 0:
+            base = base.scaled(name=f"{base.name}[window {args.window}]", swa_window=args.window)
         if args.shape and args.profile != "baseconv":
             B, H, L, dv = (int(x) for x in args.shape.split(","))
             base = base.scaled(name=f"{base.name}[{args.shape}]", B=B, H=H, L=L, d_v=dv)
@@ -593,6 +635,8 @@ def main():
             r = bench_swa_decode(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         elif args.profile == "backward":
             r = bench_backward(base, args.steps, args.warmup, torch, based, dist_on, peaks)
+        elif args.profile == "prefill_dfeat":
+            r = bench_prefill_dfeat(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         elif args.profile == "baseconv":
             shp = (8, 4096, 8192)
             if args.shape:

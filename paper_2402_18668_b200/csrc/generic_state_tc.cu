@@ -41,7 +41,7 @@ template <int DV> struct SCfg {
     static constexpr int kVB = (DV + 63) / 64;                 // 64-column blocks of the v tile (112 -> 2)
     static constexpr int kNS = DV == 64 ? 4 : 3;               // load stages
     static constexpr uint32_t kVBytes = kVB * kTB * 128;       // [64 tokens][64 * kVB] bf16, SWIZZLE_128B blocks
-    static constexpr uint32_t kKBytes = kTB * 64;              // [64 tokens][32] bf16, plain 64-byte rows
+    static constexpr uint32_t kKBytes = kTB * 64;              // [64 tokens][32] bf16, 64-byte rows, SWIZZLE_64B
     static constexpr uint32_t kStage = kVBytes + kKBytes;
     static constexpr uint32_t kABytes = kFB * 128;             // [128 features][64 tokens] bf16
     static constexpr uint32_t offA = kNS * kStage;
@@ -182,18 +182,20 @@ __global__ void __launch_bounds__(kThreadsS, 1)
             const int b = it % kNA, s = it % C::kNS;
             ok = rows_and(mbar_wait(&bars[sFull0 + s], (it / C::kNS) & 1, abort_flag));
             if (!ok) break;
-            // transpose the k tile: thread (token t / 2, half t % 2) moves 16 columns
+            // transpose the k tile ([token][m], 64-byte rows, SWIZZLE_64B): warp w moves the 16-byte pieces
+            // w / 2 and w / 2 + 2 of tokens 32 (w % 2) + lane, so a warp's loads hit distinct banks and its
+            // 2-byte stores fill consecutive words of one transposed row
             __nv_bfloat16* kt = reinterpret_cast<__nv_bfloat16*>(smem + C::offKT + (it & 1) * C::kKTBytes);
             {
-                const int j = t >> 1, h = t & 1;
-                const uint4* src = reinterpret_cast<const uint4*>(smem + s * C::kStage + C::kVBytes + j * 64 + h * 32);
-                const uint4 u0 = src[0], u1 = src[1];
-                const __nv_bfloat16* e0 = reinterpret_cast<const __nv_bfloat16*>(&u0);
-                const __nv_bfloat16* e1 = reinterpret_cast<const __nv_bfloat16*>(&u1);
+                const int j = lane + 32 * (warp & 1);
+                const uint8_t* krow = smem + s * C::kStage + C::kVBytes + j * 64;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    kt[(h * 16 + i) * kKT + j] = e0[i];
-                    kt[(h * 16 + 8 + i) * kKT + j] = e1[i];
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int c = (warp >> 1) + 2 * cc;
+                    const uint4 u = *reinterpret_cast<const uint4*>(krow + ((c ^ ((j >> 1) & 3)) << 4));
+                    const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&u);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) kt[(c * 8 + i) * kKT + j] = e[i];
                 }
                 if (t < kTB) kt[kRowOne * kKT + t] = __float2bfloat16(it * kTB + t < p.L ? 1.0f : 0.0f);
             }
@@ -203,12 +205,14 @@ __global__ void __launch_bounds__(kThreadsS, 1)
             const uint4* rm = reinterpret_cast<const uint4*>(kt + m * kKT);
             const uint4* rn = reinterpret_cast<const uint4*>(kt + n * kKT);
             uint8_t* a_row = a_row0 + b * C::kABytes;
+            uint4 xm[kTB / 8], xn[kTB / 8];                  // all sixteen loads in flight before the first product
+#pragma unroll
+            for (int c = 0; c < kTB / 8; ++c) { xm[c] = rm[c]; xn[c] = rn[c]; }
 #pragma unroll
             for (int c = 0; c < kTB / 8; ++c) {
-                const uint4 xm = rm[c], xn = rn[c];
                 uint4 pr;
-                const __nv_bfloat162* hm = reinterpret_cast<const __nv_bfloat162*>(&xm);
-                const __nv_bfloat162* hn = reinterpret_cast<const __nv_bfloat162*>(&xn);
+                const __nv_bfloat162* hm = reinterpret_cast<const __nv_bfloat162*>(&xm[c]);
+                const __nv_bfloat162* hn = reinterpret_cast<const __nv_bfloat162*>(&xn[c]);
                 __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&pr);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) hp[i] = __hmul2(hm[i], hn[i]);
@@ -264,7 +268,7 @@ based_status launch_state_dv(const void* k, const void* v, float* kv, float* z, 
                              int cont, cudaStream_t stream) {
     using C = SCfg<DV>;
     CUtensorMap tk, tv;
-    if (!make_rows_map_bf16(&tk, k, BH, L, df, 32, kTB, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+    if (!make_rows_map_bf16(&tk, k, BH, L, df, 32, kTB, CU_TENSOR_MAP_SWIZZLE_64B) ||
         !make_rows_map_bf16(&tv, v, BH, L, dvw, 64, kTB, CU_TENSOR_MAP_SWIZZLE_128B))
         return BASED_ERR_CUDA;
     SParams p{};
