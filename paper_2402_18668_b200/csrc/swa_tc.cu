@@ -15,9 +15,12 @@
 // that loads, MMAs, softmax and stores of neighbouring tiles overlap.
 //
 // Windows of 65..128 keys run the same kernel with 128 keys before the tile (PAD = 128): 256 keys
-// per tile, a 2-stage ring, S[128,256] filling the tile's 256 tensor-memory columns, and a softmax
-// in two passes over the 160 columns a warp's rows can touch (maximum first, then exponentials and
-// the packed weights, 32 columns at a time, written over columns that have been read already).
+// per tile, S[128,256] filling the tile's 256 tensor-memory columns, and a softmax in two passes
+// over the 160 columns a warp's rows can touch (maximum first, then exponentials and the packed
+// weights, 32 columns at a time, written over columns that have been read already).  Each CTA
+// walks a contiguous run of tiles, so the 128 rows of K and V before a tile are the ones the tile
+// before it loaded: a tile loads only its own rows (48 KB with Q) into one of four slots, and the
+// MMAs address two slots (two N = 128 score products per K step, the P V steps over two V blocks).
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -37,10 +40,12 @@ constexpr uint32_t kQBytes = kQT * kHD * 2;      // 16 KB
 // PAD: keys loaded before the tile's first query (>= window - 1): 64 or 128
 template <int PAD> struct SwaCfg {
     static constexpr int kPad = PAD;
-    static constexpr int kKeys = kQT + PAD;                        // 192 / 256
-    static constexpr int kStages = PAD == 64 ? 3 : 2;
-    static constexpr uint32_t kKVBytes = kKeys * kHD * 2;          // 24 / 32 KB
-    static constexpr uint32_t kStageBytes = kQBytes + 2 * kKVBytes;   // 64 / 80 KB
+    static constexpr int kKeys = kQT + PAD;                        // 192 / 256 keys under a tile's scores
+    // PAD 64: a stage holds a tile's Q and its 192 rows of K and of V.  PAD 128: a slot holds a tile's Q and its
+    // own 128 rows of K and of V; the 128 rows before them are the previous tile's, still in the slot before.
+    static constexpr int kStages = PAD == 64 ? 3 : 4;
+    static constexpr uint32_t kKVBytes = (PAD == 64 ? kKeys : kQT) * kHD * 2;   // 24 / 16 KB
+    static constexpr uint32_t kStageBytes = kQBytes + 2 * kKVBytes;   // 64 / 48 KB
     static constexpr uint32_t offOut = kStages * kStageBytes;      // two 16 KB output staging tiles (one per group)
     static constexpr uint32_t offBars = offOut + 2 * kQBytes;
     static constexpr uint32_t kSmemBytes = offBars + 256 + 1024;
@@ -49,7 +54,7 @@ template <int PAD> struct SwaCfg {
 constexpr uint32_t kBufCols = 256;               // TMEM columns per tile in flight
 constexpr uint32_t colS = 0, colO = 128;         // P overwrites the first half of S's columns; O uses dead S columns
 
-enum SwaBar { bFull = 0, bEmpty = 3, bS = 6, bP = 8, bO = 10, bOfree = 12, bCount = 14 };
+enum SwaBar { bFull = 0, bEmpty = 4, bS = 8, bP = 10, bO = 12, bOfree = 14, bCount = 16 };
 
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -104,7 +109,13 @@ __global__ void __launch_bounds__(kThreads, 1)
     volatile uint32_t* abort_flag = tmem_base_s + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int ntiles = (p.total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // tiles of this CTA
+    // PAD 64: CTA j takes tiles j, j + gridDim.x, ...; PAD 128: a contiguous run of tiles, so that a tile's
+    // first 128 keys are the rows the tile before it loaded
+    const int run_first = (int)((long long)p.total_tiles * blockIdx.x / gridDim.x);
+    const int run_last = (int)((long long)p.total_tiles * (blockIdx.x + 1) / gridDim.x);
+    const int ntiles = PAD == 64 ? (p.total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x
+                                 : run_last - run_first;
+    auto tile_of = [&](int n) -> int { return PAD == 64 ? (int)blockIdx.x + n * (int)gridDim.x : run_first + n; };
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&bars[bFull + s], 1); mbar_init(&bars[bEmpty + s], 1); }
@@ -125,18 +136,37 @@ __global__ void __launch_bounds__(kThreads, 1)
 
     if (warp == kWarpTma) {
         if (lane == 0) {
-            for (int n = 0; n < ntiles && ok; ++n) {
-                const int s = n % kStages;
-                ok = mbar_wait(&bars[bEmpty + s], ((n / kStages) & 1) ^ 1, abort_flag);
-                if (!ok) break;
-                const int tile = blockIdx.x + n * gridDim.x;
-                const int head = tile / p.tiles_per_head, i0 = (tile % p.tiles_per_head) * kQT;
-                uint8_t* st = smem + s * kStageBytes;
-                // Q tile, and K, V rows i0-PAD .. i0+127 (rows before the sequence start read as zero)
-                mbar_arrive_expect_tx(&bars[bFull + s], kStageBytes);
-                tma_load_3d(st, &tm_q, &bars[bFull + s], 0, i0, head);
-                tma_load_3d(st + kQBytes, &tm_k, &bars[bFull + s], 0, i0 - kPad, head);
-                tma_load_3d(st + kQBytes + kKVBytes, &tm_v, &bars[bFull + s], 0, i0 - kPad, head);
+            if constexpr (PAD == 64) {
+                for (int n = 0; n < ntiles && ok; ++n) {
+                    const int s = n % kStages;
+                    ok = mbar_wait(&bars[bEmpty + s], ((n / kStages) & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    const int tile = tile_of(n);
+                    const int head = tile / p.tiles_per_head, i0 = (tile % p.tiles_per_head) * kQT;
+                    uint8_t* st = smem + s * kStageBytes;
+                    // Q tile, and K, V rows i0-PAD .. i0+127 (rows before the sequence start read as zero)
+                    mbar_arrive_expect_tx(&bars[bFull + s], kStageBytes);
+                    tma_load_3d(st, &tm_q, &bars[bFull + s], 0, i0, head);
+                    tma_load_3d(st + kQBytes, &tm_k, &bars[bFull + s], 0, i0 - kPad, head);
+                    tma_load_3d(st + kQBytes + kKVBytes, &tm_v, &bars[bFull + s], 0, i0 - kPad, head);
+                }
+            } else {
+                // load m = 0: the 128 rows of K and V before the run's first tile (zeros at a head's start);
+                // load m >= 1: Q, K, V rows of tile m - 1.  Slot m % 4; a slot is free once the tile that
+                // used it as "rows before" has finished its P V products.
+                for (int m = 0; m <= ntiles && ok && ntiles > 0; ++m) {
+                    const int s = m % kStages;
+                    ok = mbar_wait(&bars[bEmpty + s], ((m / kStages) & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    const int tile = tile_of(m == 0 ? 0 : m - 1);
+                    const int head = tile / p.tiles_per_head;
+                    const int i0 = (tile % p.tiles_per_head) * kQT - (m == 0 ? kQT : 0);
+                    uint8_t* st = smem + s * kStageBytes;
+                    mbar_arrive_expect_tx(&bars[bFull + s], m == 0 ? 2 * kKVBytes : kStageBytes);
+                    if (m > 0) tma_load_3d(st, &tm_q, &bars[bFull + s], 0, i0, head);
+                    tma_load_3d(st + kQBytes, &tm_k, &bars[bFull + s], 0, i0, head);
+                    tma_load_3d(st + kQBytes + kKVBytes, &tm_v, &bars[bFull + s], 0, i0, head);
+                }
             }
         }
     } else if (warp == kWarpMma) {
@@ -144,44 +174,105 @@ __global__ void __launch_bounds__(kThreads, 1)
             constexpr uint64_t dK = make_smem_desc_base(16, 1024, kSwizzle128B);   // K-major rows / MN-major block
             constexpr uint32_t iS = make_idesc_bf16(kQT, kKeys, 0, 0);
             constexpr uint32_t iO = make_idesc_bf16(kQT, kHD, 0, 1);
-            auto issue_pv = [&](int n) {
-                const uint32_t tbuf = tb + (n & 1) * kBufCols;
-                const uint32_t lV = desc_lo(dK) + (smem_u32(smem + (n % kStages) * kStageBytes + kQBytes + kKVBytes) >> 4);
-                mma_ts_lh<false>(tbuf + colO, tbuf + colS, lV, desc_hi(dK), iO);
+            if constexpr (PAD == 64) {
+                auto issue_pv = [&](int n) {
+                    const uint32_t tbuf = tb + (n & 1) * kBufCols;
+                    const uint32_t lV = desc_lo(dK) + (smem_u32(smem + (n % kStages) * kStageBytes + kQBytes + kKVBytes) >> 4);
+                    mma_ts_lh<false>(tbuf + colO, tbuf + colS, lV, desc_hi(dK), iO);
 #pragma unroll
-                for (int k = 1; k < kKeys / 16; ++k)
-                    mma_ts_lh<true>(tbuf + colO, tbuf + colS + k * 8, lV + k * (2048 >> 4), desc_hi(dK), iO);
-                mma_commit(&bars[bO + (n & 1)]);
-                mma_commit(&bars[bEmpty + n % kStages]);     // K, V (and Q) of this stage are dead
-            };
-            for (int n = 0; n < ntiles && ok; ++n) {
-                const int s = n % kStages, b = n & 1;
-                ok = mbar_wait(&bars[bFull + s], (n / kStages) & 1, abort_flag);
-                // the buffer's previous tile (n - 2) must have been read out
-                if (ok && n >= 2) ok = mbar_wait(&bars[bOfree + b], ((n >> 1) - 1) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t tbuf = tb + b * kBufCols;
-                const uint32_t lQ = desc_lo(dK) + (smem_u32(smem + s * kStageBytes) >> 4);
-                const uint32_t lK = lQ + (kQBytes >> 4);
-                mma_ss_lh<false>(tbuf + colS, lQ, desc_hi(dK), lK, desc_hi(dK), iS);
-#pragma unroll
-                for (int k = 1; k < kHD / 16; ++k)
-                    mma_ss_lh<true>(tbuf + colS, lQ + k * 2, desc_hi(dK), lK + k * 2, desc_hi(dK), iS);
-                mma_commit(&bars[bS + b]);
-                if (n >= 1) {
-                    ok = mbar_wait(&bars[bP + (b ^ 1)], ((n - 1) >> 1) & 1, abort_flag);
+                    for (int k = 1; k < kKeys / 16; ++k)
+                        mma_ts_lh<true>(tbuf + colO, tbuf + colS + k * 8, lV + k * (2048 >> 4), desc_hi(dK), iO);
+                    mma_commit(&bars[bO + (n & 1)]);
+                    mma_commit(&bars[bEmpty + n % kStages]);     // K, V (and Q) of this stage are dead
+                };
+                for (int n = 0; n < ntiles && ok; ++n) {
+                    const int s = n % kStages, b = n & 1;
+                    ok = mbar_wait(&bars[bFull + s], (n / kStages) & 1, abort_flag);
+                    // the buffer's previous tile (n - 2) must have been read out
+                    if (ok && n >= 2) ok = mbar_wait(&bars[bOfree + b], ((n >> 1) - 1) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(n - 1);
+                    const uint32_t tbuf = tb + b * kBufCols;
+                    const uint32_t lQ = desc_lo(dK) + (smem_u32(smem + s * kStageBytes) >> 4);
+                    const uint32_t lK = lQ + (kQBytes >> 4);
+                    mma_ss_lh<false>(tbuf + colS, lQ, desc_hi(dK), lK, desc_hi(dK), iS);
+#pragma unroll
+                    for (int k = 1; k < kHD / 16; ++k)
+                        mma_ss_lh<true>(tbuf + colS, lQ + k * 2, desc_hi(dK), lK + k * 2, desc_hi(dK), iS);
+                    mma_commit(&bars[bS + b]);
+                    if (n >= 1) {
+                        ok = mbar_wait(&bars[bP + (b ^ 1)], ((n - 1) >> 1) & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(n - 1);
+                    }
                 }
-            }
-            if (ok && ntiles >= 1) {
-                const int n = ntiles - 1;
-                ok = mbar_wait(&bars[bP + (n & 1)], (n >> 1) & 1, abort_flag);
-                if (ok) {
+                if (ok && ntiles >= 1) {
+                    const int n = ntiles - 1;
+                    ok = mbar_wait(&bars[bP + (n & 1)], (n >> 1) & 1, abort_flag);
+                    if (ok) {
+                        tc_fence_after();
+                        issue_pv(n);
+                    }
+                }
+            } else {
+                // tile n: its own rows in slot (n + 1) % 4, the 128 rows before them in slot n % 4
+                constexpr uint32_t iS128 = make_idesc_bf16(kQT, 128, 0, 0);
+                auto slot_lo = [&](int m, uint32_t off) -> uint32_t {
+                    return desc_lo(dK) + (smem_u32(smem + (m % kStages) * kStageBytes + off) >> 4);
+                };
+                auto issue_pv = [&](int n) {
+                    const uint32_t tbuf = tb + (n & 1) * kBufCols;
+                    const uint32_t lV0 = slot_lo(n, kQBytes + kKVBytes), lV1 = slot_lo(n + 1, kQBytes + kKVBytes);
+                    // a head's first tile has no rows before it: their weights are zero, and the slot holds another
+                    // head's rows, so those products are left out
+                    const bool head_start = tile_of(n) % p.tiles_per_head == 0;
+                    if (!head_start) {
+                        mma_ts_lh<false>(tbuf + colO, tbuf + colS, lV0, desc_hi(dK), iO);
+#pragma unroll
+                        for (int k = 1; k < 8; ++k)
+                            mma_ts_lh<true>(tbuf + colO, tbuf + colS + k * 8, lV0 + k * (2048 >> 4), desc_hi(dK), iO);
+                        mma_ts_lh<true>(tbuf + colO, tbuf + colS + 64, lV1, desc_hi(dK), iO);
+                    } else {
+                        mma_ts_lh<false>(tbuf + colO, tbuf + colS + 64, lV1, desc_hi(dK), iO);
+                    }
+#pragma unroll
+                    for (int k = 1; k < 8; ++k)
+                        mma_ts_lh<true>(tbuf + colO, tbuf + colS + 64 + k * 8, lV1 + k * (2048 >> 4), desc_hi(dK), iO);
+                    mma_commit(&bars[bO + (n & 1)]);
+                    mma_commit(&bars[bEmpty + n % kStages]);     // the rows before tile n are dead now
+                };
+                if (ntiles > 0) ok = mbar_wait(&bars[bFull + 0], 0, abort_flag);       // rows before the first tile
+                for (int n = 0; n < ntiles && ok; ++n) {
+                    const int m = n + 1, b = n & 1;
+                    ok = mbar_wait(&bars[bFull + m % kStages], (m / kStages) & 1, abort_flag);
+                    if (ok && n >= 2) ok = mbar_wait(&bars[bOfree + b], ((n >> 1) - 1) & 1, abort_flag);
+                    if (!ok) break;
                     tc_fence_after();
-                    issue_pv(n);
+                    const uint32_t tbuf = tb + b * kBufCols;
+                    const uint32_t lQ = slot_lo(m, 0), lK0 = slot_lo(n, kQBytes), lK1 = slot_lo(m, kQBytes);
+                    mma_ss_lh<false>(tbuf + colS, lQ, desc_hi(dK), lK0, desc_hi(dK), iS128);
+                    mma_ss_lh<false>(tbuf + colS + 128, lQ, desc_hi(dK), lK1, desc_hi(dK), iS128);
+#pragma unroll
+                    for (int k = 1; k < kHD / 16; ++k) {
+                        mma_ss_lh<true>(tbuf + colS, lQ + k * 2, desc_hi(dK), lK0 + k * 2, desc_hi(dK), iS128);
+                        mma_ss_lh<true>(tbuf + colS + 128, lQ + k * 2, desc_hi(dK), lK1 + k * 2, desc_hi(dK), iS128);
+                    }
+                    mma_commit(&bars[bS + b]);
+                    if (n >= 1) {
+                        ok = mbar_wait(&bars[bP + (b ^ 1)], ((n - 1) >> 1) & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(n - 1);
+                    }
+                }
+                if (ok && ntiles >= 1) {
+                    const int n = ntiles - 1;
+                    ok = mbar_wait(&bars[bP + (n & 1)], (n >> 1) & 1, abort_flag);
+                    if (ok) {
+                        tc_fence_after();
+                        issue_pv(n);
+                    }
                 }
             }
         }
@@ -198,7 +289,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const uint32_t tbuf = tb + g * kBufCols;
         for (int n = g; n < ntiles && ok; n += 2) {
             const uint32_t ph = (n >> 1) & 1;
-            const int tile = blockIdx.x + n * gridDim.x;
+            const int tile = tile_of(n);
             const int head = tile / p.tiles_per_head, i0 = (tile % p.tiles_per_head) * kQT;
             // visible columns of this row inside its warp's batch of PAD + 32 columns: keys i-w+1 .. i, and key >= 0
             const int jhi = lane + kPad;
@@ -391,7 +482,8 @@ static based_status launch_swa_pad(const void* q, const void* k, const void* v, 
                                    float scale, cudaStream_t stream) {
     using C = SwaCfg<PAD>;
     CUtensorMap tq, tk, tv, to;
-    if (!make_map(&tq, q, BH, L, kQT) || !make_map(&tk, k, BH, L, C::kKeys) || !make_map(&tv, v, BH, L, C::kKeys) ||
+    constexpr int kv_rows = PAD == 64 ? C::kKeys : kQT;      // rows of one K / V load
+    if (!make_map(&tq, q, BH, L, kQT) || !make_map(&tk, k, BH, L, kv_rows) || !make_map(&tv, v, BH, L, kv_rows) ||
         !make_map(&to, out, BH, L, kQT))
         return BASED_ERR_CUDA;
     SwaParams p;
