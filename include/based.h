@@ -183,7 +183,8 @@ based_status swa_decode_step(const void* q, const void* k, const void* v, void* 
  * cancels almost completely for short prefixes and a rounded out would dominate the result).
  * flags: 0, or BASED_NUMERATOR_ONLY for the backward of the numerator-only forward.
  * workspace: at least based_prefill_backward_workspace_bytes(B, H, L, d_v, io) bytes of device scratch.
- * Supported: d_feat = 16; d_v in {64, 112, 128}; io in {F32, BF16}; B*H <= 65535.
+ * Supported: d_feat = 16 with io in {F32, BF16}, d_feat in {8, 24, 32} with BF16 io (w = 1 + s/sqrt(d') +
+ * s^2/(2 d'), so ds_ij = (a_i . v_j + b_i)(1/sqrt(d') + q_i.k_j / d')); d_v in {64, 112, 128}; B*H <= 65535.
  * Both paths evaluate the quadratic form, O(L^2) per head, on 128 x 128 (bf16 io: tcgen05 tensor
  * cores, bf16 operands, fp32 accumulation) or 64 x 64 (fp32 io: fp32 FMAs) tiles of (query, key)
  * pairs.  Gradient outputs must not alias inputs.

@@ -276,7 +276,8 @@ static based_status prefill_backward(const void* q, const void* k, const void* v
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
     if (flags & ~BASED_NUMERATOR_ONLY) return BASED_ERR_INVALID_ARG;
     if (dq == q || dq == k || dk == q || dk == k || dv == v || dv == dout) return BASED_ERR_INVALID_ARG;
-    if (d_feat != kDFeat || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
+    // the other feature dimensions: bf16 io only (the tensor-core kernels take d' as a parameter)
+    if (!(d_feat == kDFeat || (df_generic(d_feat) && io == BASED_BF16)) || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
     if ((long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) || !aligned16(dk) ||
         !aligned16(dv) || !aligned16(workspace) || !aligned16(out))
@@ -285,7 +286,7 @@ static based_status prefill_backward(const void* q, const void* k, const void* v
         return BASED_ERR_WORKSPACE;
     if (io == BASED_BF16)
         return launch_prefill_backward_tc(q, k, v, out, dout, dq, dk, dv, static_cast<float*>(workspace), B * H, L,
-                                          d_v, (flags & BASED_NUMERATOR_ONLY) ? 1 : 0,
+                                          d_feat, d_v, (flags & BASED_NUMERATOR_ONLY) ? 1 : 0,
                                           static_cast<cudaStream_t>(cuda_stream));
     return launch_prefill_backward(q, k, v, dout, dq, dk, dv, static_cast<float*>(workspace), B * H, L, d_v, io,
                                    (flags & BASED_NUMERATOR_ONLY) ? 1 : 0, static_cast<cudaStream_t>(cuda_stream));

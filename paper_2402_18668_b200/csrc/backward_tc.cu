@@ -25,7 +25,9 @@
 // operands of the scores and as MN-major B operands of dQ / dK.  The work is O(L^2) per head, as
 // in the fp32 path.  A fourth mode of the same kernel evaluates the forward pass in this form
 // (scores, weights as bf16 in tensor memory, Y += P V, row sums): the tensor-core path of the
-// feature dimensions 8, 24 and 32, which the chunked d' = 16 kernel does not cover.
+// feature dimensions 8, 24 and 32, which the chunked d' = 16 kernel does not cover.  All modes take
+// d' (8, 16, 24, 32) as a parameter: the polynomial's coefficients 1/sqrt(d'), 1/(2 d'), a second K
+// step of the scores above 16, and up to 32 gradient columns of dq and dk.
 #include <math.h>
 
 #include <mutex>
@@ -85,8 +87,8 @@ struct BParams {
     __nv_bfloat16* dvo;          // [BH, L, dvw]
     unsigned int* err;
     int L, dvw, numerator_only;  // dvw: value head dimension of the caller's tensors (64, 112, 128)
-    int kdim;                    // forward mode: feature dimension rounded up to 16 (K extent of the scores)
-    float s1, s2;                // forward mode: w = 1 + s * s1 + s^2 * s2 (1 / sqrt d', 1 / (2 d'))
+    int df, kdim;                // feature dimension d', and d' rounded up to 16 (K extent of the scores)
+    float s1, s2;                // w = 1 + s * s1 + s^2 * s2 (1 / sqrt d', 1 / (2 d'))
 };
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -108,8 +110,9 @@ __device__ __forceinline__ bool rows_all(bool pred) {
         : "memory");
     return r != 0;
 }
-__device__ __forceinline__ float tw(float s) { return fmaf(s, fmaf(s, 0.03125f, 0.25f), 1.0f); }
-__device__ __forceinline__ float tdw(float s) { return fmaf(s, 0.0625f, 0.25f); }
+// w = 1 + s / sqrt(d') + s^2 / (2 d') and its derivative, s1 = 1 / sqrt(d'), s2 = 1 / (2 d') (d' = 16: 1/4, 1/32)
+__device__ __forceinline__ float tw(float s, float s1, float s2) { return fmaf(s, fmaf(s, s2, s1), 1.0f); }
+__device__ __forceinline__ float tdw(float s, float s1, float s2) { return fmaf(s, 2.0f * s2, s1); }
 }  // namespace
 
 // tm_n0 / tm_w0: narrow (q or k) and wide (a/g or v) tensor of the CTA's own (resident) tile;
@@ -190,7 +193,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                 // scores: rows = own tile, columns = looped tile
                 mma_ss_lh<false>(tb + C::colS, desc_lo(dN) + (aResN >> 4), desc_hi(dN), desc_lo(dN) + (aN >> 4),
                                  desc_hi(dN), iS);
-                if (MODE == kModeFwd && p.kdim > 16)         // feature dimensions 24 and 32: second K-step
+                if (p.kdim > 16)                             // feature dimensions 24 and 32: second K-step
                     mma_ss_lh<true>(tb + C::colS, desc_lo(dN) + (aResN >> 4) + 2, desc_hi(dN), desc_lo(dN) + (aN >> 4) + 2,
                                     desc_hi(dN), iS);
                 // own wide tile x looped wide tile^T over d_v
@@ -332,7 +335,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                         const float s = __uint_as_float(sr[i]), gvv = MODE == kModeFwd ? 0.f : __uint_as_float(gr[i]);
                         // pair (query, key): own row is the query except in the dk/dv pass
                         const bool live = !MASKED || (MODE == kModeDkDv ? (row <= col && col < p.L) : (col <= row));
-                        float w = live ? (MODE == kModeFwd ? fmaf(s, fmaf(s, p.s2, p.s1), 1.0f) : tw(s)) : 0.f;
+                        float w = live ? tw(s, p.s1, p.s2) : 0.f;
                         float ds = 0.f;
                         if (MODE == kModeFwd) {
                             den += w;
@@ -342,11 +345,11 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                         } else if (MODE == kModeDqS) {
                             den += w;
                             en = fmaf(w, gvv, en);
-                            w = live ? tdw(s) : 0.f;         // second tile: w'
+                            w = live ? tdw(s, p.s1, p.s2) : 0.f;         // second tile: w'
                             ds = w * (gvv - m_own);          // first tile: w' (gv - m)
                         } else {
                             const float2 stq = MODE == kModeDq ? st_own : s_b[(it & 1) * LT + blk * 32 + i];
-                            ds = live ? fmaf(gvv, stq.x, stq.y) * tdw(s) : 0.f;
+                            ds = live ? fmaf(gvv, stq.x, stq.y) * tdw(s, p.s1, p.s2) : 0.f;
                             w *= stq.x;                      // dv_j = sum_i (w_ij / D_i) G_i
                         }
                         sr[i] = __float_as_uint(w);
@@ -391,40 +394,42 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                 // dq_i = X_i / D_i + (m_i / D_i + b_i) Y_i
                 const float cy = fmaf(m_own, dinv, bq);
                 uint32_t rx[16], ry[16];
-                tmem_ld16(tmem_addr(tb, lane_base, C::colAcc), rx);
-                tmem_ld16(tmem_addr(tb, lane_base, C::colAcc2), ry);
-                tmem_wait_ld();
-                if (store) {
-                    uint32_t o[8];
+                for (int h = 0; h < (p.df + 15) / 16; ++h) {     // p.df is uniform: 8, 16, 24, 32 gradient columns
+                    tmem_ld16(tmem_addr(tb, lane_base, C::colAcc + h * 16), rx);
+                    tmem_ld16(tmem_addr(tb, lane_base, C::colAcc2 + h * 16), ry);
+                    tmem_wait_ld();
+                    if (store) {
+                        uint32_t o[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        o[i] = pack_bf16x2(fmaf(__uint_as_float(rx[2 * i]), dinv, cy * __uint_as_float(ry[2 * i])),
-                                           fmaf(__uint_as_float(rx[2 * i + 1]), dinv, cy * __uint_as_float(ry[2 * i + 1])));
-                    uint4* dst = reinterpret_cast<uint4*>(p.dq + grow * kDFeat);
-                    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                        for (int i = 0; i < 8; ++i)
+                            o[i] = pack_bf16x2(fmaf(__uint_as_float(rx[2 * i]), dinv, cy * __uint_as_float(ry[2 * i])),
+                                               fmaf(__uint_as_float(rx[2 * i + 1]), dinv, cy * __uint_as_float(ry[2 * i + 1])));
+                        uint4* dst = reinterpret_cast<uint4*>(p.dq + grow * p.df + h * 16);
+                        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                        if (h * 16 + 8 < p.df) dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                    }
                 }
             }
         } else if (ok) {                                     // ok is uniform over the row threads (rows_all)
-            // 16 gradient columns of dq (colAcc) or dk (colK)
-            uint32_t r[16];
-            if (MODE != kModeFwd) {
-                tmem_ld16(tmem_addr(tb, lane_base, MODE == kModeDq ? C::colAcc : C::colK), r);
+            // the d' gradient columns of dq (colAcc) or dk (colK), 16 at a time (p.df is uniform)
+            for (int h = 0; h < (MODE == kModeFwd ? 0 : (p.df + 15) / 16); ++h) {
+                uint32_t r[16];
+                tmem_ld16(tmem_addr(tb, lane_base, (MODE == kModeDq ? C::colAcc : C::colK) + h * 16), r);
                 tmem_wait_ld();
-            }
-            if (store && MODE != kModeFwd) {
-                uint4 o0, o1;
-                o0.x = pack_bf16x2(__uint_as_float(r[0]), __uint_as_float(r[1]));
-                o0.y = pack_bf16x2(__uint_as_float(r[2]), __uint_as_float(r[3]));
-                o0.z = pack_bf16x2(__uint_as_float(r[4]), __uint_as_float(r[5]));
-                o0.w = pack_bf16x2(__uint_as_float(r[6]), __uint_as_float(r[7]));
-                o1.x = pack_bf16x2(__uint_as_float(r[8]), __uint_as_float(r[9]));
-                o1.y = pack_bf16x2(__uint_as_float(r[10]), __uint_as_float(r[11]));
-                o1.z = pack_bf16x2(__uint_as_float(r[12]), __uint_as_float(r[13]));
-                o1.w = pack_bf16x2(__uint_as_float(r[14]), __uint_as_float(r[15]));
-                uint4* dst = reinterpret_cast<uint4*>((MODE == kModeDq ? p.dq : p.dk) + grow * kDFeat);
-                dst[0] = o0;
-                dst[1] = o1;
+                if (store) {
+                    uint4 o0, o1;
+                    o0.x = pack_bf16x2(__uint_as_float(r[0]), __uint_as_float(r[1]));
+                    o0.y = pack_bf16x2(__uint_as_float(r[2]), __uint_as_float(r[3]));
+                    o0.z = pack_bf16x2(__uint_as_float(r[4]), __uint_as_float(r[5]));
+                    o0.w = pack_bf16x2(__uint_as_float(r[6]), __uint_as_float(r[7]));
+                    o1.x = pack_bf16x2(__uint_as_float(r[8]), __uint_as_float(r[9]));
+                    o1.y = pack_bf16x2(__uint_as_float(r[10]), __uint_as_float(r[11]));
+                    o1.z = pack_bf16x2(__uint_as_float(r[12]), __uint_as_float(r[13]));
+                    o1.w = pack_bf16x2(__uint_as_float(r[14]), __uint_as_float(r[15]));
+                    uint4* dst = reinterpret_cast<uint4*>((MODE == kModeDq ? p.dq : p.dk) + grow * p.df + h * 16);
+                    dst[0] = o0;
+                    if (h * 16 + 8 < p.df) dst[1] = o1;
+                }
             }
             if (MODE == kModeDkDv || MODE == kModeFwd) {
                 // the wide accumulator row: dv, or the forward output scaled by 1 / (denominator + eps)
@@ -522,16 +527,16 @@ based_status launch_pass(const CUtensorMap& n0, const CUtensorMap& w0, const CUt
 
 template <int DV>
 based_status launch_dvb(const void* q, const void* k, const void* v, const void* out, const void* g, void* dq, void* dk,
-                        void* dv, float* ws, int BH, int L, int dvr, int numerator_only, cudaStream_t stream) {
+                        void* dv, float* ws, int BH, int L, int df, int dvr, int numerator_only, cudaStream_t stream) {
     constexpr int LTK = (DV == 64) ? 64 : 128;       // looped tile of the dk/dv pass (d_v 128 needs all 512 columns anyway)
     float2* stats = reinterpret_cast<float2*>(ws);
     // own tiles: 128 rows; looped tiles: 64 rows (and LTK rows for the dk/dv pass)
     CUtensorMap tq, tk, tv, tg, tk64, tv64, tqL, tgL;
     const CUtensorMapSwizzle s64 = CU_TENSOR_MAP_SWIZZLE_64B, s128 = CU_TENSOR_MAP_SWIZZLE_128B;
-    if (!make_map_b(&tq, q, BH, L, kDFeat, 32, kTile, s64) || !make_map_b(&tk, k, BH, L, kDFeat, 32, kTile, s64) ||
+    if (!make_map_b(&tq, q, BH, L, df, 32, kTile, s64) || !make_map_b(&tk, k, BH, L, df, 32, kTile, s64) ||
         !make_map_b(&tv, v, BH, L, dvr, 64, kTile, s128) || !make_map_b(&tg, g, BH, L, dvr, 64, kTile, s128) ||
-        !make_map_b(&tk64, k, BH, L, kDFeat, 32, 64, s64) || !make_map_b(&tv64, v, BH, L, dvr, 64, 64, s128) ||
-        !make_map_b(&tqL, q, BH, L, kDFeat, 32, LTK, s64) || !make_map_b(&tgL, g, BH, L, dvr, 64, LTK, s128))
+        !make_map_b(&tk64, k, BH, L, df, 32, 64, s64) || !make_map_b(&tv64, v, BH, L, dvr, 64, 64, s128) ||
+        !make_map_b(&tqL, q, BH, L, df, 32, LTK, s64) || !make_map_b(&tgL, g, BH, L, dvr, 64, LTK, s128))
         return BASED_ERR_CUDA;
     BParams p{};
     if (error_word_ptr(&p.err) != BASED_OK) return BASED_ERR_CUDA;
@@ -545,6 +550,10 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
     p.L = L;
     p.dvw = dvr;
     p.numerator_only = numerator_only;
+    p.df = df;
+    p.kdim = df <= 16 ? 16 : 32;
+    p.s1 = 1.0f / sqrtf((float)df);
+    p.s2 = 0.5f / (float)df;
     const dim3 grid((L + kTile - 1) / kTile, BH);
     based_status st;
     if (out != nullptr || numerator_only) {
@@ -579,6 +588,7 @@ based_status launch_quadratic_forward_tc(const void* q, const void* k, const voi
     p.L = L;
     p.dvw = d_v;
     p.numerator_only = numerator_only;
+    p.df = d_feat;
     p.kdim = d_feat <= 16 ? 16 : 32;
     p.s1 = 1.0f / sqrtf((float)d_feat);
     p.s2 = 0.5f / (float)d_feat;
@@ -593,10 +603,10 @@ size_t backward_tc_workspace_bytes(int BH, int L, int d_v) {
 }
 
 based_status launch_prefill_backward_tc(const void* q, const void* k, const void* v, const void* out, const void* g,
-                                        void* dq, void* dk, void* dv, float* ws, int BH, int L, int d_v,
+                                        void* dq, void* dk, void* dv, float* ws, int BH, int L, int d_feat, int d_v,
                                         int numerator_only, cudaStream_t stream) {
-    if (d_v == 64) return launch_dvb<64>(q, k, v, out, g, dq, dk, dv, ws, BH, L, 64, numerator_only, stream);
-    return launch_dvb<128>(q, k, v, out, g, dq, dk, dv, ws, BH, L, d_v, numerator_only, stream);  // 112 or 128
+    if (d_v == 64) return launch_dvb<64>(q, k, v, out, g, dq, dk, dv, ws, BH, L, d_feat, 64, numerator_only, stream);
+    return launch_dvb<128>(q, k, v, out, g, dq, dk, dv, ws, BH, L, d_feat, d_v, numerator_only, stream);  // 112 or 128
 }
 
 }  // namespace based

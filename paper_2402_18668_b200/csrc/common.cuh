@@ -112,7 +112,7 @@ based_status launch_decode_generic(const void* q, const void* k, const void* v, 
 size_t backward_tc_workspace_bytes(int BH, int L, int d_v);
 // out: the forward output (may be null): with it, statistics and dq run as one sweep
 based_status launch_prefill_backward_tc(const void* q, const void* k, const void* v, const void* out, const void* g,
-                                        void* dq, void* dk, void* dv, float* ws, int BH, int L, int d_v,
+                                        void* dq, void* dk, void* dv, float* ws, int BH, int L, int d_feat, int d_v,
                                         int numerator_only, cudaStream_t stream);
 // definition-form forward on tensor cores for d' in {8, 24, 32} (bf16 io, empty initial state)
 based_status launch_quadratic_forward_tc(const void* q, const void* k, const void* v, void* out, int BH, int L,

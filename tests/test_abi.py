@@ -141,6 +141,8 @@ def test_backward_validation(lib):
     assert f(q, k, v, g, dq, dk, dv, *ok, 1, ws, 1 << 20, None) == 1               # CONTINUE is not a backward flag
     assert f(q, k, v, g, q, dk, dv, *ok, 0, ws, 1 << 20, None) == 1                # gradient aliases an input
     assert f(q, k, v, g, dq, dk, dv, 1, 1, 8, 16, 96, 1, 0, ws, 1 << 20, None) == 2
+    assert f(q, k, v, g, dq, dk, dv, 1, 1, 8, 12, 64, 1, 0, ws, 1 << 20, None) == 2   # d' in {8, 16, 24, 32}
+    assert f(q, k, v, g, dq, dk, dv, 1, 1, 8, 24, 64, 0, 0, ws, 1 << 20, None) == 2   # other d': bf16 io only
     assert f(q, k, v, g, dq, dk, dv, *ok, 0, ws, 8, None) == 6                     # workspace too small
     assert f(q, k, v, g, dq, dk, dv, *ok, 0, None, 0, None) == 6
     w = lib.based_prefill_backward_with_out

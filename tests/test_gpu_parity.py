@@ -255,6 +255,24 @@ def test_prefill_backward_with_forward_output(dtype, L, d_v, flags):
     assert _grad_err(_np(dq), rq) <= tol and _grad_err(_np(dk), rk) <= tol and _grad_err(_np(dv), rv) <= tol
 
 
+@pytest.mark.parametrize("with_out", [False, True])
+@pytest.mark.parametrize("d_feat,L,d_v", [(8, 200, 64), (24, 333, 128), (32, 130, 112), (32, 1, 64), (24, 700, 64)])
+def test_prefill_backward_other_feature_dimensions(d_feat, L, d_v, with_out):
+    """Backward for d' in {8, 24, 32} (bf16 io, tensor-core path with d' as a parameter) against the oracle."""
+    B, H = 2, 2
+    w = wl.Workload("bwdf", B, H, L, d_feat, d_v, "bf16", 0.5)
+    q, k, v = wl.prefill_inputs(w, wl.generator(7000 + d_feat + L))
+    g = torch.randn(B, H, L, d_v, generator=wl.generator(7001 + L)).to(v.dtype)
+    rq, rk, rv = oracle.linattn_backward(_np(q), _np(k), _np(v), _np(g))
+    qd, kd, vd, gd = q.to(DEV), k.to(DEV), v.to(DEV), g.to(DEV)
+    out = based.based_prefill(qd, kd, vd) if with_out else None
+    dq, dk, dv = based.based_prefill_backward(qd, kd, vd, gd, out=out)
+    _poll()
+    assert dq.shape == q.shape and dk.shape == k.shape
+    assert _grad_err(_np(dq), rq) <= TOL_BF16 and _grad_err(_np(dk), rk) <= TOL_BF16
+    assert _grad_err(_np(dv), rv) <= TOL_BF16
+
+
 def test_prefill_backward_with_forward_output_cfg2_sampled_heads():
     """360M-layer shape, bf16: the merged statistics + dq pass on sampled heads against the oracle, and its dq
     against the separate passes' dq (both within tolerance of the truth, so within twice that of each other)."""
