@@ -467,7 +467,7 @@ def bench_generation_graph(w, steps, warmup, torch, based, dist_on, peaks):
         "workload": f"B{w.B} H{w.H}: decode step on the 153-row state (d_v {w.d_v}) + window-{win} decode step, "
                     "one CUDA graph per token",
         "metric": "generation_tokens_per_s", "value": w.B / t, "unit": "tokens/s", "us_per_token_step": t * 1e6,
-        "steps": steps, "kernels_per_replay": 3,
+        "steps": steps, "kernels_per_replay": 2,
         "roofline": {"bound": "hbm", "achieved": bytes_step / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": bytes_step / t / 1e9 / peaks["hbm_gbs"], "traffic": None,
                      "algorithmic_bytes": bytes_step, "peak_source": peaks["source"]},

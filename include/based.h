@@ -254,6 +254,18 @@ based_status swa_decode_step_at(const void* q, const void* k, const void* v, voi
                                 float softmax_scale, based_dtype io, void* cuda_stream);
 
 /*
+ * The same step for a generation loop that is replayed as a CUDA graph: pos_state points to two
+ * ints in device memory, {position, ticket} (ticket 0 before the first call).  The step reads the
+ * position like swa_decode_step_at and stores position + 1 when it ends, so the loop needs no
+ * separate kernel to advance the counter: every CTA takes a ticket at its end, and the one that
+ * takes the last ticket, at which point all have read the position, resets the ticket and writes
+ * the new position.  pos_state must be 8-byte aligned and is owned by the caller.
+ */
+based_status swa_decode_step_advance(const void* q, const void* k, const void* v, void* k_cache, void* v_cache,
+                                     void* out, int B, int H, int d, int window, int* pos_state,
+                                     float softmax_scale, based_dtype io, void* cuda_stream);
+
+/*
  * The same computation as based_prefill, for callers that cannot give the library scratch
  * memory.  (The paper has no counterpart: this is a deployment convenience.)  Some hosts
  * may not allocate device memory around a call at all - a serving process that has handed

@@ -28,7 +28,7 @@ EXPORTS = (
     "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step", "based_decode_step_sym",
     "based_state_to_sym", "based_state_from_sym", "swa_decode_step_at", "based_preload_decode",
     "baseconv_gate_forward", "baseconv_gate_step", "based_decode_step_flags", "based_prefill_backward",
-    "based_prefill_backward_workspace_bytes", "based_prefill_backward_with_out",
+    "based_prefill_backward_workspace_bytes", "based_prefill_backward_with_out", "swa_decode_step_advance",
 )
 
 _lib = None
@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.swa_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
         L.swa_decode_step_at.restype = i
         L.swa_decode_step_at.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, i, vp]
+        L.swa_decode_step_advance.restype = i
+        L.swa_decode_step_advance.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, i, vp]
         L.based_preload_decode.restype = i
         L.based_prefill_backward.restype = i
         L.based_prefill_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]

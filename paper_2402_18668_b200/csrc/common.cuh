@@ -86,9 +86,10 @@ based_status launch_prefill_tc(const void* q, const void* k, const void* v, void
 bool swa_tc_supported(int window);
 based_status launch_swa_tc(const void* q, const void* k, const void* v, void* out, int BH, int L, int window,
                            float scale, cudaStream_t stream);
-// pos_dev != nullptr: the position is read from device memory by the kernel (pos is ignored)
+// pos_dev != nullptr: the position is read from device memory by the kernel (pos is ignored);
+// pos_adv != nullptr ({position, ticket}, pos_dev == pos_adv): the kernel also stores position + 1 at its end
 based_status launch_swa_decode(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
-                               int window, int pos, const int* pos_dev, float scale, based_dtype io,
+                               int window, int pos, const int* pos_dev, int* pos_adv, float scale, based_dtype io,
                                cudaStream_t stream);
 // gated short convolution (BaseConv core); step: one token on a [B, width-1, C] state, N ignored
 based_status launch_baseconv(const void* a, const void* g, const float* h, const float* b2, void* state, void* out,

@@ -80,7 +80,8 @@ template <typename T, int NPW>     // NPW >= ceil(window / (4 * kWarps)): passes
 __global__ void __launch_bounds__(32 * kWarps)
 swa_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, T* __restrict__ kc,
                   T* __restrict__ vc, T* __restrict__ out, int window, int pos_arg,
-                  const int* __restrict__ pos_dev, float scale, unsigned int* __restrict__ error_word) {
+                  const int* __restrict__ pos_dev, int* __restrict__ pos_adv, float scale,
+                  unsigned int* __restrict__ error_word) {
     // the position comes from device memory when the launch is part of a captured graph that is
     // replayed as the sequence grows
     const int pos = pos_dev ? *pos_dev : pos_arg;
@@ -208,11 +209,20 @@ swa_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
         }
         out[head * kHD + tid] = from_f32<T>(num / den);
     }
+    // advance mode: pos_adv = {position, ticket}.  Every CTA read the position at its start and takes a
+    // ticket at its end, so the CTA that takes the last one knows that all of them have read it: it
+    // resets the ticket and stores position + 1 for the next launch
+    if (pos_adv != nullptr && tid == 0) {
+        if (atomicAdd(pos_adv + 1, 1) == (int)gridDim.x - 1) {
+            pos_adv[1] = 0;
+            pos_adv[0] = pos + 1;
+        }
+    }
 }
 
 template <typename T, int NPW>
 static based_status launch_n(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
-                             int window, int pos, const int* pos_dev, float scale, unsigned int* err,
+                             int window, int pos, const int* pos_dev, int* pos_adv, float scale, unsigned int* err,
                              cudaStream_t stream) {
     const size_t smem = swa_decode_smem_bytes<T>(window);
     if (smem > 48 * 1024) {
@@ -223,17 +233,17 @@ static based_status launch_n(const void* q, const void* k, const void* v, void* 
     swa_decode_kernel<T, NPW><<<BH, 32 * kWarps, smem, stream>>>(static_cast<const T*>(q), static_cast<const T*>(k),
                                                           static_cast<const T*>(v), static_cast<T*>(kc),
                                                           static_cast<T*>(vc), static_cast<T*>(out), window, pos,
-                                                          pos_dev, scale, err);
+                                                          pos_dev, pos_adv, scale, err);
     note_launch();
     return check_launch("swa_decode_kernel");
 }
 
 template <typename T>
 static based_status launch_t(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
-                             int window, int pos, const int* pos_dev, float scale, unsigned int* err,
+                             int window, int pos, const int* pos_dev, int* pos_adv, float scale, unsigned int* err,
                              cudaStream_t stream) {
-    if (window <= 64) return launch_n<T, 4>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, scale, err, stream);
-    return launch_n<T, 8>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, scale, err, stream);
+    if (window <= 64) return launch_n<T, 4>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream);
+    return launch_n<T, 8>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream);
 }
 
 based_status preload_swa_decode() {
@@ -246,13 +256,14 @@ based_status preload_swa_decode() {
 }
 
 based_status launch_swa_decode(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
-                               int window, int pos, const int* pos_dev, float scale, based_dtype io,
+                               int window, int pos, const int* pos_dev, int* pos_adv, float scale, based_dtype io,
                                cudaStream_t stream) {
     unsigned int* err = nullptr;
     const based_status st = error_word_ptr(&err);
     if (st != BASED_OK) return st;
-    if (io == BASED_F32) return launch_t<float>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, scale, err, stream);
-    return launch_t<__nv_bfloat16>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, scale, err, stream);
+    if (io == BASED_F32)
+        return launch_t<float>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream);
+    return launch_t<__nv_bfloat16>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream);
 }
 
 }  // namespace based

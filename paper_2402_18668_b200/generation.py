@@ -4,8 +4,8 @@ The paper runs next-token prediction under CUDA graphs (Sec. 6, "Efficiency Benc
 batch sizes where a decode step lasts tens of microseconds the launch overhead of separate
 calls is a visible share of it.  `DecodeGraph` captures one step of both mixers, the Taylor
 linear-attention decode step (on the 273-row or the 153-row symmetric state) and the
-sliding-window decode step on its rolling cache, together with the increment of the position
-counter the latter reads from device memory, and replays it once per generated token.
+sliding-window decode step on its rolling cache, which reads the position from device memory and
+advances it itself (swa_decode_step_advance), and replays it once per generated token.
 
 Only plumbing lives here (static buffers, stream capture); every arithmetic step runs in the
 library's kernels.
@@ -42,14 +42,14 @@ class DecodeGraph:
         self.vw = torch.zeros_like(self.qw)
         self.out_lin = torch.empty_like(self.v)
         self.out_swa = torch.empty_like(self.qw)
-        self.pos = torch.full((1,), int(pos), dtype=torch.int32, device=dev)
+        self._pos_state = torch.tensor([int(pos), 0], dtype=torch.int32, device=dev)    # {position, ticket}
+        self.pos = self._pos_state[:1]
         self._scale, self._window, self._d = float(softmax_scale), window, d
         self._stream = torch.cuda.Stream(device=dev)
         self._graph = torch.cuda.CUDAGraph()
         # an eager warm-up pass would advance the state, so the kernels are loaded explicitly and
         # the step is captured directly (the library allocates nothing: the calls only enqueue kernels)
         _b._check(_b.lib().based_preload_decode(), "based_preload_decode")
-        self.pos.add_(0)                                   # loads torch's add kernel outside the capture
         self._stream.wait_stream(torch.cuda.current_stream(dev))
         with torch.cuda.stream(self._stream):
             with torch.cuda.graph(self._graph, stream=self._stream):
@@ -60,12 +60,11 @@ class DecodeGraph:
         dec = _b.based_decode_step_sym if self.sym else _b.based_decode_step
         dec(self.q, self.k, self.v, self.kv, self.z, out=self.out_lin)
         B, H, d = self.qw.shape
-        st = _b.lib().swa_decode_step_at(_b._ptr(self.qw), _b._ptr(self.kw), _b._ptr(self.vw), _b._ptr(self.kc),
-                                         _b._ptr(self.vc), _b._ptr(self.out_swa), B, H, d, self._window,
-                                         ctypes.c_void_p(self.pos.data_ptr()), self._scale,
-                                         _b._dtype_code(self.qw), _b._stream())
-        _b._check(st, "swa_decode_step_at")
-        self.pos.add_(1)
+        st = _b.lib().swa_decode_step_advance(_b._ptr(self.qw), _b._ptr(self.kw), _b._ptr(self.vw), _b._ptr(self.kc),
+                                              _b._ptr(self.vc), _b._ptr(self.out_swa), B, H, d, self._window,
+                                              ctypes.c_void_p(self._pos_state.data_ptr()), self._scale,
+                                              _b._dtype_code(self.qw), _b._stream())
+        _b._check(st, "swa_decode_step_advance")
 
     def step(self, q, k, v, qw, kw, vw):
         """Copies the token's inputs into the graph's buffers, replays it; returns the two outputs

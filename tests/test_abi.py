@@ -117,6 +117,14 @@ def test_swa_decode_at_validation(lib):
     assert f(P, P, P, P, P, O, 1, 1, 48, 64, P, 0.0, 1, None) == 2
 
 
+def test_swa_decode_advance_validation(lib):
+    f = lib.swa_decode_step_advance
+    O = ctypes.c_void_p(0x2000)
+    assert f(P, P, P, P, P, O, 1, 1, 64, 64, None, 0.0, 1, None) == 1            # no position state
+    assert f(P, P, P, P, P, O, 1, 1, 64, 64, ctypes.c_void_p(0x3004), 0.0, 1, None) == 3   # two ints, 8-byte aligned
+    assert f(P, P, P, P, P, O, 1, 1, 64, 200, P, 0.0, 1, None) == 2
+
+
 def test_baseconv_validation(lib):
     f = lib.baseconv_gate_forward
     O = ctypes.c_void_p(0x2000)

@@ -469,6 +469,31 @@ def test_baseconv_gate_full_size_sampled():
 
 
 # --------------------------------------------------------------------------- graph-replayed generation step
+def test_swa_decode_advance_moves_the_position_itself():
+    """swa_decode_step_advance: the position in device memory grows by one per call (every CTA takes a ticket,
+    the last one writes position + 1), and the outputs equal those of the plain step at the same positions."""
+    B, H, d, window, T = 3, 50, 64, 64, 70
+    g_ = torch.Generator(device=DEV).manual_seed(5)
+    q, k, v = (torch.randn(B, H, T, d, generator=g_, device=DEV).bfloat16() for _ in range(3))
+    kc1 = torch.zeros(B, H, window, d, dtype=torch.bfloat16, device=DEV); vc1 = torch.zeros_like(kc1)
+    kc2 = torch.zeros_like(kc1); vc2 = torch.zeros_like(kc1)
+    state = torch.tensor([0, 0], dtype=torch.int32, device=DEV)
+    out2 = torch.empty(B, H, d, dtype=torch.bfloat16, device=DEV)
+    import ctypes
+    from paper_2402_18668_b200 import binding as _b
+    for t in range(T):
+        args = (q[:, :, t].contiguous(), k[:, :, t].contiguous(), v[:, :, t].contiguous())
+        o1 = based.swa_decode_step(*args, kc1, vc1, t)
+        st = _b.lib().swa_decode_step_advance(_b._ptr(args[0]), _b._ptr(args[1]), _b._ptr(args[2]), _b._ptr(kc2), _b._ptr(vc2),
+                                              _b._ptr(out2), B, H, d, window, ctypes.c_void_p(state.data_ptr()), 0.0, 1,
+                                              _b._stream())
+        assert st == 0
+        assert torch.equal(o1, out2), f"token {t}"
+        assert state.tolist() == [t + 1, 0]
+    _poll()
+    assert torch.equal(kc1, kc2) and torch.equal(vc1, vc2)
+
+
 @pytest.mark.parametrize("sym", [False, True])
 def test_decode_graph_replays_match_oracle_chain(sym):
     """The mixer pair's generation step captured once and replayed T times (position advanced on the
