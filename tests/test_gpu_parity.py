@@ -861,3 +861,23 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     out = based.based_prefill(q, q.clone(), v)
     _poll()
     assert torch.isfinite(out.float()).all()
+
+
+# --------------------------------------------------------------------------- benchmark arms
+@pytest.mark.parametrize("args", [["--profile", "backward"], ["--profile", "prefill_dfeat", "--d-feat", "24"],
+                                  ["--profile", "swa", "--window", "128"], ["--profile", "generation_graph"]])
+def test_bench_profiles_print_one_json_line(args):
+    """The secondary benchmark arms run and report a roofline (short runs: the numbers are not checked)."""
+    import json
+    import subprocess
+    import sys
+    from pathlib import Path
+    root = Path(__file__).resolve().parent.parent
+    r = subprocess.run([sys.executable, str(root / "bench.py"), *args, "--steps", "3", "--warmup", "3"],
+                       capture_output=True, text=True, timeout=600, cwd=str(root))
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["profile"] == args[1] and d["value"] > 0 and 0 < d["roofline"]["frac"] < 1.5
+
