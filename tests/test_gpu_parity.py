@@ -863,6 +863,35 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     assert torch.isfinite(out.float()).all()
 
 
+# --------------------------------------------------------------------------- input scales
+@pytest.mark.parametrize("qk_scale,v_scale", [(0.0, 1.0), (1e-3, 1.0), (4.0, 1.0), (0.3, 1e4), (0.3, 1e-4)])
+def test_extreme_input_scales_bf16(qk_scale, v_scale):
+    """bf16 prefill, final state and backward against the oracle far from the benchmark's input scales:
+    vanishing q.k (weights all one: running means), large q.k (the quadratic term dominates), very large
+    and very small values."""
+    B, H, L, d_v = 1, 3, 300, 64
+    gen = wl.generator(int(qk_scale * 1000) + int(v_scale))
+    q = (torch.randn(B, H, L, 16, generator=gen) * qk_scale).bfloat16()
+    k = (torch.randn(B, H, L, 16, generator=gen) * qk_scale).bfloat16()
+    v = (torch.randn(B, H, L, d_v, generator=gen) * v_scale).bfloat16()
+    g = torch.randn(B, H, L, d_v, generator=gen).bfloat16()
+    y_ref, S_ref, z_ref = oracle.linattn_quadratic(_np(q), _np(k), _np(v))
+    rq, rk, rv = oracle.linattn_backward(_np(q), _np(k), _np(v), _np(g))
+    qd, kd, vd, gd = q.to(DEV), k.to(DEV), v.to(DEV), g.to(DEV)
+    kv, z = based.new_state(B, H, d_v)
+    out = based.based_prefill(qd, kd, vd, kv_state=kv, z_state=z)
+    dq, dk, dv = based.based_prefill_backward(qd, kd, vd, gd, out=out)
+    _poll()
+    assert row_err(_np(out), y_ref) <= TOL_BF16
+    assert head_err(_np(kv), S_ref) <= TOL_BF16 and head_err(_np(z), z_ref) <= TOL_BF16
+    # gradients: relative to each head's largest entry (no absolute floor: the scales span eight decades)
+    for got, want in ((dq, rq), (dk, rk), (dv, rv)):
+        got, want = _np(got).reshape(B * H, -1).astype(np.float64), np.asarray(want).reshape(B * H, -1)
+        scale = np.abs(want).max(axis=1)
+        err = np.abs(got - want).max(axis=1)
+        assert np.all(err <= TOL_BF16 * np.maximum(scale, 1e-30) + 1e-30), (err, scale)
+
+
 # --------------------------------------------------------------------------- benchmark arms
 @pytest.mark.parametrize("args", [["--profile", "backward"], ["--profile", "prefill_dfeat", "--d-feat", "24"],
                                   ["--profile", "swa", "--window", "128"], ["--profile", "generation_graph"]])
