@@ -85,6 +85,24 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
 size_t based_prefill_workspace_bytes(int B, int H, int L, int d_feat, int d_v, based_dtype io);
 
 /*
+ * The recurrent state of a token block without its outputs (Sec. 4.1, recurrent view):
+ *   kv_state (+)= sum_j phi(k_j) v_j^T,   z_state (+)= sum_j phi(k_j)
+ * exactly what based_prefill leaves in kv_state / z_state for the same k, v, flags, at about a
+ * third of its cost (no scores, no read-out).  k [B,H,L,d_feat], v [B,H,L,d_v] in the io dtype;
+ * the state layouts are based_prefill's.  flags: BASED_STATE_ZERO_INIT or BASED_STATE_CONTINUE,
+ * optionally BASED_STATE_SYM.  This is the first step of a prefill whose sequence is split across
+ * GPUs: every rank computes its block's state, the states are exchanged and summed over the
+ * earlier ranks, and based_prefill with BASED_STATE_CONTINUE produces the block's outputs.
+ * Supported: d_feat in {8, 16, 24, 32}, d_v in {64, 112, 128}, io in {F32, BF16}; BASED_STATE_SYM
+ * with d_feat = 16 and BF16 io only.  workspace: based_prefill_state_workspace_bytes (non-zero
+ * for d_feat = 16 with BF16 io: partial states of sequence segments).
+ */
+based_status based_prefill_state(const void* k, const void* v, float* kv_state, float* z_state, int B, int H, int L,
+                                 int d_feat, int d_v, based_dtype io, int flags, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream);
+size_t based_prefill_state_workspace_bytes(int B, int H, int L, int d_feat, int d_v, based_dtype io);
+
+/*
  * One recurrent step of the same mixer (Sec. 4.1 recurrences; App. B.2 step()
  * listing and Algorithm 2, here on raw q, k with the feature map applied on chip and
  * with the denominator): per (b, h), update then read,

@@ -29,6 +29,7 @@ EXPORTS = (
     "based_state_to_sym", "based_state_from_sym", "swa_decode_step_at", "based_preload_decode",
     "baseconv_gate_forward", "baseconv_gate_step", "based_decode_step_flags", "based_prefill_backward",
     "based_prefill_backward_workspace_bytes", "based_prefill_backward_with_out", "swa_decode_step_advance",
+    "based_prefill_state", "based_prefill_state_workspace_bytes",
 )
 
 _lib = None
@@ -54,6 +55,10 @@ def lib() -> ctypes.CDLL:
         L.based_prefill.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
         L.based_prefill_workspace_bytes.restype = sz
         L.based_prefill_workspace_bytes.argtypes = [i, i, i, i, i, i]
+        L.based_prefill_state.restype = i
+        L.based_prefill_state.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
+        L.based_prefill_state_workspace_bytes.restype = sz
+        L.based_prefill_state_workspace_bytes.argtypes = [i, i, i, i, i, i]
         L.based_prefill_static_scratch.restype = i
         L.based_prefill_static_scratch.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp]
         L.based_static_scratch_bytes.restype = sz
@@ -165,6 +170,26 @@ def based_prefill(q, k, v, out=None, kv_state=None, z_state=None, flags: int = B
                              d_v, io, flags, _ptr(workspace), ws_bytes, _stream(stream))
     _check(st, "based_prefill")
     return out
+
+
+def based_prefill_state(k, v, kv_state=None, z_state=None, flags: int = BASED_STATE_ZERO_INIT, workspace=None,
+                        stream=None):
+    """The state a prefill over k [B,H,L,d'], v [B,H,L,d_v] leaves (kv_state, z_state; added to the given
+    state with BASED_STATE_CONTINUE), without computing outputs.  Returns (kv_state, z_state)."""
+    _dev(k, v, kv_state, z_state, workspace)
+    B, H, L, d_feat = k.shape
+    d_v = v.shape[-1]
+    if kv_state is None:
+        kv_state, z_state = new_state(B, H, d_v, k.device, sym=bool(flags & BASED_STATE_SYM), d_feat=d_feat)
+    need = int(lib().based_prefill_state_workspace_bytes(B, H, L, d_feat, d_v, _dtype_code(k)))
+    if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
+        workspace = torch.empty(need, dtype=torch.uint8, device=k.device)
+    st = lib().based_prefill_state(_ptr(k), _ptr(v), _ptr(kv_state), _ptr(z_state), B, H, L, d_feat, d_v, _dtype_code(k),
+                                   int(flags), _ptr(workspace),
+                                   0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                   _stream(stream))
+    _check(st, "based_prefill_state")
+    return kv_state, z_state
 
 
 def based_prefill_backward(q, k, v, dout, flags: int = 0, workspace=None, stream=None, out=None):

@@ -117,6 +117,34 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
                                static_cast<cudaStream_t>(cuda_stream));
 }
 
+size_t based_prefill_state_workspace_bytes(int B, int H, int L, int d_feat, int d_v, based_dtype io) {
+    if (B <= 0 || H <= 0 || L <= 0 || d_feat != kDFeat || !dv_ok(d_v) || io != BASED_BF16) return 0;
+    if ((long long)B * H > 65535) return 0;
+    return prefill_tc_state_workspace_bytes(B * H, L, d_v);
+}
+
+based_status based_prefill_state(const void* k, const void* v, float* kv_state, float* z_state, int B, int H, int L,
+                                 int d_feat, int d_v, based_dtype io, int flags, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
+    if (!k || !v || !kv_state || !z_state || B <= 0 || H <= 0 || L <= 0) return BASED_ERR_INVALID_ARG;
+    if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
+    if (flags & ~(BASED_STATE_CONTINUE | BASED_STATE_SYM)) return BASED_ERR_INVALID_ARG;
+    if ((d_feat != kDFeat && !df_generic(d_feat)) || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
+    const bool tc16 = d_feat == kDFeat && io == BASED_BF16;
+    if ((flags & BASED_STATE_SYM) && !tc16) return BASED_ERR_UNSUPPORTED;      // symmetric rows: d' = 16, bf16 io
+    if (!aligned16(k) || !aligned16(v) || !aligned16(kv_state) || !aligned16(z_state) || !aligned16(workspace))
+        return BASED_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (tc16) {
+        if (!workspace || workspace_bytes < based_prefill_state_workspace_bytes(B, H, L, d_feat, d_v, io))
+            return BASED_ERR_WORKSPACE;
+        return launch_prefill_tc_state(k, v, kv_state, z_state, B * H, L, d_v, flags, workspace, stream);
+    }
+    return launch_state_generic(k, v, kv_state, z_state, B * H, L, d_feat, d_v, io,
+                                (flags & BASED_STATE_CONTINUE) ? 1 : 0, stream);
+}
+
 based_status based_decode_step(const void* q, const void* k, const void* v, float* kv_state, float* z_state,
                                void* out, int B, int H, int d_feat, int d_v, based_dtype io, void* cuda_stream) {
     if (!q || !k || !v || !out || !kv_state || !z_state || B <= 0 || H <= 0) return BASED_ERR_INVALID_ARG;

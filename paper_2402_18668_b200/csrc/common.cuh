@@ -106,6 +106,12 @@ based_status launch_prefill_generic(const void* q, const void* k, const void* v,
 // the final state of those feature dimensions on tensor cores (bf16 io); cont: add to the state given
 based_status launch_state_generic_tc(const void* k, const void* v, float* kv, float* z, int BH, int L, int d_feat,
                                      int d_v, int cont, cudaStream_t stream);
+// the state of a token block alone (no outputs): kv (+)= sum_j phi(k_j) v_j^T, z (+)= sum_j phi(k_j)
+based_status launch_state_generic(const void* k, const void* v, float* kv, float* z, int BH, int L, int d_feat, int d_v,
+                                  based_dtype io, int cont, cudaStream_t stream);
+size_t prefill_tc_state_workspace_bytes(int BH, int L, int d_v);
+based_status launch_prefill_tc_state(const void* k, const void* v, float* kv, float* z, int BH, int L, int d_v,
+                                     int flags, void* workspace, cudaStream_t stream);
 based_status launch_decode_generic(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
                                    int BH, int d_feat, int d_v, based_dtype io, bool numerator_only,
                                    cudaStream_t stream);

@@ -343,6 +343,26 @@ based_status launch_prefill_generic(const void* q, const void* k, const void* v,
     return prefill_t<__nv_bfloat16, 128>(q, k, v, out, kv, z, BH, L, d_feat, flags, outputs_done, stream);
 }
 
+// The state of a token block alone, any supported feature dimension (16 included): bf16 io on tensor cores,
+// fp32 io with fp32 FMAs.
+template <int DV>
+static based_status state_f32(const void* k, const void* v, float* kv, float* z, int BH, int L, int df, int cont,
+                              cudaStream_t stream) {
+    const int D = expanded_dim(df);
+    generic_state_kernel<float, DV><<<dim3((D + 31) / 32, BH), DV + 32, 0, stream>>>(
+        static_cast<const float*>(k), static_cast<const float*>(v), kv, z, L, df, cont);
+    note_launch();
+    return check_launch("generic_state_kernel");
+}
+
+based_status launch_state_generic(const void* k, const void* v, float* kv, float* z, int BH, int L, int d_feat, int d_v,
+                                  based_dtype io, int cont, cudaStream_t stream) {
+    if (io == BASED_BF16) return launch_state_generic_tc(k, v, kv, z, BH, L, d_feat, d_v, cont, stream);
+    if (d_v == 64) return state_f32<64>(k, v, kv, z, BH, L, d_feat, cont, stream);
+    if (d_v == 112) return state_f32<112>(k, v, kv, z, BH, L, d_feat, cont, stream);
+    return state_f32<128>(k, v, kv, z, BH, L, d_feat, cont, stream);
+}
+
 based_status launch_decode_generic(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
                                    int BH, int d_feat, int d_v, based_dtype io, bool numerator_only,
                                    cudaStream_t stream) {

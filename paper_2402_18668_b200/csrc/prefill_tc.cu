@@ -1075,6 +1075,97 @@ static SegPlan prefill_tc_plan(int BH, int L, int d_v) {
     return best;
 }
 
+// ---- the state of a token block without its outputs ---------------------------------------------
+// Segments of the state-update-only pass for a state-only call: up to eight per head, about one CTA per SM.
+static SegPlan prefill_tc_state_plan(int BH, int L) {
+    const int nch = (L + kC - 1) / kC;
+    int n = 148 / BH;
+    n = n < 1 ? 1 : (n > 8 ? 8 : n);
+    if (n > nch) n = nch;
+    const int per = (nch + n - 1) / n;
+    return {(nch + per - 1) / per, per, false};
+}
+
+// Sum of a head's partial states (internal basis, [160][DV] + [160] per segment) into the caller's state
+// (273 rows, or the 153 symmetric ones), added to it when `cont`.
+template <int DV>
+__global__ void __launch_bounds__(256) state_reduce_kernel(const float* __restrict__ ws, int nseg, float* __restrict__ kv,
+                                                           float* __restrict__ z, int dv, int sym, int cont) {
+    const size_t head = blockIdx.x;
+    const size_t stride = seg_state_floats(DV);
+    const float* wh = ws + head * nseg * stride;
+    const int nrows = sym ? kDSym : kD;
+    float* kvh = kv + head * (size_t)nrows * dv;
+    float* zh = z + head * (size_t)nrows;
+    // blockIdx.y: a block of 8 internal features (their DV value columns and their K-state entries)
+    const int f0 = blockIdx.y * 8;
+    for (int e = threadIdx.x; e < 8 * (DV + 1); e += 256) {
+        const bool zrow = e >= 8 * DV;
+        const int f = f0 + (zrow ? e - 8 * DV : e / DV), col = zrow ? 0 : e % DV;
+        const int idx = zrow ? kF * DV + f : f * DV + col;
+        const AbiRows ar = sym ? sym_rows(f) : abi_rows(f);
+        if (ar.a < 0 || (!zrow && col >= dv)) continue;
+        float acc = 0.f;
+        for (int sg = 0; sg < nseg; ++sg) acc += wh[sg * stride + idx];
+        if (ar.b >= 0) acc *= kRsqrt2;
+        float* dst = zrow ? zh : kvh + col;
+        const size_t pitch = zrow ? 1 : (size_t)dv;
+        dst[ar.a * pitch] = acc + (cont ? dst[ar.a * pitch] : 0.f);
+        if (ar.b >= 0) dst[ar.b * pitch] = acc + (cont ? dst[ar.b * pitch] : 0.f);
+    }
+}
+
+template <int DV>
+static based_status launch_state_dv(const void* k, const void* v, float* kv, float* z, int BH, int L, int dv, int flags,
+                                    float* ws, cudaStream_t stream) {
+    using C = Cfg<DV>;
+    const SegPlan plan = prefill_tc_state_plan(BH, L);
+    CUtensorMap tk, tv;
+    if (!make_map(&tk, k, BH, L, kDFeat, kDFeat, CU_TENSOR_MAP_SWIZZLE_32B) ||
+        !make_map(&tv, v, BH, L, dv, 64, CU_TENSOR_MAP_SWIZZLE_128B))
+        return BASED_ERR_CUDA;
+    Params p{};
+    p.ws = ws;
+    if (error_word_ptr(&p.err) != BASED_OK) return BASED_ERR_CUDA;
+    p.L = L;
+    p.nseg = plan.nseg + 1;            // the workspace holds nseg - 1 partial states per head
+    p.seg_len = plan.per * kC;
+    p.dv = dv;
+    {
+        static bool configured[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BASED_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(setup_mutex());
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(prefill_tc_kernel<DV, kModeState>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)C::kSmemBytes) != cudaSuccess)
+                return BASED_ERR_CUDA;
+            configured[dev] = true;
+        }
+    }
+    // the q and output maps are not used by the state-update-only pass
+    prefill_tc_kernel<DV, kModeState><<<dim3(plan.nseg, BH), kThreads, C::kSmemBytes, stream>>>(tk, tk, tv, tv, p);
+    note_launch();
+    based_status st = check_launch("prefill_tc_kernel<state>");
+    if (st != BASED_OK) return st;
+    state_reduce_kernel<DV><<<dim3(BH, kF / 8), 256, 0, stream>>>(ws, plan.nseg, kv, z, dv, (flags & BASED_STATE_SYM) ? 1 : 0,
+                                                                  (flags & BASED_STATE_CONTINUE) ? 1 : 0);
+    note_launch();
+    return check_launch("state_reduce_kernel");
+}
+
+size_t prefill_tc_state_workspace_bytes(int BH, int L, int d_v) {
+    if (d_v == 112) d_v = 128;
+    return (size_t)BH * prefill_tc_state_plan(BH, L).nseg * seg_state_floats(d_v) * sizeof(float);
+}
+
+based_status launch_prefill_tc_state(const void* k, const void* v, float* kv, float* z, int BH, int L, int d_v,
+                                     int flags, void* workspace, cudaStream_t stream) {
+    float* ws = static_cast<float*>(workspace);
+    if (d_v == 64) return launch_state_dv<64>(k, v, kv, z, BH, L, 64, flags, ws, stream);
+    return launch_state_dv<128>(k, v, kv, z, BH, L, d_v, flags, ws, stream);      // 112 or 128
+}
+
 size_t prefill_tc_workspace_bytes(int BH, int L, int d_v) {
     if (d_v == 112) d_v = 128;                      // runs on the d_v 128 kernel, partial states in its layout
     const SegPlan plan = prefill_tc_plan(BH, L, d_v);

@@ -125,6 +125,21 @@ def test_swa_decode_advance_validation(lib):
     assert f(P, P, P, P, P, O, 1, 1, 64, 200, P, 0.0, 1, None) == 2
 
 
+def test_prefill_state_validation(lib):
+    f = lib.based_prefill_state
+    O = ctypes.c_void_p(0x2000)
+    assert lib.based_prefill_state_workspace_bytes(4, 16, 2048, 16, 64, 1) > 0
+    assert lib.based_prefill_state_workspace_bytes(4, 16, 2048, 16, 64, 0) == 0          # fp32 io: no scratch
+    assert lib.based_prefill_state_workspace_bytes(4, 16, 2048, 24, 64, 1) == 0          # other d': no scratch
+    assert f(P, P, None, O, 1, 1, 8, 16, 64, 1, 0, P, 1 << 30, None) == 1                # state missing
+    assert f(P, P, O, O, 1, 1, 8, 16, 64, 1, 4, P, 1 << 30, None) == 1                   # NUMERATOR_ONLY is not a state flag
+    assert f(P, P, O, O, 1, 1, 8, 12, 64, 1, 0, P, 1 << 30, None) == 2
+    assert f(P, P, O, O, 1, 1, 8, 16, 64, 0, 2, P, 1 << 30, None) == 2                   # symmetric rows: bf16 io only
+    assert f(P, P, O, O, 1, 1, 8, 24, 64, 1, 2, P, 1 << 30, None) == 2                   # ... and d' = 16 only
+    assert f(P, U, O, O, 1, 1, 8, 16, 64, 1, 0, P, 1 << 30, None) == 3
+    assert f(P, P, O, O, 1, 1, 8, 16, 64, 1, 0, None, 0, None) == 6                      # workspace missing
+
+
 def test_baseconv_validation(lib):
     f = lib.baseconv_gate_forward
     O = ctypes.c_void_p(0x2000)

@@ -863,6 +863,58 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     assert torch.isfinite(out.float()).all()
 
 
+# --------------------------------------------------------------------------- state of a token block alone
+@pytest.mark.parametrize("dtype,d_feat,L,d_v,sym", [("bf16", 16, 700, 64, False), ("bf16", 16, 129, 128, True),
+                                                    ("bf16", 16, 1, 112, False), ("bf16", 16, 5000, 64, True),
+                                                    ("f32", 16, 300, 64, False), ("bf16", 24, 333, 128, False),
+                                                    ("f32", 8, 200, 112, False)])
+def test_prefill_state_matches_oracle_and_prefill(dtype, d_feat, L, d_v, sym):
+    """based_prefill_state: the state of a token block without outputs, from empty and added to a given state,
+    against the oracle's final state; and a sequence cut in two (state of the first half, then based_prefill
+    with BASED_STATE_CONTINUE on the second) against the oracle's outputs for the second half."""
+    B, H = 2, 3
+    w = wl.Workload("st", B, H, L, d_feat, d_v, dtype, 0.5)
+    q, k, v = wl.prefill_inputs(w, wl.generator(31 * L + d_feat))
+    y_ref, S_ref, z_ref = oracle.linattn_quadratic(_np(q), _np(k), _np(v))
+    if sym:
+        S_ref, z_ref = oracle.state_to_sym(S_ref, z_ref)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    fl = based.BASED_STATE_SYM if sym else 0
+    tol = tol_for(dtype)
+    kv, z = based.based_prefill_state(kd, vd, flags=fl)
+    _poll()
+    assert head_err(_np(kv), S_ref) <= tol and head_err(_np(z), z_ref) <= tol
+    # twice the block on top of itself: CONTINUE adds
+    kv2, z2 = based.based_prefill_state(kd, vd, kv_state=kv.clone(), z_state=z.clone(), flags=fl | based.BASED_STATE_CONTINUE)
+    assert head_err(_np(kv2), 2 * S_ref) <= tol and head_err(_np(z2), 2 * z_ref) <= tol
+    if L >= 2:
+        half = L // 2
+        kvh, zh = based.based_prefill_state(kd[:, :, :half].contiguous(), vd[:, :, :half].contiguous(), flags=fl)
+        out = based.based_prefill(qd[:, :, half:].contiguous(), kd[:, :, half:].contiguous(), vd[:, :, half:].contiguous(),
+                                  kv_state=kvh, z_state=zh, flags=fl | based.BASED_STATE_CONTINUE)
+        _poll()
+        assert row_err(_np(out), y_ref[:, :, half:]) <= tol
+        assert head_err(_np(kvh), S_ref) <= tol and head_err(_np(zh), z_ref) <= tol
+
+
+def test_sequence_parallel_helpers_on_one_process():
+    """dist.sequence_parallel_prefill / _swa with the library's kernels on a single process (world size 1: the
+    block is the whole sequence; the exchange across ranks is covered on CPU with gloo)."""
+    from paper_2402_18668_b200 import dist as bd
+    B, H, L, d_v = 2, 3, 900, 64
+    w = wl.Workload("sp", B, H, L, 16, d_v, "bf16", 0.5)
+    q, k, v = wl.prefill_inputs(w, wl.generator(77))
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    out, kv, z = bd.sequence_parallel_prefill(qd, kd, vd)
+    kv2, z2 = based.new_state(B, H, d_v)
+    ref = based.based_prefill(qd, kd, vd, kv_state=kv2, z_state=z2)
+    _poll()
+    assert torch.equal(out, ref) and torch.equal(kv, kv2) and torch.equal(z, z2)
+    qs, ks, vs = wl.swa_standalone_inputs(B, H, L, 64, torch.bfloat16, wl.generator(78))
+    o = bd.sequence_parallel_swa(qs.to(DEV), ks.to(DEV), vs.to(DEV), 64)
+    assert torch.equal(o, based.swa_forward(qs.to(DEV), ks.to(DEV), vs.to(DEV), window=64))
+
+
 # --------------------------------------------------------------------------- input scales
 @pytest.mark.parametrize("qk_scale,v_scale", [(0.0, 1.0), (1e-3, 1.0), (4.0, 1.0), (0.3, 1e4), (0.3, 1e-4)])
 def test_extreme_input_scales_bf16(qk_scale, v_scale):
