@@ -69,12 +69,16 @@ enum {
  *           both non-NULL.  With BASED_STATE_CONTINUE they are read as the state
  *           before token 0 (then they must be non-NULL); on return they hold the
  *           state after token L-1.  Accumulation and state are fp32 for both io dtypes.
+ *           The rows of the products k_m k_n and k_n k_m hold equal values in every state a
+ *           prefill or a decode step produces; the bf16 d_feat = 16 path relies on that and
+ *           returns both as their mean when it continues from a state where they differ.
  * workspace device scratch of at least based_prefill_workspace_bytes(...) bytes
  *           (may be NULL when that size is 0); contents are undefined afterwards.
  * Supported: d_feat = 16; d_v in {64, 112, 128}; io in {F32, BF16}; any L >= 1.
  * d_feat in {8, 24, 32} (the other dimensions of the paper's feature-map ablation; state rows
- * D = 1 + d_feat + d_feat^2 = 73, 601, 1057) is served by fp32 definition-form kernels for
- * both io dtypes: no workspace, no BASED_STATE_SYM, B*H <= 65535.
+ * D = 1 + d_feat + d_feat^2 = 73, 601, 1057) is served by the definition form: bf16 io from the
+ * empty state on tensor cores (outputs and state), the other cases by fp32 FMA kernels; no
+ * workspace, no BASED_STATE_SYM, B*H <= 65535.
  * out must not alias an input.
  */
 based_status based_prefill(const void* q, const void* k, const void* v, void* out, float* kv_state,
