@@ -8,7 +8,8 @@
 //             sums, and the product of the weight tile (through shared memory) with the value
 //             tile.  A given initial state adds phi(q_i).S0 and phi(q_i).z0 per row.
 //   state     S = S0 + sum_j phi(k_j) v_j^T, z = z0 + sum_j phi(k_j): one CTA per (head, 32 features).
-//   decode    the recurrent step as a plain stream over the [D, d_v] state, D = 1 + d' + d'^2.
+//   decode    the recurrent step as a stream over the [D, d_v] state, D = 1 + d' + d'^2 (both io dtypes; the
+//             loop of the d' = 16 decode kernel with the number of rows as a parameter).
 //
 // The state layout is the 273-row layout's generalisation: constant, linear terms, row-major
 // outer product.  The chunked tensor-core prefill and the symmetric format exist for d' = 16 only.
@@ -232,22 +233,33 @@ __global__ void __launch_bounds__(DV + 32) generic_state_kernel(const T* __restr
     }
 }
 
-// one recurrent step on the [D, d_v] state of a head (update, then read)
-template <typename T>
-__global__ void __launch_bounds__(256) generic_decode_kernel(const T* __restrict__ q, const T* __restrict__ k,
-                                                             const T* __restrict__ v, float* __restrict__ kv,
-                                                             float* __restrict__ z, T* __restrict__ out, int df,
-                                                             int dv, int numerator_only) {
+// one recurrent step on the [D, d_v] state of a head (update, then read): the d' = 16 decode kernel's
+// stream with the number of rows as a parameter.  d_v / 4 consecutive threads cover a state row with one
+// 128-bit load each, six rows are in flight per thread; STREAM: the state of all heads is larger than L2,
+// so every line is used once per step and takes the evict-first policy.
+template <typename T, int DV, bool STREAM>
+__global__ void __launch_bounds__(256, 4) generic_decode_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                                const T* __restrict__ v, float* __restrict__ kv,
+                                                                float* __restrict__ z, T* __restrict__ out, int df,
+                                                                int numerator_only) {
+    constexpr int TPR = DV / 4;                        // threads per state row
+    constexpr int RPP = 256 / TPR;                     // rows per pass: 8 (d_v 128), 9 (112), 16 (64)
+    constexpr int UNROLL = 6;
     __shared__ float s_x[2][kMaxDF];
     __shared__ float s_pq[1 + kMaxDF + kMaxDF * kMaxDF], s_pk[1 + kMaxDF + kMaxDF * kMaxDF];
-    __shared__ __align__(16) float s_num[8][128];      // written with 16-byte stores
+    __shared__ __align__(16) float s_num[RPP][DV];     // written with 16-byte stores
     __shared__ float s_den[8];
     const int tid = threadIdx.x;
     const size_t head = blockIdx.x;
     const int D = expanded_dim(df);
     const FeatScale sc = feat_scale(df);
+    const int c4 = tid % TPR, rslot = tid / TPR;
+    const bool row_thread = rslot < RPP;               // false only for the idle tail threads of d_v 112
     if (tid < df) s_x[0][tid] = to_f32(q[head * df + tid]);
     else if (tid >= 32 && tid < 32 + df) s_x[1][tid - 32] = to_f32(k[head * df + tid - 32]);
+    float vv[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) vv[e] = to_f32(v[head * DV + c4 * 4 + e]);
     __syncthreads();
     for (int f = tid; f < D; f += 256) {
         s_pq[f] = phi_gen(s_x[0], df, f, sc);
@@ -264,33 +276,44 @@ __global__ void __launch_bounds__(256) generic_decode_kernel(const T* __restrict
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) dpart += __shfl_xor_sync(0xffffffffu, dpart, o);
     if ((tid & 31) == 0) s_den[tid >> 5] = dpart;
-    // 32 column lanes (4 columns each for d_v 128; fewer are live for narrower heads) x 8 row slots
-    const int c4 = tid & 31, rslot = tid >> 5;
-    const bool live = c4 * 4 < dv;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), vv = acc;
-    if (live) {
-        vv.x = to_f32(v[head * dv + c4 * 4]); vv.y = to_f32(v[head * dv + c4 * 4 + 1]);
-        vv.z = to_f32(v[head * dv + c4 * 4 + 2]); vv.w = to_f32(v[head * dv + c4 * 4 + 3]);
-        float* S = kv + head * (size_t)D * dv + c4 * 4;
-        for (int r = rslot; r < D; r += 8) {
-            float4 s = *reinterpret_cast<float4*>(S + (size_t)r * dv);
-            const float pk = s_pk[r], pq = s_pq[r];
-            s.x = fmaf(pk, vv.x, s.x); s.y = fmaf(pk, vv.y, s.y); s.z = fmaf(pk, vv.z, s.z); s.w = fmaf(pk, vv.w, s.w);
-            acc.x = fmaf(pq, s.x, acc.x); acc.y = fmaf(pq, s.y, acc.y);
-            acc.z = fmaf(pq, s.z, acc.z); acc.w = fmaf(pq, s.w, acc.w);
-            *reinterpret_cast<float4*>(S + (size_t)r * dv) = s;
+
+    float4* S = reinterpret_cast<float4*>(kv + head * (size_t)D * DV) + c4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int npass = (D + RPP - 1) / RPP;
+    for (int p0 = 0; p0 < npass; p0 += UNROLL) {
+        float4 s[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int r = (p0 + u) * RPP + rslot;
+            if (r < D && row_thread) s[u] = STREAM ? __ldcs(&S[(size_t)r * TPR]) : S[(size_t)r * TPR];
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int r = (p0 + u) * RPP + rslot;
+            if (r < D && row_thread) {
+                const float pk = s_pk[r], pq = s_pq[r];
+                s[u].x = fmaf(pk, vv[0], s[u].x);
+                s[u].y = fmaf(pk, vv[1], s[u].y);
+                s[u].z = fmaf(pk, vv[2], s[u].z);
+                s[u].w = fmaf(pk, vv[3], s[u].w);
+                acc.x = fmaf(pq, s[u].x, acc.x);
+                acc.y = fmaf(pq, s[u].y, acc.y);
+                acc.z = fmaf(pq, s[u].z, acc.z);
+                acc.w = fmaf(pq, s[u].w, acc.w);
+                if (STREAM) __stcs(&S[(size_t)r * TPR], s[u]);
+                else S[(size_t)r * TPR] = s[u];
+            }
         }
     }
-    *reinterpret_cast<float4*>(&s_num[rslot][c4 * 4]) = acc;
+    if (row_thread) *reinterpret_cast<float4*>(&s_num[rslot][c4 * 4]) = acc;
     __syncthreads();
-    if (tid < dv) {
+    if (tid < DV) {
         float num = 0.f, den = 0.f;
 #pragma unroll
-        for (int r = 0; r < 8; ++r) {
-            num += s_num[r][tid];
-            den += s_den[r];
-        }
-        out[head * dv + tid] = from_f32<T>(numerator_only ? num : num / (den + kEps));
+        for (int r = 0; r < RPP; ++r) num += s_num[r][tid];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) den += s_den[w];
+        out[head * DV + tid] = from_f32<T>(numerator_only ? num : num / (den + kEps));
     }
 }
 
@@ -363,19 +386,33 @@ based_status launch_state_generic(const void* k, const void* v, float* kv, float
     return state_f32<128>(k, v, kv, z, BH, L, d_feat, cont, stream);
 }
 
+template <typename T, int DV>
+static based_status decode_t(const void* q, const void* k, const void* v, float* kv, float* z, void* out, int BH,
+                             int df, int num_only, cudaStream_t stream) {
+    // 96 MB: safely above what L2 (126 MB, shared with everything else) keeps from one step to the next
+    const bool streaming = (size_t)BH * expanded_dim(df) * DV * sizeof(float) > (size_t)96 << 20;
+    const T* qq = static_cast<const T*>(q);
+    const T* kk = static_cast<const T*>(k);
+    const T* vv = static_cast<const T*>(v);
+    if (streaming) generic_decode_kernel<T, DV, true><<<BH, 256, 0, stream>>>(qq, kk, vv, kv, z, static_cast<T*>(out), df, num_only);
+    else generic_decode_kernel<T, DV, false><<<BH, 256, 0, stream>>>(qq, kk, vv, kv, z, static_cast<T*>(out), df, num_only);
+    note_launch();
+    return check_launch("generic_decode_kernel");
+}
+
+template <typename T>
+static based_status decode_dv(const void* q, const void* k, const void* v, float* kv, float* z, void* out, int BH,
+                              int df, int d_v, int num_only, cudaStream_t stream) {
+    if (d_v == 64) return decode_t<T, 64>(q, k, v, kv, z, out, BH, df, num_only, stream);
+    if (d_v == 112) return decode_t<T, 112>(q, k, v, kv, z, out, BH, df, num_only, stream);
+    return decode_t<T, 128>(q, k, v, kv, z, out, BH, df, num_only, stream);
+}
+
 based_status launch_decode_generic(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
                                    int BH, int d_feat, int d_v, based_dtype io, bool numerator_only,
                                    cudaStream_t stream) {
-    if (io == BASED_F32)
-        generic_decode_kernel<float><<<BH, 256, 0, stream>>>(static_cast<const float*>(q), static_cast<const float*>(k),
-                                                             static_cast<const float*>(v), kv, z,
-                                                             static_cast<float*>(out), d_feat, d_v, numerator_only);
-    else
-        generic_decode_kernel<__nv_bfloat16><<<BH, 256, 0, stream>>>(
-            static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
-            static_cast<const __nv_bfloat16*>(v), kv, z, static_cast<__nv_bfloat16*>(out), d_feat, d_v, numerator_only);
-    note_launch();
-    return check_launch("generic_decode_kernel");
+    if (io == BASED_F32) return decode_dv<float>(q, k, v, kv, z, out, BH, d_feat, d_v, numerator_only ? 1 : 0, stream);
+    return decode_dv<__nv_bfloat16>(q, k, v, kv, z, out, BH, d_feat, d_v, numerator_only ? 1 : 0, stream);
 }
 
 }  // namespace based
