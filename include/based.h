@@ -209,7 +209,8 @@ based_status swa_decode_step(const void* q, const void* k, const void* v, void* 
  * s^2/(2 d'), so ds_ij = (a_i . v_j + b_i)(1/sqrt(d') + q_i.k_j / d')); d_v in {64, 112, 128}; B*H <= 65535.
  * Both paths evaluate the quadratic form, O(L^2) per head, on 128 x 128 (bf16 io: tcgen05 tensor
  * cores, bf16 operands, fp32 accumulation) or 64 x 64 (fp32 io: fp32 FMAs) tiles of (query, key)
- * pairs.  Gradient outputs must not alias inputs.
+ * pairs; with bf16 io, d_feat = 16 and BASED_NUMERATOR_ONLY, long sequences take the block-wise
+ * path described at based_prefill_backward_with_out.  Gradient outputs must not alias inputs.
  */
 based_status based_prefill_backward(const void* q, const void* k, const void* v, const void* dout, void* dq,
                                     void* dk, void* dv, int B, int H, int L, int d_feat, int d_v, based_dtype io,
@@ -226,6 +227,18 @@ size_t based_prefill_backward_workspace_bytes(int B, int H, int L, int d_v, base
  * rounding of out, keeps the cancellation against b_i in fp32.  out is used for this centring
  * only: D_i and dout_i . N_i are still recomputed in fp32.  fp32 io ignores out's values.
  * out must not alias a gradient output.
+ *
+ * Block-wise path (bf16 io, d_feat = 16; L >= 1536 at d_v 64, L >= 2048 at d_v 112 / 128): O(L) per
+ * head, the recurrent view of Sec. 4.1 applied to the gradients.  The sequence is cut into blocks of
+ * W = 256 (d_v 64) or 512 tokens.  Pairs inside a block go through the tiles above.  All earlier
+ * blocks reach a query through their summed state S = sum_j phi(k_j) v_j^T, z = sum_j phi(k_j):
+ *   sum_j w'_ij (dout_i.v_j - m_i) k_j = J(q_i)^T (S dout_i - m_i z),   D_i += phi(q_i) . z
+ * (J the Jacobian of phi), and all later blocks reach a key through R = sum_i phi(q_i) (dout_i / D_i)^T
+ * and R_b = sum_i b_i phi(q_i):  dk_j += J(k_j)^T (R v_j + R_b),  dv_j += R^T phi(k_j).
+ * The block states are fp32 sums, rounded once to bf16 as tensor-core operands, like the state copy of
+ * the forward pass; the products S dout_i and m_i z cancel in fp32 after the product, so the error
+ * relative to the gradient grows with |mean v| / std v over the earlier blocks (1.5e-2 at mean 3,
+ * std 1; 3e-3 for centred values).  Seven launches instead of two.
  */
 based_status based_prefill_backward_with_out(const void* q, const void* k, const void* v, const void* out,
                                              const void* dout, void* dq, void* dk, void* dv, int B, int H, int L,

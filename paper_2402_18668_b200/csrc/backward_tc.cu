@@ -48,23 +48,28 @@ constexpr uint32_t kQKTile = kTile * 64;                 // [128][32] bf16, 64-b
 // LT: rows of the tiles the CTA loops over (columns of the accumulators): 64 where that lets two CTAs
 // share an SM (256 tensor-memory columns each), so that one CTA's row-thread pass overlaps the
 // other's MMA bursts; 128 for the dk/dv pass at d_v 128, whose accumulators need more columns.
-template <int DV, int MODE, int LT> struct BCfg {
+template <int DV, int MODE, int LT, bool XB = false> struct BCfg {
     static constexpr int kVB = (DV + 63) / 64;           // 64-column blocks of a [rows][DV] tile (112 -> 2, second partly zero)
     static constexpr uint32_t kWide = kVB * kTile * 128; // own tile: [128][64 * kVB] bf16 in SWIZZLE_128B blocks
     static constexpr uint32_t kNarrowL = LT * 64, kWideL = kVB * LT * 128;       // looped tiles
     // shared memory: resident narrow + wide tile, two stages of (narrow + wide), (1/D, b) of two stages, barriers
     static constexpr uint32_t offResN = 0, offResW = offResN + kQKTile;
     static constexpr uint32_t offStage = offResW + kWide, kStage = kNarrowL + kWideL;
-    static constexpr uint32_t offB = offStage + 2 * kStage;
+    // a block state [160][64 * kVB] bf16 (block-wise path) lies from the second stage on, so that the first looped
+    // tile loads beside it
+    static constexpr uint32_t kStateTile = kVB * 160 * 128;
+    static constexpr uint32_t kStageArea = (XB && kStage + kStateTile > 2 * kStage) ? kStage + kStateTile : 2 * kStage;
+    static constexpr uint32_t offB = offStage + kStageArea;
     static constexpr uint32_t offMisc = offB + 2 * LT * 8;
-    static constexpr uint32_t kSmem = offMisc + 256 + 1024;
+    static constexpr uint32_t kSmem = offMisc + 1024 + 1024;                    // barriers, the block state's row sums (160 floats)
+
     // tensor memory columns: scores, dout.v products, ds (dq pass; the dk/dv pass packs in place), accumulators
     static constexpr uint32_t colS = 0, colG = LT, colD = MODE == kModeFwd ? LT : 2 * LT;   // forward: no dout.v product
     static constexpr uint32_t colD2 = colD + LT / 2;                                      // second packed tile (merged pass)
     static constexpr uint32_t colAcc = MODE == kModeDq ? 2 * LT + LT / 2                  // dQ (32)
                                        : MODE == kModeDqS ? 3 * LT                        // X (32), then Y (32)
                                        : MODE == kModeFwd ? LT + LT / 2                   // Y (64 * kVB)
-                                                          : 2 * LT;                       // dV (64 * kVB)
+                                                          : (2 * LT < 160 ? 160 : 2 * LT);  // dV (64 * kVB), above the block product
     static constexpr uint32_t colAcc2 = colAcc + 32;                                      // merged pass: Y
     static constexpr uint32_t colK = colAcc + 64 * kVB;                                   // dK (32), dk/dv pass
     static constexpr uint32_t kColsUsed = MODE == kModeStats ? 2 * LT
@@ -75,7 +80,7 @@ template <int DV, int MODE, int LT> struct BCfg {
     static constexpr uint32_t kCols = kColsUsed <= 128 ? 128 : kColsUsed <= 256 ? 256 : 512;
     static_assert(kColsUsed <= 512, "tensor memory budget");
 };
-enum { bRes = 0, bFull0, bFull1, bMma, bAlu, bFinal, bNum };
+enum { bRes = 0, bFull0, bFull1, bMma, bAlu, bFinal, bXs, bX0, bX1, bNum };
 
 struct BParams {
     const __nv_bfloat16* g_raw;  // dout and the forward output as plain pointers [BH, L, dvw] (merged pass)
@@ -89,6 +94,9 @@ struct BParams {
     int L, dvw, numerator_only;  // dvw: value head dimension of the caller's tensors (64, 112, 128)
     int df, kdim;                // feature dimension d', and d' rounded up to 16 (K extent of the scores)
     float s1, s2;                // w = 1 + s * s1 + s^2 * s2 (1 / sqrt d', 1 / (2 d'))
+    // block-wise path: pairs inside a block of W tokens by tiles, the other blocks through their summed state
+    int W, nblk;
+    const float* sv;             // [BH x nblk][160]: row sums of the block states (z, or the b-weighted sums of phi(q))
 };
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -113,22 +121,79 @@ __device__ __forceinline__ bool rows_all(bool pred) {
 // w = 1 + s / sqrt(d') + s^2 / (2 d') and its derivative, s1 = 1 / sqrt(d'), s2 = 1 / (2 d') (d' = 16: 1/4, 1/32)
 __device__ __forceinline__ float tw(float s, float s1, float s2) { return fmaf(s, fmaf(s, s2, s1), 1.0f); }
 __device__ __forceinline__ float tdw(float s, float s1, float s2) { return fmaf(s, 2.0f * s2, s1); }
+
+// Block-wise path, one row thread: T (160 fp32 columns of tensor memory, from column 0) holds the product of the
+// row's wide operand with a block state in the monomial basis of generic_state_tc_kernel<.., true>
+// (f < 16: x_f | 16 + 16 o + m: x_m x_(m+o) | 144 + m: x_m x_(m+8) | 152: 1), sv the state's row sums.
+//   query row (merged statistics + dq pass): T_f = (S g_i)_f, sv = z:
+//     den += mono(q_i) . z,  en += mono(q_i) . T,  gx = J^T (T - m_i z),  gy = J^T z      (J = d mono / d q_i)
+//   key row (dk/dv pass): T_f = (R v_j)_f, sv = R_b:  gx = J^T (T + R_b); the monomials of k_j go back to tensor
+//     memory as packed bf16 (80 columns from column 0, over the columns already read): the A operand of dV += mono(K) R
+template <bool KEYS>
+__device__ __forceinline__ void block_rows(uint32_t tb, uint32_t lane_base, const float (&x)[16], const float* sv,
+                                           float m_own, float& den, float& en, float (&gx)[16], float (&gy)[16]) {
+#pragma unroll
+    for (int blk = 0; blk < 5; ++blk) {
+        uint32_t tr[32];
+        tmem_ld32(tmem_addr(tb, lane_base, blk * 32), tr);
+        tmem_wait_ld();
+        float mono[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const int f = blk * 32 + i;
+            const int m = f < 16 ? f : f < 144 ? ((f - 16) & 15) : f < 152 ? f - 144 : -1;
+            const int n = f < 16 ? -1 : f < 144 ? ((m + ((f - 16) >> 4)) & 15) : f < 152 ? m + 8 : -1;
+            mono[i] = 0.f;
+            if (f <= 152) {
+                const float xm = m >= 0 ? x[m] : 1.0f, xn = n >= 0 ? x[n] : 1.0f;
+                mono[i] = xm * xn;
+                const float a = __uint_as_float(tr[i]), zf = sv[f];
+                const float bq = KEYS ? a + zf : fmaf(-m_own, zf, a);
+                if (!KEYS) {
+                    den = fmaf(mono[i], zf, den);
+                    en = fmaf(mono[i], a, en);
+                }
+                if (m >= 0 && n < 0) {
+                    gx[m] += bq;
+                    if (!KEYS) gy[m] += zf;
+                } else if (m >= 0 && m != n) {
+                    gx[m] = fmaf(xn, bq, gx[m]);
+                    gx[n] = fmaf(xm, bq, gx[n]);
+                    if (!KEYS) { gy[m] = fmaf(xn, zf, gy[m]); gy[n] = fmaf(xm, zf, gy[n]); }
+                } else if (m >= 0) {
+                    gx[m] = fmaf(2.0f * xm, bq, gx[m]);
+                    if (!KEYS) gy[m] = fmaf(2.0f * xm, zf, gy[m]);
+                }
+            }
+        }
+        if (KEYS) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(mono[2 * i], mono[2 * i + 1]);
+            tmem_st16(tmem_addr(tb, lane_base, blk * 16), pk);
+        }
+    }
+}
 }  // namespace
 
 // tm_n0 / tm_w0: narrow (q or k) and wide (a/g or v) tensor of the CTA's own (resident) tile;
 // tm_n1 / tm_w1: of the tiles it loops over.
-template <int DV, int MODE, int LT>
+// XB: the block-wise path (merged statistics + dq pass and dk/dv pass, d' = 16); tm_st: the block states
+// [BH x nblk][160][d_v] bf16.
+template <int DV, int MODE, int LT, bool XB>
 __global__ void __launch_bounds__(kThreadsB, 1)
     backward_tc_kernel(const __grid_constant__ CUtensorMap tm_n0, const __grid_constant__ CUtensorMap tm_w0,
                        const __grid_constant__ CUtensorMap tm_n1, const __grid_constant__ CUtensorMap tm_w1,
-                       const BParams p) {
-    using C = BCfg<DV, MODE, LT>;
+                       const __grid_constant__ CUtensorMap tm_st, const BParams p) {
+    static_assert(!XB || MODE == kModeDqS || MODE == kModeDkDv, "block-wise path: the two passes that use it");
+    using C = BCfg<DV, MODE, LT, XB>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offMisc);
     uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + bNum);
     volatile uint32_t* abort_flag = tmem_base_s + 1;
     float2* s_b = reinterpret_cast<float2*>(smem + C::offB);
+    float* s_sv = reinterpret_cast<float*>(smem + C::offMisc + 256);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int ntiles = (p.L + kTile - 1) / kTile;
@@ -137,15 +202,23 @@ __global__ void __launch_bounds__(kThreadsB, 1)
     const int head = blockIdx.y;
     const int r0 = own * kTile;
     // looped tiles (LT rows each): keys 0 .. end of the own tile, or queries from the own tile's first row on
-    const int first = MODE == kModeDkDv ? r0 / LT : 0;
-    const int last = MODE == kModeDkDv ? (p.L - 1) / LT : (min(p.L, r0 + kTile) - 1) / LT;
+    // block-wise path: the loop stays inside the own tile's block of W tokens; the blocks before it (queries) or
+    // after it (keys) enter through their summed state, if there are any (cross)
+    const int blk = XB ? r0 / p.W : 0;
+    const bool cross = XB && (MODE == kModeDkDv ? blk + 1 < p.nblk : blk > 0);
+    const int first = MODE == kModeDkDv ? r0 / LT : (XB ? blk * p.W / LT : 0);
+    const int last = MODE == kModeDkDv ? (min(p.L, XB ? (blk + 1) * p.W : p.L) - 1) / LT : (min(p.L, r0 + kTile) - 1) / LT;
     const int nloop = last - first + 1;
 
     if (tid == 0) {
         mbar_init(&bars[bRes], 1); mbar_init(&bars[bFull0], 1); mbar_init(&bars[bFull1], 1);
         mbar_init(&bars[bMma], 1); mbar_init(&bars[bAlu], 128); mbar_init(&bars[bFinal], 1);
+        mbar_init(&bars[bXs], 1); mbar_init(&bars[bX0], 1); mbar_init(&bars[bX1], 128);
         *abort_flag = 0;
         fence_mbar_init();
+    }
+    if (cross) {
+        for (int i = tid; i < 160; i += kThreadsB) s_sv[i] = p.sv[((size_t)head * p.nblk + blk) * 160 + i];
     }
     if (warp == 4) { tmem_alloc(tmem_base_s, C::kCols); tmem_relinquish(); }
     tc_fence_before();
@@ -161,6 +234,8 @@ __global__ void __launch_bounds__(kThreadsB, 1)
     constexpr uint32_t iS = make_idesc_bf16(128, LT, 0, 0);                             // both operands K-major
     constexpr uint32_t iN32 = make_idesc_bf16(128, 32, 0, 1);                           // A from TMEM, B MN-major narrow
     constexpr uint32_t iNV = make_idesc_bf16(128, 64 * C::kVB, 0, 1);                   // A from TMEM, B MN-major wide
+    constexpr uint64_t dSt = make_smem_desc_base(160 * 128, 1024, kSwizzle128B);        // block state (160 rows per block)
+    constexpr uint32_t iT = make_idesc_bf16(128, 160, 0, 0);                            // own wide x state^T
 
     if (warp == 4) {
         if (lane == 0) {
@@ -182,8 +257,53 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                 for (int b = 0; b < C::kVB; ++b)
                     tma_load_3d(smem + C::offResW + b * (kTile * 128), &tm_w0, &bars[bRes], b * 64, r0, head);
             }
+            if (cross) {
+                mbar_arrive_expect_tx(&bars[bXs], C::kStateTile);
+#pragma unroll
+                for (int b = 0; b < C::kVB; ++b)
+                    tma_load_3d(smem + C::offStage + C::kStage + b * (160 * 128), &tm_st, &bars[bXs], b * 64, 0,
+                                head * p.nblk + blk);
+            }
             load_stage(0);
             ok = mbar_wait(&bars[bRes], 0, abort_flag);
+            if (cross && ok) {
+                const uint32_t aSt = smem_u32(smem + C::offStage + C::kStage);
+                ok = mbar_wait(&bars[bXs], 0, abort_flag);
+                tc_fence_after();
+                // T = own wide tile x state^T (K = d_v), 160 columns from column 0
+#pragma unroll
+                for (int kk = 0; kk < DV / 16; ++kk) {
+                    const uint32_t off = ((kk >> 2) * (kTile * 128) + (kk & 3) * 32) >> 4;
+                    const uint32_t offS = ((kk >> 2) * (160 * 128) + (kk & 3) * 32) >> 4;
+                    if (kk == 0)
+                        mma_ss_lh<false>(tb, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW), desc_lo(dSt) + (aSt >> 4) + offS,
+                                         desc_hi(dSt), iT);
+                    else
+                        mma_ss_lh<true>(tb, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW), desc_lo(dSt) + (aSt >> 4) + offS,
+                                        desc_hi(dSt), iT);
+                }
+                mma_commit(&bars[bX0]);
+                if (MODE == kModeDkDv) {
+                    // dV = mono(K) (tensor memory, written by the row threads) x state (MN-major, 160 = 10 K-steps)
+                    if (ok) ok = mbar_wait(&bars[bX1], 0, abort_flag);
+                    tc_fence_after();
+                    if (ok) {
+#pragma unroll
+                        for (int k = 0; k < 10; ++k) {
+                            if (k == 0)
+                                mma_ts_lh<false>(tb + C::colAcc, tb + k * 8, desc_lo(dSt) + ((aSt + k * 2048) >> 4),
+                                                 desc_hi(dSt), iNV);
+                            else
+                                mma_ts_lh<true>(tb + C::colAcc, tb + k * 8, desc_lo(dSt) + ((aSt + k * 2048) >> 4),
+                                                desc_hi(dSt), iNV);
+                        }
+                    }
+                } else {
+                    if (ok) ok = mbar_wait(&bars[bX1], 0, abort_flag);     // the rows have read T: the scores may overwrite it
+                    tc_fence_after();
+                }
+                // the state tile's stages are loaded again after the first iteration's products (in-order pipe)
+            }
             for (int it = 0; it < nloop && ok; ++it) {
                 const int s = it & 1;
                 const uint32_t aN = smem_u32(smem + C::offStage + s * C::kStage), aW = aN + C::kNarrowL;
@@ -231,7 +351,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                     // X += (w' (gv - m)) K_j and Y += w' K_j: two packed tiles in tensor memory, the same B operand
 #pragma unroll
                     for (int k = 0; k < LT / 16; ++k) {
-                        if (it == 0 && k == 0) {
+                        if (it == 0 && k == 0 && !cross) {
                             mma_ts_lh<false>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                              desc_hi(dN), iN32);
                             mma_ts_lh<false>(tb + C::colAcc2, tb + C::colD2 + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
@@ -258,7 +378,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                     // dV += W'^T (over the scores) x G_i;  dK += DS^T (over GV) x Q_i
 #pragma unroll
                     for (int k = 0; k < LT / 16; ++k) {
-                        if (it == 0 && k == 0) {
+                        if (it == 0 && k == 0 && !cross) {
                             mma_ts_lh<false>(tb + C::colAcc, tb + C::colS + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
                                              desc_hi(dWL), iNV);
                             mma_ts_lh<false>(tb + C::colK, tb + C::colG + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
@@ -311,6 +431,45 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                 }
             }
             m_own = (part[0] + part[1]) + (part[2] + part[3]);
+        }
+        if (XB && cross) {
+            // the blocks before (queries) or after (keys) the own one, through their summed state
+            ok = rows_all(mbar_wait(&bars[bRes], 0, abort_flag) && mbar_wait(&bars[bX0], 0, abort_flag));
+            tc_fence_after();
+            if (ok) {
+                // this thread's q or k row: 64-byte rows, SWIZZLE_64B (16-byte pieces 0 and 1)
+                float x[16], gx[16], gy[16];
+                const uint8_t* xrow = smem + C::offResN + t * 64;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const uint4 u = *reinterpret_cast<const uint4*>(xrow + ((c ^ ((t >> 1) & 3)) << 4));
+                    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float2 fv = __bfloat1622float2(h[i]);
+                        x[c * 8 + 2 * i] = fv.x;
+                        x[c * 8 + 2 * i + 1] = fv.y;
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 16; ++i) { gx[i] = 0.f; gy[i] = 0.f; }
+                block_rows<MODE == kModeDkDv>(tb, lane_base, x, s_sv, m_own, den, en, gx, gy);
+                // the sums start the accumulators that the loop's products add to: X and Y, or dK
+                uint32_t o[16], zero[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) { o[i] = __float_as_uint(gx[i]); zero[i] = 0u; }
+                tmem_st16(tmem_addr(tb, lane_base, MODE == kModeDkDv ? C::colK : C::colAcc), o);
+                tmem_st16(tmem_addr(tb, lane_base, (MODE == kModeDkDv ? C::colK : C::colAcc) + 16), zero);
+                if (MODE == kModeDqS) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(gy[i]);
+                    tmem_st16(tmem_addr(tb, lane_base, C::colAcc2), o);
+                    tmem_st16(tmem_addr(tb, lane_base, C::colAcc2 + 16), zero);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(&bars[bX1]);
+            }
         }
         for (int it = 0; it < nloop && ok; ++it) {
             const int c0 = (first + it) * LT;                // first row of the looped tile (columns of the accumulators)
@@ -504,25 +663,98 @@ bool make_rows_map_bf16(CUtensorMap* m, const void* base, int BH, int L, int wid
 }
 
 namespace {
-template <int DV, int MODE, int LT>
+// Block-wise path, between the passes.  state_scan_kernel: the per-block states of
+// generic_state_tc_kernel<.., true> summed over the blocks before (suffix = 0) or after (suffix = 1) each
+// block, as bf16 [BH x nblk][160][dvw] (tensor-core operand) and fp32 row sums [BH x nblk][160].
+__global__ void __launch_bounds__(256)
+    state_scan_kernel(const float* __restrict__ part, const float* __restrict__ zpart, __nv_bfloat16* __restrict__ st,
+                      float* __restrict__ sv, int nblk, int per, int suffix) {
+    const int e = blockIdx.x * 256 + threadIdx.x;
+    const size_t h0 = (size_t)blockIdx.y * nblk;
+    if (e < per) {
+        float run = 0.f;
+        for (int i = 0; i < nblk; ++i) {
+            const int c = suffix ? nblk - 1 - i : i;
+            st[(h0 + c) * per + e] = __float2bfloat16(run);
+            run += part[(h0 + c) * per + e];
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < 160) {
+        float run = 0.f;
+        for (int i = 0; i < nblk; ++i) {
+            const int c = suffix ? nblk - 1 - i : i;
+            sv[(h0 + c) * 160 + threadIdx.x] = run;
+            run += zpart[(h0 + c) * 160 + threadIdx.x];
+        }
+    }
+}
+// scaled_dout_kernel: dout_i / D_i as bf16 (the value operand of the query-side states), eight columns per thread
+__global__ void __launch_bounds__(256)
+    scaled_dout_kernel(const uint4* __restrict__ g, const float2* __restrict__ stats, uint4* __restrict__ ga, size_t n8,
+                       int dv8) {
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= n8) return;
+    const float dinv = stats[i / dv8].x;
+    const uint4 u = g[i];
+    uint4 o;
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+    uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const float2 f = __bfloat1622float2(h[c]);
+        ow[c] = pack_bf16x2(f.x * dinv, f.y * dinv);
+    }
+    ga[i] = o;
+}
+
+template <int DV, int MODE, int LT, bool XB = false>
 based_status launch_pass(const CUtensorMap& n0, const CUtensorMap& w0, const CUtensorMap& n1, const CUtensorMap& w1,
-                         const BParams& p, dim3 grid, const char* what, cudaStream_t stream) {
-    using C = BCfg<DV, MODE, LT>;
+                         const BParams& p, dim3 grid, const char* what, cudaStream_t stream,
+                         const CUtensorMap* st = nullptr) {
+    using C = BCfg<DV, MODE, LT, XB>;
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BASED_ERR_CUDA;
     {
         std::lock_guard<std::mutex> lock(setup_mutex());
         if (!configured[dev]) {
-            if (cudaFuncSetAttribute(backward_tc_kernel<DV, MODE, LT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            if (cudaFuncSetAttribute(backward_tc_kernel<DV, MODE, LT, XB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)C::kSmem) != cudaSuccess)
                 return BASED_ERR_CUDA;
             configured[dev] = true;
         }
     }
-    backward_tc_kernel<DV, MODE, LT><<<grid, kThreadsB, C::kSmem, stream>>>(n0, w0, n1, w1, p);
+    backward_tc_kernel<DV, MODE, LT, XB><<<grid, kThreadsB, C::kSmem, stream>>>(n0, w0, n1, w1, st ? *st : n0, p);
     note_launch();
     return check_launch(what);
+}
+
+// Block length of the block-wise path, or 0 for the tile path alone.  The block-wise path needs d' = 16 and the
+// statistics in one sweep (the forward output, or the numerator-only form); its cost grows with L where the tile
+// path's grows with L^2, and the lengths below are where it starts to win on B200 (d_v 64: 274 against 317 us at
+// L = 1536 for 128 heads; d_v 128: 508 against 616 us at L = 2048).
+int backward_block_len(int L, int df, bool merged, int d_v) {
+    if (df != 16 || !merged) return 0;
+    if (d_v == 64) return L >= 1536 ? 256 : 0;
+    return L >= 2048 ? 512 : 0;
+}
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+struct BlockWs {
+    float* sv; float* zpart; float* part; __nv_bfloat16* st; __nv_bfloat16* ga;
+    size_t bytes;
+};
+// scratch after the [BH, L] float2 statistics
+BlockWs block_ws(float* ws, int BH, int L, int dvr, int nblk) {
+    BlockWs w{};
+    const uintptr_t base = reinterpret_cast<uintptr_t>(ws);
+    size_t off = align256((size_t)BH * L * 8);
+    w.sv = reinterpret_cast<float*>(base + off);     off = align256(off + (size_t)BH * nblk * 160 * 4);
+    w.zpart = reinterpret_cast<float*>(base + off);  off = align256(off + (size_t)BH * nblk * 160 * 4);
+    w.part = reinterpret_cast<float*>(base + off);   off = align256(off + (size_t)BH * nblk * 160 * dvr * 4);
+    w.st = reinterpret_cast<__nv_bfloat16*>(base + off);  off = align256(off + (size_t)BH * nblk * 160 * dvr * 2);
+    w.ga = reinterpret_cast<__nv_bfloat16*>(base + off);  off = align256(off + (size_t)BH * L * dvr * 2);
+    w.bytes = off;
+    return w;
 }
 
 template <int DV>
@@ -556,6 +788,37 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
     p.s2 = 0.5f / (float)df;
     const dim3 grid((L + kTile - 1) / kTile, BH);
     based_status st;
+    const int W = backward_block_len(L, df, out != nullptr || numerator_only, dvr);
+    if (W > 0) {
+        // block-wise: pairs inside a block of W tokens by tiles, everything else through summed block states
+        const int nblk = (L + W - 1) / W;
+        const BlockWs w = block_ws(ws, BH, L, dvr, nblk);
+        CUtensorMap tst;
+        if (!make_map_b(&tst, w.st, BH * nblk, 160, dvr, 64, 160, s128)) return BASED_ERR_CUDA;
+        p.W = W;
+        p.nblk = nblk;
+        p.sv = w.sv;
+        // states of the keys: S = sum mono(k) v^T, z = sum mono(k), summed over the blocks before each block
+        st = launch_state_blocks_tc(k, v, nullptr, 0, w.part, w.zpart, BH, L, W, dvr, stream);
+        if (st != BASED_OK) return st;
+        state_scan_kernel<<<dim3((160 * dvr + 255) / 256, BH), 256, 0, stream>>>(w.part, w.zpart, w.st, w.sv, nblk, 160 * dvr, 0);
+        note_launch();
+        if ((st = check_launch("state_scan_kernel")) != BASED_OK) return st;
+        st = launch_pass<DV, kModeDqS, 64, true>(tq, tg, tk64, tv64, p, grid, "backward_tc_kernel<stats+dq, blocks>", stream, &tst);
+        if (st != BASED_OK) return st;
+        // states of the queries: R = sum mono(q) (dout / D)^T, R_b = sum b mono(q), summed over the blocks after each block
+        const size_t n8 = (size_t)BH * L * dvr / 8;
+        scaled_dout_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, stream>>>(
+            static_cast<const uint4*>(g), stats, reinterpret_cast<uint4*>(w.ga), n8, dvr / 8);
+        note_launch();
+        if ((st = check_launch("scaled_dout_kernel")) != BASED_OK) return st;
+        st = launch_state_blocks_tc(q, w.ga, reinterpret_cast<const float*>(stats) + 1, 2, w.part, w.zpart, BH, L, W, dvr, stream);
+        if (st != BASED_OK) return st;
+        state_scan_kernel<<<dim3((160 * dvr + 255) / 256, BH), 256, 0, stream>>>(w.part, w.zpart, w.st, w.sv, nblk, 160 * dvr, 1);
+        note_launch();
+        if ((st = check_launch("state_scan_kernel")) != BASED_OK) return st;
+        return launch_pass<DV, kModeDkDv, LTK, true>(tk, tv, tqL, tgL, p, grid, "backward_tc_kernel<dkdv, blocks>", stream, &tst);
+    }
     if (out != nullptr || numerator_only) {
         // statistics and dq in one sweep (needs the forward output as the centre of the packed products)
         st = launch_pass<DV, kModeDqS, 64>(tq, tg, tk64, tv64, p, grid, "backward_tc_kernel<stats+dq>", stream);
@@ -598,7 +861,8 @@ based_status launch_quadratic_forward_tc(const void* q, const void* k, const voi
 }
 
 size_t backward_tc_workspace_bytes(int BH, int L, int d_v) {
-    (void)d_v;
+    const int W = backward_block_len(L, 16, true, d_v);
+    if (W > 0) return block_ws(nullptr, BH, L, d_v, (L + W - 1) / W).bytes;         // statistics, block states, dout / D
     return (size_t)BH * L * 2 * sizeof(float);                 // (1 / D, b) per row
 }
 
