@@ -55,9 +55,10 @@ template <int DV, int MODE, int LT, bool XB = false> struct BCfg {
     // shared memory: resident narrow + wide tile, two stages of (narrow + wide), (1/D, b) of two stages, barriers
     static constexpr uint32_t offResN = 0, offResW = offResN + kQKTile;
     static constexpr uint32_t offStage = offResW + kWide, kStage = kNarrowL + kWideL;
-    // a block state [160][64 * kVB] bf16 (block-wise path) lies from the second stage on, so that the first looped
-    // tile loads beside it
-    static constexpr uint32_t kStateTile = kVB * 160 * 128;
+    // a block state, transposed: [64 * kVB value columns][160 features] bf16 in five SWIZZLE_64B blocks of 32 features
+    // (block-wise path); it lies from the second stage on, so that the first looped tile loads beside it
+    static constexpr uint32_t kStateBlk = kVB * 64 * 64;
+    static constexpr uint32_t kStateTile = 5 * kStateBlk;
     static constexpr uint32_t kStageArea = (XB && kStage + kStateTile > 2 * kStage) ? kStage + kStateTile : 2 * kStage;
     static constexpr uint32_t offB = offStage + kStageArea;
     static constexpr uint32_t offMisc = offB + 2 * LT * 8;
@@ -123,7 +124,7 @@ __device__ __forceinline__ float tw(float s, float s1, float s2) { return fmaf(s
 __device__ __forceinline__ float tdw(float s, float s1, float s2) { return fmaf(s, 2.0f * s2, s1); }
 
 // Block-wise path, one row thread: T (160 fp32 columns of tensor memory, from column 0) holds the product of the
-// row's wide operand with a block state in the monomial basis of generic_state_tc_kernel<.., true>
+// row's wide operand with a block state in the monomial basis of block_state_tc_kernel
 // (f < 16: x_f | 16 + 16 o + m: x_m x_(m+o) | 144 + m: x_m x_(m+8) | 152: 1), sv the state's row sums.
 //   query row (merged statistics + dq pass): T_f = (S g_i)_f, sv = z:
 //     den += mono(q_i) . z,  en += mono(q_i) . T,  gx = J^T (T - m_i z),  gy = J^T z      (J = d mono / d q_i)
@@ -178,8 +179,8 @@ __device__ __forceinline__ void block_rows(uint32_t tb, uint32_t lane_base, cons
 
 // tm_n0 / tm_w0: narrow (q or k) and wide (a/g or v) tensor of the CTA's own (resident) tile;
 // tm_n1 / tm_w1: of the tiles it loops over.
-// XB: the block-wise path (merged statistics + dq pass and dk/dv pass, d' = 16); tm_st: the block states
-// [BH x nblk][160][d_v] bf16.
+// XB: the block-wise path (merged statistics + dq pass and dk/dv pass, d' = 16); tm_st: the block states,
+// transposed: [BH x nblk][d_v][160] bf16.
 template <int DV, int MODE, int LT, bool XB>
 __global__ void __launch_bounds__(kThreadsB, 1)
     backward_tc_kernel(const __grid_constant__ CUtensorMap tm_n0, const __grid_constant__ CUtensorMap tm_w0,
@@ -234,8 +235,9 @@ __global__ void __launch_bounds__(kThreadsB, 1)
     constexpr uint32_t iS = make_idesc_bf16(128, LT, 0, 0);                             // both operands K-major
     constexpr uint32_t iN32 = make_idesc_bf16(128, 32, 0, 1);                           // A from TMEM, B MN-major narrow
     constexpr uint32_t iNV = make_idesc_bf16(128, 64 * C::kVB, 0, 1);                   // A from TMEM, B MN-major wide
-    constexpr uint64_t dSt = make_smem_desc_base(160 * 128, 1024, kSwizzle128B);        // block state (160 rows per block)
-    constexpr uint32_t iT = make_idesc_bf16(128, 160, 0, 0);                            // own wide x state^T
+    constexpr uint64_t dStN = make_smem_desc_base(C::kStateBlk, 512, kSwizzle64B);      // block state as B over d_v: MN-major
+    constexpr uint32_t iT = make_idesc_bf16(128, 160, 0, 1);                            // own wide x state^T
+    constexpr uint32_t iXV = make_idesc_bf16(128, 64 * C::kVB, 0, 0);                   // A from TMEM, B K-major: the state over features
 
     if (warp == 4) {
         if (lane == 0) {
@@ -260,8 +262,8 @@ __global__ void __launch_bounds__(kThreadsB, 1)
             if (cross) {
                 mbar_arrive_expect_tx(&bars[bXs], C::kStateTile);
 #pragma unroll
-                for (int b = 0; b < C::kVB; ++b)
-                    tma_load_3d(smem + C::offStage + C::kStage + b * (160 * 128), &tm_st, &bars[bXs], b * 64, 0,
+                for (int b = 0; b < 5; ++b)
+                    tma_load_3d(smem + C::offStage + C::kStage + b * C::kStateBlk, &tm_st, &bars[bXs], b * 32, 0,
                                 head * p.nblk + blk);
             }
             load_stage(0);
@@ -274,28 +276,28 @@ __global__ void __launch_bounds__(kThreadsB, 1)
 #pragma unroll
                 for (int kk = 0; kk < DV / 16; ++kk) {
                     const uint32_t off = ((kk >> 2) * (kTile * 128) + (kk & 3) * 32) >> 4;
-                    const uint32_t offS = ((kk >> 2) * (160 * 128) + (kk & 3) * 32) >> 4;
+                    const uint32_t offS = (kk * 1024) >> 4;        // sixteen value columns = sixteen 64-byte rows of every block
                     if (kk == 0)
-                        mma_ss_lh<false>(tb, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW), desc_lo(dSt) + (aSt >> 4) + offS,
-                                         desc_hi(dSt), iT);
+                        mma_ss_lh<false>(tb, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW), desc_lo(dStN) + (aSt >> 4) + offS,
+                                         desc_hi(dStN), iT);
                     else
-                        mma_ss_lh<true>(tb, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW), desc_lo(dSt) + (aSt >> 4) + offS,
-                                        desc_hi(dSt), iT);
+                        mma_ss_lh<true>(tb, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW), desc_lo(dStN) + (aSt >> 4) + offS,
+                                        desc_hi(dStN), iT);
                 }
                 mma_commit(&bars[bX0]);
                 if (MODE == kModeDkDv) {
-                    // dV = mono(K) (tensor memory, written by the row threads) x state (MN-major, 160 = 10 K-steps)
+                    // dV = mono(K) (tensor memory, written by the row threads) x state (K-major: 64-byte rows of 32
+                    // features, 160 = 10 K-steps of 32 bytes)
                     if (ok) ok = mbar_wait(&bars[bX1], 0, abort_flag);
                     tc_fence_after();
                     if (ok) {
 #pragma unroll
                         for (int k = 0; k < 10; ++k) {
+                            const uint32_t offK = ((k >> 1) * C::kStateBlk + (k & 1) * 32) >> 4;
                             if (k == 0)
-                                mma_ts_lh<false>(tb + C::colAcc, tb + k * 8, desc_lo(dSt) + ((aSt + k * 2048) >> 4),
-                                                 desc_hi(dSt), iNV);
+                                mma_ts_lh<false>(tb + C::colAcc, tb + k * 8, desc_lo(dN) + (aSt >> 4) + offK, desc_hi(dN), iXV);
                             else
-                                mma_ts_lh<true>(tb + C::colAcc, tb + k * 8, desc_lo(dSt) + ((aSt + k * 2048) >> 4),
-                                                desc_hi(dSt), iNV);
+                                mma_ts_lh<true>(tb + C::colAcc, tb + k * 8, desc_lo(dN) + (aSt >> 4) + offK, desc_hi(dN), iXV);
                         }
                     }
                 } else {
@@ -664,8 +666,9 @@ bool make_rows_map_bf16(CUtensorMap* m, const void* base, int BH, int L, int wid
 
 namespace {
 // Block-wise path, between the passes.  state_scan_kernel: the per-block states of
-// generic_state_tc_kernel<.., true> summed over the blocks before (suffix = 0) or after (suffix = 1) each
-// block, as bf16 [BH x nblk][160][dvw] (tensor-core operand) and fp32 row sums [BH x nblk][160].
+// block_state_tc_kernel summed over the blocks before (suffix = 0) or after (suffix = 1) each
+// block, as bf16 [BH x nblk][dvw][160] (tensor-core operand, transposed as the state kernel holds it) and fp32 row
+// sums [BH x nblk][160].
 __global__ void __launch_bounds__(256)
     state_scan_kernel(const float* __restrict__ part, const float* __restrict__ zpart, __nv_bfloat16* __restrict__ st,
                       float* __restrict__ sv, int nblk, int per, int suffix) {
@@ -688,25 +691,6 @@ __global__ void __launch_bounds__(256)
         }
     }
 }
-// scaled_dout_kernel: dout_i / D_i as bf16 (the value operand of the query-side states), eight columns per thread
-__global__ void __launch_bounds__(256)
-    scaled_dout_kernel(const uint4* __restrict__ g, const float2* __restrict__ stats, uint4* __restrict__ ga, size_t n8,
-                       int dv8) {
-    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
-    if (i >= n8) return;
-    const float dinv = stats[i / dv8].x;
-    const uint4 u = g[i];
-    uint4 o;
-    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
-    uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        const float2 f = __bfloat1622float2(h[c]);
-        ow[c] = pack_bf16x2(f.x * dinv, f.y * dinv);
-    }
-    ga[i] = o;
-}
-
 template <int DV, int MODE, int LT, bool XB = false>
 based_status launch_pass(const CUtensorMap& n0, const CUtensorMap& w0, const CUtensorMap& n1, const CUtensorMap& w1,
                          const BParams& p, dim3 grid, const char* what, cudaStream_t stream,
@@ -740,7 +724,7 @@ int backward_block_len(int L, int df, bool merged, int d_v) {
 }
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 struct BlockWs {
-    float* sv; float* zpart; float* part; __nv_bfloat16* st; __nv_bfloat16* ga;
+    float* sv; float* zpart; float* part; __nv_bfloat16* st;
     size_t bytes;
 };
 // scratch after the [BH, L] float2 statistics
@@ -752,7 +736,6 @@ BlockWs block_ws(float* ws, int BH, int L, int dvr, int nblk) {
     w.zpart = reinterpret_cast<float*>(base + off);  off = align256(off + (size_t)BH * nblk * 160 * 4);
     w.part = reinterpret_cast<float*>(base + off);   off = align256(off + (size_t)BH * nblk * 160 * dvr * 4);
     w.st = reinterpret_cast<__nv_bfloat16*>(base + off);  off = align256(off + (size_t)BH * nblk * 160 * dvr * 2);
-    w.ga = reinterpret_cast<__nv_bfloat16*>(base + off);  off = align256(off + (size_t)BH * L * dvr * 2);
     w.bytes = off;
     return w;
 }
@@ -794,29 +777,28 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
         const int nblk = (L + W - 1) / W;
         const BlockWs w = block_ws(ws, BH, L, dvr, nblk);
         CUtensorMap tst;
-        if (!make_map_b(&tst, w.st, BH * nblk, 160, dvr, 64, 160, s128)) return BASED_ERR_CUDA;
+        // the block states lie transposed, [BH x nblk][d_v][160]: boxes of 32 features x all value columns
+        if (!make_map_b(&tst, w.st, BH * nblk, dvr, 160, 32, 64 * BCfg<DV, kModeDkDv, LTK>::kVB, s64)) return BASED_ERR_CUDA;
         p.W = W;
         p.nblk = nblk;
         p.sv = w.sv;
+        // With many heads one CTA per head walks the blocks and writes the running sums; with few, one CTA per head
+        // and block writes the block's own sums and a scan adds them up.
+        const bool running = BH >= 64;
+        auto states = [&](const void* x, const void* val, const void* sts, int rev) -> based_status {
+            if (running) return launch_block_states_tc(x, val, sts, w.st, w.sv, nullptr, nullptr, BH, L, W, dvr, rev, stream);
+            based_status s2 = launch_block_states_tc(x, val, sts, w.st, w.sv, w.part, w.zpart, BH, L, W, dvr, rev, stream);
+            if (s2 != BASED_OK) return s2;
+            state_scan_kernel<<<dim3((160 * dvr + 255) / 256, BH), 256, 0, stream>>>(w.part, w.zpart, w.st, w.sv, nblk, 160 * dvr, rev);
+            note_launch();
+            return check_launch("state_scan_kernel");
+        };
         // states of the keys: S = sum mono(k) v^T, z = sum mono(k), summed over the blocks before each block
-        st = launch_state_blocks_tc(k, v, nullptr, 0, w.part, w.zpart, BH, L, W, dvr, stream);
-        if (st != BASED_OK) return st;
-        state_scan_kernel<<<dim3((160 * dvr + 255) / 256, BH), 256, 0, stream>>>(w.part, w.zpart, w.st, w.sv, nblk, 160 * dvr, 0);
-        note_launch();
-        if ((st = check_launch("state_scan_kernel")) != BASED_OK) return st;
+        if ((st = states(k, v, nullptr, 0)) != BASED_OK) return st;
         st = launch_pass<DV, kModeDqS, 64, true>(tq, tg, tk64, tv64, p, grid, "backward_tc_kernel<stats+dq, blocks>", stream, &tst);
         if (st != BASED_OK) return st;
         // states of the queries: R = sum mono(q) (dout / D)^T, R_b = sum b mono(q), summed over the blocks after each block
-        const size_t n8 = (size_t)BH * L * dvr / 8;
-        scaled_dout_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, stream>>>(
-            static_cast<const uint4*>(g), stats, reinterpret_cast<uint4*>(w.ga), n8, dvr / 8);
-        note_launch();
-        if ((st = check_launch("scaled_dout_kernel")) != BASED_OK) return st;
-        st = launch_state_blocks_tc(q, w.ga, reinterpret_cast<const float*>(stats) + 1, 2, w.part, w.zpart, BH, L, W, dvr, stream);
-        if (st != BASED_OK) return st;
-        state_scan_kernel<<<dim3((160 * dvr + 255) / 256, BH), 256, 0, stream>>>(w.part, w.zpart, w.st, w.sv, nblk, 160 * dvr, 1);
-        note_launch();
-        if ((st = check_launch("state_scan_kernel")) != BASED_OK) return st;
+        if ((st = states(q, g, stats, 1)) != BASED_OK) return st;
         return launch_pass<DV, kModeDkDv, LTK, true>(tk, tv, tqL, tgL, p, grid, "backward_tc_kernel<dkdv, blocks>", stream, &tst);
     }
     if (out != nullptr || numerator_only) {
@@ -862,7 +844,7 @@ based_status launch_quadratic_forward_tc(const void* q, const void* k, const voi
 
 size_t backward_tc_workspace_bytes(int BH, int L, int d_v) {
     const int W = backward_block_len(L, 16, true, d_v);
-    if (W > 0) return block_ws(nullptr, BH, L, d_v, (L + W - 1) / W).bytes;         // statistics, block states, dout / D
+    if (W > 0) return block_ws(nullptr, BH, L, d_v, (L + W - 1) / W).bytes;         // statistics, block states
     return (size_t)BH * L * 2 * sizeof(float);                 // (1 / D, b) per row
 }
 

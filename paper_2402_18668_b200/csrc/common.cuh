@@ -106,10 +106,13 @@ based_status launch_prefill_generic(const void* q, const void* k, const void* v,
 // the final state of those feature dimensions on tensor cores (bf16 io); cont: add to the state given
 based_status launch_state_generic_tc(const void* k, const void* v, float* kv, float* z, int BH, int L, int d_feat,
                                      int d_v, int cont, cudaStream_t stream);
-// per-block states of the backward pass (d' = 16, bf16): [BH x nblk][160][d_v] and [BH x nblk][160] over blocks of W
-// tokens in the monomial basis; x = k or q, val = v or dout / D; wts: token weights of the row sums (null: ones)
-based_status launch_state_blocks_tc(const void* x, const void* val, const float* wts, int wstride, float* kv, float* z,
-                                    int BH, int L, int W, int d_v, cudaStream_t stream);
+// block_state_tc.cu: block states of the block-wise backward pass (d' = 16, bf16), transposed: st [BH x nblk][d_v][160]
+// bf16 and sv [BH x nblk][160]: for every block of W tokens the sums over the blocks before it (rev = 0) or after it
+// (rev = 1), one CTA per head; stats: (1 / D, b) per
+// token for the query side (x = q, val = dout), null for the key side (x = k, val = v); part, zpart: null, or the
+// blocks' own sums in fp32 instead (one CTA per head and block), for state_scan_kernel
+based_status launch_block_states_tc(const void* x, const void* val, const void* stats, void* st, float* sv, float* part,
+                                    float* zpart, int BH, int L, int W, int d_v, int rev, cudaStream_t stream);
 // the state of a token block alone (no outputs): kv (+)= sum_j phi(k_j) v_j^T, z (+)= sum_j phi(k_j)
 based_status launch_state_generic(const void* k, const void* v, float* kv, float* z, int BH, int L, int d_feat, int d_v,
                                   based_dtype io, int cont, cudaStream_t stream);

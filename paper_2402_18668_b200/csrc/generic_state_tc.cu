@@ -45,8 +45,8 @@ template <int DV> struct SCfg {
     static constexpr uint32_t kStage = kVBytes + kKBytes;
     static constexpr uint32_t kABytes = kFB * 128;             // [128 features][64 tokens] bf16
     static constexpr uint32_t offA = kNS * kStage;
-    static constexpr uint32_t offOnes = offA + kNA * kABytes;    // per A buffer: [16][64] bf16 token weights (ones: the row sums)
-    static constexpr uint32_t offKT = offOnes + kNA * 2048;    // two transposed k tiles [34][kKT] bf16
+    static constexpr uint32_t offOnes = offA + kNA * kABytes;    // [16][64] bf16 ones (B operand of the row sums)
+    static constexpr uint32_t offKT = offOnes + 2048;          // two transposed k tiles [34][kKT] bf16
     static constexpr uint32_t kKTBytes = 34 * kKT * 2;
     static constexpr uint32_t offMisc = offKT + 2 * kKTBytes + 64;
     static constexpr uint32_t kSmem = ((offMisc + 1023) / 1024) * 1024 + 256 + 1024;
@@ -61,9 +61,6 @@ struct SParams {
     unsigned int* err;
     int L, df, D, dvw, cont;
     float lin, quad;
-    // block mode: one state per block of W tokens, weighted row sums
-    const float* wts;              // weight of token t of head h at wts[(h * L + t) * wstride], or null (ones)
-    int wstride, W, nblk;
 };
 
 // AND of a predicate over the 128 row threads (named barrier 2); also a barrier for their shared-memory traffic
@@ -81,13 +78,7 @@ __device__ __forceinline__ bool rows_and(bool pred) {
 }
 }  // namespace
 
-// BLK: the states of the backward pass (d' = 16).  One CTA per (feature block, head x token block):
-// the sums run over the W tokens of the block; the features are the 153 distinct monomials of the
-// map (x_f | x_m x_(m+o) for o < 8 | x_m x_(m+8) for m < 8 | 1, padded to 160) and each sum is
-// scaled by the monomial's weight in phi(q) . phi(k) (1/4, 1/32 on the diagonal, 1/16, 1), so that a
-// reader contracts it with plain monomials; the row sum is weighted per token (two bf16 columns,
-// high and low part of the fp32 weight).
-template <int DV, bool BLK>
+template <int DV>
 __global__ void __launch_bounds__(kThreadsS, 1)
     generic_state_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                             const SParams p) {
@@ -99,11 +90,9 @@ __global__ void __launch_bounds__(kThreadsS, 1)
     volatile uint32_t* abort_flag = tmem_base_s + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int slot = blockIdx.y;                             // output state
-    const int head = BLK ? slot / p.nblk : slot;
-    const int t0 = BLK ? (slot % p.nblk) * p.W : 0;          // first token
+    const int head = blockIdx.y;
     const int f0 = blockIdx.x * kFB;
-    const int nit = ((BLK ? min(p.L, t0 + p.W) : p.L) - t0 + kTB - 1) / kTB;
+    const int nit = (p.L + kTB - 1) / kTB;
 
     if (tid == 0) {
         for (int s = 0; s < C::kNS; ++s) mbar_init(&bars[sFull0 + s], 1);
@@ -115,7 +104,7 @@ __global__ void __launch_bounds__(kThreadsS, 1)
     // constants in shared memory: the ones block, the zero rows of both transposed tiles
     {
         __nv_bfloat16* ones = reinterpret_cast<__nv_bfloat16*>(smem + C::offOnes);
-        for (int i = tid; i < kNA * 1024; i += kThreadsS) ones[i] = __float2bfloat16(BLK ? 0.0f : 1.0f);
+        for (int i = tid; i < 1024; i += kThreadsS) ones[i] = __float2bfloat16(1.0f);
         for (int i = tid; i < 2 * kKT; i += kThreadsS) {
             __nv_bfloat16* kt = reinterpret_cast<__nv_bfloat16*>(smem + C::offKT + (i / kKT) * C::kKTBytes);
             kt[kRowZero * kKT + (i % kKT)] = __float2bfloat16(0.0f);
@@ -135,15 +124,15 @@ __global__ void __launch_bounds__(kThreadsS, 1)
             constexpr uint64_t dV = make_smem_desc_base(kTB * 128, 1024, kSwizzle128B);       // MN-major, 64-column blocks
             constexpr uint32_t iV = make_idesc_bf16(128, 64 * C::kVB, 0, 1);
             constexpr uint32_t iZ = make_idesc_bf16(128, 16, 0, 0);
-            const uint32_t aOnes0 = smem_u32(smem + C::offOnes);
+            const uint32_t aOnes = smem_u32(smem + C::offOnes);
             auto load = [&](int it) {
                 const int s = it % C::kNS;
                 uint8_t* st = smem + s * C::kStage;
                 mbar_arrive_expect_tx(&bars[sFull0 + s], C::kStage);
 #pragma unroll
                 for (int b = 0; b < C::kVB; ++b)
-                    tma_load_3d(st + b * (kTB * 128), &tm_v, &bars[sFull0 + s], b * 64, t0 + it * kTB, head);
-                tma_load_3d(st + C::kVBytes, &tm_k, &bars[sFull0 + s], 0, t0 + it * kTB, head);
+                    tma_load_3d(st + b * (kTB * 128), &tm_v, &bars[sFull0 + s], b * 64, it * kTB, head);
+                tma_load_3d(st + C::kVBytes, &tm_k, &bars[sFull0 + s], 0, it * kTB, head);
             };
             for (int it = 0; it < C::kNS && it < nit; ++it) load(it);
             for (int it = 0; it < nit && ok; ++it) {
@@ -154,7 +143,6 @@ __global__ void __launch_bounds__(kThreadsS, 1)
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t aA = smem_u32(smem + C::offA + b * C::kABytes), aV = smem_u32(smem + s * C::kStage);
-                const uint32_t aOnes = aOnes0 + b * 2048;
 #pragma unroll
                 for (int kk = 0; kk < kTB / 16; ++kk) {
                     if (it == 0 && kk == 0) {
@@ -186,16 +174,9 @@ __global__ void __launch_bounds__(kThreadsS, 1)
         // the row's factors as rows of the transposed k tile: k_m k_n, k_m x 1, 1 x 1, or 0 past the last row
         int m = kRowZero, n = kRowZero;
         float scale = 0.f;
-        if (BLK) {
-            if (f < 16) { m = f; n = kRowOne; scale = 0.25f; }
-            else if (f < 144) { m = (f - 16) & 15; n = (m + ((f - 16) >> 4)) & 15; scale = f < 32 ? 0.03125f : 0.0625f; }
-            else if (f < 152) { m = f - 144; n = m + 8; scale = 0.0625f; }
-            else if (f == 152) { m = kRowOne; n = kRowOne; scale = 1.0f; }
-        } else {
-            if (f == 0) { m = kRowOne; n = kRowOne; scale = 1.0f; }
-            else if (f <= p.df) { m = f - 1; n = kRowOne; scale = p.lin; }
-            else if (f < p.D) { m = (f - 1 - p.df) / p.df; n = (f - 1 - p.df) % p.df; scale = p.quad; }
-        }
+        if (f == 0) { m = kRowOne; n = kRowOne; scale = 1.0f; }
+        else if (f <= p.df) { m = f - 1; n = kRowOne; scale = p.lin; }
+        else if (f < p.D) { m = (f - 1 - p.df) / p.df; n = (f - 1 - p.df) % p.df; scale = p.quad; }
         uint8_t* a_row0 = smem + C::offA + t * 128;
         for (int it = 0; it < nit && ok; ++it) {
             const int b = it % kNA, s = it % C::kNS;
@@ -216,7 +197,7 @@ __global__ void __launch_bounds__(kThreadsS, 1)
 #pragma unroll
                     for (int i = 0; i < 8; ++i) kt[(c * 8 + i) * kKT + j] = e[i];
                 }
-                if (t < kTB) kt[kRowOne * kKT + t] = __float2bfloat16(t0 + it * kTB + t < p.L ? 1.0f : 0.0f);
+                if (t < kTB) kt[kRowOne * kKT + t] = __float2bfloat16(it * kTB + t < p.L ? 1.0f : 0.0f);
             }
             // the A buffer is free once the products of kNA steps ago are done; the barrier also publishes the transpose
             ok = rows_and(it < kNA || mbar_wait(&bars[sMma0 + b], ((it / kNA) - 1) & 1, abort_flag));
@@ -237,15 +218,6 @@ __global__ void __launch_bounds__(kThreadsS, 1)
                 for (int i = 0; i < 4; ++i) hp[i] = __hmul2(hm[i], hn[i]);
                 *reinterpret_cast<uint4*>(a_row + ((c ^ (t & 7)) << 4)) = pr;
             }
-            if (BLK && t < kTB) {
-                // this step's token weights: rows 0 (high part) and 1 (low part) of the K-major SWIZZLE_128B block
-                const int tok = t0 + it * kTB + t;
-                const float wv = tok < p.L ? (p.wts ? p.wts[((size_t)head * p.L + tok) * p.wstride] : 1.0f) : 0.0f;
-                const __nv_bfloat16 hi = __float2bfloat16(wv), lo = __float2bfloat16(wv - __bfloat162float(hi));
-                uint8_t* wb = smem + C::offOnes + b * 2048;
-                *reinterpret_cast<__nv_bfloat16*>(wb + ((t >> 3) << 4) + (t & 7) * 2) = hi;
-                *reinterpret_cast<__nv_bfloat16*>(wb + 128 + (((t >> 3) ^ 1) << 4) + (t & 7) * 2) = lo;
-            }
             fence_proxy_async_smem();
             mbar_arrive(&bars[sAlu0 + b]);
         }
@@ -254,7 +226,7 @@ __global__ void __launch_bounds__(kThreadsS, 1)
         if (ok) {                                            // uniform over the row threads
             const uint32_t lane_base = (uint32_t)warp * 32u;
             const bool store = f < p.D;
-            const size_t row = (size_t)slot * p.D + (store ? f : 0);
+            const size_t row = (size_t)head * p.D + (store ? f : 0);
             float* dst = p.kv + row * p.dvw;
             for (int c = 0; c < p.dvw / 16; ++c) {           // p.dvw is uniform: the loads stay warp-collective
                 uint32_t r[16];
@@ -274,11 +246,10 @@ __global__ void __launch_bounds__(kThreadsS, 1)
                     }
                 }
             }
-            uint32_t zr, zl = 0u;
+            uint32_t zr;
             tmem_ld1(tmem_addr(tb, lane_base, C::colZ), zr);
-            if (BLK) tmem_ld1(tmem_addr(tb, lane_base, C::colZ + 1), zl);
             tmem_wait_ld();
-            if (store) p.z[row] = (__uint_as_float(zr) + __uint_as_float(zl)) * scale + (p.cont ? p.z[row] : 0.f);
+            if (store) p.z[row] = __uint_as_float(zr) * scale + (p.cont ? p.z[row] : 0.f);
         }
     }
     if (!ok && lane == 0) atomicOr(p.err, 1u);
@@ -292,11 +263,9 @@ __global__ void __launch_bounds__(kThreadsS, 1)
 }
 
 namespace {
-// blocks: 0 for one state per head over the whole sequence; else the block length W (a multiple of 64):
-// the per-block states of the backward pass, [BH x nblk][160][dvw] and [BH x nblk][160]
-template <int DV, bool BLK>
+template <int DV>
 based_status launch_state_dv(const void* k, const void* v, float* kv, float* z, int BH, int L, int df, int dvw,
-                             int cont, const float* wts, int wstride, int W, cudaStream_t stream) {
+                             int cont, cudaStream_t stream) {
     using C = SCfg<DV>;
     CUtensorMap tk, tv;
     if (!make_rows_map_bf16(&tk, k, BH, L, df, 32, kTB, CU_TENSOR_MAP_SWIZZLE_64B) ||
@@ -308,13 +277,9 @@ based_status launch_state_dv(const void* k, const void* v, float* kv, float* z, 
     p.z = z;
     p.L = L;
     p.df = df;
-    p.D = BLK ? 160 : 1 + df + df * df;
+    p.D = 1 + df + df * df;
     p.dvw = dvw;
     p.cont = cont;
-    p.wts = wts;
-    p.wstride = wstride;
-    p.W = W;
-    p.nblk = BLK ? (L + W - 1) / W : 1;
     const float rd = sqrtf((float)df);
     p.lin = 1.0f / sqrtf(rd);
     p.quad = 1.0f / (1.41421356237309505f * rd);
@@ -324,29 +289,22 @@ based_status launch_state_dv(const void* k, const void* v, float* kv, float* z, 
     {
         std::lock_guard<std::mutex> lock(setup_mutex());
         if (!configured[dev]) {
-            if (cudaFuncSetAttribute(generic_state_tc_kernel<DV, BLK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            if (cudaFuncSetAttribute(generic_state_tc_kernel<DV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)C::kSmem) != cudaSuccess)
                 return BASED_ERR_CUDA;
             configured[dev] = true;
         }
     }
-    generic_state_tc_kernel<DV, BLK><<<dim3((p.D + kFB - 1) / kFB, BH * p.nblk), kThreadsS, C::kSmem, stream>>>(tk, tv, p);
+    generic_state_tc_kernel<DV><<<dim3((p.D + kFB - 1) / kFB, BH), kThreadsS, C::kSmem, stream>>>(tk, tv, p);
     note_launch();
-    return check_launch(BLK ? "generic_state_tc_kernel<blocks>" : "generic_state_tc_kernel");
+    return check_launch("generic_state_tc_kernel");
 }
 }  // namespace
 
 based_status launch_state_generic_tc(const void* k, const void* v, float* kv, float* z, int BH, int L, int d_feat,
                                      int d_v, int cont, cudaStream_t stream) {
-    if (d_v == 64) return launch_state_dv<64, false>(k, v, kv, z, BH, L, d_feat, 64, cont, nullptr, 0, 0, stream);
-    return launch_state_dv<128, false>(k, v, kv, z, BH, L, d_feat, d_v, cont, nullptr, 0, 0, stream);   // 112 or 128
-}
-
-// per-block states of the backward pass (d' = 16): x = k or q, val = v or dout / D, weights of the row sums
-based_status launch_state_blocks_tc(const void* x, const void* val, const float* wts, int wstride, float* kv, float* z,
-                                    int BH, int L, int W, int d_v, cudaStream_t stream) {
-    if (d_v == 64) return launch_state_dv<64, true>(x, val, kv, z, BH, L, 16, 64, 0, wts, wstride, W, stream);
-    return launch_state_dv<128, true>(x, val, kv, z, BH, L, 16, d_v, 0, wts, wstride, W, stream);
+    if (d_v == 64) return launch_state_dv<64>(k, v, kv, z, BH, L, d_feat, 64, cont, stream);
+    return launch_state_dv<128>(k, v, kv, z, BH, L, d_feat, d_v, cont, stream);        // 112 or 128
 }
 
 }  // namespace based

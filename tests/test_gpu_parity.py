@@ -310,7 +310,7 @@ def test_prefill_backward_cfg3_sampled_heads(with_out):
     n0 = based.launch_count()
     dq, dk, dv = based.based_prefill_backward(q, k, v, dout, out=out)
     _poll()
-    assert based.launch_count() - n0 == (7 if with_out else 3)
+    assert based.launch_count() - n0 == (4 if with_out else 3)     # block-wise: two state walks, two tile passes
     b, h = w.B - 1, 5
     sl = (slice(b, b + 1), slice(h, h + 1))
     rq, rk, rv = oracle.linattn_backward(_np(q[sl]), _np(k[sl]), _np(v[sl]), _np(dout[sl]))
@@ -334,13 +334,39 @@ def test_prefill_backward_blockwise(L, d_v, flags):
     n0 = based.launch_count()
     dq, dk, dv = based.based_prefill_backward(qd, kd, vd, gd, flags=flags, out=out)
     _poll()
-    assert based.launch_count() - n0 == 7                   # two state passes with their sums, dout / D, two tile passes
+    assert based.launch_count() - n0 == 6                   # few heads: two state passes with their scans, two tile passes
     assert _grad_err(_np(dq), rq) <= TOL_BF16 and _grad_err(_np(dk), rk) <= TOL_BF16 and _grad_err(_np(dv), rv) <= TOL_BF16
     # row by row as well, away from the first rows (whose gradients nearly vanish): the blocks' seams show here
     for got, want in ((dq, rq), (dk, rk), (dv, rv)):
         gm, wm = _np(got)[:, :, 64:].astype(np.float64), want[:, :, 64:]
         rows = np.abs(gm - wm).max(axis=-1) / np.maximum(np.abs(wm).max(axis=-1), 0.05 * np.abs(wm).max())
         assert rows.max() <= TOL_BF16
+
+
+@pytest.mark.parametrize("L,d_v,flags", [(1700, 64, 0), (2304, 128, 0), (2100, 112, 4)])
+def test_prefill_backward_blockwise_running_states(L, d_v, flags):
+    """The same with 64 heads, where one CTA per head walks the blocks and writes the running sums (four launches):
+    three heads against the oracle."""
+    B, H = 8, 8
+    g_ = torch.Generator(device=DEV).manual_seed(L + d_v)
+    q = (torch.randn(B, H, L, 16, generator=g_, device=DEV) * 0.5).bfloat16()
+    k = (torch.randn(B, H, L, 16, generator=g_, device=DEV) * 0.5).bfloat16()
+    v = torch.randn(B, H, L, d_v, generator=g_, device=DEV).bfloat16()
+    dout = torch.randn(B, H, L, d_v, generator=g_, device=DEV).bfloat16()
+    out = based.based_prefill(q, k, v, flags=flags)
+    n0 = based.launch_count()
+    dq, dk, dv = based.based_prefill_backward(q, k, v, dout, flags=flags, out=out)
+    _poll()
+    assert based.launch_count() - n0 == 4
+    for (b, h) in [(0, 0), (3, 5), (B - 1, H - 1)]:
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        rq, rk, rv = oracle.linattn_backward(_np(q[sl]), _np(k[sl]), _np(v[sl]), _np(dout[sl]), numerator_only=bool(flags))
+        assert _grad_err(_np(dq[sl]), rq) <= TOL_BF16 and _grad_err(_np(dk[sl]), rk) <= TOL_BF16
+        assert _grad_err(_np(dv[sl]), rv) <= TOL_BF16
+        for got, want in ((dq[sl], rq), (dk[sl], rk), (dv[sl], rv)):
+            gm, wm = _np(got)[:, :, 64:].astype(np.float64), want[:, :, 64:]
+            rows = np.abs(gm - wm).max(axis=-1) / np.maximum(np.abs(wm).max(axis=-1), 0.05 * np.abs(wm).max())
+            assert rows.max() <= TOL_BF16
 
 
 def test_prefill_backward_blockwise_many_blocks_against_tile_path():
