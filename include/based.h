@@ -228,10 +228,10 @@ size_t based_prefill_backward_workspace_bytes(int B, int H, int L, int d_v, base
  * only: D_i and dout_i . N_i are still recomputed in fp32.  fp32 io ignores out's values.
  * out must not alias a gradient output.
  *
- * Block-wise path (bf16 io, d_feat = 16; L >= 1536 at d_v 64, L >= 2048 at d_v 112 / 128): O(L) per
+ * Block-wise path (bf16 io, d_feat = 16; L >= 768 at d_v 64, L >= 1024 to 1536 at d_v 112 / 128): O(L) per
  * head, the recurrent view of Sec. 4.1 applied to the gradients.  The sequence is cut into blocks of
- * W = 256 (d_v 64) or 512 tokens.  Pairs inside a block go through the tiles above.  All earlier
- * blocks reach a query through their summed state S = sum_j phi(k_j) v_j^T, z = sum_j phi(k_j):
+ * W = 256 tokens (512 for long sequences of few heads at d_v 128).  Pairs inside a block go through
+ * the tiles above.  All earlier blocks reach a query through their summed state S = sum_j phi(k_j) v_j^T, z = sum_j phi(k_j):
  *   sum_j w'_ij (dout_i.v_j - m_i) k_j = J(q_i)^T (S dout_i - m_i z),   D_i += phi(q_i) . z
  * (J the Jacobian of phi), and all later blocks reach a key through R = sum_i phi(q_i) (dout_i / D_i)^T
  * and R_b = sum_i b_i phi(q_i):  dk_j += J(k_j)^T (R v_j + R_b),  dv_j += R^T phi(k_j).

@@ -715,12 +715,15 @@ based_status launch_pass(const CUtensorMap& n0, const CUtensorMap& w0, const CUt
 
 // Block length of the block-wise path, or 0 for the tile path alone.  The block-wise path needs d' = 16 and the
 // statistics in one sweep (the forward output, or the numerator-only form); its cost grows with L where the tile
-// path's grows with L^2, and the lengths below are where it starts to win on B200 (d_v 64: 274 against 317 us at
-// L = 1536 for 128 heads; d_v 128: 508 against 616 us at L = 2048).
-int backward_block_len(int L, int df, bool merged, int d_v) {
+// path's grows with L^2, and the lengths below are where it starts to win on B200 (128 heads, d_v 64: 101 against
+// 117 us at L = 768; d_v 128: 191 against 213 us at L = 1024; 32 heads, d_v 128: 129 against 134 us at L = 1536).
+// Blocks of 256 tokens are the fastest from there on (B8 H16 L4096 d_v128: 720 / 687 / 737 us at 128 / 256 / 512),
+// except with few heads at d_v 128, where every block's state costs a CTA of its own.
+int backward_block_len(int L, int df, bool merged, int d_v, int BH) {
     if (df != 16 || !merged) return 0;
-    if (d_v == 64) return L >= 1536 ? 256 : 0;
-    return L >= 2048 ? 512 : 0;
+    if (d_v == 64) return L >= 768 ? 256 : 0;
+    if (BH >= 64) return L >= 1024 ? 256 : 0;
+    return L >= 4096 ? 512 : L >= 1536 ? 256 : 0;
 }
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 struct BlockWs {
@@ -771,7 +774,7 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
     p.s2 = 0.5f / (float)df;
     const dim3 grid((L + kTile - 1) / kTile, BH);
     based_status st;
-    const int W = backward_block_len(L, df, out != nullptr || numerator_only, dvr);
+    const int W = backward_block_len(L, df, out != nullptr || numerator_only, dvr, BH);
     if (W > 0) {
         // block-wise: pairs inside a block of W tokens by tiles, everything else through summed block states
         const int nblk = (L + W - 1) / W;
@@ -843,7 +846,7 @@ based_status launch_quadratic_forward_tc(const void* q, const void* k, const voi
 }
 
 size_t backward_tc_workspace_bytes(int BH, int L, int d_v) {
-    const int W = backward_block_len(L, 16, true, d_v);
+    const int W = backward_block_len(L, 16, true, d_v, BH);
     if (W > 0) return block_ws(nullptr, BH, L, d_v, (L + W - 1) / W).bytes;         // statistics, block states
     return (size_t)BH * L * 2 * sizeof(float);                 // (1 / D, b) per row
 }

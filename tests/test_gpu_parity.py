@@ -318,12 +318,12 @@ def test_prefill_backward_cfg3_sampled_heads(with_out):
     assert _grad_err(_np(dv[sl]), rv) <= TOL_BF16
 
 
-@pytest.mark.parametrize("L,d_v,flags", [(1536, 64, 0), (1700, 64, 0), (1601, 64, 4), (2125, 128, 0), (2100, 112, 0),
-                                          (2048, 128, 4)])
+@pytest.mark.parametrize("L,d_v,flags", [(768, 64, 0), (1536, 64, 0), (1700, 64, 0), (1601, 64, 4), (1536, 128, 0),
+                                          (2125, 128, 0), (2100, 112, 0), (2048, 128, 4), (4200, 128, 0)])
 def test_prefill_backward_blockwise(L, d_v, flags):
-    """The block-wise backward (bf16, d' = 16, forward output given, L from 1536 / 2048 up): pairs inside a block of
-    256 / 512 tokens by tiles, all others through summed block states; whole and ragged last blocks, both forms,
-    every gradient against the oracle."""
+    """The block-wise backward (bf16, d' = 16, forward output given, L from 768 / 1536 up at these head counts): pairs
+    inside a block of 256 (512 at the longest d_v 128 case) tokens by tiles, all others through summed block states;
+    whole and ragged last blocks, both forms, every gradient against the oracle."""
     B, H = 1, 2
     w = wl.Workload("bwdblk", B, H, L, 16, d_v, "bf16", 0.5)
     q, k, v = wl.prefill_inputs(w, wl.generator(4000 + L))
@@ -343,7 +343,7 @@ def test_prefill_backward_blockwise(L, d_v, flags):
         assert rows.max() <= TOL_BF16
 
 
-@pytest.mark.parametrize("L,d_v,flags", [(1700, 64, 0), (2304, 128, 0), (2100, 112, 4)])
+@pytest.mark.parametrize("L,d_v,flags", [(800, 64, 0), (1700, 64, 0), (1024, 128, 0), (2304, 128, 0), (2100, 112, 4)])
 def test_prefill_backward_blockwise_running_states(L, d_v, flags):
     """The same with 64 heads, where one CTA per head walks the blocks and writes the running sums (four launches):
     three heads against the oracle."""
