@@ -504,8 +504,9 @@ def bench_baseconv(shape, steps, warmup, torch, based, dist_on, peaks):
 
 
 def bench_backward(w, steps, warmup, torch, based, dist_on, peaks):
-    """Backward pass of the linear attention (quadratic form) on the workload's shape: bf16 io runs on
-    the tensor cores, fp32 io on the fp32 pipe (peak = SMs x 128 lanes x 2 flop x SM clock)."""
+    """Backward pass of the linear attention on the workload's shape: bf16 io runs on the tensor cores (block-wise
+    from a few blocks up, else the quadratic form), fp32 io on the fp32 pipe (peak = SMs x 128 lanes x 2 flop x SM
+    clock).  The flops counted are those of the form that ran."""
     g = torch.Generator(device="cuda").manual_seed(8)
     dt = w.torch_dtype
     q = (torch.randn(w.B, w.H, w.L, w.d_feat, generator=g, device="cuda") * w.qk_scale).to(dt)
@@ -522,13 +523,25 @@ def bench_backward(w, steps, warmup, torch, based, dist_on, peaks):
                      dist_on)
     assert based.based_poll_error() == 0
     t = ms * 1e-3 / steps
-    pairs = w.B * w.H * w.L * (w.L + 1) / 2.0
     # per pair: bf16 (statistics + dq merged): 2 score and 2 dout.v products, dv, X and Y of dq, dk = 80 + 3 d_v;
     # fp32: 3 score and 3 dout.v products, dv, dq, dk = 80 + 4 d_v
-    flops = 2.0 * pairs * (80 + (3 if bf16 else 4) * w.d_v)
+    per_pair = 2.0 * (80 + (3 if bf16 else 4) * w.d_v)
+    W = int(based.lib().based_prefill_backward_block_tokens(w.B, w.H, w.L, w.d_feat, w.d_v, 1 if bf16 else 0, 0, 1))
+    if W > 0:
+        # block-wise path: the pairs inside blocks of W tokens; per token the two state updates (153 monomials x
+        # (d_v + 2) columns each), the three read-outs (S dout, R v, R^T mono(k): 153 x d_v each) and the Jacobian
+        # contractions (about 8 flops per pair monomial, for queries and keys)
+        nfull, tail = divmod(w.L, W)
+        pairs = w.B * w.H * (nfull * W * (W + 1) / 2.0 + tail * (tail + 1) / 2.0)
+        flops = per_pair * pairs + w.B * w.H * w.L * (2.0 * 153 * (2 * (w.d_v + 2) + 3 * w.d_v) + 2 * 8 * 136 * 2)
+        form = f" backward given the forward output (tensor cores, block-wise: blocks of {W} tokens by tiles, the rest through block states)"
+    else:
+        pairs = w.B * w.H * w.L * (w.L + 1) / 2.0
+        flops = per_pair * pairs
+        form = " backward given the forward output (tensor cores, quadratic form, 2 passes)" if bf16 else " backward (fp32 FMA, quadratic form)"
     peak = peaks["bf16_tflops"] if bf16 else 148 * 128 * 2 * 1.965e9 / 1e12
     return {
-        "workload": w.name + (" backward given the forward output (tensor cores, quadratic form, 2 passes)" if bf16 else " backward (fp32 FMA, quadratic form)"),
+        "workload": w.name + form,
         "metric": "backward_tokens_per_s", "value": w.B * w.L / t, "unit": "tokens/s", "ms_per_step": t * 1e3,
         "steps": steps, "launches_per_step": (based.launch_count() - n0) // (steps + warmup),
         "roofline": {"bound": "tensor" if bf16 else "alu", "achieved": flops / t / 1e12, "peak": peak,

@@ -247,6 +247,15 @@ based_status based_prefill_backward_with_out(const void* q, const void* k, const
                                              size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Which path a backward call with these arguments takes: the block length W of the block-wise path, or 0
+ * for the tile path (fp32 io, d_feat other than 16, short sequences, or neither the forward output nor
+ * BASED_NUMERATOR_ONLY given).  with_out: nonzero for based_prefill_backward_with_out with out non-null.
+ * Host only; for callers that account the work of a call (benchmarks).
+ */
+int based_prefill_backward_block_tokens(int B, int H, int L, int d_feat, int d_v, based_dtype io, int flags,
+                                        int with_out);
+
+/*
  * The gated short convolution at the core of the BaseConv layer (App. "Extended Architecture
  * Details", paragraph "Convolution": y = ((u W1 + b1) (.) SiLU(h * (u W2) + b2)) W3 + b3).
  * The three projections are plain matrix products and stay with the caller; this call is the

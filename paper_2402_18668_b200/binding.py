@@ -28,7 +28,7 @@ EXPORTS = (
     "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step", "based_decode_step_sym",
     "based_state_to_sym", "based_state_from_sym", "swa_decode_step_at", "based_preload_decode",
     "baseconv_gate_forward", "baseconv_gate_step", "based_decode_step_flags", "based_prefill_backward",
-    "based_prefill_backward_workspace_bytes", "based_prefill_backward_with_out", "swa_decode_step_advance",
+    "based_prefill_backward_workspace_bytes", "based_prefill_backward_with_out", "based_prefill_backward_block_tokens", "swa_decode_step_advance",
     "based_prefill_state", "based_prefill_state_workspace_bytes",
 )
 
@@ -87,6 +87,8 @@ def lib() -> ctypes.CDLL:
         L.based_prefill_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
         L.based_prefill_backward_with_out.restype = i
         L.based_prefill_backward_with_out.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
+        L.based_prefill_backward_block_tokens.restype = i
+        L.based_prefill_backward_block_tokens.argtypes = [i, i, i, i, i, i, i, i]
         L.based_prefill_backward_workspace_bytes.restype = sz
         L.based_prefill_backward_workspace_bytes.argtypes = [i, i, i, i, i]
         L.baseconv_gate_forward.restype = i

@@ -312,6 +312,12 @@ size_t based_prefill_backward_workspace_bytes(int B, int H, int L, int d_v, base
     return (size_t)B * H * L * 2 * sizeof(float);
 }
 
+int based_prefill_backward_block_tokens(int B, int H, int L, int d_feat, int d_v, based_dtype io, int flags,
+                                        int with_out) {
+    if (B <= 0 || H <= 0 || L <= 0 || !dv_ok(d_v) || io != BASED_BF16) return 0;
+    return backward_tc_block_tokens(B * H, L, d_feat, d_v, (with_out || (flags & BASED_NUMERATOR_ONLY)) ? 1 : 0);
+}
+
 static based_status prefill_backward(const void* q, const void* k, const void* v, const void* out, const void* dout,
                                      void* dq, void* dk, void* dv, int B, int H, int L, int d_feat, int d_v,
                                      based_dtype io, int flags, void* workspace, size_t workspace_bytes,

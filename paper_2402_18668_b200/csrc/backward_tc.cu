@@ -845,6 +845,10 @@ based_status launch_quadratic_forward_tc(const void* q, const void* k, const voi
     return launch_pass<128, kModeFwd, 64>(tq, tq, tk64, tv64, p, grid, "quadratic forward (tc)", stream);
 }
 
+int backward_tc_block_tokens(int BH, int L, int d_feat, int d_v, int merged) {
+    return backward_block_len(L, d_feat, merged != 0, d_v, BH);
+}
+
 size_t backward_tc_workspace_bytes(int BH, int L, int d_v) {
     const int W = backward_block_len(L, 16, true, d_v, BH);
     if (W > 0) return block_ws(nullptr, BH, L, d_v, (L + W - 1) / W).bytes;         // statistics, block states

@@ -124,6 +124,9 @@ based_status launch_decode_generic(const void* q, const void* k, const void* v, 
                                    cudaStream_t stream);
 // the same on tensor cores (bf16 io); ws: backward_tc_workspace_bytes
 size_t backward_tc_workspace_bytes(int BH, int L, int d_v);
+// block length of the block-wise path for this shape, 0 where the tile path runs (merged: forward output given, or
+// the numerator-only form)
+int backward_tc_block_tokens(int BH, int L, int d_feat, int d_v, int merged);
 // out: the forward output (may be null): with it, statistics and dq run as one sweep
 based_status launch_prefill_backward_tc(const void* q, const void* k, const void* v, const void* out, const void* g,
                                         void* dq, void* dk, void* dv, float* ws, int BH, int L, int d_feat, int d_v,

@@ -160,6 +160,15 @@ def test_backward_validation(lib):
     ok = (1, 1, 8, 16, 64, 1)
     assert lib.based_prefill_backward_workspace_bytes(2, 3, 100, 64, 0) == 2 * 3 * 100 * 8
     assert lib.based_prefill_backward_workspace_bytes(2, 3, 100, 64, 1) == 2 * 3 * 100 * 8
+    # the block-wise path: bf16, d' = 16, statistics in one sweep, from a few blocks of 256 tokens up
+    assert lib.based_prefill_backward_block_tokens(4, 16, 2048, 16, 64, 1, 0, 1) == 256
+    assert lib.based_prefill_backward_block_tokens(4, 16, 2048, 16, 64, 1, 0, 0) == 0      # no forward output
+    assert lib.based_prefill_backward_block_tokens(4, 16, 2048, 16, 64, 1, 4, 0) == 256    # numerator only
+    assert lib.based_prefill_backward_block_tokens(4, 16, 2048, 16, 64, 0, 0, 1) == 0      # fp32 io
+    assert lib.based_prefill_backward_block_tokens(4, 16, 2048, 32, 64, 1, 0, 1) == 0      # other feature dimension
+    assert lib.based_prefill_backward_block_tokens(4, 16, 512, 16, 64, 1, 0, 1) == 0       # short
+    assert lib.based_prefill_backward_block_tokens(1, 8, 8192, 16, 128, 1, 0, 1) == 512    # few heads, long, d_v 128
+    assert lib.based_prefill_backward_workspace_bytes(4, 16, 2048, 64, 1) > 4 * 16 * 2048 * 8
     assert f(q, k, v, None, dq, dk, dv, *ok, 0, ws, 1 << 20, None) == 1            # output gradient missing
     assert f(q, k, v, g, dq, dk, dv, *ok, 1, ws, 1 << 20, None) == 1               # CONTINUE is not a backward flag
     assert f(q, k, v, g, q, dk, dv, *ok, 0, ws, 1 << 20, None) == 1                # gradient aliases an input
