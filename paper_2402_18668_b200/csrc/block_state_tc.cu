@@ -13,16 +13,18 @@
 // warps, two threads per token of the step (and per accumulator lane at the block ends), each with
 // half of the features; lane 0 of warp 8 issues TMA loads and MMAs.  Per step the row threads form
 // their token's 160 monomials times u_t in fp32, round once to bf16 and write them as a row of the B
-// operand ([128 tokens][160], MN-major,
-// five SWIZZLE_64B blocks of 32 features); the value tile comes by TMA and is the A operand as it
-// lies ([128 tokens][d_v], MN-major), so the accumulator in tensor memory is the transposed state,
-// [d_v lanes][160 columns] fp32.  The weights wt_t ride as two more rows of A (high and low bf16
-// part): lanes 64, 65 of the same accumulator at d_v 64, a second accumulator (M = 64) at d_v 112 /
-// 128.  At a block's end the issuer waits for the products so far, the row threads read the sums,
-// scale, round to bf16 and write the next block's state [160][d_v] through a transposing tile in
-// shared memory; the walk then adds on.  The operand tiles are double-buffered and the value tiles
-// come through a ring of three stages, so loads, row threads and tensor pipe overlap between block
-// ends.
+// operand ([128 tokens][160], MN-major, five SWIZZLE_64B blocks of 32 features); the value tile comes
+// by TMA and is the A operand as it lies ([128 tokens][d_v], MN-major), so the accumulator in tensor
+// memory is the transposed state, [d_v lanes][160 columns] fp32.  The weights wt_t ride as two more
+// rows of A (high and low bf16 part): lanes 64, 65 of the same accumulator at d_v 64, a second
+// accumulator (M = 64) at d_v 112 / 128.  Two accumulators alternate from block to block: while the
+// tensor pipe adds up the next block, the row threads read the finished one, add it to the running
+// sums they keep in registers, scale, round to bf16 and write their lane's row of the next block's
+// state, [d_v][160] - the layout the readers' descriptors take as it lies.  (The weights rows'
+// accumulator at d_v 128 is never started over: blocks alternate between two pairs of its lanes,
+// each pair a running sum of every second block.)  The operand tiles are double-buffered and the
+// value tiles come through a ring of three stages.  With few heads one CTA per (head, block) writes
+// the block's own sums in fp32 instead, for a scan by another kernel.
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -54,11 +56,12 @@ template <int DV> struct RCfg {
     static constexpr uint32_t offW = kNSR * kVBytes;
     static constexpr uint32_t offPhi = offW + 2 * kWBytes;
     static constexpr uint32_t offMisc = offPhi + 2 * kPhiBytes;
-    static constexpr uint32_t kSmem = offMisc + 2048 + 1024;   // barriers; the row sums' two parts (2 x 160 floats)
-    static constexpr uint32_t colS = 0, colZ = 160;            // second accumulator (weights rows) at d_v 128
-    static constexpr uint32_t kCols = DV == 64 ? 256 : 512;
+    static constexpr uint32_t kSmem = offMisc + 3072 + 1024;   // barriers; the row sums' parts (4 x 160 floats)
+    // two accumulators of 160 columns that alternate from block to block; at d_v 128 the weights rows' accumulator
+    static constexpr uint32_t colS = 0, colZ = 320;
+    static constexpr uint32_t kCols = 512;
 };
-enum { rFull0 = 0, rAlu0 = 3, rMma0 = 5, rFlush = 7, rFlushDone = 8, rNum = 9 };
+enum { rFull0 = 0, rAlu0 = 3, rMma0 = 5, rFlush0 = 7, rFree0 = 9, rNum = 11 };
 
 struct RParams {
     const __nv_bfloat16* x;        // [BH, L, 16] k or q
@@ -119,12 +122,12 @@ __global__ void __launch_bounds__(kThreadsR, 1)
     if (tid == 0) {
         for (int s = 0; s < kNSR; ++s) mbar_init(&bars[rFull0 + s], 1);
         for (int b = 0; b < 2; ++b) { mbar_init(&bars[rAlu0 + b], kRowThreads); mbar_init(&bars[rMma0 + b], 1); }
-        mbar_init(&bars[rFlush], 1);
-        mbar_init(&bars[rFlushDone], kRowThreads);
+        for (int a = 0; a < 2; ++a) { mbar_init(&bars[rFlush0 + a], 1); mbar_init(&bars[rFree0 + a], kRowThreads); }
         *abort_flag = 0;
         fence_mbar_init();
     }
-    // the weights blocks: only the first four bytes of a row are ever written again
+    for (int i = tid; i < 4 * 160; i += kThreadsR) reinterpret_cast<float*>(smem + C::offMisc + 256)[i] = 0.f;
+    // the weights blocks: only the first eight bytes of a row are ever written again
     for (int i = tid; i < 2 * (int)C::kWBytes / 16; i += kThreadsR)
         reinterpret_cast<uint4*>(smem + C::offW)[i] = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
@@ -150,14 +153,22 @@ __global__ void __launch_bounds__(kThreadsR, 1)
                     tma_load_3d(st + b * (kTok * 128), &tm_val, &bars[rFull0 + s], b * 64, tile_of(it) * kTok, head);
             };
             for (int it = 0; it < kNSR && it < nit; ++it) load(it);
-            int nflush = 0;
+            int nblk_done = 0;                               // blocks walked so far: the accumulators alternate
             for (int it = 0; it < nit && ok; ++it) {
                 const int b = it & 1, s = it % kNSR;
+                const int a = nblk_done & 1;
+                const bool first = it == 0 || ends_block(it - 1);        // first step of a block: the accumulator starts over
                 ok = mbar_wait(&bars[rFull0 + s], (it / kNSR) & 1, abort_flag);
                 if (!ok) break;
                 ok = mbar_wait(&bars[rAlu0 + b], (it >> 1) & 1, abort_flag);
                 if (!ok) break;
+                // the row threads have read this accumulator's sums of two blocks ago
+                if (first && nblk_done >= 2) {
+                    ok = mbar_wait(&bars[rFree0 + a], ((nblk_done >> 1) - 1) & 1, abort_flag);
+                    if (!ok) break;
+                }
                 tc_fence_after();
+                const uint32_t dS = tb + C::colS + a * 160;
                 const uint32_t aV = smem_u32(smem + C::offV + s * C::kVBytes);
                 const uint32_t aW = smem_u32(smem + C::offW + b * C::kWBytes);
                 const uint32_t lPhi = desc_lo(dPhi) + (smem_u32(smem + C::offPhi + b * kPhiBytes) >> 4);
@@ -167,32 +178,29 @@ __global__ void __launch_bounds__(kThreadsR, 1)
                     const uint32_t a_lo = desc_lo(dV1) + (aV >> 4), a_hi = desc_hi(dV1);
 #pragma unroll
                     for (int k = 0; k < kTok / 16; ++k) {
-                        if (it == 0 && k == 0)
-                            mma_ss_lh<false>(tb + C::colS, a_lo + k * 128, a_hi, lPhi + k * 64, desc_hi(dPhi), iS);
+                        if (first && k == 0)
+                            mma_ss_lh<false>(dS, a_lo + k * 128, a_hi, lPhi + k * 64, desc_hi(dPhi), iS);
                         else
-                            mma_ss_lh<true>(tb + C::colS, a_lo + k * 128, a_hi, lPhi + k * 64, desc_hi(dPhi), iS);
+                            mma_ss_lh<true>(dS, a_lo + k * 128, a_hi, lPhi + k * 64, desc_hi(dPhi), iS);
                     }
                 } else {
                     const uint32_t a_lo = desc_lo(dV) + (aV >> 4), w_lo = desc_lo(dV) + (aW >> 4);
 #pragma unroll
                     for (int k = 0; k < kTok / 16; ++k) {
-                        if (it == 0 && k == 0) {
-                            mma_ss_lh<false>(tb + C::colS, a_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iS);
+                        // the weights rows' accumulator is never started over: blocks alternate between two pairs of
+                        // its lanes (the weights block's columns 0, 1 or 2, 3), each pair a running sum
+                        if (first && k == 0) mma_ss_lh<false>(dS, a_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iS);
+                        else mma_ss_lh<true>(dS, a_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iS);
+                        if (it == 0 && k == 0)
                             mma_ss_lh<false>(tb + C::colZ, w_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iZ);
-                        } else {
-                            mma_ss_lh<true>(tb + C::colS, a_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iS);
+                        else
                             mma_ss_lh<true>(tb + C::colZ, w_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iZ);
-                        }
                     }
                 }
                 mma_commit(&bars[rMma0 + b]);
                 if (ends_block(it)) {
-                    // the row threads read the sums so far; the next step adds to them after that
-                    mma_commit(&bars[rFlush]);
-                    ok = mbar_wait(&bars[rFlushDone], nflush & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    ++nflush;
+                    mma_commit(&bars[rFlush0 + a]);          // the block's sums are complete: the row threads read them
+                    ++nblk_done;
                 }
                 // the previous step's products are done long since: its stage takes the load kNSR steps ahead
                 if (it >= 1 && it - 1 + kNSR < nit) {
@@ -228,21 +236,34 @@ __global__ void __launch_bounds__(kThreadsR, 1)
         // of the transposed state goes out as it lies, [slot][d_v][160] (bf16 running sums, or the block's own fp32
         // sums), the row sums through two small arrays in shared memory.
         float* zs = reinterpret_cast<float*>(smem + C::offMisc + 256);
+        float run[80];                                       // running sums of this thread's half of its lane's columns
+#pragma unroll
+        for (int i = 0; i < 80; ++i) run[i] = 0.f;
         auto flush = [&](int it, int nf) -> bool {
-            if (!rows_and3(mbar_wait(&bars[rFlush], nf & 1, abort_flag))) return false;
+            const int a = nf & 1;
+            if (!rows_and3(mbar_wait(&bars[rFlush0 + a], (nf >> 1) & 1, abort_flag))) return false;
             tc_fence_after();
             const int c = own ? blk : p.rev ? tile_of(it) / spb - 1 : (tile_of(it) + 1) / spb;
             const size_t slot = (size_t)head * p.nblk + c;
             const size_t rowoff = (slot * p.dvw + (t < p.dvw ? t : 0)) * 160 + half * 80;
+            // where the weights rows lie: d_v 64: lanes 64, 65 of this block's accumulator (own sums: added to the
+            // running parts in shared memory); d_v 128: lanes 2a, 2a + 1 of their own accumulator (running sums of
+            // every second block: they replace their parts, the other pair's parts stay as last read)
+            const bool zwarp = (warp & 3) == (DV == 64 ? 2 : 0);
+            const bool zlane = DV == 64 ? lane < 2 : (lane >> 1) == a;
+            float* zrow = zs + (DV == 64 ? lane : lane) * 160;
 #pragma unroll
             for (int j = 0; j < 5; ++j) {
                 uint32_t r[16];
                 const int f0 = half * 80 + j * 16;           // this thread's half of the lane's columns
-                tmem_ld16(tmem_addr(tb, lane_base, C::colS + f0), r);
+                tmem_ld16(tmem_addr(tb, lane_base, C::colS + a * 160 + f0), r);
                 tmem_wait_ld();
                 float v[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) * feature_weight(f0 + i);
+                for (int i = 0; i < 16; ++i) {
+                    run[j * 16 + i] += __uint_as_float(r[i]);
+                    v[i] = run[j * 16 + i] * feature_weight(f0 + i);
+                }
                 if (t < p.dvw) {
                     if (own) {
                         float4* d4 = reinterpret_cast<float4*>(p.part + rowoff + j * 16);
@@ -260,29 +281,27 @@ __global__ void __launch_bounds__(kThreadsR, 1)
                         d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
                     }
                 }
-                // the weights rows: lanes 0 (high part) and 1 (low part) of the quarter that holds them
-                if ((warp & 3) == (DV == 64 ? 2 : 0)) {
+                if (zwarp) {
                     if (DV != 64) {
                         tmem_ld16(tmem_addr(tb, lane_base, C::colZ + f0), r);
                         tmem_wait_ld();
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) * feature_weight(f0 + i);
                     }
-                    if (lane < 2) {
-                        float4* z4 = reinterpret_cast<float4*>(zs + lane * 160 + f0);
+                    if (lane < 4 && zlane) {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) z4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                        for (int i = 0; i < 16; ++i) zrow[f0 + i] = v[i];
                     }
                 }
             }
-            const bool good = rows_and3(true);               // the row sums' parts are written
-            if (tid < 160) (own ? p.zpart : p.sv)[slot * 160 + tid] = zs[tid] + zs[160 + tid];
             tc_fence_before();
-            mbar_arrive(&bars[rFlushDone]);
-            return good;
+            mbar_arrive(&bars[rFree0 + a]);                  // the accumulator may start over
+            const bool good = rows_and3(true);               // the row sums' parts are written
+            if (tid < 160) (own ? p.zpart : p.sv)[slot * 160 + tid] = (zs[tid] + zs[160 + tid]) + (zs[320 + tid] + zs[480 + tid]);
+            return rows_and3(good);                          // ... and read, before the next block end writes them
         };
         fetch(0);
-        int nflush = 0;
+        int nflush = 0, nflush_w = 0;                        // blocks read so far; blocks whose operands are written
         for (int it = 0; it < nit && ok; ++it) {
             const int b = it & 1;
             float x[16];
@@ -334,13 +353,18 @@ __global__ void __launch_bounds__(kThreadsR, 1)
             if (half == 0) pieces(std::integral_constant<int, 0>{});
             else pieces(std::integral_constant<int, 1>{});
             if (half == 0) {
-                // the token's weight as columns 0 (high part) and 1 (low part) of its row of the weights block
+                // the token's weight, high and low part, as two columns of its row of the weights block: 0 and 1, or
+                // at d_v 128 2 and 3 in every second block (the other pair zero)
                 __nv_bfloat16 hi = __float2bfloat16(wt), lo = __float2bfloat16(wt - __bfloat162float(hi));
                 __nv_bfloat162 h2;
                 h2.x = hi;
                 h2.y = lo;
-                *reinterpret_cast<__nv_bfloat162*>(smem + C::offW + b * C::kWBytes + t * 128 + ((t & 7) << 4)) = h2;
+                const uint32_t w2 = *reinterpret_cast<uint32_t*>(&h2);
+                const bool second = DV != 64 && (nflush_w & 1);
+                *reinterpret_cast<uint2*>(smem + C::offW + b * C::kWBytes + t * 128 + ((t & 7) << 4)) =
+                    second ? make_uint2(0u, w2) : make_uint2(w2, 0u);
             }
+            if (ends_block(it)) ++nflush_w;
             fence_proxy_async_smem();
             mbar_arrive(&bars[rAlu0 + b]);
             // a block ended with the step before: its sums are read after this step's operand is handed over, so
