@@ -62,7 +62,7 @@ template <int DV, int MODE, int LT, bool XB = false> struct BCfg {
     static constexpr uint32_t kStageArea = (XB && kStage + kStateTile > 2 * kStage) ? kStage + kStateTile : 2 * kStage;
     static constexpr uint32_t offB = offStage + kStageArea;
     static constexpr uint32_t offMisc = offB + 2 * LT * 8;
-    static constexpr uint32_t kSmem = offMisc + 1024 + 1024;                    // barriers, the block state's row sums (160 floats)
+    static constexpr uint32_t kSmem = offMisc + 2048 + 1024;                    // barriers, the block state's row sums (160 floats), m (128)
 
     // tensor memory columns: scores, dout.v products, ds (dq pass; the dk/dv pass packs in place), accumulators
     static constexpr uint32_t colS = 0, colG = LT, colD = MODE == kModeFwd ? LT : 2 * LT;   // forward: no dout.v product
@@ -180,12 +180,13 @@ __device__ __forceinline__ void block_rows(uint32_t tb, uint32_t lane_base, cons
 // tm_n0 / tm_w0: narrow (q or k) and wide (a/g or v) tensor of the CTA's own (resident) tile;
 // tm_n1 / tm_w1: of the tiles it loops over.
 // XB: the block-wise path (merged statistics + dq pass and dk/dv pass, d' = 16); tm_st: the block states,
-// transposed: [BH x nblk][d_v][160] bf16.
+// transposed: [BH x nblk][d_v][160] bf16.  tm_out: the wide output (dv, or the forward output), stored by TMA.
 template <int DV, int MODE, int LT, bool XB>
 __global__ void __launch_bounds__(kThreadsB, 1)
     backward_tc_kernel(const __grid_constant__ CUtensorMap tm_n0, const __grid_constant__ CUtensorMap tm_w0,
                        const __grid_constant__ CUtensorMap tm_n1, const __grid_constant__ CUtensorMap tm_w1,
-                       const __grid_constant__ CUtensorMap tm_st, const BParams p) {
+                       const __grid_constant__ CUtensorMap tm_st, const __grid_constant__ CUtensorMap tm_out,
+                       const BParams p) {
     static_assert(!XB || MODE == kModeDqS || MODE == kModeDkDv, "block-wise path: the two passes that use it");
     using C = BCfg<DV, MODE, LT, XB>;
     extern __shared__ uint8_t smem_raw[];
@@ -195,6 +196,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
     volatile uint32_t* abort_flag = tmem_base_s + 1;
     float2* s_b = reinterpret_cast<float2*>(smem + C::offB);
     float* s_sv = reinterpret_cast<float*>(smem + C::offMisc + 256);
+    float* s_m = reinterpret_cast<float*>(smem + C::offMisc + 1024);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int ntiles = (p.L + kTile - 1) / kTile;
@@ -217,9 +219,6 @@ __global__ void __launch_bounds__(kThreadsB, 1)
         mbar_init(&bars[bXs], 1); mbar_init(&bars[bX0], 1); mbar_init(&bars[bX1], 128);
         *abort_flag = 0;
         fence_mbar_init();
-    }
-    if (cross) {
-        for (int i = tid; i < 160; i += kThreadsB) s_sv[i] = p.sv[((size_t)head * p.nblk + blk) * 160 + i];
     }
     if (warp == 4) { tmem_alloc(tmem_base_s, C::kCols); tmem_relinquish(); }
     tc_fence_before();
@@ -407,12 +406,54 @@ __global__ void __launch_bounds__(kThreadsB, 1)
         // merged pass: the products dout_i . v_j enter the packed tile relative to m_i = dout_i . out_i, which
         // is their weighted mean E_i / D_i up to the rounding of out: the part of dq that cancels against
         // b_i is then formed in fp32 at the end, not from two separately rounded bf16 tiles
+        // the block state's row sums: read by the row threads only, after their next barrier
+        if (XB && cross) {
+            const float* svp = p.sv + ((size_t)head * p.nblk + blk) * 160;
+            s_sv[t] = svp[t];
+            if (t < 32) s_sv[128 + t] = svp[128 + t];
+        }
         float m_own = 0.f;
-        if (MODE == kModeDqS && !p.numerator_only && row < p.L) {
+        if (MODE == kModeDqS && !p.numerator_only && (DV == 64 || p.dvw == 128)) {
+            // a warp's 32 rows of out lie one after the other in global memory: every load instruction takes 512
+            // consecutive bytes (two rows at d_v 128, four at d_v 64); the matching piece of dout comes from the own
+            // tile in shared memory, and the lanes of a row add up their parts
+            constexpr int PPR = DV / 8;                       // 16-byte pieces per row
+            constexpr int NI = PPR;                           // load instructions per warp: 32 rows x PPR pieces / 32 lanes
+            const int wrow0 = r0 + warp * 32;
+            const uint4* op = reinterpret_cast<const uint4*>(p.o_raw + ((size_t)head * p.L + wrow0) * DV);
+            uint4 ob[NI];
+#pragma unroll
+            for (int i = 0; i < NI; ++i) {
+                const int pc = i * 32 + lane;                 // piece of the warp's 32 x PPR
+                ob[i] = wrow0 + pc / PPR < p.L ? op[pc] : make_uint4(0u, 0u, 0u, 0u);
+            }
+            ok = rows_all(mbar_wait(&bars[bRes], 0, abort_flag));
+#pragma unroll
+            for (int i = 0; i < NI; ++i) {
+                const int pc = i * 32 + lane;
+                const int rr = warp * 32 + pc / PPR, c = pc % PPR;           // row of the tile, piece of the row
+                const uint4 u = *reinterpret_cast<const uint4*>(smem + C::offResW + (c >> 3) * (kTile * 128) + rr * 128 +
+                                                                (((c & 7) ^ (rr & 7)) << 4));
+                const __nv_bfloat162* ha = reinterpret_cast<const __nv_bfloat162*>(&u);
+                const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&ob[i]);
+                float d = 0.f;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 fa = __bfloat1622float2(ha[e]), fb = __bfloat1622float2(hb[e]);
+                    d = fmaf(fa.x, fb.x, d);
+                    d = fmaf(fa.y, fb.y, d);
+                }
+#pragma unroll
+                for (int o = PPR / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+                if (c == 0) s_m[rr] = d;
+            }
+            __syncwarp();
+            m_own = s_m[t];
+        } else if (MODE == kModeDqS && !p.numerator_only && row < p.L) {
             const uint4* gp = reinterpret_cast<const uint4*>(p.g_raw + ((size_t)head * p.L + row) * p.dvw);
             const uint4* op = reinterpret_cast<const uint4*>(p.o_raw + ((size_t)head * p.L + row) * p.dvw);
             float part[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int c0 = 0; c0 < p.dvw / 8; c0 += 4) {          // 64, 112, 128 columns: 8, 14, 16 pieces; four in flight
+            for (int c0 = 0; c0 < p.dvw / 8; c0 += 4) {          // 112 columns: 14 pieces; four in flight
                 uint4 a[4], b[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -594,25 +635,36 @@ __global__ void __launch_bounds__(kThreadsB, 1)
             }
             if (MODE == kModeDkDv || MODE == kModeFwd) {
                 // the wide accumulator row: dv, or the forward output scaled by 1 / (denominator + eps)
+                // through the own wide tile's place in shared memory (its products are done) in the layout of a TMA box,
+                // [128 rows][64 columns] blocks with 128-byte rows, SWIZZLE_128B, and out by TMA: whole 128-byte lines
+                // per row where a store per row thread would touch 32 rows per instruction.  Rows and columns past the
+                // tensor's end are clipped by the store.
                 const float sc = (MODE == kModeFwd && !p.numerator_only) ? 1.0f / (den + kEps) : 1.0f;
-                uint4* vdst = reinterpret_cast<uint4*>(p.dvo + grow * p.dvw);
                 for (int c = 0; c < p.dvw / 16; ++c) {       // p.dvw is uniform
                     uint32_t rv[16];
                     tmem_ld16(tmem_addr(tb, lane_base, C::colAcc + c * 16), rv);
                     tmem_wait_ld();
-                    if (store) {
-                        uint4 a, b;
-                        a.x = pack_bf16x2(__uint_as_float(rv[0]) * sc, __uint_as_float(rv[1]) * sc);
-                        a.y = pack_bf16x2(__uint_as_float(rv[2]) * sc, __uint_as_float(rv[3]) * sc);
-                        a.z = pack_bf16x2(__uint_as_float(rv[4]) * sc, __uint_as_float(rv[5]) * sc);
-                        a.w = pack_bf16x2(__uint_as_float(rv[6]) * sc, __uint_as_float(rv[7]) * sc);
-                        b.x = pack_bf16x2(__uint_as_float(rv[8]) * sc, __uint_as_float(rv[9]) * sc);
-                        b.y = pack_bf16x2(__uint_as_float(rv[10]) * sc, __uint_as_float(rv[11]) * sc);
-                        b.z = pack_bf16x2(__uint_as_float(rv[12]) * sc, __uint_as_float(rv[13]) * sc);
-                        b.w = pack_bf16x2(__uint_as_float(rv[14]) * sc, __uint_as_float(rv[15]) * sc);
-                        vdst[2 * c] = a;
-                        vdst[2 * c + 1] = b;
-                    }
+                    uint4 a, b;
+                    a.x = pack_bf16x2(__uint_as_float(rv[0]) * sc, __uint_as_float(rv[1]) * sc);
+                    a.y = pack_bf16x2(__uint_as_float(rv[2]) * sc, __uint_as_float(rv[3]) * sc);
+                    a.z = pack_bf16x2(__uint_as_float(rv[4]) * sc, __uint_as_float(rv[5]) * sc);
+                    a.w = pack_bf16x2(__uint_as_float(rv[6]) * sc, __uint_as_float(rv[7]) * sc);
+                    b.x = pack_bf16x2(__uint_as_float(rv[8]) * sc, __uint_as_float(rv[9]) * sc);
+                    b.y = pack_bf16x2(__uint_as_float(rv[10]) * sc, __uint_as_float(rv[11]) * sc);
+                    b.z = pack_bf16x2(__uint_as_float(rv[12]) * sc, __uint_as_float(rv[13]) * sc);
+                    b.w = pack_bf16x2(__uint_as_float(rv[14]) * sc, __uint_as_float(rv[15]) * sc);
+                    uint8_t* rowp = smem + C::offResW + (c >> 2) * (kTile * 128) + t * 128;
+                    *reinterpret_cast<uint4*>(rowp + ((((2 * c) & 7) ^ (t & 7)) << 4)) = a;
+                    *reinterpret_cast<uint4*>(rowp + ((((2 * c + 1) & 7) ^ (t & 7)) << 4)) = b;
+                }
+                fence_proxy_async_smem();
+                rows_all(true);
+                if (t == 0) {
+#pragma unroll
+                    for (int bb = 0; bb < C::kVB; ++bb)
+                        tma_store_3d(&tm_out, smem + C::offResW + bb * (kTile * 128), bb * 64, r0, head);
+                    tma_store_commit();
+                    tma_store_wait<0>();
                 }
             }
         }
@@ -694,7 +746,7 @@ __global__ void __launch_bounds__(256)
 template <int DV, int MODE, int LT, bool XB = false>
 based_status launch_pass(const CUtensorMap& n0, const CUtensorMap& w0, const CUtensorMap& n1, const CUtensorMap& w1,
                          const BParams& p, dim3 grid, const char* what, cudaStream_t stream,
-                         const CUtensorMap* st = nullptr) {
+                         const CUtensorMap* st = nullptr, const CUtensorMap* outm = nullptr) {
     using C = BCfg<DV, MODE, LT, XB>;
     static bool configured[64] = {};
     int dev = 0;
@@ -708,7 +760,8 @@ based_status launch_pass(const CUtensorMap& n0, const CUtensorMap& w0, const CUt
             configured[dev] = true;
         }
     }
-    backward_tc_kernel<DV, MODE, LT, XB><<<grid, kThreadsB, C::kSmem, stream>>>(n0, w0, n1, w1, st ? *st : n0, p);
+    backward_tc_kernel<DV, MODE, LT, XB><<<grid, kThreadsB, C::kSmem, stream>>>(n0, w0, n1, w1, st ? *st : n0,
+                                                                               outm ? *outm : w0, p);
     note_launch();
     return check_launch(what);
 }
@@ -749,12 +802,13 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
     constexpr int LTK = (DV == 64) ? 64 : 128;       // looped tile of the dk/dv pass (d_v 128 needs all 512 columns anyway)
     float2* stats = reinterpret_cast<float2*>(ws);
     // own tiles: 128 rows; looped tiles: 64 rows (and LTK rows for the dk/dv pass)
-    CUtensorMap tq, tk, tv, tg, tk64, tv64, tqL, tgL;
+    CUtensorMap tq, tk, tv, tg, tk64, tv64, tqL, tgL, tdv;
     const CUtensorMapSwizzle s64 = CU_TENSOR_MAP_SWIZZLE_64B, s128 = CU_TENSOR_MAP_SWIZZLE_128B;
     if (!make_map_b(&tq, q, BH, L, df, 32, kTile, s64) || !make_map_b(&tk, k, BH, L, df, 32, kTile, s64) ||
         !make_map_b(&tv, v, BH, L, dvr, 64, kTile, s128) || !make_map_b(&tg, g, BH, L, dvr, 64, kTile, s128) ||
         !make_map_b(&tk64, k, BH, L, df, 32, 64, s64) || !make_map_b(&tv64, v, BH, L, dvr, 64, 64, s128) ||
-        !make_map_b(&tqL, q, BH, L, df, 32, LTK, s64) || !make_map_b(&tgL, g, BH, L, dvr, 64, LTK, s128))
+        !make_map_b(&tqL, q, BH, L, df, 32, LTK, s64) || !make_map_b(&tgL, g, BH, L, dvr, 64, LTK, s128) ||
+        !make_map_b(&tdv, dv, BH, L, dvr, 64, kTile, s128))
         return BASED_ERR_CUDA;
     BParams p{};
     if (error_word_ptr(&p.err) != BASED_OK) return BASED_ERR_CUDA;
@@ -802,7 +856,8 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
         if (st != BASED_OK) return st;
         // states of the queries: R = sum mono(q) (dout / D)^T, R_b = sum b mono(q), summed over the blocks after each block
         if ((st = states(q, g, stats, 1)) != BASED_OK) return st;
-        return launch_pass<DV, kModeDkDv, LTK, true>(tk, tv, tqL, tgL, p, grid, "backward_tc_kernel<dkdv, blocks>", stream, &tst);
+        return launch_pass<DV, kModeDkDv, LTK, true>(tk, tv, tqL, tgL, p, grid, "backward_tc_kernel<dkdv, blocks>", stream, &tst,
+                                                     &tdv);
     }
     if (out != nullptr || numerator_only) {
         // statistics and dq in one sweep (needs the forward output as the centre of the packed products)
@@ -817,7 +872,7 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
         if (st != BASED_OK) return st;
     }
     // dk, dv: own = keys (k, v), looped = queries (q, dout)
-    return launch_pass<DV, kModeDkDv, LTK>(tk, tv, tqL, tgL, p, grid, "backward_tc_kernel<dkdv>", stream);
+    return launch_pass<DV, kModeDkDv, LTK>(tk, tv, tqL, tgL, p, grid, "backward_tc_kernel<dkdv>", stream, nullptr, &tdv);
 }
 }  // namespace
 
@@ -825,10 +880,10 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
 // empty initial state): out = (sum_j w_ij v_j) / (sum_j w_ij + eps), w = 1 + s/sqrt(d') + s^2/(2 d').
 based_status launch_quadratic_forward_tc(const void* q, const void* k, const void* v, void* out, int BH, int L,
                                          int d_feat, int d_v, int numerator_only, cudaStream_t stream) {
-    CUtensorMap tq, tk64, tv64;
+    CUtensorMap tq, tk64, tv64, tout;
     const CUtensorMapSwizzle s64 = CU_TENSOR_MAP_SWIZZLE_64B, s128 = CU_TENSOR_MAP_SWIZZLE_128B;
     if (!make_map_b(&tq, q, BH, L, d_feat, 32, kTile, s64) || !make_map_b(&tk64, k, BH, L, d_feat, 32, 64, s64) ||
-        !make_map_b(&tv64, v, BH, L, d_v, 64, 64, s128))
+        !make_map_b(&tv64, v, BH, L, d_v, 64, 64, s128) || !make_map_b(&tout, out, BH, L, d_v, 64, kTile, s128))
         return BASED_ERR_CUDA;
     BParams p{};
     if (error_word_ptr(&p.err) != BASED_OK) return BASED_ERR_CUDA;
@@ -841,8 +896,8 @@ based_status launch_quadratic_forward_tc(const void* q, const void* k, const voi
     p.s1 = 1.0f / sqrtf((float)d_feat);
     p.s2 = 0.5f / (float)d_feat;
     const dim3 grid((L + kTile - 1) / kTile, BH);
-    if (d_v == 64) return launch_pass<64, kModeFwd, 64>(tq, tq, tk64, tv64, p, grid, "quadratic forward (tc)", stream);
-    return launch_pass<128, kModeFwd, 64>(tq, tq, tk64, tv64, p, grid, "quadratic forward (tc)", stream);
+    if (d_v == 64) return launch_pass<64, kModeFwd, 64>(tq, tq, tk64, tv64, p, grid, "quadratic forward (tc)", stream, nullptr, &tout);
+    return launch_pass<128, kModeFwd, 64>(tq, tq, tk64, tv64, p, grid, "quadratic forward (tc)", stream, nullptr, &tout);
 }
 
 int backward_tc_block_tokens(int BH, int L, int d_feat, int d_v, int merged) {
