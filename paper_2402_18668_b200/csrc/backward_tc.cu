@@ -70,7 +70,9 @@ template <int DV, int MODE, int LT, bool XB = false> struct BCfg {
     static constexpr uint32_t colAcc = MODE == kModeDq ? 2 * LT + LT / 2                  // dQ (32)
                                        : MODE == kModeDqS ? 3 * LT                        // X (32), then Y (32)
                                        : MODE == kModeFwd ? LT + LT / 2                   // Y (64 * kVB)
-                                                          : (2 * LT < 160 ? 160 : 2 * LT);  // dV (64 * kVB), above the block product
+                                                          : (LT == 32 ? 96 : 2 * LT < 160 ? 160 : 2 * LT);  // dV (64 * kVB): above the block
+                                       // product (160 columns), or with 32-row looped tiles above its packed monomials (80): the
+                                       // product is read before the first dV product is issued
     static constexpr uint32_t colAcc2 = colAcc + 32;                                      // merged pass: Y
     static constexpr uint32_t colK = colAcc + 64 * kVB;                                   // dK (32), dk/dv pass
     static constexpr uint32_t kColsUsed = MODE == kModeStats ? 2 * LT
@@ -770,7 +772,7 @@ based_status launch_pass(const CUtensorMap& n0, const CUtensorMap& w0, const CUt
 // statistics in one sweep (the forward output, or the numerator-only form); its cost grows with L where the tile
 // path's grows with L^2, and the lengths below are where it starts to win on B200 (128 heads, d_v 64: 101 against
 // 117 us at L = 768; d_v 128: 191 against 213 us at L = 1024; 32 heads, d_v 128: 129 against 134 us at L = 1536).
-// Blocks of 256 tokens are the fastest from there on (B8 H16 L4096 d_v128: 720 / 687 / 737 us at 128 / 256 / 512),
+// Blocks of 256 tokens are the fastest from there on (B8 H16 L4096 d_v128: 613 / 582 / 661 us at 128 / 256 / 512),
 // except with few heads at d_v 128, where every block's state costs a CTA of its own.
 int backward_block_len(int L, int df, bool merged, int d_v, int BH) {
     if (df != 16 || !merged) return 0;
@@ -856,6 +858,14 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
         if (st != BASED_OK) return st;
         // states of the queries: R = sum mono(q) (dout / D)^T, R_b = sum b mono(q), summed over the blocks after each block
         if ((st = states(q, g, stats, 1)) != BASED_OK) return st;
+        if (DV == 128) {
+            // 32-row looped tiles: the accumulators then fit 256 tensor-memory columns and two CTAs share an SM, which
+            // hides the fixed latency of these short-lived CTAs (273 -> 220 us for the pass at B8 H16 L4096)
+            CUtensorMap tq32, tg32;
+            if (!make_map_b(&tq32, q, BH, L, df, 32, 32, s64) || !make_map_b(&tg32, g, BH, L, dvr, 64, 32, s128)) return BASED_ERR_CUDA;
+            return launch_pass<DV, kModeDkDv, 32, true>(tk, tv, tq32, tg32, p, grid, "backward_tc_kernel<dkdv, blocks>", stream, &tst,
+                                                        &tdv);
+        }
         return launch_pass<DV, kModeDkDv, LTK, true>(tk, tv, tqL, tgL, p, grid, "backward_tc_kernel<dkdv, blocks>", stream, &tst,
                                                      &tdv);
     }
