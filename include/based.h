@@ -209,8 +209,9 @@ based_status swa_decode_step(const void* q, const void* k, const void* v, void* 
  * s^2/(2 d'), so ds_ij = (a_i . v_j + b_i)(1/sqrt(d') + q_i.k_j / d')); d_v in {64, 112, 128}; B*H <= 65535.
  * Both paths evaluate the quadratic form, O(L^2) per head, on 128 x 128 (bf16 io: tcgen05 tensor
  * cores, bf16 operands, fp32 accumulation) or 64 x 64 (fp32 io: fp32 FMAs) tiles of (query, key)
- * pairs; with bf16 io, d_feat = 16 and BASED_NUMERATOR_ONLY, long sequences take the block-wise
- * path described at based_prefill_backward_with_out.  Gradient outputs must not alias inputs.
+ * pairs; with bf16 io and d_feat = 16 longer sequences take the block-wise path described at
+ * based_prefill_backward_with_out (the forward output that it needs is recomputed into the workspace:
+ * one forward pass more).  Gradient outputs must not alias inputs.
  */
 based_status based_prefill_backward(const void* q, const void* k, const void* v, const void* dout, void* dq,
                                     void* dk, void* dv, int B, int H, int L, int d_feat, int d_v, based_dtype io,
@@ -248,8 +249,9 @@ based_status based_prefill_backward_with_out(const void* q, const void* k, const
 
 /*
  * Which path a backward call with these arguments takes: the block length W of the block-wise path, or 0
- * for the tile path (fp32 io, d_feat other than 16, short sequences, or neither the forward output nor
- * BASED_NUMERATOR_ONLY given).  with_out: nonzero for based_prefill_backward_with_out with out non-null.
+ * for the tile path (fp32 io, d_feat other than 16, short sequences).  with_out: nonzero for
+ * based_prefill_backward_with_out with out non-null; without the forward output (and without
+ * BASED_NUMERATOR_ONLY) the block-wise path starts at somewhat longer sequences.
  * Host only; for callers that account the work of a call (benchmarks).
  */
 int based_prefill_backward_block_tokens(int B, int H, int L, int d_feat, int d_v, based_dtype io, int flags,

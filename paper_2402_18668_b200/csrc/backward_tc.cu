@@ -774,8 +774,15 @@ based_status launch_pass(const CUtensorMap& n0, const CUtensorMap& w0, const CUt
 // 117 us at L = 768; d_v 128: 191 against 213 us at L = 1024; 32 heads, d_v 128: 129 against 134 us at L = 1536).
 // Blocks of 256 tokens are the fastest from there on (B8 H16 L4096 d_v128: 613 / 582 / 661 us at 128 / 256 / 512),
 // except with few heads at d_v 128, where every block's state costs a CTA of its own.
+// A caller without the forward output gets it recomputed into the workspace first (one forward pass, 23 us at B4 H16
+// L2048 d_v64, 83 us at B8 H16 L4096 d_v128), from somewhat longer sequences on.
 int backward_block_len(int L, int df, bool merged, int d_v, int BH) {
-    if (df != 16 || !merged) return 0;
+    if (df != 16) return 0;
+    if (!merged) {
+        if (d_v == 64) return L >= 1024 ? 256 : 0;
+        if (BH >= 64) return L >= 1536 ? 256 : 0;
+        return L >= 4096 ? 512 : L >= 2048 ? 256 : 0;
+    }
     if (d_v == 64) return L >= 768 ? 256 : 0;
     if (BH >= 64) return L >= 1024 ? 256 : 0;
     return L >= 4096 ? 512 : L >= 1536 ? 256 : 0;
@@ -783,6 +790,7 @@ int backward_block_len(int L, int df, bool merged, int d_v, int BH) {
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 struct BlockWs {
     float* sv; float* zpart; float* part; __nv_bfloat16* st;
+    __nv_bfloat16* out; void* fwd;                   // the recomputed forward output and the forward pass's own scratch
     size_t bytes;
 };
 // scratch after the [BH, L] float2 statistics
@@ -792,8 +800,11 @@ BlockWs block_ws(float* ws, int BH, int L, int dvr, int nblk) {
     size_t off = align256((size_t)BH * L * 8);
     w.sv = reinterpret_cast<float*>(base + off);     off = align256(off + (size_t)BH * nblk * 160 * 4);
     w.zpart = reinterpret_cast<float*>(base + off);  off = align256(off + (size_t)BH * nblk * 160 * 4);
-    w.part = reinterpret_cast<float*>(base + off);   off = align256(off + (size_t)BH * nblk * 160 * dvr * 4);
+    // the blocks' own fp32 sums: only where a scan adds them up (few heads)
+    w.part = reinterpret_cast<float*>(base + off);   off = align256(off + (BH >= 64 ? 0 : (size_t)BH * nblk * 160 * dvr * 4));
     w.st = reinterpret_cast<__nv_bfloat16*>(base + off);  off = align256(off + (size_t)BH * nblk * 160 * dvr * 2);
+    w.out = reinterpret_cast<__nv_bfloat16*>(base + off); off = align256(off + (size_t)BH * L * dvr * 2);
+    w.fwd = reinterpret_cast<void*>(base + off);     off = align256(off + prefill_tc_workspace_bytes(BH, L, dvr));
     w.bytes = off;
     return w;
 }
@@ -838,6 +849,12 @@ based_status launch_dvb(const void* q, const void* k, const void* v, const void*
         CUtensorMap tst;
         // the block states lie transposed, [BH x nblk][d_v][160]: boxes of 32 features x all value columns
         if (!make_map_b(&tst, w.st, BH * nblk, dvr, 160, 32, 64 * BCfg<DV, kModeDkDv, LTK>::kVB, s64)) return BASED_ERR_CUDA;
+        if (out == nullptr && !numerator_only) {
+            // the centre of the merged pass: the forward output, recomputed
+            st = launch_prefill_tc(q, k, v, w.out, nullptr, nullptr, BH, L, dvr, 0, w.fwd, stream);
+            if (st != BASED_OK) return st;
+            p.o_raw = w.out;
+        }
         p.W = W;
         p.nblk = nblk;
         p.sv = w.sv;

@@ -162,7 +162,9 @@ def test_backward_validation(lib):
     assert lib.based_prefill_backward_workspace_bytes(2, 3, 100, 64, 1) == 2 * 3 * 100 * 8
     # the block-wise path: bf16, d' = 16, statistics in one sweep, from a few blocks of 256 tokens up
     assert lib.based_prefill_backward_block_tokens(4, 16, 2048, 16, 64, 1, 0, 1) == 256
-    assert lib.based_prefill_backward_block_tokens(4, 16, 2048, 16, 64, 1, 0, 0) == 0      # no forward output
+    assert lib.based_prefill_backward_block_tokens(4, 16, 2048, 16, 64, 1, 0, 0) == 256    # forward output recomputed
+    assert lib.based_prefill_backward_block_tokens(4, 16, 800, 16, 64, 1, 0, 0) == 0       # ... from longer sequences on
+    assert lib.based_prefill_backward_block_tokens(4, 16, 800, 16, 64, 1, 0, 1) == 256
     assert lib.based_prefill_backward_block_tokens(4, 16, 2048, 16, 64, 1, 4, 0) == 256    # numerator only
     assert lib.based_prefill_backward_block_tokens(4, 16, 2048, 16, 64, 0, 0, 1) == 0      # fp32 io
     assert lib.based_prefill_backward_block_tokens(4, 16, 2048, 32, 64, 1, 0, 1) == 0      # other feature dimension

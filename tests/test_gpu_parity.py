@@ -298,8 +298,8 @@ def test_prefill_backward_with_forward_output_cfg2_sampled_heads():
 @pytest.mark.parametrize("with_out", [False, True])
 def test_prefill_backward_cfg3_sampled_heads(with_out):
     """Full 1.3B-layer shape (B8 H16 L4096 d_v128, bf16): one head recomputed by the oracle (4096^2 / 2 pairs in
-    fp64), gradients drawn on the device.  Without the forward output: the tile path (dk/dv pass on 128-row looped
-    tiles); with it: the block-wise path (eight blocks of 512 tokens)."""
+    fp64), gradients drawn on the device.  The block-wise path (sixteen blocks of 256 tokens); without the forward
+    output the library recomputes it first."""
     w = wl.CONFIGS["cfg3_1p3b_prefill"]
     g_ = torch.Generator(device=DEV).manual_seed(88)
     q = (torch.randn(w.B, w.H, w.L, 16, generator=g_, device=DEV) * w.qk_scale).bfloat16()
@@ -310,7 +310,7 @@ def test_prefill_backward_cfg3_sampled_heads(with_out):
     n0 = based.launch_count()
     dq, dk, dv = based.based_prefill_backward(q, k, v, dout, out=out)
     _poll()
-    assert based.launch_count() - n0 == (4 if with_out else 3)     # block-wise: two state walks, two tile passes
+    assert based.launch_count() - n0 == (4 if with_out else 5)     # block-wise: two state walks, two tile passes (+ forward)
     b, h = w.B - 1, 5
     sl = (slice(b, b + 1), slice(h, h + 1))
     rq, rk, rv = oracle.linattn_backward(_np(q[sl]), _np(k[sl]), _np(v[sl]), _np(dout[sl]))
@@ -369,9 +369,9 @@ def test_prefill_backward_blockwise_running_states(L, d_v, flags):
             assert rows.max() <= TOL_BF16
 
 
-def test_prefill_backward_blockwise_many_blocks_against_tile_path():
-    """64 blocks (B1 H2 L16384 d_v64): the block-wise path against the tile path (no forward output given), each
-    within tolerance of the truth."""
+def test_prefill_backward_blockwise_many_blocks_against_fp32_path():
+    """64 blocks (B1 H2 L16384 d_v64): the block-wise path, with and without the forward output, against the fp32
+    path of the library (quadratic form, fp32 FMAs) on the same bf16 values."""
     B, H, L, d_v = 1, 2, 16384, 64
     g_ = torch.Generator(device=DEV).manual_seed(16384)
     q = (torch.randn(B, H, L, 16, generator=g_, device=DEV) * 0.4).bfloat16()
@@ -380,12 +380,32 @@ def test_prefill_backward_blockwise_many_blocks_against_tile_path():
     dout = torch.randn(B, H, L, d_v, generator=g_, device=DEV).bfloat16()
     out = based.based_prefill(q, k, v)
     blk = based.based_prefill_backward(q, k, v, dout, out=out)
-    til = based.based_prefill_backward(q, k, v, dout)
+    n0 = based.launch_count()
+    blk2 = based.based_prefill_backward(q, k, v, dout)
+    assert based.launch_count() - n0 >= 7                    # forward recomputed, then the six block-wise launches
+    ref = based.based_prefill_backward(q.float(), k.float(), v.float(), dout.float())
     _poll()
-    for a, b in zip(blk, til):
-        assert _grad_err(_np(a), _np(b)) <= TOL_BF16
-        d = (a.float() - b.float()).norm() / b.float().norm()
-        assert d.item() <= 1e-2
+    for a, a2, b in zip(blk, blk2, ref):
+        assert _grad_err(_np(a), _np(b)) <= TOL_BF16 and _grad_err(_np(a2), _np(b)) <= TOL_BF16
+        assert ((a.float() - b).norm() / b.norm()).item() <= 1e-2 and ((a2.float() - b).norm() / b.norm()).item() <= 1e-2
+
+
+def test_prefill_backward_tile_path_long_loops():
+    """The tile path alone at a length where its loops are long (d' = 32 keeps it off the block-wise path): B1 H2
+    L2048 d_v128, with and without the forward output, against the oracle."""
+    B, H, L, d_v, d_feat = 1, 2, 2048, 128, 32
+    w = wl.Workload("bwdtile", B, H, L, d_feat, d_v, "bf16", 0.5)
+    q, k, v = wl.prefill_inputs(w, wl.generator(3232))
+    g = torch.randn(B, H, L, d_v, generator=wl.generator(3233)).to(v.dtype)
+    rq, rk, rv = oracle.linattn_backward(_np(q), _np(k), _np(v), _np(g))
+    qd, kd, vd, gd = q.to(DEV), k.to(DEV), v.to(DEV), g.to(DEV)
+    out = based.based_prefill(qd, kd, vd)
+    for o, n in ((None, 3), (out, 2)):
+        n0 = based.launch_count()
+        dq, dk, dv = based.based_prefill_backward(qd, kd, vd, gd, out=o)
+        _poll()
+        assert based.launch_count() - n0 == n
+        assert _grad_err(_np(dq), rq) <= TOL_BF16 and _grad_err(_np(dk), rk) <= TOL_BF16 and _grad_err(_np(dv), rv) <= TOL_BF16
 
 
 @pytest.mark.parametrize("d_feat", [8, 32])
