@@ -28,6 +28,16 @@
 // feature dimensions 8, 24 and 32, which the chunked d' = 16 kernel does not cover.  All modes take
 // d' (8, 16, 24, 32) as a parameter: the polynomial's coefficients 1/sqrt(d'), 1/(2 d'), a second K
 // step of the scores above 16, and up to 32 gradient columns of dq and dk.
+//
+// Block-wise path (template flag XB; d' = 16, statistics in one sweep): linear in L.  The loops of the merged
+// statistics + dq pass and of the dk/dv pass stop at the edges of the own tile's block of W tokens; all earlier
+// blocks reach a query, and all later blocks a key, through one state tile each (block_state_tc.cu writes them:
+// S = sum mono(k) v^T with row sums z for the queries, R = sum mono(q) (dout / D)^T with row sums R_b = sum b mono(q)
+// for the keys, in the basis of the 153 distinct monomials of the feature map).  Before its loop such a CTA
+// multiplies its own wide tile with the state tile (T = G S^T or V R^T, 128 x 160 in tensor memory), every row
+// thread contracts its row of T with the monomials and the Jacobian of its q or k row, and the results start the
+// accumulators that the loop's products add to; the dk/dv pass also writes the monomials of its k rows back to
+// tensor memory as the A operand of dV = mono(K) R.
 #include <math.h>
 
 #include <mutex>

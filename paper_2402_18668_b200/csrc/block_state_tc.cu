@@ -251,7 +251,7 @@ __global__ void __launch_bounds__(kThreadsR, 1)
             // every second block: they replace their parts, the other pair's parts stay as last read)
             const bool zwarp = (warp & 3) == (DV == 64 ? 2 : 0);
             const bool zlane = DV == 64 ? lane < 2 : (lane >> 1) == a;
-            float* zrow = zs + (DV == 64 ? lane : lane) * 160;
+            float* zrow = zs + lane * 160;                   // lanes 0..3 of the quarter: one part each
 #pragma unroll
             for (int j = 0; j < 5; ++j) {
                 uint32_t r[16];
