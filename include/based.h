@@ -239,7 +239,8 @@ size_t based_prefill_backward_workspace_bytes(int B, int H, int L, int d_v, base
  * The block states are fp32 sums, rounded once to bf16 as tensor-core operands, like the state copy of
  * the forward pass; the products S dout_i and m_i z cancel in fp32 after the product, so the error
  * relative to the gradient grows with |mean v| / std v over the earlier blocks (1.5e-2 at mean 3,
- * std 1; 3e-3 for centred values).  Four launches instead of two (six below 64 heads, where the block
+ * std 1; 3e-3 for centred values; the gradients do not depend on a common offset of the values, so a
+ * caller with such an offset can subtract it first).  Four launches instead of two (six below 64 heads, where the block
  * states come from one CTA per head and block plus a scan instead of one CTA walking each head).
  */
 based_status based_prefill_backward_with_out(const void* q, const void* k, const void* v, const void* out,
