@@ -23,8 +23,9 @@
 // state, [d_v][160] - the layout the readers' descriptors take as it lies.  (The weights rows'
 // accumulator at d_v 128 is never started over: blocks alternate between two pairs of its lanes,
 // each pair a running sum of every second block.)  The operand tiles are double-buffered and the
-// value tiles come through a ring of three stages.  With few heads one CTA per (head, block) writes
-// the block's own sums in fp32 instead, for a scan by another kernel.
+// value tiles come through a ring of three stages.  With few heads one CTA per head and group of one
+// to four consecutive blocks writes every block's own sums in fp32 instead, for a scan by another
+// kernel.
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -56,7 +57,7 @@ template <int DV> struct RCfg {
     static constexpr uint32_t offW = kNSR * kVBytes;
     static constexpr uint32_t offPhi = offW + 2 * kWBytes;
     static constexpr uint32_t offMisc = offPhi + 2 * kPhiBytes;
-    static constexpr uint32_t kSmem = offMisc + 3072 + 1024;   // barriers; the row sums' parts (4 x 160 floats)
+    static constexpr uint32_t kSmem = offMisc + 4096 + 1024;   // barriers; the row sums' parts (4 x 160 floats), their changes (2 x 160)
     // two accumulators of 160 columns that alternate from block to block; at d_v 128 the weights rows' accumulator
     static constexpr uint32_t colS = 0, colZ = 320;
     static constexpr uint32_t kCols = 512;
@@ -74,6 +75,7 @@ struct RParams {
     float* zpart;
     unsigned int* err;
     int L, dvw, W, nblk, rev;
+    int grp;                       // own sums: blocks per CTA (consecutive blocks of one head)
 };
 
 // AND of a predicate over the 256 row threads (named barrier 3); also a barrier for their shared-memory traffic
@@ -105,18 +107,18 @@ __global__ void __launch_bounds__(kThreadsR, 1)
     volatile uint32_t* abort_flag = tmem_base_s + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const bool own = p.part != nullptr;                      // one block's own sums
-    const int head = own ? blockIdx.x / p.nblk : blockIdx.x;
-    const int blk = own ? blockIdx.x % p.nblk : 0;
+    const bool own = p.part != nullptr;                      // every block's own sums, grp consecutive blocks per CTA
+    const int ngrp = own ? (p.nblk + p.grp - 1) / p.grp : 1;
+    const int head = own ? blockIdx.x / ngrp : blockIdx.x;
+    const int blk = own ? (blockIdx.x % ngrp) * p.grp : 0;  // first block of the CTA
     const int spb = p.W / kTok;                              // steps per block
     const int ntile = (p.L + kTok - 1) / kTok;
-    // the last block walked (first block in reverse) adds to no state that anyone reads
-    if (own && blk == (p.rev ? 0 : p.nblk - 1)) return;
-    const int nit = own ? min(spb, ntile - blk * spb) : p.rev ? ntile - spb : (p.nblk - 1) * spb;
+    // running sums: the last block walked (first block in reverse) adds to no state that anyone reads
+    const int nit = own ? min(p.grp * spb, ntile - blk * spb) : p.rev ? ntile - spb : (p.nblk - 1) * spb;
     auto tile_of = [&](int it) { return own ? blk * spb + it : p.rev ? ntile - 1 - it : it; };
     auto ends_block = [&](int it) {
         const int ti = tile_of(it);
-        return own ? it == nit - 1 : p.rev ? ti % spb == 0 : (ti + 1) % spb == 0;
+        return own ? ((it + 1) % spb == 0 || it == nit - 1) : p.rev ? ti % spb == 0 : (ti + 1) % spb == 0;
     };
 
     if (tid == 0) {
@@ -236,6 +238,7 @@ __global__ void __launch_bounds__(kThreadsR, 1)
         // of the transposed state goes out as it lies, [slot][d_v][160] (bf16 running sums, or the block's own fp32
         // sums), the row sums through two small arrays in shared memory.
         float* zs = reinterpret_cast<float*>(smem + C::offMisc + 256);
+        float* zd = zs + 4 * 160;
         float run[80];                                       // running sums of this thread's half of its lane's columns
 #pragma unroll
         for (int i = 0; i < 80; ++i) run[i] = 0.f;
@@ -243,7 +246,7 @@ __global__ void __launch_bounds__(kThreadsR, 1)
             const int a = nf & 1;
             if (!rows_and3(mbar_wait(&bars[rFlush0 + a], (nf >> 1) & 1, abort_flag))) return false;
             tc_fence_after();
-            const int c = own ? blk : p.rev ? tile_of(it) / spb - 1 : (tile_of(it) + 1) / spb;
+            const int c = own ? blk + it / spb : p.rev ? tile_of(it) / spb - 1 : (tile_of(it) + 1) / spb;
             const size_t slot = (size_t)head * p.nblk + c;
             const size_t rowoff = (slot * p.dvw + (t < p.dvw ? t : 0)) * 160 + half * 80;
             // where the weights rows lie: d_v 64: lanes 64, 65 of this block's accumulator (own sums: added to the
@@ -263,6 +266,7 @@ __global__ void __launch_bounds__(kThreadsR, 1)
                 for (int i = 0; i < 16; ++i) {
                     run[j * 16 + i] += __uint_as_float(r[i]);
                     v[i] = run[j * 16 + i] * feature_weight(f0 + i);
+                    if (own) run[j * 16 + i] = 0.f;              // own sums: every block starts over
                 }
                 if (t < p.dvw) {
                     if (own) {
@@ -290,14 +294,21 @@ __global__ void __launch_bounds__(kThreadsR, 1)
                     }
                     if (lane < 4 && zlane) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) zrow[f0 + i] = v[i];
+                        for (int i = 0; i < 16; ++i) {
+                            // (d_v 128, own sums: the lane pair's running sum has grown by the block's own sum)
+                            if (DV != 64 && own) zd[(lane & 1) * 160 + f0 + i] = v[i] - zrow[f0 + i];
+                            zrow[f0 + i] = v[i];
+                        }
                     }
                 }
             }
             tc_fence_before();
             mbar_arrive(&bars[rFree0 + a]);                  // the accumulator may start over
             const bool good = rows_and3(true);               // the row sums' parts are written
-            if (tid < 160) (own ? p.zpart : p.sv)[slot * 160 + tid] = (zs[tid] + zs[160 + tid]) + (zs[320 + tid] + zs[480 + tid]);
+            if (tid < 160) {
+                if (own && DV != 64) p.zpart[slot * 160 + tid] = zd[tid] + zd[160 + tid];
+                else (own ? p.zpart : p.sv)[slot * 160 + tid] = (zs[tid] + zs[160 + tid]) + (zs[320 + tid] + zs[480 + tid]);
+            }
             return rows_and3(good);                          // ... and read, before the next block end writes them
         };
         fetch(0);
@@ -406,6 +417,9 @@ based_status launch_running(const void* x, const void* val, const float2* stats,
     p.W = W;
     p.nblk = (L + W - 1) / W;
     p.rev = rev;
+    // own sums: enough consecutive blocks per CTA to spread its fixed cost, while some waves of CTAs remain
+    // (B1 H32 L32768 d_v64: 1170 / 1099 / 1061 / 1078 us per backward call at 1 / 2 / 4 / 8 blocks per CTA)
+    p.grp = !part ? 1 : BH * p.nblk >= 1200 ? 4 : BH * p.nblk >= 600 ? 2 : 1;
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BASED_ERR_CUDA;
@@ -418,7 +432,7 @@ based_status launch_running(const void* x, const void* val, const float2* stats,
             configured[dev] = true;
         }
     }
-    block_state_tc_kernel<DV><<<part ? BH * p.nblk : BH, kThreadsR, C::kSmem, stream>>>(tv, p);
+    block_state_tc_kernel<DV><<<part ? BH * ((p.nblk + p.grp - 1) / p.grp) : BH, kThreadsR, C::kSmem, stream>>>(tv, p);
     note_launch();
     return check_launch("block_state_tc_kernel");
 }

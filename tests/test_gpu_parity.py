@@ -390,6 +390,26 @@ def test_prefill_backward_blockwise_many_blocks_against_fp32_path():
         assert ((a.float() - b).norm() / b.norm()).item() <= 1e-2 and ((a2.float() - b).norm() / b.norm()).item() <= 1e-2
 
 
+@pytest.mark.parametrize("H,L,d_v", [(8, 40960, 128), (4, 40900, 64)])
+def test_prefill_backward_blockwise_grouped_block_sums(H, L, d_v):
+    """Few heads, 160 blocks: the block states come from CTAs that take four (8 heads) or two (4 heads) consecutive
+    blocks each and write every block's own sums for the scan; against the fp32 path of the library."""
+    g_ = torch.Generator(device=DEV).manual_seed(L + H)
+    q = (torch.randn(1, H, L, 16, generator=g_, device=DEV) * 0.4).bfloat16()
+    k = (torch.randn(1, H, L, 16, generator=g_, device=DEV) * 0.4).bfloat16()
+    v = torch.randn(1, H, L, d_v, generator=g_, device=DEV).bfloat16()
+    dout = torch.randn(1, H, L, d_v, generator=g_, device=DEV).bfloat16()
+    out = based.based_prefill(q, k, v)
+    n0 = based.launch_count()
+    blk = based.based_prefill_backward(q, k, v, dout, out=out)
+    assert based.launch_count() - n0 == 6
+    ref = based.based_prefill_backward(q.float(), k.float(), v.float(), dout.float())
+    _poll()
+    for a, b in zip(blk, ref):
+        assert _grad_err(_np(a), _np(b)) <= TOL_BF16
+        assert ((a.float() - b).norm() / b.norm()).item() <= 1e-2
+
+
 def test_prefill_backward_tile_path_long_loops():
     """The tile path alone at a length where its loops are long (d' = 32 keeps it off the block-wise path): B1 H2
     L2048 d_v128, with and without the forward output, against the oracle."""
