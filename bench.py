@@ -694,6 +694,9 @@ def main():
                                             sym=True)
         torch.cuda.empty_cache()
         extras["backward"] = bench_backward(w, 5, 3, torch, based, dist_on, peaks)
+        torch.cuda.empty_cache()
+        extras["backward_cfg3"] = bench_backward(wl.CONFIGS["cfg3_1p3b_prefill"], 5, 3, torch, based, dist_on, peaks)
+        torch.cuda.empty_cache()
         extras["baseconv"] = bench_baseconv((8, 4096, 8192), 10, 3, torch, based, dist_on, peaks)
         extras["generation_graph"] = bench_generation_graph(wl.CONFIGS["cfg4_generation"], 512, 16, torch, based,
                                                             dist_on, peaks)
