@@ -91,6 +91,12 @@ __device__ __forceinline__ bool rows_and3(bool pred) {
         : "memory");
     return r != 0;
 }
+// one 256-bit store (the address a multiple of 32 bytes): a whole sector per lane where the lanes' rows lie apart
+__device__ __forceinline__ void st_global_256(void* dst, const uint32_t (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                 "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+}
 __device__ __forceinline__ float feature_weight(int f) {
     return f < 16 ? 0.25f : f < 32 ? 0.03125f : f < 152 ? 0.0625f : f == 152 ? 1.0f : 0.0f;
 }
@@ -270,9 +276,13 @@ __global__ void __launch_bounds__(kThreadsR, 1)
                 }
                 if (t < p.dvw) {
                     if (own) {
-                        float4* d4 = reinterpret_cast<float4*>(p.part + rowoff + j * 16);
+                        uint32_t w8[8];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                        for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) w8[i] = __float_as_uint(v[hh * 8 + i]);
+                            st_global_256(p.part + rowoff + j * 16 + hh * 8, w8);
+                        }
                     } else {
                         uint32_t o[8];
 #pragma unroll
@@ -280,9 +290,7 @@ __global__ void __launch_bounds__(kThreadsR, 1)
                             __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
                             o[i] = *reinterpret_cast<uint32_t*>(&h2);
                         }
-                        uint4* d4 = reinterpret_cast<uint4*>(p.st + rowoff + j * 16);
-                        d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                        d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                        st_global_256(p.st + rowoff + j * 16, o);       // 16 columns = one 32-byte sector of the lane's row
                     }
                 }
                 if (zwarp) {
