@@ -149,6 +149,35 @@ def _check(status: int, where: str):
         raise BasedError(status, where)
 
 
+# The C ABI takes bare pointers and cannot know how large the caller's buffers are; a state of the wrong
+# format or an output that is too short would make the kernels write past the allocation.  The binding is
+# the one place that sees the tensors, so it checks them before the call.
+def _state_rows(d_feat: int, flags: int) -> int:
+    return D_SYM if (int(flags) & BASED_STATE_SYM) else 1 + d_feat + d_feat * d_feat
+
+
+def _check_state(kv_state, z_state, B: int, H: int, d_feat: int, d_v: int, flags: int, required: bool):
+    if kv_state is None and z_state is None:
+        if required:
+            raise ValueError("kv_state and z_state are required")
+        return
+    if kv_state is None or z_state is None:
+        raise ValueError("kv_state and z_state come together")
+    if kv_state.dtype != torch.float32 or z_state.dtype != torch.float32:
+        raise TypeError("state tensors are fp32")
+    rows = _state_rows(d_feat, flags)
+    if tuple(kv_state.shape) != (B, H, rows, d_v) or tuple(z_state.shape) != (B, H, rows):
+        raise ValueError(f"state shapes must be kv [{B},{H},{rows},{d_v}] and z [{B},{H},{rows}] for these flags, "
+                         f"got {tuple(kv_state.shape)} and {tuple(z_state.shape)}")
+
+
+def _check_qkv(q, k, v, out=None):
+    if q.dim() != k.dim() or k.shape != q.shape or v.shape[:-1] != q.shape[:-1] or k.dtype != q.dtype or v.dtype != q.dtype:
+        raise ValueError("q, k, v shapes/dtypes disagree")
+    if out is not None and (out.shape != v.shape or out.dtype != v.dtype):
+        raise ValueError("out must have the shape and dtype of v")
+
+
 def based_prefill_workspace_bytes(B: int, H: int, L: int, d_feat: int, d_v: int, io: int) -> int:
     return int(lib().based_prefill_workspace_bytes(B, H, L, d_feat, d_v, io))
 
@@ -159,8 +188,8 @@ def based_prefill(q, k, v, out=None, kv_state=None, z_state=None, flags: int = B
     _dev(q, k, v, out, kv_state, z_state, workspace)
     B, H, L, d_feat = q.shape
     d_v = v.shape[-1]
-    if k.shape != q.shape or v.shape[:3] != q.shape[:3] or k.dtype != q.dtype or v.dtype != q.dtype:
-        raise ValueError("q, k, v shapes/dtypes disagree")
+    _check_qkv(q, k, v, out)
+    _check_state(kv_state, z_state, B, H, d_feat, d_v, flags, required=bool(int(flags) & BASED_STATE_CONTINUE))
     io = _dtype_code(q)
     if out is None:
         out = torch.empty_like(v)
@@ -181,8 +210,11 @@ def based_prefill_state(k, v, kv_state=None, z_state=None, flags: int = BASED_ST
     _dev(k, v, kv_state, z_state, workspace)
     B, H, L, d_feat = k.shape
     d_v = v.shape[-1]
-    if kv_state is None:
+    if v.shape[:3] != k.shape[:3] or v.dtype != k.dtype:
+        raise ValueError("k, v shapes/dtypes disagree")
+    if kv_state is None and z_state is None:
         kv_state, z_state = new_state(B, H, d_v, k.device, sym=bool(flags & BASED_STATE_SYM), d_feat=d_feat)
+    _check_state(kv_state, z_state, B, H, d_feat, d_v, flags, required=True)
     need = int(lib().based_prefill_state_workspace_bytes(B, H, L, d_feat, d_v, _dtype_code(k)))
     if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
         workspace = torch.empty(need, dtype=torch.uint8, device=k.device)
@@ -200,6 +232,9 @@ def based_prefill_backward(q, k, v, dout, flags: int = 0, workspace=None, stream
     _dev(q, k, v, dout, workspace, out)
     B, H, L, d_feat = q.shape
     d_v = v.shape[-1]
+    _check_qkv(q, k, v, out)
+    if dout.shape != v.shape or dout.dtype != v.dtype:
+        raise ValueError("dout must have the shape and dtype of v")
     need = int(lib().based_prefill_backward_workspace_bytes(B, H, L, d_v, _dtype_code(q)))
     if workspace is None or workspace.numel() * workspace.element_size() < need:
         workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
@@ -228,6 +263,8 @@ def based_prefill_static_scratch(q, k, v, out, kv_state=None, z_state=None, flag
     overlap on the GPU must be serialised by the caller: they share that one array."""
     _dev(q, k, v, out, kv_state, z_state)
     B, H, L, d_feat = q.shape
+    _check_qkv(q, k, v, out)
+    _check_state(kv_state, z_state, B, H, d_feat, v.shape[-1], flags, required=bool(int(flags) & BASED_STATE_CONTINUE))
     st = lib().based_prefill_static_scratch(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(kv_state), _ptr(z_state), B, H,
                                             L, d_feat, v.shape[-1], _dtype_code(q), flags, _stream(stream))
     _check(st, "based_prefill_static_scratch")
@@ -239,8 +276,8 @@ def based_decode_step(q, k, v, kv_state, z_state, out=None, stream=None):
     _dev(q, k, v, kv_state, z_state, out)
     B, H, d_feat = q.shape
     d_v = v.shape[-1]
-    if kv_state.dtype != torch.float32 or z_state.dtype != torch.float32:
-        raise TypeError("state tensors are fp32")
+    _check_qkv(q, k, v, out)
+    _check_state(kv_state, z_state, B, H, d_feat, d_v, 0, required=True)
     if out is None:
         out = torch.empty_like(v)
     st = lib().based_decode_step(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_state), _ptr(z_state), _ptr(out), B, H, d_feat,
@@ -254,10 +291,8 @@ def based_decode_step_sym(q, k, v, kv_sym, z_sym, out=None, stream=None):
     _dev(q, k, v, kv_sym, z_sym, out)
     B, H, d_feat = q.shape
     d_v = v.shape[-1]
-    if kv_sym.dtype != torch.float32 or z_sym.dtype != torch.float32:
-        raise TypeError("state tensors are fp32")
-    if kv_sym.shape != (B, H, D_SYM, d_v) or z_sym.shape != (B, H, D_SYM):
-        raise ValueError("symmetric state has 153 rows")
+    _check_qkv(q, k, v, out)
+    _check_state(kv_sym, z_sym, B, H, d_feat, d_v, BASED_STATE_SYM, required=True)
     if out is None:
         out = torch.empty_like(v)
     st = lib().based_decode_step_sym(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_sym), _ptr(z_sym), _ptr(out), B, H, d_feat,
@@ -271,6 +306,8 @@ def based_decode_step_flags(q, k, v, kv_state, z_state, flags: int, out=None, st
     _dev(q, k, v, kv_state, z_state, out)
     B, H, d_feat = q.shape
     d_v = v.shape[-1]
+    _check_qkv(q, k, v, out)
+    _check_state(kv_state, z_state, B, H, d_feat, d_v, flags, required=True)
     if out is None:
         out = torch.empty_like(v)
     st = lib().based_decode_step_flags(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_state), _ptr(z_state), _ptr(out), B, H,
@@ -283,6 +320,9 @@ def based_state_to_sym(kv_state, z_state, kv_sym=None, z_sym=None, stream=None):
     """[B,H,273,d_v], [B,H,273] -> symmetric [B,H,153,d_v], [B,H,153]."""
     _dev(kv_state, z_state, kv_sym, z_sym)
     B, H, _, d_v = kv_state.shape
+    _check_state(kv_state, z_state, B, H, D_FEAT, d_v, 0, required=True)
+    if kv_sym is not None or z_sym is not None:
+        _check_state(kv_sym, z_sym, B, H, D_FEAT, d_v, BASED_STATE_SYM, required=True)
     if kv_sym is None:
         kv_sym, z_sym = new_state(B, H, d_v, device=kv_state.device, sym=True)
     st = lib().based_state_to_sym(_ptr(kv_state), _ptr(z_state), _ptr(kv_sym), _ptr(z_sym), B, H, D_FEAT, d_v,
@@ -295,6 +335,9 @@ def based_state_from_sym(kv_sym, z_sym, kv_state=None, z_state=None, stream=None
     """Symmetric [B,H,153,d_v], [B,H,153] -> [B,H,273,d_v], [B,H,273]."""
     _dev(kv_sym, z_sym, kv_state, z_state)
     B, H, _, d_v = kv_sym.shape
+    _check_state(kv_sym, z_sym, B, H, D_FEAT, d_v, BASED_STATE_SYM, required=True)
+    if kv_state is not None or z_state is not None:
+        _check_state(kv_state, z_state, B, H, D_FEAT, d_v, 0, required=True)
     if kv_state is None:
         kv_state, z_state = new_state(B, H, d_v, device=kv_sym.device)
     st = lib().based_state_from_sym(_ptr(kv_sym), _ptr(z_sym), _ptr(kv_state), _ptr(z_state), B, H, D_FEAT, d_v,
@@ -339,6 +382,9 @@ def swa_forward(q, k, v, out=None, window: int = 64, softmax_scale: float = 0.0,
     """q,k,v [B,H,L,d] -> out; causal softmax over keys i-window+1..i; scale<=0 -> 1/sqrt(d)."""
     _dev(q, k, v, out)
     B, H, L, d = q.shape
+    _check_qkv(q, k, v, out)
+    if v.shape != q.shape:
+        raise ValueError("the sliding-window mixer takes q, k, v of one shape")
     if out is None:
         out = torch.empty_like(v)
     st = lib().swa_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, L, d, int(window), float(softmax_scale),

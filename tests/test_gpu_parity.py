@@ -11,7 +11,7 @@ import torch
 import oracle
 import paper_2402_18668_b200 as based
 from paper_2402_18668_b200 import workloads as wl
-from parity import TOL_BF16, TOL_F32, head_err, row_err, tol_for
+from parity import TOL_BF16, TOL_F32, assert_state_close, head_err, row_err, state_errs, tol_for
 
 pytestmark = pytest.mark.gpu
 
@@ -38,8 +38,7 @@ def test_cfg1_prefill_then_decode_fp32():
     y = based.based_prefill(q.to(DEV), k.to(DEV), v.to(DEV), kv_state=kv, z_state=z)
     _poll()
     assert row_err(_np(y), y_ref) <= TOL_F32
-    assert head_err(_np(kv), S_ref) <= TOL_F32
-    assert head_err(_np(z), z_ref) <= TOL_F32
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, "f32")
 
     S, zz = S_ref, z_ref
     for t in range(w.decode_steps):
@@ -47,8 +46,7 @@ def test_cfg1_prefill_then_decode_fp32():
         out = based.based_decode_step(qs[t].to(DEV), ks[t].to(DEV), vs[t].to(DEV), kv, z)
         assert row_err(_np(out), y_t) <= TOL_F32, f"decode step {t}"
     _poll()
-    assert head_err(_np(kv), S) <= TOL_F32
-    assert head_err(_np(z), zz) <= TOL_F32
+    assert_state_close(_np(kv), S, _np(z), zz, "f32")
 
 
 # --------------------------------------------------------------------------- prefill, element by element
@@ -66,8 +64,7 @@ def test_prefill_small_shapes(dtype, d_v, L):
     _poll()
     tol = tol_for(dtype)
     assert row_err(_np(out), y_ref) <= tol
-    assert head_err(_np(kv), S_ref) <= tol
-    assert head_err(_np(z), z_ref) <= tol
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, dtype)
     # without state pointers the outputs are the same
     out2 = based.based_prefill(q.to(DEV), k.to(DEV), v.to(DEV))
     assert torch.equal(out2, out)
@@ -87,8 +84,7 @@ def test_prefill_bf16_many_chunks(B, H, d_v, L):
     out = based.based_prefill(q.to(DEV), k.to(DEV), v.to(DEV), kv_state=kv, z_state=z)
     _poll()
     assert row_err(_np(out), y_ref) <= TOL_BF16
-    assert head_err(_np(kv), S_ref) <= TOL_BF16
-    assert head_err(_np(z), z_ref) <= TOL_BF16
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, "bf16")
 
 
 @pytest.mark.parametrize("dtype,d_v,L,L1", [("f32", 64, 200, 77), ("bf16", 128, 384, 128), ("bf16", 64, 450, 131)])
@@ -105,8 +101,7 @@ def test_prefill_continue_equals_one_pass(dtype, d_v, L, L1):
     _poll()
     tol = tol_for(dtype)
     assert row_err(_np(torch.cat([y1, y2], dim=2)), y_ref) <= tol
-    assert head_err(_np(kv), S_ref) <= tol
-    assert head_err(_np(z), z_ref) <= tol
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, dtype)
 
 
 # --------------------------------------------------------------------------- decode
@@ -130,8 +125,7 @@ def test_decode_step_from_given_state(dtype, d_v):
         out = torch.full_like(vs[t], float("nan"), device=DEV)
         based.based_decode_step(qs[t].to(DEV), ks[t].to(DEV), vs[t].to(DEV), kv, z, out=out)
         assert row_err(_np(out), y_t) <= tol, f"step {t}"
-        assert head_err(_np(kv), S) <= TOL_F32          # the state is fp32 for both io dtypes
-        assert head_err(_np(z), zz) <= TOL_F32
+        assert_state_close(_np(kv), S, _np(z), zz, "f32")          # the state is fp32 for both io dtypes
     _poll()
 
 
@@ -151,8 +145,8 @@ def test_decode_chain_equals_prefill_on_gpu():
     _poll()
     assert row_err(_np(y_chain), y_ref) <= TOL_F32
     assert row_err(_np(y_pre), y_ref) <= TOL_F32
-    assert head_err(_np(kv), S_ref) <= TOL_F32 and head_err(_np(kv2), S_ref) <= TOL_F32
-    assert head_err(_np(z), z_ref) <= TOL_F32 and head_err(_np(z2), z_ref) <= TOL_F32
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, "f32")
+    assert_state_close(_np(kv2), S_ref, _np(z2), z_ref, "f32")
 
 
 # --------------------------------------------------------------------------- d_v = 112
@@ -179,7 +173,7 @@ def test_head_dim_112_prefill_continue_and_decode(dtype, L):
                              vd[:, :, half:L].contiguous(), kv_state=kv, z_state=z, flags=based.BASED_STATE_CONTINUE)
     out[:, :, :half], out[:, :, half:] = o1, o2
     assert row_err(_np(out), y_ref[:, :, :L]) <= tol
-    assert head_err(_np(kv), S_ref) <= tol and head_err(_np(z), z_ref) <= tol
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, dtype)
     kvs, zs = based.based_state_to_sym(kv, z)
     for t in range(L, L + T):
         args = (qd[:, :, t].contiguous(), kd[:, :, t].contiguous(), vd[:, :, t].contiguous())
@@ -388,6 +382,11 @@ def test_prefill_backward_blockwise_many_blocks_against_fp32_path():
     for a, a2, b in zip(blk, blk2, ref):
         assert _grad_err(_np(a), _np(b)) <= TOL_BF16 and _grad_err(_np(a2), _np(b)) <= TOL_BF16
         assert ((a.float() - b).norm() / b.norm()).item() <= 1e-2 and ((a2.float() - b).norm() / b.norm()).item() <= 1e-2
+    # one head against the oracle itself (the quadratic form in fp64)
+    sl = (slice(0, 1), slice(1, 2))
+    want = oracle.linattn_backward(_np(q[sl]), _np(k[sl]), _np(v[sl]), _np(dout[sl]))
+    for a, a2, wnt in zip(blk, blk2, want):
+        assert _grad_err(_np(a[sl]), wnt) <= TOL_BF16 and _grad_err(_np(a2[sl]), wnt) <= TOL_BF16
 
 
 @pytest.mark.parametrize("H,L,d_v", [(8, 40960, 128), (4, 40900, 64)])
@@ -444,7 +443,7 @@ def test_other_feature_dimensions_full_length_sampled(d_feat):
         sl = (slice(b, b + 1), slice(h, h + 1))
         y_ref, S_ref, z_ref = oracle.linattn_quadratic(_np(q[sl]), _np(k[sl]), _np(v[sl]))
         assert row_err(_np(out[sl]), y_ref) <= TOL_BF16
-        assert head_err(_np(kv[sl]), S_ref) <= TOL_BF16 and head_err(_np(z[sl]), z_ref) <= TOL_BF16
+        assert_state_close(_np(kv[sl]), S_ref, _np(z[sl]), z_ref, "bf16")
 
 
 def test_autograd_wrapper_routes_gradients_through_the_library():
@@ -491,7 +490,7 @@ def test_other_feature_dimensions_prefill_continue_decode(dtype, d_feat, L, d_v)
                                     flags=based.BASED_STATE_CONTINUE if half > 0 else based.BASED_STATE_ZERO_INIT))
     out = torch.cat(outs, dim=2)
     assert row_err(_np(out), y_ref[:, :, :L]) <= tol
-    assert head_err(_np(kv), S_ref) <= tol and head_err(_np(z), z_ref) <= tol
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, dtype)
     for t in range(L, L + T):
         o = based.based_decode_step(qd[:, :, t].contiguous(), kd[:, :, t].contiguous(), vd[:, :, t].contiguous(), kv, z)
         assert row_err(_np(o), y_ref[:, :, t]) <= tol, f"token {t}"
@@ -668,8 +667,7 @@ def test_decode_step_sym_from_folded_state(dtype, d_v):
         out = torch.full_like(vs[t], float("nan"), device=DEV)
         based.based_decode_step_sym(qs[t].to(DEV), ks[t].to(DEV), vs[t].to(DEV), kv, z, out=out)
         assert row_err(_np(out), y_t) <= tol, f"step {t}"
-        assert head_err(_np(kv), S) <= TOL_F32
-        assert head_err(_np(z), zz) <= TOL_F32
+        assert_state_close(_np(kv), S, _np(z), zz, "f32")
     _poll()
 
 
@@ -688,7 +686,7 @@ def test_state_conversions_and_prefill_to_sym_decode(d_v):
     based.based_prefill(qd[:, :, :L].contiguous(), kd[:, :, :L].contiguous(), vd[:, :, :L].contiguous(),
                         kv_state=kv, z_state=z)
     kvs, zs = based.based_state_to_sym(kv, z)
-    assert head_err(_np(kvs), Ss_ref) <= TOL_BF16 and head_err(_np(zs), zs_ref) <= TOL_BF16
+    assert_state_close(_np(kvs), Ss_ref, _np(zs), zs_ref, "bf16")
     # the fold itself is exact fp32 arithmetic on the GPU's own state
     Ss_own, zs_own = oracle.state_to_sym(_np(kv), _np(z))
     assert head_err(_np(kvs), Ss_own) <= 1e-6 and head_err(_np(zs), zs_own) <= 1e-6
@@ -719,12 +717,12 @@ def test_prefill_with_symmetric_state_in_and_out(dtype, L, d_v):
     out1 = based.based_prefill(qd[:, :, :half].contiguous(), kd[:, :, :half].contiguous(), vd[:, :, :half].contiguous(),
                                kv_state=kv, z_state=z, flags=based.BASED_STATE_SYM)
     assert row_err(_np(out1), y_ref[:, :, :half]) <= tol
-    assert head_err(_np(kv), S_half) <= tol and head_err(_np(z), z_half) <= tol
+    assert_state_close(_np(kv), S_half, _np(z), z_half, dtype)
     out2 = based.based_prefill(qd[:, :, half:].contiguous(), kd[:, :, half:].contiguous(), vd[:, :, half:].contiguous(),
                                kv_state=kv, z_state=z, flags=based.BASED_STATE_SYM | based.BASED_STATE_CONTINUE)
     _poll()
     assert row_err(_np(out2), y_ref[:, :, half:]) <= tol
-    assert head_err(_np(kv), S_ref) <= tol and head_err(_np(z), z_ref) <= tol
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, dtype)
 
 
 def test_sym_and_full_decode_agree_at_generation_batch():
@@ -868,8 +866,7 @@ def test_full_size_prefill_sampled(name):
             b, h = divmod(bh, w.H)
             _, S_ref, z_ref = oracle.linattn_recurrent(_np(q[b:b + 1, h:h + 1]), _np(k[b:b + 1, h:h + 1]),
                                                        _np(v[b:b + 1, h:h + 1]))
-            assert head_err(_np(kv[b:b + 1, h:h + 1]), S_ref) <= TOL_BF16
-            assert head_err(_np(z[b:b + 1, h:h + 1]), z_ref) <= TOL_BF16
+            assert_state_close(_np(kv[b:b + 1, h:h + 1]), S_ref, _np(z[b:b + 1, h:h + 1]), z_ref, "bf16")
 
 
 def test_full_size_mixer_pair_sampled():
@@ -881,7 +878,11 @@ def test_full_size_mixer_pair_sampled():
     vd = v.to(DEV)
     out_lin = based.based_prefill(q.to(DEV), k.to(DEV), vd).cpu()
     out_swa = based.swa_forward(qs.to(DEV), ks.to(DEV), vd, window=w.swa_window).cpu()
+    # the same call returning its state: outputs must not depend on it, and the state is checked on two heads
+    kv, z = based.new_state(w.B, w.H, w.d_v)
+    out_lin2 = based.based_prefill(q.to(DEV), k.to(DEV), vd, kv_state=kv, z_state=z).cpu()
     _poll()
+    assert torch.equal(out_lin, out_lin2)
     rng = np.random.default_rng(1)
     worst = 0.0
     for bh in (0, 13, w.B * w.H - 1):
@@ -890,6 +891,11 @@ def test_full_size_mixer_pair_sampled():
         for i in _sample_rows(w.L, 12, rng):
             worst = max(worst, row_err(_np(out_lin[b, h, i]), oracle.linattn_row(qh, kh, vh, i)))
     assert worst <= TOL_BF16
+    for bh in (5, w.B * w.H - 1):
+        b, h = divmod(bh, w.H)
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        _, S_ref, z_ref = oracle.linattn_recurrent(_np(q[sl]), _np(k[sl]), _np(v[sl]))
+        assert_state_close(_np(kv[sl]), S_ref, _np(z[sl]), z_ref, "bf16")
     # the sliding-window oracle is cheap enough to check four whole heads
     for bh in (0, 7, 22, w.B * w.H - 1):
         b, h = divmod(bh, w.H)
@@ -916,10 +922,11 @@ def test_full_size_wide_window_sampled(window):
 
 
 def test_full_size_generation_sampled():
-    """cfg 4: batch 128 prompt prefill, then decode steps from the resulting fp32 state
-    (a reduced number of steps here; the benchmark runs all 1024)."""
+    """cfg 4: batch 128 prompt prefill, then all 1024 decode steps from the resulting fp32 state; three heads
+    are followed by the oracle step by step (outputs of every step, state after the prompt and at the end)."""
     w = wl.CONFIGS["cfg4_generation"]
-    steps = 64
+    steps = w.decode_steps
+    assert steps == 1024
     gen = wl.generator(0)
     q, k, v = wl.prefill_inputs(w, gen)
     qs, ks, vs = wl.decode_inputs(w, gen, steps=steps)
@@ -932,25 +939,25 @@ def test_full_size_generation_sampled():
         sl = (slice(b, b + 1), slice(h, h + 1))
         y_ref, S, zz = oracle.linattn_recurrent(_np(q[sl]), _np(k[sl]), _np(v[sl]))
         assert row_err(_np(out[sl]), y_ref) <= TOL_BF16
-        assert head_err(_np(kv[sl]), S) <= TOL_BF16
+        assert_state_close(_np(kv[sl]), S, _np(z[sl]), zz, "bf16")
         refs[bh] = (S, zz)
     del out
     qsd, ksd, vsd = qs.to(DEV), ks.to(DEV), vs.to(DEV)
+    bs, hs = [bh // w.H for bh in heads], [bh % w.H for bh in heads]
+    got = torch.empty(steps, len(heads), w.d_v, dtype=vsd.dtype, device=DEV)
     for t in range(steps):
         o = based.based_decode_step(qsd[t], ksd[t], vsd[t], kv, z)
-        for bh in heads:
-            b, h = divmod(bh, w.H)
-            sl = (slice(b, b + 1), slice(h, h + 1))
-            S, zz = refs[bh]
-            y_t, S, zz = oracle.decode_step(_np(qs[t][sl]), _np(ks[t][sl]), _np(vs[t][sl]), S, zz)
-            refs[bh] = (S, zz)
-            assert row_err(_np(o[sl]), y_t) <= TOL_BF16, (t, bh)
+        got[t] = o[bs, hs]
     _poll()
-    for bh in heads:
+    got = _np(got)
+    for n, bh in enumerate(heads):
         b, h = divmod(bh, w.H)
         sl = (slice(b, b + 1), slice(h, h + 1))
-        assert head_err(_np(kv[sl]), refs[bh][0]) <= TOL_BF16
-        assert head_err(_np(z[sl]), refs[bh][1]) <= TOL_BF16
+        S, zz = refs[bh]
+        for t in range(steps):
+            y_t, S, zz = oracle.decode_step(_np(qs[t][sl]), _np(ks[t][sl]), _np(vs[t][sl]), S, zz)
+            assert row_err(got[t, n], y_t.reshape(-1)) <= TOL_BF16, (t, bh)
+        assert_state_close(_np(kv[sl]), S, _np(z[sl]), zz, "bf16")
 
 
 # --------------------------------------------------------------------------- errors on the device box
@@ -999,10 +1006,10 @@ def test_prefill_state_matches_oracle_and_prefill(dtype, d_feat, L, d_v, sym):
     tol = tol_for(dtype)
     kv, z = based.based_prefill_state(kd, vd, flags=fl)
     _poll()
-    assert head_err(_np(kv), S_ref) <= tol and head_err(_np(z), z_ref) <= tol
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, dtype)
     # twice the block on top of itself: CONTINUE adds
     kv2, z2 = based.based_prefill_state(kd, vd, kv_state=kv.clone(), z_state=z.clone(), flags=fl | based.BASED_STATE_CONTINUE)
-    assert head_err(_np(kv2), 2 * S_ref) <= tol and head_err(_np(z2), 2 * z_ref) <= tol
+    assert_state_close(_np(kv2), 2 * S_ref, _np(z2), 2 * z_ref, dtype)
     if L >= 2:
         half = L // 2
         kvh, zh = based.based_prefill_state(kd[:, :, :half].contiguous(), vd[:, :, :half].contiguous(), flags=fl)
@@ -1010,7 +1017,7 @@ def test_prefill_state_matches_oracle_and_prefill(dtype, d_feat, L, d_v, sym):
                                   kv_state=kvh, z_state=zh, flags=fl | based.BASED_STATE_CONTINUE)
         _poll()
         assert row_err(_np(out), y_ref[:, :, half:]) <= tol
-        assert head_err(_np(kvh), S_ref) <= tol and head_err(_np(zh), z_ref) <= tol
+        assert_state_close(_np(kvh), S_ref, _np(zh), z_ref, dtype)
 
 
 def test_sequence_parallel_helpers_on_one_process():
@@ -1051,13 +1058,69 @@ def test_extreme_input_scales_bf16(qk_scale, v_scale):
     dq, dk, dv = based.based_prefill_backward(qd, kd, vd, gd, out=out)
     _poll()
     assert row_err(_np(out), y_ref) <= TOL_BF16
-    assert head_err(_np(kv), S_ref) <= TOL_BF16 and head_err(_np(z), z_ref) <= TOL_BF16
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, "bf16")
     # gradients: relative to each head's largest entry (no absolute floor: the scales span eight decades)
     for got, want in ((dq, rq), (dk, rk), (dv, rv)):
         got, want = _np(got).reshape(B * H, -1).astype(np.float64), np.asarray(want).reshape(B * H, -1)
         scale = np.abs(want).max(axis=1)
         err = np.abs(got - want).max(axis=1)
         assert np.all(err <= TOL_BF16 * np.maximum(scale, 1e-30) + 1e-30), (err, scale)
+
+
+# --------------------------------------------------------------------------- state rows, block by block
+# B, H, L: one CTA per head (many heads), the cfg-2 shape (two CTAs per head, the second one recomputing the state
+# of the first one's chunks), a long sequence (segments with a state pass), and a short ragged one
+_STATE_SHAPES = [(1, 80, 700), (4, 16, 2048), (1, 2, 16500), (2, 3, 300)]
+
+
+@pytest.mark.parametrize("qk_scale", [1.0, 4.0])
+@pytest.mark.parametrize("d_v", [64, 112, 128])
+@pytest.mark.parametrize("B,H,L", _STATE_SHAPES)
+def test_prefill_state_rows_every_mode(B, H, L, d_v, qk_scale):
+    """The ABI-visible state of the bf16 prefill, checked per feature block and per state row (a wrong factor on
+    the second-order rows must not hide behind the much larger constant row), at input scales where those rows
+    carry weight, for every way the state leaves the kernel: from the empty state, continued from a given
+    state, in the 153-row symmetric format (both), and from the state-only entry point."""
+    if (B, H, L) == (4, 16, 2048) and d_v == 112:
+        pytest.skip("the 64-head shape runs at the two benchmark widths")
+    w = wl.Workload("staterows", B, H, L, 16, d_v, "bf16", qk_scale)
+    q, k, v = wl.prefill_inputs(w, wl.generator(B * 7 + L + d_v + int(qk_scale)))
+    L1 = (L // 3) | 1                                      # ragged split point for the continued runs
+    y_ref, S_ref, z_ref = oracle.linattn_recurrent(_np(q), _np(k), _np(v))
+    Ss_ref, zs_ref = oracle.state_to_sym(S_ref, z_ref)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    cut = lambda t, a, b: t[:, :, a:b].contiguous()
+    for sym in (False, True):
+        flag = based.BASED_STATE_SYM if sym else 0
+        want = (Ss_ref, zs_ref) if sym else (S_ref, z_ref)
+        what = f"sym={sym}"
+        # from the empty state (buffers poisoned: they must not be read)
+        kv, z = based.new_state(B, H, d_v, sym=sym)
+        kv.fill_(float("nan")); z.fill_(float("nan"))
+        out = based.based_prefill(qd, kd, vd, kv_state=kv, z_state=z, flags=flag)
+        _poll()
+        assert row_err(_np(out), y_ref) <= TOL_BF16
+        assert_state_close(_np(kv), want[0], _np(z), want[1], "bf16", what + " zero-init")
+        # continued from the state of the first L1 tokens
+        kv, z = based.new_state(B, H, d_v, sym=sym)
+        y1 = based.based_prefill(cut(qd, 0, L1), cut(kd, 0, L1), cut(vd, 0, L1), kv_state=kv, z_state=z, flags=flag)
+        y2 = based.based_prefill(cut(qd, L1, L), cut(kd, L1, L), cut(vd, L1, L), kv_state=kv, z_state=z,
+                                 flags=flag | based.BASED_STATE_CONTINUE)
+        _poll()
+        assert row_err(_np(torch.cat([y1, y2], dim=2)), y_ref) <= TOL_BF16
+        assert_state_close(_np(kv), want[0], _np(z), want[1], "bf16", what + " continue")
+        # the state-only entry point, in one piece and added to the first piece's state
+        kv, z = based.new_state(B, H, d_v, sym=sym)
+        kv.fill_(float("nan")); z.fill_(float("nan"))
+        based.based_prefill_state(kd, vd, kv_state=kv, z_state=z, flags=flag)
+        _poll()
+        assert_state_close(_np(kv), want[0], _np(z), want[1], "bf16", what + " state-only")
+        kv, z = based.new_state(B, H, d_v, sym=sym)
+        based.based_prefill_state(cut(kd, 0, L1), cut(vd, 0, L1), kv_state=kv, z_state=z, flags=flag)
+        based.based_prefill_state(cut(kd, L1, L), cut(vd, L1, L), kv_state=kv, z_state=z,
+                                  flags=flag | based.BASED_STATE_CONTINUE)
+        _poll()
+        assert_state_close(_np(kv), want[0], _np(z), want[1], "bf16", what + " state-only continue")
 
 
 # --------------------------------------------------------------------------- benchmark arms
