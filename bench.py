@@ -2,16 +2,30 @@
 """Benchmark of the Based hot path on B200 (one process per GPU).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+                    [--scaling weak|strong]
 
 Prints ONE JSON line on rank 0.  The headline `value` is prefill tokens/s of
-`based_prefill` on the named workload (device-resident inputs, rotating buffer sets
-larger than L2); the same line carries the decode-step and sliding-window results
-(`decode`, `swa`), the other prefill configurations (`prefill_configs`), the
-end-to-end number through host buffers (`e2e`), the roofline of the dominant kernel
-and the CPU oracle timed on the host cores (`cpu_baseline`).
+`based_prefill` on the named workload (default: the 1.3B-layer shape, the largest
+single-GPU prefill configuration; device-resident inputs, rotating buffer sets larger
+than L2); the same line carries the decode-step and sliding-window results (`decode`,
+`swa`), the other prefill configurations (`prefill_configs`), the end-to-end number
+through host buffers (`e2e`), the roofline of the dominant kernel, the CPU oracle timed
+on the host cores (`cpu_baseline`) and, last, a compact `summary` of every
+configuration's time and roofline fraction.
+
+Every prefill arm is timed twice: a short region (one CUDA-graph replay of the K calls:
+a burst at the full clock, held against the burst tensor peak) and a region of at least
+half a second of back-to-back replays (`sustained`: under the power limit the SM clock
+settles lower; held against the sustained tensor peak, with the SM clock sampled in
+that region alone).
 
 Every (b, h) head is independent, so N GPUs run N copies of the per-GPU workload with
-no data-path collective ("weak" scaling); time is the max over ranks.
+no data-path collective ("weak" scaling) or split one batch's heads (`--scaling strong`);
+time is the max over ranks.  Run as `python bench.py --gpus N` it starts its N ranks
+itself (torch.distributed.run on 127.0.0.1); under torchrun it takes its rank from the
+environment.  With more than one rank the line also carries `seqpar`: the mixer pair with
+the sequence cut across the ranks (one all-gather of block states, one halo exchange),
+checked on every rank against the one-GPU result.
 """
 from __future__ import annotations
 
@@ -35,6 +49,7 @@ L2_BYTES = 126 * 1024 * 1024
 # processed.  Written bytes still resident in L2 when a launch ends are not in these figures.
 NCU_TRAFFIC = {
     "cfg2_360m_prefill": 25.23e6,                 # profiles/prefill_tc_kernel_dv64_cfg2.md (output stays in L2)
+    "cfg3_1p3b_prefill": 1.6 * (104.94e6 + 43.89e6),  # profiles/prefill_tc_kernel_dv128.md, 80 -> 128 heads (part of the output still in L2)
     "cfg4_generation": 2 * (144.59e6 + 88.45e6),  # profiles/decode_step_kernel_dv128.md, 1024 -> 2048 heads
     "cfg5_mixer_pair:swa": 2 * (201.37e6 + 43.87e6),  # profiles/swa_tc_kernel.md, 16 -> 32 heads
     "baseconv": 4 * (272.67e6 + 96.72e6),         # profiles/baseconv_gate_kernel.md, batch 2 -> 8 (part of the writes still in L2)
@@ -62,6 +77,7 @@ class ClockSampler:
     def __init__(self, index: int, period_s: float = 0.02):
         self.index, self.period = index, period_s
         self.samples, self.reasons = [], set()
+        self.log = []           # (time, MHz, reason mask) of every sample, for per-region statistics
         self.max_mhz = None
         self._stop = threading.Event()
         self._thread = None
@@ -90,12 +106,20 @@ class ClockSampler:
                     mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)) if hasattr(
                         nv, "nvmlDeviceGetCurrentClocksEventReasons") else int(
                         nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                    self.log.append((time.perf_counter(), self.samples[-1], mask))
                     for name, bit in {**self.BAD, **self.NOTE}.items():
                         if mask & bit:
                             self.reasons.add(name)
             except Exception:
                 pass
             time.sleep(self.period)
+
+    def region(self, t0: float, t1: float):
+        """Median SM clock and the reasons seen between two perf_counter stamps."""
+        sel = [(m, k) for (t, m, k) in list(self.log) if t0 <= t <= t1]
+        reasons = sorted({name for _, k in sel for name, bit in {**self.BAD, **self.NOTE}.items() if k & bit})
+        return {"sm_mhz": statistics.median([m for m, _ in sel]) if sel else None, "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(sel)}
 
     def stop(self):
         self._stop.set()
@@ -130,13 +154,19 @@ def prefill_alg_bytes(w, with_state: bool) -> float:
     return b
 
 
-def time_region(fn_step, steps: int, warmup: int, torch, dist_on: bool, graph: bool = False):
+def time_region(fn_step, steps: int, warmup: int, torch, dist_on: bool, graph: bool = False, sustain_s: float = 0.0,
+                sampler=None):
     """W warm-up steps, then EXACTLY K steps between two events on the current stream, with a
     barrier and a device synchronise on both sides.  Returns ms for the K steps (max over ranks
     when distributed).  With graph=True the K calls are captured once into a CUDA graph and the
     timed region is one replay of it, so that microsecond-scale kernels are not timed through
-    the Python launch loop; every step still goes through the library's public entry point."""
+    the Python launch loop; every step still goes through the library's public entry point.
+
+    sustain_s > 0 (graph mode): a second region follows, of as many back-to-back replays as fill
+    that many seconds; returns (ms, {...}) with the time per step there and the SM clock sampled
+    in that region alone."""
     import torch.distributed as dist
+    from paper_2402_18668_b200.dist import max_over_ranks
     for i in range(warmup):
         fn_step(i)
     torch.cuda.synchronize()
@@ -152,25 +182,39 @@ def time_region(fn_step, steps: int, warmup: int, torch, dist_on: bool, graph: b
         torch.cuda.current_stream().wait_stream(side)
         g.replay()                      # untimed: first replay uploads the graph
         torch.cuda.synchronize()
-    if dist_on:
-        dist.barrier()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    if g is not None:
-        g.replay()
-    else:
-        for i in range(steps):
-            fn_step(warmup + i)
-    e1.record()
-    torch.cuda.synchronize()
-    if dist_on:
-        dist.barrier()
-    ms = e0.elapsed_time(e1)
-    if dist_on:
-        from paper_2402_18668_b200.dist import max_over_ranks
-        ms = max_over_ranks(ms, device="cuda")
-    return ms
+
+    def timed(replays: int):
+        if dist_on:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        e0.record()
+        if g is not None:
+            for _ in range(replays):
+                g.replay()
+        else:
+            for i in range(steps):
+                fn_step(warmup + i)
+        e1.record()
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+        if dist_on:
+            dist.barrier()
+        ms = e0.elapsed_time(e1)
+        return (max_over_ranks(ms, device="cuda") if dist_on else ms), t0, t1
+
+    ms, _, _ = timed(1)
+    if not (sustain_s > 0 and g is not None):
+        return ms
+    replays = max(2, int(-(-sustain_s * 1e3 // max(ms, 1e-3))))
+    if dist_on:                         # every rank must enqueue the same number of replays
+        replays = int(max_over_ranks(float(replays), device="cuda"))
+    ms_s, t0, t1 = timed(replays)
+    sus = {"us_per_step": ms_s * 1e3 / (replays * steps), "region_s": ms_s * 1e-3, "replays": replays}
+    if sampler is not None:
+        sus["clocks"] = sampler.region(t0, t1)
+    return ms, sus
 
 
 def device_inputs(w, n_sets: int, torch, seed: int = 0):
@@ -192,7 +236,9 @@ def n_sets_for(bytes_per_set: float) -> int:
 
 
 # --------------------------------------------------------------------------- the arms
-def bench_prefill(w, steps, warmup, torch, based, dist_on, peaks):
+def bench_prefill(w, steps, warmup, torch, based, dist_on, peaks, sampler=None, sustain_s: float = 0.0, world: int = 1):
+    """Device-resident prefill of workload w (this rank's share of it).  `world` only scales the whole-job
+    token count of a strong-scaling run, where w is already this rank's slice of the heads."""
     with_state = w.return_state
     per_set = prefill_alg_bytes(w, with_state)
     sets = device_inputs(w, n_sets_for(per_set), torch)
@@ -211,8 +257,9 @@ def bench_prefill(w, steps, warmup, torch, based, dist_on, peaks):
     for i in range(2):
         step(i)
     per_step = (based.launch_count() - n0) // 2
-    ms = time_region(step, steps, warmup, torch, dist_on, graph=True)
-    launches = per_step * steps
+    r = time_region(step, steps, warmup, torch, dist_on, graph=True, sustain_s=sustain_s, sampler=sampler)
+    ms, sus = r if isinstance(r, tuple) else (r, None)
+    launches = per_step * steps * (1 + (sus["replays"] if sus else 0))
     assert based.based_poll_error() == 0
     t = ms * 1e-3 / steps
     tokens = w.B * w.L
@@ -224,6 +271,17 @@ def bench_prefill(w, steps, warmup, torch, based, dist_on, peaks):
         "frac_hbm_peak": per_set / t / 1e9 / peaks["hbm_gbs"],
         "buffer_sets": len(sets), "launches_per_step": per_step, "timed_as": "one CUDA-graph replay of the K calls",
     }
+    if sus:
+        ts = sus["us_per_step"] * 1e-6
+        mhz = (sus.get("clocks") or {}).get("sm_mhz")
+        res["sustained"] = {
+            "us_per_step": sus["us_per_step"], "tokens_per_s": tokens / ts, "region_s": sus["region_s"],
+            "alg_tflops": flops / ts / 1e12, "peak": peaks["bf16_tflops_sustained"],
+            "frac_tensor_peak_sustained": flops / ts / 1e12 / peaks["bf16_tflops_sustained"],
+            "us_x_mhz": None if mhz is None else sus["us_per_step"] * mhz,
+            "clocks": sus.get("clocks"),
+            "timed_as": f"{sus['replays']} back-to-back replays of the K-call graph",
+        }
     return res, launches, sets
 
 
@@ -551,6 +609,13 @@ def bench_backward(w, steps, warmup, torch, based, dist_on, peaks):
     }
 
 
+def oracle_sample_heads(w) -> int:
+    """Heads of the workload that one timed oracle call processes: about a second of CPU work
+    (the recurrent form costs about 4 * 273 * d_v fp64 flops per token and head)."""
+    per_head = 4.0 * 273 * w.d_v * w.L
+    return max(1, min(w.B * w.H, int(3.0e10 // per_head)))
+
+
 def cpu_oracle_sample(w, budget_heads: int):
     """The oracle's recurrent form, as it stands, on the first `budget_heads` heads of the
     workload's seeded host inputs.  Returns (tokens/s scaled to whole tokens, cores, text)."""
@@ -569,24 +634,99 @@ def cpu_oracle_sample(w, budget_heads: int):
         f"{dt:.2f} s; tokens/s = token-heads/s / H")
 
 
+def bench_seqpar(w, steps, warmup, torch, based, dist_on, peaks):
+    """The mixer pair with the sequence cut across the ranks (rank r holds the r-th block of tokens):
+    linear attention through dist.sequence_parallel_prefill (block states all-gathered, one continued
+    prefill) and the sliding window through dist.sequence_parallel_swa (w - 1 keys and values from the
+    neighbour).  Every rank holds the whole seeded input, so it can check its block against the one-GPU
+    call on the same data.  Time: events around the K steps, max over ranks."""
+    import torch.distributed as dist
+    from paper_2402_18668_b200 import dist as bd
+    rank, n = bd.world()
+    g = torch.Generator(device="cuda").manual_seed(5)
+    dt = w.torch_dtype
+    q = torch.randn(w.B, w.H, w.L, w.d_feat, generator=g, device="cuda").mul_(w.qk_scale).to(dt)
+    k = torch.randn(w.B, w.H, w.L, w.d_feat, generator=g, device="cuda").mul_(w.qk_scale).to(dt)
+    v = torch.randn(w.B, w.H, w.L, w.d_v, generator=g, device="cuda").to(dt)
+    qs = torch.randn(w.B, w.H, w.L, w.swa_d, generator=g, device="cuda").to(dt)
+    ks = torch.randn(w.B, w.H, w.L, w.swa_d, generator=g, device="cuda").to(dt)
+    per = -(-w.L // n)
+    lo, hi = min(w.L, rank * per), min(w.L, (rank + 1) * per)
+    cut = lambda t: t[:, :, lo:hi].contiguous()
+    qb, kb, vb, qsb, ksb = cut(q), cut(k), cut(v), cut(qs), cut(ks)
+    window = w.swa_window or 64
+
+    def step(i):
+        out_lin, _, _ = bd.sequence_parallel_prefill(qb, kb, vb)
+        out_swa = bd.sequence_parallel_swa(qsb, ksb, vb, window)
+        return out_lin, out_swa
+
+    out_lin, out_swa = step(0)
+    ref_lin = based.based_prefill(q, k, v)[:, :, lo:hi].float()
+    ref_swa = based.swa_forward(qs, ks, v, window=window)[:, :, lo:hi].float()
+
+    def rowerr(a, b):
+        num = (a.float() - b).abs().amax(dim=-1)
+        return float((num / b.abs().amax(dim=-1).clamp_min(1e-30)).max())
+    err = max(rowerr(out_lin, ref_lin), rowerr(out_swa, ref_swa))
+    err = bd.max_over_ranks(err, device="cuda")
+    del ref_lin, ref_swa
+    ms = time_region(step, steps, warmup, torch, dist_on)
+    assert based.based_poll_error() == 0
+    t = ms * 1e-3 / steps
+    return {"workload": f"{w.name}: sequence cut into {n} blocks of {per} tokens", "metric": "mixer_pair_tokens_per_s",
+            "value": w.B * w.L / t, "unit": "tokens/s", "ms_per_step": t * 1e3, "ranks": n,
+            "max_row_err_vs_one_gpu": err, "parity_ok": bool(err <= 2e-2),
+            "exchange": "all-gather of block states + one halo send (NCCL)" if n > 1 else "none (one rank)"}
+
+
 # --------------------------------------------------------------------------- main
+def respawn_under_torchrun(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N ranks (one per GPU) on this node and
+    pass their output through.  NCCL's own log of the communicator set-up is kept (in a file per process,
+    so that stdout stays the one JSON line)."""
+    import socket
+    import subprocess
+    import tempfile
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_FILE", str(Path(tempfile.gettempdir()) / "based_bench_nccl.%h.%p.log"))
+    env["BASED_BENCH_SPAWNED"] = "1"
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), str(Path(__file__).resolve()), *sys.argv[1:]]
+    return subprocess.call(cmd, env=env)
+
+
+def frac_str(x):
+    return None if x is None else round(float(x), 4)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2_360m_prefill")
+    ap.add_argument("--workload", default="cfg3_1p3b_prefill")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="strong: the headline batch's heads (and the generation batch's) are split over the ranks")
     ap.add_argument("--skip-extras", action="store_true", help="only the headline prefill workload")
     ap.add_argument("--profile", choices=["prefill", "decode", "decode_sym", "swa", "swa_decode", "generation_graph", "baseconv", "backward",
-                             "prefill_dfeat"],
+                             "prefill_dfeat", "seqpar"],
                     help="run only this arm on --shape (small cases for ncu captures) and print its result")
     ap.add_argument("--shape", default="", help="B,H,L,d_v for --profile (defaults to the arm's benchmark shape)")
     ap.add_argument("--window", type=int, default=0, help="--profile swa: window (default: the workload's 64)")
     ap.add_argument("--d-feat", type=int, default=32, help="--profile prefill_dfeat: feature dimension (8, 24, 32)")
+    ap.add_argument("--sustain", type=float, default=0.5, help="seconds of the sustained timing region (0: skip it)")
     args = ap.parse_args()
     if args.warmup < 3 and not args.profile:
         args.warmup = 3
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(respawn_under_torchrun(args.gpus))
 
     from paper_2402_18668_b200 import workloads as wl
     w = wl.CONFIGS[args.workload]
@@ -597,16 +737,17 @@ def main():
         # the reference arm of this build is the CPU oracle: rank 0 alone runs it
         if rank != 0:
             return
+        heads = oracle_sample_heads(w)
         vals = []
         for _ in range(args.warmup + args.steps):
-            v, cores, sample = cpu_oracle_sample(w, budget_heads=16)
+            v, cores, sample = cpu_oracle_sample(w, budget_heads=heads)
             vals.append(v)
         vals = vals[args.warmup:]
         value = statistics.mean(vals)
         print(json.dumps({
             "impl": "reference", "metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s",
-            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": w.B * w.L / value * 1e3, "higher_is_better": True, "scaling": "weak",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": w.B * w.L / value * 1e3, "higher_is_better": True, "scaling": args.scaling,
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d_feat": w.d_feat, "d_v": w.d_v},
             "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
@@ -625,13 +766,21 @@ def main():
     if dist_on:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     import paper_2402_18668_b200 as based
+    from paper_2402_18668_b200 import dist as bd
     based.lib()
     peaks = load_peaks()
+
+    def my_share(wk):
+        """This rank's part of a workload: all of it (weak scaling) or its slice of the B*H heads (strong)."""
+        if args.scaling == "weak" or world == 1:
+            return wk, 1.0
+        mine = len(bd.shard_heads(wk.B * wk.H, rank, world))
+        return wk.scaled(name=f"{wk.name}[{mine} of {wk.B * wk.H} heads]", B=1, H=mine), wk.B * wk.H / (mine * world)
 
     if args.profile:
         base = {"prefill": w, "decode": wl.CONFIGS["cfg4_generation"], "decode_sym": wl.CONFIGS["cfg4_generation"], "swa": wl.CONFIGS["cfg5_mixer_pair"],
                 "swa_decode": wl.CONFIGS["cfg4_generation"],
-                "generation_graph": wl.CONFIGS["cfg4_generation"],
+                "generation_graph": wl.CONFIGS["cfg4_generation"], "seqpar": wl.CONFIGS["cfg5_mixer_pair"],
                 "baseconv": wl.CONFIGS["cfg3_1p3b_prefill"], "backward": w,
                 "prefill_dfeat": w.scaled(d_feat=args.d_feat, qk_scale=0.4)}[args.profile]
         if args.profile == "swa" and args.window > 0:
@@ -658,6 +807,8 @@ def main():
             r = bench_baseconv(shp, args.steps, args.warmup, torch, based, dist_on, peaks)
         elif args.profile == "generation_graph":
             r = bench_generation_graph(base, args.steps, args.warmup, torch, based, dist_on, peaks)
+        elif args.profile == "seqpar":
+            r = bench_seqpar(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         else:
             r = bench_swa(base, args.steps, args.warmup, torch, based, dist_on, peaks)
         if rank == 0:
@@ -676,65 +827,117 @@ def main():
     sampler = ClockSampler(phys).start()
     sampler.active = True
 
-    res, launches, _ = bench_prefill(w, args.steps, args.warmup, torch, based, dist_on, peaks)
+    w_mine, rebal = my_share(w)
+    t_head0 = time.perf_counter()
+    res, launches, _ = bench_prefill(w_mine, args.steps, args.warmup, torch, based, dist_on, peaks, sampler=sampler,
+                                     sustain_s=args.sustain)
+    t_head1 = time.perf_counter()
     torch.cuda.empty_cache()
-    e2e = bench_prefill_e2e(w, max(10, args.steps // 2), 3, torch, based, dist_on)
+    e2e = bench_prefill_e2e(w_mine, max(10, args.steps // 2), 3, torch, based, dist_on)
     torch.cuda.empty_cache()
     extras = {}
     if not args.skip_extras:
         others = {}
         for name in ("cfg2_360m_prefill", "cfg3_1p3b_prefill", "cfg5_mixer_pair"):
             if name != w.name:
-                r, _, _ = bench_prefill(wl.CONFIGS[name], max(5, args.steps // 2), 3, torch, based, dist_on, peaks)
+                r, _, _ = bench_prefill(my_share(wl.CONFIGS[name])[0], max(5, args.steps), 3, torch, based, dist_on, peaks,
+                                        sampler=sampler, sustain_s=args.sustain)
                 others[name] = r
                 torch.cuda.empty_cache()
         extras["prefill_configs"] = others
-        extras["decode"] = bench_decode(wl.CONFIGS["cfg4_generation"], 1024, 16, torch, based, dist_on, peaks)
-        extras["decode_sym"] = bench_decode(wl.CONFIGS["cfg4_generation"], 1024, 16, torch, based, dist_on, peaks,
-                                            sym=True)
+        w4 = my_share(wl.CONFIGS["cfg4_generation"])[0]
+        extras["decode"] = bench_decode(w4, 1024, 16, torch, based, dist_on, peaks)
+        extras["decode_sym"] = bench_decode(w4, 1024, 16, torch, based, dist_on, peaks, sym=True)
         torch.cuda.empty_cache()
-        extras["backward"] = bench_backward(w, 5, 3, torch, based, dist_on, peaks)
+        extras["backward"] = bench_backward(my_share(wl.CONFIGS["cfg2_360m_prefill"])[0], 5, 3, torch, based, dist_on, peaks)
         torch.cuda.empty_cache()
-        extras["backward_cfg3"] = bench_backward(wl.CONFIGS["cfg3_1p3b_prefill"], 5, 3, torch, based, dist_on, peaks)
+        extras["backward_cfg3"] = bench_backward(my_share(wl.CONFIGS["cfg3_1p3b_prefill"])[0], 5, 3, torch, based, dist_on, peaks)
         torch.cuda.empty_cache()
         extras["baseconv"] = bench_baseconv((8, 4096, 8192), 10, 3, torch, based, dist_on, peaks)
-        extras["generation_graph"] = bench_generation_graph(wl.CONFIGS["cfg4_generation"], 512, 16, torch, based,
-                                                            dist_on, peaks)
-        extras["swa_decode"] = bench_swa_decode(wl.CONFIGS["cfg4_generation"], 200, 10, torch, based, dist_on, peaks)
-        extras["swa"] = bench_swa(wl.CONFIGS["cfg5_mixer_pair"], max(5, args.steps // 2), 3, torch, based, dist_on,
+        extras["generation_graph"] = bench_generation_graph(w4, 512, 16, torch, based, dist_on, peaks)
+        extras["swa_decode"] = bench_swa_decode(w4, 200, 10, torch, based, dist_on, peaks)
+        extras["swa"] = bench_swa(my_share(wl.CONFIGS["cfg5_mixer_pair"])[0], max(5, args.steps), 3, torch, based, dist_on,
                                   peaks)
         torch.cuda.empty_cache()
+        if dist_on:
+            extras["seqpar"] = bench_seqpar(wl.CONFIGS["cfg5_mixer_pair"], 10, 3, torch, based, dist_on, peaks)
+            torch.cuda.empty_cache()
     sampler.active = False
     clocks = sampler.stop()
+    clocks["headline_region"] = sampler.region(t_head0, t_head1)
+    if args.scaling == "strong" and world > 1 and extras:
+        # the arms ran on this rank's slice of the heads in the slowest rank's time: whole-job rates
+        c4, c5 = wl.CONFIGS["cfg4_generation"], wl.CONFIGS["cfg5_mixer_pair"]
+        for key, us in (("decode", "us_per_step"), ("decode_sym", "us_per_step"), ("swa_decode", "us_per_step"),
+                        ("generation_graph", "us_per_token_step")):
+            extras[key]["value"] = c4.B / (extras[key][us] * 1e-6)
+        extras["swa"]["value"] = c5.B * c5.L / (extras["swa"]["ms_per_step"] * 1e-3)
+        for name, r in extras["prefill_configs"].items():
+            r["tokens_per_s"] = wl.CONFIGS[name].B * wl.CONFIGS[name].L / (r["ms_per_step"] * 1e-3)
 
     if rank == 0:
-        cpu_val, cores, sample = cpu_oracle_sample(w, budget_heads=w.B * w.H)
-        value = res["tokens_per_s"] * world
-        e2e["value"] *= world
-        bound_tensor = True      # the chunk contractions are the contract's yardstick; HBM figures ride along
+        cpu_val, cores, sample = cpu_oracle_sample(w, budget_heads=oracle_sample_heads(w))
+        # whole-job tokens: every rank's own copy of the batch (weak) or the one batch the ranks share (strong)
+        job_tokens = w.B * w.L * (world if args.scaling == "weak" else 1)
+        value = job_tokens / (res["ms_per_step"] * 1e-3)
+        e2e["value"] = job_tokens / (e2e["ms_per_step"] * 1e-3)
         line = {
             "metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": res["ms_per_step"],
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
+            "higher_is_better": True, "scaling": args.scaling, "vs_baseline": None, "dtype": w.dtype,
             "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d_feat": w.d_feat, "d_v": w.d_v,
-                       "per_gpu": True, "l2": f"rotating {res['buffer_sets']} input sets larger than L2 in total"},
+                       "per_gpu": args.scaling == "weak", "heads_on_this_rank": w_mine.B * w_mine.H,
+                       "l2": f"rotating {res['buffer_sets']} input sets larger than L2 in total"},
             "roofline": {
-                "bound": "tensor" if bound_tensor else "hbm",
-                "achieved": res["alg_tflops"] if bound_tensor else res["alg_gbs"],
-                "peak": peaks["bf16_tflops"] if bound_tensor else peaks["hbm_gbs"],
-                "unit": "TFLOP/s" if bound_tensor else "GB/s",
-                "frac": res["frac_tensor_peak"] if bound_tensor else res["frac_hbm_peak"],
-                "traffic": NCU_TRAFFIC.get(w.name), "peak_source": peaks["source"],
+                "bound": "tensor", "achieved": res["alg_tflops"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": res["frac_tensor_peak"],
+                "traffic": NCU_TRAFFIC.get(w.name) if w_mine.H * w_mine.B == w.B * w.H else None,
+                "peak_source": peaks["source"], "peak_kind": "burst (the timed region is a burst of K calls at the full clock)",
                 "kernel": "prefill_tc_kernel", "kernel_us": res["ms_per_step"] * 1e3 / max(1, res["launches_per_step"]),
-                "algorithmic_flops": prefill_alg_flops_per_token_head(w.d_v) * w.B * w.H * w.L,
-                "algorithmic_bytes": prefill_alg_bytes(w, w.return_state),
+                "algorithmic_flops": prefill_alg_flops_per_token_head(w.d_v) * w_mine.B * w_mine.H * w.L,
+                "algorithmic_bytes": prefill_alg_bytes(w_mine, w.return_state),
                 "tensor": {"achieved": res["alg_tflops"], "peak": peaks["bf16_tflops"], "frac": res["frac_tensor_peak"]},
                 "hbm": {"achieved": res["alg_gbs"], "peak": peaks["hbm_gbs"], "frac": res["frac_hbm_peak"]},
+                "sustained": res.get("sustained"),
             },
             "cpu_baseline": {"value": cpu_val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": e2e, "gpu_launches": launches, "clocks": clocks, **extras,
         }
+        # ---- compact summary, last in the line: time (us), roofline fraction and bound of every configuration
+        def pf(r):
+            sus = r.get("sustained") or {}
+            return {"us": round(r["ms_per_step"] * 1e3, 2), "frac": frac_str(r["frac_tensor_peak"]), "bound": "tensor",
+                    "sus_us": None if not sus else round(sus["us_per_step"], 2),
+                    "sus_frac": frac_str(sus.get("frac_tensor_peak_sustained")),
+                    "sus_mhz": (sus.get("clocks") or {}).get("sm_mhz")}
+        summ = {w.name.split("_")[0] + "_prefill": pf(res)}
+        for name, r in extras.get("prefill_configs", {}).items():
+            summ[name.split("_")[0] + "_prefill"] = pf(r)
+        def hb(r, key):
+            return {"us": round(r[key] if key.startswith("us") else r[key] * 1e3, 2), "frac": frac_str(r["roofline"]["frac"]),
+                    "bound": r["roofline"]["bound"]}
+        if "decode" in extras:
+            summ["cfg4_decode_273"] = hb(extras["decode"], "us_per_step")
+            summ["cfg4_decode_153"] = hb(extras["decode_sym"], "us_per_step")
+            summ["cfg5_swa"] = hb(extras["swa"], "ms_per_step")
+            summ["gen_graph"] = hb(extras["generation_graph"], "us_per_token_step")
+            summ["swa_decode"] = hb(extras["swa_decode"], "us_per_step")
+            summ["baseconv"] = hb(extras["baseconv"], "ms_per_step")
+            summ["bwd_cfg2"] = hb(extras["backward"], "ms_per_step")
+            summ["bwd_cfg3"] = hb(extras["backward_cfg3"], "ms_per_step")
+            w5 = wl.CONFIGS["cfg5_mixer_pair"]
+            lin = res if w.name == w5.name else extras["prefill_configs"].get(w5.name)
+            if lin is not None:
+                t_pair = lin["ms_per_step"] * 1e-3 + extras["swa"]["ms_per_step"] * 1e-3
+                summ["cfg5_pair"] = {"us": round(t_pair * 1e6, 2),
+                                     "tokens_per_s": round(w5.B * w5.L * (world if args.scaling == "weak" else 1) / t_pair)}
+        if "seqpar" in extras:
+            summ["cfg5_seqpar"] = {"us": round(extras["seqpar"]["ms_per_step"] * 1e3, 2),
+                                   "parity_ok": extras["seqpar"]["parity_ok"]}
+        summ["targets"] = {"decode_frac_hbm>=0.70": summ.get("cfg4_decode_273", {}).get("frac"),
+                           "prefill_frac_tensor>=0.50": {k: v["frac"] for k, v in summ.items() if k.endswith("_prefill")}}
+        line["summary"] = summ
         print(json.dumps(line))
     if dist_on:
         dist.destroy_process_group()
