@@ -78,7 +78,8 @@ enum {
  * d_feat in {8, 24, 32} (the other dimensions of the paper's feature-map ablation; state rows
  * D = 1 + d_feat + d_feat^2 = 73, 601, 1057) is served by the definition form: bf16 io from the
  * empty state on tensor cores (outputs and state), the other cases by fp32 FMA kernels; no
- * workspace, no BASED_STATE_SYM, B*H <= 65535.
+ * workspace, no BASED_STATE_SYM.
+ * Batches of more than 65535 heads are cut into slabs of heads that run one after another on the stream.
  * out must not alias an input.
  */
 based_status based_prefill(const void* q, const void* k, const void* v, void* out, float* kv_state,
@@ -206,7 +207,7 @@ based_status swa_decode_step(const void* q, const void* k, const void* v, void* 
  * flags: 0, or BASED_NUMERATOR_ONLY for the backward of the numerator-only forward.
  * workspace: at least based_prefill_backward_workspace_bytes(B, H, L, d_v, io) bytes of device scratch.
  * Supported: d_feat = 16 with io in {F32, BF16}, d_feat in {8, 24, 32} with BF16 io (w = 1 + s/sqrt(d') +
- * s^2/(2 d'), so ds_ij = (a_i . v_j + b_i)(1/sqrt(d') + q_i.k_j / d')); d_v in {64, 112, 128}; B*H <= 65535.
+ * s^2/(2 d'), so ds_ij = (a_i . v_j + b_i)(1/sqrt(d') + q_i.k_j / d')); d_v in {64, 112, 128}.
  * Both paths evaluate the quadratic form, O(L^2) per head, on 128 x 128 (bf16 io: tcgen05 tensor
  * cores, bf16 operands, fp32 accumulation) or 64 x 64 (fp32 io: fp32 FMAs) tiles of (query, key)
  * pairs; with bf16 io and d_feat = 16 longer sequences take the block-wise path described at

@@ -54,6 +54,16 @@ static inline bool df_generic(int d_feat) { return d_feat == 8 || d_feat == 24 |
 
 using namespace based;
 
+// Several kernels index heads by the y dimension of the grid (at most 65535).  Larger batches are cut into
+// slabs of heads here: every tensor is [B*H, ...] with the heads outermost, so a slab is a contiguous piece,
+// and the slabs run one after another on the caller's stream (sharing the caller's workspace, which is sized
+// for the largest slab).
+constexpr long long kHeadSlab = 65532;      // a multiple of 4: a slab's K-state (an odd number of floats per head) stays 16-byte aligned
+static inline const void* off(const void* p, size_t bytes) { return p ? static_cast<const char*>(p) + bytes : nullptr; }
+static inline void* off(void* p, size_t bytes) { return p ? static_cast<char*>(p) + bytes : nullptr; }
+static inline float* off(float* p, size_t floats) { return p ? p + floats : nullptr; }
+static inline size_t esize(based_dtype io) { return io == BASED_BF16 ? 2 : 4; }
+
 extern "C" {
 
 int based_version(void) { return 1; }
@@ -76,6 +86,12 @@ const char* based_status_string(based_status s) {
 size_t based_prefill_workspace_bytes(int B, int H, int L, int d_feat, int d_v, based_dtype io) {
     if (B <= 0 || H <= 0 || L <= 0 || d_feat != kDFeat || !dv_ok(d_v)) return 0;
     if (io != BASED_BF16) return 0;            // the fp32 path keeps its state in registers
+    const long long BH = (long long)B * H;
+    if (BH > kHeadSlab) {
+        const size_t a = prefill_tc_workspace_bytes((int)kHeadSlab, L, d_v);
+        const size_t b = BH % kHeadSlab ? prefill_tc_workspace_bytes((int)(BH % kHeadSlab), L, d_v) : 0;
+        return a > b ? a : b;
+    }
     return prefill_tc_workspace_bytes(B * H, L, d_v);
 }
 
@@ -93,8 +109,20 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(kv_state) ||
         !aligned16(z_state) || !aligned16(workspace))
         return BASED_ERR_ALIGNMENT;
+    if ((long long)B * H > kHeadSlab) {
+        const size_t es = esize(io), rows = (flags & BASED_STATE_SYM) ? kDSym : 1 + d_feat + d_feat * d_feat;
+        for (long long h0 = 0; h0 < (long long)B * H; h0 += kHeadSlab) {
+            const int n = (int)((long long)B * H - h0 < kHeadSlab ? (long long)B * H - h0 : kHeadSlab);
+            const based_status st = based_prefill(
+                off(q, (size_t)h0 * L * d_feat * es), off(k, (size_t)h0 * L * d_feat * es), off(v, (size_t)h0 * L * d_v * es),
+                off(out, (size_t)h0 * L * d_v * es), off(kv_state, (size_t)h0 * rows * d_v), off(z_state, (size_t)h0 * rows),
+                1, n, L, d_feat, d_v, io, flags, workspace, workspace_bytes, cuda_stream);
+            if (st != BASED_OK) return st;
+        }
+        return BASED_OK;
+    }
     if (d_feat != kDFeat) {
-        if ((flags & BASED_STATE_SYM) || (long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
+        if (flags & BASED_STATE_SYM) return BASED_ERR_UNSUPPORTED;
         // bf16 io from the empty state: outputs on the tensor cores (definition form), the state by the fp32 kernel
         bool outputs_done = false;
         if (io == BASED_BF16 && !(flags & BASED_STATE_CONTINUE)) {
@@ -109,7 +137,6 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
     }
     const size_t need = based_prefill_workspace_bytes(B, H, L, d_feat, d_v, io);
     if (need > 0 && (!workspace || workspace_bytes < need)) return BASED_ERR_WORKSPACE;
-    if ((long long)B * H > 65535 && io == BASED_BF16) return BASED_ERR_UNSUPPORTED;
     if (io == BASED_BF16)
         return launch_prefill_tc(q, k, v, out, kv_state, z_state, B * H, L, d_v, flags, workspace,
                                  static_cast<cudaStream_t>(cuda_stream));
@@ -119,7 +146,7 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
 
 size_t based_prefill_state_workspace_bytes(int B, int H, int L, int d_feat, int d_v, based_dtype io) {
     if (B <= 0 || H <= 0 || L <= 0 || d_feat != kDFeat || !dv_ok(d_v) || io != BASED_BF16) return 0;
-    if ((long long)B * H > 65535) return 0;
+    if ((long long)B * H > kHeadSlab) return prefill_tc_state_workspace_bytes((int)kHeadSlab, L, d_v);   // heads x one partial state: the largest slab's
     return prefill_tc_state_workspace_bytes(B * H, L, d_v);
 }
 
@@ -130,11 +157,22 @@ based_status based_prefill_state(const void* k, const void* v, float* kv_state, 
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
     if (flags & ~(BASED_STATE_CONTINUE | BASED_STATE_SYM)) return BASED_ERR_INVALID_ARG;
     if ((d_feat != kDFeat && !df_generic(d_feat)) || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
-    if ((long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
     const bool tc16 = d_feat == kDFeat && io == BASED_BF16;
     if ((flags & BASED_STATE_SYM) && !tc16) return BASED_ERR_UNSUPPORTED;      // symmetric rows: d' = 16, bf16 io
     if (!aligned16(k) || !aligned16(v) || !aligned16(kv_state) || !aligned16(z_state) || !aligned16(workspace))
         return BASED_ERR_ALIGNMENT;
+    if ((long long)B * H > kHeadSlab) {
+        const size_t es = esize(io), rows = (flags & BASED_STATE_SYM) ? kDSym : 1 + d_feat + d_feat * d_feat;
+        for (long long h0 = 0; h0 < (long long)B * H; h0 += kHeadSlab) {
+            const int n = (int)((long long)B * H - h0 < kHeadSlab ? (long long)B * H - h0 : kHeadSlab);
+            const based_status st = based_prefill_state(
+                off(k, (size_t)h0 * L * d_feat * es), off(v, (size_t)h0 * L * d_v * es), off(kv_state, (size_t)h0 * rows * d_v),
+                off(z_state, (size_t)h0 * rows), 1, n, L, d_feat, d_v, io, flags, workspace, workspace_bytes, cuda_stream);
+            if (st != BASED_OK) return st;
+        }
+        return BASED_OK;
+    }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (tc16) {
         if (!workspace || workspace_bytes < based_prefill_state_workspace_bytes(B, H, L, d_feat, d_v, io))
@@ -222,8 +260,18 @@ based_status swa_forward(const void* q, const void* k, const void* v, void* out,
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
     if (out == q || out == k || out == v) return BASED_ERR_INVALID_ARG;
     if (d != 64 || window > 128) return BASED_ERR_UNSUPPORTED;
-    if ((long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return BASED_ERR_ALIGNMENT;
+    if ((long long)B * H > kHeadSlab) {
+        const size_t hb = (size_t)L * d * esize(io);
+        for (long long h0 = 0; h0 < (long long)B * H; h0 += kHeadSlab) {
+            const int n = (int)((long long)B * H - h0 < kHeadSlab ? (long long)B * H - h0 : kHeadSlab);
+            const based_status st = swa_forward(off(q, h0 * hb), off(k, h0 * hb), off(v, h0 * hb), off(out, h0 * hb), 1, n, L,
+                                                d, window, softmax_scale, io, cuda_stream);
+            if (st != BASED_OK) return st;
+        }
+        return BASED_OK;
+    }
     const float scale = softmax_scale > 0.f ? softmax_scale : 0.125f;   // 1/sqrt(64)
     if (io == BASED_BF16 && swa_tc_supported(window))
         return launch_swa_tc(q, k, v, out, B * H, L, window, scale, static_cast<cudaStream_t>(cuda_stream));
@@ -308,8 +356,9 @@ based_status baseconv_gate_step(const void* a, const void* g, const float* h, co
 
 size_t based_prefill_backward_workspace_bytes(int B, int H, int L, int d_v, based_dtype io) {
     if (B <= 0 || H <= 0 || L <= 0 || !dv_ok(d_v)) return 0;
-    if (io == BASED_BF16) return backward_tc_workspace_bytes(B * H, L, d_v);
-    return (size_t)B * H * L * 2 * sizeof(float);
+    const int heads = (long long)B * H > kHeadSlab ? (int)kHeadSlab : B * H;       // the largest slab of heads
+    if (io == BASED_BF16) return backward_tc_workspace_bytes(heads, L, d_v);
+    return (size_t)heads * L * 2 * sizeof(float);
 }
 
 int based_prefill_backward_block_tokens(int B, int H, int L, int d_feat, int d_v, based_dtype io, int flags,
@@ -328,12 +377,23 @@ static based_status prefill_backward(const void* q, const void* k, const void* v
     if (dq == q || dq == k || dk == q || dk == k || dv == v || dv == dout) return BASED_ERR_INVALID_ARG;
     // the other feature dimensions: bf16 io only (the tensor-core kernels take d' as a parameter)
     if (!(d_feat == kDFeat || (df_generic(d_feat) && io == BASED_BF16)) || !dv_ok(d_v)) return BASED_ERR_UNSUPPORTED;
-    if ((long long)B * H > 65535) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) || !aligned16(dk) ||
         !aligned16(dv) || !aligned16(workspace) || !aligned16(out))
         return BASED_ERR_ALIGNMENT;
     if (!workspace || workspace_bytes < based_prefill_backward_workspace_bytes(B, H, L, d_v, io))
         return BASED_ERR_WORKSPACE;
+    if ((long long)B * H > kHeadSlab) {
+        const size_t qb = (size_t)L * d_feat * esize(io), vb = (size_t)L * d_v * esize(io);
+        for (long long h0 = 0; h0 < (long long)B * H; h0 += kHeadSlab) {
+            const int n = (int)((long long)B * H - h0 < kHeadSlab ? (long long)B * H - h0 : kHeadSlab);
+            const based_status st = prefill_backward(off(q, h0 * qb), off(k, h0 * qb), off(v, h0 * vb), off(out, h0 * vb),
+                                                     off(dout, h0 * vb), off(dq, h0 * qb), off(dk, h0 * qb), off(dv, h0 * vb), 1,
+                                                     n, L, d_feat, d_v, io, flags, workspace, workspace_bytes, cuda_stream);
+            if (st != BASED_OK) return st;
+        }
+        return BASED_OK;
+    }
     if (io == BASED_BF16)
         return launch_prefill_backward_tc(q, k, v, out, dout, dq, dk, dv, static_cast<float*>(workspace), B * H, L,
                                           d_feat, d_v, (flags & BASED_NUMERATOR_ONLY) ? 1 : 0,

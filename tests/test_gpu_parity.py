@@ -1141,3 +1141,30 @@ def test_bench_profiles_print_one_json_line(args):
     d = json.loads(lines[0])
     assert d["profile"] == args[1] and d["value"] > 0 and 0 < d["roofline"]["frac"] < 1.5
 
+
+
+# --------------------------------------------------------------------------- very many heads
+def test_more_heads_than_one_grid_dimension_holds():
+    """B*H = 70,000 heads of 128 tokens (bf16): the batch is cut into slabs of heads inside the library; heads on
+    both sides of the cut, the first and the last, against the oracle (prefill with state, the state-only call and
+    the sliding window)."""
+    B, H, L, d_v = 7, 10000, 128, 64
+    g = torch.Generator(device=DEV).manual_seed(70000)
+    q = (torch.randn(B, H, L, 16, generator=g, device=DEV) * 0.5).bfloat16()
+    k = (torch.randn(B, H, L, 16, generator=g, device=DEV) * 0.5).bfloat16()
+    v = torch.randn(B, H, L, d_v, generator=g, device=DEV).bfloat16()
+    kv, z = based.new_state(B, H, d_v)
+    out = based.based_prefill(q, k, v, kv_state=kv, z_state=z)
+    kv2, z2 = based.based_prefill_state(k, v)
+    qs = torch.randn(B, H, L, 64, generator=g, device=DEV).bfloat16()
+    ks = torch.randn(B, H, L, 64, generator=g, device=DEV).bfloat16()
+    out_swa = based.swa_forward(qs, ks, v, window=64)
+    _poll()
+    for bh in (0, 65531, 65532, 65535, 65536, B * H - 1):
+        b, h = divmod(bh, H)
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        y_ref, S_ref, z_ref = oracle.linattn_quadratic(_np(q[sl]), _np(k[sl]), _np(v[sl]))
+        assert row_err(_np(out[sl]), y_ref) <= TOL_BF16, bh
+        assert_state_close(_np(kv[sl]), S_ref, _np(z[sl]), z_ref, "bf16", f"head {bh}")
+        assert_state_close(_np(kv2[sl]), S_ref, _np(z2[sl]), z_ref, "bf16", f"head {bh}, state-only call")
+        assert row_err(_np(out_swa[sl]), oracle.swa(_np(qs[sl]), _np(ks[sl]), _np(v[sl]), 64)) <= TOL_BF16, bh
