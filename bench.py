@@ -523,9 +523,9 @@ def bench_generation_graph(w, steps, warmup, torch, based, dist_on, peaks):
     bytes_step = 2.0 * w.B * w.H * based.D_SYM * w.d_v * 4 + 2.0 * w.B * w.H * win * d * esz
     return {
         "workload": f"B{w.B} H{w.H}: decode step on the 153-row state (d_v {w.d_v}) + window-{win} decode step, "
-                    "one CUDA graph per token",
+                    "one fused launch (based_generation_step) replayed as a CUDA graph per token",
         "metric": "generation_tokens_per_s", "value": w.B / t, "unit": "tokens/s", "us_per_token_step": t * 1e6,
-        "steps": steps, "kernels_per_replay": 2,
+        "steps": steps, "kernels_per_replay": 1 if graph.fused else 2,
         "roofline": {"bound": "hbm", "achieved": bytes_step / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": bytes_step / t / 1e9 / peaks["hbm_gbs"], "traffic": None,
                      "algorithmic_bytes": bytes_step, "peak_source": peaks["source"]},

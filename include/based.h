@@ -315,6 +315,28 @@ based_status swa_decode_step_advance(const void* q, const void* k, const void* v
                                      float softmax_scale, based_dtype io, void* cuda_stream);
 
 /*
+ * One generated token through both mixers in ONE launch: based_decode_step (or its symmetric-state /
+ * numerator-only forms, by flags: BASED_STATE_SYM, BASED_NUMERATOR_ONLY) on the linear-attention
+ * layer's B x H heads (Sec. 4.1 recurrences, Algorithm 2) and swa_decode_step_advance on the
+ * sliding-window layer's B x H_w heads (Algorithm 3, rolling cache, position read from and advanced in
+ * device memory), the two kinds of CTA dealt out in turn within one grid so that the short window
+ * step hides under the long state stream (the paper runs next-token prediction under CUDA graphs,
+ * Sec. 6 "Efficiency Benchmarks"; as two kernels the steps run one after the other).
+ * q, k [B,H,16], v, out [B,H,d_v], kv_state / z_state as in based_decode_step_flags (updated in
+ * place); qw, kw, vw, out_w [B,H_w,64], k_cache, v_cache [B,H_w,window,64] as in swa_decode_step
+ * (slot position % window is overwritten); pos_state: two ints in device memory, {position,
+ * ticket}, 8-byte aligned (ticket 0 before the first call): position + 1 is stored when the step
+ * ends.  All device pointers, io dtype for both mixers, results identical to the separate calls.
+ * Supported: d_feat = 16, d_v in {64, 112, 128}, d_w = 64, window <= 128.  Errors as the separate
+ * calls; nothing is launched when validation fails.
+ */
+based_status based_generation_step(const void* q, const void* k, const void* v, float* kv_state, float* z_state,
+                                   void* out, const void* qw, const void* kw, const void* vw, void* k_cache,
+                                   void* v_cache, void* out_w, int B, int H, int d_feat, int d_v, int H_w, int d_w,
+                                   int window, int* pos_state, float softmax_scale, based_dtype io, int flags,
+                                   void* cuda_stream);
+
+/*
  * The same computation as based_prefill, for callers that cannot give the library scratch
  * memory.  (The paper has no counterpart: this is a deployment convenience.)  Some hosts
  * may not allocate device memory around a call at all - a serving process that has handed

@@ -28,7 +28,7 @@ EXPORTS = (
     "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step", "based_decode_step_sym",
     "based_state_to_sym", "based_state_from_sym", "swa_decode_step_at", "based_preload_decode",
     "baseconv_gate_forward", "baseconv_gate_step", "based_decode_step_flags", "based_prefill_backward",
-    "based_prefill_backward_workspace_bytes", "based_prefill_backward_with_out", "based_prefill_backward_block_tokens", "swa_decode_step_advance",
+    "based_prefill_backward_workspace_bytes", "based_prefill_backward_with_out", "based_prefill_backward_block_tokens", "swa_decode_step_advance", "based_generation_step",
     "based_prefill_state", "based_prefill_state_workspace_bytes",
 )
 
@@ -82,6 +82,8 @@ def lib() -> ctypes.CDLL:
         L.swa_decode_step_at.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, i, vp]
         L.swa_decode_step_advance.restype = i
         L.swa_decode_step_advance.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, i, vp]
+        L.based_generation_step.restype = i
+        L.based_generation_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, f, i, i, vp]
         L.based_preload_decode.restype = i
         L.based_prefill_backward.restype = i
         L.based_prefill_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
@@ -406,6 +408,40 @@ def swa_decode_step(q, k, v, k_cache, v_cache, pos: int, out=None, softmax_scale
                                int(pos), float(softmax_scale), _dtype_code(q), _stream(stream))
     _check(st, "swa_decode_step")
     return out
+
+
+def based_generation_step(q, k, v, kv_state, z_state, qw, kw, vw, k_cache, v_cache, pos_state, out=None, out_w=None,
+                          flags: int = 0, softmax_scale: float = 0.0, stream=None):
+    """One generated token through both mixers in one launch: the linear-attention decode step (q, k
+    [B,H,16], v [B,H,d_v], state updated in place; flags: BASED_STATE_SYM, BASED_NUMERATOR_ONLY) and the
+    sliding-window decode step (qw, kw, vw [B,H_w,64], ring caches [B,H_w,window,64] updated in place).
+    pos_state: int32 tensor {position, ticket} on the device; the step stores position + 1.
+    Returns (out, out_w)."""
+    _dev(q, k, v, kv_state, z_state, qw, kw, vw, k_cache, v_cache, pos_state, out, out_w)
+    B, H, d_feat = q.shape
+    d_v = v.shape[-1]
+    _check_qkv(q, k, v, out)
+    _check_state(kv_state, z_state, B, H, d_feat, d_v, flags, required=True)
+    Bw, Hw, d_w = qw.shape
+    window = k_cache.shape[2]
+    if Bw != B or kw.shape != qw.shape or vw.shape != qw.shape or qw.dtype != q.dtype or kw.dtype != q.dtype or vw.dtype != q.dtype:
+        raise ValueError("qw, kw, vw must be [B,H_w,d_w] in the io dtype")
+    if k_cache.shape != (B, Hw, window, d_w) or v_cache.shape != k_cache.shape or k_cache.dtype != q.dtype or v_cache.dtype != q.dtype:
+        raise ValueError("cache shapes/dtypes disagree with qw")
+    if pos_state.dtype != torch.int32 or pos_state.numel() != 2:
+        raise ValueError("pos_state is an int32 tensor {position, ticket}")
+    if out is None:
+        out = torch.empty_like(v)
+    if out_w is None:
+        out_w = torch.empty_like(vw)
+    elif out_w.shape != vw.shape or out_w.dtype != vw.dtype:
+        raise ValueError("out_w must have the shape and dtype of vw")
+    st = lib().based_generation_step(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_state), _ptr(z_state), _ptr(out), _ptr(qw),
+                                     _ptr(kw), _ptr(vw), _ptr(k_cache), _ptr(v_cache), _ptr(out_w), B, H, d_feat, d_v,
+                                     Hw, d_w, window, _ptr(pos_state), float(softmax_scale), _dtype_code(q), int(flags),
+                                     _stream(stream))
+    _check(st, "based_generation_step")
+    return out, out_w
 
 
 def based_selftest_bounded_wait(limit_ms: int = 20, stream=None) -> None:

@@ -326,6 +326,28 @@ based_status swa_decode_step_advance(const void* q, const void* k, const void* v
                              static_cast<cudaStream_t>(cuda_stream));
 }
 
+based_status based_generation_step(const void* q, const void* k, const void* v, float* kv_state, float* z_state,
+                                   void* out, const void* qw, const void* kw, const void* vw, void* k_cache,
+                                   void* v_cache, void* out_w, int B, int H, int d_feat, int d_v, int H_w, int d_w,
+                                   int window, int* pos_state, float softmax_scale, based_dtype io, int flags,
+                                   void* cuda_stream) {
+    if (!q || !k || !v || !kv_state || !z_state || !out || !qw || !kw || !vw || !k_cache || !v_cache || !out_w ||
+        !pos_state || B <= 0 || H <= 0 || H_w <= 0 || window <= 0)
+        return BASED_ERR_INVALID_ARG;
+    if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
+    if (flags & ~(BASED_STATE_SYM | BASED_NUMERATOR_ONLY)) return BASED_ERR_INVALID_ARG;
+    if (d_feat != kDFeat || !dv_ok(d_v) || d_w != 64 || window > 128) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H + ((long long)B * H_w + 1) / 2 > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(kv_state) || !aligned16(z_state) ||
+        !aligned16(out) || !aligned16(qw) || !aligned16(kw) || !aligned16(vw) || !aligned16(k_cache) ||
+        !aligned16(v_cache) || !aligned16(out_w) || (reinterpret_cast<uintptr_t>(pos_state) & 7u))
+        return BASED_ERR_ALIGNMENT;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 0.125f;   // 1/sqrt(64)
+    return launch_generation_step(q, k, v, kv_state, z_state, out, B * H, d_v, (flags & BASED_STATE_SYM) != 0,
+                                  (flags & BASED_NUMERATOR_ONLY) != 0, qw, kw, vw, k_cache, v_cache, out_w, B * H_w,
+                                  window, pos_state, scale, io, static_cast<cudaStream_t>(cuda_stream));
+}
+
 static based_status baseconv_check(const void* a, const void* g, const float* h, const float* b2, const void* out,
                                    int B, int N, int C, int width, based_dtype io) {
     if (!a || !g || !h || !b2 || !out || B <= 0 || N <= 0 || C <= 0 || width <= 0) return BASED_ERR_INVALID_ARG;
@@ -423,6 +445,7 @@ based_status based_preload_decode(void) {
     based_status st = error_word_ptr(&err);
     if (st == BASED_OK) st = preload_decode();
     if (st == BASED_OK) st = preload_swa_decode();
+    if (st == BASED_OK) st = preload_generation_step();
     return st;
 }
 

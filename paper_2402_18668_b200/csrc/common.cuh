@@ -73,6 +73,12 @@ __device__ __forceinline__ float psi_at(const float* x, int f) {
 // sym: the state has the 153 symmetric rows instead of the 273 full ones
 based_status launch_decode(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
                            int BH, int d_v, based_dtype io, bool sym, bool numerator_only, cudaStream_t stream);
+// both mixers' decode steps of one token in one launch (generation_step.cu)
+based_status launch_generation_step(const void* q, const void* k, const void* v, float* kv, float* z, void* out,
+                                    int n_lin, int d_v, bool sym, bool numerator_only, const void* qw, const void* kw,
+                                    const void* vw, void* kc, void* vc, void* outw, int n_swa, int window,
+                                    int* pos_state, float scale, based_dtype io, cudaStream_t stream);
+based_status preload_generation_step();
 // full (273-row) state -> symmetric (153-row) state, or back
 based_status launch_state_convert(const float* kv_in, const float* z_in, float* kv_out, float* z_out, int BH,
                                   int d_v, bool to_sym, cudaStream_t stream);

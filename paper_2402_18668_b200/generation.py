@@ -5,7 +5,10 @@ batch sizes where a decode step lasts tens of microseconds the launch overhead o
 calls is a visible share of it.  `DecodeGraph` captures one step of both mixers, the Taylor
 linear-attention decode step (on the 273-row or the 153-row symmetric state) and the
 sliding-window decode step on its rolling cache, which reads the position from device memory and
-advances it itself (swa_decode_step_advance), and replays it once per generated token.
+advances it itself, and replays it once per generated token.  By default the step is the
+library's fused call (based_generation_step: one kernel node in which the two mixers' CTAs are
+dealt out in turn, so the short window step rides in the shadow of the long state stream);
+fused=False captures the two separate kernels one after the other.
 
 Only plumbing lives here (static buffers, stream capture); every arithmetic step runs in the
 library's kernels.
@@ -27,13 +30,14 @@ class DecodeGraph:
     """
 
     def __init__(self, kv_state, z_state, k_cache, v_cache, pos: int, dtype=torch.bfloat16, sym: bool = False,
-                 softmax_scale: float = 0.0):
+                 softmax_scale: float = 0.0, fused: bool = True):
         B, H, rows, d_v = kv_state.shape
         if rows != (_b.D_SYM if sym else _b.D_EXPANDED):
             raise ValueError("state rows do not match the format")
         window, d = k_cache.shape[2], k_cache.shape[3]
         dev = kv_state.device
         self.sym, self.kv, self.z, self.kc, self.vc = sym, kv_state, z_state, k_cache, v_cache
+        self.fused = fused
         self.q = torch.zeros(B, H, _b.D_FEAT, dtype=dtype, device=dev)
         self.k = torch.zeros_like(self.q)
         self.v = torch.zeros(B, H, d_v, dtype=dtype, device=dev)
@@ -57,6 +61,11 @@ class DecodeGraph:
         torch.cuda.current_stream(dev).wait_stream(self._stream)
 
     def _enqueue(self):
+        if self.fused:
+            _b.based_generation_step(self.q, self.k, self.v, self.kv, self.z, self.qw, self.kw, self.vw, self.kc,
+                                     self.vc, self._pos_state, out=self.out_lin, out_w=self.out_swa,
+                                     flags=_b.BASED_STATE_SYM if self.sym else 0, softmax_scale=self._scale)
+            return
         dec = _b.based_decode_step_sym if self.sym else _b.based_decode_step
         dec(self.q, self.k, self.v, self.kv, self.z, out=self.out_lin)
         B, H, d = self.qw.shape

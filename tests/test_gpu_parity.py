@@ -609,8 +609,9 @@ def test_swa_decode_advance_moves_the_position_itself():
     assert torch.equal(kc1, kc2) and torch.equal(vc1, vc2)
 
 
+@pytest.mark.parametrize("fused", [True, False])
 @pytest.mark.parametrize("sym", [False, True])
-def test_decode_graph_replays_match_oracle_chain(sym):
+def test_decode_graph_replays_match_oracle_chain(sym, fused):
     """The mixer pair's generation step captured once and replayed T times (position advanced on the
     device): linear-attention outputs against the oracle's recurrence, sliding-window outputs against
     the whole-sequence form, across the point where the ring cache wraps."""
@@ -634,7 +635,7 @@ def test_decode_graph_replays_match_oracle_chain(sym):
     for t in range(L0):
         based.swa_decode_step(qw[:, :, t].contiguous().to(DEV), kw[:, :, t].contiguous().to(DEV),
                               vw[:, :, t].contiguous().to(DEV), kc, vc, pos=t)
-    graph = DecodeGraph(kv, z, kc, vc, pos=L0, dtype=tdt, sym=sym)
+    graph = DecodeGraph(kv, z, kc, vc, pos=L0, dtype=tdt, sym=sym, fused=fused)
     n0 = based.launch_count()
     for t in range(L0, L0 + T):
         o_lin, o_swa = graph.step(q[:, :, t].to(DEV), k[:, :, t].to(DEV), v[:, :, t].to(DEV),
@@ -644,6 +645,41 @@ def test_decode_graph_replays_match_oracle_chain(sym):
     _poll()
     assert int(graph.pos.item()) == L0 + T
     assert based.launch_count() == n0          # replays enqueue no new launches through the library
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,H,Hw,d_v,window,flags", [(2, 3, 3, 64, 16, 0), (3, 5, 7, 128, 64, 1), (1, 1, 1, 112, 100, 0),
+                                                     (4, 16, 2, 128, 64, 2), (1, 2, 9, 64, 1, 6)])
+def test_generation_step_equals_the_two_separate_steps(dtype, B, H, Hw, d_v, window, flags):
+    """based_generation_step (both mixers' CTAs in one grid) against based_decode_step_flags and
+    swa_decode_step called separately on copies of the same state and caches: bit for bit (the fused kernel
+    runs the same device code), over several tokens, for head counts that leave either role with CTAs of its
+    own after the dealt-out prefix, odd window-head counts (a CTA with one idle half), and the state formats."""
+    flags = {0: 0, 1: based.BASED_STATE_SYM, 2: based.BASED_NUMERATOR_ONLY,
+             6: based.BASED_STATE_SYM | based.BASED_NUMERATOR_ONLY}[flags]
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    g = torch.Generator(device=DEV).manual_seed(B * 100 + H * 10 + Hw)
+    sym = bool(flags & based.BASED_STATE_SYM)
+    kv1, z1 = based.new_state(B, H, d_v, sym=sym)
+    kv1.copy_(torch.randn(kv1.shape, generator=g, device=DEV)); z1.copy_(torch.rand(z1.shape, generator=g, device=DEV) + 1.0)
+    kv2, z2 = kv1.clone(), z1.clone()
+    kc1 = torch.randn(B, Hw, window, 64, generator=g, device=DEV).to(tdt)
+    vc1 = torch.randn(B, Hw, window, 64, generator=g, device=DEV).to(tdt)
+    kc2, vc2 = kc1.clone(), vc1.clone()
+    pos0 = max(0, window - 2)                                  # crosses the point where the ring wraps
+    state = torch.tensor([pos0, 0], dtype=torch.int32, device=DEV)
+    for t in range(5):
+        q = (torch.randn(B, H, 16, generator=g, device=DEV) * 0.5).to(tdt)
+        k = (torch.randn(B, H, 16, generator=g, device=DEV) * 0.5).to(tdt)
+        v = torch.randn(B, H, d_v, generator=g, device=DEV).to(tdt)
+        qw, kw, vw = (torch.randn(B, Hw, 64, generator=g, device=DEV).to(tdt) for _ in range(3))
+        o1 = based.based_decode_step_flags(q, k, v, kv1, z1, flags)
+        w1 = based.swa_decode_step(qw, kw, vw, kc1, vc1, pos0 + t)
+        o2, w2 = based.based_generation_step(q, k, v, kv2, z2, qw, kw, vw, kc2, vc2, state, flags=flags)
+        assert torch.equal(o1, o2) and torch.equal(w1, w2), f"token {t}"
+        assert state.tolist() == [pos0 + t + 1, 0]
+    _poll()
+    assert torch.equal(kv1, kv2) and torch.equal(z1, z2) and torch.equal(kc1, kc2) and torch.equal(vc1, vc2)
 
 
 # --------------------------------------------------------------------------- symmetric state
