@@ -108,7 +108,7 @@ enum Bar {
 };
 
 // segments per head, chunks per segment (the last one takes the rest), mode
-struct SegPlan { int nseg; int per; bool recompute; };
+struct SegPlan { int nseg; int per; bool recompute; int balanced; };   // balanced > 0: that many equal chunk ranges over all heads
 
 struct Params {
     float* kv_abi;        // [BH, 273, DV] or null
@@ -123,6 +123,8 @@ struct Params {
     int numerator_only;   // outputs are not divided by the denominator
     int dv;               // value head dimension of the caller's tensors (112 runs on the d_v 128 kernel:
                           // the tensor maps zero-fill columns 112..127 on load and clip them on store)
+    int balanced;         // > 0: the number of equal chunk ranges the heads' chunks are cut into (see the kernel)
+    int heads;            // B*H (balanced mode)
 #ifdef BASED_TRACE
     unsigned long long* trace;
 #endif
@@ -285,9 +287,86 @@ __global__ void __launch_bounds__(kThreads, 1)
     short2* s_abi = reinterpret_cast<short2*>(s_den + 4 * kC);         // [160] ABI rows of each internal feature
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int seg = blockIdx.x, head = blockIdx.y;
-    const int tok_begin = seg * p.seg_len;
-    const int tok_end = min(p.L, tok_begin + p.seg_len);
+    // ---- the CTA's piece of work: a head, a token range, where its initial state comes from (workspace slots
+    // ws_first .. ws_first + ws_count - 1) and where its final state goes (slot ws_out, or the caller's state if
+    // the piece ends its head).
+    // Legacy grids: blockIdx.x = sequence segment, blockIdx.y = head.
+    // Balanced grids (one row of CTAs): the concatenation of all heads' chunks, T = heads x chunks per head, is
+    // cut into n equal ranges [i T / n, (i + 1) T / n), one per SM.  A range holds at most one head boundary
+    // (n >= heads).  CTA i < n takes range i up to the boundary, if there is one; CTA n + j takes what is left
+    // of a range behind its boundary, the j-th largest such rest first: the hardware hands these later CTAs to
+    // SMs as they become free, and the SM whose first piece was shortest is free first, so every SM ends up
+    // with about T / n chunks.  A piece that ends inside its head leaves its state in slot i of its range.
+    int it_head = blockIdx.y, it_seg = blockIdx.x, it_begin = blockIdx.x * p.seg_len, it_end = 0, it_first = 0, it_count = 0,
+        it_out = -1;
+    bool it_head_end = false;
+    if (MODE != kModePre && p.balanced > 0) {      // (the recompute mode's kernel is never launched this way)
+        // 32-bit arithmetic throughout (the host takes this path only while (T + 1) n fits: 64-bit divisions
+        // would be subroutine calls, and their mere presence slows this kernel's role loops by a fifth)
+        const uint32_t n = p.balanced;
+        const uint32_t nchh = (p.L + kC - 1) / kC;
+        const uint32_t T = (uint32_t)p.heads * nchh;
+        uint32_t lo, hi, range;                    // global chunk range of this piece, index of its range
+        if (blockIdx.x < n) {
+            range = blockIdx.x;
+            lo = range * T / n;
+            hi = (range + 1) * T / n;
+            const uint32_t xb = ((hi - 1) / nchh) * nchh;         // start of the head that holds the range's last chunk
+            if (xb > lo) hi = xb;                                  // a boundary inside: stop there
+        } else {
+            // rest of the range behind head boundary h: [h nchh, end of the range that holds it); rank the rests
+            int* s_rest = reinterpret_cast<int*>(smem + C::offStage);
+            const int nb = p.heads - 1, want = (int)(blockIdx.x - n);
+            auto rest_of = [&](uint32_t h, uint32_t& rg) -> int {
+                const uint32_t x = h * nchh;
+                rg = ((x + 1) * n + T - 1) / T - 1;                 // the range that holds chunk x
+                return rg * T / n == x ? 0 : (int)((rg + 1) * T / n - x);   // 0: the boundary is a range start
+            };
+            for (int h = 1 + threadIdx.x; h <= nb; h += kThreads) { uint32_t rg; s_rest[h] = rest_of(h, rg); }
+            __syncthreads();
+            s_rest[0] = -1;
+            __syncthreads();
+            for (int h = 1 + threadIdx.x; h <= nb; h += kThreads) {
+                const int mine = s_rest[h];
+                int rank = 0;
+                for (int u = 1; u <= nb; ++u) rank += (s_rest[u] > mine || (s_rest[u] == mine && u < h)) ? 1 : 0;
+                if (rank == want) s_rest[0] = h;
+            }
+            __syncthreads();
+            const int h = s_rest[0];
+            __syncthreads();
+            if (h < 1) return;
+            const int r = rest_of(h, range);
+            if (r == 0) return;                                    // nothing is left behind this boundary
+            lo = (uint32_t)h * nchh;
+            hi = lo + r;
+        }
+        it_head = (int)(lo / nchh);
+        const int c0 = (int)(lo - (uint32_t)it_head * nchh), c1 = (int)(hi - (uint32_t)it_head * nchh);
+        it_seg = c0 > 0 ? 1 : 0;
+        it_begin = c0 * kC;
+        it_end = min(p.L, c1 * kC);
+        it_head_end = c1 == (int)nchh;
+        if (c0 > 0 && MODE != kModeState) {
+            const uint32_t x = (uint32_t)it_head * nchh;
+            it_first = (int)(((x + 1) * n + T - 1) / T - 1);       // the range that holds the head's first chunk
+            it_count = (int)range - it_first;
+        }
+        if (MODE == kModeState) {
+            if (it_head_end) return;                               // nobody starts from the state of a head's last piece
+            it_out = (int)range;
+        }
+    } else {
+        it_end = min(p.L, it_begin + p.seg_len);
+        it_head_end = it_seg == p.nseg - 1;
+        const int per_head = p.nseg > 1 ? p.nseg - 1 : 0;          // workspace slots of one head
+        it_first = it_head * per_head;
+        it_count = (MODE == kModeState || MODE == kModePre) ? 0 : it_seg;
+        it_out = MODE == kModeState ? it_head * per_head + it_seg : -1;
+    }
+    const int seg = it_seg, head = it_head, tok_begin = it_begin, tok_end = it_end;
+    const int ws_first = it_first, ws_count = it_count, ws_out = it_out;
+    const bool head_end = it_head_end;
     const int nch = (tok_end - tok_begin + kC - 1) / kC;
     // Recompute mode: before its own chunks the CTA runs the state update alone ("pre-chunks") over
     // every chunk that precedes its segment.  g counts pre-chunks and own chunks together; stage
@@ -604,12 +683,12 @@ __global__ void __launch_bounds__(kThreads, 1)
         // d_v 128: K-state features held in the two z tiles (64-row MMA: rows 0..31 in lanes 0-15, 32-47)
         const int z1f = (DV == 128 && (t & 31) < 16 && (t >> 5) < 2) ? 128 + (t >> 5) * 16 + (t & 15) : -1;
         const size_t seg_stride = seg_state_floats(DV);
-        const float* wsh = p.ws + (size_t)head * (p.nseg > 1 ? p.nseg - 1 : 0) * seg_stride;
+        const float* wsh = p.ws + (size_t)ws_first * seg_stride;      // the partial states this piece starts from
         const int dv = p.dv;                        // row pitch of the caller's state; lanes >= dv hold zeros
         const float* kvh = p.kv_abi ? p.kv_abi + (size_t)head * abi_nrows * dv : nullptr;
         const float* zh = p.z_abi ? p.z_abi + (size_t)head * abi_nrows : nullptr;
         const bool from_abi = !STATE_ONLY && p.continue_abi;
-        const int nprev = (STATE_ONLY || PRE) ? 0 : seg;
+        const int nprev = ws_count;
 
         // Initial value of this lane's row: the caller's ABI state (folded into the internal
         // basis) plus the partial states of the earlier segments.  Loads are issued 16 at a
@@ -743,9 +822,9 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (t == 0) TRACE(5, 3, 7);   // chunk loop done
         tc_fence_after();
         const bool write_ws = STATE_ONLY;
-        const bool write_abi = !STATE_ONLY && p.kv_abi != nullptr && seg == p.nseg - 1;
+        const bool write_abi = !STATE_ONLY && p.kv_abi != nullptr && head_end;
         if (ok && (write_ws || write_abi)) {
-            float* wseg = p.ws + ((size_t)head * (p.nseg > 1 ? p.nseg - 1 : 0) + seg) * seg_stride;
+            float* wseg = p.ws + (size_t)(ws_out < 0 ? 0 : ws_out) * seg_stride;
             float* kvo = write_abi ? p.kv_abi + (size_t)head * abi_nrows * dv : nullptr;
             float* zo = write_abi ? p.z_abi + (size_t)head * abi_nrows : nullptr;
             auto put = [&](int f, float v, bool zrow, int col) {
@@ -1008,6 +1087,22 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
             configured[dev] = true;
         }
     }
+    p.balanced = 0;
+    p.heads = BH;
+    if (plan.balanced > 0) {
+        // state pass over every piece that ends inside its head, then the main pass; both on one row of CTAs:
+        // one per range, then one per head boundary
+        p.balanced = plan.balanced;
+        p.nseg = 1;
+        const dim3 grid(plan.balanced + BH - 1, 1);
+        prefill_tc_kernel<DV, kModeState><<<grid, kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
+        note_launch();
+        const based_status st = check_launch("prefill_tc_kernel<state, balanced>");
+        if (st != BASED_OK) return st;
+        prefill_tc_kernel<DV, kModeMain><<<grid, kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
+        note_launch();
+        return check_launch("prefill_tc_kernel<balanced>");
+    }
     if (nseg > 1 && recompute) {
         prefill_tc_kernel<DV, kModePre><<<dim3(nseg, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
         note_launch();
@@ -1037,7 +1132,7 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
 // start-up about 14.  In recompute mode later segments do more redundant work, so the first
 // n - 1 segments get `per` chunks each and the last one the (shorter) rest, `per` chosen to
 // level the modelled times.
-static SegPlan prefill_tc_plan(int BH, int L, int d_v) {
+static SegPlan prefill_tc_plan(int BH, int L, int d_v, bool continued = false) {
     const int nch = (L + kC - 1) / kC;
     const float full = d_v == 64 ? 3.3f : 3.4f, upd = d_v == 64 ? 1.0f : 1.4f;
     int nmax = 148 / BH;
@@ -1047,7 +1142,7 @@ static SegPlan prefill_tc_plan(int BH, int L, int d_v) {
     if (nseg > nch / 16) nseg = nch / 16;
     if (nseg < 1) nseg = 1;
     while (nseg > 1 && ((nch + nseg - 1) / nseg) * (nseg - 1) >= nch) --nseg;   // every segment owns a chunk
-    SegPlan best = {nseg, (nch + nseg - 1) / nseg, false};
+    SegPlan best = {nseg, (nch + nseg - 1) / nseg, false, 0};
     float best_cost = nseg > 1 ? (float)best.per * (upd + full) + 14.f : (float)nch * full;
     for (int n = 2; n <= nmax; ++n) {
         for (int per = (nch + n - 1) / n; per * (n - 1) < nch; ++per) {
@@ -1058,10 +1153,22 @@ static SegPlan prefill_tc_plan(int BH, int L, int d_v) {
                 if (c > cost) cost = c;
             }
             if (cost < 0.95f * best_cost) {
-                best = {n, per, true};
+                best = {n, per, true, 0};
                 best_cost = cost;
             }
         }
+    }
+    //  - balanced: all heads' chunks, laid end to end, are cut into 148 equal ranges, one per SM (a range then
+    //    holds the tail of one head and the start of the next, run as two CTAs on the same SM one after the
+    //    other); state pass and main pass as above.  It fills every SM whatever the head count.  Not for
+    //    continued calls: a head's last piece writes the caller's state while the first piece of the same head,
+    //    queued behind another head's tail, may not have read it yet.
+    if (BH < 148 && !continued) {
+        const long long total = (long long)BH * nch;
+        const int ranges = 148;
+        const float share = (float)((total + ranges - 1) / ranges);
+        const float cost = share * (upd + full) + 14.f + 7.f;        // a second launch; a second CTA's start-up on some SMs
+        if (share >= 16.f && total >= ranges && total <= 14000000 && cost < 0.95f * best_cost) best = {1, nch, false, ranges};
     }
 #ifdef BASED_TRACE
     if (const char* e = getenv("BASED_NSEG")) {
@@ -1083,7 +1190,7 @@ static SegPlan prefill_tc_state_plan(int BH, int L) {
     n = n < 1 ? 1 : (n > 8 ? 8 : n);
     if (n > nch) n = nch;
     const int per = (nch + n - 1) / n;
-    return {(nch + per - 1) / per, per, false};
+    return {(nch + per - 1) / per, per, false, 0};
 }
 
 // Sum of a head's partial states (internal basis, [160][DV] + [160] per segment) into the caller's state
@@ -1129,6 +1236,7 @@ static based_status launch_state_dv(const void* k, const void* v, float* kv, flo
     if (error_word_ptr(&p.err) != BASED_OK) return BASED_ERR_CUDA;
     p.L = L;
     p.nseg = plan.nseg + 1;            // the workspace holds nseg - 1 partial states per head
+    p.heads = BH;
     p.seg_len = plan.per * kC;
     p.dv = dv;
     {
@@ -1168,14 +1276,21 @@ based_status launch_prefill_tc_state(const void* k, const void* v, float* kv, fl
 
 size_t prefill_tc_workspace_bytes(int BH, int L, int d_v) {
     if (d_v == 112) d_v = 128;                      // runs on the d_v 128 kernel, partial states in its layout
-    const SegPlan plan = prefill_tc_plan(BH, L, d_v);
-    const int nseg = plan.recompute ? 1 : plan.nseg;
-    return nseg > 1 ? (size_t)BH * (nseg - 1) * seg_state_floats(d_v) * sizeof(float) : 0;
+    // the larger of the two plans a call can take (continued calls do not use the balanced one)
+    size_t need = 0;
+    for (int cont = 0; cont < 2; ++cont) {
+        const SegPlan plan = prefill_tc_plan(BH, L, d_v, cont != 0);
+        size_t n = 0;
+        if (plan.balanced > 0) n = (size_t)plan.balanced * seg_state_floats(d_v) * sizeof(float);
+        else if (!plan.recompute && plan.nseg > 1) n = (size_t)BH * (plan.nseg - 1) * seg_state_floats(d_v) * sizeof(float);
+        need = n > need ? n : need;
+    }
+    return need;
 }
 
 based_status launch_prefill_tc(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH,
                                int L, int d_v, int flags, void* workspace, cudaStream_t stream) {
-    const SegPlan plan = prefill_tc_plan(BH, L, d_v == 112 ? 128 : d_v);
+    const SegPlan plan = prefill_tc_plan(BH, L, d_v == 112 ? 128 : d_v, (flags & BASED_STATE_CONTINUE) != 0);
     float* ws = static_cast<float*>(workspace);
     if (d_v == 64) return launch_dv<64>(q, k, v, out, kv, z, BH, L, 64, flags, ws, plan, stream);
     return launch_dv<128>(q, k, v, out, kv, z, BH, L, d_v, flags, ws, plan, stream);      // 112 or 128

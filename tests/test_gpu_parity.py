@@ -1179,6 +1179,33 @@ def test_bench_profiles_print_one_json_line(args):
 
 
 
+# --------------------------------------------------------------------------- few heads, long sequences
+@pytest.mark.parametrize("B,H,L,d_v,flags", [(1, 5, 61000, 64, 0), (1, 40, 16500, 128, 1), (2, 3, 50700, 112, 0),
+                                             (1, 147, 2100, 64, 2)])
+def test_prefill_heads_cut_into_equal_chunk_ranges(B, H, L, d_v, flags):
+    """Fewer heads than SMs and sequences long enough that all heads' chunks, laid end to end, are cut into one
+    equal range per SM (a range then holds the tail of one head and the start of the next, and a head's pieces
+    start from the summed states of the pieces before them): every output row and the final state of every head
+    against the oracle, ragged last chunks included, in the full and the symmetric state format and for
+    numerator-only outputs."""
+    flag = {0: 0, 1: based.BASED_STATE_SYM, 2: based.BASED_NUMERATOR_ONLY}[flags]
+    w = wl.Workload("ranges", B, H, L, 16, d_v, "bf16", 0.3)
+    q, k, v = wl.prefill_inputs(w, wl.generator(B + H + L))
+    sym = bool(flag & based.BASED_STATE_SYM)
+    kv, z = based.new_state(B, H, d_v, sym=sym)
+    kv.fill_(float("nan")); z.fill_(float("nan"))
+    out = torch.full_like(v, float("nan"), device=DEV)
+    based.based_prefill(q.to(DEV), k.to(DEV), v.to(DEV), out=out, kv_state=kv, z_state=z, flags=flag)
+    _poll()
+    y_ref, S_ref, z_ref = oracle.linattn_recurrent(_np(q), _np(k), _np(v))
+    if flag & based.BASED_NUMERATOR_ONLY:
+        y_ref = oracle.linattn_numerator(_np(q), _np(k), _np(v))
+    if sym:
+        S_ref, z_ref = oracle.state_to_sym(S_ref, z_ref)
+    assert row_err(_np(out), y_ref) <= TOL_BF16
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, "bf16")
+
+
 # --------------------------------------------------------------------------- very many heads
 def test_more_heads_than_one_grid_dimension_holds():
     """B*H = 70,000 heads of 128 tokens (bf16): the batch is cut into slabs of heads inside the library; heads on
