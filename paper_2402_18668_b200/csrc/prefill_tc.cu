@@ -130,19 +130,22 @@ struct Params {
 #endif
 };
 
-#ifdef BASED_TRACE
+#if defined(BASED_TRACE) && !defined(BASED_TRACE_CTA_ONLY)
 #define TRACE(role, c, ev)                                                                   \
     do {                                                                                     \
         if (p.trace && blockIdx.x == gridDim.x - 1 && blockIdx.y == 0 && (c) >= 0 && (c) < 64)           \
             p.trace[((role) * 64 + (c)) * 8 + (ev)] = clock64();                             \
     } while (0)
-// wall-clock entry / exit of every CTA, after the per-role events
-#define TRACE_CTA(which)                                                                                      \
-    do {                                                                                                      \
-        if (p.trace) p.trace[6 * 64 * 8 + (blockIdx.y * gridDim.x + blockIdx.x) * 2 + (which)] = global_timer_ns(); \
-    } while (0)
 #else
 #define TRACE(role, c, ev) do {} while (0)
+#endif
+#ifdef BASED_TRACE
+// wall-clock entry / exit of every CTA (with its SM), after the per-role events
+#define TRACE_CTA(which)                                                                                      \
+    do {                                                                                                      \
+        if (p.trace) p.trace[6 * 64 * 8 + (blockIdx.y * gridDim.x + blockIdx.x) * 2 + (which)] = (global_timer_ns() << 8) | smid_u32(); \
+    } while (0)
+#else
 #define TRACE_CTA(which) do {} while (0)
 #endif
 
@@ -278,6 +281,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     // phi(Q) in tensor memory and two state-copy tiles: the plain chunk loop only (measured: -7 % where every
     // SM has a CTA; the recompute mode's kernel loses 5 % with it)
     constexpr bool PQT = C::kPQinT && MODE == kModeMain;
+    // packed bf16 polynomial and the row sums by the tensor cores: the same kernel (measured: -6 % there, +14 % in
+    // the recompute mode's kernel)
+    constexpr bool PKW = PQT;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offMisc);
@@ -529,7 +535,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             constexpr uint64_t dV = make_smem_desc_base(kC * 128, 1024, kSwizzle128B);    // MN-major [128 tok][DV]
             constexpr uint32_t i1 = make_idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t i4 = make_idesc_bf16(128, C::kNY, 0, 0);
-            constexpr uint32_t i3 = make_idesc_bf16(128, DV, 0, 1);
+            // d_v 64, plain chunk loop: the values get 16 more columns from the ones block (column 64 = 1 for every token), so the same
+            // MMAs that apply the weights to V also add up each row's weights: the in-chunk part of the denominator
+            // lands in column 64 of Y, on top of the cross-chunk part that step (4) put there
+            constexpr uint32_t i3 = make_idesc_bf16(128, PKW ? DV + 16 : DV, 0, 1);
             const uint32_t lQK = desc_lo(dQK), lV = desc_lo(dV);
             const uint32_t lPQ = desc_lo(dPhiK) + (smem_u32(sPQ) >> 4), lSc0 = desc_lo(dPhiK) + (smem_u32(sSc) >> 4);
             // scores of chunk c: T[c & 1] (or the single T) = Q_c K_c^T
@@ -596,10 +605,12 @@ __global__ void __launch_bounds__(kThreads, 1)
                 TRACE(0, c, 5);
                 tc_fence_after();
                 {
-                    const uint32_t b_lo = lV + (aVt >> 4);
+                    // there the second 64-column block of the B operand is the ones block (leading byte offset)
+                    const uint64_t dVo = PKW ? make_smem_desc_base(smem_u32(sOnes) - aVt, 1024, kSwizzle128B) : dV;
+                    const uint32_t b_lo = desc_lo(dVo) + (aVt >> 4), b_hi = desc_hi(dVo);
 #pragma unroll
                     for (int k = 0; k < kC / 16; ++k)
-                        mma_ts_lh<true>(tb + C::colY, tb + colTc + k * 8, b_lo + k * (2048 >> 4), desc_hi(dV), i3);
+                        mma_ts_lh<true>(tb + C::colY, tb + colTc + k * 8, b_lo + k * (2048 >> 4), b_hi, i3);
                 }
                 TRACE(2, c, 2);
                 mma_commit(&bars[kG3]);
@@ -626,7 +637,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                 uint32_t dcol;
                 tmem_ld1(tmem_addr(tb, lane_base, C::colY + DV), dcol);
                 tmem_wait_ld();
-                const float inv = p.numerator_only ? 1.0f : 1.0f / (s_den[(c & 3) * kC + t] + __uint_as_float(dcol) + kEps);
+                const float den_in = PKW ? 0.f : s_den[(c & 3) * kC + t];      // packed variant: already in the column
+                const float inv = p.numerator_only ? 1.0f : 1.0f / (den_in + __uint_as_float(dcol) + kEps);
 #pragma unroll 1
                 for (int h = 0; h < DV / 64; ++h) {
                     uint32_t y0[32], y1[32];
@@ -954,7 +966,21 @@ __global__ void __launch_bounds__(kThreads, 1)
                     uint32_t sc[32];
                     tmem_ld32(tmem_addr(tb, lane_base, colTc + b * 32), sc);
                     tmem_wait_ld();
-                    if (b < q4) {                        // fully visible batch: no mask
+                    if constexpr (PKW) {
+                        // Two scores per instruction: the pair is rounded to bf16 first, w = 1 + s (1/4 + s/32) in
+                        // two packed fused multiply-adds, and the result is the packed weight as it is stored (it
+                        // would be rounded to bf16 anyway).  The row sum is the tensor cores' work (see step (3)).
+                        const __nv_bfloat162 c1 = __float2bfloat162_rn(0.25f), c2 = __float2bfloat162_rn(0.03125f),
+                                             one = __float2bfloat162_rn(1.0f);
+                        const int vis = (b < q4) ? 64 : lane + 1;      // columns of this batch the row may see
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const __nv_bfloat162 s2 = __floats2bfloat162_rn(__uint_as_float(sc[2 * i]), __uint_as_float(sc[2 * i + 1]));
+                            const __nv_bfloat162 w2 = __hfma2(s2, __hfma2(s2, c2, c1), one);
+                            const uint32_t w = *reinterpret_cast<const uint32_t*>(&w2);
+                            pk[i] = (2 * i + 1 < vis) ? w : ((2 * i < vis) ? (w & 0xFFFFu) : 0u);
+                        }
+                    } else if (b < q4) {                 // fully visible batch: no mask
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             const float s0 = __uint_as_float(sc[2 * i]), s1 = __uint_as_float(sc[2 * i + 1]);
@@ -987,8 +1013,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 }
                 tmem_st16(tmem_addr(tb, lane_base, colTc + b * 16), pk);
             }
-            const float den = den0 + den1;
-            s_den[(c & 3) * kC + tid] = den;
+            if constexpr (!PKW) s_den[(c & 3) * kC + tid] = den0 + den1;
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(&bars[kP + t_idx(c)]);
