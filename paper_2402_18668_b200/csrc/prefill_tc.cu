@@ -246,6 +246,29 @@ __device__ __forceinline__ void read_qk_row(const uint8_t* tile, int t, uint4& l
     hi = *reinterpret_cast<const uint4*>(row + (16 ^ sw));
 }
 
+// Packed fp32 pairs (sm_100 has two-wide fp32 multiply-add and add): a pair lives in one 64-bit register.
+__device__ __forceinline__ uint64_t f32x2(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void f32x2_split(uint64_t v, float& lo, float& hi) {
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
 __device__ __forceinline__ void group_sync(int id) {        // named barrier of one 128-thread group
     asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
 }
@@ -980,27 +1003,35 @@ __global__ void __launch_bounds__(kThreads, 1)
                             const uint32_t w = *reinterpret_cast<const uint32_t*>(&w2);
                             pk[i] = (2 * i + 1 < vis) ? w : ((2 * i < vis) ? (w & 0xFFFFu) : 0u);
                         }
-                    } else if (b < q4) {                 // fully visible batch: no mask
+                    } else {
+                        // fp32 polynomial on pairs of scores (two-wide fp32 multiply-add): t = s/32 + 1/4, w = s t + 1
+                        const uint64_t k2 = f32x2(__float_as_uint(0.03125f), __float_as_uint(0.03125f)),
+                                       k1 = f32x2(__float_as_uint(0.25f), __float_as_uint(0.25f)),
+                                       k0 = f32x2(__float_as_uint(1.0f), __float_as_uint(1.0f));
+                        uint64_t den2 = f32x2(__float_as_uint(den0), __float_as_uint(den1));
+                        if (b < q4) {                    // fully visible batch: no mask
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const float s0 = __uint_as_float(sc[2 * i]), s1 = __uint_as_float(sc[2 * i + 1]);
-                            const float w0 = fmaf(s0, fmaf(s0, 0.03125f, 0.25f), 1.0f);
-                            const float w1 = fmaf(s1, fmaf(s1, 0.03125f, 0.25f), 1.0f);
-                            den0 += w0;
-                            den1 += w1;
-                            pk[i] = pack_bf16(w0, w1);
-                        }
-                    } else {                             // the batch that holds the diagonal
+                            for (int i = 0; i < 16; ++i) {
+                                const uint64_t s2 = f32x2(sc[2 * i], sc[2 * i + 1]);
+                                const uint64_t w2 = fma2(s2, fma2(s2, k2, k1), k0);
+                                den2 = add2(den2, w2);
+                                float w0, w1;
+                                f32x2_split(w2, w0, w1);
+                                pk[i] = pack_bf16(w0, w1);
+                            }
+                            f32x2_split(den2, den0, den1);
+                        } else {                         // the batch that holds the diagonal
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const float s0 = __uint_as_float(sc[2 * i]), s1 = __uint_as_float(sc[2 * i + 1]);
-                            float w0 = fmaf(s0, fmaf(s0, 0.03125f, 0.25f), 1.0f);
-                            float w1 = fmaf(s1, fmaf(s1, 0.03125f, 0.25f), 1.0f);
-                            w0 = (2 * i <= lane) ? w0 : 0.f;
-                            w1 = (2 * i + 1 <= lane) ? w1 : 0.f;
-                            den0 += w0;
-                            den1 += w1;
-                            pk[i] = pack_bf16(w0, w1);
+                            for (int i = 0; i < 16; ++i) {
+                                const uint64_t s2 = f32x2(sc[2 * i], sc[2 * i + 1]);
+                                float w0, w1;
+                                f32x2_split(fma2(s2, fma2(s2, k2, k1), k0), w0, w1);
+                                w0 = (2 * i <= lane) ? w0 : 0.f;
+                                w1 = (2 * i + 1 <= lane) ? w1 : 0.f;
+                                den0 += w0;
+                                den1 += w1;
+                                pk[i] = pack_bf16(w0, w1);
+                            }
                         }
                     }
                 } else {
