@@ -194,3 +194,19 @@ def test_binding_rejects_cpu_tensors():
     v = torch.zeros(1, 1, 4, 64)
     with pytest.raises(ValueError):
         binding.based_prefill(q, q.clone(), v)
+
+
+def test_generation_step_validation(lib):
+    """based_generation_step checks its arguments before anything is launched (no GPU needed)."""
+    f = lib.based_generation_step
+    Q = ctypes.c_void_p(0x3000)
+
+    def call(q=P, kv=Q, out=ctypes.c_void_p(0x2000), qw=P, pos=ctypes.c_void_p(0x4000), B=1, H=2, d_feat=16, d_v=64, Hw=2,
+             d_w=64, window=64, io=1, flags=0):
+        return f(q, P, P, kv, Q, out, qw, P, P, Q, Q, ctypes.c_void_p(0x5000), B, H, d_feat, d_v, Hw, d_w, window, pos,
+                 ctypes.c_float(0.0), io, flags, None)
+
+    assert call(q=None) == 1 and call(kv=None) == 1 and call(pos=None) == 1 and call(B=0) == 1 and call(Hw=0) == 1
+    assert call(io=5) == 1 and call(flags=1) == 1           # BASED_STATE_CONTINUE means nothing for a step
+    assert call(d_feat=8) == 2 and call(d_v=96) == 2 and call(d_w=128) == 2 and call(window=129) == 2
+    assert call(q=U) == 3 and call(pos=ctypes.c_void_p(0x4004)) == 3
