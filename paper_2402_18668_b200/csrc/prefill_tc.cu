@@ -803,14 +803,18 @@ __global__ void __launch_bounds__(kThreads, 1)
                 tc_fence_after();
                 // bf16 copy of this lane's state row, held in registers until the tile is free
                 uint32_t pkd[kF / 2];
+                // d_v 64: lanes 65..127 of S^T hold nothing, so the group's last warp (lanes 96..127) has no row to
+                // copy: it only keeps the barriers' arrival counts whole
+                if (DV == 128 || t < 96) {
 #pragma unroll
-                for (int b = 0; b < kF / 16; ++b) {
-                    uint32_t r[16];
-                    tmem_ld16(tmem_addr(tb, lane_base, C::colS + b * 16), r);
-                    tmem_wait_ld();
+                    for (int b = 0; b < kF / 16; ++b) {
+                        uint32_t r[16];
+                        tmem_ld16(tmem_addr(tb, lane_base, C::colS + b * 16), r);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        pkd[b * 8 + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                        for (int i = 0; i < 8; ++i)
+                            pkd[b * 8 + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                    }
                 }
                 uint32_t z0 = 0, z1 = 0;
                 if (DV == 128) {
