@@ -303,6 +303,16 @@ based_status swa_decode_step_at(const void* q, const void* k, const void* v, voi
                                 float softmax_scale, based_dtype io, void* cuda_stream);
 
 /*
+ * The same step for a batch whose sequences have different lengths (Algorithm 3 takes one position; a
+ * serving batch does not share one): pos_per_sequence is an array of B ints in device memory, the
+ * position of sequence b's new token (>= 0); every head of sequence b uses slot pos[b] % window of its
+ * cache and attends to min(pos[b] + 1, window) keys.  The caller advances the positions.
+ */
+based_status swa_decode_step_ragged(const void* q, const void* k, const void* v, void* k_cache, void* v_cache,
+                                    void* out, int B, int H, int d, int window, const int* pos_per_sequence,
+                                    float softmax_scale, based_dtype io, void* cuda_stream);
+
+/*
  * The same step for a generation loop that is replayed as a CUDA graph: pos_state points to two
  * ints in device memory, {position, ticket} (ticket 0 before the first call).  The step reads the
  * position like swa_decode_step_at and stores position + 1 when it ends, so the loop needs no

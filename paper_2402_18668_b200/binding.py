@@ -28,7 +28,7 @@ EXPORTS = (
     "based_static_scratch_bytes", "based_selftest_bounded_wait", "swa_decode_step", "based_decode_step_sym",
     "based_state_to_sym", "based_state_from_sym", "swa_decode_step_at", "based_preload_decode",
     "baseconv_gate_forward", "baseconv_gate_step", "based_decode_step_flags", "based_prefill_backward",
-    "based_prefill_backward_workspace_bytes", "based_prefill_backward_with_out", "based_prefill_backward_block_tokens", "swa_decode_step_advance", "based_generation_step",
+    "based_prefill_backward_workspace_bytes", "based_prefill_backward_with_out", "based_prefill_backward_block_tokens", "swa_decode_step_advance", "swa_decode_step_ragged", "based_generation_step",
     "based_prefill_state", "based_prefill_state_workspace_bytes",
 )
 
@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
         L.swa_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
         L.swa_decode_step_at.restype = i
         L.swa_decode_step_at.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, i, vp]
+        L.swa_decode_step_ragged.restype = i
+        L.swa_decode_step_ragged.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, i, vp]
         L.swa_decode_step_advance.restype = i
         L.swa_decode_step_advance.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, i, vp]
         L.based_generation_step.restype = i
@@ -407,6 +409,25 @@ def swa_decode_step(q, k, v, k_cache, v_cache, pos: int, out=None, softmax_scale
     st = lib().swa_decode_step(_ptr(q), _ptr(k), _ptr(v), _ptr(k_cache), _ptr(v_cache), _ptr(out), B, H, d, window,
                                int(pos), float(softmax_scale), _dtype_code(q), _stream(stream))
     _check(st, "swa_decode_step")
+    return out
+
+
+def swa_decode_step_ragged(q, k, v, k_cache, v_cache, pos, out=None, softmax_scale: float = 0.0, stream=None):
+    """swa_decode_step for sequences of different lengths: pos is an int32 tensor [B] on the device, the position
+    of each sequence's new token."""
+    _dev(q, k, v, k_cache, v_cache, pos, out)
+    B, H, d = q.shape
+    window = k_cache.shape[2]
+    _check_qkv(q, k, v, out)
+    if k_cache.shape != (B, H, window, d) or v_cache.shape != k_cache.shape or k_cache.dtype != q.dtype:
+        raise ValueError("cache shapes/dtypes disagree with q")
+    if pos.dtype != torch.int32 or tuple(pos.shape) != (B,):
+        raise ValueError("pos is an int32 tensor with one entry per sequence")
+    if out is None:
+        out = torch.empty_like(v)
+    st = lib().swa_decode_step_ragged(_ptr(q), _ptr(k), _ptr(v), _ptr(k_cache), _ptr(v_cache), _ptr(out), B, H, d, window,
+                                      _ptr(pos), float(softmax_scale), _dtype_code(q), _stream(stream))
+    _check(st, "swa_decode_step_ragged")
     return out
 
 

@@ -310,6 +310,22 @@ based_status swa_decode_step_at(const void* q, const void* k, const void* v, voi
                              static_cast<cudaStream_t>(cuda_stream));
 }
 
+based_status swa_decode_step_ragged(const void* q, const void* k, const void* v, void* k_cache, void* v_cache,
+                                    void* out, int B, int H, int d, int window, const int* pos_per_sequence,
+                                    float softmax_scale, based_dtype io, void* cuda_stream) {
+    if (!q || !k || !v || !k_cache || !v_cache || !out || !pos_per_sequence || B <= 0 || H <= 0 || window <= 0)
+        return BASED_ERR_INVALID_ARG;
+    if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
+    if (d != 64 || window > 128) return BASED_ERR_UNSUPPORTED;
+    if ((long long)B * H > 0x7fffffffLL) return BASED_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(k_cache) || !aligned16(v_cache) ||
+        !aligned16(out) || (reinterpret_cast<uintptr_t>(pos_per_sequence) & 3u))
+        return BASED_ERR_ALIGNMENT;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 0.125f;   // 1/sqrt(64)
+    return launch_swa_decode(q, k, v, k_cache, v_cache, out, B * H, window, 0, pos_per_sequence, nullptr, scale, io,
+                             static_cast<cudaStream_t>(cuda_stream), H);
+}
+
 based_status swa_decode_step_advance(const void* q, const void* k, const void* v, void* k_cache, void* v_cache,
                                      void* out, int B, int H, int d, int window, int* pos_state,
                                      float softmax_scale, based_dtype io, void* cuda_stream) {

@@ -96,7 +96,7 @@ based_status launch_swa_tc(const void* q, const void* k, const void* v, void* ou
 // pos_adv != nullptr ({position, ticket}, pos_dev == pos_adv): the kernel also stores position + 1 at its end
 based_status launch_swa_decode(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
                                int window, int pos, const int* pos_dev, int* pos_adv, float scale, based_dtype io,
-                               cudaStream_t stream);
+                               cudaStream_t stream, int pos_group = 0);
 // gated short convolution (BaseConv core); step: one token on a [B, width-1, C] state, N ignored
 based_status launch_baseconv(const void* a, const void* g, const float* h, const float* b2, void* state, void* out,
                              int B, int N, int C, int width, bool step, based_dtype io, cudaStream_t stream);

@@ -22,16 +22,16 @@ template <typename T, int NPW>
 __global__ void __launch_bounds__(32 * kWarps)
 swa_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, T* __restrict__ kc,
                   T* __restrict__ vc, T* __restrict__ out, int window, int pos_arg,
-                  const int* pos_dev, int* pos_adv, float scale, unsigned int* __restrict__ error_word) {
+                  const int* pos_dev, int* pos_adv, float scale, unsigned int* __restrict__ error_word, int pos_group) {
     extern __shared__ __align__(128) unsigned char smem[];
     swa_decode_body<T, NPW, 1>(q, k, v, kc, vc, out, window, pos_arg, pos_dev, pos_adv, scale, error_word, blockIdx.x,
-                               threadIdx.x, (int)gridDim.x, smem);
+                               threadIdx.x, (int)gridDim.x, smem, pos_group);
 }
 
 template <typename T, int NPW>
 static based_status launch_n(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
                              int window, int pos, const int* pos_dev, int* pos_adv, float scale, unsigned int* err,
-                             cudaStream_t stream) {
+                             cudaStream_t stream, int pos_group) {
     const size_t smem = swa_decode_smem_bytes<T>(window);
     if (smem > 48 * 1024) {
         if (cudaFuncSetAttribute(swa_decode_kernel<T, NPW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -41,7 +41,7 @@ static based_status launch_n(const void* q, const void* k, const void* v, void* 
     swa_decode_kernel<T, NPW><<<BH, 32 * kWarps, smem, stream>>>(static_cast<const T*>(q), static_cast<const T*>(k),
                                                           static_cast<const T*>(v), static_cast<T*>(kc),
                                                           static_cast<T*>(vc), static_cast<T*>(out), window, pos,
-                                                          pos_dev, pos_adv, scale, err);
+                                                          pos_dev, pos_adv, scale, err, pos_group);
     note_launch();
     return check_launch("swa_decode_kernel");
 }
@@ -49,9 +49,9 @@ static based_status launch_n(const void* q, const void* k, const void* v, void* 
 template <typename T>
 static based_status launch_t(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
                              int window, int pos, const int* pos_dev, int* pos_adv, float scale, unsigned int* err,
-                             cudaStream_t stream) {
-    if (window <= 64) return launch_n<T, 4>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream);
-    return launch_n<T, 8>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream);
+                             cudaStream_t stream, int pos_group) {
+    if (window <= 64) return launch_n<T, 4>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream, pos_group);
+    return launch_n<T, 8>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream, pos_group);
 }
 
 based_status preload_swa_decode() {
@@ -65,13 +65,13 @@ based_status preload_swa_decode() {
 
 based_status launch_swa_decode(const void* q, const void* k, const void* v, void* kc, void* vc, void* out, int BH,
                                int window, int pos, const int* pos_dev, int* pos_adv, float scale, based_dtype io,
-                               cudaStream_t stream) {
+                               cudaStream_t stream, int pos_group) {
     unsigned int* err = nullptr;
     const based_status st = error_word_ptr(&err);
     if (st != BASED_OK) return st;
     if (io == BASED_F32)
-        return launch_t<float>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream);
-    return launch_t<__nv_bfloat16>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream);
+        return launch_t<float>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream, pos_group);
+    return launch_t<__nv_bfloat16>(q, k, v, kc, vc, out, BH, window, pos, pos_dev, pos_adv, scale, err, stream, pos_group);
 }
 
 }  // namespace based

@@ -69,12 +69,14 @@ __device__ __forceinline__ void swa_decode_body(const T* __restrict__ q, const T
                                                 const T* __restrict__ v, T* __restrict__ kc, T* __restrict__ vc,
                                                 T* __restrict__ out, int window, int pos_arg, const int* pos_dev,
                                                 int* pos_adv, float scale, unsigned int* __restrict__ error_word,
-                                                size_t head, int tid, int n_tickets, unsigned char* smem) {
+                                                size_t head, int tid, int n_tickets, unsigned char* smem, int pos_group = 0) {
     auto group_sync = [&]() { asm volatile("bar.sync %0, 128;" ::"n"(BAR) : "memory"); };
     // the position comes from device memory when the launch is part of a captured graph that is
     // replayed as the sequence grows.  In advance mode pos_dev and pos_adv name the same word, which
     // the last CTA rewrites at its end: no restrict on either, and the read is a volatile one
-    const int pos = pos_dev ? *reinterpret_cast<const volatile int*>(pos_dev) : pos_arg;
+    // pos_group > 0: one position per sequence (pos_dev[b], b = head / pos_group) for batches whose sequences
+    // have different lengths
+    const int pos = pos_dev ? *reinterpret_cast<const volatile int*>(pos_dev + (pos_group > 0 ? head / pos_group : 0)) : pos_arg;
     T* s_K = reinterpret_cast<T*>(smem);
     T* s_V = s_K + (size_t)window * kHD;
     T* s_qn = s_V + (size_t)window * kHD;

@@ -859,6 +859,34 @@ def test_swa_decode_full_batch():
     assert np.array_equal(_np(kc), kc_ref) and np.array_equal(_np(vc), vc_ref)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_swa_decode_sequences_of_different_lengths(dtype):
+    """swa_decode_step_ragged: five sequences at positions before, at and past the point where the ring wraps, each
+    against the whole-sequence oracle of its own length; the caches are updated in the right slots."""
+    B, H, window, d = 5, 3, 16, 64
+    pos = [0, 7, 15, 16, 45]
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    g = wl.generator(77)
+    Lmax = max(pos) + 1
+    qs, ks, vs = ((torch.randn(B, H, Lmax, d, generator=g)).to(tdt) for _ in range(3))
+    kc = torch.full((B, H, window, d), float("nan"), dtype=tdt, device=DEV)
+    vc = torch.full_like(kc, float("nan"))
+    # fill each sequence's ring with its own history (tokens 0 .. pos-1), sequence by sequence
+    for b in range(B):
+        for t in range(pos[b]):
+            based.swa_decode_step(qs[b:b + 1, :, t].contiguous().to(DEV), ks[b:b + 1, :, t].contiguous().to(DEV),
+                                  vs[b:b + 1, :, t].contiguous().to(DEV), kc[b:b + 1], vc[b:b + 1], pos=t)
+    idx = torch.tensor(pos)
+    take = lambda x: torch.stack([x[b, :, pos[b]] for b in range(B)]).contiguous().to(DEV)
+    out = based.swa_decode_step_ragged(take(qs), take(ks), take(vs), kc, vc, idx.to(torch.int32).to(DEV))
+    _poll()
+    for b in range(B):
+        L = pos[b] + 1
+        ref = oracle.swa(_np(qs[b:b + 1, :, :L]), _np(ks[b:b + 1, :, :L]), _np(vs[b:b + 1, :, :L]), window)
+        assert row_err(_np(out[b:b + 1]), ref[:, :, -1]) <= tol_for(dtype), b
+        assert torch.equal(kc[b, :, pos[b] % window].cpu(), ks[b, :, pos[b]]) and torch.equal(vc[b, :, pos[b] % window].cpu(), vs[b, :, pos[b]])
+
+
 def test_swa_decode_matches_forward_on_gpu():
     """The decode chain and swa_forward agree on the same sequence (both against the oracle above)."""
     B, H, L, d, w = 2, 4, 200, 64, 64
