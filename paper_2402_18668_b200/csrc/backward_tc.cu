@@ -251,9 +251,12 @@ __global__ void __launch_bounds__(kThreadsB, 1)
     constexpr uint32_t iXV = make_idesc_bf16(128, 64 * C::kVB, 0, 0);                   // A from TMEM, B K-major: the state over features
 
     if (warp == 4) {
-        if (lane == 0) {
+        {
+            // the whole warp runs this block; one elected lane issues the MMAs, commits and loads (see mma_ss_w)
+            const uint32_t lead = elect_one();
             const uint32_t aResN = smem_u32(smem + C::offResN), aResW = smem_u32(smem + C::offResW);
             auto load_stage = [&](int it) {
+                if (!lead) return;
                 const int s = it & 1;
                 uint8_t* st = smem + C::offStage + s * C::kStage;
                 const int row = (first + it) * LT;
@@ -263,6 +266,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                 for (int b = 0; b < C::kVB; ++b)
                     tma_load_3d(st + C::kNarrowL + b * (LT * 128), &tm_w1, &bars[bFull0 + s], b * 64, row, head);
             };
+            if (lead) {
             mbar_arrive_expect_tx(&bars[bRes], MODE == kModeFwd ? kQKTile : kQKTile + C::kWide);
             tma_load_3d(smem + C::offResN, &tm_n0, &bars[bRes], 0, r0, head);
             if (MODE != kModeFwd) {
@@ -277,6 +281,7 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                     tma_load_3d(smem + C::offStage + C::kStage + b * C::kStateBlk, &tm_st, &bars[bXs], b * 32, 0,
                                 head * p.nblk + blk);
             }
+            }
             load_stage(0);
             ok = mbar_wait(&bars[bRes], 0, abort_flag);
             if (cross && ok) {
@@ -289,13 +294,13 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                     const uint32_t off = ((kk >> 2) * (kTile * 128) + (kk & 3) * 32) >> 4;
                     const uint32_t offS = (kk * 1024) >> 4;        // sixteen value columns = sixteen 64-byte rows of every block
                     if (kk == 0)
-                        mma_ss_lh<false>(tb, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW), desc_lo(dStN) + (aSt >> 4) + offS,
+                        mma_ss_w<false>(lead, tb, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW), desc_lo(dStN) + (aSt >> 4) + offS,
                                          desc_hi(dStN), iT);
                     else
-                        mma_ss_lh<true>(tb, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW), desc_lo(dStN) + (aSt >> 4) + offS,
+                        mma_ss_w<true>(lead, tb, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW), desc_lo(dStN) + (aSt >> 4) + offS,
                                         desc_hi(dStN), iT);
                 }
-                mma_commit(&bars[bX0]);
+                mma_commit_w(lead, &bars[bX0]);
                 if (MODE == kModeDkDv) {
                     // dV = mono(K) (tensor memory, written by the row threads) x state (K-major: 64-byte rows of 32
                     // features, 160 = 10 K-steps of 32 bytes)
@@ -306,9 +311,9 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                         for (int k = 0; k < 10; ++k) {
                             const uint32_t offK = ((k >> 1) * C::kStateBlk + (k & 1) * 32) >> 4;
                             if (k == 0)
-                                mma_ts_lh<false>(tb + C::colAcc, tb + k * 8, desc_lo(dN) + (aSt >> 4) + offK, desc_hi(dN), iXV);
+                                mma_ts_w<false>(lead, tb + C::colAcc, tb + k * 8, desc_lo(dN) + (aSt >> 4) + offK, desc_hi(dN), iXV);
                             else
-                                mma_ts_lh<true>(tb + C::colAcc, tb + k * 8, desc_lo(dN) + (aSt >> 4) + offK, desc_hi(dN), iXV);
+                                mma_ts_w<true>(lead, tb + C::colAcc, tb + k * 8, desc_lo(dN) + (aSt >> 4) + offK, desc_hi(dN), iXV);
                         }
                     }
                 } else {
@@ -324,10 +329,10 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                 if (!ok) break;
                 tc_fence_after();
                 // scores: rows = own tile, columns = looped tile
-                mma_ss_lh<false>(tb + C::colS, desc_lo(dN) + (aResN >> 4), desc_hi(dN), desc_lo(dN) + (aN >> 4),
+                mma_ss_w<false>(lead, tb + C::colS, desc_lo(dN) + (aResN >> 4), desc_hi(dN), desc_lo(dN) + (aN >> 4),
                                  desc_hi(dN), iS);
                 if (p.kdim > 16)                             // feature dimensions 24 and 32: second K-step
-                    mma_ss_lh<true>(tb + C::colS, desc_lo(dN) + (aResN >> 4) + 2, desc_hi(dN), desc_lo(dN) + (aN >> 4) + 2,
+                    mma_ss_w<true>(lead, tb + C::colS, desc_lo(dN) + (aResN >> 4) + 2, desc_hi(dN), desc_lo(dN) + (aN >> 4) + 2,
                                     desc_hi(dN), iS);
                 // own wide tile x looped wide tile^T over d_v
 #pragma unroll
@@ -335,13 +340,13 @@ __global__ void __launch_bounds__(kThreadsB, 1)
                     const uint32_t off = ((kk >> 2) * (kTile * 128) + (kk & 3) * 32) >> 4;
                     const uint32_t offL = ((kk >> 2) * (LT * 128) + (kk & 3) * 32) >> 4;
                     if (kk == 0)
-                        mma_ss_lh<false>(tb + C::colG, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW),
+                        mma_ss_w<false>(lead, tb + C::colG, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW),
                                          desc_lo(dWL) + (aW >> 4) + offL, desc_hi(dWL), iS);
                     else
-                        mma_ss_lh<true>(tb + C::colG, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW),
+                        mma_ss_w<true>(lead, tb + C::colG, desc_lo(dW) + (aResW >> 4) + off, desc_hi(dW),
                                         desc_lo(dWL) + (aW >> 4) + offL, desc_hi(dWL), iS);
                 }
-                mma_commit(&bars[bMma]);
+                mma_commit_w(lead, &bars[bMma]);
                 // once these products are done, so are the previous iteration's (in-order pipe): its stage is free
                 ok = mbar_wait(&bars[bMma], it & 1, abort_flag);
                 if (!ok) break;
@@ -354,10 +359,10 @@ __global__ void __launch_bounds__(kThreadsB, 1)
 #pragma unroll
                     for (int k = 0; k < LT / 16; ++k) {
                         if (it == 0 && k == 0)
-                            mma_ts_lh<false>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                            mma_ts_w<false>(lead, tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                              desc_hi(dN), iN32);
                         else
-                            mma_ts_lh<true>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                            mma_ts_w<true>(lead, tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                             desc_hi(dN), iN32);
                     }
                 } else if (MODE == kModeDqS) {
@@ -365,14 +370,14 @@ __global__ void __launch_bounds__(kThreadsB, 1)
 #pragma unroll
                     for (int k = 0; k < LT / 16; ++k) {
                         if (it == 0 && k == 0 && !cross) {
-                            mma_ts_lh<false>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                            mma_ts_w<false>(lead, tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                              desc_hi(dN), iN32);
-                            mma_ts_lh<false>(tb + C::colAcc2, tb + C::colD2 + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                            mma_ts_w<false>(lead, tb + C::colAcc2, tb + C::colD2 + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                              desc_hi(dN), iN32);
                         } else {
-                            mma_ts_lh<true>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                            mma_ts_w<true>(lead, tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                             desc_hi(dN), iN32);
-                            mma_ts_lh<true>(tb + C::colAcc2, tb + C::colD2 + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                            mma_ts_w<true>(lead, tb + C::colAcc2, tb + C::colD2 + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                             desc_hi(dN), iN32);
                         }
                     }
@@ -381,10 +386,10 @@ __global__ void __launch_bounds__(kThreadsB, 1)
 #pragma unroll
                     for (int k = 0; k < LT / 16; ++k) {
                         if (it == 0 && k == 0)
-                            mma_ts_lh<false>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
+                            mma_ts_w<false>(lead, tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
                                              desc_hi(dWL), iNV);
                         else
-                            mma_ts_lh<true>(tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
+                            mma_ts_w<true>(lead, tb + C::colAcc, tb + C::colD + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
                                             desc_hi(dWL), iNV);
                     }
                 } else if (MODE == kModeDkDv) {
@@ -392,20 +397,20 @@ __global__ void __launch_bounds__(kThreadsB, 1)
 #pragma unroll
                     for (int k = 0; k < LT / 16; ++k) {
                         if (it == 0 && k == 0 && !cross) {
-                            mma_ts_lh<false>(tb + C::colAcc, tb + C::colS + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
+                            mma_ts_w<false>(lead, tb + C::colAcc, tb + C::colS + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
                                              desc_hi(dWL), iNV);
-                            mma_ts_lh<false>(tb + C::colK, tb + C::colG + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                            mma_ts_w<false>(lead, tb + C::colK, tb + C::colG + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                              desc_hi(dN), iN32);
                         } else {
-                            mma_ts_lh<true>(tb + C::colAcc, tb + C::colS + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
+                            mma_ts_w<true>(lead, tb + C::colAcc, tb + C::colS + k * 8, desc_lo(dWL) + ((aW + k * 2048) >> 4),
                                             desc_hi(dWL), iNV);
-                            mma_ts_lh<true>(tb + C::colK, tb + C::colG + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
+                            mma_ts_w<true>(lead, tb + C::colK, tb + C::colG + k * 8, desc_lo(dN) + ((aN + k * 1024) >> 4),
                                             desc_hi(dN), iN32);
                         }
                     }
                 }
             }
-            if (ok) mma_commit(&bars[bFinal]);
+            if (ok) mma_commit_w(lead, &bars[bFinal]);
         }
     } else {
         // ===================================================================== row threads

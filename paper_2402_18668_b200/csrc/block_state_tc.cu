@@ -147,12 +147,15 @@ __global__ void __launch_bounds__(kThreadsR, 1)
     bool ok = true;
 
     if (warp == 8) {
-        if (lane == 0) {
+        {
+            // the whole warp runs this block; one elected lane issues the MMAs, commits and loads (see mma_ss_w)
+            const uint32_t lead = elect_one();
             constexpr uint64_t dPhi = make_smem_desc_base(kPhiBlk, 512, kSwizzle64B);          // B, MN-major: 32-feature blocks
             constexpr uint64_t dV = make_smem_desc_base(kTok * 128, 1024, kSwizzle128B);       // A, MN-major: 64-column blocks
             constexpr uint32_t iS = make_idesc_bf16(128, 160, 1, 1);
             constexpr uint32_t iZ = make_idesc_bf16(64, 160, 1, 1);
             auto load = [&](int it) {
+                if (!lead) return;
                 const int s = it % kNSR;
                 uint8_t* st = smem + C::offV + s * C::kVBytes;
                 mbar_arrive_expect_tx(&bars[rFull0 + s], C::kVBytes);
@@ -187,9 +190,9 @@ __global__ void __launch_bounds__(kThreadsR, 1)
 #pragma unroll
                     for (int k = 0; k < kTok / 16; ++k) {
                         if (first && k == 0)
-                            mma_ss_lh<false>(dS, a_lo + k * 128, a_hi, lPhi + k * 64, desc_hi(dPhi), iS);
+                            mma_ss_w<false>(lead, dS, a_lo + k * 128, a_hi, lPhi + k * 64, desc_hi(dPhi), iS);
                         else
-                            mma_ss_lh<true>(dS, a_lo + k * 128, a_hi, lPhi + k * 64, desc_hi(dPhi), iS);
+                            mma_ss_w<true>(lead, dS, a_lo + k * 128, a_hi, lPhi + k * 64, desc_hi(dPhi), iS);
                     }
                 } else {
                     const uint32_t a_lo = desc_lo(dV) + (aV >> 4), w_lo = desc_lo(dV) + (aW >> 4);
@@ -197,17 +200,17 @@ __global__ void __launch_bounds__(kThreadsR, 1)
                     for (int k = 0; k < kTok / 16; ++k) {
                         // the weights rows' accumulator is never started over: blocks alternate between two pairs of
                         // its lanes (the weights block's columns 0, 1 or 2, 3), each pair a running sum
-                        if (first && k == 0) mma_ss_lh<false>(dS, a_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iS);
-                        else mma_ss_lh<true>(dS, a_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iS);
+                        if (first && k == 0) mma_ss_w<false>(lead, dS, a_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iS);
+                        else mma_ss_w<true>(lead, dS, a_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iS);
                         if (it == 0 && k == 0)
-                            mma_ss_lh<false>(tb + C::colZ, w_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iZ);
+                            mma_ss_w<false>(lead, tb + C::colZ, w_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iZ);
                         else
-                            mma_ss_lh<true>(tb + C::colZ, w_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iZ);
+                            mma_ss_w<true>(lead, tb + C::colZ, w_lo + k * 128, desc_hi(dV), lPhi + k * 64, desc_hi(dPhi), iZ);
                     }
                 }
-                mma_commit(&bars[rMma0 + b]);
+                mma_commit_w(lead, &bars[rMma0 + b]);
                 if (ends_block(it)) {
-                    mma_commit(&bars[rFlush0 + a]);          // the block's sums are complete: the row threads read them
+                    mma_commit_w(lead, &bars[rFlush0 + a]);          // the block's sums are complete: the row threads read them
                     ++nblk_done;
                 }
                 // the previous step's products are done long since: its stage takes the load kNSR steps ahead

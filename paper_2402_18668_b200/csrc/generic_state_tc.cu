@@ -119,13 +119,16 @@ __global__ void __launch_bounds__(kThreadsS, 1)
     bool ok = true;
 
     if (warp == 4) {
-        if (lane == 0) {
+        {
+            // the whole warp runs this block; one elected lane issues the MMAs, commits and loads (see mma_ss_w)
+            const uint32_t lead = elect_one();
             constexpr uint64_t dA = make_smem_desc_base(16, 1024, kSwizzle128B);              // K-major, one 64-token block
             constexpr uint64_t dV = make_smem_desc_base(kTB * 128, 1024, kSwizzle128B);       // MN-major, 64-column blocks
             constexpr uint32_t iV = make_idesc_bf16(128, 64 * C::kVB, 0, 1);
             constexpr uint32_t iZ = make_idesc_bf16(128, 16, 0, 0);
             const uint32_t aOnes = smem_u32(smem + C::offOnes);
             auto load = [&](int it) {
+                if (!lead) return;
                 const int s = it % C::kNS;
                 uint8_t* st = smem + s * C::kStage;
                 mbar_arrive_expect_tx(&bars[sFull0 + s], C::kStage);
@@ -146,18 +149,18 @@ __global__ void __launch_bounds__(kThreadsS, 1)
 #pragma unroll
                 for (int kk = 0; kk < kTB / 16; ++kk) {
                     if (it == 0 && kk == 0) {
-                        mma_ss_lh<false>(tb, desc_lo(dA) + ((aA + kk * 32) >> 4), desc_hi(dA),
+                        mma_ss_w<false>(lead, tb, desc_lo(dA) + ((aA + kk * 32) >> 4), desc_hi(dA),
                                          desc_lo(dV) + ((aV + kk * 2048) >> 4), desc_hi(dV), iV);
-                        mma_ss_lh<false>(tb + C::colZ, desc_lo(dA) + ((aA + kk * 32) >> 4), desc_hi(dA),
+                        mma_ss_w<false>(lead, tb + C::colZ, desc_lo(dA) + ((aA + kk * 32) >> 4), desc_hi(dA),
                                          desc_lo(dA) + ((aOnes + kk * 32) >> 4), desc_hi(dA), iZ);
                     } else {
-                        mma_ss_lh<true>(tb, desc_lo(dA) + ((aA + kk * 32) >> 4), desc_hi(dA),
+                        mma_ss_w<true>(lead, tb, desc_lo(dA) + ((aA + kk * 32) >> 4), desc_hi(dA),
                                         desc_lo(dV) + ((aV + kk * 2048) >> 4), desc_hi(dV), iV);
-                        mma_ss_lh<true>(tb + C::colZ, desc_lo(dA) + ((aA + kk * 32) >> 4), desc_hi(dA),
+                        mma_ss_w<true>(lead, tb + C::colZ, desc_lo(dA) + ((aA + kk * 32) >> 4), desc_hi(dA),
                                         desc_lo(dA) + ((aOnes + kk * 32) >> 4), desc_hi(dA), iZ);
                     }
                 }
-                mma_commit(&bars[sMma0 + b]);
+                mma_commit_w(lead, &bars[sMma0 + b]);
                 // the previous step's products are done long since: its stage takes the load kNS steps ahead
                 if (it >= 1 && it - 1 + C::kNS < nit) {
                     ok = mbar_wait(&bars[sMma0 + (it - 1) % kNA], ((it - 1) / kNA) & 1, abort_flag);
@@ -165,7 +168,7 @@ __global__ void __launch_bounds__(kThreadsS, 1)
                     load(it - 1 + C::kNS);
                 }
             }
-            if (ok) mma_commit(&bars[sFinal]);
+            if (ok) mma_commit_w(lead, &bars[sFinal]);
         }
     } else {
         // ===================================================================== row threads

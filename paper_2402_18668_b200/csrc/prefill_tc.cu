@@ -491,7 +491,9 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
     } else if (warp == kWarpMma) {
         // ===================================================================== MMA issuer, state chain
-        if (lane == 0) {
+        // (the whole warp runs the loop and one elected lane issues: see mma_ss_w)
+        const uint32_t lead = elect_one();
+        {
             constexpr uint64_t dPhiMN = make_smem_desc_base(C::kPhiBlk, 512, kSwizzle64B);// MN-major view of a phi tile
             constexpr uint64_t dV = make_smem_desc_base(kC * 128, 1024, kSwizzle128B);    // MN-major [128 tok][DV]
             constexpr uint64_t dOnes = make_smem_desc_base(16, 1024, kSwizzle128B);
@@ -519,7 +521,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     }
                 }
                 if (!ok) break;
-                TRACE(1, c, 1);
+                if (lane == 0) TRACE(1, c, 1);
                 tc_fence_after();
                 if (DV == 64) {
                     // V^T as a 128-row A operand: rows 0..63 from the V tile, rows 64..127 from the ones
@@ -528,31 +530,32 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const uint32_t a_lo = desc_lo(dV1) + (aVt >> 4), a_hi = desc_hi(dV1);
 #pragma unroll
                     for (int k = 0; k < kC / 16; ++k)
-                        mma_ss_lh<true>(tb + C::colS, a_lo + k * (2048 >> 4), a_hi, lPK + k * (1024 >> 4),
+                        mma_ss_w<true>(lead, tb + C::colS, a_lo + k * (2048 >> 4), a_hi, lPK + k * (1024 >> 4),
                                         desc_hi(dPhiMN), i5);
                 } else {
                     const uint32_t a_lo = lV + (aVt >> 4);
 #pragma unroll
                     for (int k = 0; k < kC / 16; ++k) {
-                        mma_ss_lh<true>(tb + C::colS, a_lo + k * (2048 >> 4), desc_hi(dV), lPK + k * (1024 >> 4),
+                        mma_ss_w<true>(lead, tb + C::colS, a_lo + k * (2048 >> 4), desc_hi(dV), lPK + k * (1024 >> 4),
                                         desc_hi(dPhiMN), i5);
-                        mma_ss_lh<true>(tb + C::colZ0, lPK + k * (1024 >> 4), desc_hi(dPhiMN), lOnes + (k & 1) * 2,
+                        mma_ss_w<true>(lead, tb + C::colZ0, lPK + k * (1024 >> 4), desc_hi(dPhiMN), lOnes + (k & 1) * 2,
                                         desc_hi(dOnes), iZ0);
-                        mma_ss_lh<true>(tb + C::colZ1, lPK + ((4 * C::kPhiBlk + k * 1024) >> 4), desc_hi(dPhiMN),
+                        mma_ss_w<true>(lead, tb + C::colZ1, lPK + ((4 * C::kPhiBlk + k * 1024) >> 4), desc_hi(dPhiMN),
                                         lOnes + (k & 1) * 2, desc_hi(dOnes), iZ1);
                     }
                 }
-                mma_commit(g2_bar(c));
-                mma_commit(&bars[kEmpty0 + s]);
+                mma_commit_w(lead, g2_bar(c));
+                mma_commit_w(lead, &bars[kEmpty0 + s]);
                 // every state update without a read-out in between is done (state-only pass: all of
                 // them; main pass: the pre-chunks)
-                if (c + 1 == (STATE_ONLY ? nch : npre)) mma_commit(&bars[kDone]);
-                TRACE(1, c, 2);
+                if (c + 1 == (STATE_ONLY ? nch : npre)) mma_commit_w(lead, &bars[kDone]);
+                if (lane == 0) TRACE(1, c, 2);
             }
         }
     } else if (warp == kWarpMmaY) {
         // ===================================================================== MMA issuer, output chain
-        if (lane == 0 && !STATE_ONLY) {
+        const uint32_t lead = elect_one();
+        if (!STATE_ONLY) {
             constexpr uint64_t dQK = make_smem_desc_base(16, 256, kSwizzle32B);           // K-major [128][16]
             constexpr uint64_t dPhiK = make_smem_desc_base(16, 512, kSwizzle64B);         // K-major, 64-byte rows
             constexpr uint64_t dV = make_smem_desc_base(kC * 128, 1024, kSwizzle128B);    // MN-major [128 tok][DV]
@@ -568,18 +571,18 @@ __global__ void __launch_bounds__(kThreads, 1)
             auto issue_scores = [&](int c) -> bool {
                 const int s = (c + npre) % NS;
                 if (!mbar_wait(&bars[kFull0 + s], ((c + npre) / NS) & 1, abort_flag)) return false;
-                TRACE(0, c, 0);
+                if (lane == 0) TRACE(0, c, 0);
                 tc_fence_after();
                 const uint32_t aSt = smem_u32(smem + C::offStage + s * C::kStageBytes);
-                mma_ss_lh<false>(tb + C::colT + (C::kTDouble ? (c & 1) * 128 : 0), lQK + (aSt >> 4), desc_hi(dQK),
+                mma_ss_w<false>(lead, tb + C::colT + (C::kTDouble ? (c & 1) * 128 : 0), lQK + (aSt >> 4), desc_hi(dQK),
                                  lQK + ((aSt + C::kQKBytes) >> 4), desc_hi(dQK), i1);
-                mma_commit(&bars[kG1 + t_idx(c)]);
+                mma_commit_w(lead, &bars[kG1 + t_idx(c)]);
                 return true;
             };
             // pre-chunks: nothing to issue, but the stage is released by two arrivals
             for (int g = 0; g < npre && ok; ++g) {
                 ok = mbar_wait(&bars[kFull0 + g % NS], (g / NS) & 1, abort_flag);
-                if (ok) mbar_arrive(&bars[kEmpty0 + g % NS]);
+                if (ok && lead) mbar_arrive(&bars[kEmpty0 + g % NS]);
             }
             if (nch > 0 && ok) ok = issue_scores(0);
             for (int c = 0; c < nch && ok; ++c) {
@@ -589,12 +592,12 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const uint32_t colTc = C::colT + (C::kTDouble ? (c & 1) * 128 : 0);
                 // with two score buffers the next chunk's scores are issued ahead of this chunk's
                 // steps (4) and (3), so its polynomial overlaps them
-                TRACE(2, c, 3);
+                if (lane == 0) TRACE(2, c, 3);
                 if (C::kTDouble && c + 1 < nch) {
                     ok = issue_scores(c + 1);
                     if (!ok) break;
                 }
-                TRACE(0, c, 1);
+                if (lane == 0) TRACE(0, c, 1);
                 // step (4) of chunk c needs phi(Q) of chunk c (feature group), the state copy after chunk
                 // c-1 (state group) and the Y accumulator read out for chunk c-1 (output group, which
                 // arrives once before its first chunk): one barrier, three groups of 128 arrivals
@@ -605,7 +608,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     ok = mbar_wait(&bars[kSC + (c & 1)], (c >> 1) & 1, abort_flag);
                     if (!ok) break;
                 }
-                TRACE(0, c, 3);
+                if (lane == 0) TRACE(0, c, 3);
                 tc_fence_after();
                 const uint32_t lSc = (PQT && (c & 1)) ? lPQ : lSc0;      // second copy tile: the phi(Q) tile's place
 #pragma unroll
@@ -614,18 +617,18 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const uint32_t offb = ((k >> 1) * C::kScBlk + (k & 1) * 32) >> 4;
                     if (PQT) {
                         const uint32_t a = tb + (k < 8 ? colTc + 64 + k * 8 : C::colPQhi + (k - 8) * 8);
-                        if (k == 0) mma_ts_lh<false>(tb + C::colY, a, lSc + offb, desc_hi(dPhiK), i4);
-                        else mma_ts_lh<true>(tb + C::colY, a, lSc + offb, desc_hi(dPhiK), i4);
+                        if (k == 0) mma_ts_w<false>(lead, tb + C::colY, a, lSc + offb, desc_hi(dPhiK), i4);
+                        else mma_ts_w<true>(lead, tb + C::colY, a, lSc + offb, desc_hi(dPhiK), i4);
                     } else {
-                        if (k == 0) mma_ss_lh<false>(tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
-                        else mma_ss_lh<true>(tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
+                        if (k == 0) mma_ss_w<false>(lead, tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
+                        else mma_ss_w<true>(lead, tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
                     }
                 }
-                mma_commit(g4_bar(c));
-                TRACE(0, c, 4);
+                mma_commit_w(lead, g4_bar(c));
+                if (lane == 0) TRACE(0, c, 4);
                 ok = mbar_wait(&bars[kP + t_idx(c)], t_parity(c), abort_flag);
                 if (!ok) break;
-                TRACE(0, c, 5);
+                if (lane == 0) TRACE(0, c, 5);
                 tc_fence_after();
                 {
                     // there the second 64-column block of the B operand is the ones block (leading byte offset)
@@ -633,12 +636,12 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const uint32_t b_lo = desc_lo(dVo) + (aVt >> 4), b_hi = desc_hi(dVo);
 #pragma unroll
                     for (int k = 0; k < kC / 16; ++k)
-                        mma_ts_lh<true>(tb + C::colY, tb + colTc + k * 8, b_lo + k * (2048 >> 4), b_hi, i3);
+                        mma_ts_w<true>(lead, tb + C::colY, tb + colTc + k * 8, b_lo + k * (2048 >> 4), b_hi, i3);
                 }
-                TRACE(2, c, 2);
-                mma_commit(&bars[kG3]);
-                mma_commit(&bars[kEmpty0 + s]);
-                TRACE(0, c, 6);
+                if (lane == 0) TRACE(2, c, 2);
+                mma_commit_w(lead, &bars[kG3]);
+                mma_commit_w(lead, &bars[kEmpty0 + s]);
+                if (lane == 0) TRACE(0, c, 6);
                 // single score buffer: P of this chunk has to be consumed before the next scores land
                 if (!C::kTDouble && c + 1 < nch) ok = issue_scores(c + 1);
             }
@@ -979,6 +982,13 @@ __global__ void __launch_bounds__(kThreads, 1)
         // One thread per query row: polynomial of the scores, causal mask, row sum; the
         // bf16 weights overwrite the scores in place (columns [0, 64) of the same lanes).
         const int q4 = warp;                            // lane quarter == 32-row block of the chunk
+        // packed variant: causal mask of the batch that holds the diagonal, one word per pair of columns
+        // (columns 2i and 2i+1 against this row, i.e. this lane), so that masking is one logic instruction per pair
+        uint32_t dm[PKW ? 16 : 1];
+        if constexpr (PKW) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) dm[i] = (2 * i + 1 <= lane) ? 0xFFFFFFFFu : ((2 * i <= lane) ? 0x0000FFFFu : 0u);
+        }
         for (int c = 0; c < nch && ok; ++c) {
             ok = mbar_wait(&bars[kG1 + t_idx(c)], t_parity(c), abort_flag);
             if (!ok) break;
@@ -999,13 +1009,12 @@ __global__ void __launch_bounds__(kThreads, 1)
                         // would be rounded to bf16 anyway).  The row sum is the tensor cores' work (see step (3)).
                         const __nv_bfloat162 c1 = __float2bfloat162_rn(0.25f), c2 = __float2bfloat162_rn(0.03125f),
                                              one = __float2bfloat162_rn(1.0f);
-                        const int vis = (b < q4) ? 64 : lane + 1;      // columns of this batch the row may see
+                        const uint32_t full = (b < q4) ? 0xFFFFFFFFu : 0u;      // a batch left of the diagonal is seen whole
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             const __nv_bfloat162 s2 = __floats2bfloat162_rn(__uint_as_float(sc[2 * i]), __uint_as_float(sc[2 * i + 1]));
                             const __nv_bfloat162 w2 = __hfma2(s2, __hfma2(s2, c2, c1), one);
-                            const uint32_t w = *reinterpret_cast<const uint32_t*>(&w2);
-                            pk[i] = (2 * i + 1 < vis) ? w : ((2 * i < vis) ? (w & 0xFFFFu) : 0u);
+                            pk[i] = *reinterpret_cast<const uint32_t*>(&w2) & (dm[i] | full);
                         }
                     } else {
                         // fp32 polynomial on pairs of scores (two-wide fp32 multiply-add): t = s/32 + 1/4, w = s t + 1

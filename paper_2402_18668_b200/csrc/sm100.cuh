@@ -298,6 +298,51 @@ __device__ __forceinline__ void mma_ts_lh(uint32_t d_tmem, uint32_t a_tmem, uint
         ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0)
         : "memory");
 }
+// The same for a converged warp.  A lone thread behind a branch keeps descriptors and addresses in ordinary
+// registers and pays for moving each into the uniform registers the instruction takes: measured, 45 cycles per
+// tcgen05.mma whatever its shape (82 in a rolled loop), which is more than an MMA with N <= 80 runs.  When all 32
+// lanes execute the call and only the instruction itself is predicated on the elected lane, the operands stay in
+// uniform registers: 15 cycles per issue, so an N = 80 MMA takes its 40 cycles of tensor time.
+// `lead` is non-zero in exactly one lane (elect_one(), taken once per warp so that the commits come from the
+// thread that issued the MMAs).
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.b32 %0, 1, 0, p;\n\t}" : "=r"(r));
+    return r;
+}
+template <bool ACC>
+__device__ __forceinline__ void mma_ss_w(uint32_t lead, uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                         uint32_t b_hi, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p, e;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "setp.ne.b32 e, %7, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0), "r"(lead)
+        : "memory");
+}
+template <bool ACC>
+__device__ __forceinline__ void mma_ts_w(uint32_t lead, uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
+                                         uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p, e;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "setp.ne.b32 e, %6, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0), "r"(lead)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit_w(uint32_t lead, uint64_t* bar) {
+    asm volatile(
+        "{\n\t.reg .pred e;\n\t"
+        "setp.ne.b32 e, %1, 0;\n\t"
+        "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar)), "r"(lead)
+        : "memory");
+}
 __host__ __device__ constexpr uint32_t desc_hi(uint64_t base) { return static_cast<uint32_t>(base >> 32); }
 __host__ __device__ constexpr uint32_t desc_lo(uint64_t base) { return static_cast<uint32_t>(base & 0xffffffffu); }
 

@@ -170,7 +170,9 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
         }
     } else if (warp == kWarpMma) {
-        if (lane == 0) {
+        {
+            // the whole warp runs this block and one elected lane issues (see mma_ss_w)
+            const uint32_t lead = elect_one();
             constexpr uint64_t dK = make_smem_desc_base(16, 1024, kSwizzle128B);   // K-major rows / MN-major block
             constexpr uint32_t iS = make_idesc_bf16(kQT, kKeys, 0, 0);
             constexpr uint32_t iO = make_idesc_bf16(kQT, kHD, 0, 1);
@@ -178,12 +180,12 @@ __global__ void __launch_bounds__(kThreads, 1)
                 auto issue_pv = [&](int n) {
                     const uint32_t tbuf = tb + (n & 1) * kBufCols;
                     const uint32_t lV = desc_lo(dK) + (smem_u32(smem + (n % kStages) * kStageBytes + kQBytes + kKVBytes) >> 4);
-                    mma_ts_lh<false>(tbuf + colO, tbuf + colS, lV, desc_hi(dK), iO);
+                    mma_ts_w<false>(lead, tbuf + colO, tbuf + colS, lV, desc_hi(dK), iO);
 #pragma unroll
                     for (int k = 1; k < kKeys / 16; ++k)
-                        mma_ts_lh<true>(tbuf + colO, tbuf + colS + k * 8, lV + k * (2048 >> 4), desc_hi(dK), iO);
-                    mma_commit(&bars[bO + (n & 1)]);
-                    mma_commit(&bars[bEmpty + n % kStages]);     // K, V (and Q) of this stage are dead
+                        mma_ts_w<true>(lead, tbuf + colO, tbuf + colS + k * 8, lV + k * (2048 >> 4), desc_hi(dK), iO);
+                    mma_commit_w(lead, &bars[bO + (n & 1)]);
+                    mma_commit_w(lead, &bars[bEmpty + n % kStages]);     // K, V (and Q) of this stage are dead
                 };
                 for (int n = 0; n < ntiles && ok; ++n) {
                     const int s = n % kStages, b = n & 1;
@@ -195,11 +197,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const uint32_t tbuf = tb + b * kBufCols;
                     const uint32_t lQ = desc_lo(dK) + (smem_u32(smem + s * kStageBytes) >> 4);
                     const uint32_t lK = lQ + (kQBytes >> 4);
-                    mma_ss_lh<false>(tbuf + colS, lQ, desc_hi(dK), lK, desc_hi(dK), iS);
+                    mma_ss_w<false>(lead, tbuf + colS, lQ, desc_hi(dK), lK, desc_hi(dK), iS);
 #pragma unroll
                     for (int k = 1; k < kHD / 16; ++k)
-                        mma_ss_lh<true>(tbuf + colS, lQ + k * 2, desc_hi(dK), lK + k * 2, desc_hi(dK), iS);
-                    mma_commit(&bars[bS + b]);
+                        mma_ss_w<true>(lead, tbuf + colS, lQ + k * 2, desc_hi(dK), lK + k * 2, desc_hi(dK), iS);
+                    mma_commit_w(lead, &bars[bS + b]);
                     if (n >= 1) {
                         ok = mbar_wait(&bars[bP + (b ^ 1)], ((n - 1) >> 1) & 1, abort_flag);
                         if (!ok) break;
@@ -228,19 +230,19 @@ __global__ void __launch_bounds__(kThreads, 1)
                     // head's rows, so those products are left out
                     const bool head_start = tile_of(n) % p.tiles_per_head == 0;
                     if (!head_start) {
-                        mma_ts_lh<false>(tbuf + colO, tbuf + colS, lV0, desc_hi(dK), iO);
+                        mma_ts_w<false>(lead, tbuf + colO, tbuf + colS, lV0, desc_hi(dK), iO);
 #pragma unroll
                         for (int k = 1; k < 8; ++k)
-                            mma_ts_lh<true>(tbuf + colO, tbuf + colS + k * 8, lV0 + k * (2048 >> 4), desc_hi(dK), iO);
-                        mma_ts_lh<true>(tbuf + colO, tbuf + colS + 64, lV1, desc_hi(dK), iO);
+                            mma_ts_w<true>(lead, tbuf + colO, tbuf + colS + k * 8, lV0 + k * (2048 >> 4), desc_hi(dK), iO);
+                        mma_ts_w<true>(lead, tbuf + colO, tbuf + colS + 64, lV1, desc_hi(dK), iO);
                     } else {
-                        mma_ts_lh<false>(tbuf + colO, tbuf + colS + 64, lV1, desc_hi(dK), iO);
+                        mma_ts_w<false>(lead, tbuf + colO, tbuf + colS + 64, lV1, desc_hi(dK), iO);
                     }
 #pragma unroll
                     for (int k = 1; k < 8; ++k)
-                        mma_ts_lh<true>(tbuf + colO, tbuf + colS + 64 + k * 8, lV1 + k * (2048 >> 4), desc_hi(dK), iO);
-                    mma_commit(&bars[bO + (n & 1)]);
-                    mma_commit(&bars[bEmpty + n % kStages]);     // the rows before tile n are dead now
+                        mma_ts_w<true>(lead, tbuf + colO, tbuf + colS + 64 + k * 8, lV1 + k * (2048 >> 4), desc_hi(dK), iO);
+                    mma_commit_w(lead, &bars[bO + (n & 1)]);
+                    mma_commit_w(lead, &bars[bEmpty + n % kStages]);     // the rows before tile n are dead now
                 };
                 if (ntiles > 0) ok = mbar_wait(&bars[bFull + 0], 0, abort_flag);       // rows before the first tile
                 for (int n = 0; n < ntiles && ok; ++n) {
@@ -251,14 +253,14 @@ __global__ void __launch_bounds__(kThreads, 1)
                     tc_fence_after();
                     const uint32_t tbuf = tb + b * kBufCols;
                     const uint32_t lQ = slot_lo(m, 0), lK0 = slot_lo(n, kQBytes), lK1 = slot_lo(m, kQBytes);
-                    mma_ss_lh<false>(tbuf + colS, lQ, desc_hi(dK), lK0, desc_hi(dK), iS128);
-                    mma_ss_lh<false>(tbuf + colS + 128, lQ, desc_hi(dK), lK1, desc_hi(dK), iS128);
+                    mma_ss_w<false>(lead, tbuf + colS, lQ, desc_hi(dK), lK0, desc_hi(dK), iS128);
+                    mma_ss_w<false>(lead, tbuf + colS + 128, lQ, desc_hi(dK), lK1, desc_hi(dK), iS128);
 #pragma unroll
                     for (int k = 1; k < kHD / 16; ++k) {
-                        mma_ss_lh<true>(tbuf + colS, lQ + k * 2, desc_hi(dK), lK0 + k * 2, desc_hi(dK), iS128);
-                        mma_ss_lh<true>(tbuf + colS + 128, lQ + k * 2, desc_hi(dK), lK1 + k * 2, desc_hi(dK), iS128);
+                        mma_ss_w<true>(lead, tbuf + colS, lQ + k * 2, desc_hi(dK), lK0 + k * 2, desc_hi(dK), iS128);
+                        mma_ss_w<true>(lead, tbuf + colS + 128, lQ + k * 2, desc_hi(dK), lK1 + k * 2, desc_hi(dK), iS128);
                     }
-                    mma_commit(&bars[bS + b]);
+                    mma_commit_w(lead, &bars[bS + b]);
                     if (n >= 1) {
                         ok = mbar_wait(&bars[bP + (b ^ 1)], ((n - 1) >> 1) & 1, abort_flag);
                         if (!ok) break;
