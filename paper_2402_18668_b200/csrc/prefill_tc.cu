@@ -60,7 +60,9 @@ __host__ __device__ constexpr size_t seg_state_floats(int dv) { return (size_t)k
 
 template <int DV>
 struct Cfg {
-    static constexpr int kStages = (DV == 64) ? 3 : 2;
+    // d_v 64: four stages (a tile's load takes about 2500 cycles from issue to arrival, more than a chunk's period;
+    // with three the next chunk's scores waited for their tile: measured 5-8 % on the 360M shapes)
+    static constexpr int kStages = (DV == 64) ? 4 : 2;
     static constexpr int kNY = DV + 16;                         // Y columns: d_v numerators + denominator block
     static constexpr int kSLanes = (DV == 64) ? 65 : 128;       // live lanes of S^T (d_v 64: lane 64 carries z)
     static constexpr uint32_t kQKBytes = kC * 32;               // one q or k tile (16 bf16 per token)
@@ -70,9 +72,11 @@ struct Cfg {
     static constexpr uint32_t kPhiBytes = kFBlk * kPhiBlk;      // 40 KB
     static constexpr uint32_t kScBlk = kNY * 64;
     static constexpr uint32_t kScBytes = kFBlk * kScBlk;
-    // d_v 64: a [128 tokens][64] bf16 block whose column 0 is 1.0 (second M-block of V^T);
+    // d_v 64: a [16 tokens][64] bf16 block whose column 0 is 1.0: the second 64-wide block of V^T (and of V) for one
+    // K-step of 16 tokens.  Every K-step's block would hold the same, so all of them read this one: the descriptor
+    // of K-step k starts 2 KB further and its block offset is 2 KB shorter.
     // d_v 128: a block of bf16 ones (B operand of the z step)
-    static constexpr uint32_t kOnesBytes = (DV == 64) ? kC * 128 : 2048;
+    static constexpr uint32_t kOnesBytes = 2048;
     static constexpr uint32_t kOutBytes = kC * 128;             // staging of 64 output columns
     static constexpr uint32_t offStage = 0;
     static constexpr uint32_t offOnes = kStages * kStageBytes;  // after the stages: LBO of V^T stays positive
@@ -99,11 +103,16 @@ struct Cfg {
     static constexpr bool kPQinT = (DV == 64);
     static constexpr uint32_t colPQhi = colS + kF;
     static_assert((DV == 64 ? colS + kF + 16 : colZ1 + 16) <= 512, "TMEM budget");
+    // d_v 128, plain chunk loop: the 48 columns behind the z tiles hold features 0..95 of phi(Q) (A operand of the
+    // first six K-steps of step (4)); only features 96..159 stay in shared memory, two blocks at the start of the
+    // phi(Q) tile's place, and the 16 KB behind them are a second output staging tile
+    static constexpr uint32_t colPQlo = colZ1 + 16;
+    static constexpr uint32_t offOut2 = offPQ + 2 * kPhiBlk;
     static_assert(kScBlk % 1024 == 0 && kStageBytes % 1024 == 0 && offPK % 1024 == 0, "tiles stay 1024-byte aligned");
 };
 
 enum Bar {
-    kFull0 = 0, kEmpty0 = 3, kG1 = 6, kG1b, kP, kPb, kG2, kG2b, kG4, kG4b, kG3, kR4, kPK, kPKb, kSR, kDone, kTR, kTRb, kSC, kSCb,
+    kFull0 = 0, kEmpty0 = 4, kG1 = 8, kG1b, kP, kPb, kG2, kG2b, kG4, kG4b, kG3, kR4, kPK, kPKb, kSR, kDone, kTR, kTRb, kSC, kSCb,
     kNumBars
 };
 
@@ -307,6 +316,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     // packed bf16 polynomial and the row sums by the tensor cores: the same kernel (measured: -6 % there, +14 % in
     // the recompute mode's kernel)
     constexpr bool PKW = PQT;
+    // d_v 128: most of phi(Q) in tensor memory and two output staging tiles (see Cfg::colPQlo)
+    constexpr bool PQS = DV == 128 && MODE == kModeMain;
+    static_assert(!PQS || C::colPQlo + 48 <= 512, "TMEM budget");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offMisc);
@@ -529,9 +541,9 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const uint64_t dV1 = make_smem_desc_base(aOnes - aVt, 1024, kSwizzle128B);
                     const uint32_t a_lo = desc_lo(dV1) + (aVt >> 4), a_hi = desc_hi(dV1);
 #pragma unroll
-                    for (int k = 0; k < kC / 16; ++k)
-                        mma_ss_w<true>(lead, tb + C::colS, a_lo + k * (2048 >> 4), a_hi, lPK + k * (1024 >> 4),
-                                        desc_hi(dPhiMN), i5);
+                    for (int k = 0; k < kC / 16; ++k)         // (start + 2 KB per K-step, block offset - 2 KB: see kOnesBytes)
+                        mma_ss_w<true>(lead, tb + C::colS, a_lo + k * ((2048u >> 4) - ((2048u >> 4) << 16)), a_hi,
+                                       lPK + k * (1024 >> 4), desc_hi(dPhiMN), i5);
                 } else {
                     const uint32_t a_lo = lV + (aVt >> 4);
 #pragma unroll
@@ -619,6 +631,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                         const uint32_t a = tb + (k < 8 ? colTc + 64 + k * 8 : C::colPQhi + (k - 8) * 8);
                         if (k == 0) mma_ts_w<false>(lead, tb + C::colY, a, lSc + offb, desc_hi(dPhiK), i4);
                         else mma_ts_w<true>(lead, tb + C::colY, a, lSc + offb, desc_hi(dPhiK), i4);
+                    } else if (PQS) {
+                        const uint32_t offs = (((k >> 1) - 3) * C::kPhiBlk + (k & 1) * 32) >> 4;      // blocks 3, 4 at the tile's start
+                        if (k == 0) mma_ts_w<false>(lead, tb + C::colY, tb + C::colPQlo, lSc + offb, desc_hi(dPhiK), i4);
+                        else if (k < 6) mma_ts_w<true>(lead, tb + C::colY, tb + C::colPQlo + k * 8, lSc + offb, desc_hi(dPhiK), i4);
+                        else mma_ss_w<true>(lead, tb + C::colY, lPQ + offs, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
                     } else {
                         if (k == 0) mma_ss_w<false>(lead, tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
                         else mma_ss_w<true>(lead, tb + C::colY, lPQ + off, desc_hi(dPhiK), lSc + offb, desc_hi(dPhiK), i4);
@@ -636,7 +653,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const uint32_t b_lo = desc_lo(dVo) + (aVt >> 4), b_hi = desc_hi(dVo);
 #pragma unroll
                     for (int k = 0; k < kC / 16; ++k)
-                        mma_ts_w<true>(lead, tb + C::colY, tb + colTc + k * 8, b_lo + k * (2048 >> 4), b_hi, i3);
+                        mma_ts_w<true>(lead, tb + C::colY, tb + colTc + k * 8,
+                                       b_lo + k * (PKW ? (2048u >> 4) - ((2048u >> 4) << 16) : (2048u >> 4)), b_hi, i3);
                 }
                 if (lane == 0) TRACE(2, c, 2);
                 mma_commit_w(lead, &bars[kG3]);
@@ -665,6 +683,45 @@ __global__ void __launch_bounds__(kThreads, 1)
                 tmem_wait_ld();
                 const float den_in = PKW ? 0.f : s_den[(c & 3) * kC + t];      // packed variant: already in the column
                 const float inv = p.numerator_only ? 1.0f : 1.0f / (den_in + __uint_as_float(dcol) + kEps);
+                if constexpr (PQS) {
+                    // All of Y leaves tensor memory before any staging (step (4) of the next chunk waits for that), 32
+                    // columns at a time, scaled and packed as they arrive: 128 fp32 columns do not fit a thread's registers.
+                    // Then one staging tile per 64 columns: a bulk store reads its tile at about 15 bytes per cycle, so
+                    // with one tile filled and drained twice per chunk the tile alone would take most of a chunk's time.
+                    uint32_t pkd[DV / 2];
+#pragma unroll
+                    for (int qd = 0; qd < DV / 32; ++qd) {
+                        uint32_t y[32];
+                        tmem_ld32(tmem_addr(tb, lane_base, C::colY + qd * 32), y);
+                        tmem_wait_ld();
+                        if (qd == DV / 32 - 1) {
+                            tc_fence_before();
+                            mbar_arrive(&bars[kR4]);
+                            if (t == 0) TRACE(5, c, 1);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            pkd[qd * 16 + i] = pack_bf16(__uint_as_float(y[2 * i]) * inv, __uint_as_float(y[2 * i + 1]) * inv);
+                    }
+#pragma unroll
+                    for (int h = 0; h < DV / 64; ++h) {
+                        uint8_t* tile = h == 0 ? sOut : smem + C::offOut2;
+                        uint8_t* trow = tile + (t >> 3) * 1024 + (t & 7) * 128;
+                        // the tile is free once the store before the latest one has read it
+                        if (t == 0) tma_store_wait_read<1>();
+                        group_sync(1);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            *reinterpret_cast<uint4*>(trow + ((j ^ sw) << 4)) =
+                                make_uint4(pkd[h * 32 + 4 * j], pkd[h * 32 + 4 * j + 1], pkd[h * 32 + 4 * j + 2], pkd[h * 32 + 4 * j + 3]);
+                        fence_proxy_async_smem();
+                        group_sync(1);
+                        if (t == 0) {
+                            tma_store_3d(&tm_o, tile, h * 64, tok_begin + c * kC, head);   // rows past the end are clipped
+                            tma_store_commit();
+                        }
+                    }
+                } else {
 #pragma unroll 1
                 for (int h = 0; h < DV / 64; ++h) {
                     uint32_t y0[32], y1[32];
@@ -704,6 +761,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                         tma_store_3d(&tm_o, sOut, h * 64, tok_begin + c * kC, head);
                         tma_store_commit();
                     }
+                }
                 }
                 if (t == 0) TRACE(5, c, 2);
             }
@@ -968,6 +1026,28 @@ __global__ void __launch_bounds__(kThreads, 1)
                     tmem_st16(tmem_addr(tb, lane_base, C::colPQhi), r);
                     tmem_wait_st();
                     tc_fence_before();
+                } else if constexpr (PQS) {
+                    uint4 f[20];
+                    compute_phi_row(qlo, qhi, true, f);
+                    tc_fence_after();
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) {              // pieces 0..11: features 0..95, four columns a piece
+                        const uint32_t r[16] = {f[4 * j].x, f[4 * j].y, f[4 * j].z, f[4 * j].w,
+                                                f[4 * j + 1].x, f[4 * j + 1].y, f[4 * j + 1].z, f[4 * j + 1].w,
+                                                f[4 * j + 2].x, f[4 * j + 2].y, f[4 * j + 2].z, f[4 * j + 2].w,
+                                                f[4 * j + 3].x, f[4 * j + 3].y, f[4 * j + 3].z, f[4 * j + 3].w};
+                        tmem_st16(tmem_addr(tb, lane_base, C::colPQlo + j * 16), r);
+                    }
+                    {                                          // pieces 12..19: feature blocks 3 and 4 -> blocks 0 and 1 of the tile
+                        uint8_t* row = sPQ + (t >> 3) * 512 + (t & 7) * 64;
+                        const uint32_t sw = (t >> 1) & 3;
+#pragma unroll
+                        for (int j = 12; j < 20; ++j)
+                            *reinterpret_cast<uint4*>(row + ((j >> 2) - 3) * (kC * 64) + (((j & 3) ^ sw) << 4)) = f[j];
+                    }
+                    tmem_wait_st();
+                    tc_fence_before();
+                    fence_proxy_async_smem();
                 } else {
                     if constexpr (DV == 64) store_phi_row(fq, sPQ, t);
                     else write_phi_row(qlo, qhi, sPQ, t, true);
