@@ -112,7 +112,7 @@ struct Cfg {
 };
 
 enum Bar {
-    kFull0 = 0, kEmpty0 = 4, kG1 = 8, kG1b, kP, kPb, kG2, kG2b, kG4, kG4b, kG3, kR4, kPK, kPKb, kSR, kDone, kTR, kTRb, kSC, kSCb,
+    kFull0 = 0, kEmpty0 = 4, kG1 = 8, kG1b, kP, kPb, kG2, kG2b, kG4, kG4b, kG3, kR4, kPK, kPKb, kSR, kDone, kTR, kTRb, kSC, kSCb, kFin,
     kNumBars
 };
 
@@ -430,6 +430,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         mbar_init(&bars[kG3], 1);
         mbar_init(&bars[kP], 128); mbar_init(&bars[kR4], PQT ? 256 : 384); mbar_init(&bars[kPK], 128); mbar_init(&bars[kPKb], 128); mbar_init(&bars[kDone], 1);
         mbar_init(&bars[kSR], 128);
+        mbar_init(&bars[kFin], 1);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v); prefetch_tensormap(&tm_o);
@@ -561,6 +562,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 // every state update without a read-out in between is done (state-only pass: all of
                 // them; main pass: the pre-chunks)
                 if (c + 1 == (STATE_ONLY ? nch : npre)) mma_commit_w(lead, &bars[kDone]);
+                if (c + 1 == ntot) mma_commit_w(lead, &bars[kFin]);      // the state is final
                 if (lane == 0) TRACE(1, c, 2);
             }
         }
@@ -918,46 +920,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (ok && nch > 0) ok = mbar_wait(g2_bar(ntot - 1), g2_parity(ntot - 1), abort_flag);
         }
 
-        // ---- final state
         if (t == 0) TRACE(5, 3, 7);   // chunk loop done
-        tc_fence_after();
-        const bool write_ws = STATE_ONLY;
-        const bool write_abi = !STATE_ONLY && p.kv_abi != nullptr && head_end;
-        if (ok && (write_ws || write_abi)) {
-            float* wseg = p.ws + (size_t)(ws_out < 0 ? 0 : ws_out) * seg_stride;
-            float* kvo = write_abi ? p.kv_abi + (size_t)head * abi_nrows * dv : nullptr;
-            float* zo = write_abi ? p.z_abi + (size_t)head * abi_nrows : nullptr;
-            auto put = [&](int f, float v, bool zrow, int col) {
-                if (write_ws) {
-                    if (zrow) wseg[(size_t)kF * DV + f] = v;
-                    else wseg[(size_t)f * DV + col] = v;
-                    return;
-                }
-                const short2 ar = s_abi[f];
-                if (ar.x < 0) return;
-                if (ar.y >= 0) v *= kRsqrt2;
-                if (zrow) { zo[ar.x] = v; if (ar.y >= 0) zo[ar.y] = v; }
-                else if (col < dv) { kvo[(size_t)ar.x * dv + col] = v; if (ar.y >= 0) kvo[(size_t)ar.y * dv + col] = v; }
-            };
-#pragma unroll 1
-            for (int b = 0; b < kF / 16; ++b) {
-                uint32_t r[16];
-                tmem_ld16(tmem_addr(tb, lane_base, C::colS + b * 16), r);
-                tmem_wait_ld();
-                if (srow >= 0) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) put(b * 16 + i, __uint_as_float(r[i]), is_z, srow);
-                }
-            }
-            if (DV == 128) {
-                uint32_t z0, z1;
-                tmem_ld1(tmem_addr(tb, lane_base, C::colZ0), z0);
-                tmem_ld1(tmem_addr(tb, lane_base, C::colZ1), z1);
-                tmem_wait_ld();
-                put(t, __uint_as_float(z0), true, 0);
-                if (z1f >= 0) put(z1f, __uint_as_float(z1), true, 0);
-            }
-        }
     } else if (warp >= 4) {
         // ===================================================================== feature group
         // One thread per token of the chunk: expands its k row (and q row) into feature rows.
@@ -1142,6 +1105,62 @@ __global__ void __launch_bounds__(kThreads, 1)
             tc_fence_before();
             mbar_arrive(&bars[kP + t_idx(c)]);
             if (tid == 96) TRACE(2, c, 1);
+        }
+    }
+
+    // ---- final state: into the workspace slot (state pass) or, folded back into the caller's layout, into the
+    // caller's state (a piece that ends its head).  Every thread of the first sixteen warps owns a lane of S^T (its
+    // warp's lane quarter), so the four role groups share the ten 16-column blocks: the write is 140 KB per head at
+    // d_v 128, a fifth of a chunk's time when one group does it alone.
+    if (warp < 16) {
+        const bool write_ws = STATE_ONLY;
+        const bool write_abi = !STATE_ONLY && p.kv_abi != nullptr && head_end;
+        if (write_ws || write_abi) {
+            const int part = warp >> 2;                                  // 0 row, 1 feature, 2 state, 3 output group
+            const int t = ((warp & 3) << 5) + lane;
+            const int srow = (t < C::kSLanes) ? t : -1;
+            const bool is_z = (DV == 64) && t == 64;
+            const int z1f = (DV == 128 && (t & 31) < 16 && (t >> 5) < 2) ? 128 + (t >> 5) * 16 + (t & 15) : -1;
+            const int dv = p.dv;
+            // without chunks there is no last MMA to wait for, and only the state group knows the state is initialised
+            const bool shared = ntot > 0;
+            if (ok && shared) ok = mbar_wait(&bars[kFin], 0, abort_flag);
+            tc_fence_after();
+            if (ok && (shared || part == 2)) {
+                float* wseg = p.ws + (size_t)(ws_out < 0 ? 0 : ws_out) * seg_state_floats(DV);
+                float* kvo = write_abi ? p.kv_abi + (size_t)head * abi_nrows * dv : nullptr;
+                float* zo = write_abi ? p.z_abi + (size_t)head * abi_nrows : nullptr;
+                auto put = [&](int f, float v, bool zrow, int col) {
+                    if (write_ws) {
+                        if (zrow) wseg[(size_t)kF * DV + f] = v;
+                        else wseg[(size_t)f * DV + col] = v;
+                        return;
+                    }
+                    const short2 ar = s_abi[f];
+                    if (ar.x < 0) return;
+                    if (ar.y >= 0) v *= kRsqrt2;
+                    if (zrow) { zo[ar.x] = v; if (ar.y >= 0) zo[ar.y] = v; }
+                    else if (col < dv) { kvo[(size_t)ar.x * dv + col] = v; if (ar.y >= 0) kvo[(size_t)ar.y * dv + col] = v; }
+                };
+#pragma unroll 1
+                for (int b = shared ? part : 0; b < kF / 16; b += shared ? 4 : 1) {
+                    uint32_t r[16];
+                    tmem_ld16(tmem_addr(tb, lane_base, C::colS + b * 16), r);
+                    tmem_wait_ld();
+                    if (srow >= 0) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) put(b * 16 + i, __uint_as_float(r[i]), is_z, srow);
+                    }
+                }
+                if (DV == 128 && part == 2) {
+                    uint32_t z0, z1;
+                    tmem_ld1(tmem_addr(tb, lane_base, C::colZ0), z0);
+                    tmem_ld1(tmem_addr(tb, lane_base, C::colZ1), z1);
+                    tmem_wait_ld();
+                    put(t, __uint_as_float(z0), true, 0);
+                    if (z1f >= 0) put(z1f, __uint_as_float(z1), true, 0);
+                }
+            }
         }
     }
 
