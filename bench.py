@@ -44,12 +44,12 @@ sys.path.insert(0, str(ROOT))
 L2_BYTES = 126 * 1024 * 1024
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
-# summarised under profiles/.  cfg 2 was captured at full size; the decode and sliding-window
+# summarised under profiles/.  cfg 2 and cfg 3 were captured at full size; the decode and sliding-window
 # captures used half-size cases (sizing rule for profiler runs) and are scaled by the units
 # processed.  Written bytes still resident in L2 when a launch ends are not in these figures.
 NCU_TRAFFIC = {
-    "cfg2_360m_prefill": 25.23e6,                 # profiles/prefill_tc_kernel_dv64_cfg2.md (output stays in L2)
-    "cfg3_1p3b_prefill": 1.6 * (104.94e6 + 43.89e6),  # profiles/prefill_tc_kernel_dv128.md, 80 -> 128 heads (part of the output still in L2)
+    "cfg2_360m_prefill": 25.24e6,                 # profiles/prefill_tc_kernel_dv64_cfg2.md (output stays in L2)
+    "cfg3_1p3b_prefill": 167.98e6 + 103.88e6,     # profiles/prefill_tc_kernel_dv128.md (part of the output still in L2)
     "cfg4_generation": 2 * (144.59e6 + 88.45e6),  # profiles/decode_step_kernel_dv128.md, 1024 -> 2048 heads
     "cfg5_mixer_pair:swa": 2 * (201.37e6 + 43.87e6),  # profiles/swa_tc_kernel.md, 16 -> 32 heads
     "baseconv": 4 * (272.67e6 + 96.72e6),         # profiles/baseconv_gate_kernel.md, batch 2 -> 8 (part of the writes still in L2)
