@@ -232,6 +232,36 @@ __device__ __forceinline__ void compute_phi_row(uint4 xlo, uint4 xhi, bool valid
     f[19] = make_uint4(valid ? 0x00003F80u : 0u, 0u, 0u, 0u);   // the constant feature 1.0
 }
 
+// The same expansion one 32-feature block (16 packed registers) at a time, for callers that store each block as it
+// is formed: block 0 = x' and the squares, block j = the products of offsets 2j-1 and 2j, block 4 = offset 7, the
+// eight products of offset 8, the constant.  E and O as in compute_phi_row.
+__device__ __forceinline__ void phi_prepare(uint4 xlo, uint4 xhi, bool valid, uint32_t (&E)[8], uint32_t (&O)[8]) {
+    const uint32_t x[8] = {xlo.x, xlo.y, xlo.z, xlo.w, xhi.x, xhi.y, xhi.z, xhi.w};
+    const uint32_t kHalf = 0x3F003F00u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) E[i] = valid ? mul2(x[i], kHalf) : 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) O[i] = __byte_perm(E[i], E[(i + 1) & 7], 0x5432);
+}
+template <int J>
+__device__ __forceinline__ void phi_block(const uint32_t (&E)[8], const uint32_t (&O)[8], bool valid, uint32_t (&v)[16]) {
+    const uint32_t kRs2 = 0x3F353F35u;
+    if constexpr (J == 0) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { v[i] = E[i]; v[8 + i] = mul2(E[i], mul2(E[i], kRs2)); }
+    } else if constexpr (J < 4) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { v[i] = mul2(E[i], O[(i + J - 1) & 7]); v[8 + i] = mul2(E[i], E[(i + J) & 7]); }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = mul2(E[i], O[(i + 3) & 7]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[8 + i] = mul2(E[i], E[i + 4]);
+        v[12] = valid ? 0x00003F80u : 0u;
+        v[13] = v[14] = v[15] = 0u;
+    }
+}
+
 // Write the 20 pieces as row t of a [128 tokens][160 features] tile made of five SWIZZLE_64B blocks.
 __device__ __forceinline__ void store_phi_row(const uint4 (&f)[20], uint8_t* tile, int t) {
     uint8_t* row = tile + (t >> 3) * 512 + (t & 7) * 64;
@@ -271,6 +301,17 @@ __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
     uint64_t r;
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
     return r;
+}
+__device__ __forceinline__ uint64_t mul2f(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// two fp32 accumulator columns scaled and packed to bf16: one two-wide multiply and one conversion
+__device__ __forceinline__ uint32_t scale_pack(uint32_t y0, uint32_t y1, uint64_t inv2) {
+    float lo, hi;
+    f32x2_split(mul2f(f32x2(y0, y1), inv2), lo, hi);
+    return pack_bf16(lo, hi);
 }
 __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     uint64_t r;
@@ -701,9 +742,9 @@ __global__ void __launch_bounds__(kThreads, 1)
                             mbar_arrive(&bars[kR4]);
                             if (t == 0) TRACE(5, c, 1);
                         }
+                        const uint64_t inv2 = f32x2(__float_as_uint(inv), __float_as_uint(inv));
 #pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            pkd[qd * 16 + i] = pack_bf16(__uint_as_float(y[2 * i]) * inv, __uint_as_float(y[2 * i + 1]) * inv);
+                        for (int i = 0; i < 16; ++i) pkd[qd * 16 + i] = scale_pack(y[2 * i], y[2 * i + 1], inv2);
                     }
 #pragma unroll
                     for (int h = 0; h < DV / 64; ++h) {
@@ -738,24 +779,17 @@ __global__ void __launch_bounds__(kThreads, 1)
                     // the staging tile is free once the previous TMA store has read it
                     if (t == 0) tma_store_wait_read<0>();
                     group_sync(1);
+                    const uint64_t inv2 = f32x2(__float_as_uint(inv), __float_as_uint(inv));
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint4 v4;
-                        v4.x = pack_bf16(__uint_as_float(y0[8 * j + 0]) * inv, __uint_as_float(y0[8 * j + 1]) * inv);
-                        v4.y = pack_bf16(__uint_as_float(y0[8 * j + 2]) * inv, __uint_as_float(y0[8 * j + 3]) * inv);
-                        v4.z = pack_bf16(__uint_as_float(y0[8 * j + 4]) * inv, __uint_as_float(y0[8 * j + 5]) * inv);
-                        v4.w = pack_bf16(__uint_as_float(y0[8 * j + 6]) * inv, __uint_as_float(y0[8 * j + 7]) * inv);
-                        *reinterpret_cast<uint4*>(orow + ((j ^ sw) << 4)) = v4;
-                    }
+                    for (int j = 0; j < 4; ++j)
+                        *reinterpret_cast<uint4*>(orow + ((j ^ sw) << 4)) =
+                            make_uint4(scale_pack(y0[8 * j], y0[8 * j + 1], inv2), scale_pack(y0[8 * j + 2], y0[8 * j + 3], inv2),
+                                       scale_pack(y0[8 * j + 4], y0[8 * j + 5], inv2), scale_pack(y0[8 * j + 6], y0[8 * j + 7], inv2));
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint4 v4;
-                        v4.x = pack_bf16(__uint_as_float(y1[8 * j + 0]) * inv, __uint_as_float(y1[8 * j + 1]) * inv);
-                        v4.y = pack_bf16(__uint_as_float(y1[8 * j + 2]) * inv, __uint_as_float(y1[8 * j + 3]) * inv);
-                        v4.z = pack_bf16(__uint_as_float(y1[8 * j + 4]) * inv, __uint_as_float(y1[8 * j + 5]) * inv);
-                        v4.w = pack_bf16(__uint_as_float(y1[8 * j + 6]) * inv, __uint_as_float(y1[8 * j + 7]) * inv);
-                        *reinterpret_cast<uint4*>(orow + (((4 + j) ^ sw) << 4)) = v4;
-                    }
+                    for (int j = 0; j < 4; ++j)
+                        *reinterpret_cast<uint4*>(orow + (((4 + j) ^ sw) << 4)) =
+                            make_uint4(scale_pack(y1[8 * j], y1[8 * j + 1], inv2), scale_pack(y1[8 * j + 2], y1[8 * j + 3], inv2),
+                                       scale_pack(y1[8 * j + 4], y1[8 * j + 5], inv2), scale_pack(y1[8 * j + 6], y1[8 * j + 7], inv2));
                     fence_proxy_async_smem();
                     group_sync(1);
                     if (t == 0) {
@@ -990,24 +1024,23 @@ __global__ void __launch_bounds__(kThreads, 1)
                     tmem_wait_st();
                     tc_fence_before();
                 } else if constexpr (PQS) {
-                    uint4 f[20];
-                    compute_phi_row(qlo, qhi, true, f);
+                    // block by block, each stored as it is formed (twenty pieces at once do not fit the registers)
+                    uint32_t E[8], O[8], vv[16];
+                    phi_prepare(qlo, qhi, true, E, O);
                     tc_fence_after();
+                    phi_block<0>(E, O, true, vv); tmem_st16(tmem_addr(tb, lane_base, C::colPQlo), vv);
+                    phi_block<1>(E, O, true, vv); tmem_st16(tmem_addr(tb, lane_base, C::colPQlo + 16), vv);
+                    phi_block<2>(E, O, true, vv); tmem_st16(tmem_addr(tb, lane_base, C::colPQlo + 32), vv);
+                    uint8_t* row = sPQ + (t >> 3) * 512 + (t & 7) * 64;     // feature blocks 3 and 4 -> blocks 0 and 1 of the tile
+                    const uint32_t sw = (t >> 1) & 3;
+                    phi_block<3>(E, O, true, vv);
 #pragma unroll
-                    for (int j = 0; j < 3; ++j) {              // pieces 0..11: features 0..95, four columns a piece
-                        const uint32_t r[16] = {f[4 * j].x, f[4 * j].y, f[4 * j].z, f[4 * j].w,
-                                                f[4 * j + 1].x, f[4 * j + 1].y, f[4 * j + 1].z, f[4 * j + 1].w,
-                                                f[4 * j + 2].x, f[4 * j + 2].y, f[4 * j + 2].z, f[4 * j + 2].w,
-                                                f[4 * j + 3].x, f[4 * j + 3].y, f[4 * j + 3].z, f[4 * j + 3].w};
-                        tmem_st16(tmem_addr(tb, lane_base, C::colPQlo + j * 16), r);
-                    }
-                    {                                          // pieces 12..19: feature blocks 3 and 4 -> blocks 0 and 1 of the tile
-                        uint8_t* row = sPQ + (t >> 3) * 512 + (t & 7) * 64;
-                        const uint32_t sw = (t >> 1) & 3;
+                    for (int j = 0; j < 4; ++j)
+                        *reinterpret_cast<uint4*>(row + ((j ^ sw) << 4)) = make_uint4(vv[4 * j], vv[4 * j + 1], vv[4 * j + 2], vv[4 * j + 3]);
+                    phi_block<4>(E, O, true, vv);
 #pragma unroll
-                        for (int j = 12; j < 20; ++j)
-                            *reinterpret_cast<uint4*>(row + ((j >> 2) - 3) * (kC * 64) + (((j & 3) ^ sw) << 4)) = f[j];
-                    }
+                    for (int j = 0; j < 4; ++j)
+                        *reinterpret_cast<uint4*>(row + kC * 64 + ((j ^ sw) << 4)) = make_uint4(vv[4 * j], vv[4 * j + 1], vv[4 * j + 2], vv[4 * j + 3]);
                     tmem_wait_st();
                     tc_fence_before();
                     fence_proxy_async_smem();
@@ -1032,6 +1065,11 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
             for (int i = 0; i < 16; ++i) dm[i] = (2 * i + 1 <= lane) ? 0xFFFFFFFFu : ((2 * i <= lane) ? 0x0000FFFFu : 0u);
         }
+        // sixteen registers of zeros for the batches right of the diagonal (opaque, or each store would be
+        // preceded by sixteen moves)
+        uint32_t zz[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) asm volatile("mov.b32 %0, 0;" : "=r"(zz[i]));
         for (int c = 0; c < nch && ok; ++c) {
             ok = mbar_wait(&bars[kG1 + t_idx(c)], t_parity(c), abort_flag);
             if (!ok) break;
@@ -1052,12 +1090,20 @@ __global__ void __launch_bounds__(kThreads, 1)
                         // would be rounded to bf16 anyway).  The row sum is the tensor cores' work (see step (3)).
                         const __nv_bfloat162 c1 = __float2bfloat162_rn(0.25f), c2 = __float2bfloat162_rn(0.03125f),
                                              one = __float2bfloat162_rn(1.0f);
-                        const uint32_t full = (b < q4) ? 0xFFFFFFFFu : 0u;      // a batch left of the diagonal is seen whole
+                        if (b < q4) {                    // a batch left of the diagonal is seen whole
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const __nv_bfloat162 s2 = __floats2bfloat162_rn(__uint_as_float(sc[2 * i]), __uint_as_float(sc[2 * i + 1]));
-                            const __nv_bfloat162 w2 = __hfma2(s2, __hfma2(s2, c2, c1), one);
-                            pk[i] = *reinterpret_cast<const uint32_t*>(&w2) & (dm[i] | full);
+                            for (int i = 0; i < 16; ++i) {
+                                const __nv_bfloat162 s2 = __floats2bfloat162_rn(__uint_as_float(sc[2 * i]), __uint_as_float(sc[2 * i + 1]));
+                                const __nv_bfloat162 w2 = __hfma2(s2, __hfma2(s2, c2, c1), one);
+                                pk[i] = *reinterpret_cast<const uint32_t*>(&w2);
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const __nv_bfloat162 s2 = __floats2bfloat162_rn(__uint_as_float(sc[2 * i]), __uint_as_float(sc[2 * i + 1]));
+                                const __nv_bfloat162 w2 = __hfma2(s2, __hfma2(s2, c2, c1), one);
+                                pk[i] = *reinterpret_cast<const uint32_t*>(&w2) & dm[i];
+                            }
                         }
                     } else {
                         // fp32 polynomial on pairs of scores (two-wide fp32 multiply-add): t = s/32 + 1/4, w = s t + 1
@@ -1090,15 +1136,13 @@ __global__ void __launch_bounds__(kThreads, 1)
                             }
                         }
                     }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) pk[i] = 0u;
                 }
                 if (PQT && b == 3) {               // every score column has been read: phi(Q) may take the upper half
                     tc_fence_before();
                     mbar_arrive(&bars[kTR + t_idx(c)]);
                 }
-                tmem_st16(tmem_addr(tb, lane_base, colTc + b * 16), pk);
+                if (b <= q4) tmem_st16(tmem_addr(tb, lane_base, colTc + b * 16), pk);
+                else tmem_st16(tmem_addr(tb, lane_base, colTc + b * 16), zz);
             }
             if constexpr (!PKW) s_den[(c & 3) * kC + tid] = den0 + den1;
             tmem_wait_st();
