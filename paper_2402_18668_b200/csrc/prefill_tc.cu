@@ -1347,6 +1347,9 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
 static SegPlan prefill_tc_plan(int BH, int L, int d_v, bool continued = false) {
     const int nch = (L + kC - 1) / kC;
     const float full = d_v == 64 ? 3.3f : 3.4f, upd = d_v == 64 ? 1.0f : 1.4f;
+    // a pre-chunk of the recompute mode costs more than a chunk of the state pass (d_v 64, cfg 2: 2.1 k cycles against
+    // 3.5 k for a full chunk of that kernel); of 1.0 / 1.5 / 2.0 / 2.4 this value gave the shortest calls
+    const float pre = d_v == 64 ? 1.5f : upd;
     int nmax = 148 / BH;
     if (nmax > 8) nmax = 8;
     // state pass: a split pays only when every segment keeps at least 16 chunks
@@ -1361,7 +1364,7 @@ static SegPlan prefill_tc_plan(int BH, int L, int d_v, bool continued = false) {
             float cost = 0.f;
             for (int j = 0; j < n; ++j) {
                 const int own = (j == n - 1) ? nch - per * (n - 1) : per;
-                const float c = (float)(j * per) * upd + (float)own * full;
+                const float c = (float)(j * per) * pre + (float)own * full;
                 if (c > cost) cost = c;
             }
             if (cost < 0.95f * best_cost) {
