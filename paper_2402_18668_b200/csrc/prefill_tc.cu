@@ -22,19 +22,24 @@
 // x'_m x'_(m+8), m < 8 | 1 | 0 x 7].  Its inner products equal those of the 273-feature
 // map; the state is expanded to / folded from the 273-row ABI layout at the kernel's edges.
 //
-// Warp roles (576 threads): warps 0-3 "row" group (one thread per query row: polynomial),
+// Warp roles (608 threads): warps 0-3 "row" group (one thread per query row: polynomial),
 // warps 4-7 "feature" group (one thread per token: phi expansion), warps 8-11 "state"
 // group (one thread per TMEM lane: bf16 state copy, state I/O), warps 12-15 "output"
 // group (one thread per output row: normalise, stage, TMA store), warp 16 TMA producer,
 // warp 17 issues the state-update MMAs (5)/(z), warp 18 the output-side MMAs (1)/(4)/(3):
-// two independent in-order streams, so the state chain runs ahead of the output chain.
-// All cross-role hand-offs are mbarriers with bounded waits.
+// two independent in-order streams, so the state chain runs ahead of the output chain; both
+// warps run converged and predicate only the MMA and its commit on one elected lane (sm100.cuh).
+// All cross-role hand-offs are mbarriers with bounded waits.  A piece that ends its head (or, in
+// the state pass, its range) has its final state written by all four groups, a quarter each.
 //
 // d_v 64, plain chunk loop: phi(Q) does not go through shared memory.  The feature group writes it
 // into tensor memory (the upper half of the chunk's score buffer once the row group has read the
 // scores, plus 16 spare columns) as the A operand of step (4), and the shared-memory tile that
 // frees holds a second state-copy tile, so the copy for chunk c+1 is written while step (4) of
 // chunk c reads its own.
+// d_v 128, plain chunk loop: features 0..95 of phi(Q) go to the 48 tensor-memory columns behind
+// the z tiles, features 96..159 to shared memory; the rest of the phi(Q) tile's place is a second
+// output staging tile, and the output group releases the accumulator before it stages anything.
 #include <cuda_bf16.h>
 #include <cstdlib>
 
