@@ -18,7 +18,7 @@
 // fp32 (without a centre the two separately rounded tiles would have to cancel).
 //
 // One CTA per (head, 128-row tile), 160 threads: warps 0-3 own one accumulator row each (the
-// polynomial, masks and bf16 packing), lane 0 of warp 4 issues TMA loads and MMAs.  The loop over
+// polynomial, masks and bf16 packing), warp 4 issues TMA loads and MMAs (converged, one elected lane).  The loop over
 // the other side's tiles is sequential per CTA (loads of the next tile are in flight during the
 // current one); parallelism comes from the (tile, head) grid.  q and k tiles are loaded 32
 // columns wide (columns 16..31 are zero-filled by TMA) so that they serve both as K-major

@@ -11,7 +11,7 @@
 //
 // One CTA per head walks the 128-token tiles in order (rev: last to first), 288 threads: eight row
 // warps, two threads per token of the step (and per accumulator lane at the block ends), each with
-// half of the features; lane 0 of warp 8 issues TMA loads and MMAs.  Per step the row threads form
+// half of the features; warp 8 issues TMA loads and MMAs (converged, one elected lane).  Per step the row threads form
 // their token's 160 monomials times u_t in fp32, round once to bf16 and write them as a row of the B
 // operand ([128 tokens][160], MN-major, five SWIZZLE_64B blocks of 32 features); the value tile comes
 // by TMA and is the A operand as it lies ([128 tokens][d_v], MN-major), so the accumulator in tensor

@@ -5,7 +5,7 @@
 //
 // in the state's own row order (row 0 constant, rows 1..d' linear, row 1 + d' + m d' + n the
 // product k_m k_n).  One CTA per (block of 128 feature rows, head), 160 threads: the four row
-// warps own one feature row (= accumulator lane) each, lane 0 of warp 4 issues TMA loads and
+// warps own one feature row (= accumulator lane) each, warp 4 (converged, one elected lane) issues TMA loads and
 // MMAs.  Per step of 64 tokens the row threads transpose the k tile ([token][m] -> [m][token]),
 // form their row of the A operand, [128 features][64 tokens] in the K-major SWIZZLE_128B layout,
 // as packed bf16 products k_m k_n (eight tokens per instruction), and one MMA burst adds
