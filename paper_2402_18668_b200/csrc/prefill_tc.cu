@@ -469,6 +469,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     uint8_t* sOut = smem + C::offOut;
 
     if (tid == 0) { TRACE(5, 0, 7); TRACE_CTA(0); }     // kernel entry
+    // state pass: the main pass of the same call may be scheduled behind this CTA (see launch_main_after_state)
+    if (STATE_ONLY) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(&bars[kFull0 + s], 1); mbar_init(&bars[kEmpty0 + s], STATE_ONLY ? 1 : 2); }
         mbar_init(&bars[kG1], 1); mbar_init(&bars[kG1b], 1); mbar_init(&bars[kPb], 128); mbar_init(&bars[kG2], 1); mbar_init(&bars[kG2b], 1); mbar_init(&bars[kG4], 1); mbar_init(&bars[kG4b], 1);
@@ -826,6 +828,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         const float* zh = p.z_abi ? p.z_abi + (size_t)head * abi_nrows : nullptr;
         const bool from_abi = !STATE_ONLY && p.continue_abi;
         const int nprev = ws_count;
+        // the partial states are the state pass's output (a no-op when this grid was launched the plain way)
+        if (MODE == kModeMain && nprev > 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 
         // Initial value of this lane's row: the caller's ABI state (folded into the internal
         // basis) plus the partial states of the earlier segments.  Loads are issued 16 at a
@@ -1261,6 +1265,27 @@ bool make_map(CUtensorMap* m, const void* base, int BH, int L, int width, int bo
 unsigned long long* g_trace = nullptr;
 #endif
 
+// The main pass behind a state pass of the same call, launched with programmatic stream serialization: its CTAs
+// may start (set-up, first loads) as the state pass's CTAs leave their SMs, and the one group that reads what the
+// state pass wrote waits for that grid's completion inside the kernel (griddepcontrol.wait).  Every CTA of the
+// state pass signals at its start, so the main pass's CTAs are scheduled only once every CTA of the state pass is
+// resident or done: they cannot take an SM that a CTA of the state pass still needs.
+template <int DV>
+cudaError_t launch_main_after_state(dim3 grid, cudaStream_t stream, const CUtensorMap& tq, const CUtensorMap& tk,
+                                    const CUtensorMap& tv, const CUtensorMap& to, const Params& p) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = Cfg<DV>::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<DV, kModeMain>, tq, tk, tv, to, p);
+}
+
 template <int DV>
 based_status launch_dv(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH, int L,
                        int dv, int flags, float* ws, const SegPlan plan, cudaStream_t stream) {
@@ -1316,7 +1341,7 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
         note_launch();
         const based_status st = check_launch("prefill_tc_kernel<state, balanced>");
         if (st != BASED_OK) return st;
-        prefill_tc_kernel<DV, kModeMain><<<grid, kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
+        if (launch_main_after_state<DV>(grid, stream, tq, tk, tv, to, p) != cudaSuccess) return BASED_ERR_CUDA;
         note_launch();
         return check_launch("prefill_tc_kernel<balanced>");
     }
@@ -1331,7 +1356,11 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
         const based_status st = check_launch("prefill_tc_kernel<state>");
         if (st != BASED_OK) return st;
     }
-    prefill_tc_kernel<DV, kModeMain><<<dim3(nseg, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
+    if (nseg > 1) {
+        if (launch_main_after_state<DV>(dim3(nseg, BH), stream, tq, tk, tv, to, p) != cudaSuccess) return BASED_ERR_CUDA;
+    } else {
+        prefill_tc_kernel<DV, kModeMain><<<dim3(nseg, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
+    }
     note_launch();
     return check_launch("prefill_tc_kernel");
 }
