@@ -1259,3 +1259,42 @@ def test_more_heads_than_one_grid_dimension_holds():
         assert_state_close(_np(kv[sl]), S_ref, _np(z[sl]), z_ref, "bf16", f"head {bh}")
         assert_state_close(_np(kv2[sl]), S_ref, _np(z2[sl]), z_ref, "bf16", f"head {bh}, state-only call")
         assert row_err(_np(out_swa[sl]), oracle.swa(_np(qs[sl]), _np(ks[sl]), _np(v[sl]), 64)) <= TOL_BF16, bh
+
+
+# --------------------------------------------------------------------------- calls that depend on one another
+@pytest.mark.parametrize("B,H,L,d_v,cont", [(2, 32, 2048, 64, False),     # recompute mode: a dependent launch behind the call before
+                                            (1, 40, 16500, 128, False),   # equal chunk ranges: state pass, then a dependent main pass
+                                            (1, 16, 8192, 64, True),      # continued call: state pass per segment + main pass
+                                            (1, 148, 1024, 64, False)])   # plain chunk loop
+def test_chained_calls_without_host_synchronisation(B, H, L, d_v, cont):
+    """Three prefill calls in a row on one stream, each taking the call before's output as its values (and, in the
+    continued case, its state), first with the host waiting between the calls and then without: the kernels of a call
+    may be scheduled before the call ahead of them has finished (programmatic dependent launches), so every read of
+    a predecessor's result has to sit behind the wait inside the kernel.  Bit-for-bit the same outputs and states."""
+    w = wl.Workload("chain", B, H, L, 16, d_v, "bf16", 0.3)
+    q, k, v = (t.to(DEV) for t in wl.prefill_inputs(w, wl.generator(B * H + L)))
+    flags = based.BASED_STATE_CONTINUE if cont else based.BASED_STATE_ZERO_INIT
+
+    def chain(wait):
+        kv, z = based.new_state(B, H, d_v)
+        x = v
+        outs = []
+        for _ in range(3):
+            o = torch.empty_like(v)
+            based.based_prefill(q, k, x, out=o, kv_state=kv, z_state=z, flags=flags)
+            if wait:
+                torch.cuda.synchronize()
+            # the output is a weighted mean of the values (positive weights), so it can serve as the next call's values
+            # as it is: no kernel of another library runs between two calls of the chain
+            x = o
+            outs.append(o)
+        torch.cuda.synchronize()
+        _poll()
+        return outs, kv.clone(), z.clone()
+
+    ref, kv_ref, z_ref = chain(True)
+    for _ in range(3):
+        got, kv_got, z_got = chain(False)
+        for a, b in zip(ref, got):
+            assert torch.equal(a, b)
+        assert torch.equal(kv_ref, kv_got) and torch.equal(z_ref, z_got)
