@@ -68,6 +68,10 @@ struct Cfg {
     // d_v 64: four stages (a tile's load takes about 2500 cycles from issue to arrival, more than a chunk's period;
     // with three the next chunk's scores waited for their tile: measured 5-8 % on the 360M shapes)
     static constexpr int kStages = (DV == 64) ? 4 : 2;
+    // The state pass loads no q tile and needs neither state copy nor output staging, and what bounds it is the bytes
+    // in flight (20 KB per stage and SM, about 2500 cycles per load: four stages are 4.7 TB/s over 148 SMs), so its
+    // stages are packed (k tile, v tile) and there are as many as fit in front of the ones block and two phi(K) tiles
+    static constexpr int kStagesState = (DV == 64) ? 6 : 3;
     static constexpr int kNY = DV + 16;                         // Y columns: d_v numerators + denominator block
     static constexpr int kSLanes = (DV == 64) ? 65 : 128;       // live lanes of S^T (d_v 64: lane 64 carries z)
     static constexpr uint32_t kQKBytes = kC * 32;               // one q or k tile (16 bf16 per token)
@@ -117,7 +121,7 @@ struct Cfg {
 };
 
 enum Bar {
-    kFull0 = 0, kEmpty0 = 4, kG1 = 8, kG1b, kP, kPb, kG2, kG2b, kG4, kG4b, kG3, kR4, kPK, kPKb, kSR, kDone, kTR, kTRb, kSC, kSCb, kFin,
+    kFull0 = 0, kEmpty0 = 8, kG1 = 16, kG1b, kP, kPb, kG2, kG2b, kG4, kG4b, kG3, kR4, kPK, kPKb, kSR, kDone, kTR, kTRb, kSC, kSCb, kFin,
     kNumBars
 };
 
@@ -353,7 +357,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
                       const Params p) {
     using C = Cfg<DV>;
-    constexpr int NS = C::kStages;
+    constexpr int NS = (MODE == kModeState) ? C::kStagesState : C::kStages;
     constexpr bool STATE_ONLY = MODE == kModeState;
     constexpr bool PRE = MODE == kModePre;
     // phi(Q) in tensor memory and two state-copy tiles: the plain chunk loop only (measured: -7 % where every
@@ -462,10 +466,16 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int ntot = npre + nch;
     const int tok_first = tok_begin - npre * kC;
 
-    uint8_t* sPK = smem + C::offPK;
-    uint8_t* sPQ = smem + C::offPQ;
+    // shared-memory layout: as in Cfg, except in the state pass (see Cfg::kStagesState)
+    constexpr uint32_t kStride = STATE_ONLY ? C::kQKBytes + C::kVBytes : C::kStageBytes;     // bytes of one stage
+    constexpr uint32_t kOffK = STATE_ONLY ? 0u : C::kQKBytes, kOffV = kOffK + C::kQKBytes;     // k and v tile within a stage
+    constexpr uint32_t offOnesM = STATE_ONLY ? NS * kStride : C::offOnes;
+    constexpr uint32_t offPKM = offOnesM + C::kOnesBytes, offPQM = offPKM + C::kPhiBytes;
+    static_assert(offPQM + C::kPhiBytes <= C::offMisc && offPKM % 1024 == 0 && kStride % 1024 == 0, "state pass layout");
+    uint8_t* sPK = smem + offPKM;
+    uint8_t* sPQ = smem + offPQM;
     uint8_t* sSc = smem + C::offSc;
-    uint8_t* sOnes = smem + C::offOnes;
+    uint8_t* sOnes = smem + offOnesM;
     uint8_t* sOut = smem + C::offOut;
 
     if (tid == 0) { TRACE(5, 0, 7); TRACE_CTA(0); }     // kernel entry
@@ -500,8 +510,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         for (uint32_t i = tid * 16; i < C::kOnesBytes; i += kThreads * 16)
             *reinterpret_cast<uint4*>(sOnes + i) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
     }
-    for (uint32_t i = tid * 16; i < C::kScBytes; i += kThreads * 16)
-        *reinterpret_cast<uint4*>(sSc + i) = make_uint4(0u, 0u, 0u, 0u);
+    if (!STATE_ONLY) {
+        for (uint32_t i = tid * 16; i < C::kScBytes; i += kThreads * 16)
+            *reinterpret_cast<uint4*>(sSc + i) = make_uint4(0u, 0u, 0u, 0u);
+    }
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -548,15 +560,15 @@ __global__ void __launch_bounds__(kThreads, 1)
                 ok = mbar_wait(&bars[kEmpty0 + s], ((g / NS) & 1) ^ 1, abort_flag);
                 if (!ok) break;
                 TRACE(1, g, 3);
-                uint8_t* st = smem + C::offStage + s * C::kStageBytes;
+                uint8_t* st = smem + C::offStage + s * kStride;
                 const int tok0 = tok_first + g * kC;
                 const bool with_q = !STATE_ONLY && g >= npre;
                 mbar_arrive_expect_tx(&bars[kFull0 + s], (with_q ? 2 : 1) * C::kQKBytes + C::kVBytes);
                 if (with_q) tma_load_3d(st, &tm_q, &bars[kFull0 + s], 0, tok0, head);
-                tma_load_3d(st + C::kQKBytes, &tm_k, &bars[kFull0 + s], 0, tok0, head);
+                tma_load_3d(st + kOffK, &tm_k, &bars[kFull0 + s], 0, tok0, head);
 #pragma unroll
                 for (int b = 0; b < DV / 64; ++b)
-                    tma_load_3d(st + 2 * C::kQKBytes + b * (kC * 128), &tm_v, &bars[kFull0 + s], b * 64, tok0, head);
+                    tma_load_3d(st + kOffV + b * (kC * 128), &tm_v, &bars[kFull0 + s], b * 64, tok0, head);
             }
         }
     } else if (warp == kWarpMma) {
@@ -576,7 +588,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             const uint32_t lPK0 = desc_lo(dPhiMN) + (smem_u32(sPK) >> 4), lPK1 = desc_lo(dPhiMN) + (smem_u32(sPQ) >> 4);
             for (int c = 0; c < ntot && ok; ++c) {      // c counts pre-chunks and own chunks here
                 const int s = c % NS;
-                const uint32_t aVt = smem_u32(smem + C::offStage + s * C::kStageBytes) + 2 * C::kQKBytes;
+                const uint32_t aVt = smem_u32(smem + C::offStage + s * kStride) + kOffV;
                 const uint32_t lPK = (alt(c) && (c & 1)) ? lPK1 : lPK0;
                 ok = mbar_wait(&bars[kFull0 + s], (c / NS) & 1, abort_flag);
                 if (ok) ok = mbar_wait(pk_bar(c), g2_parity(c), abort_flag);
@@ -980,13 +992,13 @@ __global__ void __launch_bounds__(kThreads, 1)
         for (int g = 0; g < ntot && ok; ++g) {
             const int c = g - npre;                     // own chunk index (negative: pre-chunk)
             const int s = g % NS;
-            const uint8_t* st = smem + C::offStage + s * C::kStageBytes;
+            const uint8_t* st = smem + C::offStage + s * kStride;
             const bool valid = tok_first + g * kC + t < tok_end;
             ok = mbar_wait(&bars[kFull0 + s], (g / NS) & 1, abort_flag);
             if (!ok) break;
             if (t == 0) TRACE(3, c, 0);
             uint4 klo, khi, qlo = make_uint4(0u, 0u, 0u, 0u), qhi = qlo;
-            read_qk_row(st + C::kQKBytes, t, klo, khi);
+            read_qk_row(st + kOffK, t, klo, khi);
             if (!STATE_ONLY && c >= 0) read_qk_row(st, t, qlo, qhi);
             // the tile being overwritten was last read by step (5) of the chunk before (two chunks
             // before where tiles alternate; own chunk 0 after pre-chunks: the last even pre-chunk)
