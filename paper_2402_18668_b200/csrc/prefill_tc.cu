@@ -72,6 +72,14 @@ struct Cfg {
     // in flight (20 KB per stage and SM, about 2500 cycles per load: four stages are 4.7 TB/s over 148 SMs), so its
     // stages are packed (k tile, v tile) and there are as many as fit in front of the ones block and two phi(K) tiles
     static constexpr int kStagesState = (DV == 64) ? 6 : 3;
+    // How a piece of the main pass gets the state of the pieces before it in its head (up to seven workspace slots,
+    // or one per earlier range, of 40-80 KB each).  Its state group reading them alone spends 2.7 us of load latency
+    // per slot before the first state update can run (11 us on cfg 5's last pieces, 46 us with 18 pieces per head).
+    // d_v 128: all four role groups share the read (init_state_blocks).  d_v 64: a small kernel between the two
+    // passes turns the slots into running sums (slot_scan_kernel) and the piece reads one slot; sharing the read
+    // as at d_v 128 was as fast there, but every form of it tried slowed that kernel's role loops by 3-18 %
+    // (register allocation), on shapes that have no slots at all.
+    static constexpr bool kSlotScan = DV == 64;
     static constexpr int kNY = DV + 16;                         // Y columns: d_v numerators + denominator block
     static constexpr int kSLanes = (DV == 64) ? 65 : 128;       // live lanes of S^T (d_v 64: lane 64 carries z)
     static constexpr uint32_t kQKBytes = kC * 32;               // one q or k tile (16 bf16 per token)
@@ -94,7 +102,7 @@ struct Cfg {
     static constexpr uint32_t offSc = offPQ + kPhiBytes;
     static constexpr uint32_t offOut = offSc + kScBytes;
     static constexpr uint32_t offMisc = offOut + kOutBytes;
-    static constexpr uint32_t kMiscBytes = 3072;                // barriers, row sums, ABI row table
+    static constexpr uint32_t kMiscBytes = 3072;                // barriers, row sums, ABI row table, the CTA's piece
     static constexpr uint32_t kSmemBytes = offMisc + kMiscBytes + 1024;   // + alignment slack
     static_assert(kSmemBytes <= 232448, "shared memory budget");
     // TMEM columns
@@ -121,7 +129,7 @@ struct Cfg {
 };
 
 enum Bar {
-    kFull0 = 0, kEmpty0 = 8, kG1 = 16, kG1b, kP, kPb, kG2, kG2b, kG4, kG4b, kG3, kR4, kPK, kPKb, kSR, kDone, kTR, kTRb, kSC, kSCb, kFin,
+    kFull0 = 0, kEmpty0 = 8, kG1 = 16, kG1b, kP, kPb, kG2, kG2b, kG4, kG4b, kG3, kR4, kPK, kPKb, kSR, kDone, kTR, kTRb, kSC, kSCb, kFin, kInit,
     kNumBars
 };
 
@@ -143,6 +151,7 @@ struct Params {
                           // the tensor maps zero-fill columns 112..127 on load and clip them on store)
     int balanced;         // > 0: the number of equal chunk ranges the heads' chunks are cut into (see the kernel)
     int heads;            // B*H (balanced mode)
+    int pad;              // balanced mode: chunks counted in front of every head for the CTA it starts
 #ifdef BASED_TRACE
     unsigned long long* trace;
 #endif
@@ -158,10 +167,10 @@ struct Params {
 #define TRACE(role, c, ev) do {} while (0)
 #endif
 #ifdef BASED_TRACE
-// wall-clock entry / exit of every CTA (with its SM), after the per-role events
+// wall-clock entry / exit of every CTA (with its SM), after the per-role events (state pass: 2048 entries further on)
 #define TRACE_CTA(which)                                                                                      \
     do {                                                                                                      \
-        if (p.trace) p.trace[6 * 64 * 8 + (blockIdx.y * gridDim.x + blockIdx.x) * 2 + (which)] = (global_timer_ns() << 8) | smid_u32(); \
+        if (p.trace) p.trace[6 * 64 * 8 + ((MODE == kModeState ? 2048 : 0) + blockIdx.y * gridDim.x + blockIdx.x) * 2 + (which)] = (global_timer_ns() << 8) | smid_u32(); \
     } while (0)
 #else
 #define TRACE_CTA(which) do {} while (0)
@@ -351,6 +360,206 @@ __device__ __forceinline__ bool group_all(int id, bool pred) {
 // MODE: kModeMain = chunk loop from a given initial state; kModeState = state-update-only pass over
 // a segment (partial state to the workspace); kModePre = kModeMain preceded by state-update-only
 // "pre-chunks" over everything before the segment (recompute mode).
+// ---- initial state.  One thread per TMEM lane of the state accumulator S^T; lane t of a warp's lane quarter holds
+// V column t (d_v 64: lane 64 the K-state).  Its initial value is the caller's ABI state (folded into the internal
+// basis; kv_abi == nullptr: none) plus the partial states of the earlier pieces (nprev workspace slots from wsh on).
+// Those are up to seven slots of 40-80 KB each, read as ten 16-column blocks per slot, and one thread group doing it
+// alone spends 0.7 us of load latency per block and slot before the first state update can run (2.7 us per slot).
+// So in the main pass all four role groups (each has a warp per lane quarter) take every fourth block (part of
+// nparts), and two slots' loads are in flight at a time; the state group waits for the others before it reads the
+// state.  Not inlined: its registers are its own and the role loops' allocation does not see it.
+template <int DV>
+__device__ __noinline__ void init_state_blocks(const float* wsh, int nprev, bool wait_for_state_pass, const float* kv_abi,
+                                               const float* z_abi, int dv, int abi_row0, const short2* s_abi, uint32_t tb,
+                                               int part, int nparts) {
+    using C = Cfg<DV>;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
+    const int t = ((warp & 3) << 5) + lane;
+    // what this thread's lane of S^T holds: V column srow, or (d_v 64) the K-state at lane 64
+    const int srow = (t < C::kSLanes) ? t : -1;
+    const bool is_z = (DV == 64) && t == 64;
+    // d_v 128: K-state features held in the two z tiles (64-row MMA: rows 0..31 in lanes 0-15, 32-47)
+    const int z1f = (DV == 128 && (t & 31) < 16 && (t >> 5) < 2) ? 128 + (t >> 5) * 16 + (t & 15) : -1;
+    const size_t seg_stride = seg_state_floats(DV);
+    const bool from_abi = kv_abi != nullptr;            // dv: row pitch of the caller's state; lanes >= dv hold zeros
+    const float* kvh = from_abi ? kv_abi + (size_t)abi_row0 * dv : nullptr;
+    const float* zh = from_abi ? z_abi + abi_row0 : nullptr;
+    // the partial states are the state pass's output (a no-op when this grid was launched the plain way)
+    if (wait_for_state_pass) asm volatile("griddepcontrol.wait;" ::: "memory");
+#pragma unroll 1
+    for (int b = part; b < kF / 16; b += nparts) {
+        float acc[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+        if (srow >= 0) {
+            if (from_abi) {
+                float va[16], vb[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const short2 ar = s_abi[b * 16 + i];
+                    const bool live = is_z || srow < dv;
+                    va[i] = (ar.x >= 0 && live) ? (is_z ? zh[ar.x] : kvh[(size_t)ar.x * dv + srow]) : 0.f;
+                    vb[i] = (ar.y >= 0 && live) ? (is_z ? zh[ar.y] : kvh[(size_t)ar.y * dv + srow]) : 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] = (s_abi[b * 16 + i].y >= 0) ? (va[i] + vb[i]) * kRsqrt2 : va[i];
+            }
+            const float* src = wsh + (is_z ? (size_t)kF * DV + b * 16 : (size_t)(b * 16) * DV + srow);
+            const size_t step = is_z ? 1 : DV;
+            int sp = 0;
+#pragma unroll 1
+            for (; sp + 1 < nprev; sp += 2, src += 2 * seg_stride) {
+                float t0[16], t1[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) { t0[i] = src[i * step]; t1[i] = src[seg_stride + i * step]; }
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] += t0[i] + t1[i];
+            }
+            if (sp < nprev) {
+                float t0[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) t0[i] = src[i * step];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] += t0[i];
+            }
+        }
+        uint32_t r[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(acc[i]);
+        tmem_st16(tmem_addr(tb, lane_base, C::colS + b * 16), r);
+    }
+    // d_v 128: K-state of feature t (tile 0) and feature z1f (tile 1), column 0 of each tile
+    auto z_init = [&](int f) -> float {
+        if (f < 0) return 0.f;
+        float acc = 0.f;
+        if (from_abi) {
+            const short2 ar = s_abi[f];
+            if (ar.x >= 0) acc = (ar.y >= 0) ? (zh[ar.x] + zh[ar.y]) * kRsqrt2 : zh[ar.x];
+        }
+        for (int sp = 0; sp < nprev; ++sp) acc += wsh[(size_t)sp * seg_stride + (size_t)kF * DV + f];
+        return acc;
+    };
+    if (DV == 128 && part == nparts - 1) {
+        uint32_t r0[16], r1[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) r0[i] = r1[i] = 0u;
+        r0[0] = __float_as_uint(z_init(t));
+        r1[0] = __float_as_uint(z_init(z1f));
+        tmem_st16(tmem_addr(tb, lane_base, C::colZ0), r0);
+        tmem_st16(tmem_addr(tb, lane_base, C::colZ1), r1);
+    }
+    tmem_wait_st();
+}
+
+// ---- the CTA's piece of work: a head, a token range, where its initial state comes from (workspace slots
+// ws_first .. ws_first + ws_count - 1) and where its final state goes (slot ws_out, or the caller's state if
+// the piece ends its head).
+// Legacy grids: blockIdx.x = sequence segment, blockIdx.y = head.
+// Balanced grids (one row of CTAs): the concatenation of all heads' chunks, T = heads x chunks per head, is
+// cut into n equal ranges [i T / n, (i + 1) T / n), one per SM.  A range holds at most one head boundary
+// (n >= heads).  CTA i < n takes range i up to the boundary, if there is one; CTA n + j takes what is left
+// of a range behind its boundary, the j-th largest such rest first: the hardware hands these later CTAs to
+// SMs as they become free, and the SM whose first piece was shortest is free first, so every SM ends up
+// with about T / n chunks.  A piece that ends inside its head leaves its state in slot i of its range.
+// A CTA's start-up and wind-down cost as much as `pad` chunks, and an SM with a head boundary pays them twice:
+// in this count every head is preceded by `pad` chunks that nobody runs, so such an SM gets that many fewer.
+struct Piece { int head, seg, begin, end, first, count, out, head_end, skip; };
+// Every thread of the CTA calls it.  find_piece is the same out of line, with the result in shared memory: how this
+// arithmetic is compiled into the kernel moves the time of the role loops by several per cent either way (register
+// allocation), so each instance of the kernel takes the form that measured faster for it (Cfg::kPieceOutOfLine).
+template <int MODE, bool SCAN>
+__device__ __forceinline__ void piece_of_cta(Piece& piece, int* s_rest, int balanced, int heads, int pad, int L, int seg_len, int nseg) {
+    bool skip = false;
+    int it_head = blockIdx.y, it_seg = blockIdx.x, it_begin = blockIdx.x * seg_len, it_end = 0, it_first = 0, it_count = 0,
+        it_out = -1;
+    bool it_head_end = false;
+    if (MODE != kModePre && balanced > 0) {      // (the recompute mode's kernel is never launched this way)
+        // 32-bit arithmetic throughout (the host takes this path only while (T + 1) n fits: 64-bit divisions
+        // would be subroutine calls, and their mere presence slows this kernel's role loops by a fifth)
+        const uint32_t n = balanced;
+        const uint32_t nchr = (L + kC - 1) / kC;                // chunks of a head
+        const uint32_t w = pad, nchh = nchr + w;                // ... and with the pad in front of them
+        const uint32_t T = (uint32_t)heads * nchh;
+        uint32_t lo, hi, range;                    // global (padded) chunk range of this piece, index of its range
+        if (blockIdx.x < n) {
+            range = blockIdx.x;
+            lo = range * T / n;
+            hi = (range + 1) * T / n;
+            const uint32_t xb = ((hi - 1) / nchh) * nchh;         // start of the head that holds the range's last chunk
+            if (xb > lo) hi = xb;                                  // a boundary inside: stop there
+        } else {
+            // rest of the range behind head boundary h: [h nchh, end of the range that holds it); rank the rests
+                        const int nb = heads - 1, want = (int)(blockIdx.x - n);
+            auto rest_of = [&](uint32_t h, uint32_t& rg) -> int {
+                const uint32_t x = h * nchh;
+                rg = ((x + 1) * n + T - 1) / T - 1;                 // the range that holds chunk x
+                if (rg * T / n == x) return 0;                      // the boundary is a range start
+                const uint32_t r = (rg + 1) * T / n - x;
+                return r > w ? (int)(r - w) : 0;                    // real chunks behind the pad
+            };
+            for (int h = 1 + threadIdx.x; h <= nb; h += kThreads) { uint32_t rg; s_rest[h] = rest_of(h, rg); }
+            __syncthreads();
+            s_rest[0] = -1;
+            __syncthreads();
+            for (int h = 1 + threadIdx.x; h <= nb; h += kThreads) {
+                const int mine = s_rest[h];
+                int rank = 0;
+                for (int u = 1; u <= nb; ++u) rank += (s_rest[u] > mine || (s_rest[u] == mine && u < h)) ? 1 : 0;
+                if (rank == want) s_rest[0] = h;
+            }
+            __syncthreads();
+            const int h = s_rest[0];
+            __syncthreads();
+            if (h < 1) { skip = true; goto done; }
+            const int r = rest_of(h, range);
+            if (r == 0) { skip = true; goto done; }               // nothing is left behind this boundary
+            lo = (uint32_t)h * nchh;
+            hi = lo + w + r;
+        }
+        it_head = (int)(lo / nchh);
+        const uint32_t o0 = lo - (uint32_t)it_head * nchh, o1 = hi - (uint32_t)it_head * nchh;
+        const int c0 = (int)(o0 > w ? o0 - w : 0), c1 = (int)(o1 > w ? o1 - w : 0);     // real chunks of the head
+        it_seg = c0 > 0 ? 1 : 0;
+        it_begin = c0 * kC;
+        it_end = min(L, c1 * kC);
+        it_head_end = c1 == (int)nchr;
+        if (c0 > 0 && MODE != kModeState) {
+            if (SCAN) {                            // the slot of the range before: the head's state up to there
+                it_first = (int)range - 1;
+                it_count = 1;
+            } else {                               // every slot of the head so far
+                const uint32_t x = (uint32_t)it_head * nchh + w;
+                it_first = (int)(((x + 1) * n + T - 1) / T - 1);   // the range that holds the head's first chunk
+                it_count = (int)range - it_first;
+            }
+        }
+        if (MODE == kModeState) {
+            if (it_head_end) skip = true;                          // nobody starts from the state of a head's last piece
+            it_out = (int)range;
+        }
+    } else {
+        it_end = min(L, it_begin + seg_len);
+        it_head_end = it_seg == nseg - 1;
+        const int per_head = nseg > 1 ? nseg - 1 : 0;          // workspace slots of one head
+        it_first = it_head * per_head + ((SCAN && it_seg > 0) ? it_seg - 1 : 0);
+        it_count = (MODE == kModeState || MODE == kModePre || it_seg == 0) ? 0 : (SCAN ? 1 : it_seg);
+        it_out = MODE == kModeState ? it_head * per_head + it_seg : -1;
+    }
+done:
+    piece.head = it_head; piece.seg = it_seg; piece.begin = it_begin; piece.end = it_end;
+    piece.first = it_first; piece.count = it_count; piece.out = it_out; piece.head_end = it_head_end ? 1 : 0;
+    piece.skip = skip ? 1 : 0;
+}
+template <int MODE, bool SCAN>
+__device__ __noinline__ void find_piece(Piece* piece, int* s_rest, int balanced, int heads, int pad, int L, int seg_len, int nseg) {
+    Piece pc;
+    piece_of_cta<MODE, SCAN>(pc, s_rest, balanced, heads, pad, L, seg_len, nseg);
+    __syncthreads();
+    if (threadIdx.x == 0) *piece = pc;
+    __syncthreads();
+}
+
 template <int DV, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
     prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -378,83 +587,24 @@ __global__ void __launch_bounds__(kThreads, 1)
     short2* s_abi = reinterpret_cast<short2*>(s_den + 4 * kC);         // [160] ABI rows of each internal feature
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // ---- the CTA's piece of work: a head, a token range, where its initial state comes from (workspace slots
-    // ws_first .. ws_first + ws_count - 1) and where its final state goes (slot ws_out, or the caller's state if
-    // the piece ends its head).
-    // Legacy grids: blockIdx.x = sequence segment, blockIdx.y = head.
-    // Balanced grids (one row of CTAs): the concatenation of all heads' chunks, T = heads x chunks per head, is
-    // cut into n equal ranges [i T / n, (i + 1) T / n), one per SM.  A range holds at most one head boundary
-    // (n >= heads).  CTA i < n takes range i up to the boundary, if there is one; CTA n + j takes what is left
-    // of a range behind its boundary, the j-th largest such rest first: the hardware hands these later CTAs to
-    // SMs as they become free, and the SM whose first piece was shortest is free first, so every SM ends up
-    // with about T / n chunks.  A piece that ends inside its head leaves its state in slot i of its range.
-    int it_head = blockIdx.y, it_seg = blockIdx.x, it_begin = blockIdx.x * p.seg_len, it_end = 0, it_first = 0, it_count = 0,
-        it_out = -1;
-    bool it_head_end = false;
-    if (MODE != kModePre && p.balanced > 0) {      // (the recompute mode's kernel is never launched this way)
-        // 32-bit arithmetic throughout (the host takes this path only while (T + 1) n fits: 64-bit divisions
-        // would be subroutine calls, and their mere presence slows this kernel's role loops by a fifth)
-        const uint32_t n = p.balanced;
-        const uint32_t nchh = (p.L + kC - 1) / kC;
-        const uint32_t T = (uint32_t)p.heads * nchh;
-        uint32_t lo, hi, range;                    // global chunk range of this piece, index of its range
-        if (blockIdx.x < n) {
-            range = blockIdx.x;
-            lo = range * T / n;
-            hi = (range + 1) * T / n;
-            const uint32_t xb = ((hi - 1) / nchh) * nchh;         // start of the head that holds the range's last chunk
-            if (xb > lo) hi = xb;                                  // a boundary inside: stop there
-        } else {
-            // rest of the range behind head boundary h: [h nchh, end of the range that holds it); rank the rests
-            int* s_rest = reinterpret_cast<int*>(smem + C::offStage);
-            const int nb = p.heads - 1, want = (int)(blockIdx.x - n);
-            auto rest_of = [&](uint32_t h, uint32_t& rg) -> int {
-                const uint32_t x = h * nchh;
-                rg = ((x + 1) * n + T - 1) / T - 1;                 // the range that holds chunk x
-                return rg * T / n == x ? 0 : (int)((rg + 1) * T / n - x);   // 0: the boundary is a range start
-            };
-            for (int h = 1 + threadIdx.x; h <= nb; h += kThreads) { uint32_t rg; s_rest[h] = rest_of(h, rg); }
-            __syncthreads();
-            s_rest[0] = -1;
-            __syncthreads();
-            for (int h = 1 + threadIdx.x; h <= nb; h += kThreads) {
-                const int mine = s_rest[h];
-                int rank = 0;
-                for (int u = 1; u <= nb; ++u) rank += (s_rest[u] > mine || (s_rest[u] == mine && u < h)) ? 1 : 0;
-                if (rank == want) s_rest[0] = h;
-            }
-            __syncthreads();
-            const int h = s_rest[0];
-            __syncthreads();
-            if (h < 1) return;
-            const int r = rest_of(h, range);
-            if (r == 0) return;                                    // nothing is left behind this boundary
-            lo = (uint32_t)h * nchh;
-            hi = lo + r;
-        }
-        it_head = (int)(lo / nchh);
-        const int c0 = (int)(lo - (uint32_t)it_head * nchh), c1 = (int)(hi - (uint32_t)it_head * nchh);
-        it_seg = c0 > 0 ? 1 : 0;
-        it_begin = c0 * kC;
-        it_end = min(p.L, c1 * kC);
-        it_head_end = c1 == (int)nchh;
-        if (c0 > 0 && MODE != kModeState) {
-            const uint32_t x = (uint32_t)it_head * nchh;
-            it_first = (int)(((x + 1) * n + T - 1) / T - 1);       // the range that holds the head's first chunk
-            it_count = (int)range - it_first;
-        }
-        if (MODE == kModeState) {
-            if (it_head_end) return;                               // nobody starts from the state of a head's last piece
-            it_out = (int)range;
-        }
+    // ---- the CTA's piece of work (see find_piece)
+    Piece pc;
+#ifdef BASED_PIECE_OUT
+    constexpr bool kPieceOut = (BASED_PIECE_OUT >> ((DV == 128 ? 3 : 0) + MODE)) & 1;
+#else
+    constexpr bool kPieceOut = DV == 64 && MODE == kModeMain;
+#endif
+    if constexpr (kPieceOut) {
+        Piece* s_piece = reinterpret_cast<Piece*>(s_abi + kF);
+        find_piece<MODE, C::kSlotScan>(s_piece, reinterpret_cast<int*>(smem + C::offStage), p.balanced, p.heads, p.pad, p.L, p.seg_len, p.nseg);
+        pc = *s_piece;
     } else {
-        it_end = min(p.L, it_begin + p.seg_len);
-        it_head_end = it_seg == p.nseg - 1;
-        const int per_head = p.nseg > 1 ? p.nseg - 1 : 0;          // workspace slots of one head
-        it_first = it_head * per_head;
-        it_count = (MODE == kModeState || MODE == kModePre) ? 0 : it_seg;
-        it_out = MODE == kModeState ? it_head * per_head + it_seg : -1;
+        piece_of_cta<MODE, C::kSlotScan>(pc, reinterpret_cast<int*>(smem + C::offStage), p.balanced, p.heads, p.pad, p.L, p.seg_len, p.nseg);
     }
+    if (pc.skip) return;
+    const int it_seg = pc.seg, it_head = pc.head, it_begin = pc.begin, it_end = pc.end;
+    const int it_first = pc.first, it_count = pc.count, it_out = pc.out;
+    const bool it_head_end = pc.head_end != 0;
     const int seg = it_seg, head = it_head, tok_begin = it_begin, tok_end = it_end;
     const int ws_first = it_first, ws_count = it_count, ws_out = it_out;
     const bool head_end = it_head_end;
@@ -489,6 +639,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         mbar_init(&bars[kP], 128); mbar_init(&bars[kR4], PQT ? 256 : 384); mbar_init(&bars[kPK], 128); mbar_init(&bars[kPKb], 128); mbar_init(&bars[kDone], 1);
         mbar_init(&bars[kSR], 128);
         mbar_init(&bars[kFin], 1);
+        mbar_init(&bars[kInit], 384);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v); prefetch_tensormap(&tm_o);
@@ -551,6 +702,22 @@ __global__ void __launch_bounds__(kThreads, 1)
     // "step (4) of own chunk c done": with two state-copy tiles (kPQinT) one barrier per tile, as above
     auto g4_bar = [&](int c) -> uint64_t* { return &bars[(PQT && (c & 1)) ? kG4b : kG4]; };
     auto g4_parity = [&](int c) -> uint32_t { return PQT ? ((c >> 1) & 1) : (c & 1); };
+
+    // ---- initial state from earlier pieces' slots, d_v 128 (see Cfg::kSlotScan): in the main pass behind a state pass
+    // all four role groups share it
+    const bool share_init = !C::kSlotScan && MODE == kModeMain && ws_count > 0;
+    auto init_state = [&](int part, int nparts) {
+        init_state_blocks<DV>(p.ws + (size_t)ws_first * seg_state_floats(DV), ws_count, MODE == kModeMain && ws_count > 0,
+                              (!STATE_ONLY && p.continue_abi) ? p.kv_abi : nullptr, p.z_abi, p.dv, head * abi_nrows, s_abi, tb,
+                              part, nparts);
+    };
+    if constexpr (!C::kSlotScan) {
+        if (share_init && warp < 16 && (warp >> 2) != 2) {      // row, feature and output group (parts 0, 1, 3)
+            init_state(warp >> 2, 4);
+            tc_fence_before();
+            mbar_arrive(&bars[kInit]);
+        }
+    }
 
     if (warp == kWarpTma) {
         // ===================================================================== TMA producer
@@ -842,71 +1009,79 @@ __global__ void __launch_bounds__(kThreads, 1)
         const bool is_z = (DV == 64) && t == 64;
         // d_v 128: K-state features held in the two z tiles (64-row MMA: rows 0..31 in lanes 0-15, 32-47)
         const int z1f = (DV == 128 && (t & 31) < 16 && (t >> 5) < 2) ? 128 + (t >> 5) * 16 + (t & 15) : -1;
-        const size_t seg_stride = seg_state_floats(DV);
-        const float* wsh = p.ws + (size_t)ws_first * seg_stride;      // the partial states this piece starts from
-        const int dv = p.dv;                        // row pitch of the caller's state; lanes >= dv hold zeros
-        const float* kvh = p.kv_abi ? p.kv_abi + (size_t)head * abi_nrows * dv : nullptr;
-        const float* zh = p.z_abi ? p.z_abi + (size_t)head * abi_nrows : nullptr;
-        const bool from_abi = !STATE_ONLY && p.continue_abi;
-        const int nprev = ws_count;
-        // the partial states are the state pass's output (a no-op when this grid was launched the plain way)
-        if (MODE == kModeMain && nprev > 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+        if constexpr (C::kSlotScan) {
+            const size_t seg_stride = seg_state_floats(DV);
+            const float* wsh = p.ws + (size_t)ws_first * seg_stride;      // the partial states this piece starts from
+            const int dv = p.dv;                        // row pitch of the caller's state; lanes >= dv hold zeros
+            const float* kvh = p.kv_abi ? p.kv_abi + (size_t)head * abi_nrows * dv : nullptr;
+            const float* zh = p.z_abi ? p.z_abi + (size_t)head * abi_nrows : nullptr;
+            const bool from_abi = !STATE_ONLY && p.continue_abi;
+            const int nprev = ws_count;
+            // the partial states are the state pass's output (a no-op when this grid was launched the plain way)
+            if (MODE == kModeMain && nprev > 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 
-        // Initial value of this lane's row: the caller's ABI state (folded into the internal
-        // basis) plus the partial states of the earlier segments.  Loads are issued 16 at a
-        // time before they are consumed, so their latencies overlap.
-#pragma unroll 1
-        for (int b = 0; b < kF / 16; ++b) {
-            float acc[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) acc[i] = 0.f;
-            if (srow >= 0) {
-                if (from_abi) {
-                    float va[16], vb[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const short2 ar = s_abi[b * 16 + i];
-                        const bool live = is_z || srow < dv;
-                        va[i] = (ar.x >= 0 && live) ? (is_z ? zh[ar.x] : kvh[(size_t)ar.x * dv + srow]) : 0.f;
-                        vb[i] = (ar.y >= 0 && live) ? (is_z ? zh[ar.y] : kvh[(size_t)ar.y * dv + srow]) : 0.f;
+            // Initial value of this lane's row: the caller's ABI state (folded into the internal
+            // basis) plus the partial states of the earlier segments.  Loads are issued 16 at a
+            // time before they are consumed, so their latencies overlap.
+    #pragma unroll 1
+            for (int b = 0; b < kF / 16; ++b) {
+                float acc[16];
+    #pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+                if (srow >= 0) {
+                    if (from_abi) {
+                        float va[16], vb[16];
+    #pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const short2 ar = s_abi[b * 16 + i];
+                            const bool live = is_z || srow < dv;
+                            va[i] = (ar.x >= 0 && live) ? (is_z ? zh[ar.x] : kvh[(size_t)ar.x * dv + srow]) : 0.f;
+                            vb[i] = (ar.y >= 0 && live) ? (is_z ? zh[ar.y] : kvh[(size_t)ar.y * dv + srow]) : 0.f;
+                        }
+    #pragma unroll
+                        for (int i = 0; i < 16; ++i) acc[i] = (s_abi[b * 16 + i].y >= 0) ? (va[i] + vb[i]) * kRsqrt2 : va[i];
                     }
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) acc[i] = (s_abi[b * 16 + i].y >= 0) ? (va[i] + vb[i]) * kRsqrt2 : va[i];
+                    for (int sp = 0; sp < nprev; ++sp) {
+                        const float* src = wsh + (size_t)sp * seg_stride + (is_z ? (size_t)kF * DV + b * 16
+                                                                                 : (size_t)(b * 16) * DV + srow);
+                        float tmp[16];
+    #pragma unroll
+                        for (int i = 0; i < 16; ++i) tmp[i] = is_z ? src[i] : src[(size_t)i * DV];
+    #pragma unroll
+                        for (int i = 0; i < 16; ++i) acc[i] += tmp[i];
+                    }
                 }
-                for (int sp = 0; sp < nprev; ++sp) {
-                    const float* src = wsh + (size_t)sp * seg_stride + (is_z ? (size_t)kF * DV + b * 16
-                                                                             : (size_t)(b * 16) * DV + srow);
-                    float tmp[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) tmp[i] = is_z ? src[i] : src[(size_t)i * DV];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) acc[i] += tmp[i];
+                uint32_t r[16];
+    #pragma unroll
+                for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(acc[i]);
+                tmem_st16(tmem_addr(tb, lane_base, C::colS + b * 16), r);
+            }
+            // d_v 128: K-state of feature t (tile 0) and feature z1f (tile 1), column 0 of each tile
+            auto z_init = [&](int f) -> float {
+                if (f < 0) return 0.f;
+                float acc = 0.f;
+                if (from_abi) {
+                    const short2 ar = s_abi[f];
+                    if (ar.x >= 0) acc = (ar.y >= 0) ? (zh[ar.x] + zh[ar.y]) * kRsqrt2 : zh[ar.x];
                 }
+                for (int sp = 0; sp < nprev; ++sp) acc += wsh[(size_t)sp * seg_stride + (size_t)kF * DV + f];
+                return acc;
+            };
+            if (DV == 128) {
+                uint32_t r0[16], r1[16];
+    #pragma unroll
+                for (int i = 0; i < 16; ++i) r0[i] = r1[i] = 0u;
+                r0[0] = __float_as_uint(z_init(t));
+                r1[0] = __float_as_uint(z_init(z1f));
+                tmem_st16(tmem_addr(tb, lane_base, C::colZ0), r0);
+                tmem_st16(tmem_addr(tb, lane_base, C::colZ1), r1);
             }
-            uint32_t r[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(acc[i]);
-            tmem_st16(tmem_addr(tb, lane_base, C::colS + b * 16), r);
-        }
-        // d_v 128: K-state of feature t (tile 0) and feature z1f (tile 1), column 0 of each tile
-        auto z_init = [&](int f) -> float {
-            if (f < 0) return 0.f;
-            float acc = 0.f;
-            if (from_abi) {
-                const short2 ar = s_abi[f];
-                if (ar.x >= 0) acc = (ar.y >= 0) ? (zh[ar.x] + zh[ar.y]) * kRsqrt2 : zh[ar.x];
-            }
-            for (int sp = 0; sp < nprev; ++sp) acc += wsh[(size_t)sp * seg_stride + (size_t)kF * DV + f];
-            return acc;
-        };
-        if (DV == 128) {
-            uint32_t r0[16], r1[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) r0[i] = r1[i] = 0u;
-            r0[0] = __float_as_uint(z_init(t));
-            r1[0] = __float_as_uint(z_init(z1f));
-            tmem_st16(tmem_addr(tb, lane_base, C::colZ0), r0);
-            tmem_st16(tmem_addr(tb, lane_base, C::colZ1), r1);
+        } else if (share_init) {
+            init_state(2, 4);
+            ok = mbar_wait(&bars[kInit], 0, abort_flag);          // the other groups' blocks are written
+            tc_fence_after();
+        } else {
+            init_state(0, 1);
         }
         tmem_wait_st();
         if (t == 0) TRACE(5, 2, 7);   // state initialised
@@ -1310,6 +1485,59 @@ cudaError_t launch_dependent(dim3 grid, cudaStream_t stream, const CUtensorMap& 
     return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<DV, MODE>, tq, tk, tv, to, p);
 }
 
+// Running sum over each head's partial states, in place, between the state pass and the main pass: afterwards a
+// head's slot i holds the state of everything in the head up to the end of piece i, so a piece of the main pass
+// starts from one slot.  (Summing the earlier pieces' slots in the main pass itself cost its state group 2.7 us of
+// load latency per slot before the first state update could run: 11 us on cfg 5's last pieces, 46 us with 18 pieces
+// per head.)  per_head > 0: head h owns slots h per_head .. (h + 1) per_head - 1; otherwise the equal chunk
+// ranges of prefill_tc_kernel (n ranges, nchr chunks per head, pad w): head h owns the slots of the ranges from
+// the one with its first chunk to the one before the range with its last chunk.
+__global__ void __launch_bounds__(256) slot_scan_kernel(float* __restrict__ ws, uint32_t floats, int per_head, uint32_t heads,
+                                                        uint32_t n, uint32_t nchr, uint32_t w) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the main pass may be scheduled behind this grid
+    asm volatile("griddepcontrol.wait;" ::: "memory");                   // the state pass is complete
+    const uint32_t h = blockIdx.y;
+    uint32_t first, count;
+    if (per_head > 0) {
+        first = h * (uint32_t)per_head;
+        count = (uint32_t)per_head;
+    } else {
+        const uint32_t nchh = nchr + w, T = heads * nchh;
+        auto range_of = [&](uint32_t x) -> uint32_t { return ((x + 1) * n + T - 1) / T - 1; };
+        first = range_of(h * nchh + w);
+        count = range_of((h + 1) * nchh - 1) - first;
+    }
+    float* col = ws + (size_t)first * floats;
+#pragma unroll 1
+    for (uint32_t e = blockIdx.x * 1024 + threadIdx.x; e < floats && e < (blockIdx.x + 1) * 1024; e += 256) {
+        float acc = 0.f;
+        uint32_t i = 0;
+#pragma unroll 1
+        for (; i + 4 <= count; i += 4) {
+            float v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = col[(size_t)(i + j) * floats + e];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { acc += v[j]; col[(size_t)(i + j) * floats + e] = acc; }
+        }
+        for (; i < count; ++i) { acc += col[(size_t)i * floats + e]; col[(size_t)i * floats + e] = acc; }
+    }
+}
+
+static cudaError_t launch_slot_scan(float* ws, int dv_kernel, int per_head, int heads, int n, int nchr, int w, cudaStream_t stream) {
+    const uint32_t floats = (uint32_t)seg_state_floats(dv_kernel);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((floats + 1023) / 1024, heads);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, slot_scan_kernel, ws, floats, per_head, (uint32_t)heads, (uint32_t)n, (uint32_t)nchr, (uint32_t)w);
+}
+
 template <int DV>
 based_status launch_dv(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH, int L,
                        int dv, int flags, float* ws, const SegPlan plan, cudaStream_t stream) {
@@ -1356,15 +1584,26 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
     p.balanced = 0;
     p.heads = BH;
     if (plan.balanced > 0) {
-        // state pass over every piece that ends inside its head, then the main pass; both on one row of CTAs:
-        // one per range, then one per head boundary
+        // state pass over every piece that ends inside its head, (d_v 64) the running sums of each head's slots, then
+        // the main pass; both passes on one row of CTAs: one per range, then one per head boundary
         p.balanced = plan.balanced;
         p.nseg = 1;
+#ifdef BASED_PAD
+        p.pad = BASED_PAD;
+#else
+        p.pad = 5;
+#endif
         const dim3 grid(plan.balanced + BH - 1, 1);
         prefill_tc_kernel<DV, kModeState><<<grid, kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
         note_launch();
-        const based_status st = check_launch("prefill_tc_kernel<state, balanced>");
+        based_status st = check_launch("prefill_tc_kernel<state, balanced>");
         if (st != BASED_OK) return st;
+        if (C::kSlotScan) {
+            if (launch_slot_scan(ws, DV, 0, BH, plan.balanced, (L + kC - 1) / kC, p.pad, stream) != cudaSuccess) return BASED_ERR_CUDA;
+            note_launch();
+            st = check_launch("slot_scan_kernel");
+            if (st != BASED_OK) return st;
+        }
         if (launch_dependent<DV, kModeMain>(grid, stream, tq, tk, tv, to, p) != cudaSuccess) return BASED_ERR_CUDA;
         note_launch();
         return check_launch("prefill_tc_kernel<balanced>");
@@ -1377,8 +1616,14 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
     if (nseg > 1) {
         prefill_tc_kernel<DV, kModeState><<<dim3(nseg - 1, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
         note_launch();
-        const based_status st = check_launch("prefill_tc_kernel<state>");
+        based_status st = check_launch("prefill_tc_kernel<state>");
         if (st != BASED_OK) return st;
+        if (C::kSlotScan && nseg > 2) {     // (two segments: the one slot per head is its own running sum)
+            if (launch_slot_scan(ws, DV, nseg - 1, BH, 0, 0, 0, stream) != cudaSuccess) return BASED_ERR_CUDA;
+            note_launch();
+            st = check_launch("slot_scan_kernel");
+            if (st != BASED_OK) return st;
+        }
     }
     if (nseg > 1) {
         if (launch_dependent<DV, kModeMain>(dim3(nseg, BH), stream, tq, tk, tv, to, p) != cudaSuccess) return BASED_ERR_CUDA;
@@ -1394,7 +1639,8 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
 // How a head's sequence is cut into segments so that about one CTA per SM is busy.
 //  - one segment: the plain chunk loop;
 //  - state pass: a first launch computes every segment's own state into the workspace, the main
-//    launch starts each segment from the sum of the earlier ones (long sequences);
+//    launch starts each segment from the sum of the earlier ones (long sequences; d_v 64: a small kernel in
+//    between turns the partial states into running sums, see Cfg::kSlotScan);
 //  - recompute: one launch, no workspace; a segment's CTA first runs the state update alone over
 //    all earlier chunks (short sequences, where a second launch and start-up cost more than that).
 // The choice compares modelled CTA times in thousands of cycles per chunk, measured on B200:
@@ -1512,6 +1758,9 @@ static based_status launch_state_dv(const void* k, const void* v, float* kv, flo
     p.heads = BH;
     p.seg_len = plan.per * kC;
     p.dv = dv;
+#ifdef BASED_TRACE
+    p.trace = g_trace;
+#endif
     {
         static bool configured[64] = {};
         int dev = 0;

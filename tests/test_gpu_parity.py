@@ -104,6 +104,27 @@ def test_prefill_continue_equals_one_pass(dtype, d_v, L, L1):
     assert_state_close(_np(kv), S_ref, _np(z), z_ref, dtype)
 
 
+@pytest.mark.parametrize("d_v", [64, 128])
+def test_prefill_continue_long_segments(d_v):
+    """A continued call long enough for several segments per head with a state pass: outputs and state of the second
+    call against the oracle's recurrence over the whole sequence.  (The segments' partial states reach the main pass
+    as running sums written by a kernel of their own at d_v 64 and are added up by the main pass itself at d_v 128;
+    the caller's state joins either way.)"""
+    B, H, L, L1 = 1, 3, 12000, 2001
+    w = wl.Workload("longsplit", B, H, L, 16, d_v, "bf16", 0.25)
+    q, k, v = wl.prefill_inputs(w, wl.generator(17 + d_v))
+    y_ref, S_ref, z_ref = oracle.linattn_recurrent(_np(q), _np(k), _np(v))
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    kv, z = based.new_state(B, H, d_v)
+    y1 = based.based_prefill(qd[:, :, :L1].contiguous(), kd[:, :, :L1].contiguous(), vd[:, :, :L1].contiguous(),
+                             kv_state=kv, z_state=z)
+    y2 = based.based_prefill(qd[:, :, L1:].contiguous(), kd[:, :, L1:].contiguous(), vd[:, :, L1:].contiguous(),
+                             kv_state=kv, z_state=z, flags=based.BASED_STATE_CONTINUE)
+    _poll()
+    assert row_err(_np(torch.cat([y1, y2], dim=2)), y_ref) <= TOL_BF16
+    assert_state_close(_np(kv), S_ref, _np(z), z_ref, "bf16")
+
+
 # --------------------------------------------------------------------------- decode
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d_v", [64, 128])
