@@ -1507,27 +1507,28 @@ __global__ void __launch_bounds__(256) slot_scan_kernel(float* __restrict__ ws, 
         first = range_of(h * nchh + w);
         count = range_of((h + 1) * nchh - 1) - first;
     }
-    float* col = ws + (size_t)first * floats;
+    // one element per thread, eight slots' loads in flight at a time
+    const uint32_t e = blockIdx.x * 256 + threadIdx.x;
+    if (e >= floats) return;
+    float* col = ws + (size_t)first * floats + e;
+    float acc = 0.f;
 #pragma unroll 1
-    for (uint32_t e = blockIdx.x * 1024 + threadIdx.x; e < floats && e < (blockIdx.x + 1) * 1024; e += 256) {
-        float acc = 0.f;
-        uint32_t i = 0;
-#pragma unroll 1
-        for (; i + 4 <= count; i += 4) {
-            float v[4];
+    for (uint32_t i = 0; i < count; i += 8) {
+        float v[8];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) v[j] = col[(size_t)(i + j) * floats + e];
+        for (int j = 0; j < 8; ++j) v[j] = (i + j < count) ? col[(size_t)(i + j) * floats] : 0.f;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) { acc += v[j]; col[(size_t)(i + j) * floats + e] = acc; }
+        for (int j = 0; j < 8; ++j) {
+            acc += v[j];
+            if (i + j < count) col[(size_t)(i + j) * floats] = acc;
         }
-        for (; i < count; ++i) { acc += col[(size_t)i * floats + e]; col[(size_t)i * floats + e] = acc; }
     }
 }
 
 static cudaError_t launch_slot_scan(float* ws, int dv_kernel, int per_head, int heads, int n, int nchr, int w, cudaStream_t stream) {
     const uint32_t floats = (uint32_t)seg_state_floats(dv_kernel);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((floats + 1023) / 1024, heads);
+    cfg.gridDim = dim3((floats + 255) / 256, heads);
     cfg.blockDim = dim3(256);
     cfg.stream = stream;
     cudaLaunchAttribute at[1];
