@@ -1023,36 +1023,36 @@ __global__ void __launch_bounds__(kThreads, 1)
             // Initial value of this lane's row: the caller's ABI state (folded into the internal
             // basis) plus the partial states of the earlier segments.  Loads are issued 16 at a
             // time before they are consumed, so their latencies overlap.
-    #pragma unroll 1
+#pragma unroll 1
             for (int b = 0; b < kF / 16; ++b) {
                 float acc[16];
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < 16; ++i) acc[i] = 0.f;
                 if (srow >= 0) {
                     if (from_abi) {
                         float va[16], vb[16];
-    #pragma unroll
+#pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             const short2 ar = s_abi[b * 16 + i];
                             const bool live = is_z || srow < dv;
                             va[i] = (ar.x >= 0 && live) ? (is_z ? zh[ar.x] : kvh[(size_t)ar.x * dv + srow]) : 0.f;
                             vb[i] = (ar.y >= 0 && live) ? (is_z ? zh[ar.y] : kvh[(size_t)ar.y * dv + srow]) : 0.f;
                         }
-    #pragma unroll
+#pragma unroll
                         for (int i = 0; i < 16; ++i) acc[i] = (s_abi[b * 16 + i].y >= 0) ? (va[i] + vb[i]) * kRsqrt2 : va[i];
                     }
                     for (int sp = 0; sp < nprev; ++sp) {
                         const float* src = wsh + (size_t)sp * seg_stride + (is_z ? (size_t)kF * DV + b * 16
                                                                                  : (size_t)(b * 16) * DV + srow);
                         float tmp[16];
-    #pragma unroll
+#pragma unroll
                         for (int i = 0; i < 16; ++i) tmp[i] = is_z ? src[i] : src[(size_t)i * DV];
-    #pragma unroll
+#pragma unroll
                         for (int i = 0; i < 16; ++i) acc[i] += tmp[i];
                     }
                 }
                 uint32_t r[16];
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(acc[i]);
                 tmem_st16(tmem_addr(tb, lane_base, C::colS + b * 16), r);
             }
@@ -1069,7 +1069,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             };
             if (DV == 128) {
                 uint32_t r0[16], r1[16];
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < 16; ++i) r0[i] = r1[i] = 0u;
                 r0[0] = __float_as_uint(z_init(t));
                 r1[0] = __float_as_uint(z_init(z1f));
