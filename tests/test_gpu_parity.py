@@ -1230,14 +1230,14 @@ def test_bench_profiles_print_one_json_line(args):
 
 # --------------------------------------------------------------------------- few heads, long sequences
 @pytest.mark.parametrize("B,H,L,d_v,flags", [(1, 5, 61000, 64, 0), (1, 40, 16500, 128, 1), (2, 3, 50700, 112, 0),
-                                             (1, 147, 2100, 64, 2), (1, 2, 152000, 64, 0)])
+                                             (1, 147, 2100, 64, 2), (1, 2, 152000, 64, 0), (1, 3, 110000, 128, 0)])
 def test_prefill_heads_cut_into_equal_chunk_ranges(B, H, L, d_v, flags):
     """Fewer heads than SMs and sequences long enough that all heads' chunks, laid end to end, are cut into one
     equal range per SM (a range then holds the tail of one head and the start of the next, and a head's pieces
     start from the summed states of the pieces before them): every output row and the final state of every head
     against the oracle, ragged last chunks included, in the full and the symmetric state format and for
     numerator-only outputs.  The two-head case gives a head 74 pieces (the running sums of their states at d_v 64
-    go through more than one batch of eight slots)."""
+    go through more than one batch of eight slots); the three-head d_v 128 case gives a piece up to 49 slots to add up."""
     flag = {0: 0, 1: based.BASED_STATE_SYM, 2: based.BASED_NUMERATOR_ONLY}[flags]
     w = wl.Workload("ranges", B, H, L, 16, d_v, "bf16", 0.3)
     q, k, v = wl.prefill_inputs(w, wl.generator(B + H + L))
