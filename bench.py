@@ -49,7 +49,7 @@ L2_BYTES = 126 * 1024 * 1024
 # processed.  Written bytes still resident in L2 when a launch ends are not in these figures.
 NCU_TRAFFIC = {
     "cfg2_360m_prefill": 25.24e6,                 # profiles/prefill_tc_kernel_dv64_cfg2.md (output stays in L2)
-    "cfg3_1p3b_prefill": 167.98e6 + 103.88e6,     # profiles/prefill_tc_kernel_dv128.md (part of the output still in L2)
+    "cfg3_1p3b_prefill": 167.85e6 + 102.19e6,     # profiles/prefill_tc_kernel_dv128.md (part of the output still in L2)
     "cfg4_generation": 2 * (144.59e6 + 88.45e6),  # profiles/decode_step_kernel_dv128.md, 1024 -> 2048 heads
     "cfg5_mixer_pair:swa": 2 * (201.37e6 + 43.87e6),  # profiles/swa_tc_kernel.md, 16 -> 32 heads
     "baseconv": 4 * (272.67e6 + 96.72e6),         # profiles/baseconv_gate_kernel.md, batch 2 -> 8 (part of the writes still in L2)
