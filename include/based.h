@@ -358,8 +358,10 @@ based_status based_generation_step(const void* q, const void* k, const void* v, 
  * everything it calls, allocates nothing.
  *
  * Arguments, layouts, supported set and results are those of based_prefill without the
- * workspace pair.  A request whose based_prefill_workspace_bytes exceeds the array returns
- * BASED_ERR_WORKSPACE (and says so on stderr); use based_prefill with your own buffer then.
+ * workspace pair.  A request whose based_prefill_workspace_bytes exceeds the array (few heads
+ * with a long sequence) is cut into fewer segments per head, as many as the array holds
+ * partial states for, and is slower than based_prefill with a workspace of the full size;
+ * the results are those of based_prefill up to the rounding order of the partial sums.
  * The first call on a device looks up the array's device address (one
  * cudaGetSymbolAddress, no allocation); make that first call outside any stream capture.
  * All calls on a device share the one array and it keeps the previous call's contents:

@@ -95,9 +95,9 @@ size_t based_prefill_workspace_bytes(int B, int H, int L, int d_feat, int d_v, b
     return prefill_tc_workspace_bytes(B * H, L, d_v);
 }
 
-based_status based_prefill(const void* q, const void* k, const void* v, void* out, float* kv_state, float* z_state,
-                           int B, int H, int L, int d_feat, int d_v, based_dtype io, int flags, void* workspace,
-                           size_t workspace_bytes, void* cuda_stream) {
+static based_status prefill_impl(const void* q, const void* k, const void* v, void* out, float* kv_state, float* z_state,
+                                 int B, int H, int L, int d_feat, int d_v, based_dtype io, int flags, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream, bool fit) {
     if (!q || !k || !v || !out || B <= 0 || H <= 0 || L <= 0) return BASED_ERR_INVALID_ARG;
     if (io != BASED_F32 && io != BASED_BF16) return BASED_ERR_INVALID_ARG;
     if (flags & ~(BASED_STATE_CONTINUE | BASED_STATE_SYM | BASED_NUMERATOR_ONLY)) return BASED_ERR_INVALID_ARG;
@@ -113,10 +113,10 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
         const size_t es = esize(io), rows = (flags & BASED_STATE_SYM) ? kDSym : 1 + d_feat + d_feat * d_feat;
         for (long long h0 = 0; h0 < (long long)B * H; h0 += kHeadSlab) {
             const int n = (int)((long long)B * H - h0 < kHeadSlab ? (long long)B * H - h0 : kHeadSlab);
-            const based_status st = based_prefill(
+            const based_status st = prefill_impl(
                 off(q, (size_t)h0 * L * d_feat * es), off(k, (size_t)h0 * L * d_feat * es), off(v, (size_t)h0 * L * d_v * es),
                 off(out, (size_t)h0 * L * d_v * es), off(kv_state, (size_t)h0 * rows * d_v), off(z_state, (size_t)h0 * rows),
-                1, n, L, d_feat, d_v, io, flags, workspace, workspace_bytes, cuda_stream);
+                1, n, L, d_feat, d_v, io, flags, workspace, workspace_bytes, cuda_stream, fit);
             if (st != BASED_OK) return st;
         }
         return BASED_OK;
@@ -136,12 +136,19 @@ based_status based_prefill(const void* q, const void* k, const void* v, void* ou
                                       static_cast<cudaStream_t>(cuda_stream));
     }
     const size_t need = based_prefill_workspace_bytes(B, H, L, d_feat, d_v, io);
-    if (need > 0 && (!workspace || workspace_bytes < need)) return BASED_ERR_WORKSPACE;
+    if (!fit && need > 0 && (!workspace || workspace_bytes < need)) return BASED_ERR_WORKSPACE;
     if (io == BASED_BF16)
         return launch_prefill_tc(q, k, v, out, kv_state, z_state, B * H, L, d_v, flags, workspace,
-                                 static_cast<cudaStream_t>(cuda_stream));
+                                 static_cast<cudaStream_t>(cuda_stream), fit ? workspace_bytes : ~(size_t)0);
     return launch_prefill_simt(q, k, v, out, kv_state, z_state, B * H, L, d_v, io, flags,
                                static_cast<cudaStream_t>(cuda_stream));
+}
+
+based_status based_prefill(const void* q, const void* k, const void* v, void* out, float* kv_state, float* z_state,
+                           int B, int H, int L, int d_feat, int d_v, based_dtype io, int flags, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream) {
+    return prefill_impl(q, k, v, out, kv_state, z_state, B, H, L, d_feat, d_v, io, flags, workspace, workspace_bytes,
+                        cuda_stream, false);
 }
 
 size_t based_prefill_state_workspace_bytes(int B, int H, int L, int d_feat, int d_v, based_dtype io) {
@@ -478,3 +485,12 @@ based_status based_poll_error(void* cuda_stream) {
 }
 
 }  // extern "C"
+
+namespace based {
+based_status prefill_fit_workspace(const void* q, const void* k, const void* v, void* out, float* kv_state, float* z_state,
+                                   int B, int H, int L, int d_feat, int d_v, based_dtype io, int flags, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream) {
+    return ::prefill_impl(q, k, v, out, kv_state, z_state, B, H, L, d_feat, d_v, io, flags, workspace, workspace_bytes,
+                          cuda_stream, true);
+}
+}  // namespace based

@@ -84,10 +84,17 @@ based_status launch_state_convert(const float* kv_in, const float* z_in, float* 
                                   int d_v, bool to_sym, cudaStream_t stream);
 based_status launch_prefill_simt(const void* q, const void* k, const void* v, void* out, float* kv, float* z,
                                  int BH, int L, int d_v, based_dtype io, int flags, cudaStream_t stream);
-// bf16 tensor-core prefill (tcgen05); workspace holds partial states of sequence segments
+// bf16 tensor-core prefill (tcgen05); workspace holds partial states of sequence segments.  prefill_tc_workspace_bytes
+// is what the fastest plan needs; workspace_limit = the bytes behind `workspace`: a call given less takes the fastest
+// plan that fits (fewer segments per head, in the end none: the plain loop and the recompute mode need no workspace).
 size_t prefill_tc_workspace_bytes(int BH, int L, int d_v);
 based_status launch_prefill_tc(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH,
-                               int L, int d_v, int flags, void* workspace, cudaStream_t stream);
+                               int L, int d_v, int flags, void* workspace, cudaStream_t stream,
+                               size_t workspace_limit = ~(size_t)0);
+// based_prefill without its workspace check: the plan is fitted to the workspace given (for based_prefill_static_scratch)
+based_status prefill_fit_workspace(const void* q, const void* k, const void* v, void* out, float* kv_state, float* z_state,
+                                   int B, int H, int L, int d_feat, int d_v, based_dtype io, int flags, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream);
 // bf16 tensor-core sliding window (window <= 128)
 bool swa_tc_supported(int window);
 based_status launch_swa_tc(const void* q, const void* k, const void* v, void* out, int BH, int L, int window,

@@ -44,14 +44,9 @@ extern "C" based_status based_prefill_static_scratch(const void* q, const void* 
                                                      float* kv_state, float* z_state, int B, int H, int L,
                                                      int d_feat, int d_v, based_dtype io, int flags,
                                                      void* cuda_stream) {
+    // What the fastest plan would need; with less, the call takes the fastest plan that fits the array (fewer segments
+    // per head, in the end the plain chunk loop or the recompute mode, which need no scratch).
     const size_t need = based_prefill_workspace_bytes(B, H, L, d_feat, d_v, io);
-    if (need > kScratchBytes) {
-        std::fprintf(stderr,
-                     "libbased: based_prefill_static_scratch needs %zu bytes of scratch for B=%d H=%d L=%d d_v=%d, "
-                     "the built-in array holds %zu; use based_prefill with a caller-owned workspace\n",
-                     need, B, H, L, d_v, kScratchBytes);
-        return BASED_ERR_WORKSPACE;
-    }
     void* scratch = nullptr;
     if (need > 0) {
         const based_status st = scratch_address(&scratch);
@@ -59,6 +54,6 @@ extern "C" based_status based_prefill_static_scratch(const void* q, const void* 
     }
     // Every scratch slot the main pass reads is first written by the segment-state pass of the
     // same call, so nothing has to be cleared between calls.
-    return based_prefill(q, k, v, out, kv_state, z_state, B, H, L, d_feat, d_v, io, flags, scratch, need,
-                         cuda_stream);
+    return based::prefill_fit_workspace(q, k, v, out, kv_state, z_state, B, H, L, d_feat, d_v, io, flags, scratch,
+                                        kScratchBytes, cuda_stream);
 }

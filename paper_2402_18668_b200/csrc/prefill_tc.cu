@@ -1644,26 +1644,33 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
 //    between turns the partial states into running sums, see Cfg::kSlotScan);
 //  - recompute: one launch, no workspace; a segment's CTA first runs the state update alone over
 //    all earlier chunks (short sequences, where a second launch and start-up cost more than that).
-// The choice compares modelled CTA times in thousands of cycles per chunk, measured on B200:
-// full chunk 3.3 (d_v 64) / 3.4 (d_v 128), state-update-only chunk 1.0 / 1.4, a second launch and
-// start-up about 14.  In recompute mode later segments do more redundant work, so the first
-// n - 1 segments get `per` chunks each and the last one the (shorter) rest, `per` chosen to
-// level the modelled times.
-static SegPlan prefill_tc_plan(int BH, int L, int d_v, bool continued = false) {
+// The choice compares modelled CTA times in thousands of cycles, constants fitted on B200 with every SM busy:
+// full chunk 3.0 (d_v 64) / 4.1 (d_v 128), state-update-only chunk of the state pass 1.1 / 2.2, of the recompute
+// mode 1.5 / 2.6, a state pass ahead of the main pass 34 / 30 (its CTAs' start-up and tail, the slot sums, the
+// launches).  In recompute mode later segments do more redundant work, so the first n - 1 segments get `per`
+// chunks each and the last one the (shorter) rest, `per` chosen to level the modelled times.  (Forced plans
+// against this choice on 23 shapes between 1 and 128 heads that do not take the equal chunk ranges: within 4 % of the
+// best forced plan on every one.)
+// ws_limit: bytes of workspace the plan may use (plans that need more are not considered).
+static SegPlan prefill_tc_plan(int BH, int L, int d_v, bool continued = false, size_t ws_limit = ~(size_t)0) {
     const int nch = (L + kC - 1) / kC;
-    const float full = d_v == 64 ? 3.3f : 3.4f, upd = d_v == 64 ? 1.0f : 1.4f;
-    // a pre-chunk of the recompute mode costs more than a chunk of the state pass (d_v 64, cfg 2: 2.1 k cycles against
-    // 3.5 k for a full chunk of that kernel); of 1.0 / 1.5 / 2.0 / 2.4 this value gave the shortest calls
-    const float pre = d_v == 64 ? 1.5f : upd;
+    const size_t slot = seg_state_floats(d_v) * sizeof(float);
+    const float full = d_v == 64 ? 3.0f : 4.1f, upd = d_v == 64 ? 1.1f : 2.2f;
+    const float second = d_v == 64 ? 34.f : 30.f;   // a state pass ahead of the main pass: its own start-up and tail, the slot sums, the launches
+    // a pre-chunk of the recompute mode costs more than a chunk of the state pass (its kernel keeps four stages of
+    // q + k + v size and the whole chunk loop's code); d_v 64: of 1.0 / 1.5 / 2.0 / 2.4 this value gave the shortest
+    // cfg-2 calls; d_v 128: the smallest value that keeps B1 H8 L4096 on four state-pass segments (35.5 against 43 us)
+    const float pre = d_v == 64 ? 1.5f : 2.6f;
     int nmax = 148 / BH;
     if (nmax > 8) nmax = 8;
-    // state pass: a split pays only when every segment keeps at least 16 chunks
+    // state pass: as many segments as SMs allow (at least two chunks each); its fixed cost decides against short ones
     int nseg = nmax;
-    if (nseg > nch / 16) nseg = nch / 16;
+    if (nseg > nch / 2) nseg = nch / 2;
     if (nseg < 1) nseg = 1;
     while (nseg > 1 && ((nch + nseg - 1) / nseg) * (nseg - 1) >= nch) --nseg;   // every segment owns a chunk
+    while (nseg > 1 && ((size_t)BH * (nseg - 1) * slot > ws_limit || ((nch + nseg - 1) / nseg) * (nseg - 1) >= nch)) --nseg;
     SegPlan best = {nseg, (nch + nseg - 1) / nseg, false, 0};
-    float best_cost = nseg > 1 ? (float)best.per * (upd + full) + 14.f : (float)nch * full;
+    float best_cost = nseg > 1 ? (float)best.per * (upd + full) + second : (float)nch * full;
     for (int n = 2; n <= nmax; ++n) {
         for (int per = (nch + n - 1) / n; per * (n - 1) < nch; ++per) {
             float cost = 0.f;
@@ -1672,7 +1679,8 @@ static SegPlan prefill_tc_plan(int BH, int L, int d_v, bool continued = false) {
                 const float c = (float)(j * per) * pre + (float)own * full;
                 if (c > cost) cost = c;
             }
-            if (cost < 0.95f * best_cost) {
+            // (between recompute plans of equal modelled cost the one with more segments keeps more SMs busy)
+            if (cost < 0.95f * best_cost || (best.recompute && n > best.nseg && cost <= best_cost)) {
                 best = {n, per, true, 0};
                 best_cost = cost;
             }
@@ -1687,8 +1695,9 @@ static SegPlan prefill_tc_plan(int BH, int L, int d_v, bool continued = false) {
         const long long total = (long long)BH * nch;
         const int ranges = 148;
         const float share = (float)((total + ranges - 1) / ranges);
-        const float cost = share * (upd + full) + 14.f + 7.f;        // a second launch; a second CTA's start-up on some SMs
-        if (share >= 16.f && total >= ranges && total <= 14000000 && cost < 0.95f * best_cost) best = {1, nch, false, ranges};
+        const float cost = share * (upd + full) + second + 7.f;      // a second CTA's start-up on some SMs
+        if (share >= 16.f && total >= ranges && total <= 14000000 && (size_t)ranges * slot <= ws_limit && cost < 0.95f * best_cost)
+            best = {1, nch, false, ranges};
     }
 #ifdef BASED_TRACE
     if (const char* e = getenv("BASED_NSEG")) {
@@ -1812,8 +1821,9 @@ size_t prefill_tc_workspace_bytes(int BH, int L, int d_v) {
 }
 
 based_status launch_prefill_tc(const void* q, const void* k, const void* v, void* out, float* kv, float* z, int BH,
-                               int L, int d_v, int flags, void* workspace, cudaStream_t stream) {
-    const SegPlan plan = prefill_tc_plan(BH, L, d_v == 112 ? 128 : d_v, (flags & BASED_STATE_CONTINUE) != 0);
+                               int L, int d_v, int flags, void* workspace, cudaStream_t stream, size_t workspace_limit) {
+    const SegPlan plan = prefill_tc_plan(BH, L, d_v == 112 ? 128 : d_v, (flags & BASED_STATE_CONTINUE) != 0,
+                                         workspace ? workspace_limit : 0);
     float* ws = static_cast<float*>(workspace);
     if (d_v == 64) return launch_dv<64>(q, k, v, out, kv, z, BH, L, 64, flags, ws, plan, stream);
     return launch_dv<128>(q, k, v, out, kv, z, BH, L, d_v, flags, ws, plan, stream);      // 112 or 128

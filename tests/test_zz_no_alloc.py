@@ -6,7 +6,8 @@ compared with based_prefill's, twice in a row with different inputs: the second 
 the first call's leftovers in the shared array and must not be affected by them.  Both entry
 points run the same kernels on the same inputs, so the comparison is bit for bit; sampled
 rows and one head's state are also held against the oracle, and the device's free memory is
-the same before and after the call.
+the same before and after the call.  A second test takes a shape whose fastest plan would need
+more than the built-in array.
 """
 import ctypes
 
@@ -69,13 +70,26 @@ def test_static_scratch_matches_workspace_variant_twice():
         assert_state_close(f64(kv[sl]), S_o, f64(z[sl]), z_o, "bf16")
 
 
-def test_static_scratch_rejects_oversized_requests():
-    B, H, L, d_v = 1, 18, 16384, 128                    # the partial states of 18 heads x 128 chunks exceed 8 MiB
+def test_static_scratch_fits_its_plan_to_the_array():
+    """A shape whose fastest plan needs more than the built-in 8 MiB (18 heads x 128 chunks at d_v 128: one partial
+    state per head and segment) is cut into fewer segments per head, as many as the array has room for, instead of
+    being refused: outputs and states against the oracle, and nothing allocated."""
+    B, H, L, d_v = 1, 18, 16384, 128
     need = based.based_prefill_workspace_bytes(B, H, L, 16, d_v, based.BASED_BF16)
     assert need > based.based_static_scratch_bytes() == 8 << 20
-    q = torch.zeros(B, H, L, 16, dtype=torch.bfloat16, device="cuda")
-    v = torch.zeros(B, H, L, d_v, dtype=torch.bfloat16, device="cuda")
-    n0 = based.launch_count()
-    with pytest.raises(based.BasedError) as e:
-        based.based_prefill_static_scratch(q, q.clone(), v, torch.empty_like(v))
-    assert e.value.status == 6 and based.launch_count() == n0
+    w = wl.Workload("noalloc_big", B, H, L, 16, d_v, "bf16", 0.25)
+    q, k, v = (t.cuda() for t in wl.prefill_inputs(w, wl.generator(23)))
+    kv, z = based.new_state(B, H, d_v)
+    out = torch.full_like(v, float("nan"))
+    # (a first call loads the d_v 128 kernels and, if no test ran before, the built-in array: see above)
+    based.based_prefill_static_scratch(q, k, v, torch.empty_like(v))
+    free0, alloc0 = _free_bytes(), torch.cuda.memory_allocated()
+    based.based_prefill_static_scratch(q, k, v, out, kv_state=kv, z_state=z)
+    assert based.based_poll_error() == based.BASED_OK
+    assert _free_bytes() == free0 and torch.cuda.memory_allocated() == alloc0
+    f64 = wl.to_f64
+    for h in (0, 7, H - 1):
+        sl = (slice(0, 1), slice(h, h + 1))
+        y_o, S_o, z_o = oracle.linattn_recurrent(f64(q[sl]), f64(k[sl]), f64(v[sl]))
+        assert row_err(f64(out[sl]), y_o) <= TOL_BF16
+        assert_state_close(f64(kv[sl]), S_o, f64(z[sl]), z_o, "bf16")
