@@ -151,7 +151,8 @@ struct Params {
                           // the tensor maps zero-fill columns 112..127 on load and clip them on store)
     int balanced;         // > 0: the number of equal chunk ranges the heads' chunks are cut into (see the kernel)
     int heads;            // B*H (balanced mode)
-    int pad;              // balanced mode: chunks counted in front of every head for the CTA it starts
+    int pad;              // balanced mode: chunks counted in front of every head for the CTA it starts;
+                          // segments with a state pass: 1 if each head's first slot holds the caller's state
 #ifdef BASED_TRACE
     unsigned long long* trace;
 #endif
@@ -541,10 +542,13 @@ __device__ __forceinline__ void piece_of_cta(Piece& piece, int* s_rest, int bala
     } else {
         it_end = min(L, it_begin + seg_len);
         it_head_end = it_seg == nseg - 1;
-        const int per_head = nseg > 1 ? nseg - 1 : 0;          // workspace slots of one head
-        it_first = it_head * per_head + ((SCAN && it_seg > 0) ? it_seg - 1 : 0);
-        it_count = (MODE == kModeState || MODE == kModePre || it_seg == 0) ? 0 : (SCAN ? 1 : it_seg);
-        it_out = MODE == kModeState ? it_head * per_head + it_seg : -1;
+        // workspace slots of one head: one per segment but the last, behind (pad = 1) one that holds the caller's
+        // state of a continued call (abi_to_slot_kernel), which the segments then take like an earlier segment's
+        const int per_head = nseg > 1 ? nseg - 1 + pad : 0;
+        const int before = it_seg + pad;                       // slots this segment starts from
+        it_first = it_head * per_head + ((SCAN && before > 0) ? before - 1 : 0);
+        it_count = (MODE == kModeState || MODE == kModePre || before == 0) ? 0 : (SCAN ? 1 : before);
+        it_out = MODE == kModeState ? it_head * per_head + before : -1;
     }
 done:
     piece.head = it_head; piece.seg = it_seg; piece.begin = it_begin; piece.end = it_end;
@@ -1485,6 +1489,28 @@ cudaError_t launch_dependent(dim3 grid, cudaStream_t stream, const CUtensorMap& 
     return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<DV, MODE>, tq, tk, tv, to, p);
 }
 
+// The caller's state of a continued call, folded into the internal basis, as the first workspace slot of each head
+// (slot layout: [160 features][DV] values, then the 160 K-state entries).  With a state pass the segments of a head
+// take it like the state of an earlier segment and never read the caller's arrays, which the head's last segment
+// overwrites with the final state at its end: a segment that started late (the call's CTAs are scheduled as SMs come
+// free) could otherwise read what a short last segment had already written.
+template <int DV>
+__global__ void __launch_bounds__(DV) abi_to_slot_kernel(const float* __restrict__ kv, const float* __restrict__ z,
+                                                          float* __restrict__ ws, int per_head, int dv, int sym) {
+    const int head = blockIdx.y, f = blockIdx.x, col = threadIdx.x;
+    const AbiRows ar = sym ? sym_rows(f) : abi_rows(f);
+    const int nrows = sym ? kDSym : kD;
+    float* slot = ws + (size_t)head * per_head * seg_state_floats(DV);
+    const float* kvh = kv + (size_t)head * nrows * dv;
+    float val = 0.f;
+    if (ar.a >= 0 && col < dv) val = ar.b >= 0 ? (kvh[(size_t)ar.a * dv + col] + kvh[(size_t)ar.b * dv + col]) * kRsqrt2 : kvh[(size_t)ar.a * dv + col];
+    slot[(size_t)f * DV + col] = val;
+    if (col == 0) {
+        const float* zh = z + (size_t)head * nrows;
+        slot[(size_t)kF * DV + f] = ar.a < 0 ? 0.f : (ar.b >= 0 ? (zh[ar.a] + zh[ar.b]) * kRsqrt2 : zh[ar.a]);
+    }
+}
+
 // Running sum over each head's partial states, in place, between the state pass and the main pass: afterwards a
 // head's slot i holds the state of everything in the head up to the end of piece i, so a piece of the main pass
 // starts from one slot.  (Summing the earlier pieces' slots in the main pass itself cost its state group 2.7 us of
@@ -1549,7 +1575,7 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
         !make_map(&tv, v, BH, L, dv, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !make_map(&to, out, BH, L, dv, 64, CU_TENSOR_MAP_SWIZZLE_128B))
         return BASED_ERR_CUDA;
-    Params p;
+    Params p{};         // (every field the kernel may read has a value: pad is read on every path)
     p.kv_abi = kv;
     p.z_abi = z;
     p.ws = ws;
@@ -1615,12 +1641,22 @@ based_status launch_dv(const void* q, const void* k, const void* v, void* out, f
         return check_launch("prefill_tc_kernel<pre>");
     }
     if (nseg > 1) {
+        based_status st;
+        if (p.continue_abi) {
+            // the caller's state goes into each head's first slot (see abi_to_slot_kernel); no segment reads it itself
+            p.pad = 1;
+            p.continue_abi = 0;
+            abi_to_slot_kernel<DV><<<dim3(kF, BH), DV, 0, stream>>>(kv, z, ws, nseg, dv, p.sym);
+            note_launch();
+            st = check_launch("abi_to_slot_kernel");
+            if (st != BASED_OK) return st;
+        }
         prefill_tc_kernel<DV, kModeState><<<dim3(nseg - 1, BH), kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, to, p);
         note_launch();
-        based_status st = check_launch("prefill_tc_kernel<state>");
+        st = check_launch("prefill_tc_kernel<state>");
         if (st != BASED_OK) return st;
-        if (C::kSlotScan && nseg > 2) {     // (two segments: the one slot per head is its own running sum)
-            if (launch_slot_scan(ws, DV, nseg - 1, BH, 0, 0, 0, stream) != cudaSuccess) return BASED_ERR_CUDA;
+        if (C::kSlotScan && nseg - 1 + p.pad > 1) {     // (one slot per head is its own running sum)
+            if (launch_slot_scan(ws, DV, nseg - 1 + p.pad, BH, 0, 0, 0, stream) != cudaSuccess) return BASED_ERR_CUDA;
             note_launch();
             st = check_launch("slot_scan_kernel");
             if (st != BASED_OK) return st;
@@ -1668,7 +1704,9 @@ static SegPlan prefill_tc_plan(int BH, int L, int d_v, bool continued = false, s
     if (nseg > nch / 2) nseg = nch / 2;
     if (nseg < 1) nseg = 1;
     while (nseg > 1 && ((nch + nseg - 1) / nseg) * (nseg - 1) >= nch) --nseg;   // every segment owns a chunk
-    while (nseg > 1 && ((size_t)BH * (nseg - 1) * slot > ws_limit || ((nch + nseg - 1) / nseg) * (nseg - 1) >= nch)) --nseg;
+    while (nseg > 1 && ((size_t)BH * (nseg - 1 + (continued ? 1 : 0)) * slot > ws_limit ||       // (a continued call: + the caller's state)
+                        ((nch + nseg - 1) / nseg) * (nseg - 1) >= nch))
+        --nseg;
     SegPlan best = {nseg, (nch + nseg - 1) / nseg, false, 0};
     float best_cost = nseg > 1 ? (float)best.per * (upd + full) + second : (float)nch * full;
     for (int n = 2; n <= nmax; ++n) {
@@ -1814,7 +1852,7 @@ size_t prefill_tc_workspace_bytes(int BH, int L, int d_v) {
         const SegPlan plan = prefill_tc_plan(BH, L, d_v, cont != 0);
         size_t n = 0;
         if (plan.balanced > 0) n = (size_t)plan.balanced * seg_state_floats(d_v) * sizeof(float);
-        else if (!plan.recompute && plan.nseg > 1) n = (size_t)BH * (plan.nseg - 1) * seg_state_floats(d_v) * sizeof(float);
+        else if (!plan.recompute && plan.nseg > 1) n = (size_t)BH * (plan.nseg - 1 + cont) * seg_state_floats(d_v) * sizeof(float);
         need = n > need ? n : need;
     }
     return need;

@@ -125,6 +125,28 @@ def test_prefill_continue_long_segments(d_v):
     assert_state_close(_np(kv), S_ref, _np(z), z_ref, "bf16")
 
 
+@pytest.mark.parametrize("d_v", [64, 112])
+def test_continued_call_with_short_segments_repeated(d_v):
+    """A continued call cut into seven segments of five chunks per head, forty times over: the head's last segment
+    (three chunks) overwrites the caller's state soon after the call starts, and no other segment may still be
+    reading its initial state from there (with a state pass the caller's state travels through a workspace slot).
+    Every run against the fp32 kernel of the same library, whose whole head is one thread block."""
+    B, H, L = 1, 16, 4100
+    g = torch.Generator(device="cuda").manual_seed(5 + d_v)
+    rnd = lambda *shape, s=1.0: torch.randn(*shape, generator=g, device="cuda") * s
+    for rep in range(40):
+        q, k, v = rnd(B, H, L, 16, s=0.4).bfloat16(), rnd(B, H, L, 16, s=0.4).bfloat16(), rnd(B, H, L, d_v).bfloat16()
+        kv, z = based.new_state(B, H, d_v)
+        based.based_prefill(rnd(B, H, 3, 16, s=0.4), rnd(B, H, 3, 16, s=0.4), rnd(B, H, 3, d_v), kv_state=kv, z_state=z)
+        kv2, z2 = kv.clone(), z.clone()
+        out = based.based_prefill(q, k, v, kv_state=kv, z_state=z, flags=based.BASED_STATE_CONTINUE)
+        ref = based.based_prefill(q.float(), k.float(), v.float(), kv_state=kv2, z_state=z2, flags=based.BASED_STATE_CONTINUE)
+        _poll()
+        err = ((out.float() - ref).abs().amax(-1) / ref.abs().amax(-1).clamp_min(1e-30)).max().item()
+        assert err <= TOL_BF16, f"run {rep}: {err}"
+        assert_state_close(_np(kv), _np(kv2), _np(z), _np(z2), "bf16", f"run {rep}")
+
+
 # --------------------------------------------------------------------------- decode
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d_v", [64, 128])
