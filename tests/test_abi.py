@@ -140,6 +140,26 @@ def test_prefill_state_validation(lib):
     assert f(P, P, O, O, 1, 1, 8, 16, 64, 1, 0, None, 0, None) == 6                      # workspace missing
 
 
+def test_prefill_plan_through_workspace_bytes(lib):
+    """The segment plan of the bf16 prefill as far as the host can see it: bytes of partial states the fastest plan
+    needs (one slot of 160 x d_v + 160 floats per partial state; the larger of the plain and the continued call)."""
+    wb = lib.based_prefill_workspace_bytes
+    slot = lambda d_v: (160 * d_v + 160) * 4
+    assert wb(8, 16, 4096, 16, 128, 1) == 0                       # cfg 3: 128 heads, one CTA per head
+    assert wb(1, 148, 4096, 16, 64, 1) == 0
+    assert wb(2, 16, 32768, 16, 64, 1) >= 148 * slot(64)          # cfg 5: equal chunk ranges, one slot per range
+    assert wb(1, 40, 16500, 16, 128, 1) >= 148 * slot(128)
+    assert wb(1, 40, 16500, 16, 112, 1) == wb(1, 40, 16500, 16, 128, 1)       # d_v 112 runs on the d_v 128 kernels
+    # few heads, mid-length: a state pass with as many segments as SMs allow; a continued call has one slot more per
+    # head (the caller's state), so 8 heads x 8 segments need 8 x 8 slots
+    assert wb(1, 8, 4096, 16, 128, 1) == 8 * 8 * slot(128)
+    assert wb(1, 8, 8192, 16, 64, 1) == 8 * 8 * slot(64)
+    assert wb(4, 16, 2048, 16, 64, 0) == 0                        # fp32 io: no scratch
+    assert wb(4, 16, 2048, 24, 64, 1) == 0                        # other d': no scratch
+    for shape in [(4, 16, 2048, 64), (1, 1, 128, 64), (1, 147, 2100, 64), (3, 5, 700, 128)]:
+        assert wb(*shape[:3], 16, shape[3], 1) % 16 == 0
+
+
 def test_baseconv_validation(lib):
     f = lib.baseconv_gate_forward
     O = ctypes.c_void_p(0x2000)
